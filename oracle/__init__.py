@@ -1,0 +1,304 @@
+"""CPU oracle of the key-frame partial-distillation step (ShadowTutor).
+
+TEST INFRASTRUCTURE ONLY: imported by the tests, the smoke check and the
+benchmark's CPU-baseline leg.  It never imports the CUDA package and the CUDA
+package never imports it.
+
+The arithmetic lives in ``st_oracle.c`` (plain C loops, fp32 storage, double
+accumulators; a pure-double build exists for finite differences).  This module
+compiles it with gcc on first use, wraps it with ctypes, and strings the
+functions together in the order of Algorithm 1's loop body:
+
+    prediction = Forward(student, frame)        head_forward + upsample
+    loss       = ComputeLoss(prediction, label) softmax_ce
+    gradients  = PartialBackward(loss)          upsample_adjoint, conv_wgrad (+ dgrad between head layers)
+    student    = OptimStep(student, gradients)  sgd
+    metric     = ComputeMetric(prediction,label) confusion + miou      (Section 3.2)
+
+and UpdatedPart(student) (Algorithm 3) = ``pack``.
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+import subprocess
+from dataclasses import dataclass, field
+from typing import List, Optional, Tuple
+
+import numpy as np
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+_SRC = os.path.join(_HERE, "st_oracle.c")
+_LIBS = {}
+
+_c_i64 = ctypes.c_int64
+_c_int = ctypes.c_int
+
+
+def build(force: bool = False) -> None:
+    """Compile st_oracle.c twice: fp32 storage and fp64 storage."""
+    for tag, ctype in (("f32", "float"), ("f64", "double")):
+        out = os.path.join(_HERE, f"libst_oracle_{tag}.so")
+        if (not force and os.path.exists(out)
+                and os.path.getmtime(out) >= os.path.getmtime(_SRC)):
+            continue
+        tmp = out + f".tmp{os.getpid()}"
+        cmd = ["gcc", "-O2", "-ffp-contract=off", "-fopenmp", "-fPIC", "-shared", "-std=c99",
+               f"-DST_REAL={ctype}", _SRC, "-o", tmp, "-lm"]
+        subprocess.run(cmd, check=True)
+        os.replace(tmp, out)
+
+
+def _lib(dtype) -> ctypes.CDLL:
+    tag = "f64" if np.dtype(dtype) == np.float64 else "f32"
+    if tag not in _LIBS:
+        build()
+        lib = ctypes.CDLL(os.path.join(_HERE, f"libst_oracle_{tag}.so"))
+        lib.so_miou.restype = ctypes.c_double
+        lib.so_softmax_ce.restype = _c_i64
+        lib.so_confusion.restype = _c_i64
+        assert lib.so_sizeof_real() == (8 if tag == "f64" else 4)
+        _LIBS[tag] = lib
+    return _LIBS[tag]
+
+
+def _p(a: np.ndarray):
+    return a.ctypes.data_as(ctypes.c_void_p)
+
+
+def _real(dtype):
+    return ctypes.c_double if np.dtype(dtype) == np.float64 else ctypes.c_float
+
+
+def _c(a, dtype=None) -> np.ndarray:
+    return np.ascontiguousarray(a, dtype=dtype)
+
+
+# ----------------------------------------------------------------------------
+# single operations
+# ----------------------------------------------------------------------------
+def teacher_labels(T: np.ndarray) -> np.ndarray:
+    """Pseudo-label map from teacher logits [C][H][W] (Algorithm 3): uint8 [H][W]."""
+    T = _c(T)
+    C, H, W = T.shape
+    out = np.empty((H, W), dtype=np.uint8)
+    _lib(T.dtype).so_labels(_p(T), _c_int(C), _c_i64(H * W), _p(out))
+    return out
+
+
+def conv_fwd(x: np.ndarray, W: np.ndarray, b: np.ndarray, relu: bool = False) -> np.ndarray:
+    x = _c(x)
+    W = _c(W, x.dtype)
+    b = _c(b, x.dtype)
+    Cin, h, w = x.shape
+    Cout, Cin2, ks, ks2 = W.shape
+    assert Cin2 == Cin and ks == ks2 and ks in (1, 3)
+    out = np.empty((Cout, h, w), dtype=x.dtype)
+    _lib(x.dtype).so_conv_fwd(_p(x), _c_int(Cin), _c_int(h), _c_int(w), _p(W), _p(b),
+                              _c_int(Cout), _c_int(ks), _c_int(int(relu)), _p(out))
+    return out
+
+
+def upsample(z: np.ndarray, s: int) -> np.ndarray:
+    z = _c(z)
+    C, h, w = z.shape
+    u = np.empty((C, h * s, w * s), dtype=z.dtype)
+    _lib(z.dtype).so_upsample(_p(z), _c_int(C), _c_int(h), _c_int(w), _c_int(s), _p(u))
+    return u
+
+
+def upsample_adjoint(g: np.ndarray, s: int) -> np.ndarray:
+    g = _c(g)
+    C, H, W = g.shape
+    h, w = H // s, W // s
+    dz = np.empty((C, h, w), dtype=g.dtype)
+    _lib(g.dtype).so_upsample_adjoint(_p(g), _c_int(C), _c_int(h), _c_int(w), _c_int(s), _p(dz))
+    return dz
+
+
+def softmax_ce(u: np.ndarray, labels: np.ndarray, want_grad: bool = True):
+    """(mean loss as float, gradient [C][H][W] or None, number of out-of-range labels)."""
+    u = _c(u)
+    labels = _c(labels, np.uint8)
+    C, H, W = u.shape
+    g = np.empty_like(u) if want_grad else None
+    loss = ctypes.c_double(0.0)
+    bad = _lib(u.dtype).so_softmax_ce(_p(u), _p(labels), _c_int(C), _c_i64(H * W),
+                                      _p(g) if want_grad else None, ctypes.byref(loss))
+    return loss.value, g, int(bad)
+
+
+def conv_wgrad(x: np.ndarray, dout: np.ndarray, ks: int):
+    x = _c(x)
+    dout = _c(dout, x.dtype)
+    Cin, h, w = x.shape
+    Cout = dout.shape[0]
+    dW = np.empty((Cout, Cin, ks, ks), dtype=x.dtype)
+    db = np.empty((Cout,), dtype=x.dtype)
+    _lib(x.dtype).so_conv_wgrad(_p(x), _p(dout), _c_int(Cin), _c_int(Cout), _c_int(h), _c_int(w),
+                                _c_int(ks), _p(dW), _p(db))
+    return dW, db
+
+
+def bias_grad(dout: np.ndarray) -> np.ndarray:
+    dout = _c(dout)
+    Cout = dout.shape[0]
+    db = np.empty((Cout,), dtype=dout.dtype)
+    _lib(dout.dtype).so_bias_grad(_p(dout), _c_int(Cout), _c_i64(dout.size // Cout), _p(db))
+    return db
+
+
+def conv1x1_dgrad(W2: np.ndarray, dz: np.ndarray) -> np.ndarray:
+    dz = _c(dz)
+    W2 = _c(W2, dz.dtype)
+    C, h, w = dz.shape
+    Ch = W2.shape[1]
+    dH = np.empty((Ch, h, w), dtype=dz.dtype)
+    _lib(dz.dtype).so_conv1x1_dgrad(_p(W2), _p(dz), _c_int(C), _c_int(Ch), _c_i64(h * w), _p(dH))
+    return dH
+
+
+def relu_mask_(dH: np.ndarray, Hact: np.ndarray) -> None:
+    assert dH.flags.c_contiguous and Hact.flags.c_contiguous and dH.dtype == Hact.dtype
+    _lib(dH.dtype).so_relu_mask(_p(dH), _p(Hact), _c_i64(dH.size))
+
+
+def sgd_(theta: np.ndarray, v: np.ndarray, g: np.ndarray, lr: float, mu: float) -> None:
+    assert theta.flags.c_contiguous and v.flags.c_contiguous
+    g = _c(g, theta.dtype)
+    R = _real(theta.dtype)
+    _lib(theta.dtype).so_sgd(_p(theta), _p(v), _p(g), _c_i64(theta.size), R(lr), R(mu))
+
+
+def confusion(labels: np.ndarray, pred: np.ndarray, C: int):
+    """(conf int64 [C][C] with conf[label][pred], number of skipped pixels)."""
+    labels = _c(labels, np.uint8)
+    pred = _c(pred, np.uint8)
+    conf = np.zeros((C, C), dtype=np.int64)
+    bad = _lib(np.float32).so_confusion(_p(labels), _p(pred), _c_i64(labels.size), _c_int(C), _p(conf))
+    return conf, int(bad)
+
+
+def miou(conf: np.ndarray) -> float:
+    conf = _c(conf, np.int64)
+    return float(_lib(np.float32).so_miou(_p(conf), _c_int(conf.shape[0])))
+
+
+def round_bf16(a: np.ndarray) -> np.ndarray:
+    out = _c(a).copy()
+    _lib(out.dtype).so_round_bf16(_p(out), _c_i64(out.size))
+    return out
+
+
+# ----------------------------------------------------------------------------
+# the head and one iteration of Algorithm 1's loop body
+# ----------------------------------------------------------------------------
+def param_shapes(c_in: int, c_hidden: int, n_classes: int):
+    if c_hidden == 0:
+        return [((n_classes, c_in, 1, 1), (n_classes,))]
+    return [((c_hidden, c_in, 3, 3), (c_hidden,)), ((n_classes, c_hidden, 1, 1), (n_classes,))]
+
+
+@dataclass
+class Head:
+    """Trainable back part of the student: conv weights/biases plus momentum buffers."""
+    c_in: int
+    c_hidden: int
+    n_classes: int
+    up: int = 4
+    lr: float = 0.01
+    momentum: float = 0.0
+    dtype: type = np.float32
+    quantize_bf16: bool = False      # test-only: round GEMM operands to bf16 like the tensor-core path
+    theta: np.ndarray = None         # flat parameters in packed order
+    vel: np.ndarray = None           # momentum, same order, starts at zero
+
+    def __post_init__(self):
+        n = sum(int(np.prod(ws)) + int(np.prod(bs))
+                for ws, bs in param_shapes(self.c_in, self.c_hidden, self.n_classes))
+        if self.theta is None:
+            self.theta = np.zeros(n, dtype=self.dtype)
+        self.theta = np.ascontiguousarray(self.theta, dtype=self.dtype).copy()
+        assert self.theta.size == n, (self.theta.size, n)
+        self.vel = np.zeros(n, dtype=self.dtype)
+
+    def layers(self) -> List[Tuple[np.ndarray, np.ndarray]]:
+        """Views (weight, bias) into theta, forward order."""
+        out, off = [], 0
+        for ws, bs in param_shapes(self.c_in, self.c_hidden, self.n_classes):
+            nw, nb = int(np.prod(ws)), int(np.prod(bs))
+            out.append((self.theta[off:off + nw].reshape(ws), self.theta[off + nw:off + nw + nb]))
+            off += nw + nb
+        return out
+
+    def _q(self, a):
+        return round_bf16(a) if self.quantize_bf16 else a
+
+
+def head_forward(head: Head, feat: np.ndarray):
+    """Forward of the trainable part over the frozen part's output.
+
+    Returns (z [C][h][w], hidden activation [Ch][h][w] or None).
+    """
+    x = head._q(np.ascontiguousarray(feat, dtype=head.dtype))
+    layers = head.layers()
+    if head.c_hidden == 0:
+        (W, b), = layers
+        return conv_fwd(x, head._q(W), b), None
+    (W1, b1), (W2, b2) = layers
+    Hd = head._q(conv_fwd(x, head._q(W1), b1, relu=True))
+    return conv_fwd(Hd, head._q(W2), b2), Hd
+
+
+def student_mask(head: Head, feat: np.ndarray) -> np.ndarray:
+    """Student prediction at frame resolution: argmax of the upsampled head logits."""
+    z, _ = head_forward(head, feat)
+    return teacher_labels(upsample(z, head.up))
+
+
+def gradients(head: Head, feat: np.ndarray, labels: np.ndarray):
+    """Loss and gradient of every trainable tensor (flat, packed order) at the current parameters.
+
+    Also returns the student mask of this forward (the prediction the loss was computed from).
+    """
+    x = head._q(np.ascontiguousarray(feat, dtype=head.dtype))
+    layers = head.layers()
+    z, Hd = head_forward(head, feat)
+    u = upsample(z, head.up)
+    loss, g, _ = softmax_ce(u, labels)
+    mask = teacher_labels(u)
+    dz = upsample_adjoint(g, head.up)
+    if head.c_hidden == 0:
+        dW, db = conv_wgrad(x, head._q(dz), 1)
+        if head.quantize_bf16:
+            db = bias_grad(dz)
+        grad = np.concatenate([dW.ravel(), db.ravel()])
+        return loss, grad, mask
+    (W1, b1), (W2, b2) = layers
+    dW2, db2 = conv_wgrad(Hd, head._q(dz), 1)
+    dH = conv1x1_dgrad(head._q(W2.reshape(W2.shape[0], W2.shape[1])), head._q(dz))
+    relu_mask_(dH, Hd)
+    dW1, db1 = conv_wgrad(x, head._q(dH), 3)
+    if head.quantize_bf16:
+        db2, db1 = bias_grad(dz), bias_grad(dH)
+    grad = np.concatenate([dW1.ravel(), db1.ravel(), dW2.ravel(), db2.ravel()])
+    return loss, grad, mask
+
+
+def distill_step(head: Head, feat: np.ndarray, labels: np.ndarray):
+    """One iteration of Algorithm 1's loop: loss and gradients at the current
+    parameters, then one optimiser step.  Returns (loss, student mask before the update)."""
+    loss, grad, mask = gradients(head, feat, labels)
+    sgd_(head.theta, head.vel, grad.astype(head.dtype), head.lr, head.momentum)
+    return loss, mask
+
+
+def pack(head: Head) -> bytes:
+    """UpdatedPart(student) (Algorithm 3): per trainable layer in forward order the weight
+    [Cout][Cin][kh][kw] then the bias [Cout], fp32 little-endian values, no header."""
+    return np.ascontiguousarray(head.theta, dtype="<f4").tobytes()
+
+
+def agreement(labels: np.ndarray, pred: np.ndarray, C: int):
+    conf, bad = confusion(labels, pred, C)
+    return conf, miou(conf), bad

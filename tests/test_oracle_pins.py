@@ -1,0 +1,384 @@
+"""Pins for the CPU oracle: each function is checked against something other than
+itself (closed forms, invariants, brute force, library routines, the paper's
+printed sizes), so that a dropped term, a wrong sign/index or a transposed
+operand fails at least one test.  CPU only.
+"""
+import itertools
+import os
+
+import numpy as np
+import pytest
+
+import oracle
+import synth_inputs as si
+
+GOLDEN = os.path.join(os.path.dirname(__file__), "golden")
+
+
+def _golden(name):
+    out = {}
+    with open(os.path.join(GOLDEN, name)) as f:
+        for line in f:
+            line = line.strip()
+            if not line or line.startswith("#"):
+                continue
+            k, *v = line.split()
+            out[k] = [float(t) for t in v]
+    return out
+
+
+# ---------------------------------------------------------------------------- labels
+def test_labels_brute_force_and_ties():
+    rng = np.random.default_rng(1)
+    T = rng.integers(-2, 3, size=(5, 7, 9)).astype(np.float32)   # many exact ties
+    got = oracle.teacher_labels(T)
+    for y in range(7):
+        for x in range(9):
+            col = T[:, y, x]
+            best = max(col)
+            first = [c for c in range(5) if col[c] == best][0]   # lowest index wins
+            assert got[y, x] == first
+    assert got.dtype == np.uint8
+    # property: chosen value >= all others, strictly greater than every lower index
+    chosen = np.take_along_axis(T, got[None].astype(np.int64), 0)[0]
+    assert (chosen[None] >= T).all()
+    for c in range(5):
+        lower = (np.arange(5)[:, None, None] < got[None]) & (T == chosen[None])
+        assert not lower.any()
+
+
+def test_labels_recover_voronoi_map():
+    cfg = si.get_config(1)
+    T = si.teacher_logits(cfg)
+    cls = si.voronoi_map(cfg.frame_h, cfg.frame_w, cfg.n_regions, cfg.n_classes, 2000)
+    # the winner is exactly 4.0 and the noise N(0, 0.5) never reaches 4.0 (8 sigma)
+    assert (oracle.teacher_labels(T) == cls).all()
+
+
+def test_label_map_is_one_byte_per_pixel_table4():
+    g = _golden("table4_sizes.txt")
+    lab = oracle.teacher_labels(np.zeros((2, 720, 1280), np.float32))
+    assert lab.nbytes == 1280 * 720
+    assert round(lab.nbytes / 2**20, 3) == g["label_map_to_client_mb"][0]
+    assert round(1280 * 720 * 3 / 2**20, 3) == g["frame_to_server_mb"][0]
+
+
+# ---------------------------------------------------------------------------- conv forward
+def test_conv1x1_is_a_matrix_product():
+    rng = np.random.default_rng(2)
+    x = rng.standard_normal((6, 5, 7)).astype(np.float32)
+    W = rng.standard_normal((4, 6, 1, 1)).astype(np.float32)
+    b = rng.standard_normal(4).astype(np.float32)
+    got = oracle.conv_fwd(x, W, b)
+    ref = (W.reshape(4, 6).astype(np.float64) @ x.reshape(6, -1).astype(np.float64)
+           + b[:, None]).reshape(4, 5, 7)
+    np.testing.assert_allclose(got, ref, rtol=1e-6, atol=1e-6)
+    # W[co][ci] is not W[ci][co]: a transposed operand would fail on a non-square case above
+
+
+def test_conv3x3_centre_tap_reduces_to_1x1_and_border_counts():
+    rng = np.random.default_rng(3)
+    x = rng.standard_normal((3, 6, 8)).astype(np.float32)
+    W1 = rng.standard_normal((5, 3, 1, 1)).astype(np.float32)
+    b = rng.standard_normal(5).astype(np.float32)
+    W3 = np.zeros((5, 3, 3, 3), np.float32)
+    W3[:, :, 1, 1] = W1[:, :, 0, 0]
+    np.testing.assert_array_equal(oracle.conv_fwd(x, W3, b), oracle.conv_fwd(x, W1, b))
+    ones = np.ones((1, 4, 5), np.float32)
+    cnt = oracle.conv_fwd(ones, np.ones((1, 1, 3, 3), np.float32), np.zeros(1, np.float32))[0]
+    assert cnt[0, 0] == 4 and cnt[0, 2] == 6 and cnt[2, 0] == 6 and cnt[1, 1] == 9 and cnt[3, 4] == 4
+
+
+def test_conv3x3_single_tap_shifts_the_right_way():
+    # weight at (ky,kx)=(0,2) reads in[y-1][x+1]
+    x = np.zeros((1, 5, 5), np.float32)
+    x[0, 1, 3] = 7.0
+    W = np.zeros((1, 1, 3, 3), np.float32)
+    W[0, 0, 0, 2] = 1.0
+    out = oracle.conv_fwd(x, W, np.zeros(1, np.float32))[0]
+    assert out[2, 2] == 7.0 and out.sum() == 7.0
+
+
+def test_conv_and_relu_vs_torch():
+    torch = pytest.importorskip("torch")
+    rng = np.random.default_rng(4)
+    x = rng.standard_normal((4, 7, 9)).astype(np.float32)
+    W = rng.standard_normal((6, 4, 3, 3)).astype(np.float32)
+    b = rng.standard_normal(6).astype(np.float32)
+    ref = torch.relu(torch.nn.functional.conv2d(torch.from_numpy(x)[None].double(),
+                                                torch.from_numpy(W).double(),
+                                                torch.from_numpy(b).double(), padding=1))[0].numpy()
+    np.testing.assert_allclose(oracle.conv_fwd(x, W, b, relu=True), ref, rtol=1e-5, atol=1e-5)
+
+
+# ---------------------------------------------------------------------------- upsample
+def test_upsample_invariants():
+    const = np.full((2, 3, 5), 1.7, np.float32)
+    assert (oracle.upsample(const, 4) == np.float32(1.7)).all()
+    rng = np.random.default_rng(5)
+    z = rng.standard_normal((2, 4, 6)).astype(np.float32)
+    np.testing.assert_array_equal(oracle.upsample(z, 1), z)
+    # affine ramp reproduced exactly in the interior (away from the clamped border)
+    yy, xx = np.meshgrid(np.arange(6.0), np.arange(7.0), indexing="ij")
+    ramp = (2.0 * yy - 3.0 * xx + 1.0)[None].astype(np.float64)
+    u = oracle.upsample(ramp, 4)[0]
+    Y, X = np.meshgrid(np.arange(24.0), np.arange(28.0), indexing="ij")
+    ref = 2.0 * ((Y + 0.5) / 4 - 0.5) - 3.0 * ((X + 0.5) / 4 - 0.5) + 1.0
+    np.testing.assert_allclose(u[2:-2, 2:-2], ref[2:-2, 2:-2], rtol=0, atol=1e-12)
+    # borders clamp to the edge value
+    assert u[0, 0] == ramp[0, 0, 0] and u[-1, -1] == ramp[0, -1, -1]
+
+
+def test_upsample_row_weights_are_eighths():
+    # for s = 4 and Y = 4q + r the two source rows carry weights (3/8,5/8), (1/8,7/8), (7/8,1/8), (5/8,3/8)
+    z = np.zeros((1, 3, 1), np.float64)
+    z[0, 1, 0] = 1.0
+    u = oracle.upsample(z, 4)[0, :, 0]
+    np.testing.assert_array_equal(u, [0, 0, 1 / 8, 3 / 8, 5 / 8, 7 / 8, 7 / 8, 5 / 8, 3 / 8, 1 / 8, 0, 0])
+
+
+def test_upsample_vs_torch_interpolate():
+    torch = pytest.importorskip("torch")
+    rng = np.random.default_rng(6)
+    z = rng.standard_normal((3, 5, 7)).astype(np.float32)
+    ref = torch.nn.functional.interpolate(torch.from_numpy(z)[None].double(), scale_factor=4,
+                                          mode="bilinear", align_corners=False)[0].numpy()
+    np.testing.assert_allclose(oracle.upsample(z, 4), ref, rtol=1e-6, atol=1e-6)
+    ref2 = torch.nn.functional.interpolate(torch.from_numpy(z)[None].double(), scale_factor=2,
+                                           mode="bilinear", align_corners=False)[0].numpy()
+    np.testing.assert_allclose(oracle.upsample(z, 2), ref2, rtol=1e-6, atol=1e-6)
+
+
+def test_adjoint_dot_product_identity():
+    rng = np.random.default_rng(7)
+    a = rng.standard_normal((2, 4, 5))
+    g = rng.standard_normal((2, 16, 20))
+    lhs = float((oracle.upsample(a, 4) * g).sum())
+    rhs = float((a * oracle.upsample_adjoint(g, 4)).sum())
+    assert abs(lhs - rhs) <= 1e-11 * max(1.0, abs(lhs))
+
+
+# ---------------------------------------------------------------------------- loss and its gradient
+def test_ce_gradient_closed_form():
+    rng = np.random.default_rng(8)
+    u = rng.standard_normal((5, 6, 7)) * 3
+    lab = rng.integers(0, 5, size=(6, 7)).astype(np.uint8)
+    loss, g, bad = oracle.softmax_ce(u, lab)
+    assert bad == 0
+    P = 42
+    e = np.exp(u - u.max(0))
+    p = e / e.sum(0)
+    onehot = (np.arange(5)[:, None, None] == lab[None])
+    np.testing.assert_allclose(g, (p - onehot) / P, rtol=1e-12, atol=1e-15)
+    np.testing.assert_allclose(g.sum(0), 0, atol=1e-15)            # rows of p - onehot sum to 0
+    ref_loss = float(np.mean(np.log(np.exp(u).sum(0)) - np.take_along_axis(u, lab[None].astype(np.int64), 0)[0]))
+    assert abs(loss - ref_loss) < 1e-12
+    # shift invariance and a large offset (the max subtraction must be there)
+    loss2, _, _ = oracle.softmax_ce(u + 900.0, lab)
+    assert abs(loss2 - loss) < 1e-9
+
+
+def test_ce_vs_torch():
+    torch = pytest.importorskip("torch")
+    rng = np.random.default_rng(9)
+    u = rng.standard_normal((4, 5, 6)).astype(np.float32)
+    lab = rng.integers(0, 4, size=(5, 6)).astype(np.uint8)
+    loss, _, _ = oracle.softmax_ce(u, lab)
+    ref = torch.nn.functional.cross_entropy(torch.from_numpy(u)[None].double(),
+                                            torch.from_numpy(lab.astype(np.int64))[None]).item()
+    assert abs(loss - ref) < 1e-7
+
+
+def test_zero_weights_closed_form():
+    # W = 0, b = 0 -> logits 0 -> loss = ln C, db[c] = 1/C - n_c/P, dW rows sum to 0 over classes
+    cfgC, cin, h, w = 5, 3, 4, 6
+    rng = np.random.default_rng(10)
+    feat = rng.standard_normal((cin, h, w))
+    lab = rng.integers(0, cfgC, size=(4 * h, 4 * w)).astype(np.uint8)
+    head = oracle.Head(cin, 0, cfgC, dtype=np.float64)
+    loss, grad, _ = oracle.gradients(head, feat, lab)
+    assert abs(loss - np.log(cfgC)) < 1e-12
+    dW = grad[:cfgC * cin].reshape(cfgC, cin)
+    db = grad[cfgC * cin:]
+    counts = np.bincount(lab.ravel(), minlength=cfgC)
+    np.testing.assert_allclose(db, 1.0 / cfgC - counts / lab.size, atol=1e-13)
+    np.testing.assert_allclose(dW.sum(0), 0, atol=1e-12)
+
+
+def test_ce_out_of_range_labels_are_skipped_and_counted():
+    u = np.zeros((3, 2, 2))
+    lab = np.array([[0, 1], [7, 2]], np.uint8)
+    loss, g, bad = oracle.softmax_ce(u, lab)
+    assert bad == 1 and (g[:, 1, 0] == 0).all()
+    assert abs(loss - 3 * np.log(3) / 4) < 1e-12
+
+
+# ---------------------------------------------------------------------------- whole gradient
+def _fd_check(c_hidden):
+    rng = np.random.default_rng(11 + c_hidden)
+    cin, C, h, w = 3, 3, 3, 5
+    feat = np.abs(rng.standard_normal((cin, h, w))) + 0.1
+    lab = rng.integers(0, C, size=(4 * h, 4 * w)).astype(np.uint8)
+    n = si.head_param_count(cin, c_hidden, C)
+    theta = rng.standard_normal(n) * 0.5
+    if c_hidden:
+        # keep hidden pre-activations away from the ReLU kink: positive weights + positive bias on layer 1
+        nw1 = c_hidden * cin * 9
+        theta[:nw1] = np.abs(theta[:nw1]) * 0.3
+        theta[nw1:nw1 + c_hidden] = 0.5
+        theta[nw1] *= -1.0        # one negative weight keeps it generic but far from 0 pre-activation
+    head = oracle.Head(cin, c_hidden, C, dtype=np.float64, theta=theta)
+    loss, grad, _ = oracle.gradients(head, feat, lab)
+
+    def f(th):
+        hd = oracle.Head(cin, c_hidden, C, dtype=np.float64, theta=th)
+        z, _ = oracle.head_forward(hd, feat)
+        return oracle.softmax_ce(oracle.upsample(z, 4), lab, want_grad=False)[0]
+
+    eps = 1e-6
+    fd = np.empty(n)
+    for i in range(n):
+        tp, tm = theta.copy(), theta.copy()
+        tp[i] += eps
+        tm[i] -= eps
+        fd[i] = (f(tp) - f(tm)) / (2 * eps)
+    err = np.abs(fd - grad).max() / max(np.abs(fd).max(), 1e-12)
+    assert err < 1e-6, err
+
+
+def test_finite_differences_1x1_head():
+    _fd_check(0)
+
+
+def test_finite_differences_two_layer_head():
+    _fd_check(2)
+
+
+def test_step_vs_torch_autograd():
+    torch = pytest.importorskip("torch")
+    rng = np.random.default_rng(13)
+    cin, ch, C, h, w = 4, 5, 3, 4, 6
+    feat = np.maximum(rng.standard_normal((cin, h, w)), 0)
+    lab = rng.integers(0, C, size=(4 * h, 4 * w)).astype(np.uint8)
+    theta = si.initial_head_params(cin, ch, C, 5).astype(np.float64)
+    theta[ch * cin * 9: ch * cin * 9 + ch] = 0.05
+    head = oracle.Head(cin, ch, C, dtype=np.float64, theta=theta, lr=0.1, momentum=0.9)
+    tt = [torch.tensor(a.copy(), requires_grad=True) for wb in head.layers() for a in wb]
+    opt = torch.optim.SGD(tt, lr=0.1, momentum=0.9)
+    x = torch.from_numpy(feat)[None]
+    y = torch.from_numpy(lab.astype(np.int64))[None]
+    for _ in range(3):
+        loss_o, _ = oracle.distill_step(head, feat, lab)
+        opt.zero_grad()
+        hdn = torch.relu(torch.nn.functional.conv2d(x, tt[0], tt[1], padding=1))
+        z = torch.nn.functional.conv2d(hdn, tt[2], tt[3])
+        u = torch.nn.functional.interpolate(z, scale_factor=4, mode="bilinear", align_corners=False)
+        loss_t = torch.nn.functional.cross_entropy(u, y)
+        loss_t.backward()
+        opt.step()
+        assert abs(loss_o - loss_t.item()) < 1e-10
+    ref = np.concatenate([t.detach().numpy().ravel() for t in tt])
+    np.testing.assert_allclose(head.theta, ref, rtol=1e-9, atol=1e-11)
+
+
+def test_partial_backward_leaves_features_untouched_and_loss_decreases():
+    cfg = si.WorkloadConfig("t", 8, 0, 3, 6, 8)
+    rng = np.random.default_rng(14)
+    feat = np.maximum(rng.standard_normal((8, 6, 8)), 0).astype(np.float32)
+    lab = rng.integers(0, 3, size=(24, 32)).astype(np.uint8)
+    feat0 = feat.copy()
+    head = oracle.Head(8, 0, 3, theta=si.initial_head_params(8, 0, 3, 1), lr=0.05)
+    losses = [oracle.distill_step(head, feat, lab)[0] for _ in range(6)]
+    np.testing.assert_array_equal(feat, feat0)
+    assert all(b < a for a, b in zip(losses, losses[1:]))
+
+
+# ---------------------------------------------------------------------------- optimiser
+def test_sgd_momentum_closed_form():
+    g = np.array([0.5, -2.0, 0.0], np.float64)
+    theta = np.array([1.0, 2.0, 3.0], np.float64)
+    th0 = theta.copy()
+    v = np.zeros(3)
+    mu, lr = 0.9, 0.01
+    total_v = np.zeros(3)
+    for t in range(1, 6):
+        oracle.sgd_(theta, v, g, lr, mu)
+        np.testing.assert_allclose(v, g * (1 - mu**t) / (1 - mu), rtol=1e-13)
+        total_v += v
+    np.testing.assert_allclose(theta, th0 - lr * total_v, rtol=1e-13)
+    # mu = 0 is plain gradient descent
+    th = np.array([1.0]); vv = np.zeros(1)
+    oracle.sgd_(th, vv, np.array([2.0]), 0.25, 0.0)
+    assert th[0] == 0.5 and vv[0] == 2.0
+
+
+# ---------------------------------------------------------------------------- pack
+def test_pack_layout_and_sizes():
+    cin, ch, C = 3, 2, 4
+    n = si.head_param_count(cin, ch, C)
+    head = oracle.Head(cin, ch, C, theta=np.arange(n, dtype=np.float32))
+    raw = oracle.pack(head)
+    assert raw == np.arange(n, dtype="<f4").tobytes()         # values, fp32, no header
+    (W1, b1), (W2, b2) = head.layers()
+    assert W1.shape == (ch, cin, 3, 3) and W1[1, 2, 0, 1] == 1 * 27 + 2 * 9 + 1
+    assert b1[0] == ch * cin * 9 and W2[0, 0, 0, 0] == ch * cin * 9 + ch
+    assert b2[-1] == n - 1
+    # sizes of the workloads' packed buffers
+    assert si.head_param_count(256, 0, 21) * 4 == 21588
+    assert si.head_param_count(64, 0, 4) * 4 == 1040
+    assert si.head_param_count(256, 256, 21) * 4 == 2381908
+    assert si.head_param_count(256, 256, 19) * 4 == 2379852
+    # K = 0 leaves parameters bit-identical; pack -> init -> pack round-trips
+    head2 = oracle.Head(cin, ch, C, theta=np.frombuffer(raw, "<f4"))
+    assert oracle.pack(head2) == raw
+
+
+def test_table4_parameter_bytes_are_fp32():
+    g = _golden("table4_sizes.txt")
+    full = g["student_params_million"][0] * 1e6 * 4 / 2**20
+    assert abs(full - g["full_student_mb"][0]) / g["full_student_mb"][0] < 0.02
+    part = full * g["trained_fraction"][0]
+    assert abs(part - g["updated_part_mb"][0]) / g["updated_part_mb"][0] < 0.02
+
+
+# ---------------------------------------------------------------------------- metric
+def test_confusion_and_miou():
+    g = _golden("miou_hand_example.txt")
+    lab = np.array(g["label"], np.uint8)
+    pred = np.array(g["pred"], np.uint8)
+    conf, m, bad = oracle.agreement(lab, pred, 2)
+    assert conf.ravel().tolist() == g["conf"] and bad == 0
+    assert abs(m - g["miou"][0]) < 1e-15
+    _, m3, _ = oracle.agreement(np.array(g["label3"], np.uint8), np.array(g["pred3"], np.uint8), 3)
+    assert abs(m3 - g["miou3"][0]) < 1e-15
+    rng = np.random.default_rng(15)
+    lab = rng.integers(0, 6, 500).astype(np.uint8)
+    pred = rng.integers(0, 6, 500).astype(np.uint8)
+    conf, m, bad = oracle.agreement(lab, pred, 6)
+    brute = np.zeros((6, 6), np.int64)
+    for l, q in zip(lab, pred):
+        brute[l, q] += 1
+    np.testing.assert_array_equal(conf, brute)                  # conf[label][pred], not transposed
+    assert conf.sum() == 500
+    np.testing.assert_array_equal(conf.sum(1), np.bincount(lab, minlength=6))
+    ious = []
+    for c in range(6):
+        inter = np.sum((lab == c) & (pred == c))
+        union = np.sum((lab == c) | (pred == c))
+        ious.append(inter / union)
+    assert abs(m - np.mean(ious)) < 1e-15
+    assert oracle.agreement(lab, lab, 6)[1] == 1.0
+    assert oracle.agreement(lab, (lab + 1) % 6, 6)[1] == 0.0
+    _, _, bad = oracle.agreement(np.array([0, 9], np.uint8), np.array([0, 0], np.uint8), 6)
+    assert bad == 1
+
+
+def test_round_bf16_ties_to_even():
+    a = np.array([1.0, 1.00390625, 1.01171875, -1.00390625, 0.0], np.float32)
+    # 1 + 2^-8 is halfway between 1 and 1 + 2^-7 -> even (1.0); 1 + 3*2^-8 -> 1 + 2^-6 (even mantissa)
+    np.testing.assert_array_equal(oracle.round_bf16(a),
+                                  np.array([1.0, 1.0, 1.015625, -1.0, 0.0], np.float32))
+    x = np.random.default_rng(0).standard_normal(1000).astype(np.float32)
+    torch = pytest.importorskip("torch")
+    ref = torch.from_numpy(x).to(torch.bfloat16).to(torch.float32).numpy()
+    np.testing.assert_array_equal(oracle.round_bf16(x), ref)
