@@ -1,0 +1,191 @@
+/*
+ * shadowtutor.h — C ABI of the key-frame partial-distillation step (ShadowTutor, ICPP'20).
+ *
+ * The library implements the body of the server loop (Algorithm 3) minus the teacher
+ * network and the transport: the teacher's per-pixel class logits are reduced to a
+ * one-byte label map, the student's trainable back part (its "head") is trained against
+ * those labels for K optimisation steps over the cached output of the frozen front part
+ * (Algorithm 1's loop body; partial distillation, Section 4.2), the trained subset is
+ * packed for the client (UpdatedPart, Algorithm 3) and student/teacher agreement is
+ * measured as mean IoU (Section 3.2).
+ *
+ * Conventions that hold for every entry point
+ *   - Plain C types only.  "device" = pointer into CUDA device memory of the current
+ *     device; "host" = ordinary (preferably pinned) host memory.  Where a parameter says
+ *     "host or device", the library looks the pointer up and copies from/to host memory
+ *     on the context's CUDA stream itself.
+ *   - The caller owns every buffer it passes.  The library reads or writes it only on the
+ *     context's CUDA stream during work enqueued by that call; it keeps no reference
+ *     afterwards.  Inputs must stay alive until the stream has passed that work.
+ *   - Calls enqueue work on `cuda_stream` and return.  Only calls with a host out-value
+ *     (`st_pack_updated_params` with a host destination, `st_agreement`'s `miou`,
+ *     `st_read_tensor`) wait for the stream.
+ *   - Errors are status codes; nothing aborts, throws or traps.  `st_last_error` gives a
+ *     text for the most recent failure on that context (or, with NULL, of the last failed
+ *     `st_init_head` on this thread).  All shapes are validated on the host before any
+ *     kernel is launched.
+ *   - A context is bound to the device that was current in `st_init_head`, and must be
+ *     used from one host thread at a time.
+ */
+#ifndef SHADOWTUTOR_H_
+#define SHADOWTUTOR_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#if defined(__GNUC__)
+#define ST_API __attribute__((visibility("default")))
+#else
+#define ST_API
+#endif
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef struct st_ctx st_ctx; /* opaque, library-owned */
+
+typedef enum st_status {
+    ST_OK = 0,
+    ST_ERR_INVALID_ARG = 1,      /* NULL where a pointer is required, bad index, bad shape, label >= n_classes */
+    ST_ERR_BAD_STATE = 2,        /* call order: features/labels missing for the stream */
+    ST_ERR_BUFFER_TOO_SMALL = 3, /* destination capacity below the required size */
+    ST_ERR_UNSUPPORTED = 4,      /* a shape the kernels do not cover (see st_init_head) */
+    ST_ERR_OOM = 5,              /* device or host allocation failed */
+    ST_ERR_CUDA = 6              /* a CUDA call or kernel reported an error */
+} st_status;
+
+/* Description of S independent heads of identical shape (one per client video stream). */
+typedef struct st_head_desc {
+    int32_t n_streams;      /* S >= 1: independent heads, each with its own features/labels/parameters */
+    int32_t c_in;           /* channels of the frozen part's output */
+    int32_t c_hidden;       /* 0: head = 1x1 conv c_in -> n_classes;
+                               >0: 3x3 conv c_in -> c_hidden (zero pad 1) + ReLU, then 1x1 conv -> n_classes */
+    int32_t n_classes;      /* 2..255 (labels are one byte, Table 4) */
+    int32_t feat_h, feat_w; /* spatial size of the frozen part's output */
+    int32_t up;             /* frame = feature map * up, bilinear (half-pixel centres); must be 4 */
+    int32_t gemm_precision; /* 0: fp32 FMA convolutions; 1: bf16 operands on tensor cores, fp32 accumulate */
+    float lr;               /* learning rate of OptimStep */
+    float momentum;         /* heavy-ball momentum; 0 = plain gradient descent */
+    void *cuda_stream;      /* cudaStream_t on which all work is enqueued (NULL = default stream) */
+} st_head_desc;
+
+/* Number of fp32 values in one head's packed parameter buffer:
+ * per layer in forward order, weight [Cout][Cin][kh][kw] then bias [Cout]. */
+ST_API size_t st_param_count(int32_t c_in, int32_t c_hidden, int32_t n_classes);
+
+/*
+ * st_init_head — create the server-side copy of the student's trainable part
+ * (Algorithm 3 starts from the pre-trained student; Section 4.2 fixes which part is trained).
+ *   desc         host; copied.
+ *   init_params  host or device; S packed buffers back to back (S * st_param_count floats),
+ *                layout as above; copied into fp32 master parameters.  Momentum starts at 0.
+ *   out          host; receives the context.
+ * Allocates all device state (parameters, momentum, caches, scratch) for S streams.
+ * ST_ERR_UNSUPPORTED: up != 4; with gemm_precision 1: c_in or c_hidden not a multiple of
+ * 64, c_hidden > 256, or n_classes > 32.
+ */
+ST_API st_status st_init_head(const st_head_desc *desc, const float *init_params, st_ctx **out);
+
+/*
+ * st_set_frozen_features — cache the frozen front part's output for one key frame.
+ * The frozen layers' outputs do not change across the K steps (Section 4.2), so they are
+ * stored once in the layout the head's GEMMs read (bf16 [h][w][c_in] with
+ * gemm_precision 1, fp32 [c_in][h][w] otherwise).
+ *   stream    0 <= stream < S.
+ *   feat_chw  host or device; fp32 [c_in][feat_h][feat_w], contiguous.
+ */
+ST_API st_status st_set_frozen_features(st_ctx *ctx, int32_t stream, const float *feat_chw);
+
+/*
+ * st_teacher_labels — pseudo-label of the key frame (Algorithm 3: label <- Forward(teacher)):
+ * label[y][x] = argmax_c logits[c][y][x], lowest class index on ties; one byte per pixel.
+ *   logits_chw  host or device; fp32 [n_classes][H][W], H = feat_h*up, W = feat_w*up.
+ *   labels_out  host or device, or NULL; uint8 [H][W].  A copy is always kept in the context
+ *               as the training target of `stream`.
+ */
+ST_API st_status st_teacher_labels(st_ctx *ctx, int32_t stream, const float *logits_chw, uint8_t *labels_out);
+
+/* Install an existing label map (uint8 [H][W], host or device) as the training target. */
+ST_API st_status st_set_labels(st_ctx *ctx, int32_t stream, const uint8_t *labels);
+
+/*
+ * st_distill_step — n_steps iterations of Algorithm 1's loop body on all S streams:
+ * head forward, bilinear x4 upsample, mean per-pixel softmax cross-entropy against the
+ * stored labels (Section 5.2), gradients of the head only (PartialBackward, Section 4.2),
+ * SGD(+momentum) update (OptimStep).
+ *   n_steps   1..64.
+ *   loss_out  host or device, or NULL; fp32 [S][n_steps]: loss of each step's forward.
+ *   conf_out  host or device, or NULL; int64 [S][n_steps][C][C]: conf[label][prediction] of the
+ *             forward that produced that step's loss (the prediction before that step's update).
+ * ST_ERR_BAD_STATE if a stream has no features or labels yet.
+ * Labels >= n_classes are skipped (no loss, no gradient) and make the call that finds them
+ * return ST_ERR_INVALID_ARG at its next synchronising point (`st_agreement`, `st_read_tensor`).
+ */
+ST_API st_status st_distill_step(st_ctx *ctx, int32_t n_steps, float *loss_out, int64_t *conf_out);
+
+/*
+ * st_pack_updated_params — UpdatedPart(student) (Algorithm 3; Table 4 sizes are fp32):
+ * the current values of every trainable tensor of `stream`, fp32 little-endian, per layer in
+ * forward order weight [Cout][Cin][kh][kw] then bias [Cout]; no header, no padding.
+ *   dst           host or device.
+ *   dst_capacity  bytes available at dst; ST_ERR_BUFFER_TOO_SMALL if below the packed size.
+ *   nbytes        host, may be NULL; receives the packed size (also on BUFFER_TOO_SMALL).
+ * Momentum is not part of the buffer.  Feeding the buffer back to st_init_head reproduces
+ * the parameters bit for bit.
+ */
+ST_API st_status st_pack_updated_params(st_ctx *ctx, int32_t stream, void *dst, size_t dst_capacity, size_t *nbytes);
+
+/*
+ * st_student_mask — prediction of the current student at frame resolution:
+ * argmax over classes of the upsampled head logits (fresh forward of the current parameters).
+ *   mask_out  host or device; uint8 [H][W].
+ */
+ST_API st_status st_student_mask(st_ctx *ctx, int32_t stream, uint8_t *mask_out);
+
+/*
+ * st_agreement — ComputeMetric (Algorithm 1): confusion matrix and mean IoU
+ * (Section 3.2: IoU_c = |pred_c ∩ label_c| / |pred_c ∪ label_c|, averaged over the classes
+ * present in the label).
+ *   pred   host or device uint8 [H][W], or NULL = the current student's mask (fresh forward).
+ *   label  host or device uint8 [H][W], or NULL = the stored teacher labels of `stream`.
+ *   conf   host or device, or NULL; int64 [C][C], conf[l][q] = #pixels with label l and prediction q.
+ *   miou   host, or NULL; mean IoU in double.
+ * Pixels whose label or prediction is >= n_classes are skipped and the call returns
+ * ST_ERR_INVALID_ARG (the counts of the valid pixels are still delivered).
+ * Waits for the stream.
+ */
+ST_API st_status st_agreement(st_ctx *ctx, int32_t stream, const uint8_t *pred, const uint8_t *label,
+                       int64_t *conf, double *miou);
+
+/* Intermediate tensors of the most recent step, for verification. */
+typedef enum st_tensor {
+    ST_TENSOR_LOGITS = 0,      /* z, fp32 [C][h][w]: head output of the last forward */
+    ST_TENSOR_LOGIT_GRAD = 1,  /* dz, fp32 [C][h][w]: gradient of the mean loss w.r.t. z */
+    ST_TENSOR_PARAM_GRAD = 2,  /* fp32, packed order: gradient applied by the last update */
+    ST_TENSOR_MOMENTUM = 3,    /* fp32, packed order */
+    ST_TENSOR_HIDDEN = 4,      /* fp32 [c_hidden][h][w]: ReLU output of the 3x3 layer (two-layer head) */
+    ST_TENSOR_HIDDEN_GRAD = 5, /* fp32 [c_hidden][h][w]: gradient w.r.t. the hidden activation (after the ReLU mask) */
+    ST_TENSOR_FEATURES = 6     /* fp32 [c_in][h][w]: the cached features as the GEMMs see them */
+} st_tensor;
+
+/*
+ * st_read_tensor — copy one intermediate tensor of `stream` to host memory as fp32 in the
+ * planar layout listed above (converted from the internal layout/precision).
+ *   dst_host      host; capacity in bytes; *nbytes (may be NULL) receives the size.
+ * Waits for the stream.
+ */
+ST_API st_status st_read_tensor(st_ctx *ctx, int32_t stream, st_tensor which, float *dst_host,
+                         size_t dst_capacity, size_t *nbytes);
+
+/* Number of kernels this library has launched on the context so far. */
+ST_API int64_t st_launch_count(const st_ctx *ctx);
+
+ST_API void st_destroy(st_ctx *ctx);
+ST_API const char *st_last_error(const st_ctx *ctx);
+ST_API const char *st_status_name(st_status s);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* SHADOWTUTOR_H_ */

@@ -1,0 +1,240 @@
+"""Thin Python binding of the key-frame partial-distillation library (libshadowtutor.so).
+
+Argument marshalling only: every function has the name and the meaning of the C entry
+point declared in ``include/shadowtutor.h`` and forwards pointers and sizes to it.  Tensors
+may be ``torch`` tensors (CUDA or CPU) or ``numpy`` arrays; they must be contiguous and of
+the dtype the C interface states.  No arithmetic of the method happens here, and there is
+no fallback: if the CUDA library has not been built the first call raises.
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+from typing import Optional
+
+import numpy as np
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(_HERE, "libshadowtutor.so")
+
+ST_OK = 0
+ST_ERR_INVALID_ARG = 1
+ST_ERR_BAD_STATE = 2
+ST_ERR_BUFFER_TOO_SMALL = 3
+ST_ERR_UNSUPPORTED = 4
+ST_ERR_OOM = 5
+ST_ERR_CUDA = 6
+
+ST_TENSOR_LOGITS = 0
+ST_TENSOR_LOGIT_GRAD = 1
+ST_TENSOR_PARAM_GRAD = 2
+ST_TENSOR_MOMENTUM = 3
+ST_TENSOR_HIDDEN = 4
+ST_TENSOR_HIDDEN_GRAD = 5
+ST_TENSOR_FEATURES = 6
+
+EXPORTED = [
+    "st_param_count", "st_init_head", "st_set_frozen_features", "st_teacher_labels", "st_set_labels",
+    "st_distill_step", "st_pack_updated_params", "st_student_mask", "st_agreement", "st_read_tensor",
+    "st_launch_count", "st_destroy", "st_last_error", "st_status_name",
+]
+
+
+class st_head_desc(ctypes.Structure):
+    _fields_ = [
+        ("n_streams", ctypes.c_int32), ("c_in", ctypes.c_int32), ("c_hidden", ctypes.c_int32),
+        ("n_classes", ctypes.c_int32), ("feat_h", ctypes.c_int32), ("feat_w", ctypes.c_int32),
+        ("up", ctypes.c_int32), ("gemm_precision", ctypes.c_int32),
+        ("lr", ctypes.c_float), ("momentum", ctypes.c_float), ("cuda_stream", ctypes.c_void_p),
+    ]
+
+
+class StError(RuntimeError):
+    def __init__(self, status: int, name: str, message: str):
+        super().__init__(f"{name}: {message}")
+        self.status = status
+        self.status_name = name
+
+
+_lib = None
+
+
+def load_library() -> ctypes.CDLL:
+    """Load libshadowtutor.so (built by ``python -m paper_2003_10735_b200.build``)."""
+    global _lib
+    if _lib is not None:
+        return _lib
+    if not os.path.exists(LIB_PATH):
+        raise ImportError(f"{LIB_PATH} is missing: build it with `python -m paper_2003_10735_b200.build` "
+                          "(there is no CPU fallback)")
+    lib = ctypes.CDLL(LIB_PATH)
+    vp, i32, i64 = ctypes.c_void_p, ctypes.c_int32, ctypes.c_int64
+    lib.st_param_count.restype = ctypes.c_size_t
+    lib.st_param_count.argtypes = [i32, i32, i32]
+    lib.st_init_head.restype = ctypes.c_int
+    lib.st_init_head.argtypes = [ctypes.POINTER(st_head_desc), vp, ctypes.POINTER(vp)]
+    lib.st_set_frozen_features.restype = ctypes.c_int
+    lib.st_set_frozen_features.argtypes = [vp, i32, vp]
+    lib.st_teacher_labels.restype = ctypes.c_int
+    lib.st_teacher_labels.argtypes = [vp, i32, vp, vp]
+    lib.st_set_labels.restype = ctypes.c_int
+    lib.st_set_labels.argtypes = [vp, i32, vp]
+    lib.st_distill_step.restype = ctypes.c_int
+    lib.st_distill_step.argtypes = [vp, i32, vp, vp]
+    lib.st_pack_updated_params.restype = ctypes.c_int
+    lib.st_pack_updated_params.argtypes = [vp, i32, vp, ctypes.c_size_t, ctypes.POINTER(ctypes.c_size_t)]
+    lib.st_student_mask.restype = ctypes.c_int
+    lib.st_student_mask.argtypes = [vp, i32, vp]
+    lib.st_agreement.restype = ctypes.c_int
+    lib.st_agreement.argtypes = [vp, i32, vp, vp, vp, ctypes.POINTER(ctypes.c_double)]
+    lib.st_read_tensor.restype = ctypes.c_int
+    lib.st_read_tensor.argtypes = [vp, i32, ctypes.c_int, vp, ctypes.c_size_t, ctypes.POINTER(ctypes.c_size_t)]
+    lib.st_launch_count.restype = i64
+    lib.st_launch_count.argtypes = [vp]
+    lib.st_destroy.restype = None
+    lib.st_destroy.argtypes = [vp]
+    lib.st_last_error.restype = ctypes.c_char_p
+    lib.st_last_error.argtypes = [vp]
+    lib.st_status_name.restype = ctypes.c_char_p
+    lib.st_status_name.argtypes = [ctypes.c_int]
+    _lib = lib
+    return lib
+
+
+# ---------------------------------------------------------------------------- marshalling
+_NP_OF = {"float32": np.float32, "uint8": np.uint8, "int64": np.int64}
+
+
+def _ptr(buf, dtype: str, min_elems: int, what: str) -> Optional[int]:
+    """Address of a contiguous torch tensor / numpy array of the given dtype, or None."""
+    if buf is None:
+        return None
+    if isinstance(buf, np.ndarray):
+        if buf.dtype != _NP_OF[dtype] or not buf.flags.c_contiguous:
+            raise TypeError(f"{what}: need a C-contiguous {dtype} array, got {buf.dtype}")
+        if buf.size < min_elems:
+            raise ValueError(f"{what}: {buf.size} elements, need {min_elems}")
+        return buf.ctypes.data
+    if hasattr(buf, "data_ptr"):
+        if str(buf.dtype) != "torch." + dtype or not buf.is_contiguous():
+            raise TypeError(f"{what}: need a contiguous {dtype} tensor, got {buf.dtype}")
+        if buf.numel() < min_elems:
+            raise ValueError(f"{what}: {buf.numel()} elements, need {min_elems}")
+        return buf.data_ptr()
+    raise TypeError(f"{what}: expected a torch tensor or numpy array")
+
+
+class _Ctx:
+    """Handle of an st_ctx plus the shape facts needed to size buffers."""
+
+    def __init__(self, handle, desc: st_head_desc):
+        self.handle = handle
+        self.desc = desc
+        self.S, self.C = desc.n_streams, desc.n_classes
+        self.p = desc.feat_h * desc.feat_w
+        self.P = self.p * desc.up * desc.up
+        self.n_params = st_param_count(desc.c_in, desc.c_hidden, desc.n_classes)
+
+    def __del__(self):
+        try:
+            st_destroy(self)
+        except Exception:
+            pass
+
+
+def _check(status: int, ctx: Optional[_Ctx]) -> None:
+    if status == ST_OK:
+        return
+    lib = load_library()
+    msg = lib.st_last_error(ctx.handle if ctx is not None else None)
+    raise StError(status, lib.st_status_name(status).decode(), (msg or b"").decode())
+
+
+# ---------------------------------------------------------------------------- entry points
+def st_param_count(c_in: int, c_hidden: int, n_classes: int) -> int:
+    return int(load_library().st_param_count(c_in, c_hidden, n_classes))
+
+
+def st_init_head(*, n_streams: int = 1, c_in: int, c_hidden: int = 0, n_classes: int, feat_h: int,
+                 feat_w: int, up: int = 4, gemm_precision: int = 0, lr: float = 0.01, momentum: float = 0.0,
+                 cuda_stream: int = 0, init_params) -> _Ctx:
+    lib = load_library()
+    desc = st_head_desc(n_streams, c_in, c_hidden, n_classes, feat_h, feat_w, up, gemm_precision,
+                        lr, momentum, cuda_stream or None)
+    n = n_streams * int(lib.st_param_count(c_in, c_hidden, n_classes))
+    out = ctypes.c_void_p()
+    status = lib.st_init_head(ctypes.byref(desc), _ptr(init_params, "float32", n, "init_params"), ctypes.byref(out))
+    _check(status, None)
+    return _Ctx(out.value, desc)
+
+
+def st_set_frozen_features(ctx: _Ctx, stream: int, feat_chw) -> None:
+    n = ctx.desc.c_in * ctx.p
+    _check(load_library().st_set_frozen_features(ctx.handle, stream, _ptr(feat_chw, "float32", n, "feat_chw")), ctx)
+
+
+def st_teacher_labels(ctx: _Ctx, stream: int, logits_chw, labels_out=None) -> None:
+    _check(load_library().st_teacher_labels(ctx.handle, stream, _ptr(logits_chw, "float32", ctx.C * ctx.P, "logits_chw"),
+                                            _ptr(labels_out, "uint8", ctx.P, "labels_out")), ctx)
+
+
+def st_set_labels(ctx: _Ctx, stream: int, labels) -> None:
+    _check(load_library().st_set_labels(ctx.handle, stream, _ptr(labels, "uint8", ctx.P, "labels")), ctx)
+
+
+def st_distill_step(ctx: _Ctx, n_steps: int, loss_out=None, conf_out=None) -> None:
+    _check(load_library().st_distill_step(ctx.handle, n_steps,
+                                          _ptr(loss_out, "float32", ctx.S * max(n_steps, 0), "loss_out"),
+                                          _ptr(conf_out, "int64", ctx.S * max(n_steps, 0) * ctx.C * ctx.C, "conf_out")), ctx)
+
+
+def st_pack_updated_params(ctx: _Ctx, stream: int, dst, dst_capacity: Optional[int] = None) -> int:
+    """Returns the packed size in bytes."""
+    if dst is None:
+        cap, addr = 0, None
+    else:
+        nelem = dst.size if isinstance(dst, np.ndarray) else dst.numel()
+        cap = nelem * 4 if dst_capacity is None else dst_capacity
+        addr = _ptr(dst, "float32", 0, "dst")
+    nbytes = ctypes.c_size_t(0)
+    _check(load_library().st_pack_updated_params(ctx.handle, stream, addr, cap, ctypes.byref(nbytes)), ctx)
+    return int(nbytes.value)
+
+
+def st_student_mask(ctx: _Ctx, stream: int, mask_out) -> None:
+    _check(load_library().st_student_mask(ctx.handle, stream, _ptr(mask_out, "uint8", ctx.P, "mask_out")), ctx)
+
+
+def st_agreement(ctx: _Ctx, stream: int, pred=None, label=None, conf=None) -> float:
+    """Returns the mean IoU; `conf` (int64 [C][C]) is filled if given."""
+    miou = ctypes.c_double(0.0)
+    _check(load_library().st_agreement(ctx.handle, stream, _ptr(pred, "uint8", ctx.P, "pred"),
+                                       _ptr(label, "uint8", ctx.P, "label"),
+                                       _ptr(conf, "int64", ctx.C * ctx.C, "conf"), ctypes.byref(miou)), ctx)
+    return float(miou.value)
+
+
+def st_read_tensor(ctx: _Ctx, stream: int, which: int) -> np.ndarray:
+    """Copy of one intermediate tensor as a flat fp32 numpy array (verification only)."""
+    lib = load_library()
+    nbytes = ctypes.c_size_t(0)
+    status = lib.st_read_tensor(ctx.handle, stream, which, None, 0, ctypes.byref(nbytes))
+    if nbytes.value == 0:
+        _check(status, ctx)
+    out = np.empty(nbytes.value // 4, dtype=np.float32)
+    _check(lib.st_read_tensor(ctx.handle, stream, which, out.ctypes.data, out.nbytes, ctypes.byref(nbytes)), ctx)
+    return out
+
+
+def st_launch_count(ctx: _Ctx) -> int:
+    return int(load_library().st_launch_count(ctx.handle))
+
+
+def st_destroy(ctx: _Ctx) -> None:
+    if ctx is not None and ctx.handle:
+        load_library().st_destroy(ctx.handle)
+        ctx.handle = None
+
+
+def st_last_error(ctx: Optional[_Ctx]) -> str:
+    return (load_library().st_last_error(ctx.handle if ctx else None) or b"").decode()

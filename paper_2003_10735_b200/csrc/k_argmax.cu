@@ -1,0 +1,61 @@
+// K1 — teacher logits -> one-byte label map (Algorithm 3: label <- Forward(teacher, frame);
+// Table 4: the label map is one byte per pixel).
+//
+// label[p] = argmax_c T[c][p], lowest class index on ties (strict '>' while walking c upward).
+// Pure streaming: C*P*4 bytes in, P bytes out, every input byte used once.  Each thread owns
+// four consecutive pixels, reads one 16-byte vector per class plane with a streaming
+// (evict-first) hint and writes four labels as one 32-bit word, so a warp reads 512
+// contiguous bytes per plane and writes 128.
+#include "st_internal.h"
+
+namespace st {
+
+__global__ void __launch_bounds__(256)
+argmax_u8_vec4_kernel(const float4* __restrict__ T, int C, int64_t n_quads, uint32_t* __restrict__ out)
+{
+    int64_t q = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+    if (q >= n_quads) return;
+    const float4* p = T + q;
+    float4 best = __ldcs(p);
+    uint32_t ix = 0, iy = 0, iz = 0, iw = 0;
+#pragma unroll 8
+    for (int c = 1; c < C; ++c) {
+        float4 v = __ldcs(p + (int64_t)c * n_quads);
+        if (v.x > best.x) { best.x = v.x; ix = c; }
+        if (v.y > best.y) { best.y = v.y; iy = c; }
+        if (v.z > best.z) { best.z = v.z; iz = c; }
+        if (v.w > best.w) { best.w = v.w; iw = c; }
+    }
+    out[q] = ix | (iy << 8) | (iz << 16) | (iw << 24);
+}
+
+// Fallback for pixel counts or pointers that do not allow 16-byte vectors.
+__global__ void __launch_bounds__(256)
+argmax_u8_scalar_kernel(const float* __restrict__ T, int C, int64_t P, uint8_t* __restrict__ out)
+{
+    int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+    if (i >= P) return;
+    float best = __ldcs(T + i);
+    int idx = 0;
+    for (int c = 1; c < C; ++c) {
+        float v = __ldcs(T + (int64_t)c * P + i);
+        if (v > best) { best = v; idx = c; }
+    }
+    out[i] = (uint8_t)idx;
+}
+
+void launch_argmax_u8(const float* logits, int C, int64_t P, uint8_t* labels, cudaStream_t s)
+{
+    if (P <= 0) return;
+    bool vec = (P % 4 == 0) && ((uintptr_t)logits % 16 == 0) && ((uintptr_t)labels % 4 == 0);
+    if (vec) {
+        int64_t nq = P / 4;
+        unsigned blocks = (unsigned)((nq + 255) / 256);
+        argmax_u8_vec4_kernel<<<blocks, 256, 0, s>>>((const float4*)logits, C, nq, (uint32_t*)labels);
+    } else {
+        unsigned blocks = (unsigned)((P + 255) / 256);
+        argmax_u8_scalar_kernel<<<blocks, 256, 0, s>>>(logits, C, P, labels);
+    }
+}
+
+}  // namespace st

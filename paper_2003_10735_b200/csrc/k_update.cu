@@ -1,0 +1,175 @@
+// K5 — OptimStep of Algorithm 1 ("most simply gradient descent", Section 4.1.4) with heavy-ball
+// momentum:  v <- mu*v + g ;  theta <- theta - lr*v   (mu = 0: plain gradient descent),
+// on the fp32 master parameters; the bf16 copies read by the tensor-core GEMMs are refreshed in
+// the same pass.  The kernel also finishes the reductions the step left open, always in a fixed
+// order so that results are bit-reproducible: split-K partial sums of the weight gradients,
+// per-block partial sums of the bias gradients, and the per-block loss partials.
+// K7 — UpdatedPart(student) (Algorithm 3): the packed fp32 buffer of all trainable tensors.
+#include "st_internal.h"
+
+namespace st {
+
+constexpr int kUpdThreads = 256;
+
+__device__ __forceinline__ void apply_update(const UpdateArgs& a, int64_t gi, float g)
+{
+    float v = fmaf(a.mu, a.vel[gi], g);
+    a.vel[gi] = v;
+    a.grad[gi] = g;
+    a.theta[gi] = fmaf(-a.lr, v, a.theta[gi]);
+}
+
+__global__ void __launch_bounds__(kUpdThreads)
+sgd_update_kernel(UpdateArgs a, int n_param_blocks)
+{
+    const int s = blockIdx.y;
+    const int64_t base = (int64_t)s * a.n_params;
+    if ((int)blockIdx.x < n_param_blocks) {
+        const int64_t i = (int64_t)blockIdx.x * kUpdThreads + threadIdx.x;
+        if (i >= a.n_params) return;
+        for (int L = 0; L < a.n_layers; ++L) {
+            const LayerUpdate& ly = a.layer[L];
+            const int64_t nw = (int64_t)ly.cout * ly.cin * ly.taps;
+            if (i >= ly.w_off && i < ly.w_off + nw) {
+                const int64_t e = i - ly.w_off;
+                float g;
+                if (ly.w_partials) {
+                    const float* src = ly.w_partials + (int64_t)s * ly.w_stream_stride + e;
+                    g = 0.f;
+                    for (int k = 0; k < ly.n_split; ++k) g += __ldg(src + (int64_t)k * ly.w_split_stride);
+                } else {
+                    g = a.grad[base + i];
+                }
+                apply_update(a, base + i, g);
+                if (ly.shadow) ly.shadow[(int64_t)s * ly.shadow_stream_stride + e] = __float2bfloat16_rn(a.theta[base + i]);
+                return;
+            }
+            if (i >= ly.b_off && i < ly.b_off + ly.cout) {
+                if (!ly.b_partials) apply_update(a, base + i, a.grad[base + i]);
+                return;   // biases with partial sums are finished by the reduction warps below
+            }
+        }
+        return;
+    }
+    // ---- reduction warps: one warp per bias element that has partial sums, plus one for the loss
+    const int warp = ((int)blockIdx.x - n_param_blocks) * (kUpdThreads / 32) + (threadIdx.x >> 5);
+    const int lane = threadIdx.x & 31;
+    int item = warp;
+    for (int L = 0; L < a.n_layers; ++L) {
+        const LayerUpdate& ly = a.layer[L];
+        if (!ly.b_partials) continue;
+        if (item < ly.cout) {
+            const float* src = ly.b_partials + (int64_t)s * ly.n_bpart * ly.cout + item;
+            float g = 0.f;
+            for (int k = lane; k < ly.n_bpart; k += 32) g += __ldg(src + (int64_t)k * ly.cout);
+#pragma unroll
+            for (int o = 16; o > 0; o >>= 1) g += __shfl_xor_sync(0xffffffffu, g, o);
+            if (lane == 0) apply_update(a, base + ly.b_off + item, g);
+            return;
+        }
+        item -= ly.cout;
+    }
+    if (item == 0 && a.loss_part) {
+        double t = 0.0;
+        for (int k = lane; k < a.n_loss_part; k += 32) t += (double)__ldg(a.loss_part + (int64_t)s * a.n_loss_part + k);
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) t += __shfl_xor_sync(0xffffffffu, t, o);
+        if (lane == 0) {
+            if (a.loss_slot >= 0 && a.loss_slot < kMaxSteps)
+                a.loss_buf[(int64_t)s * kMaxSteps + a.loss_slot] = (float)(t * a.inv_P);
+        }
+    }
+}
+
+void launch_sgd_update(const UpdateArgs& a, cudaStream_t s)
+{
+    const int n_param_blocks = (int)((a.n_params + kUpdThreads - 1) / kUpdThreads);
+    int items = 1;
+    for (int L = 0; L < a.n_layers; ++L) if (a.layer[L].b_partials) items += a.layer[L].cout;
+    const int n_red_blocks = (items + kUpdThreads / 32 - 1) / (kUpdThreads / 32);
+    sgd_update_kernel<<<dim3((unsigned)(n_param_blocks + n_red_blocks), (unsigned)a.S), kUpdThreads, 0, s>>>(a, n_param_blocks);
+}
+
+__global__ void refresh_shadow_kernel(UpdateArgs a)
+{
+    const int s = blockIdx.y;
+    const int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+    if (i >= a.n_params) return;
+    for (int L = 0; L < a.n_layers; ++L) {
+        const LayerUpdate& ly = a.layer[L];
+        const int64_t nw = (int64_t)ly.cout * ly.cin * ly.taps;
+        if (ly.shadow && i >= ly.w_off && i < ly.w_off + nw)
+            ly.shadow[(int64_t)s * ly.shadow_stream_stride + (i - ly.w_off)] =
+                __float2bfloat16_rn(a.theta[(int64_t)s * a.n_params + i]);
+    }
+}
+
+void launch_refresh_shadow(const UpdateArgs& a, cudaStream_t s)
+{
+    refresh_shadow_kernel<<<dim3((unsigned)((a.n_params + 255) / 256), (unsigned)a.S), 256, 0, s>>>(a);
+}
+
+// Mean IoU (Section 3.2): IoU_c = conf[c][c] / (row_c + col_c - conf[c][c]), averaged over the
+// classes present in the label (row_c > 0).  Integer counts, double arithmetic, fixed order.
+__global__ void miou_kernel(const unsigned long long* __restrict__ conf, int C, double* out)
+{
+    __shared__ double iou[256];
+    __shared__ int present[256];
+    const int c = threadIdx.x;
+    double v = 0.0; int pr = 0;
+    if (c < C) {
+        unsigned long long row = 0, col = 0;
+        for (int q = 0; q < C; ++q) { row += conf[c * C + q]; col += conf[q * C + c]; }
+        if (row > 0) {
+            const unsigned long long inter = conf[c * C + c];
+            v = (double)inter / (double)(row + col - inter);
+            pr = 1;
+        }
+    }
+    iou[c] = v; present[c] = pr;
+    __syncthreads();
+    if (c == 0) {
+        double sum = 0.0; int n = 0;
+        for (int k = 0; k < C; ++k) { sum += iou[k]; n += present[k]; }
+        *out = n ? sum / n : 0.0;
+    }
+}
+
+void launch_miou(const unsigned long long* conf, int C, double* out, cudaStream_t s)
+{
+    miou_kernel<<<1, 256, 0, s>>>(conf, C, out);
+}
+
+// ---- pack / unpack ---------------------------------------------------------------------------------
+template <bool TO_PACKED>
+__global__ void pack_kernel(const float* __restrict__ src, float* __restrict__ dst, PackLayout L)
+{
+    const int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;   // index in packed order
+    if (i >= L.n_params) return;
+    const int64_t base = (int64_t)blockIdx.y * L.n_params;
+    int64_t j = i;                                                       // index in internal order
+    for (int k = 0; k < L.n_layers; ++k) {
+        const int64_t nw = (int64_t)L.cout[k] * L.cin[k] * L.taps[k];
+        if (i >= L.w_off[k] && i < L.w_off[k] + nw) {
+            const int64_t e = i - L.w_off[k];
+            const int tap = (int)(e % L.taps[k]);
+            const int64_t r = e / L.taps[k];
+            const int ci = (int)(r % L.cin[k]), co = (int)(r / L.cin[k]);
+            j = L.w_off[k] + ((int64_t)tap * L.cout[k] + co) * L.cin[k] + ci;
+        }
+    }
+    if (TO_PACKED) dst[base + i] = src[base + j];
+    else dst[base + j] = src[base + i];
+}
+
+void launch_pack(const float* internal, float* packed, const PackLayout& L, int n_bufs, cudaStream_t s)
+{
+    pack_kernel<true><<<dim3((unsigned)((L.n_params + 255) / 256), (unsigned)n_bufs), 256, 0, s>>>(internal, packed, L);
+}
+
+void launch_unpack(const float* packed, float* internal, const PackLayout& L, int n_bufs, cudaStream_t s)
+{
+    pack_kernel<false><<<dim3((unsigned)((L.n_params + 255) / 256), (unsigned)n_bufs), 256, 0, s>>>(packed, internal, L);
+}
+
+}  // namespace st

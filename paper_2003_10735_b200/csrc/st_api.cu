@@ -1,0 +1,676 @@
+// C-ABI layer of the key-frame partial-distillation library: context, host-side validation and the
+// order in which the kernels of one step are enqueued (Algorithm 1's loop body; Algorithm 3's
+// label and UpdatedPart).  See include/shadowtutor.h for the contract of every entry point.
+#include "../../include/shadowtutor.h"
+#include "st_internal.h"
+
+#include <cstdarg>
+#include <cstdio>
+#include <cstring>
+#include <map>
+#include <new>
+#include <string>
+#include <vector>
+
+using namespace st;
+
+namespace {
+thread_local std::string g_init_error;
+
+struct GraphKey { int n_steps; bool conf; bool operator<(const GraphKey& o) const { return n_steps != o.n_steps ? n_steps < o.n_steps : conf < o.conf; } };
+}  // namespace
+
+struct st_ctx {
+    st_head_desc d;
+    cudaStream_t stream = nullptr;
+    int device = 0;
+    int S = 0, C = 0, Cin = 0, Ch = 0, h = 0, w = 0, H = 0, W = 0;
+    int64_t p = 0, P = 0, n_params = 0;
+    bool bf16_mode = false;
+    PackLayout layout;
+
+    float *theta = nullptr, *vel = nullptr, *grad = nullptr;
+    float* x_f32 = nullptr;
+    bf16* x_bf16 = nullptr;
+    uint8_t* labels = nullptr;
+    float *z = nullptr, *dz = nullptr;
+    bf16* dz_bf16 = nullptr;
+    float *hid_f32 = nullptr, *dhid_f32 = nullptr;
+    bf16 *hid_bf16 = nullptr, *dhid_bf16 = nullptr;
+    bf16 *w1_shadow = nullptr, *w2_shadow = nullptr;
+    float *w1_partials = nullptr, *w2_partials = nullptr, *b1_partials = nullptr;
+    int n_split1 = 0, n_split2 = 0, n_b1part = 0;
+    float *loss_part = nullptr, *db_part = nullptr;
+    int n_k3_blocks = 0;
+    float* loss_buf = nullptr;              // [S][kMaxSteps]
+    unsigned long long* conf_buf = nullptr; // [S][kMaxSteps][C][C], allocated on first use
+    unsigned int* bad = nullptr;            // [2]: labels >= C met by a step / by st_agreement
+    uint8_t* mask_tmp = nullptr;            // [P]
+    uint8_t* mask_tmp2 = nullptr;           // [P]
+    unsigned long long* conf_tmp = nullptr; // [C][C]
+    double* miou_tmp = nullptr;
+    float* read_tmp = nullptr; size_t read_tmp_bytes = 0;
+    void* staging = nullptr; size_t staging_bytes = 0;
+    std::vector<char> has_feat, has_labels;
+    TcPlan* plan = nullptr;
+    struct StepGraph { cudaGraphExec_t exec; int64_t n_launches; };
+    std::map<GraphKey, StepGraph> graphs;
+    bool use_graphs = true;
+    std::string err;
+    int64_t launches = 0;
+    std::vector<void*> allocs;
+};
+
+namespace {
+
+st_status fail(st_ctx* ctx, st_status code, const char* fmt, ...)
+{
+    char buf[512];
+    va_list ap;
+    va_start(ap, fmt);
+    vsnprintf(buf, sizeof buf, fmt, ap);
+    va_end(ap);
+    if (ctx) ctx->err = buf; else g_init_error = buf;
+    return code;
+}
+
+#define ST_CUDA(ctx, call)                                                                        \
+    do {                                                                                          \
+        cudaError_t e_ = (call);                                                                  \
+        if (e_ != cudaSuccess)                                                                    \
+            return fail(ctx, e_ == cudaErrorMemoryAllocation ? ST_ERR_OOM : ST_ERR_CUDA,          \
+                        "%s failed: %s", #call, cudaGetErrorString(e_));                          \
+    } while (0)
+
+template <typename T>
+cudaError_t dev_alloc(st_ctx* ctx, T** ptr, size_t count, bool zero = true)
+{
+    void* q = nullptr;
+    size_t bytes = count * sizeof(T);
+    if (bytes == 0) bytes = 16;
+    cudaError_t e = cudaMalloc(&q, bytes);
+    if (e != cudaSuccess) return e;
+    ctx->allocs.push_back(q);
+    if (zero) {
+        e = cudaMemsetAsync(q, 0, bytes, ctx->stream);
+        if (e != cudaSuccess) return e;
+    }
+    *ptr = (T*)q;
+    return cudaSuccess;
+}
+
+bool is_device_ptr(const void* q)
+{
+    cudaPointerAttributes at;
+    if (cudaPointerGetAttributes(&at, q) != cudaSuccess) { cudaGetLastError(); return false; }
+    return at.type == cudaMemoryTypeDevice || at.type == cudaMemoryTypeManaged;
+}
+
+st_status ensure_staging(st_ctx* ctx, size_t bytes)
+{
+    if (ctx->staging_bytes >= bytes) return ST_OK;
+    // the old buffer may still be read by enqueued work
+    ST_CUDA(ctx, cudaStreamSynchronize(ctx->stream));
+    if (ctx->staging) cudaFree(ctx->staging);
+    ctx->staging = nullptr; ctx->staging_bytes = 0;
+    ST_CUDA(ctx, cudaMalloc(&ctx->staging, bytes));
+    ctx->staging_bytes = bytes;
+    return ST_OK;
+}
+
+// Bring `bytes` of a host-or-device source into device memory; *dev receives a device pointer
+// (the source itself if it already is one).
+st_status to_device(st_ctx* ctx, const void* src, size_t bytes, const void** dev)
+{
+    if (is_device_ptr(src)) { *dev = src; return ST_OK; }
+    st_status st = ensure_staging(ctx, bytes);
+    if (st != ST_OK) return st;
+    ST_CUDA(ctx, cudaMemcpyAsync(ctx->staging, src, bytes, cudaMemcpyHostToDevice, ctx->stream));
+    *dev = ctx->staging;
+    return ST_OK;
+}
+
+st_status check_stream_index(st_ctx* ctx, int32_t s)
+{
+    if (!ctx) return ST_ERR_INVALID_ARG;
+    if (s < 0 || s >= ctx->S) return fail(ctx, ST_ERR_INVALID_ARG, "stream index %d outside [0, %d)", s, ctx->S);
+    return ST_OK;
+}
+
+st_status check_launch(st_ctx* ctx, const char* what)
+{
+    cudaError_t e = cudaGetLastError();
+    if (e != cudaSuccess) return fail(ctx, ST_ERR_CUDA, "%s: %s", what, cudaGetErrorString(e));
+    return ST_OK;
+}
+
+UpdateArgs make_update_args(st_ctx* c, int slot)
+{
+    UpdateArgs u;
+    memset(&u, 0, sizeof u);
+    u.theta = c->theta; u.vel = c->vel; u.grad = c->grad;
+    u.n_params = c->n_params; u.S = c->S; u.lr = c->d.lr; u.mu = c->d.momentum;
+    u.n_layers = c->layout.n_layers;
+    for (int L = 0; L < u.n_layers; ++L) {
+        LayerUpdate& ly = u.layer[L];
+        ly.w_off = c->layout.w_off[L]; ly.b_off = c->layout.b_off[L];
+        ly.cout = c->layout.cout[L]; ly.cin = c->layout.cin[L]; ly.taps = c->layout.taps[L];
+        const bool last = (L == u.n_layers - 1);
+        if (last) { ly.b_partials = c->db_part; ly.n_bpart = c->n_k3_blocks; }
+        if (c->bf16_mode) {
+            if (last) {
+                ly.w_partials = c->w2_partials; ly.n_split = c->n_split2;
+                ly.w_split_stride = (int64_t)kClassPad * ly.cin;
+                ly.w_stream_stride = ly.w_split_stride * c->n_split2;
+                ly.shadow = c->w2_shadow; ly.shadow_stream_stride = (int64_t)kClassPad * ly.cin;
+            } else {
+                ly.w_partials = c->w1_partials; ly.n_split = c->n_split1;
+                ly.w_split_stride = (int64_t)9 * ly.cout * ly.cin;
+                ly.w_stream_stride = ly.w_split_stride * c->n_split1;
+                ly.shadow = c->w1_shadow; ly.shadow_stream_stride = (int64_t)9 * ly.cout * ly.cin;
+                ly.b_partials = c->b1_partials; ly.n_bpart = c->n_b1part;
+            }
+        }
+    }
+    u.loss_part = c->loss_part; u.n_loss_part = c->n_k3_blocks;
+    u.loss_buf = c->loss_buf; u.loss_slot = slot;
+    u.inv_P = 1.0 / (double)c->P;
+    return u;
+}
+
+// Forward of the trainable part for all streams: z (and the hidden activation).
+st_status enqueue_forward(st_ctx* c)
+{
+    cudaStream_t s = c->stream;
+    if (c->bf16_mode) {
+        c->launches += tc_forward(c->plan, s);
+    } else if (c->Ch == 0) {
+        launch_conv_fwd_f32(c->x_f32, c->Cin, c->h, c->w, c->theta + c->layout.w_off[0], c->theta + c->layout.b_off[0],
+                            c->C, 1, false, c->z, c->S, (int64_t)c->Cin * c->p, c->n_params, c->n_params,
+                            (int64_t)c->C * c->p, s);
+        c->launches += 1;
+    } else {
+        launch_conv_fwd_f32(c->x_f32, c->Cin, c->h, c->w, c->theta + c->layout.w_off[0], c->theta + c->layout.b_off[0],
+                            c->Ch, 3, true, c->hid_f32, c->S, (int64_t)c->Cin * c->p, c->n_params, c->n_params,
+                            (int64_t)c->Ch * c->p, s);
+        launch_conv_fwd_f32(c->hid_f32, c->Ch, c->h, c->w, c->theta + c->layout.w_off[1], c->theta + c->layout.b_off[1],
+                            c->C, 1, false, c->z, c->S, (int64_t)c->Ch * c->p, c->n_params, c->n_params,
+                            (int64_t)c->C * c->p, s);
+        c->launches += 2;
+    }
+    return check_launch(c, "head forward");
+}
+
+st_status enqueue_step(st_ctx* c, int slot, bool want_conf)
+{
+    cudaStream_t s = c->stream;
+    st_status st = enqueue_forward(c);
+    if (st != ST_OK) return st;
+
+    UpsampleCeArgs k3;
+    k3.z = c->z; k3.labels = c->labels; k3.dz = c->dz; k3.dz_bf16 = c->bf16_mode ? c->dz_bf16 : nullptr;
+    k3.loss_part = c->loss_part; k3.db_part = c->db_part;
+    k3.conf = want_conf ? c->conf_buf + (int64_t)slot * c->C * c->C : nullptr;
+    k3.conf_stream_stride = (int64_t)kMaxSteps * c->C * c->C;
+    k3.bad = c->bad;
+    k3.S = c->S; k3.C = c->C; k3.h = c->h; k3.w = c->w;
+    launch_upsample_ce(k3, s);
+    c->launches += 1;
+    st = check_launch(c, "upsample + cross-entropy");
+    if (st != ST_OK) return st;
+
+    if (c->bf16_mode) {
+        c->launches += tc_backward(c->plan, s);
+    } else if (c->Ch == 0) {
+        launch_conv_wgrad_f32(c->x_f32, c->dz, c->Cin, c->C, c->h, c->w, 1, c->grad + c->layout.w_off[0], c->S,
+                              (int64_t)c->Cin * c->p, (int64_t)c->C * c->p, c->n_params, s);
+        c->launches += 1;
+    } else {
+        const int64_t hs = (int64_t)c->Ch * c->p;
+        launch_conv_wgrad_f32(c->hid_f32, c->dz, c->Ch, c->C, c->h, c->w, 1, c->grad + c->layout.w_off[1], c->S,
+                              hs, (int64_t)c->C * c->p, c->n_params, s);
+        launch_conv1x1_dgrad_relu_f32(c->theta + c->layout.w_off[1], c->dz, c->hid_f32, c->C, c->Ch, c->p,
+                                      c->dhid_f32, c->S, c->n_params, (int64_t)c->C * c->p, hs, s);
+        launch_conv_wgrad_f32(c->x_f32, c->dhid_f32, c->Cin, c->Ch, c->h, c->w, 3, c->grad + c->layout.w_off[0], c->S,
+                              (int64_t)c->Cin * c->p, hs, c->n_params, s);
+        launch_bias_grad_f32(c->dhid_f32, c->Ch, c->p, c->grad + c->layout.b_off[0], c->S, hs, c->n_params, s);
+        c->launches += 4;
+    }
+    st = check_launch(c, "head backward");
+    if (st != ST_OK) return st;
+
+    launch_sgd_update(make_update_args(c, slot), s);
+    c->launches += 1;
+    return check_launch(c, "sgd update");
+}
+
+st_status report_bad_labels(st_ctx* c, int which, const char* what)
+{
+    unsigned int host_bad[2] = {0, 0};
+    ST_CUDA(c, cudaMemcpyAsync(host_bad, c->bad, sizeof host_bad, cudaMemcpyDeviceToHost, c->stream));
+    ST_CUDA(c, cudaStreamSynchronize(c->stream));
+    if (host_bad[which]) {
+        unsigned int zero = 0;
+        cudaMemcpyAsync(c->bad + which, &zero, sizeof zero, cudaMemcpyHostToDevice, c->stream);
+        cudaStreamSynchronize(c->stream);
+        return fail(c, ST_ERR_INVALID_ARG, "%u pixel(s) with a label or prediction >= n_classes were skipped (%s)",
+                    host_bad[which], what);
+    }
+    return ST_OK;
+}
+
+}  // namespace
+
+extern "C" {
+
+size_t st_param_count(int32_t c_in, int32_t c_hidden, int32_t n_classes)
+{
+    if (c_in <= 0 || n_classes <= 0 || c_hidden < 0) return 0;
+    if (c_hidden == 0) return (size_t)n_classes * c_in + n_classes;
+    return (size_t)c_hidden * c_in * 9 + c_hidden + (size_t)n_classes * c_hidden + n_classes;
+}
+
+const char* st_status_name(st_status s)
+{
+    switch (s) {
+        case ST_OK: return "ST_OK";
+        case ST_ERR_INVALID_ARG: return "ST_ERR_INVALID_ARG";
+        case ST_ERR_BAD_STATE: return "ST_ERR_BAD_STATE";
+        case ST_ERR_BUFFER_TOO_SMALL: return "ST_ERR_BUFFER_TOO_SMALL";
+        case ST_ERR_UNSUPPORTED: return "ST_ERR_UNSUPPORTED";
+        case ST_ERR_OOM: return "ST_ERR_OOM";
+        case ST_ERR_CUDA: return "ST_ERR_CUDA";
+    }
+    return "ST_ERR_?";
+}
+
+const char* st_last_error(const st_ctx* ctx) { return ctx ? ctx->err.c_str() : g_init_error.c_str(); }
+
+int64_t st_launch_count(const st_ctx* ctx) { return ctx ? ctx->launches : 0; }
+
+void st_destroy(st_ctx* ctx)
+{
+    if (!ctx) return;
+    cudaStreamSynchronize(ctx->stream);
+    for (auto& g : ctx->graphs) cudaGraphExecDestroy(g.second.exec);
+    if (ctx->plan) tc_plan_destroy(ctx->plan);
+    for (void* q : ctx->allocs) cudaFree(q);
+    if (ctx->staging) cudaFree(ctx->staging);
+    if (ctx->read_tmp) cudaFree(ctx->read_tmp);
+    delete ctx;
+}
+
+st_status st_init_head(const st_head_desc* desc, const float* init_params, st_ctx** out)
+{
+    if (!desc || !init_params || !out) return fail(nullptr, ST_ERR_INVALID_ARG, "st_init_head: NULL argument");
+    *out = nullptr;
+    const st_head_desc& d = *desc;
+    if (d.n_streams < 1 || d.c_in < 1 || d.c_hidden < 0 || d.feat_h < 1 || d.feat_w < 1)
+        return fail(nullptr, ST_ERR_INVALID_ARG, "st_init_head: n_streams, c_in, feat_h, feat_w must be >= 1 and c_hidden >= 0");
+    if (d.n_classes < 2 || d.n_classes > 255)
+        return fail(nullptr, ST_ERR_INVALID_ARG, "st_init_head: n_classes %d outside 2..255", d.n_classes);
+    if (!(d.lr >= 0.f) || !(d.momentum >= 0.f) || !(d.momentum < 1.f))
+        return fail(nullptr, ST_ERR_INVALID_ARG, "st_init_head: lr must be >= 0 and momentum in [0, 1)");
+    if (d.gemm_precision != 0 && d.gemm_precision != 1)
+        return fail(nullptr, ST_ERR_INVALID_ARG, "st_init_head: gemm_precision must be 0 or 1");
+    if (d.up != kUp) return fail(nullptr, ST_ERR_UNSUPPORTED, "st_init_head: up must be 4");
+    if ((int64_t)d.feat_h * d.feat_w * 16 > (int64_t)1 << 30)
+        return fail(nullptr, ST_ERR_UNSUPPORTED, "st_init_head: frame larger than 2^30 pixels");
+    if (d.gemm_precision == 1) {
+        if (d.c_in % 64 != 0 || d.c_hidden % 64 != 0 || d.c_hidden > 256 || d.c_in > 1024 || d.n_classes > kClassPad)
+            return fail(nullptr, ST_ERR_UNSUPPORTED,
+                        "st_init_head: the bf16 tensor-core path needs c_in and c_hidden multiples of 64, "
+                        "c_hidden <= 256, c_in <= 1024 and n_classes <= %d", kClassPad);
+    }
+
+    st_ctx* c = new (std::nothrow) st_ctx();
+    if (!c) return fail(nullptr, ST_ERR_OOM, "st_init_head: host allocation failed");
+    c->d = d;
+    c->stream = (cudaStream_t)d.cuda_stream;
+    cudaGetDevice(&c->device);
+    c->S = d.n_streams; c->C = d.n_classes; c->Cin = d.c_in; c->Ch = d.c_hidden;
+    c->h = d.feat_h; c->w = d.feat_w; c->H = d.feat_h * kUp; c->W = d.feat_w * kUp;
+    c->p = (int64_t)c->h * c->w; c->P = (int64_t)c->H * c->W;
+    c->n_params = (int64_t)st_param_count(d.c_in, d.c_hidden, d.n_classes);
+    c->bf16_mode = d.gemm_precision == 1;
+    c->has_feat.assign(c->S, 0); c->has_labels.assign(c->S, 0);
+    if (const char* e = getenv("ST_NO_GRAPH")) c->use_graphs = !(e[0] == '1');
+
+    PackLayout& L = c->layout;
+    memset(&L, 0, sizeof L);
+    L.n_params = c->n_params;
+    if (c->Ch == 0) {
+        L.n_layers = 1; L.cout[0] = c->C; L.cin[0] = c->Cin; L.taps[0] = 1;
+        L.w_off[0] = 0; L.b_off[0] = (int64_t)c->C * c->Cin;
+    } else {
+        L.n_layers = 2;
+        L.cout[0] = c->Ch; L.cin[0] = c->Cin; L.taps[0] = 9; L.w_off[0] = 0; L.b_off[0] = (int64_t)c->Ch * c->Cin * 9;
+        L.cout[1] = c->C; L.cin[1] = c->Ch; L.taps[1] = 1; L.w_off[1] = L.b_off[0] + c->Ch;
+        L.b_off[1] = L.w_off[1] + (int64_t)c->C * c->Ch;
+    }
+
+    const int S = c->S;
+    const int c_last = c->Ch ? c->Ch : c->Cin;
+    c->n_k3_blocks = upsample_ce_blocks(c->h, c->w);
+    cudaError_t e = cudaSuccess;
+#define ALLOC(ptr, count) if (e == cudaSuccess) e = dev_alloc(c, &c->ptr, (size_t)(count))
+    ALLOC(theta, S * c->n_params); ALLOC(vel, S * c->n_params); ALLOC(grad, S * c->n_params);
+    ALLOC(labels, S * c->P);
+    ALLOC(z, S * c->C * c->p); ALLOC(dz, S * c->C * c->p);
+    ALLOC(loss_part, S * c->n_k3_blocks); ALLOC(db_part, (size_t)S * c->n_k3_blocks * c->C);
+    ALLOC(loss_buf, S * kMaxSteps);
+    ALLOC(bad, 2); ALLOC(mask_tmp, c->P); ALLOC(mask_tmp2, c->P); ALLOC(conf_tmp, c->C * c->C); ALLOC(miou_tmp, 1);
+    if (c->bf16_mode) {
+        ALLOC(x_bf16, S * c->p * c->Cin);
+        ALLOC(dz_bf16, (size_t)S * kClassPad * c->p);
+        ALLOC(w2_shadow, (size_t)S * kClassPad * c_last);
+        c->n_split2 = tc_wgrad_splits(2, c->Cin, c->Ch, c->h, c->w);
+        ALLOC(w2_partials, (size_t)S * c->n_split2 * kClassPad * c_last);
+        if (c->Ch) {
+            ALLOC(hid_bf16, S * c->p * c->Ch); ALLOC(dhid_bf16, S * c->p * c->Ch);
+            ALLOC(w1_shadow, (size_t)S * 9 * c->Ch * c->Cin);
+            c->n_split1 = tc_wgrad_splits(1, c->Cin, c->Ch, c->h, c->w);
+            ALLOC(w1_partials, (size_t)S * c->n_split1 * 9 * c->Ch * c->Cin);
+            c->n_b1part = tc_b1_partials(c->h, c->w);
+            ALLOC(b1_partials, (size_t)S * c->n_b1part * c->Ch);
+        }
+    } else {
+        ALLOC(x_f32, S * c->Cin * c->p);
+        if (c->Ch) { ALLOC(hid_f32, S * c->Ch * c->p); ALLOC(dhid_f32, S * c->Ch * c->p); }
+    }
+#undef ALLOC
+    if (e == cudaSuccess) e = prepare_upsample_ce(c->C);
+    if (e != cudaSuccess) {
+        st_status code = fail(nullptr, e == cudaErrorMemoryAllocation ? ST_ERR_OOM : ST_ERR_CUDA,
+                              "st_init_head: device allocation failed: %s", cudaGetErrorString(e));
+        cudaGetLastError();
+        st_destroy(c);
+        return code;
+    }
+
+    // parameters: packed order -> internal order (the momentum buffer serves as scratch, then is zeroed)
+    const size_t pbytes = (size_t)S * c->n_params * sizeof(float);
+    e = cudaMemcpyAsync(c->vel, init_params, pbytes, cudaMemcpyDefault, c->stream);
+    if (e == cudaSuccess) { launch_unpack(c->vel, c->theta, c->layout, S, c->stream); e = cudaGetLastError(); }
+    if (e == cudaSuccess) e = cudaMemsetAsync(c->vel, 0, pbytes, c->stream);
+    if (e == cudaSuccess && c->bf16_mode) {
+        TcBuffers b;
+        memset(&b, 0, sizeof b);
+        b.S = S; b.c_in = c->Cin; b.c_hidden = c->Ch; b.C = c->C; b.h = c->h; b.w = c->w;
+        b.x = c->x_bf16; b.w1 = c->w1_shadow; b.w2 = c->w2_shadow; b.theta = c->theta; b.n_params = c->n_params;
+        b.b1_off = c->Ch ? L.b_off[0] : 0; b.b2_off = L.b_off[L.n_layers - 1];
+        b.z = c->z; b.hidden = c->hid_bf16; b.dz = c->dz; b.dz_bf16 = c->dz_bf16; b.dhidden = c->dhid_bf16;
+        b.w1_partials = c->w1_partials; b.w2_partials = c->w2_partials; b.b1_partials = c->b1_partials;
+        char msg[256] = {0};
+        c->plan = tc_plan_create(b, msg, sizeof msg);
+        if (!c->plan) {
+            st_status code = fail(nullptr, ST_ERR_CUDA, "st_init_head: tensor-core plan: %s", msg);
+            st_destroy(c);
+            return code;
+        }
+        launch_refresh_shadow(make_update_args(c, -1), c->stream);
+        e = cudaGetLastError();
+    }
+    if (e == cudaSuccess) e = cudaStreamSynchronize(c->stream);   // init_params may be released on return
+    if (e != cudaSuccess) {
+        st_status code = fail(nullptr, ST_ERR_CUDA, "st_init_head: %s", cudaGetErrorString(e));
+        st_destroy(c);
+        return code;
+    }
+    c->launches += 2;
+    *out = c;
+    return ST_OK;
+}
+
+st_status st_set_frozen_features(st_ctx* ctx, int32_t stream, const float* feat_chw)
+{
+    st_status st = check_stream_index(ctx, stream);
+    if (st != ST_OK) return st;
+    if (!feat_chw) return fail(ctx, ST_ERR_INVALID_ARG, "st_set_frozen_features: NULL features");
+    const size_t bytes = (size_t)ctx->Cin * ctx->p * sizeof(float);
+    if (ctx->bf16_mode) {
+        const void* src = nullptr;
+        st = to_device(ctx, feat_chw, bytes, &src);
+        if (st != ST_OK) return st;
+        launch_feat_to_bf16_nhwc((const float*)src, ctx->Cin, ctx->p, ctx->x_bf16 + (int64_t)stream * ctx->p * ctx->Cin, ctx->stream);
+        ctx->launches += 1;
+        st = check_launch(ctx, "feature cache");
+        if (st != ST_OK) return st;
+    } else {
+        ST_CUDA(ctx, cudaMemcpyAsync(ctx->x_f32 + (int64_t)stream * ctx->Cin * ctx->p, feat_chw, bytes, cudaMemcpyDefault, ctx->stream));
+    }
+    ctx->has_feat[stream] = 1;
+    return ST_OK;
+}
+
+st_status st_teacher_labels(st_ctx* ctx, int32_t stream, const float* logits_chw, uint8_t* labels_out)
+{
+    st_status st = check_stream_index(ctx, stream);
+    if (st != ST_OK) return st;
+    if (!logits_chw) return fail(ctx, ST_ERR_INVALID_ARG, "st_teacher_labels: NULL logits");
+    const void* src = nullptr;
+    st = to_device(ctx, logits_chw, (size_t)ctx->C * ctx->P * sizeof(float), &src);
+    if (st != ST_OK) return st;
+    uint8_t* dst = ctx->labels + (int64_t)stream * ctx->P;
+    launch_argmax_u8((const float*)src, ctx->C, ctx->P, dst, ctx->stream);
+    ctx->launches += 1;
+    st = check_launch(ctx, "teacher argmax");
+    if (st != ST_OK) return st;
+    if (labels_out) ST_CUDA(ctx, cudaMemcpyAsync(labels_out, dst, (size_t)ctx->P, cudaMemcpyDefault, ctx->stream));
+    ctx->has_labels[stream] = 1;
+    return ST_OK;
+}
+
+st_status st_set_labels(st_ctx* ctx, int32_t stream, const uint8_t* labels)
+{
+    st_status st = check_stream_index(ctx, stream);
+    if (st != ST_OK) return st;
+    if (!labels) return fail(ctx, ST_ERR_INVALID_ARG, "st_set_labels: NULL labels");
+    ST_CUDA(ctx, cudaMemcpyAsync(ctx->labels + (int64_t)stream * ctx->P, labels, (size_t)ctx->P, cudaMemcpyDefault, ctx->stream));
+    ctx->has_labels[stream] = 1;
+    return ST_OK;
+}
+
+st_status st_distill_step(st_ctx* ctx, int32_t n_steps, float* loss_out, int64_t* conf_out)
+{
+    if (!ctx) return ST_ERR_INVALID_ARG;
+    if (n_steps < 1 || n_steps > kMaxSteps)
+        return fail(ctx, ST_ERR_INVALID_ARG, "st_distill_step: n_steps %d outside 1..%d", n_steps, kMaxSteps);
+    for (int s = 0; s < ctx->S; ++s)
+        if (!ctx->has_feat[s] || !ctx->has_labels[s])
+            return fail(ctx, ST_ERR_BAD_STATE, "st_distill_step: stream %d has no %s yet", s,
+                        ctx->has_feat[s] ? "labels" : "frozen features");
+    const bool want_conf = conf_out != nullptr;
+    const size_t cc = (size_t)ctx->C * ctx->C;
+    if (want_conf) {
+        if (!ctx->conf_buf) {
+            cudaError_t e = dev_alloc(ctx, &ctx->conf_buf, (size_t)ctx->S * kMaxSteps * cc);
+            if (e != cudaSuccess) return fail(ctx, ST_ERR_OOM, "st_distill_step: %s", cudaGetErrorString(e));
+        }
+        ST_CUDA(ctx, cudaMemsetAsync(ctx->conf_buf, 0, (size_t)ctx->S * kMaxSteps * cc * sizeof(unsigned long long), ctx->stream));
+    }
+
+    st_status st = ST_OK;
+    if (ctx->use_graphs) {
+        GraphKey key{n_steps, want_conf};
+        auto it = ctx->graphs.find(key);
+        if (it == ctx->graphs.end()) {
+            cudaGraph_t graph = nullptr;
+            const int64_t before = ctx->launches;
+            ST_CUDA(ctx, cudaStreamBeginCapture(ctx->stream, cudaStreamCaptureModeThreadLocal));
+            for (int k = 0; k < n_steps && st == ST_OK; ++k) st = enqueue_step(ctx, k, want_conf);
+            cudaError_t e = cudaStreamEndCapture(ctx->stream, &graph);
+            const int64_t n_launches = ctx->launches - before;
+            ctx->launches = before;
+            if (st != ST_OK) { if (graph) cudaGraphDestroy(graph); return st; }
+            if (e != cudaSuccess) return fail(ctx, ST_ERR_CUDA, "st_distill_step: graph capture: %s", cudaGetErrorString(e));
+            cudaGraphExec_t exec = nullptr;
+            e = cudaGraphInstantiate(&exec, graph, 0);
+            cudaGraphDestroy(graph);
+            if (e != cudaSuccess) return fail(ctx, ST_ERR_CUDA, "st_distill_step: graph instantiate: %s", cudaGetErrorString(e));
+            it = ctx->graphs.emplace(key, st_ctx::StepGraph{exec, n_launches}).first;
+        }
+        ctx->launches += it->second.n_launches;   // a replay launches the captured kernels again
+        ST_CUDA(ctx, cudaGraphLaunch(it->second.exec, ctx->stream));
+    } else {
+        for (int k = 0; k < n_steps; ++k) {
+            st = enqueue_step(ctx, k, want_conf);
+            if (st != ST_OK) return st;
+        }
+    }
+    if (loss_out)
+        ST_CUDA(ctx, cudaMemcpy2DAsync(loss_out, (size_t)n_steps * sizeof(float), ctx->loss_buf, kMaxSteps * sizeof(float),
+                                       (size_t)n_steps * sizeof(float), ctx->S, cudaMemcpyDefault, ctx->stream));
+    if (conf_out)
+        ST_CUDA(ctx, cudaMemcpy2DAsync(conf_out, (size_t)n_steps * cc * 8, ctx->conf_buf, (size_t)kMaxSteps * cc * 8,
+                                       (size_t)n_steps * cc * 8, ctx->S, cudaMemcpyDefault, ctx->stream));
+    return ST_OK;
+}
+
+st_status st_pack_updated_params(st_ctx* ctx, int32_t stream, void* dst, size_t dst_capacity, size_t* nbytes)
+{
+    st_status st = check_stream_index(ctx, stream);
+    if (st != ST_OK) return st;
+    const size_t need = (size_t)ctx->n_params * sizeof(float);
+    if (nbytes) *nbytes = need;
+    if (!dst) return fail(ctx, ST_ERR_INVALID_ARG, "st_pack_updated_params: NULL destination");
+    if (dst_capacity < need)
+        return fail(ctx, ST_ERR_BUFFER_TOO_SMALL, "st_pack_updated_params: capacity %zu < %zu bytes", dst_capacity, need);
+    const float* src = ctx->theta + (int64_t)stream * ctx->n_params;
+    if (is_device_ptr(dst)) {
+        launch_pack(src, (float*)dst, ctx->layout, 1, ctx->stream);
+        ctx->launches += 1;
+        return check_launch(ctx, "pack");
+    }
+    // host destination: pack into the staging buffer, then copy out
+    st = ensure_staging(ctx, need);
+    if (st != ST_OK) return st;
+    launch_pack(src, (float*)ctx->staging, ctx->layout, 1, ctx->stream);
+    ctx->launches += 1;
+    st = check_launch(ctx, "pack");
+    if (st != ST_OK) return st;
+    ST_CUDA(ctx, cudaMemcpyAsync(dst, ctx->staging, need, cudaMemcpyDeviceToHost, ctx->stream));
+    ST_CUDA(ctx, cudaStreamSynchronize(ctx->stream));
+    return ST_OK;
+}
+
+st_status st_student_mask(st_ctx* ctx, int32_t stream, uint8_t* mask_out)
+{
+    st_status st = check_stream_index(ctx, stream);
+    if (st != ST_OK) return st;
+    if (!mask_out) return fail(ctx, ST_ERR_INVALID_ARG, "st_student_mask: NULL destination");
+    if (!ctx->has_feat[stream]) return fail(ctx, ST_ERR_BAD_STATE, "st_student_mask: stream %d has no frozen features yet", stream);
+    for (int s = 0; s < ctx->S; ++s)
+        if (!ctx->has_feat[s]) return fail(ctx, ST_ERR_BAD_STATE, "st_student_mask: the forward runs on all streams; stream %d has no features", s);
+    st = enqueue_forward(ctx);
+    if (st != ST_OK) return st;
+    const bool dev = is_device_ptr(mask_out);
+    uint8_t* dst = dev ? mask_out : ctx->mask_tmp;
+    launch_upsample_argmax(ctx->z + (int64_t)stream * ctx->C * ctx->p, ctx->C, ctx->h, ctx->w, dst, ctx->stream);
+    ctx->launches += 1;
+    st = check_launch(ctx, "student mask");
+    if (st != ST_OK) return st;
+    if (!dev) {
+        ST_CUDA(ctx, cudaMemcpyAsync(mask_out, dst, (size_t)ctx->P, cudaMemcpyDeviceToHost, ctx->stream));
+        ST_CUDA(ctx, cudaStreamSynchronize(ctx->stream));
+    }
+    return ST_OK;
+}
+
+st_status st_agreement(st_ctx* ctx, int32_t stream, const uint8_t* pred, const uint8_t* label, int64_t* conf, double* miou)
+{
+    st_status st = check_stream_index(ctx, stream);
+    if (st != ST_OK) return st;
+    const uint8_t* d_label = nullptr;
+    const uint8_t* d_pred = nullptr;
+    if (label) {
+        if (is_device_ptr(label)) d_label = label;
+        else {
+            ST_CUDA(ctx, cudaMemcpyAsync(ctx->mask_tmp2, label, (size_t)ctx->P, cudaMemcpyHostToDevice, ctx->stream));
+            d_label = ctx->mask_tmp2;
+        }
+    } else {
+        if (!ctx->has_labels[stream]) return fail(ctx, ST_ERR_BAD_STATE, "st_agreement: stream %d has no labels yet", stream);
+        d_label = ctx->labels + (int64_t)stream * ctx->P;
+    }
+    if (pred) {
+        if (is_device_ptr(pred)) d_pred = pred;
+        else {
+            ST_CUDA(ctx, cudaMemcpyAsync(ctx->mask_tmp, pred, (size_t)ctx->P, cudaMemcpyHostToDevice, ctx->stream));
+            d_pred = ctx->mask_tmp;
+        }
+    } else {
+        st = st_student_mask(ctx, stream, ctx->mask_tmp);
+        if (st != ST_OK) return st;
+        d_pred = ctx->mask_tmp;
+    }
+    const size_t cbytes = (size_t)ctx->C * ctx->C * sizeof(unsigned long long);
+    ST_CUDA(ctx, cudaMemsetAsync(ctx->conf_tmp, 0, cbytes, ctx->stream));
+    launch_confusion(d_label, d_pred, ctx->P, ctx->C, ctx->conf_tmp, ctx->bad + 1, ctx->stream);
+    launch_miou(ctx->conf_tmp, ctx->C, ctx->miou_tmp, ctx->stream);
+    ctx->launches += 2;
+    st = check_launch(ctx, "confusion");
+    if (st != ST_OK) return st;
+    if (conf) ST_CUDA(ctx, cudaMemcpyAsync(conf, ctx->conf_tmp, cbytes, cudaMemcpyDefault, ctx->stream));
+    double m = 0.0;
+    ST_CUDA(ctx, cudaMemcpyAsync(&m, ctx->miou_tmp, sizeof m, cudaMemcpyDeviceToHost, ctx->stream));
+    ST_CUDA(ctx, cudaStreamSynchronize(ctx->stream));
+    if (miou) *miou = m;
+    st = report_bad_labels(ctx, 1, "st_agreement");
+    if (st != ST_OK) return st;
+    return report_bad_labels(ctx, 0, "an earlier st_distill_step");
+}
+
+st_status st_read_tensor(st_ctx* ctx, int32_t stream, st_tensor which, float* dst_host, size_t dst_capacity, size_t* nbytes)
+{
+    st_status st = check_stream_index(ctx, stream);
+    if (st != ST_OK) return st;
+    size_t count = 0;
+    switch (which) {
+        case ST_TENSOR_LOGITS: case ST_TENSOR_LOGIT_GRAD: count = (size_t)ctx->C * ctx->p; break;
+        case ST_TENSOR_PARAM_GRAD: case ST_TENSOR_MOMENTUM: count = (size_t)ctx->n_params; break;
+        case ST_TENSOR_HIDDEN: case ST_TENSOR_HIDDEN_GRAD:
+            if (!ctx->Ch) return fail(ctx, ST_ERR_INVALID_ARG, "st_read_tensor: the head has no hidden layer");
+            count = (size_t)ctx->Ch * ctx->p; break;
+        case ST_TENSOR_FEATURES: count = (size_t)ctx->Cin * ctx->p; break;
+        default: return fail(ctx, ST_ERR_INVALID_ARG, "st_read_tensor: unknown tensor %d", (int)which);
+    }
+    const size_t need = count * sizeof(float);
+    if (nbytes) *nbytes = need;
+    if (!dst_host) return fail(ctx, ST_ERR_INVALID_ARG, "st_read_tensor: NULL destination");
+    if (dst_capacity < need) return fail(ctx, ST_ERR_BUFFER_TOO_SMALL, "st_read_tensor: capacity %zu < %zu bytes", dst_capacity, need);
+    if (ctx->read_tmp_bytes < need) {
+        ST_CUDA(ctx, cudaStreamSynchronize(ctx->stream));
+        if (ctx->read_tmp) cudaFree(ctx->read_tmp);
+        ctx->read_tmp = nullptr; ctx->read_tmp_bytes = 0;
+        ST_CUDA(ctx, cudaMalloc((void**)&ctx->read_tmp, need));
+        ctx->read_tmp_bytes = need;
+    }
+    const float* src = nullptr;
+    const int64_t s = stream;
+    switch (which) {
+        case ST_TENSOR_LOGITS: src = ctx->z + s * ctx->C * ctx->p; break;
+        case ST_TENSOR_LOGIT_GRAD: src = ctx->dz + s * ctx->C * ctx->p; break;
+        case ST_TENSOR_PARAM_GRAD: launch_pack(ctx->grad + s * ctx->n_params, ctx->read_tmp, ctx->layout, 1, ctx->stream); src = ctx->read_tmp; break;
+        case ST_TENSOR_MOMENTUM: launch_pack(ctx->vel + s * ctx->n_params, ctx->read_tmp, ctx->layout, 1, ctx->stream); src = ctx->read_tmp; break;
+        case ST_TENSOR_HIDDEN:
+            if (ctx->bf16_mode) { launch_nhwc_bf16_to_chw(ctx->hid_bf16 + s * ctx->p * ctx->Ch, ctx->Ch, ctx->p, ctx->read_tmp, ctx->stream); src = ctx->read_tmp; }
+            else src = ctx->hid_f32 + s * ctx->Ch * ctx->p;
+            break;
+        case ST_TENSOR_HIDDEN_GRAD:
+            if (ctx->bf16_mode) { launch_nhwc_bf16_to_chw(ctx->dhid_bf16 + s * ctx->p * ctx->Ch, ctx->Ch, ctx->p, ctx->read_tmp, ctx->stream); src = ctx->read_tmp; }
+            else src = ctx->dhid_f32 + s * ctx->Ch * ctx->p;
+            break;
+        case ST_TENSOR_FEATURES:
+            if (ctx->bf16_mode) { launch_nhwc_bf16_to_chw(ctx->x_bf16 + s * ctx->p * ctx->Cin, ctx->Cin, ctx->p, ctx->read_tmp, ctx->stream); src = ctx->read_tmp; }
+            else src = ctx->x_f32 + s * ctx->Cin * ctx->p;
+            break;
+    }
+    st = check_launch(ctx, "read tensor");
+    if (st != ST_OK) return st;
+    ST_CUDA(ctx, cudaMemcpyAsync(dst_host, src, need, cudaMemcpyDeviceToHost, ctx->stream));
+    ST_CUDA(ctx, cudaStreamSynchronize(ctx->stream));
+    return report_bad_labels(ctx, 0, "an earlier st_distill_step");
+}
+
+}  // extern "C"

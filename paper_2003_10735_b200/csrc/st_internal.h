@@ -1,0 +1,129 @@
+// Internal declarations shared by the kernels' translation units and the C-ABI layer.
+// Nothing here is part of the public interface (see include/shadowtutor.h).
+#pragma once
+
+#include <cuda_bf16.h>
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+namespace st {
+
+typedef __nv_bfloat16 bf16;
+
+constexpr int kUp = 4;            // bilinear upsample factor of the head (frame = feature map * 4)
+constexpr int kMaxSteps = 64;     // upper bound of n_steps in one st_distill_step call
+constexpr int kClassPad = 32;     // class rows of bf16 GEMM operands are padded to this (UMMA N)
+
+// ---- K1: teacher logits -> uint8 labels -------------------------------------------------------
+void launch_argmax_u8(const float* logits, int C, int64_t P, uint8_t* labels, cudaStream_t s);
+
+// ---- K6: confusion matrix of two uint8 masks ---------------------------------------------------
+// conf: int64 [C][C], accumulated into (caller zeroes it); bad: count of pixels with l or q >= C.
+void launch_confusion(const uint8_t* label, const uint8_t* pred, int64_t P, int C,
+                      unsigned long long* conf, unsigned int* bad, cudaStream_t s);
+
+// ---- K8: frozen features fp32 [Cin][p] -> bf16 [p][Cin] ---------------------------------------
+void launch_feat_to_bf16_nhwc(const float* feat_chw, int Cin, int64_t p, bf16* out, cudaStream_t s);
+// reverse (verification only): bf16 [p][C] -> fp32 [C][p]
+void launch_nhwc_bf16_to_chw(const bf16* in, int C, int64_t p, float* out, cudaStream_t s);
+
+// ---- K3: upsample x4 + softmax cross-entropy + gradient w.r.t. the low-res logits ---------------
+struct UpsampleCeArgs {
+    const float* z;          // [S][C][h][w]
+    const uint8_t* labels;   // [S][H][W]
+    float* dz;               // [S][C][h][w]     gradient of the mean loss
+    bf16* dz_bf16;           // [S][kClassPad][p] or nullptr (rows >= C untouched)
+    float* loss_part;        // [S][n_blocks]    per-block partial sums of per-pixel losses
+    float* db_part;          // [S][n_blocks][C] per-block partial sums of dz over the block's pixels
+    unsigned long long* conf;// nullptr, or int64 [C][C] per stream: confusion of label vs argmax of the upsampled logits
+    int64_t conf_stream_stride; // elements between the matrices of consecutive streams
+    unsigned int* bad;       // count of labels >= C
+    int S, C, h, w;
+};
+int upsample_ce_blocks(int h, int w);   // blocks per stream
+cudaError_t prepare_upsample_ce(int C);   // once per device and class count, outside any stream capture
+void launch_upsample_ce(const UpsampleCeArgs& a, cudaStream_t s);
+// student mask: argmax_c of the upsampled logits, uint8 [H][W]
+void launch_upsample_argmax(const float* z, int C, int h, int w, uint8_t* mask, cudaStream_t s);
+
+// ---- fp32 CUDA-core convolutions (gemm_precision 0), planar [C][h][w] -------------------------
+void launch_conv_fwd_f32(const float* in, int Cin, int h, int w, const float* Wt, const float* b,
+                         int Cout, int ks, bool relu, float* out, int S, int64_t in_stride,
+                         int64_t w_stride, int64_t b_stride, int64_t out_stride, cudaStream_t s);
+void launch_conv_wgrad_f32(const float* in, const float* dout, int Cin, int Cout, int h, int w, int ks,
+                           float* dW, int S, int64_t in_stride, int64_t dout_stride,
+                           int64_t dw_stride, cudaStream_t s);
+void launch_conv1x1_dgrad_relu_f32(const float* W2, const float* dz, const float* Hact, int C, int Ch,
+                                   int64_t p, float* dH, int S, int64_t w_stride, int64_t dz_stride,
+                                   int64_t h_stride, cudaStream_t s);
+// db[c] = sum_p d[c][p] (one block per channel, fixed-order reduction)
+void launch_bias_grad_f32(const float* d, int C, int64_t p, float* db, int S, int64_t d_stride,
+                          int64_t db_stride, cudaStream_t s);
+
+// ---- K5: SGD(+momentum) update, loss finalisation, bf16 shadow refresh -------------------------
+struct LayerUpdate {
+    int64_t w_off, b_off;      // offsets (floats) of weight / bias in one stream's parameter buffer
+    int cout, cin, taps;       // weight in internal order [tap][cout][cin]
+    const float* w_partials;   // nullptr: grad buffer already holds dW; else split-K partial sums whose
+    int n_split;               //   element index equals the internal weight index
+    int64_t w_split_stride;    // floats between splits
+    int64_t w_stream_stride;   // floats between streams
+    const float* b_partials;   // nullptr: grad buffer already holds db; else [S][n_bpart][cout]
+    int n_bpart;
+    bf16* shadow;              // nullptr or the bf16 copy of the weight read by the GEMMs (same linear index)
+    int64_t shadow_stream_stride;
+};
+struct UpdateArgs {
+    float* theta;      // [S][n_params]   internal order
+    float* vel;        // [S][n_params]
+    float* grad;       // [S][n_params]   holds the applied gradient after the call
+    int64_t n_params;
+    int S;
+    float lr, mu;
+    LayerUpdate layer[2];
+    int n_layers;
+    const float* loss_part;  // [S][n_loss_part] per-block sums of per-pixel losses
+    int n_loss_part;
+    float* loss_buf;         // [S][kMaxSteps]
+    int loss_slot;           // slot of loss_buf written by this step
+    double inv_P;
+};
+void launch_sgd_update(const UpdateArgs& a, cudaStream_t s);
+// refresh the bf16 shadows from the fp32 master parameters (after init)
+void launch_refresh_shadow(const UpdateArgs& a, cudaStream_t s);
+// mean IoU (Section 3.2) from an int64 confusion matrix, in double, one block
+void launch_miou(const unsigned long long* conf, int C, double* out, cudaStream_t s);
+
+// ---- K7: packed parameter buffer <-> internal order ---------------------------------------------
+// packed: per layer weight [cout][cin][kh][kw] then bias; internal: weight [tap][cout][cin] then bias.
+struct PackLayout { int n_layers; int64_t w_off[2], b_off[2]; int cout[2], cin[2], taps[2]; int64_t n_params; };
+void launch_pack(const float* internal, float* packed, const PackLayout& L, int n_bufs, cudaStream_t s);
+void launch_unpack(const float* packed, float* internal, const PackLayout& L, int n_bufs, cudaStream_t s);
+
+// ---- bf16 tensor-core GEMMs (gemm_precision 1) -------------------------------------------------
+struct TcPlan;   // tensor maps and launch geometry; built once per context
+struct TcBuffers {
+    int S, c_in, c_hidden, C, h, w;
+    const bf16* x;        // [S][p][c_in]     cached features, pixel-major
+    const bf16* w1;       // [S][9][c_hidden][c_in]  (two-layer head) bf16 copy of the 3x3 weight
+    const bf16* w2;       // [S][kClassPad][c_last]  bf16 copy of the 1x1 weight, rows >= C zero
+    const float* theta;   // [S][n_params]    biases are read from the master parameters
+    int64_t n_params, b1_off, b2_off;
+    float* z;             // [S][C][p]
+    bf16* hidden;         // [S][p][c_hidden]
+    const float* dz;      // [S][C][p]
+    const bf16* dz_bf16;  // [S][kClassPad][p]
+    bf16* dhidden;        // [S][p][c_hidden]
+    float* w1_partials;   // [S][n_split1][9][c_hidden][c_in]
+    float* w2_partials;   // [S][n_split2][kClassPad][c_last]
+    float* b1_partials;   // [S][n_b1part][c_hidden]
+};
+// Geometry is fixed by the shapes alone, so scratch can be sized before the plan exists.
+int tc_wgrad_splits(int layer /*1: 3x3, 2: 1x1*/, int c_in, int c_hidden, int h, int w);
+int tc_b1_partials(int h, int w);
+TcPlan* tc_plan_create(const TcBuffers& b, char* err, size_t err_len);
+void tc_plan_destroy(TcPlan*);
+int tc_forward(const TcPlan*, cudaStream_t s);    // returns the number of kernels launched
+int tc_backward(const TcPlan*, cudaStream_t s);
+
+}  // namespace st

@@ -1,0 +1,297 @@
+"""GPU parity: the CUDA path (through the C ABI) against the CPU oracle, element by element,
+on the same seeded inputs.  Integer/byte results must be bit-exact; floating point within the
+tolerances written next to each assertion."""
+import numpy as np
+import pytest
+
+import oracle
+import synth_inputs as si
+import paper_2003_10735_b200 as st
+
+pytestmark = pytest.mark.gpu
+torch = pytest.importorskip("torch")
+
+
+def dev(a):
+    return torch.from_numpy(np.ascontiguousarray(a)).cuda()
+
+
+def make_ctx(c_in, c_hidden, C, h, w, theta, S=1, prec=0, lr=0.01, mu=0.0):
+    return st.st_init_head(n_streams=S, c_in=c_in, c_hidden=c_hidden, n_classes=C, feat_h=h, feat_w=w,
+                           gemm_precision=prec, lr=lr, momentum=mu,
+                           cuda_stream=torch.cuda.current_stream().cuda_stream, init_params=theta)
+
+
+def packed(ctx, stream=0):
+    out = np.empty(ctx.n_params, np.float32)
+    assert st.st_pack_updated_params(ctx, stream, out) == out.nbytes
+    return out
+
+
+def rand_problem(seed, c_in, C, h, w, blobs=True):
+    rng = np.random.default_rng(seed)
+    feat = np.maximum(rng.standard_normal((c_in, h, w)), 0).astype(np.float32)
+    if blobs:
+        cfg = si.WorkloadConfig("t", c_in, 0, C, h, w, n_regions=max(4, C), teacher="onehot_noise")
+        T = si.teacher_logits(cfg, stream=seed)
+    else:
+        T = rng.standard_normal((C, 4 * h, 4 * w)).astype(np.float32)
+    return feat, T
+
+
+# ---------------------------------------------------------------------------- K1 labels
+@pytest.mark.parametrize("C,h,w", [(4, 90, 160), (21, 13, 17), (2, 1, 1), (255, 3, 5)])
+def test_teacher_labels_bit_exact(C, h, w):
+    rng = np.random.default_rng(C)
+    T = rng.integers(-3, 4, size=(C, 4 * h, 4 * w)).astype(np.float32)       # plenty of exact ties
+    T += (rng.random(T.shape) < 0.5) * rng.standard_normal(T.shape).astype(np.float32)
+    ctx = make_ctx(8, 0, C, h, w, np.zeros(st.st_param_count(8, 0, C), np.float32))
+    out = torch.empty((4 * h, 4 * w), dtype=torch.uint8, device="cuda")
+    st.st_teacher_labels(ctx, 0, dev(T), out)
+    ref = oracle.teacher_labels(T)
+    np.testing.assert_array_equal(out.cpu().numpy(), ref)
+    # host input and host output go through the same kernel
+    out_h = np.empty((4 * h, 4 * w), np.uint8)
+    st.st_teacher_labels(ctx, 0, T, out_h)
+    torch.cuda.synchronize()
+    np.testing.assert_array_equal(out_h, ref)
+    st.st_destroy(ctx)
+
+
+def test_teacher_labels_blurred_boundaries_full_1080p():
+    cfg = si.get_config(4)
+    T = si.teacher_logits(cfg)
+    ctx = make_ctx(8, 0, cfg.n_classes, cfg.feat_h, cfg.feat_w, np.zeros(st.st_param_count(8, 0, cfg.n_classes), np.float32))
+    out = torch.empty((cfg.frame_h, cfg.frame_w), dtype=torch.uint8, device="cuda")
+    st.st_teacher_labels(ctx, 0, dev(T), out)
+    np.testing.assert_array_equal(out.cpu().numpy(), oracle.teacher_labels(T))
+    st.st_destroy(ctx)
+
+
+# ---------------------------------------------------------------------------- K6 agreement
+@pytest.mark.parametrize("C,h,w", [(4, 90, 160), (21, 45, 80), (3, 1, 1), (200, 5, 7)])
+def test_confusion_and_miou_bit_exact(C, h, w):
+    rng = np.random.default_rng(C + 1)
+    P = 16 * h * w
+    lab = np.repeat(rng.integers(0, C, P // 8 + 1), 8)[:P].astype(np.uint8).reshape(4 * h, 4 * w)   # coherent runs
+    pred = np.where(rng.random((4 * h, 4 * w)) < 0.7, lab, rng.integers(0, C, (4 * h, 4 * w))).astype(np.uint8)
+    ctx = make_ctx(8, 0, C, h, w, np.zeros(st.st_param_count(8, 0, C), np.float32))
+    conf = torch.zeros((C, C), dtype=torch.int64, device="cuda")
+    m = st.st_agreement(ctx, 0, dev(pred), dev(lab), conf)
+    ref_conf, ref_m, _ = oracle.agreement(lab, pred, C)
+    np.testing.assert_array_equal(conf.cpu().numpy(), ref_conf)
+    assert m == ref_m                                              # same integer counts, same double arithmetic order
+    conf_h = np.zeros((C, C), np.int64)
+    m2 = st.st_agreement(ctx, 0, pred, lab, conf_h)                # host masks
+    np.testing.assert_array_equal(conf_h, ref_conf)
+    assert m2 == ref_m
+    st.st_destroy(ctx)
+
+
+def test_agreement_reports_out_of_range_labels():
+    C, h, w = 3, 2, 2
+    lab = np.zeros((8, 8), np.uint8)
+    pred = np.zeros((8, 8), np.uint8)
+    lab[3, 3] = 9
+    ctx = make_ctx(8, 0, C, h, w, np.zeros(st.st_param_count(8, 0, C), np.float32))
+    conf = np.zeros((C, C), np.int64)
+    with pytest.raises(st.StError) as ei:
+        st.st_agreement(ctx, 0, pred, lab, conf)
+    assert ei.value.status == st.ST_ERR_INVALID_ARG
+    assert conf[0, 0] == 63                                        # the valid pixels are still counted
+    assert st.st_agreement(ctx, 0, pred, pred, conf) == 1.0        # the error does not stick
+    st.st_destroy(ctx)
+
+
+# ---------------------------------------------------------------------------- call order, pack
+def test_call_order_and_pack_errors():
+    C, cin, h, w = 3, 8, 4, 4
+    theta = si.initial_head_params(cin, 0, C, 1)
+    ctx = make_ctx(cin, 0, C, h, w, theta)
+    with pytest.raises(st.StError) as ei:
+        st.st_distill_step(ctx, 1)
+    assert ei.value.status == st.ST_ERR_BAD_STATE
+    with pytest.raises(st.StError) as ei:
+        st.st_set_frozen_features(ctx, 1, np.zeros((cin, h, w), np.float32))
+    assert ei.value.status == st.ST_ERR_INVALID_ARG
+    small = np.zeros(3, np.float32)
+    with pytest.raises(st.StError) as ei:
+        st.st_pack_updated_params(ctx, 0, small)
+    assert ei.value.status == st.ST_ERR_BUFFER_TOO_SMALL
+    with pytest.raises(st.StError) as ei:
+        st.st_distill_step(ctx, 0)
+    assert ei.value.status == st.ST_ERR_INVALID_ARG
+    # K = 0 steps taken: pack returns the initial values bit for bit (host and device destination)
+    np.testing.assert_array_equal(packed(ctx), theta)
+    d = torch.empty(ctx.n_params, dtype=torch.float32, device="cuda")
+    st.st_pack_updated_params(ctx, 0, d)
+    np.testing.assert_array_equal(d.cpu().numpy(), theta)
+    st.st_destroy(ctx)
+
+
+@pytest.mark.parametrize("prec", [0, 1])
+def test_pack_roundtrip_two_layer(prec):
+    cin, ch, C, h, w = 64, 64, 5, 4, 4
+    n = st.st_param_count(cin, ch, C)
+    theta = np.arange(n, dtype=np.float32)
+    ctx = make_ctx(cin, ch, C, h, w, theta, prec=prec)
+    raw = packed(ctx)
+    assert raw.tobytes() == np.arange(n, dtype="<f4").tobytes()
+    ctx2 = make_ctx(cin, ch, C, h, w, raw, prec=prec)
+    np.testing.assert_array_equal(packed(ctx2), raw)
+    st.st_destroy(ctx); st.st_destroy(ctx2)
+
+
+# ---------------------------------------------------------------------------- fp32 steps
+def run_both(cfg_like, feat, T, theta, n_steps, prec, want_conf=False, quantize=False):
+    c_in, ch, C, h, w, lr, mu = cfg_like
+    ctx = make_ctx(c_in, ch, C, h, w, theta, prec=prec, lr=lr, mu=mu)
+    st.st_set_frozen_features(ctx, 0, dev(feat))
+    labels = torch.empty((4 * h, 4 * w), dtype=torch.uint8, device="cuda")
+    st.st_teacher_labels(ctx, 0, dev(T), labels)
+    loss = torch.zeros(n_steps, dtype=torch.float32, device="cuda")
+    conf = torch.zeros((n_steps, C, C), dtype=torch.int64, device="cuda") if want_conf else None
+    st.st_distill_step(ctx, n_steps, loss, conf)
+    head = oracle.Head(c_in, ch, C, lr=lr, momentum=mu, theta=theta, quantize_bf16=quantize)
+    lab_ref = oracle.teacher_labels(T)
+    np.testing.assert_array_equal(labels.cpu().numpy(), lab_ref)
+    ref_loss, ref_masks = [], []
+    for _ in range(n_steps):
+        l, m = oracle.distill_step(head, feat, lab_ref)
+        ref_loss.append(l); ref_masks.append(m)
+    return ctx, head, loss.cpu().numpy(), np.array(ref_loss), (conf.cpu().numpy() if want_conf else None), ref_masks, lab_ref
+
+
+def check_weights(ctx, head, theta0, max_rel, mean_abs, upd_rel):
+    got = packed(ctx)
+    ref = head.theta
+    off = 0
+    for ws, bs in oracle.param_shapes(head.c_in, head.c_hidden, head.n_classes):
+        for n in (int(np.prod(ws)), int(np.prod(bs))):
+            g, r = got[off:off + n], ref[off:off + n]
+            scale = max(np.abs(r).max(), 1e-6)
+            assert np.abs(g - r).max() / scale <= max_rel, (off, np.abs(g - r).max() / scale)
+            off += n
+    assert np.abs(got - ref).mean() <= mean_abs
+    du, dr = got - theta0, ref - theta0
+    rel = np.linalg.norm(du - dr) / max(np.linalg.norm(dr), 1e-30)
+    assert rel <= upd_rel, rel        # a wrong gradient cannot pass this one
+    return rel
+
+
+def test_config1_tiny_fp32_step():
+    cfg = si.get_config(1)
+    feat, T, theta = si.stream_inputs(cfg)
+    like = (cfg.c_in, 0, cfg.n_classes, cfg.feat_h, cfg.feat_w, cfg.lr, cfg.momentum)
+    ctx, head, loss, ref_loss, conf, ref_masks, lab = run_both(like, feat, T, theta, 1, 0, want_conf=True)
+    assert abs(loss[0] - ref_loss[0]) <= 1e-4 * abs(ref_loss[0])             # stated tolerance: 1e-4 relative
+    check_weights(ctx, head, theta, max_rel=1e-5, mean_abs=1e-5, upd_rel=1e-4)  # fp32 GEMMs: 1e-5
+    # logits and their gradient, element by element
+    z = st.st_read_tensor(ctx, 0, st.ST_TENSOR_LOGITS)
+    # (z was produced by the forward of step 1, i.e. with the initial weights)
+    head0 = oracle.Head(cfg.c_in, 0, cfg.n_classes, theta=theta)
+    z_ref, _ = oracle.head_forward(head0, feat)
+    np.testing.assert_allclose(z, z_ref.ravel(), rtol=1e-5, atol=1e-5)
+    u = oracle.upsample(z_ref, 4)
+    _, g, _ = oracle.softmax_ce(u, lab)
+    dz_ref = oracle.upsample_adjoint(g, 4)
+    dz = st.st_read_tensor(ctx, 0, st.ST_TENSOR_LOGIT_GRAD)
+    np.testing.assert_allclose(dz, dz_ref.ravel(), rtol=1e-4, atol=1e-9)
+    # fused confusion of the pre-update forward vs. oracle mask: differing pixels only at near-ties
+    ref_conf, _, _ = oracle.agreement(lab, ref_masks[0], cfg.n_classes)
+    assert conf[0].sum() == lab.size
+    assert np.abs(conf[0] - ref_conf).sum() <= 2 * max(2, lab.size // 1000)
+    # agreement after the step: the GPU's own mask, counted by the oracle, must match bit for bit
+    mask = torch.empty(lab.shape, dtype=torch.uint8, device="cuda")
+    st.st_student_mask(ctx, 0, mask)
+    gconf = np.zeros((cfg.n_classes, cfg.n_classes), np.int64)
+    m = st.st_agreement(ctx, 0, None, None, gconf)
+    oconf, om, _ = oracle.agreement(lab, mask.cpu().numpy(), cfg.n_classes)
+    np.testing.assert_array_equal(gconf, oconf)
+    assert m == om
+    # and the mask itself agrees with the oracle's except at near-ties of the top-2 logits
+    omask = oracle.student_mask(head, feat)
+    diff = mask.cpu().numpy() != omask
+    assert diff.mean() <= 1e-3
+    if diff.any():
+        zz, _ = oracle.head_forward(head, feat)
+        uu = np.sort(oracle.upsample(zz, 4), axis=0)
+        gap = (uu[-1] - uu[-2])[diff]
+        assert gap.max() <= 1e-5 * max(1.0, np.abs(uu).max())
+    st.st_destroy(ctx)
+
+
+@pytest.mark.parametrize("c_in,ch,C,h,w,K,mu", [
+    (5, 0, 3, 7, 9, 3, 0.9),        # odd sizes: ragged tiles in every kernel
+    (8, 0, 21, 17, 33, 2, 0.0),
+    (6, 7, 4, 9, 11, 3, 0.9),       # two-layer head, fp32
+    (4, 0, 40, 3, 5, 2, 0.5),       # more classes than one register tile
+    (3, 0, 2, 1, 1, 2, 0.0),        # single feature pixel: every frame pixel is border
+])
+def test_small_fp32_steps(c_in, ch, C, h, w, K, mu):
+    feat, T = rand_problem(7, c_in, C, h, w)
+    theta = si.initial_head_params(c_in, ch, C, 3)
+    if ch:
+        theta[ch * c_in * 9: ch * c_in * 9 + ch] = 0.05
+    like = (c_in, ch, C, h, w, 0.05, mu)
+    ctx, head, loss, ref_loss, conf, _, lab = run_both(like, feat, T, theta, K, 0)
+    np.testing.assert_allclose(loss, ref_loss, rtol=1e-4)
+    check_weights(ctx, head, theta, max_rel=1e-5, mean_abs=1e-5, upd_rel=2e-4)
+    # the applied gradient of the last step and the momentum buffer
+    v = st.st_read_tensor(ctx, 0, st.ST_TENSOR_MOMENTUM)
+    np.testing.assert_allclose(v, head.vel, rtol=2e-3, atol=1e-7)
+    st.st_destroy(ctx)
+
+
+def test_two_streams_are_independent_fp32():
+    c_in, C, h, w = 6, 3, 5, 7
+    probs = [rand_problem(20 + s, c_in, C, h, w) for s in range(2)]
+    thetas = [si.initial_head_params(c_in, 0, C, 30 + s) for s in range(2)]
+    ctx = make_ctx(c_in, 0, C, h, w, np.concatenate(thetas), S=2, lr=0.05, mu=0.9)
+    for s in range(2):
+        st.st_set_frozen_features(ctx, s, dev(probs[s][0]))
+        st.st_teacher_labels(ctx, s, dev(probs[s][1]))
+    loss = torch.zeros((2, 3), dtype=torch.float32, device="cuda")
+    st.st_distill_step(ctx, 3, loss)
+    for s in range(2):
+        head = oracle.Head(c_in, 0, C, lr=0.05, momentum=0.9, theta=thetas[s])
+        lab = oracle.teacher_labels(probs[s][1])
+        ref = [oracle.distill_step(head, probs[s][0], lab)[0] for _ in range(3)]
+        np.testing.assert_allclose(loss[s].cpu().numpy(), ref, rtol=1e-4)
+        np.testing.assert_allclose(packed(ctx, s), head.theta, rtol=1e-4, atol=1e-6)
+    st.st_destroy(ctx)
+
+
+def test_out_of_range_training_labels_are_skipped_and_reported():
+    c_in, C, h, w = 4, 3, 2, 3
+    feat, T = rand_problem(5, c_in, C, h, w)
+    lab = oracle.teacher_labels(T).copy()
+    lab[2, 5] = 200
+    theta = si.initial_head_params(c_in, 0, C, 1)
+    ctx = make_ctx(c_in, 0, C, h, w, theta, lr=0.05)
+    st.st_set_frozen_features(ctx, 0, feat)
+    st.st_set_labels(ctx, 0, lab)
+    loss = np.zeros(1, np.float32)
+    st.st_distill_step(ctx, 1, loss)
+    with pytest.raises(st.StError) as ei:
+        st.st_read_tensor(ctx, 0, st.ST_TENSOR_LOGITS)
+    assert ei.value.status == st.ST_ERR_INVALID_ARG
+    head = oracle.Head(c_in, 0, C, lr=0.05, theta=theta)
+    ref, _ = oracle.distill_step(head, feat, lab)
+    assert abs(loss[0] - ref) <= 1e-4 * abs(ref)
+    np.testing.assert_allclose(packed(ctx), head.theta, rtol=1e-4, atol=1e-6)
+    st.st_destroy(ctx)
+
+
+def test_steps_are_bit_reproducible():
+    c_in, C, h, w = 8, 5, 9, 13
+    feat, T = rand_problem(9, c_in, C, h, w)
+    theta = si.initial_head_params(c_in, 0, C, 2)
+    outs = []
+    for _ in range(2):
+        ctx = make_ctx(c_in, 0, C, h, w, theta, lr=0.05, mu=0.9)
+        st.st_set_frozen_features(ctx, 0, dev(feat)); st.st_teacher_labels(ctx, 0, dev(T))
+        st.st_distill_step(ctx, 4)
+        outs.append(packed(ctx))
+        st.st_destroy(ctx)
+    assert outs[0].tobytes() == outs[1].tobytes()
