@@ -334,7 +334,9 @@ st_status st_init_head(const st_head_desc* desc, const float* init_params, st_ct
     c->n_params = (int64_t)st_param_count(d.c_in, d.c_hidden, d.n_classes);
     c->bf16_mode = d.gemm_precision == 1;
     c->has_feat.assign(c->S, 0); c->has_labels.assign(c->S, 0);
-    if (const char* e = getenv("ST_NO_GRAPH")) c->use_graphs = !(e[0] == '1');
+    // The legacy default stream cannot be captured: steps are then enqueued kernel by kernel.
+    c->use_graphs = c->stream != nullptr && c->stream != cudaStreamLegacy && c->stream != cudaStreamPerThread;
+    if (const char* e = getenv("ST_NO_GRAPH")) if (e[0] == '1') c->use_graphs = false;
 
     PackLayout& L = c->layout;
     memset(&L, 0, sizeof L);

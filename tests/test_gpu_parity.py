@@ -12,6 +12,15 @@ pytestmark = pytest.mark.gpu
 torch = pytest.importorskip("torch")
 
 
+@pytest.fixture(autouse=True)
+def side_stream():
+    """Run every test on a non-default stream (step loops are then replayed as CUDA graphs)."""
+    s = torch.cuda.Stream()
+    with torch.cuda.stream(s):
+        yield s
+    s.synchronize()
+
+
 def dev(a):
     return torch.from_numpy(np.ascontiguousarray(a)).cuda()
 
@@ -281,6 +290,22 @@ def test_out_of_range_training_labels_are_skipped_and_reported():
     assert abs(loss[0] - ref) <= 1e-4 * abs(ref)
     np.testing.assert_allclose(packed(ctx), head.theta, rtol=1e-4, atol=1e-6)
     st.st_destroy(ctx)
+
+
+def test_default_stream_runs_without_graph_capture():
+    c_in, C, h, w = 8, 5, 9, 13
+    feat, T = rand_problem(9, c_in, C, h, w)
+    theta = si.initial_head_params(c_in, 0, C, 2)
+    outs = []
+    for stream in (torch.cuda.default_stream(), torch.cuda.current_stream()):
+        with torch.cuda.stream(stream):
+            ctx = make_ctx(c_in, 0, C, h, w, theta, lr=0.05, mu=0.9)
+            st.st_set_frozen_features(ctx, 0, feat); st.st_teacher_labels(ctx, 0, T)
+            st.st_distill_step(ctx, 2)
+            st.st_distill_step(ctx, 2)
+            outs.append(packed(ctx))
+            st.st_destroy(ctx)
+    assert outs[0].tobytes() == outs[1].tobytes()
 
 
 def test_steps_are_bit_reproducible():
