@@ -1,12 +1,647 @@
-// placeholder until the tcgen05 kernels land
+// bf16 tensor-core GEMMs of the head (gemm_precision 1): Forward and PartialBackward of Algorithm 1
+// for the trainable back part (Section 4.2), as TMA-fed tcgen05 kernels with fp32 accumulators in
+// tensor memory.  Operands are bf16 (cached features, bf16 copies of the weights, rounded
+// gradients); every accumulation is fp32.
+//
+//   fwd 1x1   z[c][pix]       = b[c] + sum_k A[pix][k] W[c][k]                 A = features or hidden
+//   fwd 3x3   Hd[pix][co]     = ReLU(b1[co] + sum_{tap,ci} X[pix+tap][ci] W1[tap][co][ci])
+//   wgrad 1x1 dW[c][k]        = sum_pix dz[c][pix] A[pix][k]                   split over pixel ranges
+//   dgrad     dHd[pix][k]     = [Hd[pix][k] > 0] sum_c dz[c][pix] W2[c][k]     (fp32 FMA, bf16 out)
+//   wgrad 3x3 dW1[tap][co][ci]= sum_pix dHd[pix][co] X[pix+tap][ci]            split over pixel ranges
+//
+// Pixel-major activations [pix][channel] are K-major operands when the GEMM reduces over channels
+// (forward) and MN-major operands when it reduces over pixels (weight gradients); both forms are
+// read straight from the same TMA 128-byte-swizzled tiles, no transposing pass exists.
+// The zero padding of the 3x3 convolution is TMA's out-of-bounds fill: taps are plain box loads at
+// shifted (x, y) coordinates of a [channel][x][y][stream] tensor map.
 #include "st_internal.h"
+#include "tc_common.cuh"
+
 #include <cstdio>
+#include <cstring>
+
 namespace st {
-struct TcPlan { int dummy; };
-int tc_wgrad_splits(int, int, int, int, int) { return 1; }
-int tc_b1_partials(int, int) { return 1; }
-TcPlan* tc_plan_create(const TcBuffers&, char* err, size_t n) { snprintf(err, n, "tensor-core path not built"); return nullptr; }
-void tc_plan_destroy(TcPlan* p) { delete p; }
-int tc_forward(const TcPlan*, cudaStream_t) { return 0; }
-int tc_backward(const TcPlan*, cudaStream_t) { return 0; }
+
+using namespace tc;
+
+namespace {
+
+constexpr int kThreadsTc = 128;          // 4 warps: TMEM lanes 32w .. 32w+31 belong to warp w
+constexpr int kBlockK = 64;              // bf16 elements per 128-byte swizzled row
+constexpr int kTileM = 128;              // UMMA M
+constexpr int kChunkPix = 64;            // pixels per pipeline stage of the weight-gradient GEMMs
+constexpr int kTileW = 32, kTileH = 4;   // 3x3 forward: 128 pixels = 4 rows x 32 columns
+constexpr int kChunkW = 32, kChunkH = 2; // 3x3 wgrad: 64 pixels = 2 rows x 32 columns
+constexpr int kSmemAlign = 1024;
+constexpr int kMaxKBlocks = 16;
+
+__device__ __forceinline__ uint8_t* align_smem(uint8_t* p)
+{
+    return (uint8_t*)(((uintptr_t)p + kSmemAlign - 1) & ~(uintptr_t)(kSmemAlign - 1));
 }
+
+// ------------------------------------------------------------------------------------------------
+// fwd 1x1: one 128-pixel tile per block; the whole K extent is loaded at once (one barrier per
+// 64-channel block so that the MMAs start while later blocks are still in flight).
+// ------------------------------------------------------------------------------------------------
+__global__ void __launch_bounds__(kThreadsTc)
+tc_fwd1x1_kernel(const __grid_constant__ CUtensorMap tmA,   // {K, p, S}  box {64, 128, 1}
+                 const __grid_constant__ CUtensorMap tmB,   // {K, 32, S} box {64, 32, 1}
+                 const float* __restrict__ theta, int64_t n_params, int64_t b_off,
+                 float* __restrict__ z, int C, int p, int kblocks, unsigned int* err)
+{
+    extern __shared__ uint8_t smem_raw[];
+    uint8_t* smem = align_smem(smem_raw);
+    const uint32_t a_base = smem_u32(smem);
+    const uint32_t b_base = a_base + kblocks * (kTileM * 128);
+    __shared__ __align__(8) uint64_t bars[kMaxKBlocks + 1];
+    __shared__ uint32_t tmem_slot;
+    const int tid = threadIdx.x, warp = tid >> 5;
+    const int s = blockIdx.y, pix0 = blockIdx.x * kTileM;
+
+    if (warp == 0) tmem_alloc(smem_u32(&tmem_slot), 32);
+    if (tid == 0) {
+        for (int i = 0; i <= kblocks; ++i) mbar_init(smem_u32(&bars[i]), 1);
+        fence_barrier_init();
+    }
+    tc_fence_before_sync();
+    __syncthreads();
+    tc_fence_after_sync();
+    const uint32_t tmem = tmem_slot;
+    const uint32_t done_bar = smem_u32(&bars[kblocks]);
+    bool ok = true;
+
+    if (tid == 0) {
+        for (int kb = 0; kb < kblocks; ++kb) {
+            const uint32_t bar = smem_u32(&bars[kb]);
+            mbar_expect_tx(bar, kTileM * 128 + kClassPad * 128);
+            tma_load_3d(a_base + kb * (kTileM * 128), &tmA, bar, kb * kBlockK, pix0, s);
+            tma_load_3d(b_base + kb * (kClassPad * 128), &tmB, bar, kb * kBlockK, 0, s);
+        }
+    } else if (tid == 32) {
+        constexpr uint32_t idesc = instr_desc(kTileM, kClassPad, 0, 0);
+        for (int kb = 0; kb < kblocks; ++kb) {
+            ok = mbar_wait(smem_u32(&bars[kb]), 0, err, kWaitFull);
+            if (!ok) break;
+            tc_fence_after_sync();
+#pragma unroll
+            for (int k = 0; k < 4; ++k) {
+                const uint64_t da = smem_desc(a_base + kb * (kTileM * 128) + k * 32, 16, 1024);
+                const uint64_t db = smem_desc(b_base + kb * (kClassPad * 128) + k * 32, 16, 1024);
+                umma(tmem, da, db, idesc, (kb | k) != 0);
+            }
+        }
+        umma_commit(done_bar);
+    }
+    __syncwarp();
+    ok = mbar_wait(done_bar, 0, err, kWaitDone);
+    tc_fence_after_sync();
+    if (ok) {
+        float v[32];
+        tmem_ld_32x32(tmem + ((uint32_t)(warp * 32) << 16), v);
+        const int pix = pix0 + tid;
+        if (pix < p) {
+            const float* bias = theta + (int64_t)s * n_params + b_off;
+            float* dst = z + (int64_t)s * C * p + pix;
+#pragma unroll
+            for (int c = 0; c < kClassPad; ++c)
+                if (c < C) dst[(int64_t)c * p] = v[c] + __ldg(bias + c);
+        }
+    } else {
+        drain_after_error();
+    }
+    tc_fence_before_sync();
+    __syncthreads();
+    if (warp == 0) tmem_dealloc(tmem, 32);
+}
+
+// ------------------------------------------------------------------------------------------------
+// wgrad 1x1: D[k][c] += sum over this block's pixel chunks of A[pix][k] * dz[c][pix].
+// A (pixel-major activations) is the MN-major operand with M = channel; dz rows are K-major.
+// ------------------------------------------------------------------------------------------------
+template <int STAGES>
+__global__ void __launch_bounds__(kThreadsTc)
+tc_wgrad1x1_kernel(const __grid_constant__ CUtensorMap tmA,   // {K, p, S}      box {64, 64, 1}
+                   const __grid_constant__ CUtensorMap tmB,   // {p, 32, S}     box {64, 32, 1}
+                   float* __restrict__ partials,              // [S][n_split][32][K]
+                   int K, int n_chunks, int chunks_per_block, int tmem_cols, unsigned int* err)
+{
+    extern __shared__ uint8_t smem_raw[];
+    uint8_t* smem = align_smem(smem_raw);
+    const int m_tiles = (K + kTileM - 1) / kTileM;   // accumulators (128 channels each)
+    const int a_blocks = m_tiles * 2;                // 64-channel blocks loaded per stage (absent ones are zero-filled)
+    const uint32_t a_stage_bytes = a_blocks * (kChunkPix * 128);
+    const uint32_t stage_bytes = a_stage_bytes + kClassPad * 128;
+    const uint32_t base = smem_u32(smem);
+    __shared__ __align__(8) uint64_t full[STAGES], empty[STAGES], done;
+    __shared__ uint32_t tmem_slot;
+    const int tid = threadIdx.x, warp = tid >> 5;
+    const int s = blockIdx.y, split = blockIdx.x, n_split = gridDim.x;
+    const int c_begin = split * chunks_per_block;
+    const int c_end = min(n_chunks, c_begin + chunks_per_block);
+
+    if (warp == 0) tmem_alloc(smem_u32(&tmem_slot), tmem_cols);
+    if (tid == 0) {
+        for (int i = 0; i < STAGES; ++i) { mbar_init(smem_u32(&full[i]), 1); mbar_init(smem_u32(&empty[i]), 1); }
+        mbar_init(smem_u32(&done), 1);
+        fence_barrier_init();
+    }
+    tc_fence_before_sync();
+    __syncthreads();
+    tc_fence_after_sync();
+    const uint32_t tmem = tmem_slot;
+    bool ok = true;
+
+    if (tid == 0) {
+        for (int i = c_begin; i < c_end; ++i) {
+            const int it = i - c_begin, st = it % STAGES;
+            if (it >= STAGES) ok = mbar_wait(smem_u32(&empty[st]), ((it / STAGES) - 1) & 1, err, kWaitEmpty);
+            if (!ok) break;
+            const uint32_t bar = smem_u32(&full[st]);
+            const uint32_t sa = base + st * stage_bytes;
+            mbar_expect_tx(bar, stage_bytes);
+            for (int cb = 0; cb < a_blocks; ++cb)
+                tma_load_3d(sa + cb * (kChunkPix * 128), &tmA, bar, cb * kBlockK, i * kChunkPix, s);
+            tma_load_3d(sa + a_stage_bytes, &tmB, bar, i * kChunkPix, 0, s);
+        }
+    } else if (tid == 32) {
+        constexpr uint32_t idesc = instr_desc(kTileM, kClassPad, 1, 0);
+        for (int i = c_begin; i < c_end; ++i) {
+            const int it = i - c_begin, st = it % STAGES;
+            ok = mbar_wait(smem_u32(&full[st]), (it / STAGES) & 1, err, kWaitFull);
+            if (!ok) break;
+            tc_fence_after_sync();
+            const uint32_t sa = base + st * stage_bytes, sb = sa + a_stage_bytes;
+            for (int m = 0; m < m_tiles; ++m)
+#pragma unroll
+                for (int j = 0; j < kChunkPix / 16; ++j) {
+                    const uint64_t da = smem_desc(sa + (2 * m) * (kChunkPix * 128) + j * (16 * 128), kChunkPix * 128, 1024);
+                    const uint64_t db = smem_desc(sb + j * 32, 16, 1024);
+                    umma(tmem + m * kClassPad, da, db, idesc, (it | j) != 0);
+                }
+            umma_commit(smem_u32(&empty[st]));
+        }
+        umma_commit(smem_u32(&done));
+    }
+    __syncwarp();
+    ok = mbar_wait(smem_u32(&done), 0, err, kWaitDone);
+    tc_fence_after_sync();
+    if (ok) {
+        float* dst = partials + ((int64_t)s * n_split + split) * kClassPad * K;
+        const bool any = c_end > c_begin;
+        for (int m = 0; m < m_tiles; ++m) {
+            float v[32];
+            tmem_ld_32x32(tmem + ((uint32_t)(warp * 32) << 16) + m * kClassPad, v);
+            const int k = m * kTileM + tid;
+            if (k < K)
+#pragma unroll
+                for (int c = 0; c < kClassPad; ++c) dst[(int64_t)c * K + k] = any ? v[c] : 0.f;
+        }
+    } else {
+        drain_after_error();
+    }
+    tc_fence_before_sync();
+    __syncthreads();
+    if (warp == 0) tmem_dealloc(tmem, tmem_cols);
+}
+
+// ------------------------------------------------------------------------------------------------
+// fwd 3x3 (+bias, ReLU): one tile of 4 rows x 32 columns of pixels per block, N = Ch output channels,
+// K loop = 9 taps x (Cin / 64) channel blocks through a ring of stages.
+// ------------------------------------------------------------------------------------------------
+template <int STAGES>
+__global__ void __launch_bounds__(kThreadsTc)
+tc_fwd3x3_kernel(const __grid_constant__ CUtensorMap tmA,   // {Cin, w, h, S}    box {64, 32, 4, 1}
+                 const __grid_constant__ CUtensorMap tmB,   // {Cin, 9*Ch, S}    box {64, Ch, 1}
+                 const float* __restrict__ theta, int64_t n_params, int64_t b_off,
+                 bf16* __restrict__ hidden,                  // [S][p][Ch]
+                 int Cin, int Ch, int h, int w, int tmem_cols, unsigned int* err)
+{
+    extern __shared__ uint8_t smem_raw[];
+    uint8_t* smem = align_smem(smem_raw);
+    const uint32_t base = smem_u32(smem);
+    const uint32_t a_bytes = kTileM * 128, b_bytes = (uint32_t)Ch * 128, stage_bytes = a_bytes + b_bytes;
+    __shared__ __align__(8) uint64_t full[STAGES], empty[STAGES], done;
+    __shared__ uint32_t tmem_slot;
+    const int tid = threadIdx.x, warp = tid >> 5;
+    const int tiles_x = (w + kTileW - 1) / kTileW;
+    const int x0 = (blockIdx.x % tiles_x) * kTileW, y0 = (blockIdx.x / tiles_x) * kTileH, s = blockIdx.y;
+    const int kblocks = Cin / kBlockK, n_iter = 9 * kblocks;
+
+    if (warp == 0) tmem_alloc(smem_u32(&tmem_slot), tmem_cols);
+    if (tid == 0) {
+        for (int i = 0; i < STAGES; ++i) { mbar_init(smem_u32(&full[i]), 1); mbar_init(smem_u32(&empty[i]), 1); }
+        mbar_init(smem_u32(&done), 1);
+        fence_barrier_init();
+    }
+    tc_fence_before_sync();
+    __syncthreads();
+    tc_fence_after_sync();
+    const uint32_t tmem = tmem_slot;
+    bool ok = true;
+
+    if (tid == 0) {
+        for (int it = 0; it < n_iter; ++it) {
+            const int st = it % STAGES, tap = it / kblocks, kb = it % kblocks;
+            if (it >= STAGES) ok = mbar_wait(smem_u32(&empty[st]), ((it / STAGES) - 1) & 1, err, kWaitEmpty);
+            if (!ok) break;
+            const uint32_t bar = smem_u32(&full[st]), sa = base + st * stage_bytes;
+            mbar_expect_tx(bar, stage_bytes);
+            tma_load_4d(sa, &tmA, bar, kb * kBlockK, x0 + tap % 3 - 1, y0 + tap / 3 - 1, s);
+            tma_load_3d(sa + a_bytes, &tmB, bar, kb * kBlockK, tap * Ch, s);
+        }
+    } else if (tid == 32) {
+        const uint32_t idesc = instr_desc(kTileM, Ch, 0, 0);
+        for (int it = 0; it < n_iter; ++it) {
+            const int st = it % STAGES;
+            ok = mbar_wait(smem_u32(&full[st]), (it / STAGES) & 1, err, kWaitFull);
+            if (!ok) break;
+            tc_fence_after_sync();
+            const uint32_t sa = base + st * stage_bytes, sb = sa + a_bytes;
+#pragma unroll
+            for (int k = 0; k < 4; ++k)
+                umma(tmem, smem_desc(sa + k * 32, 16, 1024), smem_desc(sb + k * 32, 16, 1024), idesc, (it | k) != 0);
+            umma_commit(smem_u32(&empty[st]));
+        }
+        umma_commit(smem_u32(&done));
+    }
+    __syncwarp();
+    ok = mbar_wait(smem_u32(&done), 0, err, kWaitDone);
+    tc_fence_after_sync();
+    if (ok) {
+        const int y = y0 + tid / kTileW, x = x0 + tid % kTileW;
+        const bool in = y < h && x < w;
+        const float* bias = theta + (int64_t)s * n_params + b_off;
+        bf16* dst = hidden + ((int64_t)s * h * w + (int64_t)y * w + x) * Ch;
+        for (int n0 = 0; n0 < Ch; n0 += 32) {
+            float v[32];
+            tmem_ld_32x32(tmem + ((uint32_t)(warp * 32) << 16) + n0, v);
+            if (in) {
+                uint4 out[4];
+                __nv_bfloat162* o2 = reinterpret_cast<__nv_bfloat162*>(out);
+#pragma unroll
+                for (int k = 0; k < 16; ++k) {
+                    float a = v[2 * k] + __ldg(bias + n0 + 2 * k), b = v[2 * k + 1] + __ldg(bias + n0 + 2 * k + 1);
+                    o2[k] = __floats2bfloat162_rn(fmaxf(a, 0.f), fmaxf(b, 0.f));
+                }
+#pragma unroll
+                for (int k = 0; k < 4; ++k) reinterpret_cast<uint4*>(dst + n0)[k] = out[k];
+            }
+        }
+    } else {
+        drain_after_error();
+    }
+    tc_fence_before_sync();
+    __syncthreads();
+    if (warp == 0) tmem_dealloc(tmem, tmem_cols);
+}
+
+// ------------------------------------------------------------------------------------------------
+// wgrad 3x3: for one tap, D[ci][co] += sum over this block's pixel chunks of X[pix+tap][ci] * dHd[pix][co].
+// Both operands are MN-major (pixel-major activations, reduction over pixels).  A block keeps
+// ceil(Cin/128) accumulators of Ch columns (all input channels of one tap) so that the dHd tile of a
+// stage is shared by all of them.
+// ------------------------------------------------------------------------------------------------
+template <int STAGES>
+__global__ void __launch_bounds__(kThreadsTc)
+tc_wgrad3x3_kernel(const __grid_constant__ CUtensorMap tmA,   // X   {Cin, w, h, S} box {64, 32, 2, 1}
+                   const __grid_constant__ CUtensorMap tmB,   // dHd {Ch,  w, h, S} box {64, 32, 2, 1}
+                   float* __restrict__ partials,              // [S][n_split][9][Ch][Cin]
+                   int Cin, int Ch, int h, int w, int n_chunks, int chunks_per_block, int n_split,
+                   int tmem_cols, unsigned int* err)
+{
+    extern __shared__ uint8_t smem_raw[];
+    uint8_t* smem = align_smem(smem_raw);
+    const uint32_t base = smem_u32(smem);
+    const int m_tiles = (Cin + kTileM - 1) / kTileM;
+    const int a_blocks = m_tiles * 2, b_blocks = Ch / kBlockK;
+    const uint32_t blk_bytes = kChunkPix * 128;
+    const uint32_t a_bytes = a_blocks * blk_bytes, stage_bytes = a_bytes + b_blocks * blk_bytes;
+    __shared__ __align__(8) uint64_t full[STAGES], empty[STAGES], done;
+    __shared__ uint32_t tmem_slot;
+    const int tid = threadIdx.x, warp = tid >> 5;
+    const int tap = blockIdx.x % 9, split = blockIdx.x / 9, s = blockIdx.y;
+    const int chunks_x = (w + kChunkW - 1) / kChunkW;
+    const int c_begin = split * chunks_per_block, c_end = min(n_chunks, c_begin + chunks_per_block);
+
+    if (warp == 0) tmem_alloc(smem_u32(&tmem_slot), tmem_cols);
+    if (tid == 0) {
+        for (int i = 0; i < STAGES; ++i) { mbar_init(smem_u32(&full[i]), 1); mbar_init(smem_u32(&empty[i]), 1); }
+        mbar_init(smem_u32(&done), 1);
+        fence_barrier_init();
+    }
+    tc_fence_before_sync();
+    __syncthreads();
+    tc_fence_after_sync();
+    const uint32_t tmem = tmem_slot;
+    bool ok = true;
+
+    if (tid == 0) {
+        for (int i = c_begin; i < c_end; ++i) {
+            const int it = i - c_begin, st = it % STAGES;
+            if (it >= STAGES) ok = mbar_wait(smem_u32(&empty[st]), ((it / STAGES) - 1) & 1, err, kWaitEmpty);
+            if (!ok) break;
+            const int x0 = (i % chunks_x) * kChunkW, y0 = (i / chunks_x) * kChunkH;
+            const uint32_t bar = smem_u32(&full[st]), sa = base + st * stage_bytes;
+            mbar_expect_tx(bar, stage_bytes);
+            for (int cb = 0; cb < a_blocks; ++cb)
+                tma_load_4d(sa + cb * blk_bytes, &tmA, bar, cb * kBlockK, x0 + tap % 3 - 1, y0 + tap / 3 - 1, s);
+            for (int cb = 0; cb < b_blocks; ++cb)
+                tma_load_4d(sa + a_bytes + cb * blk_bytes, &tmB, bar, cb * kBlockK, x0, y0, s);
+        }
+    } else if (tid == 32) {
+        const uint32_t idesc = instr_desc(kTileM, Ch, 1, 1);
+        for (int i = c_begin; i < c_end; ++i) {
+            const int it = i - c_begin, st = it % STAGES;
+            ok = mbar_wait(smem_u32(&full[st]), (it / STAGES) & 1, err, kWaitFull);
+            if (!ok) break;
+            tc_fence_after_sync();
+            const uint32_t sa = base + st * stage_bytes, sb = sa + a_bytes;
+            for (int m = 0; m < m_tiles; ++m)
+#pragma unroll
+                for (int j = 0; j < kChunkPix / 16; ++j) {
+                    const uint64_t da = smem_desc(sa + (2 * m) * blk_bytes + j * (16 * 128), blk_bytes, 1024);
+                    const uint64_t db = smem_desc(sb + j * (16 * 128), blk_bytes, 1024);
+                    umma(tmem + m * Ch, da, db, idesc, (it | j) != 0);
+                }
+            umma_commit(smem_u32(&empty[st]));
+        }
+        umma_commit(smem_u32(&done));
+    }
+    __syncwarp();
+    ok = mbar_wait(smem_u32(&done), 0, err, kWaitDone);
+    tc_fence_after_sync();
+    if (ok) {
+        float* dst = partials + (((int64_t)s * n_split + split) * 9 + tap) * Ch * Cin;
+        const bool any = c_end > c_begin;
+        for (int m = 0; m < m_tiles; ++m) {
+            const int ci = m * kTileM + tid;
+            for (int n0 = 0; n0 < Ch; n0 += 32) {
+                float v[32];
+                tmem_ld_32x32(tmem + ((uint32_t)(warp * 32) << 16) + m * Ch + n0, v);
+                if (ci < Cin)
+#pragma unroll
+                    for (int c = 0; c < 32; ++c) dst[(int64_t)(n0 + c) * Cin + ci] = any ? v[c] : 0.f;
+            }
+        }
+    } else {
+        drain_after_error();
+    }
+    tc_fence_before_sync();
+    __syncthreads();
+    if (warp == 0) tmem_dealloc(tmem, tmem_cols);
+}
+
+// ------------------------------------------------------------------------------------------------
+// dgrad through the 1x1 output layer with the ReLU mask of the hidden activation, fp32 FMA from the
+// unrounded dz and the fp32 master weight; output rounded to bf16 (it is a GEMM operand next).
+// Also emits per-block partial sums of the (unrounded) result over pixels: the bias gradient of the
+// 3x3 layer.  Block = 64 pixels x all hidden channels; thread = one channel pair x a share of the pixels.
+// ------------------------------------------------------------------------------------------------
+constexpr int kDgradPix = 64;
+
+__global__ void __launch_bounds__(256)
+dgrad_relu_kernel(const float* __restrict__ theta, int64_t n_params, int64_t w2_off,
+                  const float* __restrict__ dz,        // [S][C][p]
+                  const bf16* __restrict__ hidden,     // [S][p][Ch]
+                  bf16* __restrict__ dhidden,          // [S][p][Ch]
+                  float* __restrict__ b1_partials,     // [S][n_blocks][Ch]
+                  int C, int Ch, int p)
+{
+    extern __shared__ float sm[];
+    float* w2 = sm;                     // [C][Ch]
+    float* dzt = w2 + C * Ch;           // [C][kDgradPix]
+    float* red = dzt + C * kDgradPix;   // [groups][Ch]
+    const int s = blockIdx.y, blk = blockIdx.x, pix0 = blk * kDgradPix;
+    const int pairs = Ch / 2, groups = 256 / pairs;    // Ch in {64,128,192,256} -> groups 8, 4, 2, 2
+    const float* W2 = theta + (int64_t)s * n_params + w2_off;
+    for (int i = threadIdx.x; i < C * Ch; i += 256) w2[i] = __ldg(W2 + i);
+    for (int i = threadIdx.x; i < C * kDgradPix; i += 256) {
+        const int c = i / kDgradPix, q = i % kDgradPix;
+        dzt[i] = (pix0 + q < p) ? __ldg(dz + ((int64_t)s * C + c) * p + pix0 + q) : 0.f;
+    }
+    __syncthreads();
+    const int cp = threadIdx.x % pairs, g = threadIdx.x / pairs;
+    if (g < groups) {
+        float sum0 = 0.f, sum1 = 0.f;
+        for (int q = g; q < kDgradPix; q += groups) {
+            const int pix = pix0 + q;
+            if (pix >= p) break;
+            float a0 = 0.f, a1 = 0.f;
+            for (int c = 0; c < C; ++c) {
+                const float d = dzt[c * kDgradPix + q];
+                const float2 wv = *reinterpret_cast<const float2*>(w2 + c * Ch + 2 * cp);
+                a0 = fmaf(d, wv.x, a0); a1 = fmaf(d, wv.y, a1);
+            }
+            const int64_t off = ((int64_t)s * p + pix) * Ch + 2 * cp;
+            const __nv_bfloat162 hv = *reinterpret_cast<const __nv_bfloat162*>(hidden + off);
+            if (!(__low2float(hv) > 0.f)) a0 = 0.f;
+            if (!(__high2float(hv) > 0.f)) a1 = 0.f;
+            *reinterpret_cast<__nv_bfloat162*>(dhidden + off) = __floats2bfloat162_rn(a0, a1);
+            sum0 += a0; sum1 += a1;
+        }
+        red[g * Ch + 2 * cp] = sum0; red[g * Ch + 2 * cp + 1] = sum1;
+    }
+    __syncthreads();
+    for (int k = threadIdx.x; k < Ch; k += 256) {
+        float t = 0.f;
+        for (int gg = 0; gg < groups; ++gg) t += red[gg * Ch + k];
+        b1_partials[((int64_t)s * gridDim.x + blk) * Ch + k] = t;
+    }
+}
+
+// ---- host side -------------------------------------------------------------------------------------
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
+                                  const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
+                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+EncodeTiledFn get_encode_fn()
+{
+    static EncodeTiledFn fn = nullptr;
+    if (fn) return fn;
+    void* ptr = nullptr;
+    cudaDriverEntryPointQueryResult q;
+    if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &ptr, cudaEnableDefault, &q) != cudaSuccess || !ptr) return nullptr;
+    fn = (EncodeTiledFn)ptr;
+    return fn;
+}
+
+// bf16 tensor, innermost dimension first; strides (bytes) for dimensions 1..rank-1; 128-byte swizzle.
+bool make_map(CUtensorMap* m, const void* base, int rank, const uint64_t* dims, const uint64_t* strides,
+              const uint32_t* box, char* err, size_t err_len, const char* what)
+{
+    EncodeTiledFn fn = get_encode_fn();
+    if (!fn) { snprintf(err, err_len, "cuTensorMapEncodeTiled is not available"); return false; }
+    cuuint64_t d[5], st[4];
+    cuuint32_t b[5], es[5];
+    for (int i = 0; i < rank; ++i) { d[i] = dims[i]; b[i] = box[i]; es[i] = 1; }
+    for (int i = 0; i + 1 < rank; ++i) st[i] = strides[i];
+    CUresult r = fn(m, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, (cuuint32_t)rank, const_cast<void*>(base), d, st, b, es,
+                    CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                    CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    if (r != CUDA_SUCCESS) { snprintf(err, err_len, "tensor map for %s rejected (CUresult %d)", what, (int)r); return false; }
+    return true;
+}
+
+int pow2_cols(int n) { int c = 32; while (c < n) c <<= 1; return c; }
+
+void split_geometry(int n_chunks, int target_blocks, int* per, int* n_split)
+{
+    int pb = (n_chunks + target_blocks - 1) / target_blocks;
+    if (pb < 1) pb = 1;
+    *per = pb;
+    *n_split = (n_chunks + pb - 1) / pb;
+    if (*n_split < 1) *n_split = 1;
+}
+
+}  // namespace
+
+struct TcPlan {
+    TcBuffers b;
+    int p, p_pad, c_last;
+    CUtensorMap act_fwd;     // last-layer input {c_last, p, S} box {64, 128, 1}
+    CUtensorMap act_wg;      // same tensor, box {64, 64, 1}
+    CUtensorMap w2_map;      // {c_last, 32, S} box {64, 32, 1}
+    CUtensorMap dz_map;      // {p, 32, S} box {64, 32, 1}
+    CUtensorMap x_fwd3;      // {Cin, w, h, S} box {64, 32, 4, 1}
+    CUtensorMap x_wg3;       // box {64, 32, 2, 1}
+    CUtensorMap w1_map;      // {Cin, 9*Ch, S} box {64, Ch, 1}
+    CUtensorMap dh_wg3;      // {Ch, w, h, S} box {64, 32, 2, 1}
+    int split2, chunks2, per2, cols2;
+    int split1, chunks1, per1, cols1;
+    size_t smem_fwd1, smem_wg1, smem_fwd3, smem_wg3, smem_dgrad;
+};
+
+int tc_wgrad_splits(int layer, int c_in, int c_hidden, int h, int w)
+{
+    (void)c_in; (void)c_hidden;
+    int per, n;
+    if (layer == 2) {
+        const int64_t p = (int64_t)h * w;
+        split_geometry((int)((p + kChunkPix - 1) / kChunkPix), 148, &per, &n);
+    } else {
+        const int chunks = ((w + kChunkW - 1) / kChunkW) * ((h + kChunkH - 1) / kChunkH);
+        split_geometry(chunks, 148 / 9, &per, &n);
+    }
+    return n;
+}
+
+int tc_b1_partials(int h, int w) { return (int)(((int64_t)h * w + kDgradPix - 1) / kDgradPix); }
+
+int tc_dz_pitch(int h, int w) { return (int)((((int64_t)h * w + 63) / 64) * 64); }
+
+TcPlan* tc_plan_create(const TcBuffers& b, char* err, size_t err_len)
+{
+    TcPlan* P = new TcPlan();
+    memset((void*)P, 0, sizeof *P);
+    P->b = b;
+    P->p = b.h * b.w; P->p_pad = tc_dz_pitch(b.h, b.w);
+    P->c_last = b.c_hidden ? b.c_hidden : b.c_in;
+    const uint64_t S = (uint64_t)b.S, p = (uint64_t)P->p, cl = (uint64_t)P->c_last;
+    const bf16* act = b.c_hidden ? b.hidden : b.x;
+    bool ok = true;
+    {
+        uint64_t dims[3] = {cl, p, S}, str[2] = {cl * 2, p * cl * 2};
+        uint32_t box_f[3] = {64, 128, 1}, box_w[3] = {64, 64, 1};
+        ok = ok && make_map(&P->act_fwd, act, 3, dims, str, box_f, err, err_len, "last-layer input (forward)");
+        ok = ok && make_map(&P->act_wg, act, 3, dims, str, box_w, err, err_len, "last-layer input (wgrad)");
+    }
+    if (ok) {
+        uint64_t dims[3] = {cl, (uint64_t)kClassPad, S}, str[2] = {cl * 2, (uint64_t)kClassPad * cl * 2};
+        uint32_t box[3] = {64, (uint32_t)kClassPad, 1};
+        ok = make_map(&P->w2_map, b.w2, 3, dims, str, box, err, err_len, "1x1 weight");
+    }
+    if (ok) {
+        uint64_t dims[3] = {p, (uint64_t)kClassPad, S}, str[2] = {(uint64_t)P->p_pad * 2, (uint64_t)kClassPad * P->p_pad * 2};
+        uint32_t box[3] = {64, (uint32_t)kClassPad, 1};
+        ok = make_map(&P->dz_map, b.dz_bf16, 3, dims, str, box, err, err_len, "logit gradient");
+    }
+    if (ok && b.c_hidden) {
+        const uint64_t ci = (uint64_t)b.c_in, ch = (uint64_t)b.c_hidden, w = (uint64_t)b.w, h = (uint64_t)b.h;
+        uint64_t dx[4] = {ci, w, h, S}, sx[3] = {ci * 2, w * ci * 2, h * w * ci * 2};
+        uint32_t bf[4] = {64, (uint32_t)kTileW, (uint32_t)kTileH, 1}, bw[4] = {64, (uint32_t)kChunkW, (uint32_t)kChunkH, 1};
+        ok = ok && make_map(&P->x_fwd3, b.x, 4, dx, sx, bf, err, err_len, "features (3x3 forward)");
+        ok = ok && make_map(&P->x_wg3, b.x, 4, dx, sx, bw, err, err_len, "features (3x3 wgrad)");
+        uint64_t dh[4] = {ch, w, h, S}, sh[3] = {ch * 2, w * ch * 2, h * w * ch * 2};
+        ok = ok && make_map(&P->dh_wg3, b.dhidden, 4, dh, sh, bw, err, err_len, "hidden gradient");
+        uint64_t dw[3] = {ci, 9 * ch, S}, sw[2] = {ci * 2, 9 * ch * ci * 2};
+        uint32_t bwt[3] = {64, (uint32_t)b.c_hidden, 1};
+        ok = ok && make_map(&P->w1_map, b.w1, 3, dw, sw, bwt, err, err_len, "3x3 weight");
+    }
+    if (!ok) { delete P; return nullptr; }
+
+    const int m_last = (P->c_last + kTileM - 1) / kTileM;
+    P->chunks2 = (P->p + kChunkPix - 1) / kChunkPix;
+    split_geometry(P->chunks2, 148, &P->per2, &P->split2);
+    P->cols2 = pow2_cols(m_last * kClassPad);
+    P->smem_fwd1 = (size_t)(P->c_last / kBlockK) * (kTileM * 128 + kClassPad * 128) + kSmemAlign;
+    P->smem_wg1 = 3 * ((size_t)m_last * 2 * kChunkPix * 128 + kClassPad * 128) + kSmemAlign;
+    if (b.c_hidden) {
+        const int m_in = (b.c_in + kTileM - 1) / kTileM;
+        P->chunks1 = ((b.w + kChunkW - 1) / kChunkW) * ((b.h + kChunkH - 1) / kChunkH);
+        split_geometry(P->chunks1, 148 / 9, &P->per1, &P->split1);
+        P->cols1 = pow2_cols(m_in * b.c_hidden);
+        P->smem_fwd3 = 4 * ((size_t)kTileM * 128 + (size_t)b.c_hidden * 128) + kSmemAlign;
+        P->smem_wg3 = 3 * ((size_t)(m_in * 2 + b.c_hidden / kBlockK) * kChunkPix * 128) + kSmemAlign;
+        P->smem_dgrad = ((size_t)b.C * b.c_hidden + (size_t)b.C * kDgradPix + 512) * sizeof(float);
+        if (P->cols1 > 512) {
+            snprintf(err, err_len, "c_in %d with c_hidden %d needs %d TMEM columns (> 512)", b.c_in, b.c_hidden, P->cols1);
+            delete P; return nullptr;
+        }
+    }
+    const size_t lim = 227 * 1024;
+    if (P->c_last / kBlockK > kMaxKBlocks || P->smem_fwd1 > lim || P->smem_wg1 > lim || P->smem_fwd3 > lim ||
+        P->smem_wg3 > lim || P->smem_dgrad > lim) {
+        snprintf(err, err_len, "shared memory per block exceeds 227 KB for these channel counts");
+        delete P; return nullptr;
+    }
+    cudaError_t e = cudaFuncSetAttribute(tc_fwd1x1_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)P->smem_fwd1);
+    if (e == cudaSuccess) e = cudaFuncSetAttribute(tc_wgrad1x1_kernel<3>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)P->smem_wg1);
+    if (b.c_hidden) {
+        if (e == cudaSuccess) e = cudaFuncSetAttribute(tc_fwd3x3_kernel<4>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)P->smem_fwd3);
+        if (e == cudaSuccess) e = cudaFuncSetAttribute(tc_wgrad3x3_kernel<3>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)P->smem_wg3);
+        if (e == cudaSuccess) e = cudaFuncSetAttribute(dgrad_relu_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)P->smem_dgrad);
+    }
+    if (e != cudaSuccess) { snprintf(err, err_len, "shared-memory attribute: %s", cudaGetErrorString(e)); delete P; return nullptr; }
+    return P;
+}
+
+void tc_plan_destroy(TcPlan* P) { delete P; }
+
+int tc_forward(const TcPlan* P, cudaStream_t s)
+{
+    const TcBuffers& b = P->b;
+    int n = 0;
+    if (b.c_hidden) {
+        const int tiles = ((b.w + kTileW - 1) / kTileW) * ((b.h + kTileH - 1) / kTileH);
+        tc_fwd3x3_kernel<4><<<dim3(tiles, b.S), kThreadsTc, P->smem_fwd3, s>>>(
+            P->x_fwd3, P->w1_map, b.theta, b.n_params, b.b1_off, b.hidden, b.c_in, b.c_hidden, b.h, b.w,
+            pow2_cols(b.c_hidden), b.err);
+        ++n;
+    }
+    const int tiles1 = (P->p + kTileM - 1) / kTileM;
+    tc_fwd1x1_kernel<<<dim3(tiles1, b.S), kThreadsTc, P->smem_fwd1, s>>>(
+        P->act_fwd, P->w2_map, b.theta, b.n_params, b.b2_off, b.z, b.C, P->p, P->c_last / kBlockK, b.err);
+    return n + 1;
+}
+
+int tc_backward(const TcPlan* P, cudaStream_t s)
+{
+    const TcBuffers& b = P->b;
+    int n = 0;
+    tc_wgrad1x1_kernel<3><<<dim3(P->split2, b.S), kThreadsTc, P->smem_wg1, s>>>(
+        P->act_wg, P->dz_map, b.w2_partials, P->c_last, P->chunks2, P->per2, P->cols2, b.err);
+    ++n;
+    if (b.c_hidden) {
+        const int blocks = tc_b1_partials(b.h, b.w);
+        dgrad_relu_kernel<<<dim3(blocks, b.S), 256, P->smem_dgrad, s>>>(
+            b.theta, b.n_params, b.w2_off, b.dz, b.hidden, b.dhidden, b.b1_partials, b.C, b.c_hidden, P->p);
+        tc_wgrad3x3_kernel<3><<<dim3(9 * P->split1, b.S), kThreadsTc, P->smem_wg3, s>>>(
+            P->x_wg3, P->dh_wg3, b.w1_partials, b.c_in, b.c_hidden, b.h, b.w, P->chunks1, P->per1, P->split1,
+            P->cols1, b.err);
+        n += 2;
+    }
+    return n;
+}
+
+}  // namespace st

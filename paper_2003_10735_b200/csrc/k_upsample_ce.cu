@@ -225,7 +225,7 @@ upsample_ce_kernel(UpsampleCeArgs a, int chunk)
                 const int c = c0 + cc;
                 a.dz[((int64_t)s * C + c) * p + (int64_t)y * w + x] = v;
                 if (a.dz_bf16)
-                    a.dz_bf16[((int64_t)s * kClassPad + c) * p + (int64_t)y * w + x] = __float2bfloat16_rn(v);
+                    a.dz_bf16[((int64_t)s * kClassPad + c) * a.dz_bf16_pitch + (int64_t)y * w + x] = __float2bfloat16_rn(v);
             }
             dzt[idx] = v;
         }

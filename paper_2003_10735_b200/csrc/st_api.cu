@@ -35,6 +35,7 @@ struct st_ctx {
     uint8_t* labels = nullptr;
     float *z = nullptr, *dz = nullptr;
     bf16* dz_bf16 = nullptr;
+    int64_t dz_pitch = 0;
     float *hid_f32 = nullptr, *dhid_f32 = nullptr;
     bf16 *hid_bf16 = nullptr, *dhid_bf16 = nullptr;
     bf16 *w1_shadow = nullptr, *w2_shadow = nullptr;
@@ -44,7 +45,7 @@ struct st_ctx {
     int n_k3_blocks = 0;
     float* loss_buf = nullptr;              // [S][kMaxSteps]
     unsigned long long* conf_buf = nullptr; // [S][kMaxSteps][C][C], allocated on first use
-    unsigned int* bad = nullptr;            // [2]: labels >= C met by a step / by st_agreement
+    unsigned int* bad = nullptr;            // [3]: labels >= C met by a step / by st_agreement; [2] = first device wait that gave up
     uint8_t* mask_tmp = nullptr;            // [P]
     uint8_t* mask_tmp2 = nullptr;           // [P]
     unsigned long long* conf_tmp = nullptr; // [C][C]
@@ -209,6 +210,7 @@ st_status enqueue_step(st_ctx* c, int slot, bool want_conf)
 
     UpsampleCeArgs k3;
     k3.z = c->z; k3.labels = c->labels; k3.dz = c->dz; k3.dz_bf16 = c->bf16_mode ? c->dz_bf16 : nullptr;
+    k3.dz_bf16_pitch = c->dz_pitch;
     k3.loss_part = c->loss_part; k3.db_part = c->db_part;
     k3.conf = want_conf ? c->conf_buf + (int64_t)slot * c->C * c->C : nullptr;
     k3.conf_stream_stride = (int64_t)kMaxSteps * c->C * c->C;
@@ -246,9 +248,16 @@ st_status enqueue_step(st_ctx* c, int slot, bool want_conf)
 
 st_status report_bad_labels(st_ctx* c, int which, const char* what)
 {
-    unsigned int host_bad[2] = {0, 0};
+    unsigned int host_bad[4] = {0, 0, 0, 0};
     ST_CUDA(c, cudaMemcpyAsync(host_bad, c->bad, sizeof host_bad, cudaMemcpyDeviceToHost, c->stream));
     ST_CUDA(c, cudaStreamSynchronize(c->stream));
+    if (host_bad[2]) {
+        unsigned int zero = 0;
+        cudaMemcpyAsync(c->bad + 2, &zero, sizeof zero, cudaMemcpyHostToDevice, c->stream);
+        cudaStreamSynchronize(c->stream);
+        return fail(c, ST_ERR_CUDA, "a tensor-core kernel gave up waiting (code %u, block %u); results of that step are invalid",
+                    host_bad[2] & 0xffu, host_bad[2] >> 8);
+    }
     if (host_bad[which]) {
         unsigned int zero = 0;
         cudaMemcpyAsync(c->bad + which, &zero, sizeof zero, cudaMemcpyHostToDevice, c->stream);
@@ -361,10 +370,11 @@ st_status st_init_head(const st_head_desc* desc, const float* init_params, st_ct
     ALLOC(z, S * c->C * c->p); ALLOC(dz, S * c->C * c->p);
     ALLOC(loss_part, S * c->n_k3_blocks); ALLOC(db_part, (size_t)S * c->n_k3_blocks * c->C);
     ALLOC(loss_buf, S * kMaxSteps);
-    ALLOC(bad, 2); ALLOC(mask_tmp, c->P); ALLOC(mask_tmp2, c->P); ALLOC(conf_tmp, c->C * c->C); ALLOC(miou_tmp, 1);
+    ALLOC(bad, 4); ALLOC(mask_tmp, c->P); ALLOC(mask_tmp2, c->P); ALLOC(conf_tmp, c->C * c->C); ALLOC(miou_tmp, 1);
     if (c->bf16_mode) {
         ALLOC(x_bf16, S * c->p * c->Cin);
-        ALLOC(dz_bf16, (size_t)S * kClassPad * c->p);
+        c->dz_pitch = tc_dz_pitch(c->h, c->w);
+        ALLOC(dz_bf16, (size_t)S * kClassPad * c->dz_pitch);
         ALLOC(w2_shadow, (size_t)S * kClassPad * c_last);
         c->n_split2 = tc_wgrad_splits(2, c->Cin, c->Ch, c->h, c->w);
         ALLOC(w2_partials, (size_t)S * c->n_split2 * kClassPad * c_last);
@@ -400,7 +410,8 @@ st_status st_init_head(const st_head_desc* desc, const float* init_params, st_ct
         memset(&b, 0, sizeof b);
         b.S = S; b.c_in = c->Cin; b.c_hidden = c->Ch; b.C = c->C; b.h = c->h; b.w = c->w;
         b.x = c->x_bf16; b.w1 = c->w1_shadow; b.w2 = c->w2_shadow; b.theta = c->theta; b.n_params = c->n_params;
-        b.b1_off = c->Ch ? L.b_off[0] : 0; b.b2_off = L.b_off[L.n_layers - 1];
+        b.b1_off = c->Ch ? L.b_off[0] : 0; b.b2_off = L.b_off[L.n_layers - 1]; b.w2_off = L.w_off[L.n_layers - 1];
+        b.err = c->bad + 2;
         b.z = c->z; b.hidden = c->hid_bf16; b.dz = c->dz; b.dz_bf16 = c->dz_bf16; b.dhidden = c->dhid_bf16;
         b.w1_partials = c->w1_partials; b.w2_partials = c->w2_partials; b.b1_partials = c->b1_partials;
         char msg[256] = {0};

@@ -32,7 +32,8 @@ struct UpsampleCeArgs {
     const float* z;          // [S][C][h][w]
     const uint8_t* labels;   // [S][H][W]
     float* dz;               // [S][C][h][w]     gradient of the mean loss
-    bf16* dz_bf16;           // [S][kClassPad][p] or nullptr (rows >= C untouched)
+    bf16* dz_bf16;           // [S][kClassPad][dz_bf16_pitch] or nullptr (rows >= C untouched)
+    int64_t dz_bf16_pitch;
     float* loss_part;        // [S][n_blocks]    per-block partial sums of per-pixel losses
     float* db_part;          // [S][n_blocks][C] per-block partial sums of dz over the block's pixels
     unsigned long long* conf;// nullptr, or int64 [C][C] per stream: confusion of label vs argmax of the upsampled logits
@@ -108,19 +109,21 @@ struct TcBuffers {
     const bf16* w1;       // [S][9][c_hidden][c_in]  (two-layer head) bf16 copy of the 3x3 weight
     const bf16* w2;       // [S][kClassPad][c_last]  bf16 copy of the 1x1 weight, rows >= C zero
     const float* theta;   // [S][n_params]    biases are read from the master parameters
-    int64_t n_params, b1_off, b2_off;
+    int64_t n_params, b1_off, b2_off, w2_off;
     float* z;             // [S][C][p]
     bf16* hidden;         // [S][p][c_hidden]
     const float* dz;      // [S][C][p]
-    const bf16* dz_bf16;  // [S][kClassPad][p]
+    const bf16* dz_bf16;  // [S][kClassPad][tc_dz_pitch]
     bf16* dhidden;        // [S][p][c_hidden]
     float* w1_partials;   // [S][n_split1][9][c_hidden][c_in]
     float* w2_partials;   // [S][n_split2][kClassPad][c_last]
     float* b1_partials;   // [S][n_b1part][c_hidden]
+    unsigned int* err;    // device word: first wait that gave up (0 = none)
 };
 // Geometry is fixed by the shapes alone, so scratch can be sized before the plan exists.
 int tc_wgrad_splits(int layer /*1: 3x3, 2: 1x1*/, int c_in, int c_hidden, int h, int w);
 int tc_b1_partials(int h, int w);
+int tc_dz_pitch(int h, int w);      // row pitch (elements) of the bf16 logit gradient [S][kClassPad][pitch]
 TcPlan* tc_plan_create(const TcBuffers& b, char* err, size_t err_len);
 void tc_plan_destroy(TcPlan*);
 int tc_forward(const TcPlan*, cudaStream_t s);    // returns the number of kernels launched
