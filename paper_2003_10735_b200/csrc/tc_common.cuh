@@ -11,7 +11,7 @@ namespace tc {
 
 // A wait that does not complete within this many polls gives up: the kernel records an error code
 // and every role falls through to the common teardown (TMEM is freed, the kernel returns).
-constexpr uint32_t kSpinLimit = 1u << 22;
+constexpr uint32_t kSpinLimit = 1u << 20;
 
 enum WaitCode : unsigned int { kWaitFull = 1, kWaitEmpty = 2, kWaitDone = 3 };
 

@@ -1,0 +1,240 @@
+"""GPU parity of the bf16 tensor-core path (gemm_precision 1) against the CPU oracle.
+
+Two comparisons are made.  Against the plain fp32 oracle with the stated tolerances (loss 1e-4
+relative; weights 2e-2 max relative / 1e-3 mean absolute; update vector 2e-2 relative L2), and
+against the oracle with its GEMM operands rounded to bf16 at the same places, where the
+remaining difference is accumulation order only and the tolerance is much tighter."""
+import numpy as np
+import pytest
+
+import oracle
+import synth_inputs as si
+import paper_2003_10735_b200 as st
+
+pytestmark = pytest.mark.gpu
+torch = pytest.importorskip("torch")
+
+
+@pytest.fixture(autouse=True)
+def side_stream():
+    s = torch.cuda.Stream()
+    with torch.cuda.stream(s):
+        yield s
+    s.synchronize()
+
+
+def dev(a):
+    return torch.from_numpy(np.ascontiguousarray(a)).cuda()
+
+
+def make_ctx(c_in, ch, C, h, w, theta, S=1, lr=0.01, mu=0.0, prec=1):
+    return st.st_init_head(n_streams=S, c_in=c_in, c_hidden=ch, n_classes=C, feat_h=h, feat_w=w,
+                           gemm_precision=prec, lr=lr, momentum=mu,
+                           cuda_stream=torch.cuda.current_stream().cuda_stream, init_params=theta)
+
+
+def packed(ctx, stream=0):
+    out = np.empty(ctx.n_params, np.float32)
+    st.st_pack_updated_params(ctx, stream, out)
+    return out
+
+
+def problem(seed, c_in, C, h, w):
+    rng = np.random.default_rng(seed)
+    feat = np.maximum(rng.standard_normal((c_in, h, w)), 0).astype(np.float32)
+    cfg = si.WorkloadConfig("t", c_in, 0, C, h, w, n_regions=max(4, C), teacher="onehot_noise")
+    return feat, si.teacher_logits(cfg, stream=seed)
+
+
+def rel_l2(a, b):
+    return float(np.linalg.norm(a.astype(np.float64) - b) / max(np.linalg.norm(b), 1e-30))
+
+
+def check_weights(got, ref, theta0, c_in, ch, C, max_rel=2e-2, mean_abs=1e-3, upd_rel=2e-2):
+    off = 0
+    for ws, bs in oracle.param_shapes(c_in, ch, C):
+        for n in (int(np.prod(ws)), int(np.prod(bs))):
+            g, r = got[off:off + n], ref[off:off + n]
+            assert np.abs(g - r).max() / max(np.abs(r).max(), 1e-6) <= max_rel
+            off += n
+    assert np.abs(got - ref).mean() <= mean_abs
+    r = rel_l2(got - theta0, ref.astype(np.float64) - theta0)
+    assert r <= upd_rel, r
+    return r
+
+
+@pytest.mark.parametrize("c_in,h,w", [(64, 5, 7), (256, 12, 20)])
+def test_feature_cache_rounds_to_nearest_even(c_in, h, w):
+    feat, _ = problem(1, c_in, 3, h, w)
+    feat[0, 0, :4] = [1.00390625, 1.01171875, -1.00390625, 3.0e-39]     # ties and a denormal
+    ctx = make_ctx(c_in, 0, 3, h, w, np.zeros(st.st_param_count(c_in, 0, 3), np.float32))
+    st.st_set_frozen_features(ctx, 0, dev(feat))
+    got = st.st_read_tensor(ctx, 0, st.ST_TENSOR_FEATURES)
+    np.testing.assert_array_equal(got, oracle.round_bf16(feat).ravel())
+    st.st_destroy(ctx)
+
+
+@pytest.mark.parametrize("c_in,C,h,w", [
+    (64, 5, 9, 13),      # fewer pixels than one 128-pixel tile, ragged chunk
+    (128, 21, 24, 40),   # several tiles and a half one
+    (256, 32, 17, 31),   # all 32 class rows in use, two channel accumulators
+    (192, 2, 8, 8),      # channel count that is not a multiple of 128
+])
+def test_1x1_head_single_step_intermediates(c_in, C, h, w):
+    feat, T = problem(3, c_in, C, h, w)
+    theta = si.initial_head_params(c_in, 0, C, 5)
+    theta[-C:] = np.linspace(-0.5, 0.5, C)                        # non-zero biases
+    ctx = make_ctx(c_in, 0, C, h, w, theta, lr=0.05)
+    st.st_set_frozen_features(ctx, 0, dev(feat))
+    st.st_teacher_labels(ctx, 0, dev(T))
+    loss = np.zeros(1, np.float32)
+    st.st_distill_step(ctx, 1, loss)
+    lab = oracle.teacher_labels(T)
+    hq = oracle.Head(c_in, 0, C, lr=0.05, theta=theta, quantize_bf16=True)
+    z_ref, _ = oracle.head_forward(hq, feat)
+    z = st.st_read_tensor(ctx, 0, st.ST_TENSOR_LOGITS)
+    np.testing.assert_allclose(z, z_ref.ravel(), rtol=2e-5, atol=2e-5)        # same bf16 operands, fp32 accumulation
+    l_ref, g_ref, _ = oracle.gradients(hq, feat, lab)
+    assert abs(loss[0] - l_ref) <= 2e-5 * abs(l_ref)
+    g = st.st_read_tensor(ctx, 0, st.ST_TENSOR_PARAM_GRAD)
+    assert rel_l2(g, g_ref) <= 2e-3
+    assert np.abs(g - g_ref).max() <= 2e-3 * np.abs(g_ref).max()
+    # against the plain fp32 oracle: stated tolerances
+    hp = oracle.Head(c_in, 0, C, lr=0.05, theta=theta)
+    l_plain, _ = oracle.distill_step(hp, feat, lab)
+    assert abs(loss[0] - l_plain) <= 1e-4 * abs(l_plain) + 0  # loss: 1e-4 relative
+    check_weights(packed(ctx), hp.theta, theta, c_in, 0, C)
+    st.st_destroy(ctx)
+
+
+@pytest.mark.parametrize("c_in,ch,C,h,w", [
+    (64, 64, 5, 10, 37),      # ragged tile in x and y, one accumulator
+    (128, 128, 21, 9, 33),
+    (256, 256, 19, 6, 70),    # the full channel counts of the two-layer workloads, all of TMEM
+    (64, 192, 3, 4, 4),
+])
+def test_two_layer_head_single_step_intermediates(c_in, ch, C, h, w):
+    feat, T = problem(4, c_in, C, h, w)
+    theta = si.initial_head_params(c_in, ch, C, 6)
+    nb1 = ch * c_in * 9
+    theta[nb1:nb1 + ch] = np.linspace(-0.2, 0.3, ch)
+    ctx = make_ctx(c_in, ch, C, h, w, theta, lr=0.02)
+    st.st_set_frozen_features(ctx, 0, dev(feat))
+    st.st_teacher_labels(ctx, 0, dev(T))
+    loss = np.zeros(1, np.float32)
+    st.st_distill_step(ctx, 1, loss)
+    lab = oracle.teacher_labels(T)
+    hq = oracle.Head(c_in, ch, C, lr=0.02, theta=theta, quantize_bf16=True)
+    z_ref, hd_ref = oracle.head_forward(hq, feat)
+    hd = st.st_read_tensor(ctx, 0, st.ST_TENSOR_HIDDEN)
+    # bf16 outputs of fp32 sums in different orders: at most one bf16 ulp apart, and rarely
+    d = np.abs(hd - hd_ref.ravel())
+    assert (d <= 2.0 ** -7 * np.maximum(np.abs(hd_ref.ravel()), 1e-3)).all()
+    assert (d > 0).mean() < 0.02
+    z = st.st_read_tensor(ctx, 0, st.ST_TENSOR_LOGITS)
+    np.testing.assert_allclose(z, z_ref.ravel(), rtol=1e-3, atol=1e-3)
+    l_ref, g_ref, _ = oracle.gradients(hq, feat, lab)
+    assert abs(loss[0] - l_ref) <= 1e-4 * abs(l_ref)
+    g = st.st_read_tensor(ctx, 0, st.ST_TENSOR_PARAM_GRAD)
+    off = 0
+    for ws, bs in oracle.param_shapes(c_in, ch, C):
+        for n in (int(np.prod(ws)), int(np.prod(bs))):
+            assert rel_l2(g[off:off + n], g_ref[off:off + n]) <= 1e-2, (off, n)
+            off += n
+    hp = oracle.Head(c_in, ch, C, lr=0.02, theta=theta)
+    l_plain, _ = oracle.distill_step(hp, feat, lab)
+    assert abs(loss[0] - l_plain) <= 1e-4 * abs(l_plain)
+    check_weights(packed(ctx), hp.theta, theta, c_in, ch, C)
+    st.st_destroy(ctx)
+
+
+def test_hidden_gradient_and_relu_mask():
+    c_in, ch, C, h, w = 64, 64, 4, 7, 9
+    feat, T = problem(8, c_in, C, h, w)
+    theta = si.initial_head_params(c_in, ch, C, 2)
+    ctx = make_ctx(c_in, ch, C, h, w, theta)
+    st.st_set_frozen_features(ctx, 0, dev(feat)); st.st_teacher_labels(ctx, 0, dev(T))
+    st.st_distill_step(ctx, 1)
+    hd = st.st_read_tensor(ctx, 0, st.ST_TENSOR_HIDDEN).reshape(ch, h, w)
+    dz = st.st_read_tensor(ctx, 0, st.ST_TENSOR_LOGIT_GRAD).reshape(C, h, w)
+    dh = st.st_read_tensor(ctx, 0, st.ST_TENSOR_HIDDEN_GRAD).reshape(ch, h, w)
+    W2 = theta[ch * c_in * 9 + ch: ch * c_in * 9 + ch + C * ch].reshape(C, ch)
+    ref = oracle.conv1x1_dgrad(W2, dz)
+    oracle.relu_mask_(ref, np.ascontiguousarray(hd))
+    assert (dh[hd <= 0] == 0).all()
+    np.testing.assert_allclose(dh, oracle.round_bf16(ref), rtol=2.0 ** -7, atol=1e-12)
+    st.st_destroy(ctx)
+
+
+def test_config2_720p_full_size_k8():
+    cfg = si.get_config(2)
+    feat, T, theta = si.stream_inputs(cfg)
+    ctx = make_ctx(cfg.c_in, 0, cfg.n_classes, cfg.feat_h, cfg.feat_w, theta, lr=cfg.lr, mu=cfg.momentum)
+    st.st_set_frozen_features(ctx, 0, dev(feat))
+    labels = torch.empty((cfg.frame_h, cfg.frame_w), dtype=torch.uint8, device="cuda")
+    st.st_teacher_labels(ctx, 0, dev(T), labels)
+    K = cfg.k_steps
+    loss = torch.zeros(K, dtype=torch.float32, device="cuda")
+    conf = torch.zeros((K, cfg.n_classes, cfg.n_classes), dtype=torch.int64, device="cuda")
+    st.st_distill_step(ctx, K, loss, conf)
+    lab = oracle.teacher_labels(T)
+    np.testing.assert_array_equal(labels.cpu().numpy(), lab)                   # bit-exact labels
+    head = oracle.Head(cfg.c_in, 0, cfg.n_classes, lr=cfg.lr, momentum=cfg.momentum, theta=theta)
+    ref_loss, masks = [], []
+    for _ in range(K):
+        l, m = oracle.distill_step(head, feat, lab)
+        ref_loss.append(l); masks.append(m)
+    np.testing.assert_allclose(loss.cpu().numpy(), ref_loss, rtol=1e-4)         # loss: 1e-4 relative
+    raw = packed(ctx)
+    assert raw.nbytes == 21588                                                  # 256*21 weights + 21 biases
+    check_weights(raw, head.theta, theta, cfg.c_in, 0, cfg.n_classes)
+    # per-step fused confusion: totals exact, cells within the near-tie budget of the student mask
+    c = conf.cpu().numpy()
+    for k in range(K):
+        assert c[k].sum() == lab.size
+        np.testing.assert_array_equal(c[k].sum(1), np.bincount(lab.ravel(), minlength=cfg.n_classes))
+        ref_c, _, _ = oracle.agreement(lab, masks[k], cfg.n_classes)
+        assert np.abs(c[k] - ref_c).sum() <= 2 * lab.size // 500
+    # agreement from the GPU's own mask is bit-exact with the oracle's count of that mask
+    mask = torch.empty_like(labels)
+    st.st_student_mask(ctx, 0, mask)
+    gconf = np.zeros((cfg.n_classes,) * 2, np.int64)
+    m = st.st_agreement(ctx, 0, None, None, gconf)
+    oconf, om, _ = oracle.agreement(lab, mask.cpu().numpy(), cfg.n_classes)
+    np.testing.assert_array_equal(gconf, oconf)
+    assert m == om
+    st.st_destroy(ctx)
+
+
+def test_three_streams_grouped_launch():
+    c_in, C, h, w = 64, 6, 11, 19
+    S = 3
+    probs = [problem(40 + s, c_in, C, h, w) for s in range(S)]
+    thetas = [si.initial_head_params(c_in, 0, C, 50 + s) for s in range(S)]
+    ctx = make_ctx(c_in, 0, C, h, w, np.concatenate(thetas), S=S, lr=0.05, mu=0.9)
+    for s in range(S):
+        st.st_set_frozen_features(ctx, s, dev(probs[s][0]))
+        st.st_teacher_labels(ctx, s, dev(probs[s][1]))
+    loss = torch.zeros((S, 4), dtype=torch.float32, device="cuda")
+    st.st_distill_step(ctx, 4, loss)
+    for s in range(S):
+        head = oracle.Head(c_in, 0, C, lr=0.05, momentum=0.9, theta=thetas[s])
+        lab = oracle.teacher_labels(probs[s][1])
+        ref = [oracle.distill_step(head, probs[s][0], lab)[0] for _ in range(4)]
+        np.testing.assert_allclose(loss[s].cpu().numpy(), ref, rtol=1e-4)
+        check_weights(packed(ctx, s), head.theta, thetas[s], c_in, 0, C)
+    st.st_destroy(ctx)
+
+
+def test_bf16_steps_are_bit_reproducible():
+    c_in, ch, C, h, w = 64, 64, 5, 9, 35
+    feat, T = problem(9, c_in, C, h, w)
+    theta = si.initial_head_params(c_in, ch, C, 2)
+    outs = []
+    for _ in range(2):
+        ctx = make_ctx(c_in, ch, C, h, w, theta, lr=0.02, mu=0.9)
+        st.st_set_frozen_features(ctx, 0, dev(feat)); st.st_teacher_labels(ctx, 0, dev(T))
+        st.st_distill_step(ctx, 3)
+        outs.append(packed(ctx))
+        st.st_destroy(ctx)
+    assert outs[0].tobytes() == outs[1].tobytes()
