@@ -1,0 +1,403 @@
+#!/usr/bin/env python
+"""Benchmark of the key-frame partial-distillation step on B200.
+
+One bench "step" is one pass of the whole hot path over one synthetic 720p key frame:
+cache the frozen features, reduce the teacher logits to labels, K = 8 SGD iterations of the
+head, pack the updated parameters, and measure student/teacher agreement.  The reported
+metric counts SGD iterations per second (8 per bench step), whole job, all GPUs.
+
+    python bench.py --gpus 1 --steps 2000 --warmup 10
+    python -m torch.distributed.run --nnodes=1 --nproc-per-node N ... bench.py --gpus N ...
+    python bench.py --impl reference        # the CPU oracle, timed on the host cores
+
+Every rank prints nothing except rank 0, which prints ONE JSON line.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import statistics
+import subprocess
+import sys
+import tempfile
+import time
+
+import numpy as np
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+sys.path.insert(0, ROOT)
+
+import synth_inputs as si  # noqa: E402
+
+METRIC = "720p key-frame partial-distill steps/s (K=8)"
+N_SETS = 4            # distinct key frames the device-resident run rotates over (4 x 136 MB > 126 MB L2)
+ALU_FLOP_PER_CLASS_PIXEL = 20.0   # algorithmic fp32 work of the fused upsample+CE kernel (10 FMA-equivalents)
+
+
+def read_peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        with open(path) as f:
+            p = json.load(f)
+        return {"hbm_gbs": float(p["hbm_gbs"]), "bf16_tflops": float(p["bf16_tflops"]),
+                "bf16_tflops_sustained": float(p.get("bf16_tflops_sustained", p["bf16_tflops"])),
+                "sm_max_mhz": float(p.get("sm_max_mhz", 1965.0)), "source": "measured"}
+    return {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0, "sm_max_mhz": 1965.0,
+            "source": "fallback"}
+
+
+# --------------------------------------------------------------------------------------------
+# clocks
+# --------------------------------------------------------------------------------------------
+class ClockSampler:
+    FIELDS = ("timestamp,index,clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,"
+              "clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
+              "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, gpu_index: int):
+        self.path = tempfile.NamedTemporaryFile(prefix="st_clocks_", suffix=".csv", delete=False).name
+        self.proc = None
+        try:
+            self.proc = subprocess.Popen(
+                ["nvidia-smi", "-i", str(gpu_index), f"--query-gpu={self.FIELDS}", "--format=csv,noheader,nounits",
+                 "-lms", "100"], stdout=open(self.path, "w"), stderr=subprocess.DEVNULL)
+        except OSError:
+            self.proc = None
+        self.t0 = self.t1 = None
+
+    def begin(self):
+        self.t0 = time.time()
+
+    def end(self):
+        self.t1 = time.time()
+
+    def finish(self):
+        if self.proc is None:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"], "samples": 0}
+        time.sleep(0.25)
+        self.proc.terminate()
+        try:
+            self.proc.wait(timeout=5)
+        except Exception:
+            self.proc.kill()
+        rows = []
+        import datetime
+        with open(self.path) as f:
+            for line in f:
+                parts = [x.strip() for x in line.split(",")]
+                if len(parts) < 10:
+                    continue
+                try:
+                    ts = datetime.datetime.strptime(parts[0], "%Y/%m/%d %H:%M:%S.%f").timestamp()
+                    rows.append((ts, float(parts[2]), float(parts[3]), parts[6:10]))
+                except ValueError:
+                    continue
+        try:
+            os.unlink(self.path)
+        except OSError:
+            pass
+        inside = [r for r in rows if self.t0 - 0.05 <= r[0] <= self.t1 + 0.05] or rows[-3:]
+        if not inside:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["no samples"], "samples": 0}
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        reasons = sorted({n for r in inside for n, v in zip(names, r[3]) if v.lower().startswith("active")})
+        return {"sm_mhz": statistics.median(r[1] for r in inside), "sm_max_mhz": inside[0][2],
+                "reasons": reasons, "samples": len(inside)}
+
+
+# --------------------------------------------------------------------------------------------
+# the CPU oracle, timed (cpu_baseline leg and --impl reference)
+# --------------------------------------------------------------------------------------------
+def oracle_key_frame(cfg, feat, T, theta, rows=None):
+    """One key frame through the oracle as it stands; returns seconds.  `rows` crops the feature map
+    to its first `rows` rows (and the frame to 4*rows) for a bounded sample."""
+    import oracle
+    if rows is not None:
+        feat = np.ascontiguousarray(feat[:, :rows])
+        T = np.ascontiguousarray(T[:, :rows * cfg.up])
+    t0 = time.perf_counter()
+    labels = oracle.teacher_labels(T)
+    head = oracle.Head(cfg.c_in, cfg.c_hidden, cfg.n_classes, up=cfg.up, lr=cfg.lr, momentum=cfg.momentum, theta=theta)
+    for _ in range(cfg.k_steps):
+        oracle.distill_step(head, feat, labels)
+    oracle.pack(head)
+    oracle.agreement(labels, oracle.student_mask(head, feat), cfg.n_classes)
+    return time.perf_counter() - t0
+
+
+def host_cores():
+    try:
+        return len(os.sched_getaffinity(0))
+    except AttributeError:
+        return os.cpu_count() or 1
+
+
+def run_reference(args, cfg):
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    import oracle
+    oracle.build()
+    feat, T, theta = si.stream_inputs(cfg)
+    # calibrate on a thin band, then size the per-step sample so that the whole run stays within ~3 minutes
+    t_band = oracle_key_frame(cfg, feat, T, theta, rows=4)
+    per_row = t_band / 4
+    budget = 150.0 / max(1, args.steps + args.warmup)
+    rows = int(max(4, min(cfg.feat_h, budget / max(per_row, 1e-9))))
+    for _ in range(args.warmup):
+        oracle_key_frame(cfg, feat, T, theta, rows=rows)
+    t0 = time.perf_counter()
+    for _ in range(args.steps):
+        oracle_key_frame(cfg, feat, T, theta, rows=rows)
+    dt = time.perf_counter() - t0
+    frac = rows / cfg.feat_h
+    key_frames_per_s = args.steps / dt * frac          # scaled to the full frame by pixel count
+    value = key_frames_per_s * cfg.k_steps
+    sample = f"{rows} of {cfg.feat_h} feature rows per step, scaled to the full frame by pixel count"
+    line = {
+        "impl": "reference", "metric": METRIC, "value": value, "unit": "steps/s", "n_gpus": args.gpus,
+        "steps": args.steps, "warmup": args.warmup, "ms_per_step": dt / args.steps * 1e3 / frac,
+        "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f32", "data": "synthetic",
+        "config": {"workload": cfg.name, "k_steps": cfg.k_steps, "frame": [cfg.frame_h, cfg.frame_w]},
+        "cpu_baseline": {"value": value, "unit": "steps/s", "cores": host_cores(), "kind": "oracle", "sample": sample},
+        "e2e": {"value": value, "unit": "steps/s", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+        "gpu_launches": 0,
+    }
+    print(json.dumps(line), flush=True)
+
+
+# --------------------------------------------------------------------------------------------
+# the CUDA path
+# --------------------------------------------------------------------------------------------
+def run_ours(args, cfg):
+    import torch
+    import paper_2003_10735_b200 as st
+
+    rank = int(os.environ.get("RANK", "0"))
+    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    dist = None
+    if world > 1:
+        import torch.distributed as dist
+        os.environ.setdefault("MASTER_ADDR", "127.0.0.1")
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local_rank))
+    torch.cuda.set_device(local_rank)
+    stream = torch.cuda.Stream()
+    peaks = read_peaks()
+    S, C, K = cfg.n_streams, cfg.n_classes, cfg.k_steps
+    H, W, p, P = cfg.frame_h, cfg.frame_w, cfg.feat_h * cfg.feat_w, cfg.frame_h * cfg.frame_w
+
+    with torch.cuda.stream(stream):
+        # ---- seeded synthetic inputs (each rank its own streams: the path shards by stream, no exchange)
+        feats_h, logits_h, thetas = [], [], []
+        for i in range(N_SETS):
+            per_stream_f, per_stream_t = [], []
+            for s in range(S):
+                f = si.frozen_features(cfg.c_in, cfg.feat_h, cfg.feat_w, seed=1000 * rank + 10 * i + s)
+                t = si.teacher_logits(cfg, stream=100 * rank + s, frame=i)
+                per_stream_f.append(torch.from_numpy(f).pin_memory())
+                per_stream_t.append(torch.from_numpy(t).pin_memory())
+            feats_h.append(per_stream_f)
+            logits_h.append(per_stream_t)
+        for s in range(S):
+            thetas.append(si.initial_head_params(cfg.c_in, cfg.c_hidden, C, 1000 + s))
+        theta0 = np.concatenate(thetas)
+        feats_d = [[f.cuda(non_blocking=True) for f in fs] for fs in feats_h]
+        logits_d = [[t.cuda(non_blocking=True) for t in ts] for ts in logits_h]
+        ctx = st.st_init_head(n_streams=S, c_in=cfg.c_in, c_hidden=cfg.c_hidden, n_classes=C, feat_h=cfg.feat_h,
+                              feat_w=cfg.feat_w, gemm_precision=cfg.gemm_precision, lr=cfg.lr, momentum=cfg.momentum,
+                              cuda_stream=stream.cuda_stream, init_params=theta0)
+        n_params = ctx.n_params
+        packed_d = torch.empty((S, n_params), dtype=torch.float32, device="cuda")
+        packed_h = torch.empty((S, n_params), dtype=torch.float32).pin_memory()
+        conf_d = torch.zeros((S, C, C), dtype=torch.int64, device="cuda")
+        loss_d = torch.zeros((S, K), dtype=torch.float32, device="cuda")
+        mious = [0.0] * S
+
+        def key_frame(i, feats, logits, packed):
+            fs, ts = feats[i % N_SETS], logits[i % N_SETS]
+            for s in range(S):
+                st.st_set_frozen_features(ctx, s, fs[s])
+                st.st_teacher_labels(ctx, s, ts[s])
+            st.st_distill_step(ctx, K, loss_d)
+            for s in range(S):
+                st.st_pack_updated_params(ctx, s, packed[s])
+                mious[s] = st.st_agreement(ctx, s, None, None, conf_d[s])
+
+        def barrier():
+            if dist is not None:
+                dist.barrier()
+            torch.cuda.synchronize()
+
+        # ---- device-resident run
+        for i in range(args.warmup):
+            key_frame(i, feats_d, logits_d, packed_d)
+        clocks = ClockSampler(local_rank) if rank == 0 else None
+        barrier()
+        launches0 = st.st_launch_count(ctx)
+        ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        if clocks:
+            clocks.begin()
+        ev0.record(stream)
+        for i in range(args.steps):
+            key_frame(i, feats_d, logits_d, packed_d)
+        ev1.record(stream)
+        barrier()
+        if clocks:
+            clocks.end()
+        ms_total = ev0.elapsed_time(ev1)
+        launches = st.st_launch_count(ctx) - launches0
+        if dist is not None:
+            t = torch.tensor([ms_total], dtype=torch.float64, device="cuda")
+            dist.all_reduce(t, op=dist.ReduceOp.MAX)
+            ms_total = float(t.item())
+        clock_info = clocks.finish() if clocks else None
+
+        # ---- the K-step loop alone (inputs already cached), for the per-step view
+        barrier()
+        n_loop = max(10, min(args.steps, 500))
+        ev0.record(stream)
+        for i in range(n_loop):
+            st.st_distill_step(ctx, K, loss_d)
+        ev1.record(stream)
+        torch.cuda.synchronize()
+        ms_loop = ev0.elapsed_time(ev1) / n_loop
+
+        # ---- end to end through the C ABI with host buffers (pinned): H2D of the inputs, D2H of the results
+        e2e_steps = max(3, min(args.steps, 100))
+        for i in range(min(args.warmup, 3)):
+            key_frame(i, feats_h, logits_h, packed_h)
+        barrier()
+        ev0.record(stream)
+        for i in range(e2e_steps):
+            key_frame(i, feats_h, logits_h, packed_h)
+        ev1.record(stream)
+        barrier()
+        ms_e2e = ev0.elapsed_time(ev1)
+        if dist is not None:
+            t = torch.tensor([ms_e2e], dtype=torch.float64, device="cuda")
+            dist.all_reduce(t, op=dist.ReduceOp.MAX)
+            ms_e2e = float(t.item())
+        h2d = S * (cfg.c_in * p * 4 + C * P * 4)
+        d2h = S * (n_params * 4 + 8)
+
+        # ---- per-kernel times with CUDA events on the launching stream
+        kernels = {}
+        if rank == 0:
+            def timed(fn, reps=20):
+                ev0.record(stream)
+                for r in range(reps):
+                    fn(r)
+                ev1.record(stream)
+                torch.cuda.synchronize()
+                return ev0.elapsed_time(ev1) / reps
+            t_arg = timed(lambda r: st.st_teacher_labels(ctx, 0, logits_d[r % N_SETS][0]))
+            t_feat = timed(lambda r: st.st_set_frozen_features(ctx, 0, feats_d[r % N_SETS][0]))
+            masks = [torch.randint(0, C, (H, W), dtype=torch.uint8, device="cuda") for _ in range(2)]
+            t_agree = timed(lambda r: st.st_agreement(ctx, 0, masks[0], masks[1], conf_d[0]))
+            hbm = peaks["hbm_gbs"]
+            kernels["argmax_u8"] = {"ms": t_arg, "bound": "hbm", "achieved": (C * P * 4 + P) / t_arg / 1e6,
+                                    "peak": hbm, "unit": "GB/s", "per_key_frame": S}
+            if cfg.gemm_precision == 1:
+                kernels["feat_to_bf16_nhwc"] = {"ms": t_feat, "bound": "hbm", "achieved": cfg.c_in * p * 6 / t_feat / 1e6,
+                                                "peak": hbm, "unit": "GB/s", "per_key_frame": S}
+            kernels["agreement(confusion+miou+sync)"] = {"ms": t_agree, "bound": "latency", "achieved": 2 * P / t_agree / 1e6,
+                                                         "peak": hbm, "unit": "GB/s", "per_key_frame": S}
+            c_last = cfg.c_hidden or cfg.c_in
+            alu_peak = 148 * 128 * 2 * peaks["sm_max_mhz"] * 1e6 / 1e12          # fp32 FMA lanes x 2 flop x clock
+            tensor_peak = peaks["bf16_tflops"]
+            for name, ms in st.st_profile_step(ctx, 20):
+                k = {"ms": ms, "per_key_frame": K}
+                if name == "upsample_ce":
+                    k.update(bound="alu", achieved=ALU_FLOP_PER_CLASS_PIXEL * C * P * S / ms / 1e9, peak=alu_peak, unit="TFLOP/s",
+                             hbm_gbs=S * (2 * C * p * 4 + P) / ms / 1e6)
+                elif name == "tc_fwd1x1":
+                    k.update(bound="hbm", achieved=S * (p * c_last * 2 + C * p * 4) / ms / 1e6, peak=hbm, unit="GB/s",
+                             tflops=2.0 * S * p * C * c_last / ms / 1e9)
+                elif name == "tc_wgrad1x1":
+                    k.update(bound="hbm", achieved=S * (p * c_last * 2 + C * p * 2) / ms / 1e6, peak=hbm, unit="GB/s",
+                             tflops=2.0 * S * p * C * c_last / ms / 1e9)
+                elif name in ("tc_fwd3x3", "tc_wgrad3x3"):
+                    k.update(bound="tensor", achieved=2.0 * S * p * cfg.c_hidden * cfg.c_in * 9 / ms / 1e9, peak=tensor_peak,
+                             unit="TFLOP/s")
+                elif name == "dgrad_relu":
+                    k.update(bound="hbm", achieved=S * (2 * p * cfg.c_hidden * 2 + C * p * 4) / ms / 1e6, peak=hbm, unit="GB/s")
+                else:
+                    k.update(bound="latency")
+                kernels[name] = k
+            for k in kernels.values():
+                if "achieved" in k and k.get("peak"):
+                    k["frac"] = k["achieved"] / k["peak"]
+
+        result = None
+        if rank == 0:
+            ms_step = ms_total / args.steps
+            value = world * K * args.steps / (ms_total / 1e3)
+            dominant = max((n for n in kernels if "frac" in kernels[n] or True),
+                           key=lambda n: kernels[n]["ms"] * kernels[n]["per_key_frame"])
+            dk = kernels[dominant]
+            roofline = {"kernel": dominant, "bound": dk.get("bound"), "achieved": dk.get("achieved"), "peak": dk.get("peak"),
+                        "unit": dk.get("unit"), "frac": dk.get("frac"), "traffic": None,
+                        "peak_source": f"of {peaks['source']}" if dk.get("bound") in ("hbm", "tensor") else
+                                       "148 SMs x 128 fp32 lanes x 2 flop x max SM clock",
+                        "ms_per_launch": dk["ms"]}
+            result = {
+                "metric": METRIC, "value": value, "unit": "steps/s", "n_gpus": world, "steps": args.steps,
+                "warmup": args.warmup, "ms_per_step": ms_step, "higher_is_better": True, "scaling": "weak",
+                "vs_baseline": None, "dtype": "bf16" if cfg.gemm_precision == 1 else "f32", "data": "synthetic",
+                "config": {"workload": cfg.name, "k_steps": K, "frame": [H, W], "features": [cfg.c_in, cfg.feat_h, cfg.feat_w],
+                           "classes": C, "streams_per_gpu": S, "c_hidden": cfg.c_hidden,
+                           "step": "features cache + labels + K SGD iterations + pack + agreement per key frame",
+                           "l2": f"inputs rotate over {N_SETS} key frames ({N_SETS * S * (cfg.c_in * p + C * P) * 4 / 1e6:.0f} MB) > 126 MB L2",
+                           "parallelism": f"replicas x{world}, no collective"},
+                "clocks": clock_info,
+                "e2e": {"value": world * K * e2e_steps / (ms_e2e / 1e3), "unit": "steps/s", "h2d_bytes_per_step": h2d,
+                        "d2h_bytes_per_step": d2h, "ms_per_step": ms_e2e / e2e_steps},
+                "gpu_launches": int(launches),
+                "roofline": roofline,
+                "key_frames_per_s": world * args.steps / (ms_total / 1e3),
+                "distill_loop_only": {"steps_per_s": K / (ms_loop / 1e3), "ms_per_k_steps": ms_loop},
+                "kernels": kernels,
+                "last_loss": float(loss_d[0, -1].item()), "last_miou": mious[0],
+            }
+        st.st_destroy(ctx)
+
+    if rank == 0:
+        if world == 1 and not args.no_cpu_baseline:
+            import oracle
+            oracle.build()
+            feat, T, theta = si.stream_inputs(cfg)
+            rows = cfg.feat_h if cfg.c_hidden == 0 else max(4, cfg.feat_h // 16)
+            t = oracle_key_frame(cfg, feat, T, theta, rows=rows)
+            frac = rows / cfg.feat_h
+            result["cpu_baseline"] = {
+                "value": cfg.k_steps / t * frac, "unit": "steps/s", "cores": host_cores(), "kind": "oracle",
+                "sample": (f"one key frame (labels, {cfg.k_steps} steps, pack, agreement) of one stream on {rows} of "
+                           f"{cfg.feat_h} feature rows, {t:.1f} s, scaled by pixel count"),
+            }
+        print(json.dumps(result), flush=True)
+    if dist is not None:
+        dist.barrier()
+        dist.destroy_process_group()
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=2000)
+    ap.add_argument("--warmup", type=int, default=10)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--workload", type=int, default=2, help="index into the synthetic workload table (2 = 720p, 1x1 head, K=8)")
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    args = ap.parse_args()
+    args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
+    cfg = si.get_config(args.workload)
+    if args.impl == "reference":
+        run_reference(args, cfg)
+    else:
+        run_ours(args, cfg)
+
+
+if __name__ == "__main__":
+    main()

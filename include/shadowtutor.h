@@ -178,6 +178,19 @@ typedef enum st_tensor {
 ST_API st_status st_read_tensor(st_ctx *ctx, int32_t stream, st_tensor which, float *dst_host,
                          size_t dst_capacity, size_t *nbytes);
 
+/*
+ * st_profile_step — time the kernels of the step one by one.  Runs n_steps ordinary steps of
+ * Algorithm 1's loop body (they do update the parameters) without graph replay, with a CUDA event
+ * recorded on the context's stream after every kernel, and returns the mean time per kernel.
+ *   n_stages   host; receives the number of kernels in one step (<= ST_MAX_STAGES).
+ *   ms_out     host float[ST_MAX_STAGES]; mean milliseconds of each kernel, in launch order.
+ *   names_out  host const char*[ST_MAX_STAGES]; static strings naming the kernels.
+ * Waits for the stream after every step.  A measuring aid, not part of the method.
+ */
+#define ST_MAX_STAGES 12
+ST_API st_status st_profile_step(st_ctx *ctx, int32_t n_steps, int32_t *n_stages, float *ms_out,
+                                 const char **names_out);
+
 /* Number of kernels this library has launched on the context so far. */
 ST_API int64_t st_launch_count(const st_ctx *ctx);
 

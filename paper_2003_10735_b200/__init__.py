@@ -36,8 +36,9 @@ ST_TENSOR_FEATURES = 6
 EXPORTED = [
     "st_param_count", "st_init_head", "st_set_frozen_features", "st_teacher_labels", "st_set_labels",
     "st_distill_step", "st_pack_updated_params", "st_student_mask", "st_agreement", "st_read_tensor",
-    "st_launch_count", "st_destroy", "st_last_error", "st_status_name",
+    "st_launch_count", "st_destroy", "st_last_error", "st_status_name", "st_profile_step",
 ]
+ST_MAX_STAGES = 12
 
 
 class st_head_desc(ctypes.Structure):
@@ -89,6 +90,9 @@ def load_library() -> ctypes.CDLL:
     lib.st_agreement.argtypes = [vp, i32, vp, vp, vp, ctypes.POINTER(ctypes.c_double)]
     lib.st_read_tensor.restype = ctypes.c_int
     lib.st_read_tensor.argtypes = [vp, i32, ctypes.c_int, vp, ctypes.c_size_t, ctypes.POINTER(ctypes.c_size_t)]
+    lib.st_profile_step.restype = ctypes.c_int
+    lib.st_profile_step.argtypes = [vp, i32, ctypes.POINTER(i32), ctypes.POINTER(ctypes.c_float),
+                                    ctypes.POINTER(ctypes.c_char_p)]
     lib.st_launch_count.restype = i64
     lib.st_launch_count.argtypes = [vp]
     lib.st_destroy.restype = None
@@ -224,6 +228,15 @@ def st_read_tensor(ctx: _Ctx, stream: int, which: int) -> np.ndarray:
     out = np.empty(nbytes.value // 4, dtype=np.float32)
     _check(lib.st_read_tensor(ctx.handle, stream, which, out.ctypes.data, out.nbytes, ctypes.byref(nbytes)), ctx)
     return out
+
+
+def st_profile_step(ctx: _Ctx, n_steps: int):
+    """[(kernel name, mean milliseconds), ...] of one step, in launch order."""
+    n = ctypes.c_int32(0)
+    ms = (ctypes.c_float * ST_MAX_STAGES)()
+    names = (ctypes.c_char_p * ST_MAX_STAGES)()
+    _check(load_library().st_profile_step(ctx.handle, n_steps, ctypes.byref(n), ms, names), ctx)
+    return [(names[i].decode(), float(ms[i])) for i in range(n.value)]
 
 
 def st_launch_count(ctx: _Ctx) -> int:

@@ -608,7 +608,7 @@ TcPlan* tc_plan_create(const TcBuffers& b, char* err, size_t err_len)
 
 void tc_plan_destroy(TcPlan* P) { delete P; }
 
-int tc_forward(const TcPlan* P, cudaStream_t s)
+int tc_forward(const TcPlan* P, cudaStream_t s, StageTimer* t)
 {
     const TcBuffers& b = P->b;
     int n = 0;
@@ -617,28 +617,33 @@ int tc_forward(const TcPlan* P, cudaStream_t s)
         tc_fwd3x3_kernel<4><<<dim3(tiles, b.S), kThreadsTc, P->smem_fwd3, s>>>(
             P->x_fwd3, P->w1_map, b.theta, b.n_params, b.b1_off, b.hidden, b.c_in, b.c_hidden, b.h, b.w,
             pow2_cols(b.c_hidden), b.err);
+        if (t) t->mark("tc_fwd3x3", s);
         ++n;
     }
     const int tiles1 = (P->p + kTileM - 1) / kTileM;
     tc_fwd1x1_kernel<<<dim3(tiles1, b.S), kThreadsTc, P->smem_fwd1, s>>>(
         P->act_fwd, P->w2_map, b.theta, b.n_params, b.b2_off, b.z, b.C, P->p, P->c_last / kBlockK, b.err);
+    if (t) t->mark("tc_fwd1x1", s);
     return n + 1;
 }
 
-int tc_backward(const TcPlan* P, cudaStream_t s)
+int tc_backward(const TcPlan* P, cudaStream_t s, StageTimer* t)
 {
     const TcBuffers& b = P->b;
     int n = 0;
     tc_wgrad1x1_kernel<3><<<dim3(P->split2, b.S), kThreadsTc, P->smem_wg1, s>>>(
         P->act_wg, P->dz_map, b.w2_partials, P->c_last, P->chunks2, P->per2, P->cols2, b.err);
+    if (t) t->mark("tc_wgrad1x1", s);
     ++n;
     if (b.c_hidden) {
         const int blocks = tc_b1_partials(b.h, b.w);
         dgrad_relu_kernel<<<dim3(blocks, b.S), 256, P->smem_dgrad, s>>>(
             b.theta, b.n_params, b.w2_off, b.dz, b.hidden, b.dhidden, b.b1_partials, b.C, b.c_hidden, P->p);
+        if (t) t->mark("dgrad_relu", s);
         tc_wgrad3x3_kernel<3><<<dim3(9 * P->split1, b.S), kThreadsTc, P->smem_wg3, s>>>(
             P->x_wg3, P->dh_wg3, b.w1_partials, b.c_in, b.c_hidden, b.h, b.w, P->chunks1, P->per1, P->split1,
             P->cols1, b.err);
+        if (t) t->mark("tc_wgrad3x3", s);
         n += 2;
     }
     return n;

@@ -180,32 +180,35 @@ UpdateArgs make_update_args(st_ctx* c, int slot)
 }
 
 // Forward of the trainable part for all streams: z (and the hidden activation).
-st_status enqueue_forward(st_ctx* c)
+st_status enqueue_forward(st_ctx* c, StageTimer* t = nullptr)
 {
     cudaStream_t s = c->stream;
     if (c->bf16_mode) {
-        c->launches += tc_forward(c->plan, s);
+        c->launches += tc_forward(c->plan, s, t);
     } else if (c->Ch == 0) {
         launch_conv_fwd_f32(c->x_f32, c->Cin, c->h, c->w, c->theta + c->layout.w_off[0], c->theta + c->layout.b_off[0],
                             c->C, 1, false, c->z, c->S, (int64_t)c->Cin * c->p, c->n_params, c->n_params,
                             (int64_t)c->C * c->p, s);
+        if (t) t->mark("conv1x1_fwd_f32", s);
         c->launches += 1;
     } else {
         launch_conv_fwd_f32(c->x_f32, c->Cin, c->h, c->w, c->theta + c->layout.w_off[0], c->theta + c->layout.b_off[0],
                             c->Ch, 3, true, c->hid_f32, c->S, (int64_t)c->Cin * c->p, c->n_params, c->n_params,
                             (int64_t)c->Ch * c->p, s);
+        if (t) t->mark("conv3x3_fwd_f32", s);
         launch_conv_fwd_f32(c->hid_f32, c->Ch, c->h, c->w, c->theta + c->layout.w_off[1], c->theta + c->layout.b_off[1],
                             c->C, 1, false, c->z, c->S, (int64_t)c->Ch * c->p, c->n_params, c->n_params,
                             (int64_t)c->C * c->p, s);
+        if (t) t->mark("conv1x1_fwd_f32", s);
         c->launches += 2;
     }
     return check_launch(c, "head forward");
 }
 
-st_status enqueue_step(st_ctx* c, int slot, bool want_conf)
+st_status enqueue_step(st_ctx* c, int slot, bool want_conf, StageTimer* t = nullptr)
 {
     cudaStream_t s = c->stream;
-    st_status st = enqueue_forward(c);
+    st_status st = enqueue_forward(c, t);
     if (st != ST_OK) return st;
 
     UpsampleCeArgs k3;
@@ -217,15 +220,17 @@ st_status enqueue_step(st_ctx* c, int slot, bool want_conf)
     k3.bad = c->bad;
     k3.S = c->S; k3.C = c->C; k3.h = c->h; k3.w = c->w;
     launch_upsample_ce(k3, s);
+    if (t) t->mark("upsample_ce", s);
     c->launches += 1;
     st = check_launch(c, "upsample + cross-entropy");
     if (st != ST_OK) return st;
 
     if (c->bf16_mode) {
-        c->launches += tc_backward(c->plan, s);
+        c->launches += tc_backward(c->plan, s, t);
     } else if (c->Ch == 0) {
         launch_conv_wgrad_f32(c->x_f32, c->dz, c->Cin, c->C, c->h, c->w, 1, c->grad + c->layout.w_off[0], c->S,
                               (int64_t)c->Cin * c->p, (int64_t)c->C * c->p, c->n_params, s);
+        if (t) t->mark("conv1x1_wgrad_f32", s);
         c->launches += 1;
     } else {
         const int64_t hs = (int64_t)c->Ch * c->p;
@@ -236,12 +241,14 @@ st_status enqueue_step(st_ctx* c, int slot, bool want_conf)
         launch_conv_wgrad_f32(c->x_f32, c->dhid_f32, c->Cin, c->Ch, c->h, c->w, 3, c->grad + c->layout.w_off[0], c->S,
                               (int64_t)c->Cin * c->p, hs, c->n_params, s);
         launch_bias_grad_f32(c->dhid_f32, c->Ch, c->p, c->grad + c->layout.b_off[0], c->S, hs, c->n_params, s);
+        if (t) t->mark("backward_f32", s);
         c->launches += 4;
     }
     st = check_launch(c, "head backward");
     if (st != ST_OK) return st;
 
     launch_sgd_update(make_update_args(c, slot), s);
+    if (t) t->mark("sgd_update", s);
     c->launches += 1;
     return check_launch(c, "sgd update");
 }
@@ -537,6 +544,39 @@ st_status st_distill_step(st_ctx* ctx, int32_t n_steps, float* loss_out, int64_t
     if (conf_out)
         ST_CUDA(ctx, cudaMemcpy2DAsync(conf_out, (size_t)n_steps * cc * 8, ctx->conf_buf, (size_t)kMaxSteps * cc * 8,
                                        (size_t)n_steps * cc * 8, ctx->S, cudaMemcpyDefault, ctx->stream));
+    return ST_OK;
+}
+
+st_status st_profile_step(st_ctx* ctx, int32_t n_steps, int32_t* n_stages, float* ms_out, const char** names_out)
+{
+    if (!ctx) return ST_ERR_INVALID_ARG;
+    if (n_steps < 1 || !n_stages || !ms_out || !names_out)
+        return fail(ctx, ST_ERR_INVALID_ARG, "st_profile_step: n_steps >= 1 and non-NULL outputs are required");
+    for (int s = 0; s < ctx->S; ++s)
+        if (!ctx->has_feat[s] || !ctx->has_labels[s])
+            return fail(ctx, ST_ERR_BAD_STATE, "st_profile_step: stream %d has no features or labels yet", s);
+    StageTimer t;
+    for (int i = 0; i <= StageTimer::kMax; ++i) ST_CUDA(ctx, cudaEventCreate(&t.ev[i]));
+    double acc[StageTimer::kMax] = {0};
+    st_status st = ST_OK;
+    int n = 0;
+    for (int k = 0; k < n_steps && st == ST_OK; ++k) {
+        t.n = 0;
+        cudaEventRecord(t.ev[0], ctx->stream);
+        st = enqueue_step(ctx, 0, false, &t);
+        if (st != ST_OK) break;
+        if (cudaStreamSynchronize(ctx->stream) != cudaSuccess) { st = fail(ctx, ST_ERR_CUDA, "st_profile_step: synchronize failed"); break; }
+        n = t.n;
+        for (int i = 0; i < n; ++i) {
+            float ms = 0.f;
+            cudaEventElapsedTime(&ms, t.ev[i], t.ev[i + 1]);
+            acc[i] += ms;
+        }
+    }
+    for (int i = 0; i <= StageTimer::kMax; ++i) cudaEventDestroy(t.ev[i]);
+    if (st != ST_OK) return st;
+    *n_stages = n;
+    for (int i = 0; i < n; ++i) { ms_out[i] = (float)(acc[i] / n_steps); names_out[i] = t.name[i]; }
     return ST_OK;
 }
 

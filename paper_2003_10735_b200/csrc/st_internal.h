@@ -126,7 +126,15 @@ int tc_b1_partials(int h, int w);
 int tc_dz_pitch(int h, int w);      // row pitch (elements) of the bf16 logit gradient [S][kClassPad][pitch]
 TcPlan* tc_plan_create(const TcBuffers& b, char* err, size_t err_len);
 void tc_plan_destroy(TcPlan*);
-int tc_forward(const TcPlan*, cudaStream_t s);    // returns the number of kernels launched
-int tc_backward(const TcPlan*, cudaStream_t s);
+// Optional per-kernel timing: an event is recorded on the stream after each kernel launch.
+struct StageTimer {
+    static constexpr int kMax = 12;
+    cudaEvent_t ev[kMax + 1];
+    const char* name[kMax];
+    int n = 0;
+    void mark(const char* what, cudaStream_t s) { if (n < kMax) { name[n] = what; cudaEventRecord(ev[n + 1], s); ++n; } }
+};
+int tc_forward(const TcPlan*, cudaStream_t s, StageTimer* t = nullptr);    // returns the number of kernels launched
+int tc_backward(const TcPlan*, cudaStream_t s, StageTimer* t = nullptr);
 
 }  // namespace st
