@@ -191,6 +191,35 @@ ST_API st_status st_read_tensor(st_ctx *ctx, int32_t stream, st_tensor which, fl
 ST_API st_status st_profile_step(st_ctx *ctx, int32_t n_steps, int32_t *n_stages, float *ms_out,
                                  const char **names_out);
 
+/*
+ * st_agreement_noalloc — confusion matrix and mean IoU of two masks without any allocation.
+ * (The paper has no counterpart: this entry point exists for the sake of callers, not of the method.)
+ *
+ * Some callers cannot allocate device memory: a process that gave all of HBM to its own pool at
+ * start-up, a latency-critical loop that cannot take the device-wide synchronisation that
+ * cudaMalloc/cudaFree imply, or code running while allocation calls are forbidden.  st_agreement
+ * needs a context and creating one allocates; this variant takes no context and calls no cudaMalloc,
+ * cudaFree or any allocating routine.  Its counters live in a fixed __device__ array inside the
+ * library (about 33 KB, held by every GPU that loads the library until the process exits).
+ *
+ *   pred, label  device; uint8 [n_pixels] each.  Pixels with a value >= n_classes are skipped
+ *                (and, unlike st_agreement, not reported: this call never waits for the stream).
+ *   n_classes    2..ST_NOALLOC_MAX_CLASSES; larger values return ST_ERR_UNSUPPORTED.
+ *   cuda_stream  cudaStream_t on which the work is enqueued (NULL = default stream).
+ *   conf_out     device; int64 [n_classes][n_classes], conf[l][q] = #pixels with label l, prediction q.
+ *   miou_out     device; one double (Section 3.2's mean IoU over the classes present in the label).
+ * Returns after enqueueing; results are valid once the stream has passed the work.
+ * The first call on each device looks up the address of the internal array
+ * (cudaGetSymbolAddress, with that device current); make that first call before any stream capture.
+ * All calls share the internal array, which is cleared at the start of each call: calls whose work
+ * overlaps on the GPU (different streams without ordering between them) race and give wrong counts.
+ * Errors: ST_ERR_INVALID_ARG (NULL pointer, n_classes < 2, n_pixels < 0), ST_ERR_UNSUPPORTED, ST_ERR_CUDA.
+ */
+#define ST_NOALLOC_MAX_CLASSES 64
+ST_API st_status st_agreement_noalloc(const uint8_t *pred, const uint8_t *label, int64_t n_pixels,
+                                      int32_t n_classes, void *cuda_stream, int64_t *conf_out,
+                                      double *miou_out);
+
 /* Number of kernels this library has launched on the context so far. */
 ST_API int64_t st_launch_count(const st_ctx *ctx);
 

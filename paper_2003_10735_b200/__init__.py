@@ -37,7 +37,9 @@ EXPORTED = [
     "st_param_count", "st_init_head", "st_set_frozen_features", "st_teacher_labels", "st_set_labels",
     "st_distill_step", "st_pack_updated_params", "st_student_mask", "st_agreement", "st_read_tensor",
     "st_launch_count", "st_destroy", "st_last_error", "st_status_name", "st_profile_step",
+    "st_agreement_noalloc",
 ]
+ST_NOALLOC_MAX_CLASSES = 64
 ST_MAX_STAGES = 12
 
 
@@ -93,6 +95,8 @@ def load_library() -> ctypes.CDLL:
     lib.st_profile_step.restype = ctypes.c_int
     lib.st_profile_step.argtypes = [vp, i32, ctypes.POINTER(i32), ctypes.POINTER(ctypes.c_float),
                                     ctypes.POINTER(ctypes.c_char_p)]
+    lib.st_agreement_noalloc.restype = ctypes.c_int
+    lib.st_agreement_noalloc.argtypes = [vp, vp, i64, i32, vp, vp, vp]
     lib.st_launch_count.restype = i64
     lib.st_launch_count.argtypes = [vp]
     lib.st_destroy.restype = None
@@ -237,6 +241,26 @@ def st_profile_step(ctx: _Ctx, n_steps: int):
     names = (ctypes.c_char_p * ST_MAX_STAGES)()
     _check(load_library().st_profile_step(ctx.handle, n_steps, ctypes.byref(n), ms, names), ctx)
     return [(names[i].decode(), float(ms[i])) for i in range(n.value)]
+
+
+def st_agreement_noalloc(pred, label, n_classes: int, cuda_stream: int, conf_out, miou_out) -> None:
+    """Confusion matrix and mean IoU of two device uint8 masks for callers that must not allocate
+    device memory (no context, no cudaMalloc; the counters live in a fixed array inside the library).
+    `conf_out` (int64 [C][C]) and `miou_out` (float64 [1]) are device tensors filled asynchronously on
+    `cuda_stream`.  Calls share the internal array: do not let two of them overlap on the GPU."""
+    n = pred.numel()
+    if label.numel() != n:
+        raise ValueError("pred and label differ in size")
+    for t, what in ((pred, "pred"), (label, "label"), (conf_out, "conf_out"), (miou_out, "miou_out")):
+        if not getattr(t, "is_cuda", False):
+            raise TypeError(f"{what}: a CUDA tensor is required")
+    if str(miou_out.dtype) != "torch.float64" or miou_out.numel() < 1:
+        raise TypeError("miou_out: need a float64 tensor with one element")
+    status = load_library().st_agreement_noalloc(
+        _ptr(pred, "uint8", n, "pred"), _ptr(label, "uint8", n, "label"), n, n_classes, cuda_stream or None,
+        _ptr(conf_out, "int64", max(n_classes, 0) ** 2, "conf_out"), miou_out.data_ptr())
+    if status != ST_OK:
+        raise StError(status, load_library().st_status_name(status).decode(), "st_agreement_noalloc")
 
 
 def st_launch_count(ctx: _Ctx) -> int:
