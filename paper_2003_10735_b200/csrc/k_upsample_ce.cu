@@ -26,7 +26,11 @@ constexpr int kCells = (NY + 1) * (NX + 1);
 constexpr int kThreads = 160;
 constexpr int ZT_H = NY + 2, ZT_W = NX + 2;
 
-int upsample_ce_blocks(int h, int w) { return ((h + NY - 1) / NY) * ((w + NX - 1) / NX); }
+int upsample_ce_blocks(int h, int w, int C)
+{
+    if (upsample_ce_rows_supported(C)) return upsample_ce_rows_blocks(h, w);
+    return ((h + NY - 1) / NY) * ((w + NX - 1) / NX);
+}
 
 __device__ __forceinline__ float lerp_f(float a, float b, float t) { return fmaf(t, b - a, a); }
 
@@ -245,6 +249,7 @@ upsample_ce_kernel(UpsampleCeArgs a, int chunk)
 
 cudaError_t prepare_upsample_ce(int C)
 {
+    if (upsample_ce_rows_supported(C)) return prepare_upsample_ce_rows(C);
     size_t smem = 0;
     chunk_classes(C, &smem);
     cudaError_t e = cudaFuncSetAttribute(upsample_ce_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
@@ -254,6 +259,7 @@ cudaError_t prepare_upsample_ce(int C)
 
 void launch_upsample_ce(const UpsampleCeArgs& a, cudaStream_t s)
 {
+    if (upsample_ce_rows_supported(a.C)) { launch_upsample_ce_rows(a, s); return; }
     size_t smem = 0;
     const int chunk = chunk_classes(a.C, &smem);
     dim3 grid((unsigned)((a.w + NX - 1) / NX), (unsigned)((a.h + NY - 1) / NY), (unsigned)a.S);

@@ -369,7 +369,7 @@ st_status st_init_head(const st_head_desc* desc, const float* init_params, st_ct
 
     const int S = c->S;
     const int c_last = c->Ch ? c->Ch : c->Cin;
-    c->n_k3_blocks = upsample_ce_blocks(c->h, c->w);
+    c->n_k3_blocks = upsample_ce_blocks(c->h, c->w, c->C);
     cudaError_t e = cudaSuccess;
 #define ALLOC(ptr, count) if (e == cudaSuccess) e = dev_alloc(c, &c->ptr, (size_t)(count))
     ALLOC(theta, S * c->n_params); ALLOC(vel, S * c->n_params); ALLOC(grad, S * c->n_params);

@@ -41,9 +41,14 @@ struct UpsampleCeArgs {
     unsigned int* bad;       // count of labels >= C
     int S, C, h, w;
 };
-int upsample_ce_blocks(int h, int w);   // blocks per stream
+int upsample_ce_blocks(int h, int w, int C);   // blocks per stream (sizes loss_part / db_part)
 cudaError_t prepare_upsample_ce(int C);   // once per device and class count, outside any stream capture
 void launch_upsample_ce(const UpsampleCeArgs& a, cudaStream_t s);
+// register-resident variant for C <= 32 (k_upsample_ce_rows.cu); launch_upsample_ce dispatches to it
+bool upsample_ce_rows_supported(int C);
+int upsample_ce_rows_blocks(int h, int w);
+cudaError_t prepare_upsample_ce_rows(int C);
+void launch_upsample_ce_rows(const UpsampleCeArgs& a, cudaStream_t s);
 // student mask: argmax_c of the upsampled logits, uint8 [H][W]
 void launch_upsample_argmax(const float* z, int C, int h, int w, uint8_t* mask, cudaStream_t s);
 

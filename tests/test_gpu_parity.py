@@ -252,6 +252,29 @@ def test_small_fp32_steps(c_in, ch, C, h, w, K, mu):
     st.st_destroy(ctx)
 
 
+def test_wildly_varying_logits_take_the_exact_maximum_path():
+    # neighbouring nodes carry logits +-300 in different classes: halfway between them every class is
+    # 150 below the largest node logit, so a softmax normalised by a neighbourhood bound would underflow
+    c_in, C, h, w = 2, 3, 6, 40
+    rng = np.random.default_rng(3)
+    f = (rng.random((h, w)) < 0.5).astype(np.float32)
+    feat = np.stack([f, 1.0 - f])
+    theta = np.array([300.0, 0.0, 0.0, 300.0, 10.0, 10.0, 0.0, 0.0, 0.0], np.float32)   # W [3][2], b [3]
+    lab = rng.integers(0, C, (4 * h, 4 * w)).astype(np.uint8)
+    ctx = make_ctx(c_in, 0, C, h, w, theta, lr=1e-4)
+    st.st_set_frozen_features(ctx, 0, feat)
+    st.st_set_labels(ctx, 0, lab)
+    loss = np.zeros(1, np.float32)
+    st.st_distill_step(ctx, 1, loss)
+    head = oracle.Head(c_in, 0, C, lr=1e-4, theta=theta)
+    ref, _ = oracle.distill_step(head, feat, lab)
+    assert np.isfinite(loss[0]) and abs(loss[0] - ref) <= 1e-4 * abs(ref)
+    dz = st.st_read_tensor(ctx, 0, st.ST_TENSOR_LOGIT_GRAD)
+    assert np.isfinite(dz).all()
+    np.testing.assert_allclose(packed(ctx), head.theta, rtol=1e-4, atol=1e-5)
+    st.st_destroy(ctx)
+
+
 def test_two_streams_are_independent_fp32():
     c_in, C, h, w = 6, 3, 5, 7
     probs = [rand_problem(20 + s, c_in, C, h, w) for s in range(2)]
