@@ -46,8 +46,10 @@ upsample_ce_rows_kernel(UpsampleCeArgs a)
 {
     extern __shared__ __align__(16) float smem_r[];
     const int C = a.C, h = a.h, w = a.w, H = h * kUp, W = w * kUp;
-    float* zt = smem_r;                         // [C][TZ_H][TZ_W]  logits * log2(e), borders replicated
-    float* nmax = zt + C * TZ;                  // [TZ_H][TZ_W]     max over classes
+    float* zt = smem_r;                         // [CB][TZ_H][TZ_W] logits * log2(e), borders replicated;
+                                                //                  classes >= C hold -1e30 (their exponentials are 0),
+                                                //                  which keeps the class loops free of branches
+    float* nmax = zt + CB * TZ;                 // [TZ_H][TZ_W]     max over classes
     int* corr = (int*)(nmax + TZ);              // [C][TZ_H][TZ_W]  -64 * (adjoint of onehot)
     float* bsh = (float*)(corr + C * TZ);       // [R_WARPS][C][32] lower-row accumulators
     float* dbs = bsh + R_WARPS * C * 32;        // [R_WARPS][C]
@@ -60,25 +62,38 @@ upsample_ce_rows_kernel(UpsampleCeArgs a)
     const uint8_t* labels = a.labels + (int64_t)s * H * W;
     const int tid = threadIdx.x, wi = tid >> 5, l = tid & 31;
 
-    // ---- tile: nodes y0-1 .. y0+RN_Y, x0-2 .. x0+31 (clamped), scaled; per-node maximum; zeroed corrections
-    for (int e = tid; e < TZ; e += R_THREADS) {
-        const int ry = e / TZ_W, rx = e % TZ_W;
-        const int yy = min(max(y0 - 1 + ry, 0), h - 1), xx = min(max(x0 - 2 + rx, 0), w - 1);
-        const float* src = z + (int64_t)yy * w + xx;
-        float m = -INFINITY;
-        for (int c = 0; c < C; ++c) {
-            const float v = __ldg(src + (int64_t)c * p) * kLog2e;
-            zt[c * TZ + e] = v;
-            m = fmaxf(m, v);
-        }
-        nmax[e] = m;
-    }
-    for (int e = tid; e < C * TZ; e += R_THREADS) corr[e] = 0;
-    __syncthreads();
-
     const int i = y0 - 1 + wi;                  // cell row: frame rows 4i+2 .. 4i+5, nodes (i, i+1)
     const int xg = x0 - 1 + l;                  // node column whose four frame pixels this lane handles
     const bool lane_valid = xg >= 0 && xg < w;
+
+    // ---- tile: nodes y0-1 .. y0+RN_Y, x0-2 .. x0+31 (clamped), scaled; zeroed corrections; per-node maximum
+    // (fully unrolled: all of a thread's loads are in flight together, one memory latency for the whole tile)
+    {
+        constexpr int kIter = (CB * TZ + R_THREADS - 1) / R_THREADS;
+        float v[kIter];
+#pragma unroll
+        for (int it = 0; it < kIter; ++it) {
+            const int e = tid + it * R_THREADS;
+            const int c = e / TZ, n = e % TZ;
+            const int ry = n / TZ_W, rx = n % TZ_W;
+            const int yy = min(max(y0 - 1 + ry, 0), h - 1), xx = min(max(x0 - 2 + rx, 0), w - 1);
+            v[it] = (e < CB * TZ && c < C) ? __ldg(z + (int64_t)c * p + (int64_t)yy * w + xx) * kLog2e : -1e30f;
+        }
+#pragma unroll
+        for (int it = 0; it < kIter; ++it) {
+            const int e = tid + it * R_THREADS;
+            if (e < CB * TZ) zt[e] = v[it];
+        }
+    }
+    for (int e = tid; e < C * TZ; e += R_THREADS) corr[e] = 0;
+    __syncthreads();
+    for (int e = tid; e < TZ; e += R_THREADS) {
+        float m = -INFINITY;
+        for (int c = 0; c < C; ++c) m = fmaxf(m, zt[c * TZ + e]);
+        nmax[e] = m;
+    }
+    __syncthreads();
+
     const bool lane_owned = lane_valid && l >= 1 && l <= RN_X;
     const bool cell_row_valid = i <= h - 1;
     const float* zp = zt + wi * TZ_W + l;       // node (i, xg-1) of class 0
@@ -100,7 +115,7 @@ upsample_ce_rows_kernel(UpsampleCeArgs a)
         const float ly = (2 * r + 1) * 0.125f;
         const bool row_owned = (Y >> 2) >= y0 && (Y >> 2) < y0 + RN_Y;
         uint32_t lw = 0xffffffffu;
-        if (lane_valid) lw = *reinterpret_cast<const uint32_t*>(labels + (int64_t)Y * W + 4 * xg);
+        if (lane_valid) lw = __ldg(reinterpret_cast<const uint32_t*>(labels + (int64_t)Y * W + 4 * xg));
         int lab[4];
 #pragma unroll
         for (int k = 0; k < 4; ++k) {
@@ -120,18 +135,16 @@ upsample_ce_rows_kernel(UpsampleCeArgs a)
             float best[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};
 #pragma unroll
             for (int c = 0; c < CB; ++c) {
-                if (c < C) {
-                    const float* q = zp + c * TZ;
-                    const float vl = lerp_r(q[0], q[TZ_W], ly), vc = lerp_r(q[1], q[TZ_W + 1], ly), vr = lerp_r(q[2], q[TZ_W + 2], ly);
-                    const float dl = vc - vl, dr = vr - vc;
-                    float u[4] = {fmaf(0.625f, dl, vl), fmaf(0.875f, dl, vl), fmaf(0.125f, dr, vc), fmaf(0.375f, dr, vc)};
+                const float* q = zp + c * TZ;
+                const float vl = lerp_r(q[0], q[TZ_W], ly), vc = lerp_r(q[1], q[TZ_W + 1], ly), vr = lerp_r(q[2], q[TZ_W + 2], ly);
+                const float dl = vc - vl, dr = vr - vc;
+                float u[4] = {fmaf(0.625f, dl, vl), fmaf(0.875f, dl, vl), fmaf(0.125f, dr, vc), fmaf(0.375f, dr, vc)};
 #pragma unroll
-                    for (int k = 0; k < 4; ++k) {
-                        if (CONF && attempt == 0) { if (u[k] > best[k]) { best[k] = u[k]; arg[k] = c; } }
-                        const float e = ex2_approx(u[k] - mk[k]);
-                        ev[k][c] = e;
-                        Zs[k] += e;
-                    }
+                for (int k = 0; k < 4; ++k) {
+                    if (CONF && attempt == 0) { if (u[k] > best[k]) { best[k] = u[k]; arg[k] = c; } }
+                    const float e = ex2_approx(u[k] - mk[k]);
+                    ev[k][c] = e;
+                    Zs[k] += e;
                 }
             }
             // the bound can sit far above a pixel's true maximum only for wildly varying logits; then redo exactly
@@ -176,21 +189,20 @@ upsample_ce_rows_kernel(UpsampleCeArgs a)
             }
         }
         // ---- B: softmax part of the adjoint
-        const float w0l = 0.375f * rz[0], w0c = 0.625f * rz[0], w1l = 0.125f * rz[1], w1c = 0.875f * rz[1];
-        const float w2c = 0.875f * rz[2], w2r = 0.125f * rz[2], w3c = 0.625f * rz[3], w3r = 0.375f * rz[3];
+        // at the clamped left/right border the outer node is the inner one: its weight joins the centre weight
         const bool fold_l = xg == 0, fold_r = xg == w - 1;
+        const float w0l = fold_l ? 0.f : 0.375f * rz[0], w0c = (fold_l ? 1.0f : 0.625f) * rz[0];
+        const float w1l = fold_l ? 0.f : 0.125f * rz[1], w1c = (fold_l ? 1.0f : 0.875f) * rz[1];
+        const float w2r = fold_r ? 0.f : 0.125f * rz[2], w2c = (fold_r ? 1.0f : 0.875f) * rz[2];
+        const float w3r = fold_r ? 0.f : 0.375f * rz[3], w3c = (fold_r ? 1.0f : 0.625f) * rz[3];
 #pragma unroll
         for (int c = 0; c < CB; ++c) {
-            if (c < C) {
-                float aL = fmaf(w0l, ev[0][c], w1l * ev[1][c]);
-                float aR = fmaf(w2r, ev[2][c], w3r * ev[3][c]);
-                float aC = fmaf(w0c, ev[0][c], fmaf(w1c, ev[1][c], fmaf(w2c, ev[2][c], w3c * ev[3][c])));
-                if (fold_l) { aC += aL; aL = 0.f; }       // clamped border: the outer node is the inner one
-                if (fold_r) { aC += aR; aR = 0.f; }
-                const float hsum = aC + __shfl_up_sync(0xffffffffu, aR, 1) + __shfl_down_sync(0xffffffffu, aL, 1);
-                top[c] = fmaf(1.0f - ly, hsum, top[c]);
-                bot[c] = fmaf(ly, hsum, bot[c]);
-            }
+            const float aL = fmaf(w0l, ev[0][c], w1l * ev[1][c]);
+            const float aR = fmaf(w2r, ev[2][c], w3r * ev[3][c]);
+            const float aC = fmaf(w0c, ev[0][c], fmaf(w1c, ev[1][c], fmaf(w2c, ev[2][c], w3c * ev[3][c])));
+            const float hsum = aC + __shfl_up_sync(0xffffffffu, aR, 1) + __shfl_down_sync(0xffffffffu, aL, 1);
+            top[c] = fmaf(1.0f - ly, hsum, top[c]);
+            bot[c] = fmaf(ly, hsum, bot[c]);
         }
     }
     // clamped borders in y
@@ -245,25 +257,26 @@ upsample_ce_rows_kernel(UpsampleCeArgs a)
     }
 }
 
+template <int CB>
 size_t rows_smem_bytes(int C)
 {
-    return ((size_t)C * TZ * 2 + TZ + (size_t)R_WARPS * C * 32 + (size_t)R_WARPS * C) * sizeof(float) + 16;
+    return ((size_t)(CB + C) * TZ + TZ + (size_t)R_WARPS * C * 32 + (size_t)R_WARPS * C) * sizeof(float) + 16;
 }
 
 template <int CB>
 cudaError_t prepare_cb(int C)
 {
-    cudaError_t e = cudaFuncSetAttribute(upsample_ce_rows_kernel<CB, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)rows_smem_bytes(C));
+    cudaError_t e = cudaFuncSetAttribute(upsample_ce_rows_kernel<CB, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)rows_smem_bytes<CB>(C));
     if (e != cudaSuccess) return e;
-    return cudaFuncSetAttribute(upsample_ce_rows_kernel<CB, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)rows_smem_bytes(C));
+    return cudaFuncSetAttribute(upsample_ce_rows_kernel<CB, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)rows_smem_bytes<CB>(C));
 }
 
 template <int CB>
 void launch_cb(const UpsampleCeArgs& a, cudaStream_t s)
 {
     dim3 grid((unsigned)((a.w + RN_X - 1) / RN_X), (unsigned)((a.h + RN_Y - 1) / RN_Y), (unsigned)a.S);
-    if (a.conf) upsample_ce_rows_kernel<CB, true><<<grid, R_THREADS, rows_smem_bytes(a.C), s>>>(a);
-    else upsample_ce_rows_kernel<CB, false><<<grid, R_THREADS, rows_smem_bytes(a.C), s>>>(a);
+    if (a.conf) upsample_ce_rows_kernel<CB, true><<<grid, R_THREADS, rows_smem_bytes<CB>(a.C), s>>>(a);
+    else upsample_ce_rows_kernel<CB, false><<<grid, R_THREADS, rows_smem_bytes<CB>(a.C), s>>>(a);
 }
 
 }  // namespace
@@ -274,18 +287,30 @@ int upsample_ce_rows_blocks(int h, int w) { return ((h + RN_Y - 1) / RN_Y) * ((w
 
 cudaError_t prepare_upsample_ce_rows(int C)
 {
-    if (C <= 8) return prepare_cb<8>(C);
-    if (C <= 16) return prepare_cb<16>(C);
-    if (C <= 24) return prepare_cb<24>(C);
-    return prepare_cb<32>(C);
+    switch ((C + 3) / 4) {
+        case 1: return prepare_cb<4>(C);
+        case 2: return prepare_cb<8>(C);
+        case 3: return prepare_cb<12>(C);
+        case 4: return prepare_cb<16>(C);
+        case 5: return prepare_cb<20>(C);
+        case 6: return prepare_cb<24>(C);
+        case 7: return prepare_cb<28>(C);
+        default: return prepare_cb<32>(C);
+    }
 }
 
 void launch_upsample_ce_rows(const UpsampleCeArgs& a, cudaStream_t s)
 {
-    if (a.C <= 8) launch_cb<8>(a, s);
-    else if (a.C <= 16) launch_cb<16>(a, s);
-    else if (a.C <= 24) launch_cb<24>(a, s);
-    else launch_cb<32>(a, s);
+    switch ((a.C + 3) / 4) {
+        case 1: launch_cb<4>(a, s); break;
+        case 2: launch_cb<8>(a, s); break;
+        case 3: launch_cb<12>(a, s); break;
+        case 4: launch_cb<16>(a, s); break;
+        case 5: launch_cb<20>(a, s); break;
+        case 6: launch_cb<24>(a, s); break;
+        case 7: launch_cb<28>(a, s); break;
+        default: launch_cb<32>(a, s); break;
+    }
 }
 
 }  // namespace st
