@@ -1,26 +1,27 @@
-// K3, register-resident form (n_classes <= 32) — ComputeLoss and the first half of PartialBackward
+// K3, row-walking form (n_classes <= 32) — ComputeLoss and the first half of PartialBackward
 // (Algorithm 1; loss of Section 5.2): bilinear x4 upsample of the low-resolution logits, per-pixel
 // softmax cross-entropy against the labels, and the gradient of the mean loss with respect to the
-// low-resolution logits.  Same result as the cell-per-thread kernel in k_upsample_ce.cu, organised
-// so that every exponential is evaluated once.
+// low-resolution logits.  Same result as the cell-per-thread kernel in k_upsample_ce.cu.
 //
-// A block owns 7 rows x 30 columns of feature-map nodes and runs 8 warps (two per scheduler, so that each
-// thread may hold the exponentials of four pixels x all classes in registers).  Warp i handles "cell row"
-// y0-1+i: the four frame rows between node rows (y0-1+i, y0+i); lane l handles the four frame pixels
-// of node column x0-1+l in each of those rows.  (Warp 0 and lanes 0/31 are the halo: their pixels are
-// recomputed by the neighbouring block, so that a block finishes its nodes alone, in a fixed order.)
-// Per frame row a thread
-//   A. interpolates the logits of its four pixels class by class (logits pre-scaled by log2 e in shared
-//      memory), exponentiates against an upper bound of the maximum (the largest logit of the six
-//      nodes it reads; the pixel is redone with its exact maximum if the sum underflows), keeps the
-//      exponentials in registers and sums them;
-//   B. forms softmax * (adjoint interpolation weights) toward its left/own/right node column, trades
-//      the side parts with the neighbouring lanes by shuffle, and adds the row into two per-class
-//      accumulators: toward the upper and the lower node row.
-// The "- onehot(label)" part of the gradient is exact in units of 1/64 (products of the eighths
-// weights), so it is accumulated with integer shared-memory atomics, order-independent.
-// At the end warp i adds its upper accumulator to the lower accumulator of warp i-1 (through shared
-// memory) and writes node row y0-1+i: one 120-byte run per class.
+// Geometry.  With half-pixel centres and factor 4 the frame pixels 4n+2 .. 4n+5 lie between node
+// columns n and n+1 ("cell" n) with weights 1/8, 3/8, 5/8, 7/8 toward n+1; rows alike.  Cells -1 and
+// w-1 are the clamped borders (their outer node is the inner one).
+// A block owns RN_Y rows x 30 columns of nodes and runs RN_Y+1 warps.  Warp i walks the four frame rows
+// of cell row y0-1+i; lane l owns node column x0-1+l and handles the four pixels of the cell to its
+// right.  Warp 0, lane 0 and lane 31 are halo (recomputed by the neighbouring block) so that a block
+// finishes its nodes alone, in a fixed summation order, without floating-point atomics.
+// Per frame row:
+//   pass 1  each lane interpolates its own node column vertically, takes the right neighbour's by
+//           shuffle, interpolates its four pixels horizontally, and sums exp2(u - M) over the classes
+//           (logits are pre-scaled by log2 e; M is the largest logit of the warp's two node rows);
+//   pass 2  the exponentials are formed again (cheaper than keeping 4 x C registers alive: three
+//           or three blocks per SM stay resident), multiplied by the adjoint interpolation weights / Z, the
+//           right-hand part is handed to the next lane by shuffle, and the row is added into two
+//           per-class accumulators: toward the upper and the lower node row.
+// If a pixel's sum underflows (logits varying by more than ~100 inside the warp's span) the warp
+// redoes that row with the exact per-pixel maximum.
+// The "- onehot(label)" part of the gradient is exact in units of 1/64, so it is accumulated with
+// integer shared-memory atomics (order-independent).
 #include "st_internal.h"
 
 namespace st {
@@ -29,10 +30,9 @@ namespace {
 
 constexpr int RN_Y = 7, RN_X = 30;
 constexpr int R_WARPS = RN_Y + 1, R_THREADS = R_WARPS * 32;
-constexpr int TZ_H = RN_Y + 2, TZ_W = RN_X + 4, TZ = TZ_H * TZ_W;
+constexpr int TZ_H = RN_Y + 2, TZ_W = 32, TZ = TZ_H * TZ_W;
 constexpr float kLog2e = 1.4426950408889634f, kLn2 = 0.6931471805599453f;
 
-__device__ __forceinline__ float lerp_r(float a, float b, float t) { return fmaf(t, b - a, a); }
 __device__ __forceinline__ float ex2_approx(float x)
 {
     float y;
@@ -40,20 +40,73 @@ __device__ __forceinline__ float ex2_approx(float x)
     return y;
 }
 
+struct RowCtx {
+    const float* za;     // zt + wi*TZ_W + l : own column, upper node row, class 0
+    float ly;            // weight toward the lower node row
+    float M;             // warp-uniform shift
+};
+
+// interpolated, shifted logits of the lane's four pixels for class c
+template <bool SHIFT>
+__device__ __forceinline__ void pixel_logits(const RowCtx& rc, int c, const float (&sk)[4], float (&u)[4])
+{
+    const float a = rc.za[c * TZ], b = rc.za[c * TZ + TZ_W];
+    const float vl = fmaf(rc.ly, b - a, a) - rc.M;
+    const float vr = __shfl_down_sync(0xffffffffu, vl, 1);
+    const float d = vr - vl;
+    u[0] = fmaf(0.125f, d, vl); u[1] = fmaf(0.375f, d, vl); u[2] = fmaf(0.625f, d, vl); u[3] = fmaf(0.875f, d, vl);
+    if (SHIFT) {
+#pragma unroll
+        for (int k = 0; k < 4; ++k) u[k] -= sk[k];
+    }
+}
+
+template <int CB, bool CONF, bool SHIFT>
+__device__ __forceinline__ void pass1(const RowCtx& rc, const float (&sk)[4], float (&Zs)[4], uint32_t (&arg)[4])
+{
+    float best[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};
+    Zs[0] = Zs[1] = Zs[2] = Zs[3] = 0.f;
+#pragma unroll
+    for (int c = 0; c < CB; ++c) {
+        float u[4];
+        pixel_logits<SHIFT>(rc, c, sk, u);
+#pragma unroll
+        for (int k = 0; k < 4; ++k) {
+            if (CONF && !SHIFT) { if (u[k] > best[k]) { best[k] = u[k]; arg[k] = c; } }
+            Zs[k] += ex2_approx(u[k]);
+        }
+    }
+}
+
+template <int CB, bool SHIFT>
+__device__ __forceinline__ void pass2(const RowCtx& rc, const float (&sk)[4], const float (&wl)[4], const float (&wr)[4],
+                                      float (&top)[CB], float (&bot)[CB])
+{
+#pragma unroll
+    for (int c = 0; c < CB; ++c) {
+        float u[4];
+        pixel_logits<SHIFT>(rc, c, sk, u);
+        const float e0 = ex2_approx(u[0]), e1 = ex2_approx(u[1]), e2 = ex2_approx(u[2]), e3 = ex2_approx(u[3]);
+        const float aL = fmaf(wl[0], e0, fmaf(wl[1], e1, fmaf(wl[2], e2, wl[3] * e3)));
+        const float aR = fmaf(wr[0], e0, fmaf(wr[1], e1, fmaf(wr[2], e2, wr[3] * e3)));
+        const float hs = aL + __shfl_up_sync(0xffffffffu, aR, 1);      // own cell's left part + left cell's right part
+        top[c] = fmaf(1.0f - rc.ly, hs, top[c]);
+        bot[c] = fmaf(rc.ly, hs, bot[c]);
+    }
+}
+
 template <int CB, bool CONF>
-__global__ void __launch_bounds__(R_THREADS, 1)
+__global__ void __launch_bounds__(R_THREADS, CB > 16 ? 2 : 3)
 upsample_ce_rows_kernel(UpsampleCeArgs a)
 {
     extern __shared__ __align__(16) float smem_r[];
     const int C = a.C, h = a.h, w = a.w, H = h * kUp, W = w * kUp;
-    float* zt = smem_r;                         // [CB][TZ_H][TZ_W] logits * log2(e), borders replicated;
-                                                //                  classes >= C hold -1e30 (their exponentials are 0),
-                                                //                  which keeps the class loops free of branches
-    float* nmax = zt + CB * TZ;                 // [TZ_H][TZ_W]     max over classes
-    int* corr = (int*)(nmax + TZ);              // [C][TZ_H][TZ_W]  -64 * (adjoint of onehot)
-    float* bsh = (float*)(corr + C * TZ);       // [R_WARPS][C][32] lower-row accumulators
-    float* dbs = bsh + R_WARPS * C * 32;        // [R_WARPS][C]
+    float* zt = smem_r;                         // [CB][TZ_H][32]   logits * log2(e), borders replicated; classes >= C
+                                                //                  hold -1e30 (their exponentials are 0)
+    int* corr = (int*)(zt + CB * TZ);           // [C][TZ_H][32]    -64 * (adjoint of onehot)
+    float* bsh = zt;                            // [R_WARPS][C][32] lower-row accumulators (reuses the tile once the rows are done)
     __shared__ float red[R_WARPS];
+    __shared__ float dbs[R_WARPS][32];
 
     const int s = blockIdx.z, x0 = blockIdx.x * RN_X, y0 = blockIdx.y * RN_Y;
     const int blk = blockIdx.y * gridDim.x + blockIdx.x, n_blk = gridDim.x * gridDim.y;
@@ -62,12 +115,8 @@ upsample_ce_rows_kernel(UpsampleCeArgs a)
     const uint8_t* labels = a.labels + (int64_t)s * H * W;
     const int tid = threadIdx.x, wi = tid >> 5, l = tid & 31;
 
-    const int i = y0 - 1 + wi;                  // cell row: frame rows 4i+2 .. 4i+5, nodes (i, i+1)
-    const int xg = x0 - 1 + l;                  // node column whose four frame pixels this lane handles
-    const bool lane_valid = xg >= 0 && xg < w;
-
-    // ---- tile: nodes y0-1 .. y0+RN_Y, x0-2 .. x0+31 (clamped), scaled; zeroed corrections; per-node maximum
-    // (fully unrolled: all of a thread's loads are in flight together, one memory latency for the whole tile)
+    // ---- tile: node rows y0-1 .. y0+RN_Y, node columns x0-1 .. x0+30 (clamped), scaled by log2(e).
+    // Fully unrolled so that all of a thread's loads are in flight together.
     {
         constexpr int kIter = (CB * TZ + R_THREADS - 1) / R_THREADS;
         float v[kIter];
@@ -75,8 +124,7 @@ upsample_ce_rows_kernel(UpsampleCeArgs a)
         for (int it = 0; it < kIter; ++it) {
             const int e = tid + it * R_THREADS;
             const int c = e / TZ, n = e % TZ;
-            const int ry = n / TZ_W, rx = n % TZ_W;
-            const int yy = min(max(y0 - 1 + ry, 0), h - 1), xx = min(max(x0 - 2 + rx, 0), w - 1);
+            const int yy = min(max(y0 - 1 + n / TZ_W, 0), h - 1), xx = min(max(x0 - 1 + n % TZ_W, 0), w - 1);
             v[it] = (e < CB * TZ && c < C) ? __ldg(z + (int64_t)c * p + (int64_t)yy * w + xx) * kLog2e : -1e30f;
         }
 #pragma unroll
@@ -87,20 +135,26 @@ upsample_ce_rows_kernel(UpsampleCeArgs a)
     }
     for (int e = tid; e < C * TZ; e += R_THREADS) corr[e] = 0;
     __syncthreads();
-    for (int e = tid; e < TZ; e += R_THREADS) {
-        float m = -INFINITY;
-        for (int c = 0; c < C; ++c) m = fmaxf(m, zt[c * TZ + e]);
-        nmax[e] = m;
-    }
-    __syncthreads();
 
-    const bool lane_owned = lane_valid && l >= 1 && l <= RN_X;
+    const int i = y0 - 1 + wi;                  // cell row: frame rows 4i+2 .. 4i+5, node rows (i, i+1)
+    const int n = x0 - 1 + l;                   // own node column; cell n lies between node columns n and n+1
     const bool cell_row_valid = i <= h - 1;
-    const float* zp = zt + wi * TZ_W + l;       // node (i, xg-1) of class 0
-    // tile coordinates of the (clamped) nodes this thread's pixels pull toward
+    const bool cell_valid = l <= 30 && n >= -1 && n <= w - 1;
+    const bool node_owned = l >= 1 && l <= RN_X && n < w;
+    // tile coordinates of the (clamped) nodes this lane's pixels pull toward
     const int ry_top = min(max(i, 0), h - 1) - (y0 - 1), ry_bot = min(max(i + 1, 0), h - 1) - (y0 - 1);
-    const int rx_l = min(max(xg - 1, 0), w - 1) - (x0 - 2), rx_c = min(max(xg, 0), w - 1) - (x0 - 2),
-              rx_r = min(max(xg + 1, 0), w - 1) - (x0 - 2);
+    const int rx_l = min(max(n, 0), w - 1) - (x0 - 1), rx_r = min(max(n + 1, 0), w - 1) - (x0 - 1);
+
+    RowCtx rc;
+    rc.za = zt + wi * TZ_W + l;
+    rc.ly = 0.f;
+    {
+        float m = -INFINITY;
+        for (int c = 0; c < C; ++c) m = fmaxf(m, fmaxf(rc.za[c * TZ], rc.za[c * TZ + TZ_W]));
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) m = fmaxf(m, __shfl_xor_sync(0xffffffffu, m, o));
+        rc.M = m;
+    }
 
     float top[CB], bot[CB];
 #pragma unroll
@@ -110,100 +164,83 @@ upsample_ce_rows_kernel(UpsampleCeArgs a)
 
     for (int r = 0; r < 4; ++r) {
         const int Y = 4 * i + 2 + r;
-        const bool row_valid = cell_row_valid && Y >= 0 && Y < H;     // warp-uniform
-        if (!row_valid) continue;
-        const float ly = (2 * r + 1) * 0.125f;
+        if (!(cell_row_valid && Y >= 0 && Y < H)) continue;          // warp-uniform
+        rc.ly = (2 * r + 1) * 0.125f;
         const bool row_owned = (Y >> 2) >= y0 && (Y >> 2) < y0 + RN_Y;
-        uint32_t lw = 0xffffffffu;
-        if (lane_valid) lw = __ldg(reinterpret_cast<const uint32_t*>(labels + (int64_t)Y * W + 4 * xg));
+        // labels of pixels 4n+2 .. 4n+5 (two aligned 16-bit loads)
+        const int X0 = 4 * n + 2;
         int lab[4];
+        bool pv[4];
+        {
+            uint32_t lo = 0xffff, hi = 0xffff;
+            const bool v01 = cell_valid && X0 >= 0 && X0 + 1 < W, v23 = cell_valid && X0 + 2 >= 0 && X0 + 3 < W;
+            if (v01) lo = __ldg(reinterpret_cast<const unsigned short*>(labels + (int64_t)Y * W + X0));
+            if (v23) hi = __ldg(reinterpret_cast<const unsigned short*>(labels + (int64_t)Y * W + X0 + 2));
+            lab[0] = lo & 0xff; lab[1] = lo >> 8; lab[2] = hi & 0xff; lab[3] = hi >> 8;
+            pv[0] = pv[1] = v01; pv[2] = pv[3] = v23;
+        }
+        // ownership of a pixel = ownership of its node-aligned group (X >> 2)
+        bool own[4];
 #pragma unroll
         for (int k = 0; k < 4; ++k) {
-            lab[k] = (lw >> (8 * k)) & 0xff;
-            if (lab[k] >= C) { if (lane_valid && row_owned && lane_owned) n_bad++; lab[k] = -1; }
+            const int gx = (X0 + k) >> 2;
+            own[k] = pv[k] && row_owned && gx >= x0 && gx < x0 + RN_X;
+            if (pv[k] && lab[k] >= C) { if (own[k]) n_bad++; lab[k] = -1; }
+            if (!pv[k]) lab[k] = -1;
         }
-        float mk[4];
-        {
-            const float* nm = nmax + wi * TZ_W + l;
-            const float m = fmaxf(fmaxf(fmaxf(nm[0], nm[1]), fmaxf(nm[2], nm[TZ_W])), fmaxf(nm[TZ_W + 1], nm[TZ_W + 2]));
-            mk[0] = mk[1] = mk[2] = mk[3] = m;
-        }
-        float ev[4][CB], Zs[4];
+
+        float sk[4] = {0.f, 0.f, 0.f, 0.f}, Zs[4];
         uint32_t arg[4] = {0, 0, 0, 0};
-        for (int attempt = 0; attempt < 2; ++attempt) {
-            Zs[0] = Zs[1] = Zs[2] = Zs[3] = 0.f;
-            float best[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};
+        pass1<CB, CONF, false>(rc, sk, Zs, arg);
+        bool under = false;
 #pragma unroll
-            for (int c = 0; c < CB; ++c) {
-                const float* q = zp + c * TZ;
-                const float vl = lerp_r(q[0], q[TZ_W], ly), vc = lerp_r(q[1], q[TZ_W + 1], ly), vr = lerp_r(q[2], q[TZ_W + 2], ly);
-                const float dl = vc - vl, dr = vr - vc;
-                float u[4] = {fmaf(0.625f, dl, vl), fmaf(0.875f, dl, vl), fmaf(0.125f, dr, vc), fmaf(0.375f, dr, vc)};
-#pragma unroll
-                for (int k = 0; k < 4; ++k) {
-                    if (CONF && attempt == 0) { if (u[k] > best[k]) { best[k] = u[k]; arg[k] = c; } }
-                    const float e = ex2_approx(u[k] - mk[k]);
-                    ev[k][c] = e;
-                    Zs[k] += e;
-                }
-            }
-            // the bound can sit far above a pixel's true maximum only for wildly varying logits; then redo exactly
-            const bool under = !(Zs[0] > 1e-30f) || !(Zs[1] > 1e-30f) || !(Zs[2] > 1e-30f) || !(Zs[3] > 1e-30f);
-            if (!under || attempt == 1) break;
+        for (int k = 0; k < 4; ++k) under |= pv[k] && !(Zs[k] > 1e-30f);
+        const bool slow = __any_sync(0xffffffffu, under);
+        if (slow) {
+            // exact per-pixel maxima, then the sums again
             float ex[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};
+            const float zero[4] = {0.f, 0.f, 0.f, 0.f};
             for (int c = 0; c < C; ++c) {
-                const float* q = zp + c * TZ;
-                const float vl = lerp_r(q[0], q[TZ_W], ly), vc = lerp_r(q[1], q[TZ_W + 1], ly), vr = lerp_r(q[2], q[TZ_W + 2], ly);
-                const float dl = vc - vl, dr = vr - vc;
-                ex[0] = fmaxf(ex[0], fmaf(0.625f, dl, vl)); ex[1] = fmaxf(ex[1], fmaf(0.875f, dl, vl));
-                ex[2] = fmaxf(ex[2], fmaf(0.125f, dr, vc)); ex[3] = fmaxf(ex[3], fmaf(0.375f, dr, vc));
+                float u[4];
+                pixel_logits<false>(rc, c, zero, u);
+#pragma unroll
+                for (int k = 0; k < 4; ++k) ex[k] = fmaxf(ex[k], u[k]);
             }
 #pragma unroll
-            for (int k = 0; k < 4; ++k) mk[k] = ex[k];
+            for (int k = 0; k < 4; ++k) sk[k] = ex[k];
+            uint32_t dummy[4];
+            pass1<CB, false, true>(rc, sk, Zs, dummy);
         }
 
         // ---- per pixel: loss, 1/Z, the "- onehot" part of the adjoint (integer, exact), confusion
-        float rz[4];
-        const int wy1 = 2 * r + 1, wy0 = 8 - wy1;                // eighths toward node rows i+1 / i
+        float wl[4], wr[4];
+        const int wy1 = 2 * r + 1, wy0 = 8 - wy1;                    // eighths toward node rows i+1 / i
+        const bool fold_l = n == -1, fold_r = n == w - 1;            // clamped borders: the outer node is the inner one
 #pragma unroll
         for (int k = 0; k < 4; ++k) {
-            rz[k] = 0.f;
-            if (lane_valid && lab[k] >= 0) {
-                rz[k] = 1.0f / Zs[k];
-                const float* q = zp + lab[k] * TZ;
-                const float vl = lerp_r(q[0], q[TZ_W], ly), vc = lerp_r(q[1], q[TZ_W + 1], ly), vr = lerp_r(q[2], q[TZ_W + 2], ly);
-                const float ul = k == 0 ? fmaf(0.625f, vc - vl, vl) : k == 1 ? fmaf(0.875f, vc - vl, vl)
-                               : k == 2 ? fmaf(0.125f, vr - vc, vc) : fmaf(0.375f, vr - vc, vc);
-                if (row_owned && lane_owned) {
-                    loss += (__log2f(Zs[k]) + (mk[k] - ul)) * kLn2;
+            float rz = 0.f;
+            if (lab[k] >= 0) {
+                rz = 1.0f / Zs[k];
+                const float* q = rc.za + lab[k] * TZ;
+                const float vl = fmaf(rc.ly, q[TZ_W] - q[0], q[0]), vr = fmaf(rc.ly, q[TZ_W + 1] - q[1], q[1]);
+                const float ul = fmaf((2 * k + 1) * 0.125f, vr - vl, vl) - rc.M - sk[k];
+                if (own[k]) {
+                    loss += (__log2f(Zs[k]) - ul) * kLn2;
                     if (CONF) atomicAdd(a.conf + (int64_t)s * a.conf_stream_stride + lab[k] * C + arg[k], 1ull);
                 }
-                // horizontal eighths: k = 0,1 pull toward (xg-1, xg) with (3,5), (1,7); k = 2,3 toward (xg, xg+1) with (7,1), (5,3)
-                const int wa = k == 0 ? 3 : k == 1 ? 1 : k == 2 ? 7 : 5, wb = 8 - wa;
-                const int ca = k < 2 ? rx_l : rx_c, cb = k < 2 ? rx_c : rx_r;
+                const int wb = 2 * k + 1, wa = 8 - wb;               // eighths toward node columns n+1 / n
                 int* cc = corr + lab[k] * TZ;
-                atomicAdd(cc + ry_top * TZ_W + ca, -wy0 * wa);
-                atomicAdd(cc + ry_top * TZ_W + cb, -wy0 * wb);
-                atomicAdd(cc + ry_bot * TZ_W + ca, -wy1 * wa);
-                atomicAdd(cc + ry_bot * TZ_W + cb, -wy1 * wb);
+                atomicAdd(cc + ry_top * TZ_W + rx_l, -wy0 * wa);
+                atomicAdd(cc + ry_top * TZ_W + rx_r, -wy0 * wb);
+                atomicAdd(cc + ry_bot * TZ_W + rx_l, -wy1 * wa);
+                atomicAdd(cc + ry_bot * TZ_W + rx_r, -wy1 * wb);
             }
+            const float fr = (2 * k + 1) * 0.125f;
+            wl[k] = (fold_l ? 0.f : (fold_r ? 1.0f : 1.0f - fr)) * rz;
+            wr[k] = (fold_r ? 0.f : (fold_l ? 1.0f : fr)) * rz;
         }
-        // ---- B: softmax part of the adjoint
-        // at the clamped left/right border the outer node is the inner one: its weight joins the centre weight
-        const bool fold_l = xg == 0, fold_r = xg == w - 1;
-        const float w0l = fold_l ? 0.f : 0.375f * rz[0], w0c = (fold_l ? 1.0f : 0.625f) * rz[0];
-        const float w1l = fold_l ? 0.f : 0.125f * rz[1], w1c = (fold_l ? 1.0f : 0.875f) * rz[1];
-        const float w2r = fold_r ? 0.f : 0.125f * rz[2], w2c = (fold_r ? 1.0f : 0.875f) * rz[2];
-        const float w3r = fold_r ? 0.f : 0.375f * rz[3], w3c = (fold_r ? 1.0f : 0.625f) * rz[3];
-#pragma unroll
-        for (int c = 0; c < CB; ++c) {
-            const float aL = fmaf(w0l, ev[0][c], w1l * ev[1][c]);
-            const float aR = fmaf(w2r, ev[2][c], w3r * ev[3][c]);
-            const float aC = fmaf(w0c, ev[0][c], fmaf(w1c, ev[1][c], fmaf(w2c, ev[2][c], w3c * ev[3][c])));
-            const float hsum = aC + __shfl_up_sync(0xffffffffu, aR, 1) + __shfl_down_sync(0xffffffffu, aL, 1);
-            top[c] = fmaf(1.0f - ly, hsum, top[c]);
-            bot[c] = fmaf(ly, hsum, bot[c]);
-        }
+        if (slow) pass2<CB, true>(rc, sk, wl, wr, top, bot);
+        else pass2<CB, false>(rc, sk, wl, wr, top, bot);
     }
     // clamped borders in y
     if (i == -1) {
@@ -214,40 +251,43 @@ upsample_ce_rows_kernel(UpsampleCeArgs a)
 #pragma unroll
         for (int c = 0; c < CB; ++c) { top[c] += bot[c]; bot[c] = 0.f; }
     }
-#pragma unroll
-    for (int c = 0; c < CB; ++c)
-        if (c < C) bsh[(wi * C + c) * 32 + l] = bot[c];
     // loss of the block, fixed order
 #pragma unroll
     for (int o = 16; o > 0; o >>= 1) loss += __shfl_xor_sync(0xffffffffu, loss, o);
     if (l == 0) red[wi] = loss;
     if (n_bad) atomicAdd(a.bad, n_bad);
+    __syncthreads();                            // every warp is done reading the tile: reuse it
+#pragma unroll
+    for (int c = 0; c < CB; ++c)
+        if (c < C) bsh[(wi * C + c) * 32 + l] = bot[c];
     __syncthreads();
 
     // ---- node row y0-1+wi (warps 1..RN_Y): own upper part + lower part of the warp above + onehot part
     const float invP = 1.0f / ((float)H * (float)W);
     const int y = i;
-    const bool node_ok = wi >= 1 && y < h && lane_owned;
+    const bool node_ok = wi >= 1 && y < h && node_owned;
+    float dbsum = 0.f;       // lane c ends up with the class-c sum over this warp's nodes
 #pragma unroll
     for (int c = 0; c < CB; ++c) {
         if (c < C) {
             float v = 0.f;
             if (node_ok) {
-                const int cr = corr[c * TZ + (y - (y0 - 1)) * TZ_W + (xg - (x0 - 2))];
+                const int cr = corr[c * TZ + wi * TZ_W + l];
                 v = (top[c] + bsh[((wi - 1) * C + c) * 32 + l] + (float)cr * (1.0f / 64.0f)) * invP;
-                a.dz[((int64_t)s * C + c) * p + (int64_t)y * w + xg] = v;
+                a.dz[((int64_t)s * C + c) * p + (int64_t)y * w + n] = v;
                 if (a.dz_bf16)
-                    a.dz_bf16[((int64_t)s * kClassPad + c) * a.dz_bf16_pitch + (int64_t)y * w + xg] = __float2bfloat16_rn(v);
+                    a.dz_bf16[((int64_t)s * kClassPad + c) * a.dz_bf16_pitch + (int64_t)y * w + n] = __float2bfloat16_rn(v);
             }
 #pragma unroll
             for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
-            if (l == 0) dbs[wi * C + c] = v;
+            if (l == c) dbsum = v;
         }
     }
+    dbs[wi][l] = dbsum;
     __syncthreads();
     for (int c = tid; c < C; c += R_THREADS) {
         float t = 0.f;
-        for (int k = 1; k < R_WARPS; ++k) t += dbs[k * C + c];
+        for (int k = 1; k < R_WARPS; ++k) t += dbs[k][c];
         a.db_part[((int64_t)s * n_blk + blk) * C + c] = t;
     }
     if (tid == 0) {
@@ -260,7 +300,8 @@ upsample_ce_rows_kernel(UpsampleCeArgs a)
 template <int CB>
 size_t rows_smem_bytes(int C)
 {
-    return ((size_t)(CB + C) * TZ + TZ + (size_t)R_WARPS * C * 32 + (size_t)R_WARPS * C) * sizeof(float) + 16;
+    const size_t tile = (size_t)CB * TZ, bsh = (size_t)R_WARPS * C * 32;
+    return ((tile > bsh ? tile : bsh) + (size_t)C * TZ) * sizeof(float) + 16;
 }
 
 template <int CB>
@@ -272,11 +313,19 @@ cudaError_t prepare_cb(int C)
 }
 
 template <int CB>
-void launch_cb(const UpsampleCeArgs& a, cudaStream_t s)
+cudaError_t launch_cb(const UpsampleCeArgs& a, cudaStream_t s)
 {
     dim3 grid((unsigned)((a.w + RN_X - 1) / RN_X), (unsigned)((a.h + RN_Y - 1) / RN_Y), (unsigned)a.S);
     if (a.conf) upsample_ce_rows_kernel<CB, true><<<grid, R_THREADS, rows_smem_bytes<CB>(a.C), s>>>(a);
     else upsample_ce_rows_kernel<CB, false><<<grid, R_THREADS, rows_smem_bytes<CB>(a.C), s>>>(a);
+    return cudaSuccess;
+}
+
+// class-count buckets: the two workload sizes exactly, multiples of four otherwise
+int bucket(int C)
+{
+    if (C == 19 || C == 21) return C;
+    return (C + 3) / 4 * 4;
 }
 
 }  // namespace
@@ -285,32 +334,24 @@ bool upsample_ce_rows_supported(int C) { return C <= 32; }
 
 int upsample_ce_rows_blocks(int h, int w) { return ((h + RN_Y - 1) / RN_Y) * ((w + RN_X - 1) / RN_X); }
 
-cudaError_t prepare_upsample_ce_rows(int C)
-{
-    switch ((C + 3) / 4) {
-        case 1: return prepare_cb<4>(C);
-        case 2: return prepare_cb<8>(C);
-        case 3: return prepare_cb<12>(C);
-        case 4: return prepare_cb<16>(C);
-        case 5: return prepare_cb<20>(C);
-        case 6: return prepare_cb<24>(C);
-        case 7: return prepare_cb<28>(C);
-        default: return prepare_cb<32>(C);
+#define ST_ROWS_DISPATCH(FN, C, ...)                 \
+    switch (bucket(C)) {                             \
+        case 4: return FN<4>(__VA_ARGS__);           \
+        case 8: return FN<8>(__VA_ARGS__);           \
+        case 12: return FN<12>(__VA_ARGS__);         \
+        case 16: return FN<16>(__VA_ARGS__);         \
+        case 19: return FN<19>(__VA_ARGS__);         \
+        case 20: return FN<20>(__VA_ARGS__);         \
+        case 21: return FN<21>(__VA_ARGS__);         \
+        case 24: return FN<24>(__VA_ARGS__);         \
+        case 28: return FN<28>(__VA_ARGS__);         \
+        default: return FN<32>(__VA_ARGS__);         \
     }
-}
 
-void launch_upsample_ce_rows(const UpsampleCeArgs& a, cudaStream_t s)
-{
-    switch ((a.C + 3) / 4) {
-        case 1: launch_cb<4>(a, s); break;
-        case 2: launch_cb<8>(a, s); break;
-        case 3: launch_cb<12>(a, s); break;
-        case 4: launch_cb<16>(a, s); break;
-        case 5: launch_cb<20>(a, s); break;
-        case 6: launch_cb<24>(a, s); break;
-        case 7: launch_cb<28>(a, s); break;
-        default: launch_cb<32>(a, s); break;
-    }
-}
+cudaError_t prepare_upsample_ce_rows(int C) { ST_ROWS_DISPATCH(prepare_cb, C, C) }
+
+cudaError_t launch_rows_dispatch(const UpsampleCeArgs& a, cudaStream_t s) { ST_ROWS_DISPATCH(launch_cb, a.C, a, s) }
+
+void launch_upsample_ce_rows(const UpsampleCeArgs& a, cudaStream_t s) { launch_rows_dispatch(a, s); }
 
 }  // namespace st
