@@ -14,7 +14,7 @@
 //   pass 1  each lane interpolates its own node column vertically, takes the right neighbour's by
 //           shuffle, interpolates its four pixels horizontally, and sums exp2(u - M) over the classes
 //           (logits are pre-scaled by log2 e; M is the largest logit of the warp's two node rows);
-//   pass 2  the exponentials are formed again (cheaper than keeping 4 x C registers alive: three
+//   pass 2  the exponentials are formed again (cheaper than keeping 4 x C registers alive: two
 //           or three blocks per SM stay resident), multiplied by the adjoint interpolation weights / Z, the
 //           right-hand part is handed to the next lane by shuffle, and the row is added into two
 //           per-class accumulators: toward the upper and the lower node row.
@@ -30,7 +30,7 @@ namespace {
 
 constexpr int RN_Y = 7, RN_X = 30;
 constexpr int R_WARPS = RN_Y + 1, R_THREADS = R_WARPS * 32;
-constexpr int TZ_H = RN_Y + 2, TZ_W = 32, TZ = TZ_H * TZ_W;
+constexpr int TZ_H = RN_Y + 2, TZ_W = 36, TZ = TZ_H * TZ_W;   // tile rows hold 36 columns: 32 used, starting at a multiple of 4
 constexpr float kLog2e = 1.4426950408889634f, kLn2 = 0.6931471805599453f;
 
 __device__ __forceinline__ float ex2_approx(float x)
@@ -41,7 +41,7 @@ __device__ __forceinline__ float ex2_approx(float x)
 }
 
 struct RowCtx {
-    const float* za;     // zt + wi*TZ_W + l : own column, upper node row, class 0
+    const float* za;     // own column, upper node row, class 0
     float ly;            // weight toward the lower node row
     float M;             // warp-uniform shift
 };
@@ -101,9 +101,9 @@ upsample_ce_rows_kernel(UpsampleCeArgs a)
 {
     extern __shared__ __align__(16) float smem_r[];
     const int C = a.C, h = a.h, w = a.w, H = h * kUp, W = w * kUp;
-    float* zt = smem_r;                         // [CB][TZ_H][32]   logits * log2(e), borders replicated; classes >= C
+    float* zt = smem_r;                         // [CB][TZ_H][36]   logits * log2(e), borders replicated; classes >= C
                                                 //                  hold -1e30 (their exponentials are 0)
-    int* corr = (int*)(zt + CB * TZ);           // [C][TZ_H][32]    -64 * (adjoint of onehot)
+    int* corr = (int*)(zt + CB * TZ);           // [C][TZ_H][36]    -64 * (adjoint of onehot)
     float* bsh = zt;                            // [R_WARPS][C][32] lower-row accumulators (reuses the tile once the rows are done)
     __shared__ float red[R_WARPS];
     __shared__ float dbs[R_WARPS][32];
@@ -115,25 +115,40 @@ upsample_ce_rows_kernel(UpsampleCeArgs a)
     const uint8_t* labels = a.labels + (int64_t)s * H * W;
     const int tid = threadIdx.x, wi = tid >> 5, l = tid & 31;
 
-    // ---- tile: node rows y0-1 .. y0+RN_Y, node columns x0-1 .. x0+30 (clamped), scaled by log2(e).
-    // Fully unrolled so that all of a thread's loads are in flight together.
+    // ---- tile: node rows y0-1 .. y0+RN_Y, node columns xa .. xa+35 where xa = (x0-1) rounded down to a
+    // multiple of 4 (so that rows are fetched as 16-byte vectors), clamped at the borders, scaled by
+    // log2(e).  Fully unrolled: all of a thread's loads are in flight together.
+    const bool vec_ok = (w % 4 == 0) && ((uintptr_t)z % 16 == 0);
+    const int xa = vec_ok ? ((x0 - 1) & ~3) : x0 - 1;      // x0-1 >= -1; (-1 & ~3) = -4
+    const int off = (x0 - 1) - xa;                         // column of node x0-1 inside the tile
     {
-        constexpr int kIter = (CB * TZ + R_THREADS - 1) / R_THREADS;
-        float v[kIter];
+        constexpr int kQuads = TZ / 4;                     // 16-byte groups per class
+        constexpr int kIter = (CB * kQuads + R_THREADS - 1) / R_THREADS;
+        float4 v[kIter];
 #pragma unroll
         for (int it = 0; it < kIter; ++it) {
             const int e = tid + it * R_THREADS;
-            const int c = e / TZ, n = e % TZ;
-            const int yy = min(max(y0 - 1 + n / TZ_W, 0), h - 1), xx = min(max(x0 - 1 + n % TZ_W, 0), w - 1);
-            v[it] = (e < CB * TZ && c < C) ? __ldg(z + (int64_t)c * p + (int64_t)yy * w + xx) * kLog2e : -1e30f;
+            const int c = e / kQuads, q = e % kQuads;
+            const int yy = min(max(y0 - 1 + q / (TZ_W / 4), 0), h - 1), xq = xa + 4 * (q % (TZ_W / 4));
+            float4 t = make_float4(-1e30f, -1e30f, -1e30f, -1e30f);
+            if (e < CB * kQuads && c < C) {
+                const float* row = z + (int64_t)c * p + (int64_t)yy * w;
+                if (vec_ok && xq >= 0 && xq + 3 < w) t = __ldg(reinterpret_cast<const float4*>(row + xq));
+                else {
+                    t.x = __ldg(row + min(max(xq, 0), w - 1));     t.y = __ldg(row + min(max(xq + 1, 0), w - 1));
+                    t.z = __ldg(row + min(max(xq + 2, 0), w - 1)); t.w = __ldg(row + min(max(xq + 3, 0), w - 1));
+                }
+                t.x *= kLog2e; t.y *= kLog2e; t.z *= kLog2e; t.w *= kLog2e;
+            }
+            v[it] = t;
         }
 #pragma unroll
         for (int it = 0; it < kIter; ++it) {
             const int e = tid + it * R_THREADS;
-            if (e < CB * TZ) zt[e] = v[it];
+            if (e < CB * kQuads) reinterpret_cast<float4*>(zt)[e] = v[it];
         }
     }
-    for (int e = tid; e < C * TZ; e += R_THREADS) corr[e] = 0;
+    for (int e = tid; e < C * TZ / 4; e += R_THREADS) reinterpret_cast<int4*>(corr)[e] = make_int4(0, 0, 0, 0);
     __syncthreads();
 
     const int i = y0 - 1 + wi;                  // cell row: frame rows 4i+2 .. 4i+5, node rows (i, i+1)
@@ -143,10 +158,10 @@ upsample_ce_rows_kernel(UpsampleCeArgs a)
     const bool node_owned = l >= 1 && l <= RN_X && n < w;
     // tile coordinates of the (clamped) nodes this lane's pixels pull toward
     const int ry_top = min(max(i, 0), h - 1) - (y0 - 1), ry_bot = min(max(i + 1, 0), h - 1) - (y0 - 1);
-    const int rx_l = min(max(n, 0), w - 1) - (x0 - 1), rx_r = min(max(n + 1, 0), w - 1) - (x0 - 1);
+    const int rx_l = min(max(n, 0), w - 1) - xa, rx_r = min(max(n + 1, 0), w - 1) - xa;
 
     RowCtx rc;
-    rc.za = zt + wi * TZ_W + l;
+    rc.za = zt + wi * TZ_W + off + l;
     rc.ly = 0.f;
     {
         float m = -INFINITY;
@@ -214,6 +229,8 @@ upsample_ce_rows_kernel(UpsampleCeArgs a)
 
         // ---- per pixel: loss, 1/Z, the "- onehot" part of the adjoint (integer, exact), confusion
         float wl[4], wr[4];
+        // four valid pixels with one label (the usual case): their onehot parts add up to 16 eighths per side
+        const bool same_label = lab[0] >= 0 && lab[0] == lab[1] && lab[1] == lab[2] && lab[2] == lab[3];
         const int wy1 = 2 * r + 1, wy0 = 8 - wy1;                    // eighths toward node rows i+1 / i
         const bool fold_l = n == -1, fold_r = n == w - 1;            // clamped borders: the outer node is the inner one
 #pragma unroll
@@ -228,16 +245,25 @@ upsample_ce_rows_kernel(UpsampleCeArgs a)
                     loss += (__log2f(Zs[k]) - ul) * kLn2;
                     if (CONF) atomicAdd(a.conf + (int64_t)s * a.conf_stream_stride + lab[k] * C + arg[k], 1ull);
                 }
-                const int wb = 2 * k + 1, wa = 8 - wb;               // eighths toward node columns n+1 / n
-                int* cc = corr + lab[k] * TZ;
-                atomicAdd(cc + ry_top * TZ_W + rx_l, -wy0 * wa);
-                atomicAdd(cc + ry_top * TZ_W + rx_r, -wy0 * wb);
-                atomicAdd(cc + ry_bot * TZ_W + rx_l, -wy1 * wa);
-                atomicAdd(cc + ry_bot * TZ_W + rx_r, -wy1 * wb);
+                if (!same_label) {
+                    const int wb = 2 * k + 1, wa = 8 - wb;           // eighths toward node columns n+1 / n
+                    int* cc = corr + lab[k] * TZ;
+                    atomicAdd(cc + ry_top * TZ_W + rx_l, -wy0 * wa);
+                    atomicAdd(cc + ry_top * TZ_W + rx_r, -wy0 * wb);
+                    atomicAdd(cc + ry_bot * TZ_W + rx_l, -wy1 * wa);
+                    atomicAdd(cc + ry_bot * TZ_W + rx_r, -wy1 * wb);
+                }
             }
             const float fr = (2 * k + 1) * 0.125f;
             wl[k] = (fold_l ? 0.f : (fold_r ? 1.0f : 1.0f - fr)) * rz;
             wr[k] = (fold_r ? 0.f : (fold_l ? 1.0f : fr)) * rz;
+        }
+        if (same_label) {
+            int* cc = corr + lab[0] * TZ;
+            atomicAdd(cc + ry_top * TZ_W + rx_l, -wy0 * 16);
+            atomicAdd(cc + ry_top * TZ_W + rx_r, -wy0 * 16);
+            atomicAdd(cc + ry_bot * TZ_W + rx_l, -wy1 * 16);
+            atomicAdd(cc + ry_bot * TZ_W + rx_r, -wy1 * 16);
         }
         if (slow) pass2<CB, true>(rc, sk, wl, wr, top, bot);
         else pass2<CB, false>(rc, sk, wl, wr, top, bot);
@@ -272,7 +298,7 @@ upsample_ce_rows_kernel(UpsampleCeArgs a)
         if (c < C) {
             float v = 0.f;
             if (node_ok) {
-                const int cr = corr[c * TZ + wi * TZ_W + l];
+                const int cr = corr[c * TZ + wi * TZ_W + off + l];
                 v = (top[c] + bsh[((wi - 1) * C + c) * 32 + l] + (float)cr * (1.0f / 64.0f)) * invP;
                 a.dz[((int64_t)s * C + c) * p + (int64_t)y * w + n] = v;
                 if (a.dz_bf16)
