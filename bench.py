@@ -321,7 +321,7 @@ def run_ours(args, cfg):
                 elif name in ("tc_fwd3x3", "tc_wgrad3x3"):
                     k.update(bound="tensor", achieved=2.0 * S * p * cfg.c_hidden * cfg.c_in * 9 / ms / 1e9, peak=tensor_peak,
                              unit="TFLOP/s")
-                elif name == "dgrad_relu":
+                elif name == "tc_dgrad":
                     k.update(bound="hbm", achieved=S * (2 * p * cfg.c_hidden * 2 + C * p * 4) / ms / 1e6, peak=hbm, unit="GB/s")
                 else:
                     k.update(bound="latency")

@@ -276,8 +276,7 @@ def gradients(head: Head, feat: np.ndarray, labels: np.ndarray):
         return loss, grad, mask
     (W1, b1), (W2, b2) = layers
     dW2, db2 = conv_wgrad(Hd, head._q(dz), 1)
-    # the gradient handed to the hidden layer is formed from unrounded operands in every mode
-    dH = conv1x1_dgrad(W2.reshape(W2.shape[0], W2.shape[1]), dz)
+    dH = conv1x1_dgrad(head._q(W2.reshape(W2.shape[0], W2.shape[1])), head._q(dz))
     relu_mask_(dH, Hd)
     dW1, db1 = conv_wgrad(x, head._q(dH), 3)
     if head.quantize_bf16:

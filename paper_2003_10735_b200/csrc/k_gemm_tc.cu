@@ -6,7 +6,7 @@
 //   fwd 1x1   z[c][pix]       = b[c] + sum_k A[pix][k] W[c][k]                 A = features or hidden
 //   fwd 3x3   Hd[pix][co]     = ReLU(b1[co] + sum_{tap,ci} X[pix+tap][ci] W1[tap][co][ci])
 //   wgrad 1x1 dW[c][k]        = sum_pix dz[c][pix] A[pix][k]                   split over pixel ranges
-//   dgrad     dHd[pix][k]     = [Hd[pix][k] > 0] sum_c dz[c][pix] W2[c][k]     (fp32 FMA, bf16 out)
+//   dgrad     dHd[pix][k]     = [Hd[pix][k] > 0] sum_c dz[c][pix] W2[c][k]     (bf16 out)
 //   wgrad 3x3 dW1[tap][co][ci]= sum_pix dHd[pix][co] X[pix+tap][ci]            split over pixel ranges
 //
 // Pixel-major activations [pix][channel] are K-major operands when the GEMM reduces over channels
@@ -393,61 +393,114 @@ tc_wgrad3x3_kernel(const __grid_constant__ CUtensorMap tmA,   // X   {Cin, w, h,
 }
 
 // ------------------------------------------------------------------------------------------------
-// dgrad through the 1x1 output layer with the ReLU mask of the hidden activation, fp32 FMA from the
-// unrounded dz and the fp32 master weight; output rounded to bf16 (it is a GEMM operand next).
-// Also emits per-block partial sums of the (unrounded) result over pixels: the bias gradient of the
-// 3x3 layer.  Block = 64 pixels x all hidden channels; thread = one channel pair x a share of the pixels.
+// dgrad through the 1x1 output layer with the ReLU mask of the hidden activation:
+//   dHd[pix][k] = [Hd[pix][k] > 0] * sum_c dz[c][pix] * W2[c][k]
+// One 128-pixel tile per block, N = Ch, K = 32 class rows (rows >= C are zero in both operands).
+// dz rows [c][pix] and weight rows [c][k] are both contiguous along the non-reduced index, so both are
+// MN-major operands.  The epilogue applies the mask, writes bf16 (a GEMM operand next) and emits the
+// block's sums over pixels of the unrounded result: the bias gradient of the 3x3 layer.
 // ------------------------------------------------------------------------------------------------
-constexpr int kDgradPix = 64;
-
-__global__ void __launch_bounds__(256)
-dgrad_relu_kernel(const float* __restrict__ theta, int64_t n_params, int64_t w2_off,
-                  const float* __restrict__ dz,        // [S][C][p]
-                  const bf16* __restrict__ hidden,     // [S][p][Ch]
-                  bf16* __restrict__ dhidden,          // [S][p][Ch]
-                  float* __restrict__ b1_partials,     // [S][n_blocks][Ch]
-                  int C, int Ch, int p)
+__global__ void __launch_bounds__(kThreadsTc)
+tc_dgrad_kernel(const __grid_constant__ CUtensorMap tmA,   // dz  {p, 32, S}  box {64, 32, 1}
+                const __grid_constant__ CUtensorMap tmB,   // W2  {Ch, 32, S} box {64, 32, 1}
+                const bf16* __restrict__ hidden,            // [S][p][Ch]
+                bf16* __restrict__ dhidden,                 // [S][p][Ch]
+                float* __restrict__ b1_partials,            // [S][n_blocks][Ch]
+                int Ch, int p, int tmem_cols, unsigned int* err)
 {
-    extern __shared__ float sm[];
-    float* w2 = sm;                     // [C][Ch]
-    float* dzt = w2 + C * Ch;           // [C][kDgradPix]
-    float* red = dzt + C * kDgradPix;   // [groups][Ch]
-    const int s = blockIdx.y, blk = blockIdx.x, pix0 = blk * kDgradPix;
-    const int pairs = Ch / 2, groups = 256 / pairs;    // Ch in {64,128,192,256} -> groups 8, 4, 2, 2
-    const float* W2 = theta + (int64_t)s * n_params + w2_off;
-    for (int i = threadIdx.x; i < C * Ch; i += 256) w2[i] = __ldg(W2 + i);
-    for (int i = threadIdx.x; i < C * kDgradPix; i += 256) {
-        const int c = i / kDgradPix, q = i % kDgradPix;
-        dzt[i] = (pix0 + q < p) ? __ldg(dz + ((int64_t)s * C + c) * p + pix0 + q) : 0.f;
+    extern __shared__ uint8_t smem_raw[];
+    uint8_t* smem = align_smem(smem_raw);
+    const uint32_t a_base = smem_u32(smem);
+    const uint32_t blk_bytes = kClassPad * 128;                 // 32 class rows x 64 elements
+    const uint32_t b_base = a_base + 2 * blk_bytes;
+    const int b_blocks = Ch / kBlockK;
+    float* red = reinterpret_cast<float*>(smem + 2 * blk_bytes + b_blocks * blk_bytes);   // [128][33]
+    __shared__ float part[4][32];
+    __shared__ __align__(8) uint64_t full, done;
+    __shared__ uint32_t tmem_slot;
+    const int tid = threadIdx.x, warp = tid >> 5;
+    const int s = blockIdx.y, pix0 = blockIdx.x * kTileM;
+
+    if (warp == 0) tmem_alloc(smem_u32(&tmem_slot), tmem_cols);
+    if (tid == 0) {
+        mbar_init(smem_u32(&full), 1); mbar_init(smem_u32(&done), 1);
+        fence_barrier_init();
     }
+    tc_fence_before_sync();
     __syncthreads();
-    const int cp = threadIdx.x % pairs, g = threadIdx.x / pairs;
-    if (g < groups) {
-        float sum0 = 0.f, sum1 = 0.f;
-        for (int q = g; q < kDgradPix; q += groups) {
-            const int pix = pix0 + q;
-            if (pix >= p) break;
-            float a0 = 0.f, a1 = 0.f;
-            for (int c = 0; c < C; ++c) {
-                const float d = dzt[c * kDgradPix + q];
-                const float2 wv = *reinterpret_cast<const float2*>(w2 + c * Ch + 2 * cp);
-                a0 = fmaf(d, wv.x, a0); a1 = fmaf(d, wv.y, a1);
-            }
-            const int64_t off = ((int64_t)s * p + pix) * Ch + 2 * cp;
-            const __nv_bfloat162 hv = *reinterpret_cast<const __nv_bfloat162*>(hidden + off);
-            if (!(__low2float(hv) > 0.f)) a0 = 0.f;
-            if (!(__high2float(hv) > 0.f)) a1 = 0.f;
-            *reinterpret_cast<__nv_bfloat162*>(dhidden + off) = __floats2bfloat162_rn(a0, a1);
-            sum0 += a0; sum1 += a1;
+    tc_fence_after_sync();
+    const uint32_t tmem = tmem_slot;
+    bool ok = true;
+
+    if (tid == 0) {
+        const uint32_t bar = smem_u32(&full);
+        mbar_expect_tx(bar, (2 + b_blocks) * blk_bytes);
+        tma_load_3d(a_base, &tmA, bar, pix0, 0, s);
+        tma_load_3d(a_base + blk_bytes, &tmA, bar, pix0 + 64, 0, s);
+        for (int cb = 0; cb < b_blocks; ++cb) tma_load_3d(b_base + cb * blk_bytes, &tmB, bar, cb * kBlockK, 0, s);
+    } else if (tid == 32) {
+        const uint32_t idesc = instr_desc(kTileM, Ch, 1, 1);
+        ok = mbar_wait(smem_u32(&full), 0, err, kWaitFull);
+        if (ok) {
+            tc_fence_after_sync();
+#pragma unroll
+            for (int j = 0; j < kClassPad / 16; ++j)
+                umma(tmem, smem_desc(a_base + j * (16 * 128), blk_bytes, 1024), smem_desc(b_base + j * (16 * 128), blk_bytes, 1024),
+                     idesc, j != 0);
         }
-        red[g * Ch + 2 * cp] = sum0; red[g * Ch + 2 * cp + 1] = sum1;
+        umma_commit(smem_u32(&done));
     }
+    __syncwarp();
+    ok = mbar_wait(smem_u32(&done), 0, err, kWaitDone);
+    tc_fence_after_sync();
+    ok = __syncthreads_and(ok);          // the epilogue below synchronises the block: all or none
+    if (ok) {
+        const int pix = pix0 + tid;
+        const bool in = pix < p;
+        const int64_t row = ((int64_t)s * p + (in ? pix : 0)) * Ch;
+        for (int n0 = 0; n0 < Ch; n0 += 32) {
+            float v[32];
+            tmem_ld_32x32(tmem + ((uint32_t)(warp * 32) << 16) + n0, v);
+            if (in) {
+                uint4 hv[4], out[4];
+#pragma unroll
+                for (int k = 0; k < 4; ++k) hv[k] = __ldg(reinterpret_cast<const uint4*>(hidden + row + n0) + k);
+                const __nv_bfloat162* h2 = reinterpret_cast<const __nv_bfloat162*>(hv);
+                __nv_bfloat162* o2 = reinterpret_cast<__nv_bfloat162*>(out);
+#pragma unroll
+                for (int k = 0; k < 16; ++k) {
+                    if (!(__low2float(h2[k]) > 0.f)) v[2 * k] = 0.f;
+                    if (!(__high2float(h2[k]) > 0.f)) v[2 * k + 1] = 0.f;
+                    o2[k] = __floats2bfloat162_rn(v[2 * k], v[2 * k + 1]);
+                }
+#pragma unroll
+                for (int k = 0; k < 4; ++k) reinterpret_cast<uint4*>(dhidden + row + n0)[k] = out[k];
+            } else {
+#pragma unroll
+                for (int k = 0; k < 32; ++k) v[k] = 0.f;
+            }
+            // sums over the tile's pixels, fixed order: rows -> four quarter sums -> one
+#pragma unroll
+            for (int k = 0; k < 32; ++k) red[tid * 33 + k] = v[k];
+            __syncthreads();
+            {
+                const int ch = tid & 31, q = tid >> 5;
+                float t = 0.f;
+#pragma unroll 8
+                for (int r = 0; r < 32; ++r) t += red[(q * 32 + r) * 33 + ch];
+                part[q][ch] = t;
+            }
+            __syncthreads();
+            if (tid < 32)
+                b1_partials[((int64_t)s * gridDim.x + blockIdx.x) * Ch + n0 + tid] =
+                    (part[0][tid] + part[1][tid]) + (part[2][tid] + part[3][tid]);
+        }
+    } else {
+        drain_after_error();
+    }
+    tc_fence_before_sync();
     __syncthreads();
-    for (int k = threadIdx.x; k < Ch; k += 256) {
-        float t = 0.f;
-        for (int gg = 0; gg < groups; ++gg) t += red[gg * Ch + k];
-        b1_partials[((int64_t)s * gridDim.x + blk) * Ch + k] = t;
-    }
+    if (warp == 0) tmem_dealloc(tmem, tmem_cols);
 }
 
 // ---- host side -------------------------------------------------------------------------------------
@@ -526,7 +579,7 @@ int tc_wgrad_splits(int layer, int c_in, int c_hidden, int h, int w)
     return n;
 }
 
-int tc_b1_partials(int h, int w) { return (int)(((int64_t)h * w + kDgradPix - 1) / kDgradPix); }
+int tc_b1_partials(int h, int w) { return (int)(((int64_t)h * w + kTileM - 1) / kTileM); }
 
 int tc_dz_pitch(int h, int w) { return (int)((((int64_t)h * w + 63) / 64) * 64); }
 
@@ -583,7 +636,7 @@ TcPlan* tc_plan_create(const TcBuffers& b, char* err, size_t err_len)
         P->cols1 = pow2_cols(m_in * b.c_hidden);
         P->smem_fwd3 = 4 * ((size_t)kTileM * 128 + (size_t)b.c_hidden * 128) + kSmemAlign;
         P->smem_wg3 = 3 * ((size_t)(m_in * 2 + b.c_hidden / kBlockK) * kChunkPix * 128) + kSmemAlign;
-        P->smem_dgrad = ((size_t)b.C * b.c_hidden + (size_t)b.C * kDgradPix + 512) * sizeof(float);
+        P->smem_dgrad = (size_t)(2 + b.c_hidden / kBlockK) * kClassPad * 128 + (size_t)kTileM * 33 * sizeof(float) + kSmemAlign;
         if (P->cols1 > 512) {
             snprintf(err, err_len, "c_in %d with c_hidden %d needs %d TMEM columns (> 512)", b.c_in, b.c_hidden, P->cols1);
             delete P; return nullptr;
@@ -600,7 +653,7 @@ TcPlan* tc_plan_create(const TcBuffers& b, char* err, size_t err_len)
     if (b.c_hidden) {
         if (e == cudaSuccess) e = cudaFuncSetAttribute(tc_fwd3x3_kernel<4>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)P->smem_fwd3);
         if (e == cudaSuccess) e = cudaFuncSetAttribute(tc_wgrad3x3_kernel<3>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)P->smem_wg3);
-        if (e == cudaSuccess) e = cudaFuncSetAttribute(dgrad_relu_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)P->smem_dgrad);
+        if (e == cudaSuccess) e = cudaFuncSetAttribute(tc_dgrad_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)P->smem_dgrad);
     }
     if (e != cudaSuccess) { snprintf(err, err_len, "shared-memory attribute: %s", cudaGetErrorString(e)); delete P; return nullptr; }
     return P;
@@ -637,9 +690,9 @@ int tc_backward(const TcPlan* P, cudaStream_t s, StageTimer* t)
     ++n;
     if (b.c_hidden) {
         const int blocks = tc_b1_partials(b.h, b.w);
-        dgrad_relu_kernel<<<dim3(blocks, b.S), 256, P->smem_dgrad, s>>>(
-            b.theta, b.n_params, b.w2_off, b.dz, b.hidden, b.dhidden, b.b1_partials, b.C, b.c_hidden, P->p);
-        if (t) t->mark("dgrad_relu", s);
+        tc_dgrad_kernel<<<dim3(blocks, b.S), kThreadsTc, P->smem_dgrad, s>>>(
+            P->dz_map, P->w2_map, b.hidden, b.dhidden, b.b1_partials, b.c_hidden, P->p, pow2_cols(b.c_hidden), b.err);
+        if (t) t->mark("tc_dgrad", s);
         tc_wgrad3x3_kernel<3><<<dim3(9 * P->split1, b.S), kThreadsTc, P->smem_wg3, s>>>(
             P->x_wg3, P->dh_wg3, b.w1_partials, b.c_in, b.c_hidden, b.h, b.w, P->chunks1, P->per1, P->split1,
             P->cols1, b.err);

@@ -22,53 +22,67 @@ __device__ __forceinline__ void apply_update(const UpdateArgs& a, int64_t gi, fl
 // Parameter blocks: a block covers kUpdThreads / G consecutive parameters; the G thread groups of a
 // block each sum every G-th split-K partial of "their" parameter (coalesced along the parameters),
 // the group sums are added in group order through shared memory, and group 0 applies the update.
-template <int G>
+template <int G, int E>
 __global__ void __launch_bounds__(kUpdThreads)
 sgd_update_kernel(UpdateArgs a, int n_param_blocks)
 {
-    constexpr int kPer = kUpdThreads / G;
+    constexpr int kRow = kUpdThreads / G;      // consecutive parameters covered by one thread group
+    constexpr int kPer = kRow * E;             // parameters per block
     __shared__ float part[G][kPer];
     const int s = blockIdx.y;
     const int64_t base = (int64_t)s * a.n_params;
     if ((int)blockIdx.x < n_param_blocks) {
-        const int e_in_block = threadIdx.x % kPer, g = threadIdx.x / kPer;
-        const int64_t i = (int64_t)blockIdx.x * kPer + e_in_block;
-        int layer = -1;
-        bool is_weight = false;
-        if (i < a.n_params) {
-            for (int L = 0; L < a.n_layers; ++L) {
-                const LayerUpdate& ly = a.layer[L];
-                const int64_t nw = (int64_t)ly.cout * ly.cin * ly.taps;
-                if (i >= ly.w_off && i < ly.w_off + nw) { layer = L; is_weight = true; }
-                if (i >= ly.b_off && i < ly.b_off + ly.cout) { layer = L; is_weight = false; }
-            }
-        }
-        float sum = 0.f;
-        bool has_partials = false;
-        if (layer >= 0 && is_weight && a.layer[layer].w_partials) {
-            const LayerUpdate& ly = a.layer[layer];
-            has_partials = true;
-            const float* src = ly.w_partials + (int64_t)s * ly.w_stream_stride + (i - ly.w_off);
-            for (int k = g; k < ly.n_split; k += G) sum += __ldg(src + (int64_t)k * ly.w_split_stride);
-        }
-        part[g][e_in_block] = sum;
-        __syncthreads();
-        if (g != 0 || layer < 0) return;
-        const LayerUpdate& ly = a.layer[layer];
-        if (is_weight) {
-            float gr;
-            if (has_partials) {
-                gr = 0.f;
+        const int col = threadIdx.x % kRow, g = threadIdx.x / kRow;
+        int layer[E];
+        bool is_weight[E], has_partials[E];
+        float sum[E];
+        // E parameters per thread, all of their split-K loads issued before any is consumed
 #pragma unroll
-                for (int k = 0; k < G; ++k) gr += part[k][e_in_block];
-            } else {
-                gr = a.grad[base + i];
+        for (int e = 0; e < E; ++e) {
+            const int64_t i = (int64_t)blockIdx.x * kPer + e * kRow + col;
+            layer[e] = -1; is_weight[e] = false; has_partials[e] = false; sum[e] = 0.f;
+            if (i < a.n_params) {
+                for (int L = 0; L < a.n_layers; ++L) {
+                    const LayerUpdate& ly = a.layer[L];
+                    const int64_t nw = (int64_t)ly.cout * ly.cin * ly.taps;
+                    if (i >= ly.w_off && i < ly.w_off + nw) { layer[e] = L; is_weight[e] = true; }
+                    if (i >= ly.b_off && i < ly.b_off + ly.cout) { layer[e] = L; is_weight[e] = false; }
+                }
             }
-            apply_update(a, base + i, gr);
-            if (ly.shadow) ly.shadow[(int64_t)s * ly.shadow_stream_stride + (i - ly.w_off)] = __float2bfloat16_rn(a.theta[base + i]);
-        } else if (!ly.b_partials) {
-            apply_update(a, base + i, a.grad[base + i]);
-        }   // biases with partial sums are finished by the reduction warps below
+            if (layer[e] >= 0 && is_weight[e] && a.layer[layer[e]].w_partials) {
+                const LayerUpdate& ly = a.layer[layer[e]];
+                has_partials[e] = true;
+                const float* src = ly.w_partials + (int64_t)s * ly.w_stream_stride + (i - ly.w_off);
+                float t = 0.f;
+#pragma unroll 4
+                for (int k = g; k < ly.n_split; k += G) t += __ldg(src + (int64_t)k * ly.w_split_stride);
+                sum[e] = t;
+            }
+        }
+#pragma unroll
+        for (int e = 0; e < E; ++e) part[g][e * kRow + col] = sum[e];
+        __syncthreads();
+        if (g != 0) return;
+#pragma unroll
+        for (int e = 0; e < E; ++e) {
+            if (layer[e] < 0) continue;
+            const int64_t i = (int64_t)blockIdx.x * kPer + e * kRow + col;
+            const LayerUpdate& ly = a.layer[layer[e]];
+            if (is_weight[e]) {
+                float gr;
+                if (has_partials[e]) {
+                    gr = 0.f;
+#pragma unroll
+                    for (int k = 0; k < G; ++k) gr += part[k][e * kRow + col];
+                } else {
+                    gr = a.grad[base + i];
+                }
+                apply_update(a, base + i, gr);
+                if (ly.shadow) ly.shadow[(int64_t)s * ly.shadow_stream_stride + (i - ly.w_off)] = __float2bfloat16_rn(a.theta[base + i]);
+            } else if (!ly.b_partials) {
+                apply_update(a, base + i, a.grad[base + i]);
+            }   // biases with partial sums are finished by the reduction warps below
+        }
         return;
     }
     // ---- reduction warps: one warp per bias element that has partial sums, plus one for the loss
@@ -109,13 +123,16 @@ void launch_sgd_update(const UpdateArgs& a, cudaStream_t s)
         if (a.layer[L].w_partials && a.layer[L].n_split > max_split) max_split = a.layer[L].n_split;
     }
     const int n_red_blocks = (items + kUpdThreads / 32 - 1) / (kUpdThreads / 32);
-    const int G = max_split >= 32 ? 8 : (max_split >= 4 ? 4 : 1);
-    const int per = kUpdThreads / G;
+    // few parameters with many splits: 8 groups, 1 parameter per thread; many parameters: 4 groups x 4 parameters
+    const bool big = a.n_params > 65536;
+    const int G = max_split <= 1 ? 1 : (big ? 4 : 8), E = big ? 4 : 1;
+    const int per = kUpdThreads / G * E;
     const int n_param_blocks = (int)((a.n_params + per - 1) / per);
     const dim3 grid((unsigned)(n_param_blocks + n_red_blocks), (unsigned)a.S);
-    if (G == 8) sgd_update_kernel<8><<<grid, kUpdThreads, 0, s>>>(a, n_param_blocks);
-    else if (G == 4) sgd_update_kernel<4><<<grid, kUpdThreads, 0, s>>>(a, n_param_blocks);
-    else sgd_update_kernel<1><<<grid, kUpdThreads, 0, s>>>(a, n_param_blocks);
+    if (G == 1 && E == 1) sgd_update_kernel<1, 1><<<grid, kUpdThreads, 0, s>>>(a, n_param_blocks);
+    else if (G == 1) sgd_update_kernel<1, 4><<<grid, kUpdThreads, 0, s>>>(a, n_param_blocks);
+    else if (G == 8) sgd_update_kernel<8, 1><<<grid, kUpdThreads, 0, s>>>(a, n_param_blocks);
+    else sgd_update_kernel<4, 4><<<grid, kUpdThreads, 0, s>>>(a, n_param_blocks);
 }
 
 __global__ void refresh_shadow_kernel(UpdateArgs a)

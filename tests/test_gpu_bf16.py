@@ -165,7 +165,7 @@ def test_hidden_gradient_and_relu_mask():
     dz = st.st_read_tensor(ctx, 0, st.ST_TENSOR_LOGIT_GRAD).reshape(C, h, w)
     dh = st.st_read_tensor(ctx, 0, st.ST_TENSOR_HIDDEN_GRAD).reshape(ch, h, w)
     W2 = theta[ch * c_in * 9 + ch: ch * c_in * 9 + ch + C * ch].reshape(C, ch)
-    ref = oracle.conv1x1_dgrad(W2, dz)
+    ref = oracle.conv1x1_dgrad(oracle.round_bf16(W2), oracle.round_bf16(dz))     # both GEMM operands are bf16
     oracle.relu_mask_(ref, np.ascontiguousarray(hd))
     assert (dh[hd <= 0] == 0).all()
     np.testing.assert_allclose(dh, oracle.round_bf16(ref), rtol=2.0 ** -7, atol=1e-12)
