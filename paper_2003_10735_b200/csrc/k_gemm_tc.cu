@@ -414,8 +414,7 @@ tc_dgrad_kernel(const __grid_constant__ CUtensorMap tmA,   // dz  {p, 32, S}  bo
     const uint32_t blk_bytes = kClassPad * 128;                 // 32 class rows x 64 elements
     const uint32_t b_base = a_base + 2 * blk_bytes;
     const int b_blocks = Ch / kBlockK;
-    float* red = reinterpret_cast<float*>(smem + 2 * blk_bytes + b_blocks * blk_bytes);   // [128][33]
-    __shared__ float part[4][32];
+    __shared__ float part[4 * 256];                             // per-warp channel sums
     __shared__ __align__(8) uint64_t full, done;
     __shared__ uint32_t tmem_slot;
     const int tid = threadIdx.x, warp = tid >> 5;
@@ -479,22 +478,25 @@ tc_dgrad_kernel(const __grid_constant__ CUtensorMap tmA,   // dz  {p, 32, S}  bo
 #pragma unroll
                 for (int k = 0; k < 32; ++k) v[k] = 0.f;
             }
-            // sums over the tile's pixels, fixed order: rows -> four quarter sums -> one
+            // sums over the warp's 32 pixels, fixed order: a reduce-scatter over the lanes (lanes whose bit
+            // is set keep the upper half of the channels), after which lane c holds the sum of channel n0 + c
+            const int lane = tid & 31;
 #pragma unroll
-            for (int k = 0; k < 32; ++k) red[tid * 33 + k] = v[k];
-            __syncthreads();
-            {
-                const int ch = tid & 31, q = tid >> 5;
-                float t = 0.f;
-#pragma unroll 8
-                for (int r = 0; r < 32; ++r) t += red[(q * 32 + r) * 33 + ch];
-                part[q][ch] = t;
+            for (int half = 16; half >= 1; half >>= 1) {
+                const bool up = (lane & half) != 0;
+#pragma unroll
+                for (int k = 0; k < half; ++k) {
+                    const float keep = up ? v[k + half] : v[k];
+                    const float send = up ? v[k] : v[k + half];
+                    v[k] = keep + __shfl_xor_sync(0xffffffffu, send, half);
+                }
             }
-            __syncthreads();
-            if (tid < 32)
-                b1_partials[((int64_t)s * gridDim.x + blockIdx.x) * Ch + n0 + tid] =
-                    (part[0][tid] + part[1][tid]) + (part[2][tid] + part[3][tid]);
+            part[warp * 256 + n0 + lane] = v[0];
         }
+        __syncthreads();
+        for (int k = tid; k < Ch; k += kThreadsTc)
+            b1_partials[((int64_t)s * gridDim.x + blockIdx.x) * Ch + k] =
+                (part[k] + part[256 + k]) + (part[512 + k] + part[768 + k]);
     } else {
         drain_after_error();
     }
@@ -636,7 +638,7 @@ TcPlan* tc_plan_create(const TcBuffers& b, char* err, size_t err_len)
         P->cols1 = pow2_cols(m_in * b.c_hidden);
         P->smem_fwd3 = 4 * ((size_t)kTileM * 128 + (size_t)b.c_hidden * 128) + kSmemAlign;
         P->smem_wg3 = 3 * ((size_t)(m_in * 2 + b.c_hidden / kBlockK) * kChunkPix * 128) + kSmemAlign;
-        P->smem_dgrad = (size_t)(2 + b.c_hidden / kBlockK) * kClassPad * 128 + (size_t)kTileM * 33 * sizeof(float) + kSmemAlign;
+        P->smem_dgrad = (size_t)(2 + b.c_hidden / kBlockK) * kClassPad * 128 + kSmemAlign;
         if (P->cols1 > 512) {
             snprintf(err, err_len, "c_in %d with c_hidden %d needs %d TMEM columns (> 512)", b.c_in, b.c_hidden, P->cols1);
             delete P; return nullptr;

@@ -24,7 +24,7 @@ __device__ __forceinline__ void apply_update(const UpdateArgs& a, int64_t gi, fl
 // the group sums are added in group order through shared memory, and group 0 applies the update.
 template <int G, int E>
 __global__ void __launch_bounds__(kUpdThreads)
-sgd_update_kernel(UpdateArgs a, int n_param_blocks)
+sgd_update_kernel(UpdateArgs a, int n_param_blocks, int64_t range_begin)
 {
     constexpr int kRow = kUpdThreads / G;      // consecutive parameters covered by one thread group
     constexpr int kPer = kRow * E;             // parameters per block
@@ -39,7 +39,7 @@ sgd_update_kernel(UpdateArgs a, int n_param_blocks)
         // E parameters per thread, all of their split-K loads issued before any is consumed
 #pragma unroll
         for (int e = 0; e < E; ++e) {
-            const int64_t i = (int64_t)blockIdx.x * kPer + e * kRow + col;
+            const int64_t i = range_begin + (int64_t)blockIdx.x * kPer + e * kRow + col;
             layer[e] = -1; is_weight[e] = false; has_partials[e] = false; sum[e] = 0.f;
             if (i < a.n_params) {
                 for (int L = 0; L < a.n_layers; ++L) {
@@ -66,7 +66,7 @@ sgd_update_kernel(UpdateArgs a, int n_param_blocks)
 #pragma unroll
         for (int e = 0; e < E; ++e) {
             if (layer[e] < 0) continue;
-            const int64_t i = (int64_t)blockIdx.x * kPer + e * kRow + col;
+            const int64_t i = range_begin + (int64_t)blockIdx.x * kPer + e * kRow + col;
             const LayerUpdate& ly = a.layer[layer[e]];
             if (is_weight[e]) {
                 float gr;
@@ -115,24 +115,73 @@ sgd_update_kernel(UpdateArgs a, int n_param_blocks)
     }
 }
 
-void launch_sgd_update(const UpdateArgs& a, cudaStream_t s)
+// A large weight tensor with a moderate number of split-K partials (the 3x3 layer): a pure stream.
+// Each thread owns VEC consecutive weights and reads them from every partial with all loads in flight.
+template <int VEC>
+__global__ void __launch_bounds__(256)
+sgd_update_stream_kernel(UpdateArgs a, int L)
 {
+    const LayerUpdate& ly = a.layer[L];
+    const int s = blockIdx.y;
+    const int64_t nw = (int64_t)ly.cout * ly.cin * ly.taps;
+    const int64_t e = ((int64_t)blockIdx.x * 256 + threadIdx.x) * VEC;
+    if (e >= nw) return;
+    const float* src = ly.w_partials + (int64_t)s * ly.w_stream_stride + e;
+    float g[VEC];
+#pragma unroll
+    for (int j = 0; j < VEC; ++j) g[j] = 0.f;
+#pragma unroll 8
+    for (int k = 0; k < ly.n_split; ++k) {
+        if (VEC == 4) {
+            const float4 t = __ldg(reinterpret_cast<const float4*>(src + (int64_t)k * ly.w_split_stride));
+            g[0] += t.x; g[1] += t.y; g[2] += t.z; g[3] += t.w;
+        } else {
+            g[0] += __ldg(src + (int64_t)k * ly.w_split_stride);
+        }
+    }
+    const int64_t gi = (int64_t)s * a.n_params + ly.w_off + e;
+#pragma unroll
+    for (int j = 0; j < VEC; ++j) {
+        apply_update(a, gi + j, g[j]);
+        if (ly.shadow) ly.shadow[(int64_t)s * ly.shadow_stream_stride + e + j] = __float2bfloat16_rn(a.theta[gi + j]);
+    }
+}
+
+int launch_sgd_update(const UpdateArgs& a, cudaStream_t s)
+{
+    int n_launches = 1;
+    // large layers with partial sums go through the streaming kernel; everything else (small layers, biases,
+    // loss) through the grouped kernel, which then starts after the streamed range
+    int64_t range_begin = 0;
+    for (int L = 0; L < a.n_layers; ++L) {
+        const LayerUpdate& ly = a.layer[L];
+        const int64_t nw = (int64_t)ly.cout * ly.cin * ly.taps;
+        if (ly.w_partials && nw >= 65536 && ly.w_off == range_begin) {
+            const bool vec = nw % 4 == 0 && ly.w_split_stride % 4 == 0 && ly.w_stream_stride % 4 == 0 &&
+                             ((uintptr_t)ly.w_partials % 16 == 0);
+            if (vec) sgd_update_stream_kernel<4><<<dim3((unsigned)((nw / 4 + 255) / 256), (unsigned)a.S), 256, 0, s>>>(a, L);
+            else sgd_update_stream_kernel<1><<<dim3((unsigned)((nw + 255) / 256), (unsigned)a.S), 256, 0, s>>>(a, L);
+            range_begin = ly.w_off + nw;
+            ++n_launches;
+        }
+    }
     int items = 1, max_split = 1;
     for (int L = 0; L < a.n_layers; ++L) {
         if (a.layer[L].b_partials) items += a.layer[L].cout;
         if (a.layer[L].w_partials && a.layer[L].n_split > max_split) max_split = a.layer[L].n_split;
     }
     const int n_red_blocks = (items + kUpdThreads / 32 - 1) / (kUpdThreads / 32);
-    // few parameters with many splits: 8 groups, 1 parameter per thread; many parameters: 4 groups x 4 parameters
-    const bool big = a.n_params > 65536;
-    const int G = max_split <= 1 ? 1 : (big ? 4 : 8), E = big ? 4 : 1;
+    const int64_t n_rest = a.n_params - range_begin;
+    const bool big = n_rest > 65536;
+    const int G = max_split <= 1 ? 1 : 8, E = big ? 4 : 1;
     const int per = kUpdThreads / G * E;
-    const int n_param_blocks = (int)((a.n_params + per - 1) / per);
+    const int n_param_blocks = (int)((n_rest + per - 1) / per);
     const dim3 grid((unsigned)(n_param_blocks + n_red_blocks), (unsigned)a.S);
-    if (G == 1 && E == 1) sgd_update_kernel<1, 1><<<grid, kUpdThreads, 0, s>>>(a, n_param_blocks);
-    else if (G == 1) sgd_update_kernel<1, 4><<<grid, kUpdThreads, 0, s>>>(a, n_param_blocks);
-    else if (G == 8) sgd_update_kernel<8, 1><<<grid, kUpdThreads, 0, s>>>(a, n_param_blocks);
-    else sgd_update_kernel<4, 4><<<grid, kUpdThreads, 0, s>>>(a, n_param_blocks);
+    if (G == 1 && E == 1) sgd_update_kernel<1, 1><<<grid, kUpdThreads, 0, s>>>(a, n_param_blocks, range_begin);
+    else if (G == 1) sgd_update_kernel<1, 4><<<grid, kUpdThreads, 0, s>>>(a, n_param_blocks, range_begin);
+    else if (E == 1) sgd_update_kernel<8, 1><<<grid, kUpdThreads, 0, s>>>(a, n_param_blocks, range_begin);
+    else sgd_update_kernel<8, 4><<<grid, kUpdThreads, 0, s>>>(a, n_param_blocks, range_begin);
+    return n_launches;
 }
 
 __global__ void refresh_shadow_kernel(UpdateArgs a)

@@ -247,9 +247,8 @@ st_status enqueue_step(st_ctx* c, int slot, bool want_conf, StageTimer* t = null
     st = check_launch(c, "head backward");
     if (st != ST_OK) return st;
 
-    launch_sgd_update(make_update_args(c, slot), s);
+    c->launches += launch_sgd_update(make_update_args(c, slot), s);
     if (t) t->mark("sgd_update", s);
-    c->launches += 1;
     return check_launch(c, "sgd update");
 }
 

@@ -94,7 +94,7 @@ struct UpdateArgs {
     int loss_slot;           // slot of loss_buf written by this step
     double inv_P;
 };
-void launch_sgd_update(const UpdateArgs& a, cudaStream_t s);
+int launch_sgd_update(const UpdateArgs& a, cudaStream_t s);   // returns the number of kernels launched
 // refresh the bf16 shadows from the fp32 master parameters (after init)
 void launch_refresh_shadow(const UpdateArgs& a, cudaStream_t s);
 // mean IoU (Section 3.2) from an int64 confusion matrix, in double, one block
