@@ -215,6 +215,7 @@ tc_fwd3x3_kernel(const __grid_constant__ CUtensorMap tmA,   // {Cin, w, h, S}   
                  const __grid_constant__ CUtensorMap tmB,   // {Cin, 9*Ch, S}    box {64, Ch, 1}
                  const float* __restrict__ theta, int64_t n_params, int64_t b_off,
                  bf16* __restrict__ hidden,                  // [S][p][Ch]
+                 uint32_t* __restrict__ relu_bits,           // [S][p][Ch/32]: bit k of word j = hidden[32j + k] > 0
                  int Cin, int Ch, int h, int w, int tmem_cols, unsigned int* err)
 {
     extern __shared__ uint8_t smem_raw[];
@@ -272,20 +273,26 @@ tc_fwd3x3_kernel(const __grid_constant__ CUtensorMap tmA,   // {Cin, w, h, S}   
         const int y = y0 + tid / kTileW, x = x0 + tid % kTileW;
         const bool in = y < h && x < w;
         const float* bias = theta + (int64_t)s * n_params + b_off;
-        bf16* dst = hidden + ((int64_t)s * h * w + (int64_t)y * w + x) * Ch;
+        const int64_t pixel = (int64_t)s * h * w + (int64_t)y * w + x;
+        bf16* dst = hidden + pixel * Ch;
         for (int n0 = 0; n0 < Ch; n0 += 32) {
             float v[32];
             tmem_ld_32x32(tmem + ((uint32_t)(warp * 32) << 16) + n0, v);
             if (in) {
                 uint4 out[4];
                 __nv_bfloat162* o2 = reinterpret_cast<__nv_bfloat162*>(out);
+                uint32_t bits = 0;
 #pragma unroll
                 for (int k = 0; k < 16; ++k) {
-                    float a = v[2 * k] + __ldg(bias + n0 + 2 * k), b = v[2 * k + 1] + __ldg(bias + n0 + 2 * k + 1);
-                    o2[k] = __floats2bfloat162_rn(fmaxf(a, 0.f), fmaxf(b, 0.f));
+                    const float a = fmaxf(v[2 * k] + __ldg(bias + n0 + 2 * k), 0.f), b = fmaxf(v[2 * k + 1] + __ldg(bias + n0 + 2 * k + 1), 0.f);
+                    o2[k] = __floats2bfloat162_rn(a, b);
+                    // the mask is taken on the stored (rounded) activation, the value the next layer sees
+                    bits |= (__low2float(o2[k]) > 0.f ? 1u : 0u) << (2 * k);
+                    bits |= (__high2float(o2[k]) > 0.f ? 1u : 0u) << (2 * k + 1);
                 }
 #pragma unroll
                 for (int k = 0; k < 4; ++k) reinterpret_cast<uint4*>(dst + n0)[k] = out[k];
+                relu_bits[pixel * (Ch / 32) + n0 / 32] = bits;
             }
         }
     } else {
@@ -403,7 +410,7 @@ tc_wgrad3x3_kernel(const __grid_constant__ CUtensorMap tmA,   // X   {Cin, w, h,
 __global__ void __launch_bounds__(kThreadsTc)
 tc_dgrad_kernel(const __grid_constant__ CUtensorMap tmA,   // dz  {p, 32, S}  box {64, 32, 1}
                 const __grid_constant__ CUtensorMap tmB,   // W2  {Ch, 32, S} box {64, 32, 1}
-                const bf16* __restrict__ hidden,            // [S][p][Ch]
+                const uint32_t* __restrict__ relu_bits,     // [S][p][Ch/32]
                 bf16* __restrict__ dhidden,                 // [S][p][Ch]
                 float* __restrict__ b1_partials,            // [S][n_blocks][Ch]
                 int Ch, int p, int tmem_cols, unsigned int* err)
@@ -450,26 +457,33 @@ tc_dgrad_kernel(const __grid_constant__ CUtensorMap tmA,   // dz  {p, 32, S}  bo
         umma_commit(smem_u32(&done));
     }
     __syncwarp();
+    // the ReLU mask of this thread's pixel (one bit per hidden channel), fetched while the MMAs run
+    const int pix = pix0 + tid;
+    const bool in = pix < p;
+    uint32_t mbits[8] = {0, 0, 0, 0, 0, 0, 0, 0};
+    if (in) {
+        const uint32_t* mp = relu_bits + ((int64_t)s * p + pix) * (Ch / 32);
+#pragma unroll
+        for (int j = 0; j < 8; ++j) if (j < Ch / 32) mbits[j] = __ldg(mp + j);
+    }
     ok = mbar_wait(smem_u32(&done), 0, err, kWaitDone);
     tc_fence_after_sync();
     ok = __syncthreads_and(ok);          // the epilogue below synchronises the block: all or none
     if (ok) {
-        const int pix = pix0 + tid;
-        const bool in = pix < p;
         const int64_t row = ((int64_t)s * p + (in ? pix : 0)) * Ch;
         for (int n0 = 0; n0 < Ch; n0 += 32) {
             float v[32];
             tmem_ld_32x32(tmem + ((uint32_t)(warp * 32) << 16) + n0, v);
             if (in) {
-                uint4 hv[4], out[4];
-#pragma unroll
-                for (int k = 0; k < 4; ++k) hv[k] = __ldg(reinterpret_cast<const uint4*>(hidden + row + n0) + k);
-                const __nv_bfloat162* h2 = reinterpret_cast<const __nv_bfloat162*>(hv);
+                uint4 out[4];
                 __nv_bfloat162* o2 = reinterpret_cast<__nv_bfloat162*>(out);
+                uint32_t bits = 0;
+#pragma unroll
+                for (int j = 0; j < 8; ++j) if (j == n0 / 32) bits = mbits[j];
 #pragma unroll
                 for (int k = 0; k < 16; ++k) {
-                    if (!(__low2float(h2[k]) > 0.f)) v[2 * k] = 0.f;
-                    if (!(__high2float(h2[k]) > 0.f)) v[2 * k + 1] = 0.f;
+                    if (!((bits >> (2 * k)) & 1u)) v[2 * k] = 0.f;
+                    if (!((bits >> (2 * k + 1)) & 1u)) v[2 * k + 1] = 0.f;
                     o2[k] = __floats2bfloat162_rn(v[2 * k], v[2 * k + 1]);
                 }
 #pragma unroll
@@ -693,7 +707,7 @@ int tc_backward(const TcPlan* P, cudaStream_t s, StageTimer* t)
     if (b.c_hidden) {
         const int blocks = tc_b1_partials(b.h, b.w);
         tc_dgrad_kernel<<<dim3(blocks, b.S), kThreadsTc, P->smem_dgrad, s>>>(
-            P->dz_map, P->w2_map, b.hidden, b.dhidden, b.b1_partials, b.c_hidden, P->p, pow2_cols(b.c_hidden), b.err);
+            P->dz_map, P->w2_map, b.relu_bits, b.dhidden, b.b1_partials, b.c_hidden, P->p, pow2_cols(b.c_hidden), b.err);
         if (t) t->mark("tc_dgrad", s);
         tc_wgrad3x3_kernel<3><<<dim3(9 * P->split1, b.S), kThreadsTc, P->smem_wg3, s>>>(
             P->x_wg3, P->dh_wg3, b.w1_partials, b.c_in, b.c_hidden, b.h, b.w, P->chunks1, P->per1, P->split1,

@@ -38,6 +38,7 @@ struct st_ctx {
     int64_t dz_pitch = 0;
     float *hid_f32 = nullptr, *dhid_f32 = nullptr;
     bf16 *hid_bf16 = nullptr, *dhid_bf16 = nullptr;
+    uint32_t* relu_bits = nullptr;
     bf16 *w1_shadow = nullptr, *w2_shadow = nullptr;
     float *w1_partials = nullptr, *w2_partials = nullptr, *b1_partials = nullptr;
     int n_split1 = 0, n_split2 = 0, n_b1part = 0;
@@ -386,6 +387,7 @@ st_status st_init_head(const st_head_desc* desc, const float* init_params, st_ct
         ALLOC(w2_partials, (size_t)S * c->n_split2 * kClassPad * c_last);
         if (c->Ch) {
             ALLOC(hid_bf16, S * c->p * c->Ch); ALLOC(dhid_bf16, S * c->p * c->Ch);
+            ALLOC(relu_bits, S * c->p * (c->Ch / 32));
             ALLOC(w1_shadow, (size_t)S * 9 * c->Ch * c->Cin);
             c->n_split1 = tc_wgrad_splits(1, c->Cin, c->Ch, c->h, c->w);
             ALLOC(w1_partials, (size_t)S * c->n_split1 * 9 * c->Ch * c->Cin);
@@ -418,7 +420,7 @@ st_status st_init_head(const st_head_desc* desc, const float* init_params, st_ct
         b.x = c->x_bf16; b.w1 = c->w1_shadow; b.w2 = c->w2_shadow; b.theta = c->theta; b.n_params = c->n_params;
         b.b1_off = c->Ch ? L.b_off[0] : 0; b.b2_off = L.b_off[L.n_layers - 1]; b.w2_off = L.w_off[L.n_layers - 1];
         b.err = c->bad + 2;
-        b.z = c->z; b.hidden = c->hid_bf16; b.dz = c->dz; b.dz_bf16 = c->dz_bf16; b.dhidden = c->dhid_bf16;
+        b.z = c->z; b.hidden = c->hid_bf16; b.relu_bits = c->relu_bits; b.dz = c->dz; b.dz_bf16 = c->dz_bf16; b.dhidden = c->dhid_bf16;
         b.w1_partials = c->w1_partials; b.w2_partials = c->w2_partials; b.b1_partials = c->b1_partials;
         char msg[256] = {0};
         c->plan = tc_plan_create(b, msg, sizeof msg);

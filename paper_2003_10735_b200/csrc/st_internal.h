@@ -117,6 +117,7 @@ struct TcBuffers {
     int64_t n_params, b1_off, b2_off, w2_off;
     float* z;             // [S][C][p]
     bf16* hidden;         // [S][p][c_hidden]
+    uint32_t* relu_bits;  // [S][p][c_hidden/32]: one bit per hidden value, set where it is > 0
     const float* dz;      // [S][C][p]
     const bf16* dz_bf16;  // [S][kClassPad][tc_dz_pitch]
     bf16* dhidden;        // [S][p][c_hidden]
