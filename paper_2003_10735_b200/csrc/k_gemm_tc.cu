@@ -684,7 +684,7 @@ int tc_forward(const TcPlan* P, cudaStream_t s, StageTimer* t)
     if (b.c_hidden) {
         const int tiles = ((b.w + kTileW - 1) / kTileW) * ((b.h + kTileH - 1) / kTileH);
         tc_fwd3x3_kernel<4><<<dim3(tiles, b.S), kThreadsTc, P->smem_fwd3, s>>>(
-            P->x_fwd3, P->w1_map, b.theta, b.n_params, b.b1_off, b.hidden, b.c_in, b.c_hidden, b.h, b.w,
+            P->x_fwd3, P->w1_map, b.theta, b.n_params, b.b1_off, b.hidden, b.relu_bits, b.c_in, b.c_hidden, b.h, b.w,
             pow2_cols(b.c_hidden), b.err);
         if (t) t->mark("tc_fwd3x3", s);
         ++n;
