@@ -54,7 +54,7 @@ sgd_update_kernel(UpdateArgs a, int n_param_blocks, int64_t range_begin)
                 has_partials[e] = true;
                 const float* src = ly.w_partials + (int64_t)s * ly.w_stream_stride + (i - ly.w_off);
                 float t = 0.f;
-#pragma unroll 4
+#pragma unroll 16
                 for (int k = g; k < ly.n_split; k += G) t += __ldg(src + (int64_t)k * ly.w_split_stride);
                 sum[e] = t;
             }
@@ -95,6 +95,7 @@ sgd_update_kernel(UpdateArgs a, int n_param_blocks, int64_t range_begin)
         if (item < ly.cout) {
             const float* src = ly.b_partials + (int64_t)s * ly.n_bpart * ly.cout + item;
             float g = 0.f;
+#pragma unroll 16
             for (int k = lane; k < ly.n_bpart; k += 32) g += __ldg(src + (int64_t)k * ly.cout);
 #pragma unroll
             for (int o = 16; o > 0; o >>= 1) g += __shfl_xor_sync(0xffffffffu, g, o);
@@ -105,6 +106,7 @@ sgd_update_kernel(UpdateArgs a, int n_param_blocks, int64_t range_begin)
     }
     if (item == 0 && a.loss_part) {
         double t = 0.0;
+#pragma unroll 16
         for (int k = lane; k < a.n_loss_part; k += 32) t += (double)__ldg(a.loss_part + (int64_t)s * a.n_loss_part + k);
 #pragma unroll
         for (int o = 16; o > 0; o >>= 1) t += __shfl_xor_sync(0xffffffffu, t, o);
