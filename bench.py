@@ -168,6 +168,29 @@ def run_reference(args, cfg):
 
 
 # --------------------------------------------------------------------------------------------
+# multi-GPU plumbing: the path shards by client stream, ranks exchange nothing but the timing
+# --------------------------------------------------------------------------------------------
+def rank_streams(streams_per_rank: int, world: int, rank: int):
+    """Global ids of the client streams a rank owns (disjoint, covering 0 .. world*streams_per_rank - 1)."""
+    return [rank * streams_per_rank + s for s in range(streams_per_rank)]
+
+
+def max_over_ranks(value: float, dist, device=None) -> float:
+    """Largest value over all ranks (the job is as slow as its slowest rank); identity without a group."""
+    if dist is None:
+        return float(value)
+    import torch
+    t = torch.tensor([value], dtype=torch.float64, device=device or "cpu")
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return float(t.item())
+
+
+def whole_job_rate(units_per_rank: float, world: int, ms_max: float) -> float:
+    """Units all ranks processed per second, timed by the slowest rank."""
+    return world * units_per_rank / (ms_max / 1e3)
+
+
+# --------------------------------------------------------------------------------------------
 # the CUDA path
 # --------------------------------------------------------------------------------------------
 def run_ours(args, cfg):
@@ -193,9 +216,9 @@ def run_ours(args, cfg):
         feats_h, logits_h, thetas = [], [], []
         for i in range(N_SETS):
             per_stream_f, per_stream_t = [], []
-            for s in range(S):
-                f = si.frozen_features(cfg.c_in, cfg.feat_h, cfg.feat_w, seed=1000 * rank + 10 * i + s)
-                t = si.teacher_logits(cfg, stream=100 * rank + s, frame=i)
+            for gs in rank_streams(S, world, rank):
+                f = si.frozen_features(cfg.c_in, cfg.feat_h, cfg.feat_w, seed=10 * gs + i)
+                t = si.teacher_logits(cfg, stream=gs, frame=i)
                 per_stream_f.append(torch.from_numpy(f).pin_memory())
                 per_stream_t.append(torch.from_numpy(t).pin_memory())
             feats_h.append(per_stream_f)
@@ -248,10 +271,7 @@ def run_ours(args, cfg):
             clocks.end()
         ms_total = ev0.elapsed_time(ev1)
         launches = st.st_launch_count(ctx) - launches0
-        if dist is not None:
-            t = torch.tensor([ms_total], dtype=torch.float64, device="cuda")
-            dist.all_reduce(t, op=dist.ReduceOp.MAX)
-            ms_total = float(t.item())
+        ms_total = max_over_ranks(ms_total, dist, "cuda")
         clock_info = clocks.finish() if clocks else None
 
         # ---- the K-step loop alone (inputs already cached), for the per-step view
@@ -275,10 +295,7 @@ def run_ours(args, cfg):
         ev1.record(stream)
         barrier()
         ms_e2e = ev0.elapsed_time(ev1)
-        if dist is not None:
-            t = torch.tensor([ms_e2e], dtype=torch.float64, device="cuda")
-            dist.all_reduce(t, op=dist.ReduceOp.MAX)
-            ms_e2e = float(t.item())
+        ms_e2e = max_over_ranks(ms_e2e, dist, "cuda")
         h2d = S * (cfg.c_in * p * 4 + C * P * 4)
         d2h = S * (n_params * 4 + 8)
 
@@ -333,7 +350,7 @@ def run_ours(args, cfg):
         result = None
         if rank == 0:
             ms_step = ms_total / args.steps
-            value = world * K * args.steps / (ms_total / 1e3)
+            value = whole_job_rate(K * args.steps, world, ms_total)
             dominant = max((n for n in kernels if "frac" in kernels[n] or True),
                            key=lambda n: kernels[n]["ms"] * kernels[n]["per_key_frame"])
             dk = kernels[dominant]
