@@ -68,6 +68,8 @@ tc_fwd1x1_kernel(const __grid_constant__ CUtensorMap tmA,   // {K, p, S}  box {6
     __syncthreads();
     tc_fence_after_sync();
     const uint32_t tmem = tmem_slot;
+    pdl_wait();                  // inputs come from the previous kernel of the step
+    pdl_launch_dependents();
     const uint32_t done_bar = smem_u32(&bars[kblocks]);
     bool ok = true;
 
@@ -150,6 +152,8 @@ tc_wgrad1x1_kernel(const __grid_constant__ CUtensorMap tmA,   // {K, p, S}      
     __syncthreads();
     tc_fence_after_sync();
     const uint32_t tmem = tmem_slot;
+    pdl_wait();                  // inputs come from the previous kernel of the step
+    pdl_launch_dependents();
     bool ok = true;
 
     if (tid == 0) {
@@ -239,6 +243,8 @@ tc_fwd3x3_kernel(const __grid_constant__ CUtensorMap tmA,   // {Cin, w, h, S}   
     __syncthreads();
     tc_fence_after_sync();
     const uint32_t tmem = tmem_slot;
+    pdl_wait();                  // inputs come from the previous kernel of the step
+    pdl_launch_dependents();
     bool ok = true;
 
     if (tid == 0) {
@@ -341,6 +347,8 @@ tc_wgrad3x3_kernel(const __grid_constant__ CUtensorMap tmA,   // X   {Cin, w, h,
     __syncthreads();
     tc_fence_after_sync();
     const uint32_t tmem = tmem_slot;
+    pdl_wait();                  // inputs come from the previous kernel of the step
+    pdl_launch_dependents();
     bool ok = true;
 
     if (tid == 0) {
@@ -436,6 +444,8 @@ tc_dgrad_kernel(const __grid_constant__ CUtensorMap tmA,   // dz  {p, 32, S}  bo
     __syncthreads();
     tc_fence_after_sync();
     const uint32_t tmem = tmem_slot;
+    pdl_wait();                  // inputs come from the previous kernel of the step
+    pdl_launch_dependents();
     bool ok = true;
 
     if (tid == 0) {
@@ -683,14 +693,14 @@ int tc_forward(const TcPlan* P, cudaStream_t s, StageTimer* t)
     int n = 0;
     if (b.c_hidden) {
         const int tiles = ((b.w + kTileW - 1) / kTileW) * ((b.h + kTileH - 1) / kTileH);
-        tc_fwd3x3_kernel<4><<<dim3(tiles, b.S), kThreadsTc, P->smem_fwd3, s>>>(
+        launch_chain(tc_fwd3x3_kernel<4>, dim3(tiles, b.S), dim3(kThreadsTc), P->smem_fwd3, s,
             P->x_fwd3, P->w1_map, b.theta, b.n_params, b.b1_off, b.hidden, b.relu_bits, b.c_in, b.c_hidden, b.h, b.w,
             pow2_cols(b.c_hidden), b.err);
         if (t) t->mark("tc_fwd3x3", s);
         ++n;
     }
     const int tiles1 = (P->p + kTileM - 1) / kTileM;
-    tc_fwd1x1_kernel<<<dim3(tiles1, b.S), kThreadsTc, P->smem_fwd1, s>>>(
+    launch_chain(tc_fwd1x1_kernel, dim3(tiles1, b.S), dim3(kThreadsTc), P->smem_fwd1, s,
         P->act_fwd, P->w2_map, b.theta, b.n_params, b.b2_off, b.z, b.C, P->p, P->c_last / kBlockK, b.err);
     if (t) t->mark("tc_fwd1x1", s);
     return n + 1;
@@ -700,16 +710,16 @@ int tc_backward(const TcPlan* P, cudaStream_t s, StageTimer* t)
 {
     const TcBuffers& b = P->b;
     int n = 0;
-    tc_wgrad1x1_kernel<3><<<dim3(P->split2, b.S), kThreadsTc, P->smem_wg1, s>>>(
+    launch_chain(tc_wgrad1x1_kernel<3>, dim3(P->split2, b.S), dim3(kThreadsTc), P->smem_wg1, s,
         P->act_wg, P->dz_map, b.w2_partials, P->c_last, P->chunks2, P->per2, P->cols2, b.err);
     if (t) t->mark("tc_wgrad1x1", s);
     ++n;
     if (b.c_hidden) {
         const int blocks = tc_b1_partials(b.h, b.w);
-        tc_dgrad_kernel<<<dim3(blocks, b.S), kThreadsTc, P->smem_dgrad, s>>>(
+        launch_chain(tc_dgrad_kernel, dim3(blocks, b.S), dim3(kThreadsTc), P->smem_dgrad, s,
             P->dz_map, P->w2_map, b.relu_bits, b.dhidden, b.b1_partials, b.c_hidden, P->p, pow2_cols(b.c_hidden), b.err);
         if (t) t->mark("tc_dgrad", s);
-        tc_wgrad3x3_kernel<3><<<dim3(9 * P->split1, b.S), kThreadsTc, P->smem_wg3, s>>>(
+        launch_chain(tc_wgrad3x3_kernel<3>, dim3(9 * P->split1, b.S), dim3(kThreadsTc), P->smem_wg3, s,
             P->x_wg3, P->dh_wg3, b.w1_partials, b.c_in, b.c_hidden, b.h, b.w, P->chunks1, P->per1, P->split1,
             P->cols1, b.err);
         if (t) t->mark("tc_wgrad3x3", s);

@@ -7,7 +7,15 @@
 // K7 — UpdatedPart(student) (Algorithm 3): the packed fp32 buffer of all trainable tensors.
 #include "st_internal.h"
 
+#include <cstdlib>
+
 namespace st {
+
+bool pdl_enabled()
+{
+    static const bool on = [] { const char* e = getenv("ST_NO_PDL"); return !(e && e[0] == '1'); }();
+    return on;
+}
 
 constexpr int kUpdThreads = 256;
 
@@ -29,6 +37,8 @@ sgd_update_kernel(UpdateArgs a, int n_param_blocks, int64_t range_begin)
     constexpr int kRow = kUpdThreads / G;      // consecutive parameters covered by one thread group
     constexpr int kPer = kRow * E;             // parameters per block
     __shared__ float part[G][kPer];
+    pdl_wait();
+    pdl_launch_dependents();
     const int s = blockIdx.y;
     const int64_t base = (int64_t)s * a.n_params;
     if ((int)blockIdx.x < n_param_blocks) {
@@ -123,6 +133,8 @@ template <int VEC>
 __global__ void __launch_bounds__(256)
 sgd_update_stream_kernel(UpdateArgs a, int L)
 {
+    pdl_wait();
+    pdl_launch_dependents();
     const LayerUpdate& ly = a.layer[L];
     const int s = blockIdx.y;
     const int64_t nw = (int64_t)ly.cout * ly.cin * ly.taps;
@@ -161,8 +173,8 @@ int launch_sgd_update(const UpdateArgs& a, cudaStream_t s)
         if (ly.w_partials && nw >= 65536 && ly.w_off == range_begin) {
             const bool vec = nw % 4 == 0 && ly.w_split_stride % 4 == 0 && ly.w_stream_stride % 4 == 0 &&
                              ((uintptr_t)ly.w_partials % 16 == 0);
-            if (vec) sgd_update_stream_kernel<4><<<dim3((unsigned)((nw / 4 + 255) / 256), (unsigned)a.S), 256, 0, s>>>(a, L);
-            else sgd_update_stream_kernel<1><<<dim3((unsigned)((nw + 255) / 256), (unsigned)a.S), 256, 0, s>>>(a, L);
+            if (vec) launch_chain(sgd_update_stream_kernel<4>, dim3((unsigned)((nw / 4 + 255) / 256), (unsigned)a.S), dim3(256), 0, s, a, L);
+            else launch_chain(sgd_update_stream_kernel<1>, dim3((unsigned)((nw + 255) / 256), (unsigned)a.S), dim3(256), 0, s, a, L);
             range_begin = ly.w_off + nw;
             ++n_launches;
         }
@@ -179,10 +191,11 @@ int launch_sgd_update(const UpdateArgs& a, cudaStream_t s)
     const int per = kUpdThreads / G * E;
     const int n_param_blocks = (int)((n_rest + per - 1) / per);
     const dim3 grid((unsigned)(n_param_blocks + n_red_blocks), (unsigned)a.S);
-    if (G == 1 && E == 1) sgd_update_kernel<1, 1><<<grid, kUpdThreads, 0, s>>>(a, n_param_blocks, range_begin);
-    else if (G == 1) sgd_update_kernel<1, 4><<<grid, kUpdThreads, 0, s>>>(a, n_param_blocks, range_begin);
-    else if (E == 1) sgd_update_kernel<8, 1><<<grid, kUpdThreads, 0, s>>>(a, n_param_blocks, range_begin);
-    else sgd_update_kernel<8, 4><<<grid, kUpdThreads, 0, s>>>(a, n_param_blocks, range_begin);
+    const dim3 blk(kUpdThreads);
+    if (G == 1 && E == 1) launch_chain(sgd_update_kernel<1, 1>, grid, blk, 0, s, a, n_param_blocks, range_begin);
+    else if (G == 1) launch_chain(sgd_update_kernel<1, 4>, grid, blk, 0, s, a, n_param_blocks, range_begin);
+    else if (E == 1) launch_chain(sgd_update_kernel<8, 1>, grid, blk, 0, s, a, n_param_blocks, range_begin);
+    else launch_chain(sgd_update_kernel<8, 4>, grid, blk, 0, s, a, n_param_blocks, range_begin);
     return n_launches;
 }
 

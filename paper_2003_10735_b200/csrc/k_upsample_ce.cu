@@ -66,6 +66,8 @@ upsample_ce_kernel(UpsampleCeArgs a, int chunk)
     const float* z = a.z + (int64_t)s * C * p;
     const uint8_t* labels = a.labels + (int64_t)s * H * W;
     const int tid = threadIdx.x;
+    pdl_wait();
+    pdl_launch_dependents();
 
     // ---- z tile with replicated borders
     for (int idx = tid; idx < C * ZT_H * ZT_W; idx += kThreads) {
@@ -263,8 +265,8 @@ void launch_upsample_ce(const UpsampleCeArgs& a, cudaStream_t s)
     size_t smem = 0;
     const int chunk = chunk_classes(a.C, &smem);
     dim3 grid((unsigned)((a.w + NX - 1) / NX), (unsigned)((a.h + NY - 1) / NY), (unsigned)a.S);
-    if (a.conf) upsample_ce_kernel<true><<<grid, kThreads, smem, s>>>(a, chunk);
-    else upsample_ce_kernel<false><<<grid, kThreads, smem, s>>>(a, chunk);
+    if (a.conf) launch_chain(upsample_ce_kernel<true>, grid, dim3(kThreads), smem, s, a, chunk);
+    else launch_chain(upsample_ce_kernel<false>, grid, dim3(kThreads), smem, s, a, chunk);
 }
 
 // ------------------------------------------------------------------------------------------------

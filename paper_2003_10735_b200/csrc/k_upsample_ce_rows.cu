@@ -114,6 +114,8 @@ upsample_ce_rows_kernel(UpsampleCeArgs a)
     const float* z = a.z + (int64_t)s * C * p;
     const uint8_t* labels = a.labels + (int64_t)s * H * W;
     const int tid = threadIdx.x, wi = tid >> 5, l = tid & 31;
+    pdl_wait();                  // the logits come from the previous kernel of the step
+    pdl_launch_dependents();
 
     // ---- tile: node rows y0-1 .. y0+RN_Y, node columns xa .. xa+35 where xa = (x0-1) rounded down to a
     // multiple of 4 (so that rows are fetched as 16-byte vectors), clamped at the borders, scaled by
@@ -342,9 +344,8 @@ template <int CB>
 cudaError_t launch_cb(const UpsampleCeArgs& a, cudaStream_t s)
 {
     dim3 grid((unsigned)((a.w + RN_X - 1) / RN_X), (unsigned)((a.h + RN_Y - 1) / RN_Y), (unsigned)a.S);
-    if (a.conf) upsample_ce_rows_kernel<CB, true><<<grid, R_THREADS, rows_smem_bytes<CB>(a.C), s>>>(a);
-    else upsample_ce_rows_kernel<CB, false><<<grid, R_THREADS, rows_smem_bytes<CB>(a.C), s>>>(a);
-    return cudaSuccess;
+    if (a.conf) return launch_chain(upsample_ce_rows_kernel<CB, true>, grid, dim3(R_THREADS), rows_smem_bytes<CB>(a.C), s, a);
+    return launch_chain(upsample_ce_rows_kernel<CB, false>, grid, dim3(R_THREADS), rows_smem_bytes<CB>(a.C), s, a);
 }
 
 // class-count buckets: the two workload sizes exactly, multiples of four otherwise

@@ -50,7 +50,8 @@ struct st_ctx {
     uint8_t* mask_tmp = nullptr;            // [P]
     uint8_t* mask_tmp2 = nullptr;           // [P]
     unsigned long long* conf_tmp = nullptr; // [C][C]
-    double* miou_tmp = nullptr;
+    double* miou_tmp = nullptr;             // status block on the device: [0] mean IoU, then the four words of `bad`
+    double* status_host = nullptr;          // pinned copy of the status block (32 bytes)
     float* read_tmp = nullptr; size_t read_tmp_bytes = 0;
     void* staging = nullptr; size_t staging_bytes = 0;
     std::vector<char> has_feat, has_labels;
@@ -253,26 +254,35 @@ st_status enqueue_step(st_ctx* c, int slot, bool want_conf, StageTimer* t = null
     return check_launch(c, "sgd update");
 }
 
+// One 32-byte device-to-host copy and one wait: the mean IoU of the last st_agreement and the error words.
+st_status fetch_status(st_ctx* c)
+{
+    ST_CUDA(c, cudaMemcpyAsync(c->status_host, c->miou_tmp, 32, cudaMemcpyDeviceToHost, c->stream));
+    ST_CUDA(c, cudaStreamSynchronize(c->stream));
+    return ST_OK;
+}
+
+// Turn the error words of the fetched status block into a status code, clearing what is reported.
+st_status report_status(st_ctx* c, bool agreement_call)
+{
+    const unsigned int* host_bad = reinterpret_cast<const unsigned int*>(c->status_host + 1);
+    const unsigned int gave_up = host_bad[2], bad_step = host_bad[0], bad_agree = host_bad[1];
+    if (!gave_up && !bad_step && !(agreement_call && bad_agree)) return ST_OK;
+    cudaMemsetAsync(c->bad, 0, 4 * sizeof(unsigned int), c->stream);
+    if (gave_up)
+        return fail(c, ST_ERR_CUDA, "a tensor-core kernel gave up waiting (code %u, block %u); results of that step are invalid",
+                    gave_up & 0xffu, gave_up >> 8);
+    if (agreement_call && bad_agree)
+        return fail(c, ST_ERR_INVALID_ARG, "%u pixel(s) with a label or prediction >= n_classes were skipped (st_agreement)", bad_agree);
+    return fail(c, ST_ERR_INVALID_ARG, "%u pixel(s) with a label >= n_classes were skipped (an earlier st_distill_step)", bad_step);
+}
+
 st_status report_bad_labels(st_ctx* c, int which, const char* what)
 {
-    unsigned int host_bad[4] = {0, 0, 0, 0};
-    ST_CUDA(c, cudaMemcpyAsync(host_bad, c->bad, sizeof host_bad, cudaMemcpyDeviceToHost, c->stream));
-    ST_CUDA(c, cudaStreamSynchronize(c->stream));
-    if (host_bad[2]) {
-        unsigned int zero = 0;
-        cudaMemcpyAsync(c->bad + 2, &zero, sizeof zero, cudaMemcpyHostToDevice, c->stream);
-        cudaStreamSynchronize(c->stream);
-        return fail(c, ST_ERR_CUDA, "a tensor-core kernel gave up waiting (code %u, block %u); results of that step are invalid",
-                    host_bad[2] & 0xffu, host_bad[2] >> 8);
-    }
-    if (host_bad[which]) {
-        unsigned int zero = 0;
-        cudaMemcpyAsync(c->bad + which, &zero, sizeof zero, cudaMemcpyHostToDevice, c->stream);
-        cudaStreamSynchronize(c->stream);
-        return fail(c, ST_ERR_INVALID_ARG, "%u pixel(s) with a label or prediction >= n_classes were skipped (%s)",
-                    host_bad[which], what);
-    }
-    return ST_OK;
+    (void)what;
+    st_status st = fetch_status(c);
+    if (st != ST_OK) return st;
+    return report_status(c, which == 1);
 }
 
 }  // namespace
@@ -313,6 +323,7 @@ void st_destroy(st_ctx* ctx)
     for (void* q : ctx->allocs) cudaFree(q);
     if (ctx->staging) cudaFree(ctx->staging);
     if (ctx->read_tmp) cudaFree(ctx->read_tmp);
+    if (ctx->status_host) cudaFreeHost(ctx->status_host);
     delete ctx;
 }
 
@@ -377,7 +388,8 @@ st_status st_init_head(const st_head_desc* desc, const float* init_params, st_ct
     ALLOC(z, S * c->C * c->p); ALLOC(dz, S * c->C * c->p);
     ALLOC(loss_part, S * c->n_k3_blocks); ALLOC(db_part, (size_t)S * c->n_k3_blocks * c->C);
     ALLOC(loss_buf, S * kMaxSteps);
-    ALLOC(bad, 4); ALLOC(mask_tmp, c->P); ALLOC(mask_tmp2, c->P); ALLOC(conf_tmp, c->C * c->C); ALLOC(miou_tmp, 1);
+    ALLOC(miou_tmp, 4); ALLOC(mask_tmp, c->P); ALLOC(mask_tmp2, c->P); ALLOC(conf_tmp, c->C * c->C);
+    if (e == cudaSuccess) { c->bad = reinterpret_cast<unsigned int*>(c->miou_tmp + 1); e = cudaHostAlloc((void**)&c->status_host, 32, cudaHostAllocDefault); }
     if (c->bf16_mode) {
         ALLOC(x_bf16, S * c->p * c->Cin);
         c->dz_pitch = tc_dz_pitch(c->h, c->w);
@@ -666,13 +678,10 @@ st_status st_agreement(st_ctx* ctx, int32_t stream, const uint8_t* pred, const u
     st = check_launch(ctx, "confusion");
     if (st != ST_OK) return st;
     if (conf) ST_CUDA(ctx, cudaMemcpyAsync(conf, ctx->conf_tmp, cbytes, cudaMemcpyDefault, ctx->stream));
-    double m = 0.0;
-    ST_CUDA(ctx, cudaMemcpyAsync(&m, ctx->miou_tmp, sizeof m, cudaMemcpyDeviceToHost, ctx->stream));
-    ST_CUDA(ctx, cudaStreamSynchronize(ctx->stream));
-    if (miou) *miou = m;
-    st = report_bad_labels(ctx, 1, "st_agreement");
+    st = fetch_status(ctx);
     if (st != ST_OK) return st;
-    return report_bad_labels(ctx, 0, "an earlier st_distill_step");
+    if (miou) *miou = ctx->status_host[0];
+    return report_status(ctx, true);
 }
 
 st_status st_read_tensor(st_ctx* ctx, int32_t stream, st_tensor which, float* dst_host, size_t dst_capacity, size_t* nbytes)

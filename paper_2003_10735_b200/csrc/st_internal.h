@@ -6,9 +6,36 @@
 #include <cuda_runtime.h>
 #include <stdint.h>
 
+#include <utility>
+
 namespace st {
 
 typedef __nv_bfloat16 bf16;
+
+// ---- programmatic dependent launch -----------------------------------------------------------------
+// The kernels of a step form a chain.  Launched with the programmatic-serialization attribute a kernel
+// may start while its predecessor is still draining; everything it does before pdl_wait() (barrier
+// set-up, tensor-memory allocation, index arithmetic) then overlaps the predecessor's tail.
+// pdl_wait() returns once the predecessor grid has completed and its writes are visible; no global
+// memory is read or written before it.  pdl_launch_dependents() lets the successor start launching.
+#ifdef __CUDACC__
+__device__ __forceinline__ void pdl_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+__device__ __forceinline__ void pdl_launch_dependents() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
+
+bool pdl_enabled();   // false if the environment variable ST_NO_PDL is set to 1
+
+template <typename... KArgs, typename... Args>
+inline cudaError_t launch_chain(void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t smem, cudaStream_t s, Args&&... args)
+{
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = grid; cfg.blockDim = block; cfg.dynamicSmemBytes = smem; cfg.stream = s;
+    cudaLaunchAttribute at[1];
+    at[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    at[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = at; cfg.numAttrs = pdl_enabled() ? 1 : 0;
+    return cudaLaunchKernelEx(&cfg, kernel, std::forward<Args>(args)...);
+}
+#endif
 
 constexpr int kUp = 4;            // bilinear upsample factor of the head (frame = feature map * 4)
 constexpr int kMaxSteps = 64;     // upper bound of n_steps in one st_distill_step call
