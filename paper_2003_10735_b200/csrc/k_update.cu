@@ -13,7 +13,7 @@ namespace st {
 
 bool pdl_enabled()
 {
-    static const bool on = [] { const char* e = getenv("ST_NO_PDL"); return !(e && e[0] == '1'); }();
+    static const bool on = [] { const char* e = getenv("ST_PDL"); return e && e[0] == '1'; }();
     return on;
 }
 
