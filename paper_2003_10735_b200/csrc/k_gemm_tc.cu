@@ -210,33 +210,43 @@ tc_wgrad1x1_kernel(const __grid_constant__ CUtensorMap tmA,   // {K, p, S}      
 }
 
 // ------------------------------------------------------------------------------------------------
-// fwd 3x3 (+bias, ReLU): one tile of 4 rows x 32 columns of pixels per block, N = Ch output channels,
-// K loop = 9 taps x (Cin / 64) channel blocks through a ring of stages.
+// fwd 3x3 (+bias, ReLU), persistent: one block per SM walks the tiles (4 rows x 32 columns of pixels,
+// N = Ch output channels; K loop = 9 taps x Cin/64 channel blocks).  Three roles: warp 0 feeds a ring of
+// shared-memory stages by TMA across tile boundaries (the pipeline never drains), warp 1 issues the
+// MMAs into one of two tensor-memory accumulators, warps 2-5 drain the other accumulator (bias, ReLU,
+// bf16, ReLU bit mask) while the next tile is being multiplied.
 // ------------------------------------------------------------------------------------------------
+constexpr int kFwd3Threads = 192;
+
+__device__ __forceinline__ void mbar_arrive(uint32_t bar)
+{
+    asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
+}
+
 template <int STAGES>
-__global__ void __launch_bounds__(kThreadsTc)
+__global__ void __launch_bounds__(kFwd3Threads)
 tc_fwd3x3_kernel(const __grid_constant__ CUtensorMap tmA,   // {Cin, w, h, S}    box {64, 32, 4, 1}
                  const __grid_constant__ CUtensorMap tmB,   // {Cin, 9*Ch, S}    box {64, Ch, 1}
                  const float* __restrict__ theta, int64_t n_params, int64_t b_off,
                  bf16* __restrict__ hidden,                  // [S][p][Ch]
                  uint32_t* __restrict__ relu_bits,           // [S][p][Ch/32]: bit k of word j = hidden[32j + k] > 0
-                 int Cin, int Ch, int h, int w, int tmem_cols, unsigned int* err)
+                 int Cin, int Ch, int h, int w, int n_tiles_total, int acc_cols, unsigned int* err)
 {
     extern __shared__ uint8_t smem_raw[];
     uint8_t* smem = align_smem(smem_raw);
     const uint32_t base = smem_u32(smem);
     const uint32_t a_bytes = kTileM * 128, b_bytes = (uint32_t)Ch * 128, stage_bytes = a_bytes + b_bytes;
-    __shared__ __align__(8) uint64_t full[STAGES], empty[STAGES], done;
+    __shared__ __align__(8) uint64_t full[STAGES], empty[STAGES], acc_full[2], acc_empty[2];
     __shared__ uint32_t tmem_slot;
-    const int tid = threadIdx.x, warp = tid >> 5;
-    const int tiles_x = (w + kTileW - 1) / kTileW;
-    const int x0 = (blockIdx.x % tiles_x) * kTileW, y0 = (blockIdx.x / tiles_x) * kTileH, s = blockIdx.y;
+    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+    const int tiles_x = (w + kTileW - 1) / kTileW, tiles_y = (h + kTileH - 1) / kTileH;
+    const int tiles_per_stream = tiles_x * tiles_y;
     const int kblocks = Cin / kBlockK, n_iter = 9 * kblocks;
 
-    if (warp == 0) tmem_alloc(smem_u32(&tmem_slot), tmem_cols);
+    if (warp == 0) tmem_alloc(smem_u32(&tmem_slot), 2 * acc_cols);
     if (tid == 0) {
         for (int i = 0; i < STAGES; ++i) { mbar_init(smem_u32(&full[i]), 1); mbar_init(smem_u32(&empty[i]), 1); }
-        mbar_init(smem_u32(&done), 1);
+        for (int i = 0; i < 2; ++i) { mbar_init(smem_u32(&acc_full[i]), 1); mbar_init(smem_u32(&acc_empty[i]), 4); }
         fence_barrier_init();
     }
     tc_fence_before_sync();
@@ -248,65 +258,88 @@ tc_fwd3x3_kernel(const __grid_constant__ CUtensorMap tmA,   // {Cin, w, h, S}   
     bool ok = true;
 
     if (tid == 0) {
-        for (int it = 0; it < n_iter; ++it) {
-            const int st = it % STAGES, tap = it / kblocks, kb = it % kblocks;
-            if (it >= STAGES) ok = mbar_wait(smem_u32(&empty[st]), ((it / STAGES) - 1) & 1, err, kWaitEmpty);
-            if (!ok) break;
-            const uint32_t bar = smem_u32(&full[st]), sa = base + st * stage_bytes;
-            mbar_expect_tx(bar, stage_bytes);
-            tma_load_4d(sa, &tmA, bar, kb * kBlockK, x0 + tap % 3 - 1, y0 + tap / 3 - 1, s);
-            tma_load_3d(sa + a_bytes, &tmB, bar, kb * kBlockK, tap * Ch, s);
-        }
-    } else if (tid == 32) {
-        const uint32_t idesc = instr_desc(kTileM, Ch, 0, 0);
-        for (int it = 0; it < n_iter; ++it) {
-            const int st = it % STAGES;
-            ok = mbar_wait(smem_u32(&full[st]), (it / STAGES) & 1, err, kWaitFull);
-            if (!ok) break;
-            tc_fence_after_sync();
-            const uint32_t sa = base + st * stage_bytes, sb = sa + a_bytes;
-#pragma unroll
-            for (int k = 0; k < 4; ++k)
-                umma(tmem, smem_desc(sa + k * 32, 16, 1024), smem_desc(sb + k * 32, 16, 1024), idesc, (it | k) != 0);
-            umma_commit(smem_u32(&empty[st]));
-        }
-        umma_commit(smem_u32(&done));
-    }
-    __syncwarp();
-    ok = mbar_wait(smem_u32(&done), 0, err, kWaitDone);
-    tc_fence_after_sync();
-    if (ok) {
-        const int y = y0 + tid / kTileW, x = x0 + tid % kTileW;
-        const bool in = y < h && x < w;
-        const float* bias = theta + (int64_t)s * n_params + b_off;
-        const int64_t pixel = (int64_t)s * h * w + (int64_t)y * w + x;
-        bf16* dst = hidden + pixel * Ch;
-        for (int n0 = 0; n0 < Ch; n0 += 32) {
-            float v[32];
-            tmem_ld_32x32(tmem + ((uint32_t)(warp * 32) << 16) + n0, v);
-            if (in) {
-                uint4 out[4];
-                __nv_bfloat162* o2 = reinterpret_cast<__nv_bfloat162*>(out);
-                uint32_t bits = 0;
-#pragma unroll
-                for (int k = 0; k < 16; ++k) {
-                    const float a = fmaxf(v[2 * k] + __ldg(bias + n0 + 2 * k), 0.f), b = fmaxf(v[2 * k + 1] + __ldg(bias + n0 + 2 * k + 1), 0.f);
-                    o2[k] = __floats2bfloat162_rn(a, b);
-                    // the mask is taken on the stored (rounded) activation, the value the next layer sees
-                    bits |= (__low2float(o2[k]) > 0.f ? 1u : 0u) << (2 * k);
-                    bits |= (__high2float(o2[k]) > 0.f ? 1u : 0u) << (2 * k + 1);
-                }
-#pragma unroll
-                for (int k = 0; k < 4; ++k) reinterpret_cast<uint4*>(dst + n0)[k] = out[k];
-                relu_bits[pixel * (Ch / 32) + n0 / 32] = bits;
+        // ---- producer: the ring index runs on across tiles
+        int g = 0;
+        for (int t = blockIdx.x; t < n_tiles_total && ok; t += gridDim.x) {
+            const int s = t / tiles_per_stream, tt = t % tiles_per_stream;
+            const int x0 = (tt % tiles_x) * kTileW, y0 = (tt / tiles_x) * kTileH;
+            for (int it = 0; it < n_iter; ++it, ++g) {
+                const int st = g % STAGES, tap = it / kblocks, kb = it % kblocks;
+                if (g >= STAGES) ok = mbar_wait(smem_u32(&empty[st]), ((g / STAGES) - 1) & 1, err, kWaitEmpty);
+                if (!ok) break;
+                const uint32_t bar = smem_u32(&full[st]), sa = base + st * stage_bytes;
+                mbar_expect_tx(bar, stage_bytes);
+                tma_load_4d(sa, &tmA, bar, kb * kBlockK, x0 + tap % 3 - 1, y0 + tap / 3 - 1, s);
+                tma_load_3d(sa + a_bytes, &tmB, bar, kb * kBlockK, tap * Ch, s);
             }
         }
-    } else {
-        drain_after_error();
+    } else if (tid == 32) {
+        // ---- MMA issuer
+        const uint32_t idesc = instr_desc(kTileM, Ch, 0, 0);
+        int g = 0, j = 0;
+        for (int t = blockIdx.x; t < n_tiles_total && ok; t += gridDim.x, ++j) {
+            const int buf = j & 1;
+            if (j >= 2) ok = mbar_wait(smem_u32(&acc_empty[buf]), ((j >> 1) - 1) & 1, err, kWaitEmpty);
+            if (!ok) break;
+            tc_fence_after_sync();
+            const uint32_t acc = tmem + buf * acc_cols;
+            for (int it = 0; it < n_iter; ++it, ++g) {
+                const int st = g % STAGES;
+                ok = mbar_wait(smem_u32(&full[st]), (g / STAGES) & 1, err, kWaitFull);
+                if (!ok) break;
+                tc_fence_after_sync();
+                const uint32_t sa = base + st * stage_bytes, sb = sa + a_bytes;
+#pragma unroll
+                for (int k = 0; k < 4; ++k)
+                    umma(acc, smem_desc(sa + k * 32, 16, 1024), smem_desc(sb + k * 32, 16, 1024), idesc, (it | k) != 0);
+                umma_commit(smem_u32(&empty[st]));
+            }
+            if (ok) umma_commit(smem_u32(&acc_full[buf]));
+        }
+    } else if (warp >= 2) {
+        // ---- epilogue warps: TMEM lanes 32*(warp % 4) .. +31 = pixel rows of the tile
+        const int q = warp & 3, row = q * 32 + lane;
+        int j = 0;
+        for (int t = blockIdx.x; t < n_tiles_total && ok; t += gridDim.x, ++j) {
+            const int buf = j & 1;
+            const int s = t / tiles_per_stream, tt = t % tiles_per_stream;
+            const int x = (tt % tiles_x) * kTileW + row % kTileW, y = (tt / tiles_x) * kTileH + row / kTileW;
+            ok = mbar_wait(smem_u32(&acc_full[buf]), (j >> 1) & 1, err, kWaitDone);
+            if (!ok) break;
+            tc_fence_after_sync();
+            const bool in = y < h && x < w;
+            const float* bias = theta + (int64_t)s * n_params + b_off;
+            const int64_t pixel = (int64_t)s * h * w + (int64_t)y * w + x;
+            bf16* dst = hidden + pixel * Ch;
+            for (int n0 = 0; n0 < Ch; n0 += 32) {
+                float v[32];
+                tmem_ld_32x32(tmem + ((uint32_t)(q * 32) << 16) + buf * acc_cols + n0, v);
+                if (in) {
+                    uint4 out[4];
+                    __nv_bfloat162* o2 = reinterpret_cast<__nv_bfloat162*>(out);
+                    uint32_t bits = 0;
+#pragma unroll
+                    for (int k = 0; k < 16; ++k) {
+                        const float a = fmaxf(v[2 * k] + __ldg(bias + n0 + 2 * k), 0.f), b = fmaxf(v[2 * k + 1] + __ldg(bias + n0 + 2 * k + 1), 0.f);
+                        o2[k] = __floats2bfloat162_rn(a, b);
+                        // the mask is taken on the stored (rounded) activation, the value the next layer sees
+                        bits |= (__low2float(o2[k]) > 0.f ? 1u : 0u) << (2 * k);
+                        bits |= (__high2float(o2[k]) > 0.f ? 1u : 0u) << (2 * k + 1);
+                    }
+#pragma unroll
+                    for (int k = 0; k < 4; ++k) reinterpret_cast<uint4*>(dst + n0)[k] = out[k];
+                    relu_bits[pixel * (Ch / 32) + n0 / 32] = bits;
+                }
+            }
+            tc_fence_before_sync();
+            __syncwarp();
+            if (lane == 0) mbar_arrive(smem_u32(&acc_empty[buf]));     // this warp's quarter of the accumulator is free
+        }
     }
+    if (!ok) drain_after_error();
     tc_fence_before_sync();
     __syncthreads();
-    if (warp == 0) tmem_dealloc(tmem, tmem_cols);
+    if (warp == 0) tmem_dealloc(tmem, 2 * acc_cols);
 }
 
 // ------------------------------------------------------------------------------------------------
@@ -589,6 +622,7 @@ struct TcPlan {
     int split2, chunks2, per2, cols2;
     int split1, chunks1, per1, cols1;
     size_t smem_fwd1, smem_wg1, smem_fwd3, smem_wg3, smem_dgrad;
+    int n_sms;
 };
 
 int tc_wgrad_splits(int layer, int c_in, int c_hidden, int h, int w)
@@ -615,6 +649,11 @@ TcPlan* tc_plan_create(const TcBuffers& b, char* err, size_t err_len)
     memset((void*)P, 0, sizeof *P);
     P->b = b;
     P->p = b.h * b.w; P->p_pad = tc_dz_pitch(b.h, b.w);
+    {
+        int dev = 0;
+        cudaGetDevice(&dev);
+        if (cudaDeviceGetAttribute(&P->n_sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || P->n_sms < 1) P->n_sms = 148;
+    }
     P->c_last = b.c_hidden ? b.c_hidden : b.c_in;
     const uint64_t S = (uint64_t)b.S, p = (uint64_t)P->p, cl = (uint64_t)P->c_last;
     const bf16* act = b.c_hidden ? b.hidden : b.x;
@@ -693,9 +732,10 @@ int tc_forward(const TcPlan* P, cudaStream_t s, StageTimer* t)
     int n = 0;
     if (b.c_hidden) {
         const int tiles = ((b.w + kTileW - 1) / kTileW) * ((b.h + kTileH - 1) / kTileH);
-        launch_chain(tc_fwd3x3_kernel<4>, dim3(tiles, b.S), dim3(kThreadsTc), P->smem_fwd3, s,
+        const int total = tiles * b.S;
+        launch_chain(tc_fwd3x3_kernel<4>, dim3(total < P->n_sms ? total : P->n_sms), dim3(kFwd3Threads), P->smem_fwd3, s,
             P->x_fwd3, P->w1_map, b.theta, b.n_params, b.b1_off, b.hidden, b.relu_bits, b.c_in, b.c_hidden, b.h, b.w,
-            pow2_cols(b.c_hidden), b.err);
+            total, pow2_cols(b.c_hidden), b.err);
         if (t) t->mark("tc_fwd3x3", s);
         ++n;
     }
