@@ -33,6 +33,8 @@ import synth_inputs as si  # noqa: E402
 METRIC = "720p key-frame partial-distill steps/s (K=8)"
 N_SETS = 4            # distinct key frames the device-resident run rotates over (4 x 136 MB > 126 MB L2)
 ALU_FLOP_PER_CLASS_PIXEL = 20.0   # algorithmic fp32 work of the fused upsample+CE kernel (10 FMA-equivalents)
+# dram__bytes_read.sum + dram__bytes_write.sum per launch, ncu capture of (workload, kernel); see profiles/
+NCU_DRAM_BYTES = {(2, "upsample_ce"): 5.88e6}
 
 
 def read_peaks():
@@ -354,8 +356,10 @@ def run_ours(args, cfg):
             dominant = max((n for n in kernels if "frac" in kernels[n] or True),
                            key=lambda n: kernels[n]["ms"] * kernels[n]["per_key_frame"])
             dk = kernels[dominant]
+            # DRAM bytes per launch from the ncu capture summarised in profiles/ (same kernel, same workload)
+            traffic = NCU_DRAM_BYTES.get((args.workload, dominant))
             roofline = {"kernel": dominant, "bound": dk.get("bound"), "achieved": dk.get("achieved"), "peak": dk.get("peak"),
-                        "unit": dk.get("unit"), "frac": dk.get("frac"), "traffic": None,
+                        "unit": dk.get("unit"), "frac": dk.get("frac"), "traffic": traffic,
                         "peak_source": f"of {peaks['source']}" if dk.get("bound") in ("hbm", "tensor") else
                                        "148 SMs x 128 fp32 lanes x 2 flop x max SM clock",
                         "ms_per_launch": dk["ms"]}
