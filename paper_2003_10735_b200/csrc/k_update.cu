@@ -63,9 +63,18 @@ sgd_update_kernel(UpdateArgs a, int n_param_blocks, int64_t range_begin)
                 const LayerUpdate& ly = a.layer[layer[e]];
                 has_partials[e] = true;
                 const float* src = ly.w_partials + (int64_t)s * ly.w_stream_stride + (i - ly.w_off);
+                // batches of 8 predicated loads: all in flight together, no one-at-a-time remainder loop
                 float t = 0.f;
-#pragma unroll 16
-                for (int k = g; k < ly.n_split; k += G) t += __ldg(src + (int64_t)k * ly.w_split_stride);
+                for (int k0 = g; k0 < ly.n_split; k0 += 8 * G) {
+                    float v[8];
+#pragma unroll
+                    for (int j = 0; j < 8; ++j) {
+                        const int k = k0 + j * G;
+                        v[j] = k < ly.n_split ? __ldg(src + (int64_t)k * ly.w_split_stride) : 0.f;
+                    }
+#pragma unroll
+                    for (int j = 0; j < 8; ++j) t += v[j];
+                }
                 sum[e] = t;
             }
         }
@@ -105,8 +114,16 @@ sgd_update_kernel(UpdateArgs a, int n_param_blocks, int64_t range_begin)
         if (item < ly.cout) {
             const float* src = ly.b_partials + (int64_t)s * ly.n_bpart * ly.cout + item;
             float g = 0.f;
-#pragma unroll 16
-            for (int k = lane; k < ly.n_bpart; k += 32) g += __ldg(src + (int64_t)k * ly.cout);
+            for (int k0 = lane; k0 < ly.n_bpart; k0 += 8 * 32) {
+                float v[8];
+#pragma unroll
+                for (int j = 0; j < 8; ++j) {
+                    const int k = k0 + j * 32;
+                    v[j] = k < ly.n_bpart ? __ldg(src + (int64_t)k * ly.cout) : 0.f;
+                }
+#pragma unroll
+                for (int j = 0; j < 8; ++j) g += v[j];
+            }
 #pragma unroll
             for (int o = 16; o > 0; o >>= 1) g += __shfl_xor_sync(0xffffffffu, g, o);
             if (lane == 0) apply_update(a, base + ly.b_off + item, g);
@@ -116,8 +133,16 @@ sgd_update_kernel(UpdateArgs a, int n_param_blocks, int64_t range_begin)
     }
     if (item == 0 && a.loss_part) {
         double t = 0.0;
-#pragma unroll 16
-        for (int k = lane; k < a.n_loss_part; k += 32) t += (double)__ldg(a.loss_part + (int64_t)s * a.n_loss_part + k);
+        for (int k0 = lane; k0 < a.n_loss_part; k0 += 8 * 32) {
+            float v[8];
+#pragma unroll
+            for (int j = 0; j < 8; ++j) {
+                const int k = k0 + j * 32;
+                v[j] = k < a.n_loss_part ? __ldg(a.loss_part + (int64_t)s * a.n_loss_part + k) : 0.f;
+            }
+#pragma unroll
+            for (int j = 0; j < 8; ++j) t += (double)v[j];
+        }
 #pragma unroll
         for (int o = 16; o > 0; o >>= 1) t += __shfl_xor_sync(0xffffffffu, t, o);
         if (lane == 0) {
@@ -144,13 +169,21 @@ sgd_update_stream_kernel(UpdateArgs a, int L)
     float g[VEC];
 #pragma unroll
     for (int j = 0; j < VEC; ++j) g[j] = 0.f;
-#pragma unroll 8
-    for (int k = 0; k < ly.n_split; ++k) {
+    for (int k0 = 0; k0 < ly.n_split; k0 += 8) {
         if (VEC == 4) {
-            const float4 t = __ldg(reinterpret_cast<const float4*>(src + (int64_t)k * ly.w_split_stride));
-            g[0] += t.x; g[1] += t.y; g[2] += t.z; g[3] += t.w;
+            float4 t[8];
+#pragma unroll
+            for (int j = 0; j < 8; ++j)
+                t[j] = k0 + j < ly.n_split ? __ldg(reinterpret_cast<const float4*>(src + (int64_t)(k0 + j) * ly.w_split_stride))
+                                           : make_float4(0.f, 0.f, 0.f, 0.f);
+#pragma unroll
+            for (int j = 0; j < 8; ++j) { g[0] += t[j].x; g[1] += t[j].y; g[2] += t[j].z; g[3] += t[j].w; }
         } else {
-            g[0] += __ldg(src + (int64_t)k * ly.w_split_stride);
+            float t[8];
+#pragma unroll
+            for (int j = 0; j < 8; ++j) t[j] = k0 + j < ly.n_split ? __ldg(src + (int64_t)(k0 + j) * ly.w_split_stride) : 0.f;
+#pragma unroll
+            for (int j = 0; j < 8; ++j) g[0] += t[j];
         }
     }
     const int64_t gi = (int64_t)s * a.n_params + ly.w_off + e;
