@@ -343,3 +343,22 @@ def test_steps_are_bit_reproducible():
         outs.append(packed(ctx))
         st.st_destroy(ctx)
     assert outs[0].tobytes() == outs[1].tobytes()
+
+
+def test_profile_step_times_every_kernel_and_takes_real_steps():
+    c_in, C, h, w = 8, 5, 9, 13
+    feat, T = rand_problem(9, c_in, C, h, w)
+    theta = si.initial_head_params(c_in, 0, C, 2)
+    ctx = make_ctx(c_in, 0, C, h, w, theta, lr=0.05)
+    st.st_set_frozen_features(ctx, 0, dev(feat)); st.st_teacher_labels(ctx, 0, dev(T))
+    stages = st.st_profile_step(ctx, 2)
+    names = [n for n, _ in stages]
+    assert names == ["conv1x1_fwd_f32", "upsample_ce", "conv1x1_wgrad_f32", "sgd_update"]
+    assert all(ms > 0 for _, ms in stages)
+    head = oracle.Head(c_in, 0, C, lr=0.05, theta=theta)
+    lab = oracle.teacher_labels(T)
+    for _ in range(2):
+        oracle.distill_step(head, feat, lab)
+    np.testing.assert_allclose(packed(ctx), head.theta, rtol=1e-4, atol=1e-6)     # the profiled steps are ordinary steps
+    assert st.st_launch_count(ctx) >= 8
+    st.st_destroy(ctx)
