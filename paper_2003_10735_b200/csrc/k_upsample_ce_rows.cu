@@ -10,7 +10,14 @@
 // of cell row y0-1+i; lane l owns node column x0-1+l and handles the four pixels of the cell to its
 // right.  Warp 0, lane 0 and lane 31 are halo (recomputed by the neighbouring block) so that a block
 // finishes its nodes alone, in a fixed summation order, without floating-point atomics.
-// Per frame row:
+// Fast path (smooth logits, the usual case), class by class for all 16 pixels of the lane's cell at once:
+// inside a cell the interpolated logit of a class is u(r,k) = A + B k + G r + D k r (r = frame row,
+// k = pixel in the row), so its 16 exponentials form geometric progressions: four exp2 (of A, B, G, D)
+// and 18 multiplications replace 16 exp2.  Pass 1 sums them per pixel; pass 2 forms them again,
+// multiplies by the adjoint interpolation weights / Z and reduces them to the cell's contribution to
+// its upper node row (kept in registers) and lower node row (shared memory).
+// Slow path (a class changing by more than 16 log2-units across a cell, or a sum that underflows): the
+// warp walks its four frame rows one by one with exact per-pixel maxima:
 //   pass 1  each lane interpolates its own node column vertically, takes the right neighbour's by
 //           shuffle, interpolates its four pixels horizontally, and sums exp2(u - M) over the classes
 //           (logits are pre-scaled by log2 e; M is the largest logit of the warp's two node rows);
@@ -95,8 +102,56 @@ __device__ __forceinline__ void pass2(const RowCtx& rc, const float (&sk)[4], co
     }
 }
 
+// The 16 exponentials exp2(u(r,k) - M) of one class inside the lane's cell, u bilinear between the four
+// corner logits (own column: rows i, i+1 from shared memory; right column from the next lane).
+// With ly_r = (2r+1)/8 and fr_k = (2k+1)/8:  u(r,k) = A + B k + G r + D k r, so the values are geometric
+// progressions along k and r: 4 exp2 and 18 multiplications.  Returns the largest corner difference
+// (the caller leaves the fast path if a class changes by more than 16 across the cell: the progressions
+// would lose their small terms).
+__device__ __forceinline__ float cell_exponentials(const float* q, float M, float (&E)[16])
+{
+    const float a = q[0] - M, b = q[TZ_W] - M;
+    const float ar = __shfl_down_sync(0xffffffffu, a, 1), br = __shfl_down_sync(0xffffffffu, b, 1);
+    const float p = b - a, qq = br - ar, e0 = ar - a;
+    const float qp = qq - p;
+    const float wv = fmaf(qp, 0.125f, e0);
+    const float A = fmaf(wv, 0.125f, fmaf(p, 0.125f, a));
+    const float E00 = ex2_approx(A), QB = ex2_approx(0.25f * wv), TG = ex2_approx(fmaf(qp, 0.03125f, 0.25f * p)),
+                SD = ex2_approx(0.0625f * qp);
+    float Er = E00, Qr = QB;
+#pragma unroll
+    for (int r = 0; r < 4; ++r) {
+        E[4 * r] = Er;
+        E[4 * r + 1] = Er * Qr;
+        E[4 * r + 2] = E[4 * r + 1] * Qr;
+        E[4 * r + 3] = E[4 * r + 2] * Qr;
+        Er *= TG;
+        Qr *= SD;
+    }
+    return fmaxf(fabsf(p), fmaxf(fabsf(qq), fabsf(e0)));
+}
+
+// pass 2 of one row on the slow path: like pass2, accumulating the upper part in registers and the lower part in
+// this thread's shared-memory slots
+template <int CB>
+__device__ __forceinline__ void pass2_slow(const RowCtx& rc, const float (&sk)[4], const float (&wl)[4], const float (&wr)[4],
+                                           float tw, float bw, float (&top)[CB], float* my_bot, int C)
+{
+#pragma unroll
+    for (int c = 0; c < CB; ++c) {
+        float u[4];
+        pixel_logits<true>(rc, c, sk, u);
+        const float e0 = ex2_approx(u[0]), e1 = ex2_approx(u[1]), e2 = ex2_approx(u[2]), e3 = ex2_approx(u[3]);
+        const float aL = fmaf(wl[0], e0, fmaf(wl[1], e1, fmaf(wl[2], e2, wl[3] * e3)));
+        const float aR = fmaf(wr[0], e0, fmaf(wr[1], e1, fmaf(wr[2], e2, wr[3] * e3)));
+        const float hs = aL + __shfl_up_sync(0xffffffffu, aR, 1);
+        top[c] = fmaf(tw, hs, top[c]);
+        if (c < C) my_bot[c * 32] = fmaf(bw, hs, my_bot[c * 32]);
+    }
+}
+
 template <int CB, bool CONF>
-__global__ void __launch_bounds__(R_THREADS, CB > 16 ? 2 : 3)
+__global__ void __launch_bounds__(R_THREADS, 2)
 upsample_ce_rows_kernel(UpsampleCeArgs a)
 {
     extern __shared__ __align__(16) float smem_r[];
@@ -104,7 +159,7 @@ upsample_ce_rows_kernel(UpsampleCeArgs a)
     float* zt = smem_r;                         // [CB][TZ_H][36]   logits * log2(e), borders replicated; classes >= C
                                                 //                  hold -1e30 (their exponentials are 0)
     int* corr = (int*)(zt + CB * TZ);           // [C][TZ_H][36]    -64 * (adjoint of onehot)
-    float* bsh = zt;                            // [R_WARPS][C][32] lower-row accumulators (reuses the tile once the rows are done)
+    float* bsh = (float*)(corr + C * TZ);       // [R_WARPS][C][32] lower-row accumulators
     __shared__ float red[R_WARPS];
     __shared__ float dbs[R_WARPS][32];
 
@@ -173,121 +228,176 @@ upsample_ce_rows_kernel(UpsampleCeArgs a)
         rc.M = m;
     }
 
-    float top[CB], bot[CB];
+    float top[CB];
 #pragma unroll
-    for (int c = 0; c < CB; ++c) { top[c] = 0.f; bot[c] = 0.f; }
+    for (int c = 0; c < CB; ++c) top[c] = 0.f;
     float loss = 0.f;
     unsigned n_bad = 0;
+    float* my_bot = bsh + (size_t)wi * C * 32 + l;             // this thread's slot of class c: my_bot[c * 32]
 
+    // labels of the lane's 16 pixels (rows 4i+2 .. 4i+5, columns 4n+2 .. 4n+5), two aligned 16-bit loads per row;
+    // bit 4r+k of vmask: pixel k of row r lies inside the frame
+    uint32_t labw[4], vmask = 0;
+    const int X0 = 4 * n + 2;
+    const bool v01 = cell_valid && X0 >= 0 && X0 + 1 < W, v23 = cell_valid && X0 + 2 >= 0 && X0 + 3 < W;
+#pragma unroll
     for (int r = 0; r < 4; ++r) {
         const int Y = 4 * i + 2 + r;
-        if (!(cell_row_valid && Y >= 0 && Y < H)) continue;          // warp-uniform
-        rc.ly = (2 * r + 1) * 0.125f;
+        uint32_t lo = 0, hi = 0;
+        if (cell_row_valid && Y >= 0 && Y < H) {
+            if (v01) { lo = __ldg(reinterpret_cast<const unsigned short*>(labels + (int64_t)Y * W + X0)); vmask |= 0x3u << (4 * r); }
+            if (v23) { hi = __ldg(reinterpret_cast<const unsigned short*>(labels + (int64_t)Y * W + X0 + 2)); vmask |= 0xcu << (4 * r); }
+        }
+        labw[r] = lo | (hi << 16);
+    }
+    // at the clamped left and right borders the outer node column is the inner one
+    const bool fold_l = n == -1, fold_r = n == w - 1;
+
+    // per pixel of one row: loss, 1/Z, the "- onehot" part of the adjoint (integer, exact), confusion; returns the
+    // horizontal adjoint weights (already divided by Z) of the row's four pixels
+    auto finish_row = [&](int r, const float (&Zs)[4], const float (&sk)[4], const uint32_t (&arg)[4], float (&wl)[4], float (&wr)[4]) {
+        const int Y = 4 * i + 2 + r;
+        const float ly = (2 * r + 1) * 0.125f;
         const bool row_owned = (Y >> 2) >= y0 && (Y >> 2) < y0 + RN_Y;
-        // labels of pixels 4n+2 .. 4n+5 (two aligned 16-bit loads)
-        const int X0 = 4 * n + 2;
+        const int wy1 = 2 * r + 1, wy0 = 8 - wy1;                // eighths toward node rows i+1 / i
         int lab[4];
-        bool pv[4];
-        {
-            uint32_t lo = 0xffff, hi = 0xffff;
-            const bool v01 = cell_valid && X0 >= 0 && X0 + 1 < W, v23 = cell_valid && X0 + 2 >= 0 && X0 + 3 < W;
-            if (v01) lo = __ldg(reinterpret_cast<const unsigned short*>(labels + (int64_t)Y * W + X0));
-            if (v23) hi = __ldg(reinterpret_cast<const unsigned short*>(labels + (int64_t)Y * W + X0 + 2));
-            lab[0] = lo & 0xff; lab[1] = lo >> 8; lab[2] = hi & 0xff; lab[3] = hi >> 8;
-            pv[0] = pv[1] = v01; pv[2] = pv[3] = v23;
-        }
-        // ownership of a pixel = ownership of its node-aligned group (X >> 2)
-        bool own[4];
 #pragma unroll
         for (int k = 0; k < 4; ++k) {
+            lab[k] = (labw[r] >> (8 * k)) & 0xff;
             const int gx = (X0 + k) >> 2;
-            own[k] = pv[k] && row_owned && gx >= x0 && gx < x0 + RN_X;
-            if (pv[k] && lab[k] >= C) { if (own[k]) n_bad++; lab[k] = -1; }
-            if (!pv[k]) lab[k] = -1;
-        }
-
-        float sk[4] = {0.f, 0.f, 0.f, 0.f}, Zs[4];
-        uint32_t arg[4] = {0, 0, 0, 0};
-        pass1<CB, CONF, false>(rc, sk, Zs, arg);
-        bool under = false;
-#pragma unroll
-        for (int k = 0; k < 4; ++k) under |= pv[k] && !(Zs[k] > 1e-30f);
-        const bool slow = __any_sync(0xffffffffu, under);
-        if (slow) {
-            // exact per-pixel maxima, then the sums again
-            float ex[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};
-            const float zero[4] = {0.f, 0.f, 0.f, 0.f};
-            for (int c = 0; c < C; ++c) {
-                float u[4];
-                pixel_logits<false>(rc, c, zero, u);
-#pragma unroll
-                for (int k = 0; k < 4; ++k) ex[k] = fmaxf(ex[k], u[k]);
-            }
-#pragma unroll
-            for (int k = 0; k < 4; ++k) sk[k] = ex[k];
-            uint32_t dummy[4];
-            pass1<CB, false, true>(rc, sk, Zs, dummy);
-        }
-
-        // ---- per pixel: loss, 1/Z, the "- onehot" part of the adjoint (integer, exact), confusion
-        float wl[4], wr[4];
-        // four valid pixels with one label (the usual case): their onehot parts add up to 16 eighths per side
-        const bool same_label = lab[0] >= 0 && lab[0] == lab[1] && lab[1] == lab[2] && lab[2] == lab[3];
-        const int wy1 = 2 * r + 1, wy0 = 8 - wy1;                    // eighths toward node rows i+1 / i
-        const bool fold_l = n == -1, fold_r = n == w - 1;            // clamped borders: the outer node is the inner one
-#pragma unroll
-        for (int k = 0; k < 4; ++k) {
+            const bool valid = (vmask >> (4 * r + k)) & 1u;
+            const bool own = valid && row_owned && gx >= x0 && gx < x0 + RN_X;
+            if (valid && lab[k] >= C) { if (own) n_bad++; lab[k] = -1; }
+            if (!valid) lab[k] = -1;
             float rz = 0.f;
             if (lab[k] >= 0) {
-                rz = 1.0f / Zs[k];
-                const float* q = rc.za + lab[k] * TZ;
-                const float vl = fmaf(rc.ly, q[TZ_W] - q[0], q[0]), vr = fmaf(rc.ly, q[TZ_W + 1] - q[1], q[1]);
-                const float ul = fmaf((2 * k + 1) * 0.125f, vr - vl, vl) - rc.M - sk[k];
-                if (own[k]) {
+                rz = __frcp_rn(Zs[k]);
+                if (own) {
+                    const float* q = rc.za + lab[k] * TZ;
+                    const float vl = fmaf(ly, q[TZ_W] - q[0], q[0]), vr = fmaf(ly, q[TZ_W + 1] - q[1], q[1]);
+                    const float ul = fmaf((2 * k + 1) * 0.125f, vr - vl, vl) - rc.M - sk[k];
                     loss += (__log2f(Zs[k]) - ul) * kLn2;
                     if (CONF) atomicAdd(a.conf + (int64_t)s * a.conf_stream_stride + lab[k] * C + arg[k], 1ull);
-                }
-                if (!same_label) {
-                    const int wb = 2 * k + 1, wa = 8 - wb;           // eighths toward node columns n+1 / n
-                    int* cc = corr + lab[k] * TZ;
-                    atomicAdd(cc + ry_top * TZ_W + rx_l, -wy0 * wa);
-                    atomicAdd(cc + ry_top * TZ_W + rx_r, -wy0 * wb);
-                    atomicAdd(cc + ry_bot * TZ_W + rx_l, -wy1 * wa);
-                    atomicAdd(cc + ry_bot * TZ_W + rx_r, -wy1 * wb);
                 }
             }
             const float fr = (2 * k + 1) * 0.125f;
             wl[k] = (fold_l ? 0.f : (fold_r ? 1.0f : 1.0f - fr)) * rz;
             wr[k] = (fold_r ? 0.f : (fold_l ? 1.0f : fr)) * rz;
         }
-        if (same_label) {
+        // four valid pixels with one label (the usual case): their onehot parts add up to 16 eighths per side
+        if (lab[0] >= 0 && lab[0] == lab[1] && lab[1] == lab[2] && lab[2] == lab[3]) {
             int* cc = corr + lab[0] * TZ;
             atomicAdd(cc + ry_top * TZ_W + rx_l, -wy0 * 16);
             atomicAdd(cc + ry_top * TZ_W + rx_r, -wy0 * 16);
             atomicAdd(cc + ry_bot * TZ_W + rx_l, -wy1 * 16);
             atomicAdd(cc + ry_bot * TZ_W + rx_r, -wy1 * 16);
+        } else {
+#pragma unroll
+            for (int k = 0; k < 4; ++k)
+                if (lab[k] >= 0) {
+                    const int wb = 2 * k + 1, wa = 8 - wb;       // eighths toward node columns n+1 / n
+                    int* cc = corr + lab[k] * TZ;
+                    atomicAdd(cc + ry_top * TZ_W + rx_l, -wy0 * wa);
+                    atomicAdd(cc + ry_top * TZ_W + rx_r, -wy0 * wb);
+                    atomicAdd(cc + ry_bot * TZ_W + rx_l, -wy1 * wa);
+                    atomicAdd(cc + ry_bot * TZ_W + rx_r, -wy1 * wb);
+                }
         }
-        if (slow) pass2<CB, true>(rc, sk, wl, wr, top, bot);
-        else pass2<CB, false>(rc, sk, wl, wr, top, bot);
-    }
-    // clamped borders in y
-    if (i == -1) {
+    };
+
+    if (cell_row_valid) {                                        // warp-uniform
+        // ---------------- fast path, pass 1: sums of exponentials of the 16 pixels
+        float Z[16];
 #pragma unroll
-        for (int c = 0; c < CB; ++c) bot[c] += top[c];
-    }
-    if (i == h - 1) {
+        for (int j = 0; j < 16; ++j) Z[j] = 0.f;
+        float wmax = 0.f;
 #pragma unroll
-        for (int c = 0; c < CB; ++c) { top[c] += bot[c]; bot[c] = 0.f; }
+        for (int c = 0; c < CB; ++c) {
+            float E[16];
+            wmax = fmaxf(wmax, cell_exponentials(rc.za + c * TZ, rc.M, E));
+#pragma unroll
+            for (int j = 0; j < 16; ++j) Z[j] += E[j];
+        }
+        bool bad = !(wmax <= 16.0f);
+#pragma unroll
+        for (int j = 0; j < 16; ++j) bad |= ((vmask >> j) & 1u) && !(Z[j] > 1e-18f);
+        const bool slow = __any_sync(0xffffffffu, bad);
+        if (!slow) {
+            float wl[16], wr[16];
+            const float zero4[4] = {0.f, 0.f, 0.f, 0.f};
+#pragma unroll
+            for (int r = 0; r < 4; ++r) {
+                const float Zr[4] = {Z[4 * r], Z[4 * r + 1], Z[4 * r + 2], Z[4 * r + 3]};
+                uint32_t ar4[4] = {0, 0, 0, 0};
+                if (CONF) {                                          // the student's class: arg-max of the interpolated logits
+                    float Zd[4];
+                    rc.ly = (2 * r + 1) * 0.125f;
+                    pass1<CB, true, false>(rc, zero4, Zd, ar4);
+                }
+                float wl4[4], wr4[4];
+                finish_row(r, Zr, zero4, ar4, wl4, wr4);
+#pragma unroll
+                for (int k = 0; k < 4; ++k) { wl[4 * r + k] = wl4[k]; wr[4 * r + k] = wr4[k]; }
+            }
+            // vertical weights of the rows toward the upper / lower node row (clamped borders fold into the inner row)
+            float tw[4], bw[4];
+#pragma unroll
+            for (int r = 0; r < 4; ++r) {
+                const float ly = (2 * r + 1) * 0.125f;
+                tw[r] = i == -1 ? 0.f : (i == h - 1 ? 1.0f : 1.0f - ly);
+                bw[r] = i == h - 1 ? 0.f : (i == -1 ? 1.0f : ly);
+            }
+            // ---------------- fast path, pass 2
+#pragma unroll
+            for (int c = 0; c < CB; ++c) {
+                float E[16];
+                cell_exponentials(rc.za + c * TZ, rc.M, E);
+                float tc = 0.f, bc = 0.f;
+#pragma unroll
+                for (int r = 0; r < 4; ++r) {
+                    const float aL = fmaf(wl[4 * r], E[4 * r], fmaf(wl[4 * r + 1], E[4 * r + 1], fmaf(wl[4 * r + 2], E[4 * r + 2], wl[4 * r + 3] * E[4 * r + 3])));
+                    const float aR = fmaf(wr[4 * r], E[4 * r], fmaf(wr[4 * r + 1], E[4 * r + 1], fmaf(wr[4 * r + 2], E[4 * r + 2], wr[4 * r + 3] * E[4 * r + 3])));
+                    const float hs = aL + __shfl_up_sync(0xffffffffu, aR, 1);
+                    tc = fmaf(tw[r], hs, tc);
+                    bc = fmaf(bw[r], hs, bc);
+                }
+                top[c] = tc;
+                if (c < C) my_bot[c * 32] = bc;
+            }
+        } else {
+            // ---------------- slow path: row by row, exact per-pixel maxima
+            for (int c = 0; c < C; ++c) my_bot[c * 32] = 0.f;
+            for (int r = 0; r < 4; ++r) {
+                const int Y = 4 * i + 2 + r;
+                if (!(Y >= 0 && Y < H)) continue;                    // warp-uniform
+                rc.ly = (2 * r + 1) * 0.125f;
+                float ex[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};
+                const float zero4[4] = {0.f, 0.f, 0.f, 0.f};
+                for (int c = 0; c < C; ++c) {
+                    float u[4];
+                    pixel_logits<false>(rc, c, zero4, u);
+#pragma unroll
+                    for (int k = 0; k < 4; ++k) ex[k] = fmaxf(ex[k], u[k]);
+                }
+                float Zs[4];
+                uint32_t ar4[4] = {0, 0, 0, 0};
+                if (CONF) pass1<CB, true, false>(rc, zero4, Zs, ar4);    // arg-max of the interpolated logits
+                pass1<CB, false, true>(rc, ex, Zs, ar4);
+                float wl4[4], wr4[4];
+                finish_row(r, Zs, ex, ar4, wl4, wr4);
+                const float twr = i == -1 ? 0.f : (i == h - 1 ? 1.0f : 1.0f - rc.ly);
+                const float bwr = i == h - 1 ? 0.f : (i == -1 ? 1.0f : rc.ly);
+                pass2_slow<CB>(rc, ex, wl4, wr4, twr, bwr, top, my_bot, C);
+            }
+        }
+    } else {
+        for (int c = 0; c < C; ++c) my_bot[c * 32] = 0.f;
     }
     // loss of the block, fixed order
 #pragma unroll
     for (int o = 16; o > 0; o >>= 1) loss += __shfl_xor_sync(0xffffffffu, loss, o);
     if (l == 0) red[wi] = loss;
     if (n_bad) atomicAdd(a.bad, n_bad);
-    __syncthreads();                            // every warp is done reading the tile: reuse it
-#pragma unroll
-    for (int c = 0; c < CB; ++c)
-        if (c < C) bsh[(wi * C + c) * 32 + l] = bot[c];
     __syncthreads();
 
     // ---- node row y0-1+wi (warps 1..RN_Y): own upper part + lower part of the warp above + onehot part
@@ -328,8 +438,7 @@ upsample_ce_rows_kernel(UpsampleCeArgs a)
 template <int CB>
 size_t rows_smem_bytes(int C)
 {
-    const size_t tile = (size_t)CB * TZ, bsh = (size_t)R_WARPS * C * 32;
-    return ((tile > bsh ? tile : bsh) + (size_t)C * TZ) * sizeof(float) + 16;
+    return ((size_t)CB * TZ + (size_t)C * TZ + (size_t)R_WARPS * C * 32) * sizeof(float) + 16;
 }
 
 template <int CB>
