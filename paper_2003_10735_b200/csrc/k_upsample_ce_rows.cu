@@ -47,6 +47,13 @@ __device__ __forceinline__ float ex2_approx(float x)
     return y;
 }
 
+__device__ __forceinline__ float rcp_approx(float x)
+{
+    float y;
+    asm("rcp.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
+    return y;
+}
+
 struct RowCtx {
     const float* za;     // own column, upper node row, class 0
     float ly;            // weight toward the lower node row
@@ -161,7 +168,6 @@ upsample_ce_rows_kernel(UpsampleCeArgs a)
     int* corr = (int*)(zt + CB * TZ);           // [C][TZ_H][36]    -64 * (adjoint of onehot)
     float* bsh = (float*)(corr + C * TZ);       // [R_WARPS][C][32] lower-row accumulators
     __shared__ float red[R_WARPS];
-    __shared__ float dbs[R_WARPS][32];
 
     const int s = blockIdx.z, x0 = blockIdx.x * RN_X, y0 = blockIdx.y * RN_Y;
     const int blk = blockIdx.y * gridDim.x + blockIdx.x, n_blk = gridDim.x * gridDim.y;
@@ -178,6 +184,33 @@ upsample_ce_rows_kernel(UpsampleCeArgs a)
     const bool vec_ok = (w % 4 == 0) && ((uintptr_t)z % 16 == 0);
     const int xa = vec_ok ? ((x0 - 1) & ~3) : x0 - 1;      // x0-1 >= -1; (-1 & ~3) = -4
     const int off = (x0 - 1) - xa;                         // column of node x0-1 inside the tile
+    const int i = y0 - 1 + wi;                  // cell row: frame rows 4i+2 .. 4i+5, node rows (i, i+1)
+    const int n = x0 - 1 + l;                   // own node column; cell n lies between node columns n and n+1
+    const bool cell_row_valid = i <= h - 1;
+    const bool cell_valid = l <= 30 && n >= -1 && n <= w - 1;
+    const bool node_owned = l >= 1 && l <= RN_X && n < w;
+    // tile coordinates of the (clamped) nodes this lane's pixels pull toward
+    const int ry_top = min(max(i, 0), h - 1) - (y0 - 1), ry_bot = min(max(i + 1, 0), h - 1) - (y0 - 1);
+    const int rx_l = min(max(n, 0), w - 1) - xa, rx_r = min(max(n + 1, 0), w - 1) - xa;
+
+    // the block that owns node (min(i+1, h-1), min(n+1, w-1)) counts the cell's loss
+    const int t_row = min(i + 1, h - 1), t_col = min(n + 1, w - 1);
+    const bool own_cell = cell_row_valid && cell_valid && t_row >= y0 && t_row < y0 + RN_Y && t_col >= x0 && t_col < x0 + RN_X;
+    // labels of the lane's 16 pixels (rows 4i+2 .. 4i+5, columns 4n+2 .. 4n+5), two aligned 16-bit loads per row;
+    // bit 4r+k of vmask: pixel k of row r lies inside the frame
+    uint32_t labw[4], vmask = 0;
+    const int X0 = 4 * n + 2;
+    const bool v01 = cell_valid && X0 >= 0 && X0 + 1 < W, v23 = cell_valid && X0 + 2 >= 0 && X0 + 3 < W;
+#pragma unroll
+    for (int r = 0; r < 4; ++r) {
+        const int Y = 4 * i + 2 + r;
+        uint32_t lo = 0, hi = 0;
+        if (cell_row_valid && Y >= 0 && Y < H) {
+            if (v01) { lo = __ldg(reinterpret_cast<const unsigned short*>(labels + (int64_t)Y * W + X0)); vmask |= 0x3u << (4 * r); }
+            if (v23) { hi = __ldg(reinterpret_cast<const unsigned short*>(labels + (int64_t)Y * W + X0 + 2)); vmask |= 0xcu << (4 * r); }
+        }
+        labw[r] = lo | (hi << 16);
+    }
     {
         constexpr int kQuads = TZ / 4;                     // 16-byte groups per class
         constexpr int kIter = (CB * kQuads + R_THREADS - 1) / R_THREADS;
@@ -208,15 +241,6 @@ upsample_ce_rows_kernel(UpsampleCeArgs a)
     for (int e = tid; e < C * TZ / 4; e += R_THREADS) reinterpret_cast<int4*>(corr)[e] = make_int4(0, 0, 0, 0);
     __syncthreads();
 
-    const int i = y0 - 1 + wi;                  // cell row: frame rows 4i+2 .. 4i+5, node rows (i, i+1)
-    const int n = x0 - 1 + l;                   // own node column; cell n lies between node columns n and n+1
-    const bool cell_row_valid = i <= h - 1;
-    const bool cell_valid = l <= 30 && n >= -1 && n <= w - 1;
-    const bool node_owned = l >= 1 && l <= RN_X && n < w;
-    // tile coordinates of the (clamped) nodes this lane's pixels pull toward
-    const int ry_top = min(max(i, 0), h - 1) - (y0 - 1), ry_bot = min(max(i + 1, 0), h - 1) - (y0 - 1);
-    const int rx_l = min(max(n, 0), w - 1) - xa, rx_r = min(max(n + 1, 0), w - 1) - xa;
-
     RowCtx rc;
     rc.za = zt + wi * TZ_W + off + l;
     rc.ly = 0.f;
@@ -235,43 +259,25 @@ upsample_ce_rows_kernel(UpsampleCeArgs a)
     unsigned n_bad = 0;
     float* my_bot = bsh + (size_t)wi * C * 32 + l;             // this thread's slot of class c: my_bot[c * 32]
 
-    // labels of the lane's 16 pixels (rows 4i+2 .. 4i+5, columns 4n+2 .. 4n+5), two aligned 16-bit loads per row;
-    // bit 4r+k of vmask: pixel k of row r lies inside the frame
-    uint32_t labw[4], vmask = 0;
-    const int X0 = 4 * n + 2;
-    const bool v01 = cell_valid && X0 >= 0 && X0 + 1 < W, v23 = cell_valid && X0 + 2 >= 0 && X0 + 3 < W;
-#pragma unroll
-    for (int r = 0; r < 4; ++r) {
-        const int Y = 4 * i + 2 + r;
-        uint32_t lo = 0, hi = 0;
-        if (cell_row_valid && Y >= 0 && Y < H) {
-            if (v01) { lo = __ldg(reinterpret_cast<const unsigned short*>(labels + (int64_t)Y * W + X0)); vmask |= 0x3u << (4 * r); }
-            if (v23) { hi = __ldg(reinterpret_cast<const unsigned short*>(labels + (int64_t)Y * W + X0 + 2)); vmask |= 0xcu << (4 * r); }
-        }
-        labw[r] = lo | (hi << 16);
-    }
     // at the clamped left and right borders the outer node column is the inner one
     const bool fold_l = n == -1, fold_r = n == w - 1;
 
     // per pixel of one row: loss, 1/Z, the "- onehot" part of the adjoint (integer, exact), confusion; returns the
     // horizontal adjoint weights (already divided by Z) of the row's four pixels
     auto finish_row = [&](int r, const float (&Zs)[4], const float (&sk)[4], const uint32_t (&arg)[4], float (&wl)[4], float (&wr)[4]) {
-        const int Y = 4 * i + 2 + r;
         const float ly = (2 * r + 1) * 0.125f;
-        const bool row_owned = (Y >> 2) >= y0 && (Y >> 2) < y0 + RN_Y;
         const int wy1 = 2 * r + 1, wy0 = 8 - wy1;                // eighths toward node rows i+1 / i
         int lab[4];
 #pragma unroll
         for (int k = 0; k < 4; ++k) {
             lab[k] = (labw[r] >> (8 * k)) & 0xff;
-            const int gx = (X0 + k) >> 2;
             const bool valid = (vmask >> (4 * r + k)) & 1u;
-            const bool own = valid && row_owned && gx >= x0 && gx < x0 + RN_X;
+            const bool own = valid && own_cell;
             if (valid && lab[k] >= C) { if (own) n_bad++; lab[k] = -1; }
             if (!valid) lab[k] = -1;
             float rz = 0.f;
             if (lab[k] >= 0) {
-                rz = __frcp_rn(Zs[k]);
+                rz = rcp_approx(Zs[k]);
                 if (own) {
                     const float* q = rc.za + lab[k] * TZ;
                     const float vl = fmaf(ly, q[TZ_W] - q[0], q[0]), vr = fmaf(ly, q[TZ_W + 1] - q[1], q[1]);
@@ -325,19 +331,57 @@ upsample_ce_rows_kernel(UpsampleCeArgs a)
         if (!slow) {
             float wl[16], wr[16];
             const float zero4[4] = {0.f, 0.f, 0.f, 0.f};
+            uint32_t arg[CONF ? 16 : 1] = {};
+            if (CONF) {                                              // the student's class: arg-max of the interpolated logits
 #pragma unroll
-            for (int r = 0; r < 4; ++r) {
-                const float Zr[4] = {Z[4 * r], Z[4 * r + 1], Z[4 * r + 2], Z[4 * r + 3]};
-                uint32_t ar4[4] = {0, 0, 0, 0};
-                if (CONF) {                                          // the student's class: arg-max of the interpolated logits
+                for (int r = 0; r < 4; ++r) {
                     float Zd[4];
+                    uint32_t ar4[4] = {0, 0, 0, 0};
                     rc.ly = (2 * r + 1) * 0.125f;
                     pass1<CB, true, false>(rc, zero4, Zd, ar4);
-                }
-                float wl4[4], wr4[4];
-                finish_row(r, Zr, zero4, ar4, wl4, wr4);
 #pragma unroll
-                for (int k = 0; k < 4; ++k) { wl[4 * r + k] = wl4[k]; wr[4 * r + k] = wr4[k]; }
+                    for (int k = 0; k < 4; ++k) arg[CONF ? 4 * r + k : 0] = ar4[k];
+                }
+            }
+            const uint32_t l0 = labw[0] & 0xffu;
+            const bool uniform = vmask == 0xffffu && labw[0] == l0 * 0x01010101u && labw[1] == labw[0] && labw[2] == labw[0] &&
+                                 labw[3] == labw[0] && (int)l0 < C;
+            if (uniform) {
+                // an interior cell whose 16 pixels carry one label (the usual case): the onehot parts add up to
+                // 256/64 per corner, and the label's logits add up to 16 x their value at the cell centre
+                int* cc = corr + l0 * TZ;
+                atomicAdd(cc + ry_top * TZ_W + rx_l, -256);
+                atomicAdd(cc + ry_top * TZ_W + rx_r, -256);
+                atomicAdd(cc + ry_bot * TZ_W + rx_l, -256);
+                atomicAdd(cc + ry_bot * TZ_W + rx_r, -256);
+                float lz = 0.f;
+#pragma unroll
+                for (int j = 0; j < 16; ++j) {
+                    const float rz = rcp_approx(Z[j]), fr = (2 * (j & 3) + 1) * 0.125f;
+                    lz += __log2f(Z[j]);
+                    wl[j] = (1.0f - fr) * rz;
+                    wr[j] = fr * rz;
+                }
+                if (own_cell) {
+                    const float* q = rc.za + l0 * TZ;
+                    const float sum4 = (q[0] + q[1]) + (q[TZ_W] + q[TZ_W + 1]);
+                    loss += (lz - (4.0f * sum4 - 16.0f * rc.M)) * kLn2;
+                    if (CONF) {
+#pragma unroll
+                        for (int j = 0; j < 16; ++j)
+                            atomicAdd(a.conf + (int64_t)s * a.conf_stream_stride + l0 * C + arg[CONF ? j : 0], 1ull);
+                    }
+                }
+            } else {
+#pragma unroll
+                for (int r = 0; r < 4; ++r) {
+                    const float Zr[4] = {Z[4 * r], Z[4 * r + 1], Z[4 * r + 2], Z[4 * r + 3]};
+                    const uint32_t ar4[4] = {arg[CONF ? 4 * r : 0], arg[CONF ? 4 * r + 1 : 0], arg[CONF ? 4 * r + 2 : 0], arg[CONF ? 4 * r + 3 : 0]};
+                    float wl4[4], wr4[4];
+                    finish_row(r, Zr, zero4, ar4, wl4, wr4);
+#pragma unroll
+                    for (int k = 0; k < 4; ++k) { wl[4 * r + k] = wl4[k]; wr[4 * r + k] = wr4[k]; }
+                }
             }
             // vertical weights of the rows toward the upper / lower node row (clamped borders fold into the inner row)
             float tw[4], bw[4];
@@ -404,7 +448,7 @@ upsample_ce_rows_kernel(UpsampleCeArgs a)
     const float invP = 1.0f / ((float)H * (float)W);
     const int y = i;
     const bool node_ok = wi >= 1 && y < h && node_owned;
-    float dbsum = 0.f;       // lane c ends up with the class-c sum over this warp's nodes
+    float* vs = zt;          // [C][R_THREADS] this block's gradient values, for the bias-gradient partial (the tile is no longer read)
 #pragma unroll
     for (int c = 0; c < CB; ++c) {
         if (c < C) {
@@ -416,17 +460,22 @@ upsample_ce_rows_kernel(UpsampleCeArgs a)
                 if (a.dz_bf16)
                     a.dz_bf16[((int64_t)s * kClassPad + c) * a.dz_bf16_pitch + (int64_t)y * w + n] = __float2bfloat16_rn(v);
             }
-#pragma unroll
-            for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
-            if (l == c) dbsum = v;
+            vs[c * R_THREADS + tid] = v;
         }
     }
-    dbs[wi][l] = dbsum;
     __syncthreads();
-    for (int c = tid; c < C; c += R_THREADS) {
+    {
+        // eight threads per class, 32 values each (rotated start: conflict-free), then a three-step tree: fixed order
+        const int c = tid >> 3, sub = tid & 7;
         float t = 0.f;
-        for (int k = 1; k < R_WARPS; ++k) t += dbs[k][c];
-        a.db_part[((int64_t)s * n_blk + blk) * C + c] = t;
+        if (c < C) {
+#pragma unroll 8
+            for (int j = 0; j < 32; ++j) t += vs[c * R_THREADS + sub * 32 + ((j + l) & 31)];
+        }
+        t += __shfl_xor_sync(0xffffffffu, t, 1);
+        t += __shfl_xor_sync(0xffffffffu, t, 2);
+        t += __shfl_xor_sync(0xffffffffu, t, 4);
+        if (c < C && sub == 0) a.db_part[((int64_t)s * n_blk + blk) * C + c] = t;
     }
     if (tid == 0) {
         float t = 0.f;
