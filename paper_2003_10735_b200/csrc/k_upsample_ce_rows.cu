@@ -54,6 +54,14 @@ __device__ __forceinline__ float rcp_approx(float x)
     return y;
 }
 
+// Byte k: (row eighths) x (column eighths of pixel k toward the left node column: 7, 5, 3, 1; toward the right one:
+// 1, 3, 5, 7) -- the integer adjoint weights (units of 1/64) of a row's four pixels for one corner node.
+__host__ __device__ constexpr uint32_t corner_weights(int row_eighths, bool right)
+{
+    return right ? (uint32_t)(row_eighths * 1) | (uint32_t)(row_eighths * 3) << 8 | (uint32_t)(row_eighths * 5) << 16 | (uint32_t)(row_eighths * 7) << 24
+                 : (uint32_t)(row_eighths * 7) | (uint32_t)(row_eighths * 5) << 8 | (uint32_t)(row_eighths * 3) << 16 | (uint32_t)(row_eighths * 1) << 24;
+}
+
 struct RowCtx {
     const float* za;     // own column, upper node row, class 0
     float ly;            // weight toward the lower node row
@@ -198,7 +206,7 @@ upsample_ce_rows_kernel(UpsampleCeArgs a)
     const bool own_cell = cell_row_valid && cell_valid && t_row >= y0 && t_row < y0 + RN_Y && t_col >= x0 && t_col < x0 + RN_X;
     // labels of the lane's 16 pixels (rows 4i+2 .. 4i+5, columns 4n+2 .. 4n+5), two aligned 16-bit loads per row;
     // bit 4r+k of vmask: pixel k of row r lies inside the frame
-    uint32_t labw[4], vmask = 0;
+    uint32_t labw[4], vb[4], vmask = 0;      // vb: 0x01 in the byte of each pixel inside the frame
     const int X0 = 4 * n + 2;
     const bool v01 = cell_valid && X0 >= 0 && X0 + 1 < W, v23 = cell_valid && X0 + 2 >= 0 && X0 + 3 < W;
 #pragma unroll
@@ -210,6 +218,7 @@ upsample_ce_rows_kernel(UpsampleCeArgs a)
             if (v23) { hi = __ldg(reinterpret_cast<const unsigned short*>(labels + (int64_t)Y * W + X0 + 2)); vmask |= 0xcu << (4 * r); }
         }
         labw[r] = lo | (hi << 16);
+        vb[r] = (((vmask >> (4 * r)) & 0x3u) ? 0x00000101u : 0u) | (((vmask >> (4 * r)) & 0xcu) ? 0x01010000u : 0u);
     }
     {
         constexpr int kQuads = TZ / 4;                     // 16-byte groups per class
@@ -331,7 +340,16 @@ upsample_ce_rows_kernel(UpsampleCeArgs a)
         if (!slow) {
             float wl[16], wr[16];
             const float zero4[4] = {0.f, 0.f, 0.f, 0.f};
-            uint32_t arg[CONF ? 16 : 1] = {};
+            // pixels that count: inside the frame, label below n_classes
+            uint32_t rem[4];
+            const uint32_t C4 = (uint32_t)C * 0x01010101u;
+            int n_ok = 0;
+#pragma unroll
+            for (int r = 0; r < 4; ++r) {
+                rem[r] = __vcmpltu4(labw[r], C4) & vb[r];
+                n_ok += __popc(rem[r]);
+                if (own_cell) n_bad += __popc(rem[r] ^ vb[r]);
+            }
             if (CONF) {                                              // the student's class: arg-max of the interpolated logits
 #pragma unroll
                 for (int r = 0; r < 4; ++r) {
@@ -340,49 +358,53 @@ upsample_ce_rows_kernel(UpsampleCeArgs a)
                     rc.ly = (2 * r + 1) * 0.125f;
                     pass1<CB, true, false>(rc, zero4, Zd, ar4);
 #pragma unroll
-                    for (int k = 0; k < 4; ++k) arg[CONF ? 4 * r + k : 0] = ar4[k];
+                    for (int k = 0; k < 4; ++k)
+                        if (own_cell && ((rem[r] >> (8 * k)) & 1u))
+                            atomicAdd(a.conf + (int64_t)s * a.conf_stream_stride + ((labw[r] >> (8 * k)) & 0xffu) * C + ar4[k], 1ull);
                 }
             }
-            const uint32_t l0 = labw[0] & 0xffu;
-            const bool uniform = vmask == 0xffffu && labw[0] == l0 * 0x01010101u && labw[1] == labw[0] && labw[2] == labw[0] &&
-                                 labw[3] == labw[0] && (int)l0 < C;
-            if (uniform) {
-                // an interior cell whose 16 pixels carry one label (the usual case): the onehot parts add up to
-                // 256/64 per corner, and the label's logits add up to 16 x their value at the cell centre
-                int* cc = corr + l0 * TZ;
-                atomicAdd(cc + ry_top * TZ_W + rx_l, -256);
-                atomicAdd(cc + ry_top * TZ_W + rx_r, -256);
-                atomicAdd(cc + ry_bot * TZ_W + rx_l, -256);
-                atomicAdd(cc + ry_bot * TZ_W + rx_r, -256);
-                float lz = 0.f;
+            float lz = 0.f;
 #pragma unroll
-                for (int j = 0; j < 16; ++j) {
-                    const float rz = rcp_approx(Z[j]), fr = (2 * (j & 3) + 1) * 0.125f;
-                    lz += __log2f(Z[j]);
-                    wl[j] = (1.0f - fr) * rz;
-                    wr[j] = fr * rz;
-                }
-                if (own_cell) {
-                    const float* q = rc.za + l0 * TZ;
-                    const float sum4 = (q[0] + q[1]) + (q[TZ_W] + q[TZ_W + 1]);
-                    loss += (lz - (4.0f * sum4 - 16.0f * rc.M)) * kLn2;
-                    if (CONF) {
-#pragma unroll
-                        for (int j = 0; j < 16; ++j)
-                            atomicAdd(a.conf + (int64_t)s * a.conf_stream_stride + l0 * C + arg[CONF ? j : 0], 1ull);
-                    }
-                }
-            } else {
+            for (int j = 0; j < 16; ++j) {
+                const bool ok = (rem[j >> 2] >> (8 * (j & 3))) & 1u;
+                const float fr = (2 * (j & 3) + 1) * 0.125f;
+                const float rz = ok ? rcp_approx(Z[j]) : 0.f;
+                lz += ok ? __log2f(Z[j]) : 0.f;
+                wl[j] = (fold_l ? 0.f : (fold_r ? 1.0f : 1.0f - fr)) * rz;
+                wr[j] = (fold_r ? 0.f : (fold_l ? 1.0f : fr)) * rz;
+            }
+            // One round per distinct label of the cell (one round for most cells).  The pixels carrying the label pull
+            // the four corner nodes with integer weights (row eighths x column eighths, summed by byte-wise dot products);
+            // the same four sums weight the label's corner logits in the loss.
+            int* c_tl = corr + ry_top * TZ_W + rx_l;
+            const int d_tr = rx_r - rx_l, d_bl = (ry_bot - ry_top) * TZ_W;
+            float lsum = 0.f;
+            while (rem[0] | rem[1] | rem[2] | rem[3]) {
+                const uint32_t wsel = rem[0] ? labw[0] : rem[1] ? labw[1] : rem[2] ? labw[2] : labw[3];
+                const uint32_t rsel = rem[0] ? rem[0] : rem[1] ? rem[1] : rem[2] ? rem[2] : rem[3];
+                const uint32_t cur = (wsel >> (__ffs(rsel) - 1)) & 0xffu;
+                const uint32_t cur4 = cur * 0x01010101u;
+                uint32_t tl = 0, tr = 0, bl = 0, br = 0;
 #pragma unroll
                 for (int r = 0; r < 4; ++r) {
-                    const float Zr[4] = {Z[4 * r], Z[4 * r + 1], Z[4 * r + 2], Z[4 * r + 3]};
-                    const uint32_t ar4[4] = {arg[CONF ? 4 * r : 0], arg[CONF ? 4 * r + 1 : 0], arg[CONF ? 4 * r + 2 : 0], arg[CONF ? 4 * r + 3 : 0]};
-                    float wl4[4], wr4[4];
-                    finish_row(r, Zr, zero4, ar4, wl4, wr4);
-#pragma unroll
-                    for (int k = 0; k < 4; ++k) { wl[4 * r + k] = wl4[k]; wr[4 * r + k] = wr4[k]; }
+                    const uint32_t eq = __vcmpeq4(labw[r], cur4) & rem[r];
+                    rem[r] ^= eq;
+                    tl = __dp4a(eq, corner_weights(7 - 2 * r, false), tl);
+                    tr = __dp4a(eq, corner_weights(7 - 2 * r, true), tr);
+                    bl = __dp4a(eq, corner_weights(2 * r + 1, false), bl);
+                    br = __dp4a(eq, corner_weights(2 * r + 1, true), br);
+                }
+                int* cc = c_tl + cur * TZ;
+                atomicAdd(cc, -(int)tl);
+                atomicAdd(cc + d_tr, -(int)tr);
+                atomicAdd(cc + d_bl, -(int)bl);
+                atomicAdd(cc + d_bl + d_tr, -(int)br);
+                if (own_cell) {
+                    const float* q = zt + (c_tl - corr) + cur * TZ;
+                    lsum = fmaf((float)tl, q[0], fmaf((float)tr, q[d_tr], fmaf((float)bl, q[d_bl], fmaf((float)br, q[d_bl + d_tr], lsum))));
                 }
             }
+            if (own_cell) loss += (lz - (lsum * (1.0f / 64.0f) - (float)n_ok * rc.M)) * kLn2;
             // vertical weights of the rows toward the upper / lower node row (clamped borders fold into the inner row)
             float tw[4], bw[4];
 #pragma unroll
