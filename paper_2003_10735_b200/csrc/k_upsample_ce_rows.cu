@@ -20,12 +20,12 @@
 // warp walks its four frame rows one by one with exact per-pixel maxima:
 //   pass 1  each lane interpolates its own node column vertically, takes the right neighbour's by
 //           shuffle, interpolates its four pixels horizontally, and sums exp2(u - M) over the classes
-//           (logits are pre-scaled by log2 e; M is the largest logit of the warp's two node rows);
+//           (logits are pre-scaled by log2 e; M is the largest logit of the block's tile);
 //   pass 2  the exponentials are formed again (cheaper than keeping 4 x C registers alive: two
 //           or three blocks per SM stay resident), multiplied by the adjoint interpolation weights / Z, the
 //           right-hand part is handed to the next lane by shuffle, and the row is added into two
 //           per-class accumulators: toward the upper and the lower node row.
-// If a pixel's sum underflows (logits varying by more than ~100 inside the warp's span) the warp
+// If a pixel's sum underflows (logits varying by more than ~100 inside the block's tile) the warp
 // redoes that row with the exact per-pixel maximum.
 // The "- onehot(label)" part of the gradient is exact in units of 1/64, so it is accumulated with
 // integer shared-memory atomics (order-independent).
@@ -175,7 +175,7 @@ upsample_ce_rows_kernel(UpsampleCeArgs a)
                                                 //                  hold -1e30 (their exponentials are 0)
     int* corr = (int*)(zt + CB * TZ);           // [C][TZ_H][36]    -64 * (adjoint of onehot)
     float* bsh = (float*)(corr + C * TZ);       // [R_WARPS][C][32] lower-row accumulators
-    __shared__ float red[R_WARPS];
+    __shared__ float red[R_WARPS], red_m[R_WARPS];
 
     const int s = blockIdx.z, x0 = blockIdx.x * RN_X, y0 = blockIdx.y * RN_Y;
     const int blk = blockIdx.y * gridDim.x + blockIdx.x, n_blk = gridDim.x * gridDim.y;
@@ -220,44 +220,53 @@ upsample_ce_rows_kernel(UpsampleCeArgs a)
         labw[r] = lo | (hi << 16);
         vb[r] = (((vmask >> (4 * r)) & 0x3u) ? 0x00000101u : 0u) | (((vmask >> (4 * r)) & 0xcu) ? 0x01010000u : 0u);
     }
+    float m_loc = -INFINITY;                               // largest logit this thread fetched
     {
-        constexpr int kQuads = TZ / 4;                     // 16-byte groups per class
-        constexpr int kIter = (CB * kQuads + R_THREADS - 1) / R_THREADS;
+        // a thread keeps one 16-byte group of the tile plane (81 groups) and walks the classes three at a time;
+        // fully unrolled: all of a thread's loads are in flight together
+        constexpr int kQuads = TZ / 4, kPlanes = R_THREADS / kQuads;       // 81, 3
+        constexpr int kIter = (CB + kPlanes - 1) / kPlanes;
+        const int g = tid / kQuads, q = tid % kQuads;
+        const int yy = min(max(y0 - 1 + q / (TZ_W / 4), 0), h - 1), xq = xa + 4 * (q % (TZ_W / 4));
+        const bool vec = vec_ok && xq >= 0 && xq + 3 < w;
+        const float* row = z + (int64_t)yy * w;
+        const int x_0 = min(max(xq, 0), w - 1), x_1 = min(max(xq + 1, 0), w - 1), x_2 = min(max(xq + 2, 0), w - 1),
+                  x_3 = min(max(xq + 3, 0), w - 1);
         float4 v[kIter];
 #pragma unroll
         for (int it = 0; it < kIter; ++it) {
-            const int e = tid + it * R_THREADS;
-            const int c = e / kQuads, q = e % kQuads;
-            const int yy = min(max(y0 - 1 + q / (TZ_W / 4), 0), h - 1), xq = xa + 4 * (q % (TZ_W / 4));
+            const int c = g + it * kPlanes;
             float4 t = make_float4(-1e30f, -1e30f, -1e30f, -1e30f);
-            if (e < CB * kQuads && c < C) {
-                const float* row = z + (int64_t)c * p + (int64_t)yy * w;
-                if (vec_ok && xq >= 0 && xq + 3 < w) t = __ldg(reinterpret_cast<const float4*>(row + xq));
-                else {
-                    t.x = __ldg(row + min(max(xq, 0), w - 1));     t.y = __ldg(row + min(max(xq + 1, 0), w - 1));
-                    t.z = __ldg(row + min(max(xq + 2, 0), w - 1)); t.w = __ldg(row + min(max(xq + 3, 0), w - 1));
-                }
+            if (g < kPlanes && c < C) {
+                const float* rp = row + (int64_t)c * p;
+                if (vec) t = __ldg(reinterpret_cast<const float4*>(rp + xq));
+                else { t.x = __ldg(rp + x_0); t.y = __ldg(rp + x_1); t.z = __ldg(rp + x_2); t.w = __ldg(rp + x_3); }
                 t.x *= kLog2e; t.y *= kLog2e; t.z *= kLog2e; t.w *= kLog2e;
+                m_loc = fmaxf(fmaxf(m_loc, fmaxf(t.x, t.y)), fmaxf(t.z, t.w));
             }
             v[it] = t;
         }
 #pragma unroll
         for (int it = 0; it < kIter; ++it) {
-            const int e = tid + it * R_THREADS;
-            if (e < CB * kQuads) reinterpret_cast<float4*>(zt)[e] = v[it];
+            const int c = g + it * kPlanes;
+            if (g < kPlanes && c < CB) reinterpret_cast<float4*>(zt)[c * kQuads + q] = v[it];
         }
     }
     for (int e = tid; e < C * TZ / 4; e += R_THREADS) reinterpret_cast<int4*>(corr)[e] = make_int4(0, 0, 0, 0);
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) m_loc = fmaxf(m_loc, __shfl_xor_sync(0xffffffffu, m_loc, o));
+    if (l == 0) red_m[wi] = m_loc;
     __syncthreads();
 
     RowCtx rc;
     rc.za = zt + wi * TZ_W + off + l;
     rc.ly = 0.f;
     {
-        float m = -INFINITY;
-        for (int c = 0; c < C; ++c) m = fmaxf(m, fmaxf(rc.za[c * TZ], rc.za[c * TZ + TZ_W]));
+        // shift of the exponentials: the largest logit of the block's tile (a pixel whose own logits lie far below it
+        // is caught by the underflow check and redone with its exact maximum)
+        float m = red_m[0];
 #pragma unroll
-        for (int o = 16; o > 0; o >>= 1) m = fmaxf(m, __shfl_xor_sync(0xffffffffu, m, o));
+        for (int k = 1; k < R_WARPS; ++k) m = fmaxf(m, red_m[k]);
         rc.M = m;
     }
 
