@@ -269,81 +269,4 @@ void launch_upsample_ce(const UpsampleCeArgs& a, cudaStream_t s)
     else launch_chain(upsample_ce_kernel<false>, grid, dim3(kThreads), smem, s, a, chunk);
 }
 
-// ------------------------------------------------------------------------------------------------
-// Student mask: arg-max over classes of the upsampled logits (lowest class on ties), uint8 [H][W].
-// A block covers 8 x 32 feature-map nodes (32 x 128 frame pixels) with the logits of the 10 x 34
-// surrounding nodes in shared memory; a thread handles the 4 x 4 frame pixels around one node.
-// ------------------------------------------------------------------------------------------------
-constexpr int AM_Y = 8, AM_X = 32, AM_TH = AM_Y + 2, AM_TW = AM_X + 2;
-
-__global__ void __launch_bounds__(256)
-upsample_argmax_kernel(const float* __restrict__ z, int C, int chunk, int h, int w, uint8_t* __restrict__ mask)
-{
-    extern __shared__ float zs[];                       // [chunk][AM_TH][AM_TW], borders replicated
-    const int x0 = blockIdx.x * AM_X, y0 = blockIdx.y * AM_Y;
-    const int64_t p = (int64_t)h * w;
-    const int W = w * kUp;
-    const int tx = threadIdx.x % AM_X, ty = threadIdx.x / AM_X;
-    const int x = x0 + tx, y = y0 + ty;
-    const bool active = x < w && y < h;
-    float best[16];
-    uint32_t arg[16];
-#pragma unroll
-    for (int k = 0; k < 16; ++k) { best[k] = -INFINITY; arg[k] = 0; }
-    const float* q0 = zs + ty * AM_TW + tx;             // node (y-1, x-1)
-    for (int c0 = 0; c0 < C; c0 += chunk) {             // classes in chunks that fit shared memory
-    const int nc = min(chunk, C - c0);
-    __syncthreads();
-    for (int e = threadIdx.x; e < nc * AM_TH * AM_TW; e += 256) {
-        const int c = e / (AM_TH * AM_TW), n = e % (AM_TH * AM_TW);
-        const int yy = min(max(y0 - 1 + n / AM_TW, 0), h - 1), xx = min(max(x0 - 1 + n % AM_TW, 0), w - 1);
-        zs[e] = __ldg(z + (int64_t)(c0 + c) * p + (int64_t)yy * w + xx);
-    }
-    __syncthreads();
-    if (active)
-    for (int cc = 0; cc < nc; ++cc) {
-        const int c = c0 + cc;
-        const float* q = q0 + cc * (AM_TH * AM_TW);
-        float n[3][3];
-#pragma unroll
-        for (int a = 0; a < 3; ++a)
-#pragma unroll
-            for (int b = 0; b < 3; ++b) n[a][b] = q[a * AM_TW + b];
-        // frame row 4y+r: rows (y-1, y) with weight 5/8, 7/8 toward y for r = 0, 1; rows (y, y+1) with 1/8, 3/8 for r = 2, 3
-#pragma unroll
-        for (int r = 0; r < 4; ++r) {
-            const int ra = r < 2 ? 0 : 1;
-            const float ly = r == 0 ? 0.625f : r == 1 ? 0.875f : r == 2 ? 0.125f : 0.375f;
-            // horizontal first, then vertical
-            const float tl0 = lerp_f(n[ra][0], n[ra][1], 0.625f), bl0 = lerp_f(n[ra + 1][0], n[ra + 1][1], 0.625f);
-            const float tl1 = lerp_f(n[ra][0], n[ra][1], 0.875f), bl1 = lerp_f(n[ra + 1][0], n[ra + 1][1], 0.875f);
-            const float tr0 = lerp_f(n[ra][1], n[ra][2], 0.125f), br0 = lerp_f(n[ra + 1][1], n[ra + 1][2], 0.125f);
-            const float tr1 = lerp_f(n[ra][1], n[ra][2], 0.375f), br1 = lerp_f(n[ra + 1][1], n[ra + 1][2], 0.375f);
-            const float u[4] = {lerp_f(tl0, bl0, ly), lerp_f(tl1, bl1, ly), lerp_f(tr0, br0, ly), lerp_f(tr1, br1, ly)};
-#pragma unroll
-            for (int k = 0; k < 4; ++k)
-                if (u[k] > best[r * 4 + k]) { best[r * 4 + k] = u[k]; arg[r * 4 + k] = c; }
-        }
-    }
-    }
-    if (!active) return;
-#pragma unroll
-    for (int r = 0; r < 4; ++r)
-        reinterpret_cast<uint32_t*>(mask + (int64_t)(4 * y + r) * W)[x] =
-            arg[r * 4] | (arg[r * 4 + 1] << 8) | (arg[r * 4 + 2] << 16) | (arg[r * 4 + 3] << 24);
-}
-
-void launch_upsample_argmax(const float* z, int C, int h, int w, uint8_t* mask, cudaStream_t s)
-{
-    const int chunk = C < 128 ? C : 128;
-    const size_t smem = (size_t)chunk * AM_TH * AM_TW * sizeof(float);
-    static size_t configured = 0;
-    if (smem > 48 * 1024 && smem > configured) {
-        cudaFuncSetAttribute(upsample_argmax_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
-        configured = smem;
-    }
-    dim3 grid((unsigned)((w + AM_X - 1) / AM_X), (unsigned)((h + AM_Y - 1) / AM_Y));
-    upsample_argmax_kernel<<<grid, 256, smem, s>>>(z, C, chunk, h, w, mask);
-}
-
 }  // namespace st

@@ -388,7 +388,7 @@ st_status st_init_head(const st_head_desc* desc, const float* init_params, st_ct
     ALLOC(z, S * c->C * c->p); ALLOC(dz, S * c->C * c->p);
     ALLOC(loss_part, S * c->n_k3_blocks); ALLOC(db_part, (size_t)S * c->n_k3_blocks * c->C);
     ALLOC(loss_buf, S * kMaxSteps);
-    ALLOC(miou_tmp, 4); ALLOC(mask_tmp, c->P); ALLOC(mask_tmp2, c->P); ALLOC(conf_tmp, c->C * c->C);
+    ALLOC(miou_tmp, 4); ALLOC(mask_tmp, c->P); ALLOC(mask_tmp2, c->P); ALLOC(conf_tmp, c->C * c->C + 1);   // + the block counter of the fused agreement kernel
     if (e == cudaSuccess) { c->bad = reinterpret_cast<unsigned int*>(c->miou_tmp + 1); e = cudaHostAlloc((void**)&c->status_host, 32, cudaHostAllocDefault); }
     if (c->bf16_mode) {
         ALLOC(x_bf16, S * c->p * c->Cin);
@@ -412,6 +412,7 @@ st_status st_init_head(const st_head_desc* desc, const float* init_params, st_ct
     }
 #undef ALLOC
     if (e == cudaSuccess) e = prepare_upsample_ce(c->C);
+    if (e == cudaSuccess) e = prepare_student_mask(c->C);
     if (e != cudaSuccess) {
         st_status code = fail(nullptr, e == cudaErrorMemoryAllocation ? ST_ERR_OOM : ST_ERR_CUDA,
                               "st_init_head: device allocation failed: %s", cudaGetErrorString(e));
@@ -620,19 +621,36 @@ st_status st_pack_updated_params(st_ctx* ctx, int32_t stream, void* dst, size_t 
     return ST_OK;
 }
 
+namespace {
+// forward of all streams with the current parameters, then the mask kernel on `stream`
+st_status student_forward(st_ctx* ctx, int32_t stream, const char* who)
+{
+    if (!ctx->has_feat[stream]) return fail(ctx, ST_ERR_BAD_STATE, "%s: stream %d has no frozen features yet", who, stream);
+    for (int s = 0; s < ctx->S; ++s)
+        if (!ctx->has_feat[s]) return fail(ctx, ST_ERR_BAD_STATE, "%s: the forward runs on all streams; stream %d has no features", who, s);
+    return enqueue_forward(ctx);
+}
+
+StudentMaskArgs mask_args(st_ctx* ctx, int32_t stream, uint8_t* mask)
+{
+    StudentMaskArgs a{};
+    a.z = ctx->z + (int64_t)stream * ctx->C * ctx->p;
+    a.C = ctx->C; a.h = ctx->h; a.w = ctx->w;
+    a.mask = mask;
+    return a;
+}
+}  // namespace
+
 st_status st_student_mask(st_ctx* ctx, int32_t stream, uint8_t* mask_out)
 {
     st_status st = check_stream_index(ctx, stream);
     if (st != ST_OK) return st;
     if (!mask_out) return fail(ctx, ST_ERR_INVALID_ARG, "st_student_mask: NULL destination");
-    if (!ctx->has_feat[stream]) return fail(ctx, ST_ERR_BAD_STATE, "st_student_mask: stream %d has no frozen features yet", stream);
-    for (int s = 0; s < ctx->S; ++s)
-        if (!ctx->has_feat[s]) return fail(ctx, ST_ERR_BAD_STATE, "st_student_mask: the forward runs on all streams; stream %d has no features", s);
-    st = enqueue_forward(ctx);
+    st = student_forward(ctx, stream, "st_student_mask");
     if (st != ST_OK) return st;
     const bool dev = is_device_ptr(mask_out);
     uint8_t* dst = dev ? mask_out : ctx->mask_tmp;
-    launch_upsample_argmax(ctx->z + (int64_t)stream * ctx->C * ctx->p, ctx->C, ctx->h, ctx->w, dst, ctx->stream);
+    launch_student_mask(mask_args(ctx, stream, dst), ctx->stream);
     ctx->launches += 1;
     st = check_launch(ctx, "student mask");
     if (st != ST_OK) return st;
@@ -659,22 +677,34 @@ st_status st_agreement(st_ctx* ctx, int32_t stream, const uint8_t* pred, const u
         if (!ctx->has_labels[stream]) return fail(ctx, ST_ERR_BAD_STATE, "st_agreement: stream %d has no labels yet", stream);
         d_label = ctx->labels + (int64_t)stream * ctx->P;
     }
-    if (pred) {
-        if (is_device_ptr(pred)) d_pred = pred;
-        else {
-            ST_CUDA(ctx, cudaMemcpyAsync(ctx->mask_tmp, pred, (size_t)ctx->P, cudaMemcpyHostToDevice, ctx->stream));
+    const size_t cbytes = (size_t)ctx->C * ctx->C * sizeof(unsigned long long);
+    if (!pred && student_mask_fused_supported(ctx->C)) {
+        // the student's own mask: arg-max, confusion and mean IoU in one kernel, the mask itself is not stored
+        st = student_forward(ctx, stream, "st_agreement");
+        if (st != ST_OK) return st;
+        ST_CUDA(ctx, cudaMemsetAsync(ctx->conf_tmp, 0, cbytes, ctx->stream));
+        StudentMaskArgs a = mask_args(ctx, stream, nullptr);
+        a.labels = d_label; a.conf = ctx->conf_tmp; a.bad = ctx->bad + 1; a.miou = ctx->miou_tmp;
+        a.ticket = reinterpret_cast<unsigned int*>(ctx->conf_tmp + (size_t)ctx->C * ctx->C);
+        launch_student_mask(a, ctx->stream);
+        ctx->launches += 1;
+    } else {
+        if (pred) {
+            if (is_device_ptr(pred)) d_pred = pred;
+            else {
+                ST_CUDA(ctx, cudaMemcpyAsync(ctx->mask_tmp, pred, (size_t)ctx->P, cudaMemcpyHostToDevice, ctx->stream));
+                d_pred = ctx->mask_tmp;
+            }
+        } else {
+            st = st_student_mask(ctx, stream, ctx->mask_tmp);
+            if (st != ST_OK) return st;
             d_pred = ctx->mask_tmp;
         }
-    } else {
-        st = st_student_mask(ctx, stream, ctx->mask_tmp);
-        if (st != ST_OK) return st;
-        d_pred = ctx->mask_tmp;
+        ST_CUDA(ctx, cudaMemsetAsync(ctx->conf_tmp, 0, cbytes, ctx->stream));
+        launch_confusion(d_label, d_pred, ctx->P, ctx->C, ctx->conf_tmp, ctx->bad + 1, ctx->stream);
+        launch_miou(ctx->conf_tmp, ctx->C, ctx->miou_tmp, ctx->stream);
+        ctx->launches += 2;
     }
-    const size_t cbytes = (size_t)ctx->C * ctx->C * sizeof(unsigned long long);
-    ST_CUDA(ctx, cudaMemsetAsync(ctx->conf_tmp, 0, cbytes, ctx->stream));
-    launch_confusion(d_label, d_pred, ctx->P, ctx->C, ctx->conf_tmp, ctx->bad + 1, ctx->stream);
-    launch_miou(ctx->conf_tmp, ctx->C, ctx->miou_tmp, ctx->stream);
-    ctx->launches += 2;
     st = check_launch(ctx, "confusion");
     if (st != ST_OK) return st;
     if (conf) ST_CUDA(ctx, cudaMemcpyAsync(conf, ctx->conf_tmp, cbytes, cudaMemcpyDefault, ctx->stream));

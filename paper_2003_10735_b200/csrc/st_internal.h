@@ -76,8 +76,21 @@ bool upsample_ce_rows_supported(int C);
 int upsample_ce_rows_blocks(int h, int w);
 cudaError_t prepare_upsample_ce_rows(int C);
 void launch_upsample_ce_rows(const UpsampleCeArgs& a, cudaStream_t s);
-// student mask: argmax_c of the upsampled logits, uint8 [H][W]
-void launch_upsample_argmax(const float* z, int C, int h, int w, uint8_t* mask, cudaStream_t s);
+// student mask: argmax_c of the upsampled logits, uint8 [H][W]; with `labels` also the confusion matrix of
+// (label, mask) added into `conf`, and with `miou` the mean IoU written by the last block (k_student_mask.cu)
+struct StudentMaskArgs {
+    const float* z;            // [C][h][w] logits of one stream
+    int C, h, w;
+    uint8_t* mask;             // [H][W] or nullptr (confusion only)
+    const uint8_t* labels;     // [H][W] or nullptr (mask only)
+    unsigned long long* conf;  // [C][C], zeroed by the caller
+    unsigned int* bad;         // count of labels >= C
+    double* miou;              // nullptr: no mean IoU
+    unsigned int* ticket;      // zero between launches (block counter for the mean IoU)
+};
+bool student_mask_fused_supported(int C);   // confusion counters fit shared memory
+cudaError_t prepare_student_mask(int C);    // once per device and class count, outside any stream capture
+void launch_student_mask(const StudentMaskArgs& a, cudaStream_t s);
 
 // ---- fp32 CUDA-core convolutions (gemm_precision 0), planar [C][h][w] -------------------------
 void launch_conv_fwd_f32(const float* in, int Cin, int h, int w, const float* Wt, const float* b,
