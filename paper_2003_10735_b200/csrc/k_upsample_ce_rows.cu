@@ -120,10 +120,11 @@ __device__ __forceinline__ void pass2(const RowCtx& rc, const float (&sk)[4], co
 // The 16 exponentials exp2(u(r,k) - M) of one class inside the lane's cell, u bilinear between the four
 // corner logits (own column: rows i, i+1 from shared memory; right column from the next lane).
 // With ly_r = (2r+1)/8 and fr_k = (2k+1)/8:  u(r,k) = A + B k + G r + D k r, so the values are geometric
-// progressions along k and r: 4 exp2 and 18 multiplications.  Returns the largest corner difference
+// progressions along k and r: 4 exp2 and 12 multiplications (8 of them packed: X01[k] = (E(0,k), E(1,k)),
+// X23[k] = (E(2,k), E(3,k))).  Returns the largest corner difference
 // (the caller leaves the fast path if a class changes by more than 16 across the cell: the progressions
 // would lose their small terms).
-__device__ __forceinline__ float cell_exponentials(const float* q, float M, float (&E)[16])
+__device__ __forceinline__ float cell_exponentials(const float* q, float M, float2 (&X01)[4], float2 (&X23)[4])
 {
     const float a = q[0] - M, b = q[TZ_W] - M;
     const float ar = __shfl_down_sync(0xffffffffu, a, 1), br = __shfl_down_sync(0xffffffffu, b, 1);
@@ -133,15 +134,16 @@ __device__ __forceinline__ float cell_exponentials(const float* q, float M, floa
     const float A = fmaf(wv, 0.125f, fmaf(p, 0.125f, a));
     const float E00 = ex2_approx(A), QB = ex2_approx(0.25f * wv), TG = ex2_approx(fmaf(qp, 0.03125f, 0.25f * p)),
                 SD = ex2_approx(0.0625f * qp);
-    float Er = E00, Qr = QB;
+    // rows (0, 1) and (2, 3) ride in the two halves of packed fp32x2 registers: one multiply advances two rows
+    const float TG2 = TG * TG, SD2 = SD * SD;
+    const float2 q01 = make_float2(QB, QB * SD);
+    const float2 q23 = __fmul2_rn(q01, make_float2(SD2, SD2));
+    X01[0] = make_float2(E00, E00 * TG);
+    X23[0] = __fmul2_rn(X01[0], make_float2(TG2, TG2));
 #pragma unroll
-    for (int r = 0; r < 4; ++r) {
-        E[4 * r] = Er;
-        E[4 * r + 1] = Er * Qr;
-        E[4 * r + 2] = E[4 * r + 1] * Qr;
-        E[4 * r + 3] = E[4 * r + 2] * Qr;
-        Er *= TG;
-        Qr *= SD;
+    for (int k = 1; k < 4; ++k) {
+        X01[k] = __fmul2_rn(X01[k - 1], q01);
+        X23[k] = __fmul2_rn(X23[k - 1], q23);
     }
     return fmaxf(fabsf(p), fmaxf(fabsf(qq), fabsf(e0)));
 }
@@ -331,17 +333,20 @@ upsample_ce_rows_kernel(UpsampleCeArgs a)
 
     if (cell_row_valid) {                                        // warp-uniform
         // ---------------- fast path, pass 1: sums of exponentials of the 16 pixels
-        float Z[16];
+        float2 Z01[4], Z23[4];                                       // Z01[k] = (Z(0,k), Z(1,k)), Z23[k] = (Z(2,k), Z(3,k))
 #pragma unroll
-        for (int j = 0; j < 16; ++j) Z[j] = 0.f;
+        for (int k = 0; k < 4; ++k) Z01[k] = Z23[k] = make_float2(0.f, 0.f);
         float wmax = 0.f;
 #pragma unroll
         for (int c = 0; c < CB; ++c) {
-            float E[16];
-            wmax = fmaxf(wmax, cell_exponentials(rc.za + c * TZ, rc.M, E));
+            float2 X01[4], X23[4];
+            wmax = fmaxf(wmax, cell_exponentials(rc.za + c * TZ, rc.M, X01, X23));
 #pragma unroll
-            for (int j = 0; j < 16; ++j) Z[j] += E[j];
+            for (int k = 0; k < 4; ++k) { Z01[k] = __fadd2_rn(Z01[k], X01[k]); Z23[k] = __fadd2_rn(Z23[k], X23[k]); }
         }
+        float Z[16];                                                 // Z[4r + k]
+#pragma unroll
+        for (int k = 0; k < 4; ++k) { Z[k] = Z01[k].x; Z[4 + k] = Z01[k].y; Z[8 + k] = Z23[k].x; Z[12 + k] = Z23[k].y; }
         bool bad = !(wmax <= 16.0f);
 #pragma unroll
         for (int j = 0; j < 16; ++j) bad |= ((vmask >> j) & 1u) && !(Z[j] > 1e-18f);
@@ -422,22 +427,33 @@ upsample_ce_rows_kernel(UpsampleCeArgs a)
                 tw[r] = i == -1 ? 0.f : (i == h - 1 ? 1.0f : 1.0f - ly);
                 bw[r] = i == h - 1 ? 0.f : (i == -1 ? 1.0f : ly);
             }
-            // ---------------- fast path, pass 2
+            // ---------------- fast path, pass 2 (packed fp32x2: rows (0,1) and (2,3) side by side)
+            float2 WL01[4], WL23[4], WR01[4], WR23[4];
+#pragma unroll
+            for (int k = 0; k < 4; ++k) {
+                WL01[k] = make_float2(wl[k], wl[4 + k]); WL23[k] = make_float2(wl[8 + k], wl[12 + k]);
+                WR01[k] = make_float2(wr[k], wr[4 + k]); WR23[k] = make_float2(wr[8 + k], wr[12 + k]);
+            }
+            const float2 tw01 = make_float2(tw[0], tw[1]), tw23 = make_float2(tw[2], tw[3]);
+            const float2 bw01 = make_float2(bw[0], bw[1]), bw23 = make_float2(bw[2], bw[3]);
 #pragma unroll
             for (int c = 0; c < CB; ++c) {
-                float E[16];
-                cell_exponentials(rc.za + c * TZ, rc.M, E);
-                float tc = 0.f, bc = 0.f;
+                float2 X01[4], X23[4];
+                cell_exponentials(rc.za + c * TZ, rc.M, X01, X23);
+                float2 aL01 = __fmul2_rn(WL01[3], X01[3]), aL23 = __fmul2_rn(WL23[3], X23[3]);
+                float2 aR01 = __fmul2_rn(WR01[3], X01[3]), aR23 = __fmul2_rn(WR23[3], X23[3]);
 #pragma unroll
-                for (int r = 0; r < 4; ++r) {
-                    const float aL = fmaf(wl[4 * r], E[4 * r], fmaf(wl[4 * r + 1], E[4 * r + 1], fmaf(wl[4 * r + 2], E[4 * r + 2], wl[4 * r + 3] * E[4 * r + 3])));
-                    const float aR = fmaf(wr[4 * r], E[4 * r], fmaf(wr[4 * r + 1], E[4 * r + 1], fmaf(wr[4 * r + 2], E[4 * r + 2], wr[4 * r + 3] * E[4 * r + 3])));
-                    const float hs = aL + __shfl_up_sync(0xffffffffu, aR, 1);
-                    tc = fmaf(tw[r], hs, tc);
-                    bc = fmaf(bw[r], hs, bc);
+                for (int k = 2; k >= 0; --k) {
+                    aL01 = __ffma2_rn(WL01[k], X01[k], aL01); aL23 = __ffma2_rn(WL23[k], X23[k], aL23);
+                    aR01 = __ffma2_rn(WR01[k], X01[k], aR01); aR23 = __ffma2_rn(WR23[k], X23[k], aR23);
                 }
-                top[c] = tc;
-                if (c < C) my_bot[c * 32] = bc;
+                // own cell's left part + left cell's right part, per row
+                const float2 hs01 = __fadd2_rn(aL01, make_float2(__shfl_up_sync(0xffffffffu, aR01.x, 1), __shfl_up_sync(0xffffffffu, aR01.y, 1)));
+                const float2 hs23 = __fadd2_rn(aL23, make_float2(__shfl_up_sync(0xffffffffu, aR23.x, 1), __shfl_up_sync(0xffffffffu, aR23.y, 1)));
+                const float2 t2 = __ffma2_rn(hs23, tw23, __fmul2_rn(hs01, tw01));
+                const float2 b2 = __ffma2_rn(hs23, bw23, __fmul2_rn(hs01, bw01));
+                top[c] = t2.x + t2.y;
+                if (c < C) my_bot[c * 32] = b2.x + b2.y;
             }
         } else {
             // ---------------- slow path: row by row, exact per-pixel maxima
