@@ -30,6 +30,7 @@
 // The "- onehot(label)" part of the gradient is exact in units of 1/64, so it is accumulated with
 // integer shared-memory atomics (order-independent).
 #include "st_internal.h"
+#include "tc_common.cuh"
 
 namespace st {
 
@@ -73,7 +74,7 @@ template <bool SHIFT>
 __device__ __forceinline__ void pixel_logits(const RowCtx& rc, int c, const float (&sk)[4], float (&u)[4])
 {
     const float a = rc.za[c * TZ], b = rc.za[c * TZ + TZ_W];
-    const float vl = fmaf(rc.ly, b - a, a) - rc.M;
+    const float vl = fmaf(fmaf(rc.ly, b - a, a), kLog2e, -rc.M);
     const float vr = __shfl_down_sync(0xffffffffu, vl, 1);
     const float d = vr - vl;
     u[0] = fmaf(0.125f, d, vl); u[1] = fmaf(0.375f, d, vl); u[2] = fmaf(0.625f, d, vl); u[3] = fmaf(0.875f, d, vl);
@@ -122,18 +123,18 @@ __device__ __forceinline__ void pass2(const RowCtx& rc, const float (&sk)[4], co
 // With ly_r = (2r+1)/8 and fr_k = (2k+1)/8:  u(r,k) = A + B k + G r + D k r, so the values are geometric
 // progressions along k and r: 4 exp2 and 12 multiplications (8 of them packed: X01[k] = (E(0,k), E(1,k)),
 // X23[k] = (E(2,k), E(3,k))).  Returns the largest corner difference
-// (the caller leaves the fast path if a class changes by more than 16 across the cell: the progressions
-// would lose their small terms).
+// in the logits' own units (the caller leaves the fast path if a class changes by more than 16 log2-units across
+// the cell: the progressions would lose their small terms).  q points at raw logits; M is in log2 units.
 __device__ __forceinline__ float cell_exponentials(const float* q, float M, float2 (&X01)[4], float2 (&X23)[4])
 {
-    const float a = q[0] - M, b = q[TZ_W] - M;
+    const float a = q[0], b = q[TZ_W];
     const float ar = __shfl_down_sync(0xffffffffu, a, 1), br = __shfl_down_sync(0xffffffffu, b, 1);
     const float p = b - a, qq = br - ar, e0 = ar - a;
     const float qp = qq - p;
     const float wv = fmaf(qp, 0.125f, e0);
     const float A = fmaf(wv, 0.125f, fmaf(p, 0.125f, a));
-    const float E00 = ex2_approx(A), QB = ex2_approx(0.25f * wv), TG = ex2_approx(fmaf(qp, 0.03125f, 0.25f * p)),
-                SD = ex2_approx(0.0625f * qp);
+    const float E00 = ex2_approx(fmaf(A, kLog2e, -M)), QB = ex2_approx((0.25f * kLog2e) * wv),
+                TG = ex2_approx(fmaf(qp, 0.03125f * kLog2e, (0.25f * kLog2e) * p)), SD = ex2_approx((0.0625f * kLog2e) * qp);
     // rows (0, 1) and (2, 3) ride in the two halves of packed fp32x2 registers: one multiply advances two rows
     const float TG2 = TG * TG, SD2 = SD * SD;
     const float2 q01 = make_float2(QB, QB * SD);
@@ -171,13 +172,14 @@ template <int CB, bool CONF>
 __global__ void __launch_bounds__(R_THREADS, 2)
 upsample_ce_rows_kernel(UpsampleCeArgs a)
 {
-    extern __shared__ __align__(16) float smem_r[];
+    extern __shared__ __align__(128) float smem_r[];
     const int C = a.C, h = a.h, w = a.w, H = h * kUp, W = w * kUp;
-    float* zt = smem_r;                         // [CB][TZ_H][36]   logits * log2(e), borders replicated; classes >= C
-                                                //                  hold -1e30 (their exponentials are 0)
+    float* zt = smem_r;                         // [CB][TZ_H][36]   logits, borders replicated; classes >= C hold -1e30
+                                                //                  (their exponentials are 0)
     int* corr = (int*)(zt + CB * TZ);           // [C][TZ_H][36]    -64 * (adjoint of onehot)
     float* bsh = (float*)(corr + C * TZ);       // [R_WARPS][C][32] lower-row accumulators
     __shared__ float red[R_WARPS], red_m[R_WARPS];
+    __shared__ __align__(8) uint64_t tile_bar;
 
     const int s = blockIdx.z, x0 = blockIdx.x * RN_X, y0 = blockIdx.y * RN_Y;
     const int blk = blockIdx.y * gridDim.x + blockIdx.x, n_blk = gridDim.x * gridDim.y;
@@ -222,39 +224,71 @@ upsample_ce_rows_kernel(UpsampleCeArgs a)
         labw[r] = lo | (hi << 16);
         vb[r] = (((vmask >> (4 * r)) & 0x3u) ? 0x00000101u : 0u) | (((vmask >> (4 * r)) & 0xcu) ? 0x01010000u : 0u);
     }
-    float m_loc = -INFINITY;                               // largest logit this thread fetched
+    float m_loc = -INFINITY;                               // largest logit of this thread's share of the tile
     {
-        // a thread keeps one 16-byte group of the tile plane (81 groups) and walks the classes three at a time;
-        // fully unrolled: all of a thread's loads are in flight together
+        // a thread keeps one 16-byte group of the tile plane (81 groups) and walks the classes three at a time
         constexpr int kQuads = TZ / 4, kPlanes = R_THREADS / kQuads;       // 81, 3
         constexpr int kIter = (CB + kPlanes - 1) / kPlanes;
         const int g = tid / kQuads, q = tid % kQuads;
-        const int yy = min(max(y0 - 1 + q / (TZ_W / 4), 0), h - 1), xq = xa + 4 * (q % (TZ_W / 4));
-        const bool vec = vec_ok && xq >= 0 && xq + 3 < w;
-        const float* row = z + (int64_t)yy * w;
-        const int x_0 = min(max(xq, 0), w - 1), x_1 = min(max(xq + 1, 0), w - 1), x_2 = min(max(xq + 2, 0), w - 1),
-                  x_3 = min(max(xq + 3, 0), w - 1);
-        float4 v[kIter];
-#pragma unroll
-        for (int it = 0; it < kIter; ++it) {
-            const int c = g + it * kPlanes;
-            float4 t = make_float4(-1e30f, -1e30f, -1e30f, -1e30f);
-            if (g < kPlanes && c < C) {
-                const float* rp = row + (int64_t)c * p;
-                if (vec) t = __ldg(reinterpret_cast<const float4*>(rp + xq));
-                else { t.x = __ldg(rp + x_0); t.y = __ldg(rp + x_1); t.z = __ldg(rp + x_2); t.w = __ldg(rp + x_3); }
-                t.x *= kLog2e; t.y *= kLog2e; t.z *= kLog2e; t.w *= kLog2e;
-                m_loc = fmaxf(fmaxf(m_loc, fmaxf(t.x, t.y)), fmaxf(t.z, t.w));
+        float4* zt4 = reinterpret_cast<float4*>(zt);
+        const bool bulk = vec_ok && xa >= 0 && xa + TZ_W <= w;             // block-uniform: every tile row is one aligned run
+        if (bulk) {
+            // ---- one asynchronous bulk copy per (class, node row): 144 contiguous bytes each, no registers involved
+            const uint32_t bar = tc::smem_u32(&tile_bar);
+            if (tid == 0) { tc::mbar_init(bar, 1); tc::fence_barrier_init(); }
+            __syncthreads();
+            if (tid == 0) tc::mbar_expect_tx(bar, (uint32_t)(C * TZ * sizeof(float)));
+            for (int e = tid; e < C * TZ_H; e += R_THREADS) {
+                const int c = e / TZ_H, j = e % TZ_H;
+                const float* src = z + (int64_t)c * p + (int64_t)min(max(y0 - 1 + j, 0), h - 1) * w + xa;
+                asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
+                             ::"r"(tc::smem_u32(zt + c * TZ + j * TZ_W)), "l"(src), "r"((uint32_t)(TZ_W * sizeof(float))), "r"(bar) : "memory");
             }
-            v[it] = t;
-        }
+            for (int e = tid; e < (CB - C) * kQuads; e += R_THREADS) zt4[C * kQuads + e] = make_float4(-1e30f, -1e30f, -1e30f, -1e30f);
+            for (int e = tid; e < C * TZ / 4; e += R_THREADS) reinterpret_cast<int4*>(corr)[e] = make_int4(0, 0, 0, 0);
+            bool ok = false;
+            for (uint32_t it = 0; it < 2 * tc::kSpinLimit && !ok; ++it) ok = tc::mbar_try_wait(bar, 0);
+            if (!__syncthreads_and(ok)) {                    // block-uniform: the copies never arrived
+                if (tid == 0) atomicCAS(a.err, 0u, (unsigned int)tc::kWaitFull | (blockIdx.x << 8));
+                return;
+            }
 #pragma unroll
-        for (int it = 0; it < kIter; ++it) {
-            const int c = g + it * kPlanes;
-            if (g < kPlanes && c < CB) reinterpret_cast<float4*>(zt)[c * kQuads + q] = v[it];
+            for (int it = 0; it < kIter; ++it) {
+                const int c = g + it * kPlanes;
+                if (g < kPlanes && c < C) {
+                    const float4 t = zt4[c * kQuads + q];
+                    m_loc = fmaxf(fmaxf(m_loc, fmaxf(t.x, t.y)), fmaxf(t.z, t.w));
+                }
+            }
+        } else {
+            // ---- plain loads (edge columns, any width and alignment), fully unrolled: all of a thread's loads are in
+            // flight together
+            const int yy = min(max(y0 - 1 + q / (TZ_W / 4), 0), h - 1), xq = xa + 4 * (q % (TZ_W / 4));
+            const bool vec = vec_ok && xq >= 0 && xq + 3 < w;
+            const float* row = z + (int64_t)yy * w;
+            const int x_0 = min(max(xq, 0), w - 1), x_1 = min(max(xq + 1, 0), w - 1), x_2 = min(max(xq + 2, 0), w - 1),
+                      x_3 = min(max(xq + 3, 0), w - 1);
+            float4 v[kIter];
+#pragma unroll
+            for (int it = 0; it < kIter; ++it) {
+                const int c = g + it * kPlanes;
+                float4 t = make_float4(-1e30f, -1e30f, -1e30f, -1e30f);
+                if (g < kPlanes && c < C) {
+                    const float* rp = row + (int64_t)c * p;
+                    if (vec) t = __ldg(reinterpret_cast<const float4*>(rp + xq));
+                    else { t.x = __ldg(rp + x_0); t.y = __ldg(rp + x_1); t.z = __ldg(rp + x_2); t.w = __ldg(rp + x_3); }
+                    m_loc = fmaxf(fmaxf(m_loc, fmaxf(t.x, t.y)), fmaxf(t.z, t.w));
+                }
+                v[it] = t;
+            }
+#pragma unroll
+            for (int it = 0; it < kIter; ++it) {
+                const int c = g + it * kPlanes;
+                if (g < kPlanes && c < CB) zt4[c * kQuads + q] = v[it];
+            }
+            for (int e = tid; e < C * TZ / 4; e += R_THREADS) reinterpret_cast<int4*>(corr)[e] = make_int4(0, 0, 0, 0);
         }
     }
-    for (int e = tid; e < C * TZ / 4; e += R_THREADS) reinterpret_cast<int4*>(corr)[e] = make_int4(0, 0, 0, 0);
 #pragma unroll
     for (int o = 16; o > 0; o >>= 1) m_loc = fmaxf(m_loc, __shfl_xor_sync(0xffffffffu, m_loc, o));
     if (l == 0) red_m[wi] = m_loc;
@@ -269,7 +303,7 @@ upsample_ce_rows_kernel(UpsampleCeArgs a)
         float m = red_m[0];
 #pragma unroll
         for (int k = 1; k < R_WARPS; ++k) m = fmaxf(m, red_m[k]);
-        rc.M = m;
+        rc.M = m * kLog2e;                                 // log2 units
     }
 
     float top[CB];
@@ -301,7 +335,7 @@ upsample_ce_rows_kernel(UpsampleCeArgs a)
                 if (own) {
                     const float* q = rc.za + lab[k] * TZ;
                     const float vl = fmaf(ly, q[TZ_W] - q[0], q[0]), vr = fmaf(ly, q[TZ_W + 1] - q[1], q[1]);
-                    const float ul = fmaf((2 * k + 1) * 0.125f, vr - vl, vl) - rc.M - sk[k];
+                    const float ul = fmaf(fmaf((2 * k + 1) * 0.125f, vr - vl, vl), kLog2e, -rc.M) - sk[k];
                     loss += (__log2f(Zs[k]) - ul) * kLn2;
                     if (CONF) atomicAdd(a.conf + (int64_t)s * a.conf_stream_stride + lab[k] * C + arg[k], 1ull);
                 }
@@ -347,7 +381,7 @@ upsample_ce_rows_kernel(UpsampleCeArgs a)
         float Z[16];                                                 // Z[4r + k]
 #pragma unroll
         for (int k = 0; k < 4; ++k) { Z[k] = Z01[k].x; Z[4 + k] = Z01[k].y; Z[8 + k] = Z23[k].x; Z[12 + k] = Z23[k].y; }
-        bool bad = !(wmax <= 16.0f);
+        bool bad = !(wmax <= 16.0f / kLog2e);                       // 16 log2-units
 #pragma unroll
         for (int j = 0; j < 16; ++j) bad |= ((vmask >> j) & 1u) && !(Z[j] > 1e-18f);
         const bool slow = __any_sync(0xffffffffu, bad);
@@ -418,7 +452,7 @@ upsample_ce_rows_kernel(UpsampleCeArgs a)
                     lsum = fmaf((float)tl, q[0], fmaf((float)tr, q[d_tr], fmaf((float)bl, q[d_bl], fmaf((float)br, q[d_bl + d_tr], lsum))));
                 }
             }
-            if (own_cell) loss += (lz - (lsum * (1.0f / 64.0f) - (float)n_ok * rc.M)) * kLn2;
+            if (own_cell) loss += (lz - (lsum * (kLog2e / 64.0f) - (float)n_ok * rc.M)) * kLn2;
             // vertical weights of the rows toward the upper / lower node row (clamped borders fold into the inner row)
             float tw[4], bw[4];
 #pragma unroll
@@ -534,7 +568,7 @@ upsample_ce_rows_kernel(UpsampleCeArgs a)
 template <int CB>
 size_t rows_smem_bytes(int C)
 {
-    return ((size_t)CB * TZ + (size_t)C * TZ + (size_t)R_WARPS * C * 32) * sizeof(float) + 16;
+    return ((size_t)CB * TZ + (size_t)C * TZ + (size_t)R_WARPS * C * 32) * sizeof(float) + 128;
 }
 
 template <int CB>

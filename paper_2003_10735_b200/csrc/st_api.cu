@@ -219,7 +219,7 @@ st_status enqueue_step(st_ctx* c, int slot, bool want_conf, StageTimer* t = null
     k3.loss_part = c->loss_part; k3.db_part = c->db_part;
     k3.conf = want_conf ? c->conf_buf + (int64_t)slot * c->C * c->C : nullptr;
     k3.conf_stream_stride = (int64_t)kMaxSteps * c->C * c->C;
-    k3.bad = c->bad;
+    k3.bad = c->bad; k3.err = c->bad + 2;
     k3.S = c->S; k3.C = c->C; k3.h = c->h; k3.w = c->w;
     launch_upsample_ce(k3, s);
     if (t) t->mark("upsample_ce", s);

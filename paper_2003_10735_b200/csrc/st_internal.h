@@ -66,6 +66,7 @@ struct UpsampleCeArgs {
     unsigned long long* conf;// nullptr, or int64 [C][C] per stream: confusion of label vs argmax of the upsampled logits
     int64_t conf_stream_stride; // elements between the matrices of consecutive streams
     unsigned int* bad;       // count of labels >= C
+    unsigned int* err;       // device word: first wait that gave up (0 = none)
     int S, C, h, w;
 };
 int upsample_ce_blocks(int h, int w, int C);   // blocks per stream (sizes loss_part / db_part)
