@@ -4,8 +4,8 @@
 //
 // Geometry as in the fused upsample + cross-entropy kernel: the frame pixels 4n+2 .. 4n+5 lie between node
 // columns n and n+1 ("cell" n) with weights 1/8, 3/8, 5/8, 7/8 toward n+1, rows alike; cells -1 and w-1 / h-1
-// are the clamped borders.  A block covers 8 cell rows x 32 cell columns (one warp per cell row, one lane per
-// cell, 16 pixels each) with the logits of the 9 x 34 surrounding nodes in shared memory, borders replicated.
+// are the clamped borders.  A block covers 4 cell rows x 32 cell columns (one warp per cell row, one lane per
+// cell, 16 pixels each) with the logits of the 5 x 34 surrounding nodes in shared memory, borders replicated.
 // Per class a lane reads the cell's four corner logits and interpolates vertically, then horizontally, with one
 // fused multiply-add per step.  No pixel is shared between cells, so blocks are independent.
 #include "st_internal.h"
@@ -14,8 +14,8 @@ namespace st {
 
 namespace {
 
-constexpr int SM_WARPS = 8, SM_THREADS = SM_WARPS * 32;
-constexpr int SM_TH = SM_WARPS + 1, SM_TW = 40, SM_T = SM_TH * SM_TW;   // tile: 9 node rows x 40 columns (34 used, start at a multiple of 4)
+constexpr int SM_WARPS = 4, SM_THREADS = SM_WARPS * 32;
+constexpr int SM_TH = SM_WARPS + 1, SM_TW = 40, SM_T = SM_TH * SM_TW;   // tile: 5 node rows x 40 columns (34 used, start at a multiple of 4)
 constexpr int kMaxChunk = 32;                                            // classes held in shared memory at a time
 
 template <typename CounterT>
@@ -44,6 +44,20 @@ student_mask_kernel(StudentMaskArgs a, int chunk)
     const bool v01 = cell_ok && X0 >= 0 && X0 + 1 < W, v23 = cell_ok && X0 + 2 >= 0 && X0 + 3 < W;
 
     if (CONF) for (int e = tid; e < C * C; e += SM_THREADS) hist[e] = 0;
+    // labels of the lane's 16 pixels, fetched before the sweep over the classes (two aligned 16-bit loads per row)
+    uint32_t labw[4] = {0, 0, 0, 0};
+    if (CONF) {
+#pragma unroll
+        for (int r = 0; r < 4; ++r) {
+            const int Y = 4 * i + 2 + r;
+            if (Y >= 0 && Y < H) {
+                uint32_t llo = 0, lhi = 0;
+                if (v01) llo = __ldg(reinterpret_cast<const unsigned short*>(a.labels + (int64_t)Y * W + X0));
+                if (v23) lhi = __ldg(reinterpret_cast<const unsigned short*>(a.labels + (int64_t)Y * W + X0 + 2));
+                labw[r] = llo | (lhi << 16);
+            }
+        }
+    }
 
     float best[16];
     uint32_t arg[16];
@@ -99,11 +113,8 @@ student_mask_kernel(StudentMaskArgs a, int chunk)
             if (v23) *reinterpret_cast<unsigned short*>(a.mask + (int64_t)Y * W + X0 + 2) = (unsigned short)hi;
         }
         if (CONF) {
-            uint32_t llo = 0, lhi = 0;
             const bool ok01 = row_ok && v01, ok23 = row_ok && v23;
-            if (ok01) llo = __ldg(reinterpret_cast<const unsigned short*>(a.labels + (int64_t)Y * W + X0));
-            if (ok23) lhi = __ldg(reinterpret_cast<const unsigned short*>(a.labels + (int64_t)Y * W + X0 + 2));
-            const uint32_t lw = llo | (lhi << 16), aw = lo | (hi << 16);
+            const uint32_t lw = labw[r], aw = lo | (hi << 16);
             // a row whose four pixels are inside the frame and share one (label, class) pair is counted at once
             const bool full = ok01 && ok23, same = full && lw == (lw & 0xffu) * 0x01010101u && aw == (aw & 0xffu) * 0x01010101u;
             if (__all_sync(0xffffffffu, same || !(ok01 || ok23))) {
