@@ -220,13 +220,15 @@ int launch_sgd_update(const UpdateArgs& a, cudaStream_t s)
     const int n_red_blocks = (items + kUpdThreads / 32 - 1) / (kUpdThreads / 32);
     const int64_t n_rest = a.n_params - range_begin;
     const bool big = n_rest > 65536;
-    const int G = max_split <= 1 ? 1 : 8, E = big ? 4 : 1;
+    // many partial sums per parameter: 16 thread groups, so that a group's share fits one batch of loads
+    const int G = max_split <= 1 ? 1 : (max_split > 64 && !big ? 16 : 8), E = big ? 4 : 1;
     const int per = kUpdThreads / G * E;
     const int n_param_blocks = (int)((n_rest + per - 1) / per);
     const dim3 grid((unsigned)(n_param_blocks + n_red_blocks), (unsigned)a.S);
     const dim3 blk(kUpdThreads);
     if (G == 1 && E == 1) launch_chain(sgd_update_kernel<1, 1>, grid, blk, 0, s, a, n_param_blocks, range_begin);
     else if (G == 1) launch_chain(sgd_update_kernel<1, 4>, grid, blk, 0, s, a, n_param_blocks, range_begin);
+    else if (G == 16) launch_chain(sgd_update_kernel<16, 1>, grid, blk, 0, s, a, n_param_blocks, range_begin);
     else if (E == 1) launch_chain(sgd_update_kernel<8, 1>, grid, blk, 0, s, a, n_param_blocks, range_begin);
     else launch_chain(sgd_update_kernel<8, 4>, grid, blk, 0, s, a, n_param_blocks, range_begin);
     return n_launches;
