@@ -582,17 +582,8 @@ EncodeTiledFn get_encode_fn()
 bool make_map(CUtensorMap* m, const void* base, int rank, const uint64_t* dims, const uint64_t* strides,
               const uint32_t* box, char* err, size_t err_len, const char* what)
 {
-    EncodeTiledFn fn = get_encode_fn();
-    if (!fn) { snprintf(err, err_len, "cuTensorMapEncodeTiled is not available"); return false; }
-    cuuint64_t d[5], st[4];
-    cuuint32_t b[5], es[5];
-    for (int i = 0; i < rank; ++i) { d[i] = dims[i]; b[i] = box[i]; es[i] = 1; }
-    for (int i = 0; i + 1 < rank; ++i) st[i] = strides[i];
-    CUresult r = fn(m, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, (cuuint32_t)rank, const_cast<void*>(base), d, st, b, es,
-                    CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
-                    CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
-    if (r != CUDA_SUCCESS) { snprintf(err, err_len, "tensor map for %s rejected (CUresult %d)", what, (int)r); return false; }
-    return true;
+    return encode_tensor_map(m, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, CU_TENSOR_MAP_SWIZZLE_128B, base, rank, dims, strides, box,
+                             err, err_len, what);
 }
 
 int pow2_cols(int n) { int c = 32; while (c < n) c <<= 1; return c; }
@@ -607,6 +598,22 @@ void split_geometry(int n_chunks, int target_blocks, int* per, int* n_split)
 }
 
 }  // namespace
+
+bool encode_tensor_map(CUtensorMap* m, CUtensorMapDataType dtype, CUtensorMapSwizzle swizzle, const void* base, int rank,
+                       const uint64_t* dims, const uint64_t* strides, const uint32_t* box, char* err, size_t err_len,
+                       const char* what)
+{
+    EncodeTiledFn fn = get_encode_fn();
+    if (!fn) { snprintf(err, err_len, "cuTensorMapEncodeTiled is not available"); return false; }
+    cuuint64_t d[5], st[4];
+    cuuint32_t b[5], es[5];
+    for (int i = 0; i < rank; ++i) { d[i] = dims[i]; b[i] = box[i]; es[i] = 1; }
+    for (int i = 0; i + 1 < rank; ++i) st[i] = strides[i];
+    CUresult r = fn(m, dtype, (cuuint32_t)rank, const_cast<void*>(base), d, st, b, es, CU_TENSOR_MAP_INTERLEAVE_NONE, swizzle,
+                    CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    if (r != CUDA_SUCCESS) { snprintf(err, err_len, "tensor map for %s rejected (CUresult %d)", what, (int)r); return false; }
+    return true;
+}
 
 struct TcPlan {
     TcBuffers b;

@@ -229,7 +229,7 @@ upsample_ce_kernel(UpsampleCeArgs a, int chunk)
                 const float4 lr = A[(ny + 1) * (NX + 1) + nx + 1];  // low-right: upper-left corner
                 v = ((ul.w + ur.z) + (ll.y + lr.x)) * invP;
                 const int c = c0 + cc;
-                a.dz[((int64_t)s * C + c) * p + (int64_t)y * w + x] = v;
+                if (a.dz) a.dz[((int64_t)s * C + c) * p + (int64_t)y * w + x] = v;
                 if (a.dz_bf16)
                     a.dz_bf16[((int64_t)s * kClassPad + c) * a.dz_bf16_pitch + (int64_t)y * w + x] = __float2bfloat16_rn(v);
             }
@@ -259,9 +259,9 @@ cudaError_t prepare_upsample_ce(int C)
     return cudaFuncSetAttribute(upsample_ce_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
 }
 
-void launch_upsample_ce(const UpsampleCeArgs& a, cudaStream_t s)
+void launch_upsample_ce(const UpsampleCeArgs& a, const CUtensorMap* z_map, cudaStream_t s)
 {
-    if (upsample_ce_rows_supported(a.C)) { launch_upsample_ce_rows(a, s); return; }
+    if (upsample_ce_rows_supported(a.C)) { launch_upsample_ce_rows(a, z_map, s); return; }
     size_t smem = 0;
     const int chunk = chunk_classes(a.C, &smem);
     dim3 grid((unsigned)((a.w + NX - 1) / NX), (unsigned)((a.h + NY - 1) / NY), (unsigned)a.S);

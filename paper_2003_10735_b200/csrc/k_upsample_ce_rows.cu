@@ -32,6 +32,8 @@
 #include "st_internal.h"
 #include "tc_common.cuh"
 
+#include <string.h>
+
 namespace st {
 
 namespace {
@@ -40,6 +42,12 @@ constexpr int RN_Y = 7, RN_X = 30;
 constexpr int R_WARPS = RN_Y + 1, R_THREADS = R_WARPS * 32;
 constexpr int TZ_H = RN_Y + 2, TZ_W = 36, TZ = TZ_H * TZ_W;   // tile rows hold 36 columns: 32 used, starting at a multiple of 4
 constexpr float kLog2e = 1.4426950408889634f, kLn2 = 0.6931471805599453f;
+// Classes per iteration of the two fast-path class sweeps.  The sweeps are rolled loops: unrolled over all classes
+// they were ~70 KB of straight-line code that every warp ran through once, and instruction fetch was the main stall.
+#ifndef ST_K3_CLASS_UNROLL
+#define ST_K3_CLASS_UNROLL 3
+#endif
+constexpr int kClassUnroll = ST_K3_CLASS_UNROLL;
 
 __device__ __forceinline__ float ex2_approx(float x)
 {
@@ -101,23 +109,6 @@ __device__ __forceinline__ void pass1(const RowCtx& rc, const float (&sk)[4], fl
     }
 }
 
-template <int CB, bool SHIFT>
-__device__ __forceinline__ void pass2(const RowCtx& rc, const float (&sk)[4], const float (&wl)[4], const float (&wr)[4],
-                                      float (&top)[CB], float (&bot)[CB])
-{
-#pragma unroll
-    for (int c = 0; c < CB; ++c) {
-        float u[4];
-        pixel_logits<SHIFT>(rc, c, sk, u);
-        const float e0 = ex2_approx(u[0]), e1 = ex2_approx(u[1]), e2 = ex2_approx(u[2]), e3 = ex2_approx(u[3]);
-        const float aL = fmaf(wl[0], e0, fmaf(wl[1], e1, fmaf(wl[2], e2, wl[3] * e3)));
-        const float aR = fmaf(wr[0], e0, fmaf(wr[1], e1, fmaf(wr[2], e2, wr[3] * e3)));
-        const float hs = aL + __shfl_up_sync(0xffffffffu, aR, 1);      // own cell's left part + left cell's right part
-        top[c] = fmaf(1.0f - rc.ly, hs, top[c]);
-        bot[c] = fmaf(rc.ly, hs, bot[c]);
-    }
-}
-
 // The 16 exponentials exp2(u(r,k) - M) of one class inside the lane's cell, u bilinear between the four
 // corner logits (own column: rows i, i+1 from shared memory; right column from the next lane).
 // With ly_r = (2r+1)/8 and fr_k = (2k+1)/8:  u(r,k) = A + B k + G r + D k r, so the values are geometric
@@ -149,11 +140,12 @@ __device__ __forceinline__ float cell_exponentials(const float* q, float M, floa
     return fmaxf(fabsf(p), fmaxf(fabsf(qq), fabsf(e0)));
 }
 
-// pass 2 of one row on the slow path: like pass2, accumulating the upper part in registers and the lower part in
-// this thread's shared-memory slots
+// pass 2 of one row on the slow path: the exponentials are formed again, multiplied by the adjoint interpolation
+// weights / Z, the right-hand part goes to the next lane, and the row is added into this thread's shared-memory
+// slots of the upper and the lower node row
 template <int CB>
 __device__ __forceinline__ void pass2_slow(const RowCtx& rc, const float (&sk)[4], const float (&wl)[4], const float (&wr)[4],
-                                           float tw, float bw, float (&top)[CB], float* my_bot, int C)
+                                           float tw, float bw, float2* my_acc, int C)
 {
 #pragma unroll
     for (int c = 0; c < CB; ++c) {
@@ -163,26 +155,31 @@ __device__ __forceinline__ void pass2_slow(const RowCtx& rc, const float (&sk)[4
         const float aL = fmaf(wl[0], e0, fmaf(wl[1], e1, fmaf(wl[2], e2, wl[3] * e3)));
         const float aR = fmaf(wr[0], e0, fmaf(wr[1], e1, fmaf(wr[2], e2, wr[3] * e3)));
         const float hs = aL + __shfl_up_sync(0xffffffffu, aR, 1);
-        top[c] = fmaf(tw, hs, top[c]);
-        if (c < C) my_bot[c * 32] = fmaf(bw, hs, my_bot[c * 32]);
+        if (c < C) {
+            const float2 t = my_acc[c * 32];
+            my_acc[c * 32] = make_float2(fmaf(tw, hs, t.x), fmaf(bw, hs, t.y));
+        }
     }
 }
 
 template <int CB, bool CONF>
 __global__ void __launch_bounds__(R_THREADS, 2)
-upsample_ce_rows_kernel(UpsampleCeArgs a)
+upsample_ce_rows_kernel(UpsampleCeArgs a, const __grid_constant__ CUtensorMap z_map)
 {
     extern __shared__ __align__(128) float smem_r[];
     const int C = a.C, h = a.h, w = a.w, H = h * kUp, W = w * kUp;
     float* zt = smem_r;                         // [CB][TZ_H][36]   logits, borders replicated; classes >= C hold -1e30
                                                 //                  (their exponentials are 0)
     int* corr = (int*)(zt + CB * TZ);           // [C][TZ_H][36]    -64 * (adjoint of onehot)
-    float* bsh = (float*)(corr + C * TZ);       // [R_WARPS][C][32] lower-row accumulators
+    float2* acc = (float2*)(corr + C * TZ);     // [R_WARPS][C][32] (x, y): the cell's pull on its upper / lower node row
     __shared__ float red[R_WARPS], red_m[R_WARPS];
     __shared__ __align__(8) uint64_t tile_bar;
 
-    const int s = blockIdx.z, x0 = blockIdx.x * RN_X, y0 = blockIdx.y * RN_Y;
-    const int blk = blockIdx.y * gridDim.x + blockIdx.x, n_blk = gridDim.x * gridDim.y;
+    // Launch order: the last block row first, then rows 0, 1, ...  Blocks at the frame border do extra work, and the
+    // blocks that reach an SM first finish earlier than their later companions, so the border rows go first.
+    const int by = blockIdx.y == 0 ? gridDim.y - 1 : blockIdx.y - 1;
+    const int s = blockIdx.z, x0 = blockIdx.x * RN_X, y0 = by * RN_Y;
+    const int blk = by * gridDim.x + blockIdx.x, n_blk = gridDim.x * gridDim.y;
     const int64_t p = (int64_t)h * w;
     const float* z = a.z + (int64_t)s * C * p;
     const uint8_t* labels = a.labels + (int64_t)s * H * W;
@@ -196,6 +193,16 @@ upsample_ce_rows_kernel(UpsampleCeArgs a)
     const bool vec_ok = (w % 4 == 0) && ((uintptr_t)z % 16 == 0);
     const int xa = vec_ok ? ((x0 - 1) & ~3) : x0 - 1;      // x0-1 >= -1; (-1 & ~3) = -4
     const int off = (x0 - 1) - xa;                         // column of node x0-1 inside the tile
+    if (a.has_map && tid == 0) {                           // block-uniform flag (implies vec_ok)
+        // one tile copy for the whole block, started before anything else: box {36 columns, RN_Y + 2 node rows,
+        // C classes} at (xa, y0 - 1, s C).  Rows and columns outside the map arrive as zeros and are replaced
+        // below by the clamped border values.
+        const uint32_t bar = tc::smem_u32(&tile_bar);
+        tc::mbar_init(bar, 1);
+        tc::fence_barrier_init();
+        tc::mbar_expect_tx(bar, (uint32_t)(C * TZ * sizeof(float)));
+        tc::tma_load_3d(tc::smem_u32(zt), &z_map, bar, xa, y0 - 1, s * C);
+    }
     const int i = y0 - 1 + wi;                  // cell row: frame rows 4i+2 .. 4i+5, node rows (i, i+1)
     const int n = x0 - 1 + l;                   // own node column; cell n lies between node columns n and n+1
     const bool cell_row_valid = i <= h - 1;
@@ -231,26 +238,42 @@ upsample_ce_rows_kernel(UpsampleCeArgs a)
         constexpr int kIter = (CB + kPlanes - 1) / kPlanes;
         const int g = tid / kQuads, q = tid % kQuads;
         float4* zt4 = reinterpret_cast<float4*>(zt);
-        const bool bulk = vec_ok && xa >= 0 && xa + TZ_W <= w;             // block-uniform: every tile row is one aligned run
-        if (bulk) {
-            // ---- one asynchronous bulk copy per (class, node row): 144 contiguous bytes each, no registers involved
+        if (a.has_map) {
+            // ---- the tile copy is in flight since the start of the block
             const uint32_t bar = tc::smem_u32(&tile_bar);
-            if (tid == 0) { tc::mbar_init(bar, 1); tc::fence_barrier_init(); }
-            __syncthreads();
-            if (tid == 0) tc::mbar_expect_tx(bar, (uint32_t)(C * TZ * sizeof(float)));
-            for (int e = tid; e < C * TZ_H; e += R_THREADS) {
-                const int c = e / TZ_H, j = e % TZ_H;
-                const float* src = z + (int64_t)c * p + (int64_t)min(max(y0 - 1 + j, 0), h - 1) * w + xa;
-                asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
-                             ::"r"(tc::smem_u32(zt + c * TZ + j * TZ_W)), "l"(src), "r"((uint32_t)(TZ_W * sizeof(float))), "r"(bar) : "memory");
-            }
             for (int e = tid; e < (CB - C) * kQuads; e += R_THREADS) zt4[C * kQuads + e] = make_float4(-1e30f, -1e30f, -1e30f, -1e30f);
             for (int e = tid; e < C * TZ / 4; e += R_THREADS) reinterpret_cast<int4*>(corr)[e] = make_int4(0, 0, 0, 0);
+            __syncthreads();                                   // the barrier's initialisation is visible to every waiter
             bool ok = false;
             for (uint32_t it = 0; it < 2 * tc::kSpinLimit && !ok; ++it) ok = tc::mbar_try_wait(bar, 0);
-            if (!__syncthreads_and(ok)) {                    // block-uniform: the copies never arrived
+            if (!__syncthreads_and(ok)) {                    // block-uniform: the copy never arrived
                 if (tid == 0) atomicCAS(a.err, 0u, (unsigned int)tc::kWaitFull | (blockIdx.x << 8));
+                tc::drain_after_error();
                 return;
+            }
+            const bool edge_rows = y0 == 0 || y0 + RN_Y > h - 1, edge_cols = xa < 0 || xa + TZ_W > w;
+            if (edge_rows) {                                   // block-uniform: node rows above 0 / below h-1 repeat the border row
+                const int j_lo = y0 == 0 ? 1 : 0;              // first tile row inside the map
+                const int j_hi = min(TZ_H - 1, h - y0);        // last one
+                const int n_out = TZ_H - (j_hi - j_lo + 1);    // rows to fill: 0 .. j_lo-1 and j_hi+1 .. TZ_H-1
+                for (int e = tid; e < C * n_out * (TZ_W / 4); e += R_THREADS) {
+                    const int c = e / (n_out * (TZ_W / 4)), r = (e / (TZ_W / 4)) % n_out, x4 = e % (TZ_W / 4);
+                    const int j = r < j_lo ? r : j_hi + 1 + (r - j_lo);
+                    const int jc = j < j_lo ? j_lo : j_hi;
+                    zt4[(c * TZ + j * TZ_W) / 4 + x4] = zt4[(c * TZ + jc * TZ_W) / 4 + x4];
+                }
+                __syncthreads();
+            }
+            if (edge_cols) {                                   // node columns left of 0 / right of w-1 repeat the border column
+                const int x_lo = xa < 0 ? -xa : 0;             // first tile column inside the map
+                const int x_hi = min(TZ_W - 1, w - 1 - xa);    // last one
+                const int n_out = TZ_W - (x_hi - x_lo + 1);
+                for (int e = tid; e < C * TZ_H * n_out; e += R_THREADS) {
+                    const int row = e / n_out, r = e % n_out;  // row = c * TZ_H + j
+                    const int x = r < x_lo ? r : x_hi + 1 + (r - x_lo);
+                    zt[row * TZ_W + x] = zt[row * TZ_W + (x < x_lo ? x_lo : x_hi)];
+                }
+                __syncthreads();
             }
 #pragma unroll
             for (int it = 0; it < kIter; ++it) {
@@ -306,12 +329,9 @@ upsample_ce_rows_kernel(UpsampleCeArgs a)
         rc.M = m * kLog2e;                                 // log2 units
     }
 
-    float top[CB];
-#pragma unroll
-    for (int c = 0; c < CB; ++c) top[c] = 0.f;
     float loss = 0.f;
     unsigned n_bad = 0;
-    float* my_bot = bsh + (size_t)wi * C * 32 + l;             // this thread's slot of class c: my_bot[c * 32]
+    float2* my_acc = acc + (size_t)wi * C * 32 + l;            // this thread's slot of class c: my_acc[c * 32]
 
     // at the clamped left and right borders the outer node column is the inner one
     const bool fold_l = n == -1, fold_r = n == w - 1;
@@ -371,7 +391,7 @@ upsample_ce_rows_kernel(UpsampleCeArgs a)
 #pragma unroll
         for (int k = 0; k < 4; ++k) Z01[k] = Z23[k] = make_float2(0.f, 0.f);
         float wmax = 0.f;
-#pragma unroll
+#pragma unroll kClassUnroll
         for (int c = 0; c < CB; ++c) {
             float2 X01[4], X23[4];
             wmax = fmaxf(wmax, cell_exponentials(rc.za + c * TZ, rc.M, X01, X23));
@@ -470,7 +490,7 @@ upsample_ce_rows_kernel(UpsampleCeArgs a)
             }
             const float2 tw01 = make_float2(tw[0], tw[1]), tw23 = make_float2(tw[2], tw[3]);
             const float2 bw01 = make_float2(bw[0], bw[1]), bw23 = make_float2(bw[2], bw[3]);
-#pragma unroll
+#pragma unroll kClassUnroll
             for (int c = 0; c < CB; ++c) {
                 float2 X01[4], X23[4];
                 cell_exponentials(rc.za + c * TZ, rc.M, X01, X23);
@@ -486,12 +506,11 @@ upsample_ce_rows_kernel(UpsampleCeArgs a)
                 const float2 hs23 = __fadd2_rn(aL23, make_float2(__shfl_up_sync(0xffffffffu, aR23.x, 1), __shfl_up_sync(0xffffffffu, aR23.y, 1)));
                 const float2 t2 = __ffma2_rn(hs23, tw23, __fmul2_rn(hs01, tw01));
                 const float2 b2 = __ffma2_rn(hs23, bw23, __fmul2_rn(hs01, bw01));
-                top[c] = t2.x + t2.y;
-                if (c < C) my_bot[c * 32] = b2.x + b2.y;
+                if (c < C) my_acc[c * 32] = make_float2(t2.x + t2.y, b2.x + b2.y);
             }
         } else {
             // ---------------- slow path: row by row, exact per-pixel maxima
-            for (int c = 0; c < C; ++c) my_bot[c * 32] = 0.f;
+            for (int c = 0; c < C; ++c) my_acc[c * 32] = make_float2(0.f, 0.f);
             for (int r = 0; r < 4; ++r) {
                 const int Y = 4 * i + 2 + r;
                 if (!(Y >= 0 && Y < H)) continue;                    // warp-uniform
@@ -512,11 +531,11 @@ upsample_ce_rows_kernel(UpsampleCeArgs a)
                 finish_row(r, Zs, ex, ar4, wl4, wr4);
                 const float twr = i == -1 ? 0.f : (i == h - 1 ? 1.0f : 1.0f - rc.ly);
                 const float bwr = i == h - 1 ? 0.f : (i == -1 ? 1.0f : rc.ly);
-                pass2_slow<CB>(rc, ex, wl4, wr4, twr, bwr, top, my_bot, C);
+                pass2_slow<CB>(rc, ex, wl4, wr4, twr, bwr, my_acc, C);
             }
         }
     } else {
-        for (int c = 0; c < C; ++c) my_bot[c * 32] = 0.f;
+        for (int c = 0; c < C; ++c) my_acc[c * 32] = make_float2(0.f, 0.f);
     }
     // loss of the block, fixed order
 #pragma unroll
@@ -525,40 +544,68 @@ upsample_ce_rows_kernel(UpsampleCeArgs a)
     if (n_bad) atomicAdd(a.bad, n_bad);
     __syncthreads();
 
-    // ---- node row y0-1+wi (warps 1..RN_Y): own upper part + lower part of the warp above + onehot part
+    // ---- node row y0-1+wi (warps 1..RN_Y): own upper part + lower part of the warp above + onehot part.
+    // All shared-memory reads of the 21 classes are issued before the first store.
     const float invP = 1.0f / ((float)H * (float)W);
     const int y = i;
     const bool node_ok = wi >= 1 && y < h && node_owned;
-    float* vs = zt;          // [C][R_THREADS] this block's gradient values, for the bias-gradient partial (the tile is no longer read)
-#pragma unroll
-    for (int c = 0; c < CB; ++c) {
-        if (c < C) {
-            float v = 0.f;
-            if (node_ok) {
-                const int cr = corr[c * TZ + wi * TZ_W + off + l];
-                v = (top[c] + bsh[((wi - 1) * C + c) * 32 + l] + (float)cr * (1.0f / 64.0f)) * invP;
-                a.dz[((int64_t)s * C + c) * p + (int64_t)y * w + n] = v;
-                if (a.dz_bf16)
-                    a.dz_bf16[((int64_t)s * kClassPad + c) * a.dz_bf16_pitch + (int64_t)y * w + n] = __float2bfloat16_rn(v);
-            }
-            vs[c * R_THREADS + tid] = v;
-        }
-    }
-    __syncthreads();
+    constexpr int CP = 32;                       // classes padded to the warp width for the lane reduce-scatter
+    float v[CP];
     {
-        // eight threads per class, 32 values each (rotated start: conflict-free), then a three-step tree: fixed order
-        const int c = tid >> 3, sub = tid & 7;
-        float t = 0.f;
-        if (c < C) {
-#pragma unroll 8
-            for (int j = 0; j < 32; ++j) t += vs[c * R_THREADS + sub * 32 + ((j + l) & 31)];
+        int cr[CB];
+        float2 up[CB], lo[CB];
+#pragma unroll
+        for (int c = 0; c < CB; ++c) {
+            cr[c] = 0; up[c] = lo[c] = make_float2(0.f, 0.f);
+            if (c < C && node_ok) {
+                cr[c] = corr[c * TZ + wi * TZ_W + off + l];
+                up[c] = acc[(wi * C + c) * 32 + l];
+                lo[c] = acc[((wi - 1) * C + c) * 32 + l];
+            }
         }
-        t += __shfl_xor_sync(0xffffffffu, t, 1);
-        t += __shfl_xor_sync(0xffffffffu, t, 2);
-        t += __shfl_xor_sync(0xffffffffu, t, 4);
-        if (c < C && sub == 0) a.db_part[((int64_t)s * n_blk + blk) * C + c] = t;
+#pragma unroll
+        for (int c = 0; c < CB; ++c) v[c] = (up[c].x + lo[c].y + (float)cr[c] * (1.0f / 64.0f)) * invP;
+#pragma unroll
+        for (int c = CB; c < CP; ++c) v[c] = 0.f;
     }
-    if (tid == 0) {
+    if (node_ok) {
+        if (a.dz) {
+            float* dzp = a.dz + (int64_t)s * C * p + (int64_t)y * w + n;
+#pragma unroll
+            for (int c = 0; c < CB; ++c)
+                if (c < C) dzp[(int64_t)c * p] = v[c];
+        }
+        if (a.dz_bf16) {
+            bf16* dzb = a.dz_bf16 + (int64_t)s * kClassPad * a.dz_bf16_pitch + (int64_t)y * w + n;
+#pragma unroll
+            for (int c = 0; c < CB; ++c)
+                if (c < C) dzb[(int64_t)c * a.dz_bf16_pitch] = __float2bfloat16_rn(v[c]);
+        }
+    }
+    // bias-gradient partial of the block: sum of the block's gradient values per class.  Lane reduce-scatter inside
+    // each warp (31 exchanges for 32 classes: at distance o a lane keeps the half of its values whose class has bit o
+    // equal to its own lane bit and adds the partner's), after which lane c holds class c; then the warps' sums are
+    // added in warp order.  Fixed order throughout.
+#pragma unroll
+    for (int o = CP / 2; o > 0; o >>= 1) {
+        const bool hi = l & o;
+#pragma unroll
+        for (int j = 0; j < o; ++j) {
+            const float send = hi ? v[j] : v[j + o];
+            const float keep = hi ? v[j + o] : v[j];
+            v[j] = keep + __shfl_xor_sync(0xffffffffu, send, o);
+        }
+    }
+    float* wsum = zt;                            // [R_WARPS][32] (the tile is no longer read)
+    wsum[wi * 32 + l] = v[0];
+    __syncthreads();
+    if (tid < C) {
+        float t = 0.f;
+#pragma unroll
+        for (int k = 1; k < R_WARPS; ++k) t += wsum[k * 32 + tid];
+        a.db_part[((int64_t)s * n_blk + blk) * C + tid] = t;
+    }
+    if (tid == 32) {
         float t = 0.f;
         for (int k = 0; k < R_WARPS; ++k) t += red[k];
         a.loss_part[(int64_t)s * n_blk + blk] = t;
@@ -568,7 +615,7 @@ upsample_ce_rows_kernel(UpsampleCeArgs a)
 template <int CB>
 size_t rows_smem_bytes(int C)
 {
-    return ((size_t)CB * TZ + (size_t)C * TZ + (size_t)R_WARPS * C * 32) * sizeof(float) + 128;
+    return ((size_t)CB * TZ + (size_t)C * TZ + (size_t)R_WARPS * C * 32 * 2) * sizeof(float) + 128;
 }
 
 template <int CB>
@@ -580,11 +627,11 @@ cudaError_t prepare_cb(int C)
 }
 
 template <int CB>
-cudaError_t launch_cb(const UpsampleCeArgs& a, cudaStream_t s)
+cudaError_t launch_cb(const UpsampleCeArgs& a, const CUtensorMap& z_map, cudaStream_t s)
 {
     dim3 grid((unsigned)((a.w + RN_X - 1) / RN_X), (unsigned)((a.h + RN_Y - 1) / RN_Y), (unsigned)a.S);
-    if (a.conf) return launch_chain(upsample_ce_rows_kernel<CB, true>, grid, dim3(R_THREADS), rows_smem_bytes<CB>(a.C), s, a);
-    return launch_chain(upsample_ce_rows_kernel<CB, false>, grid, dim3(R_THREADS), rows_smem_bytes<CB>(a.C), s, a);
+    if (a.conf) return launch_chain(upsample_ce_rows_kernel<CB, true>, grid, dim3(R_THREADS), rows_smem_bytes<CB>(a.C), s, a, z_map);
+    return launch_chain(upsample_ce_rows_kernel<CB, false>, grid, dim3(R_THREADS), rows_smem_bytes<CB>(a.C), s, a, z_map);
 }
 
 // class-count buckets: the two workload sizes exactly, multiples of four otherwise
@@ -616,8 +663,27 @@ int upsample_ce_rows_blocks(int h, int w) { return ((h + RN_Y - 1) / RN_Y) * ((w
 
 cudaError_t prepare_upsample_ce_rows(int C) { ST_ROWS_DISPATCH(prepare_cb, C, C) }
 
-cudaError_t launch_rows_dispatch(const UpsampleCeArgs& a, cudaStream_t s) { ST_ROWS_DISPATCH(launch_cb, a.C, a, s) }
+cudaError_t launch_rows_dispatch(const UpsampleCeArgs& a, const CUtensorMap& z_map, cudaStream_t s) { ST_ROWS_DISPATCH(launch_cb, a.C, a, z_map, s) }
 
-void launch_upsample_ce_rows(const UpsampleCeArgs& a, cudaStream_t s) { launch_rows_dispatch(a, s); }
+void launch_upsample_ce_rows(const UpsampleCeArgs& a, const CUtensorMap* z_map, cudaStream_t s)
+{
+    if (a.has_map && z_map) { launch_rows_dispatch(a, *z_map, s); return; }
+    UpsampleCeArgs b = a;
+    b.has_map = 0;
+    CUtensorMap none;
+    memset(&none, 0, sizeof(none));
+    launch_rows_dispatch(b, none, s);
+}
+
+bool make_logit_tile_map(CUtensorMap* m, const float* z, int S, int C, int h, int w)
+{
+    if (!upsample_ce_rows_supported(C) || w % 4 != 0 || w < TZ_W || h < TZ_H || ((uintptr_t)z & 15u)) return false;
+    const uint64_t dims[3] = {(uint64_t)w, (uint64_t)h, (uint64_t)S * C};
+    const uint64_t strides[2] = {(uint64_t)w * sizeof(float), (uint64_t)h * w * sizeof(float)};
+    const uint32_t box[3] = {(uint32_t)TZ_W, (uint32_t)TZ_H, (uint32_t)C};
+    char err[128];
+    return encode_tensor_map(m, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, CU_TENSOR_MAP_SWIZZLE_NONE, z, 3, dims, strides, box, err,
+                             sizeof(err), "logit tile");
+}
 
 }  // namespace st

@@ -44,6 +44,8 @@ struct st_ctx {
     int n_split1 = 0, n_split2 = 0, n_b1part = 0;
     float *loss_part = nullptr, *db_part = nullptr;
     int n_k3_blocks = 0;
+    CUtensorMap k3_map;        // tile map of z for the fused upsample + cross-entropy kernel
+    int k3_has_map = 0;
     float* loss_buf = nullptr;              // [S][kMaxSteps]
     unsigned long long* conf_buf = nullptr; // [S][kMaxSteps][C][C], allocated on first use
     unsigned int* bad = nullptr;            // [3]: labels >= C met by a step / by st_agreement; [2] = first device wait that gave up
@@ -207,21 +209,33 @@ st_status enqueue_forward(st_ctx* c, StageTimer* t = nullptr)
     return check_launch(c, "head forward");
 }
 
+// Arguments of the fused upsample + cross-entropy kernel.  With bf16 GEMMs the weight gradient and the dgrad read the
+// bf16 copy of the logit gradient only, so the fp32 copy is not written during a step (st_read_tensor produces it on
+// demand by running the kernel once more on the same logits and labels).
+UpsampleCeArgs k3_args(st_ctx* c, bool fp32_grad, bool bf16_grad, unsigned long long* conf)
+{
+    UpsampleCeArgs k3;
+    k3.z = c->z; k3.labels = c->labels;
+    k3.dz = fp32_grad ? c->dz : nullptr;
+    k3.dz_bf16 = bf16_grad ? c->dz_bf16 : nullptr;
+    k3.dz_bf16_pitch = c->dz_pitch;
+    k3.loss_part = c->loss_part; k3.db_part = c->db_part;
+    k3.conf = conf;
+    k3.conf_stream_stride = (int64_t)kMaxSteps * c->C * c->C;
+    k3.bad = c->bad; k3.err = c->bad + 2;
+    k3.S = c->S; k3.C = c->C; k3.h = c->h; k3.w = c->w;
+    k3.has_map = c->k3_has_map;
+    return k3;
+}
+
 st_status enqueue_step(st_ctx* c, int slot, bool want_conf, StageTimer* t = nullptr)
 {
     cudaStream_t s = c->stream;
     st_status st = enqueue_forward(c, t);
     if (st != ST_OK) return st;
 
-    UpsampleCeArgs k3;
-    k3.z = c->z; k3.labels = c->labels; k3.dz = c->dz; k3.dz_bf16 = c->bf16_mode ? c->dz_bf16 : nullptr;
-    k3.dz_bf16_pitch = c->dz_pitch;
-    k3.loss_part = c->loss_part; k3.db_part = c->db_part;
-    k3.conf = want_conf ? c->conf_buf + (int64_t)slot * c->C * c->C : nullptr;
-    k3.conf_stream_stride = (int64_t)kMaxSteps * c->C * c->C;
-    k3.bad = c->bad; k3.err = c->bad + 2;
-    k3.S = c->S; k3.C = c->C; k3.h = c->h; k3.w = c->w;
-    launch_upsample_ce(k3, s);
+    const UpsampleCeArgs k3 = k3_args(c, !c->bf16_mode, c->bf16_mode, want_conf ? c->conf_buf + (int64_t)slot * c->C * c->C : nullptr);
+    launch_upsample_ce(k3, &c->k3_map, s);
     if (t) t->mark("upsample_ce", s);
     c->launches += 1;
     st = check_launch(c, "upsample + cross-entropy");
@@ -412,6 +426,7 @@ st_status st_init_head(const st_head_desc* desc, const float* init_params, st_ct
     }
 #undef ALLOC
     if (e == cudaSuccess) e = prepare_upsample_ce(c->C);
+    if (e == cudaSuccess) c->k3_has_map = make_logit_tile_map(&c->k3_map, c->z, S, c->C, c->h, c->w) ? 1 : 0;
     if (e == cudaSuccess) e = prepare_student_mask(c->C);
     if (e != cudaSuccess) {
         st_status code = fail(nullptr, e == cudaErrorMemoryAllocation ? ST_ERR_OOM : ST_ERR_CUDA,
@@ -743,7 +758,13 @@ st_status st_read_tensor(st_ctx* ctx, int32_t stream, st_tensor which, float* ds
     const int64_t s = stream;
     switch (which) {
         case ST_TENSOR_LOGITS: src = ctx->z + s * ctx->C * ctx->p; break;
-        case ST_TENSOR_LOGIT_GRAD: src = ctx->dz + s * ctx->C * ctx->p; break;
+        case ST_TENSOR_LOGIT_GRAD:
+            if (ctx->bf16_mode) {     // the step wrote the bf16 copy only: same logits, same labels, same arithmetic once more
+                launch_upsample_ce(k3_args(ctx, true, false, nullptr), &ctx->k3_map, ctx->stream);
+                ctx->launches += 1;
+            }
+            src = ctx->dz + s * ctx->C * ctx->p;
+            break;
         case ST_TENSOR_PARAM_GRAD: launch_pack(ctx->grad + s * ctx->n_params, ctx->read_tmp, ctx->layout, 1, ctx->stream); src = ctx->read_tmp; break;
         case ST_TENSOR_MOMENTUM: launch_pack(ctx->vel + s * ctx->n_params, ctx->read_tmp, ctx->layout, 1, ctx->stream); src = ctx->read_tmp; break;
         case ST_TENSOR_HIDDEN:

@@ -2,6 +2,7 @@
 // Nothing here is part of the public interface (see include/shadowtutor.h).
 #pragma once
 
+#include <cuda.h>
 #include <cuda_bf16.h>
 #include <cuda_runtime.h>
 #include <stdint.h>
@@ -58,7 +59,7 @@ void launch_nhwc_bf16_to_chw(const bf16* in, int C, int64_t p, float* out, cudaS
 struct UpsampleCeArgs {
     const float* z;          // [S][C][h][w]
     const uint8_t* labels;   // [S][H][W]
-    float* dz;               // [S][C][h][w]     gradient of the mean loss
+    float* dz;               // [S][C][h][w]     gradient of the mean loss, or nullptr (only the bf16 copy is wanted)
     bf16* dz_bf16;           // [S][kClassPad][dz_bf16_pitch] or nullptr (rows >= C untouched)
     int64_t dz_bf16_pitch;
     float* loss_part;        // [S][n_blocks]    per-block partial sums of per-pixel losses
@@ -68,15 +69,24 @@ struct UpsampleCeArgs {
     unsigned int* bad;       // count of labels >= C
     unsigned int* err;       // device word: first wait that gave up (0 = none)
     int S, C, h, w;
+    int has_map;             // the launch carries a tile map of z (see make_logit_tile_map)
 };
+// Tile map of the logits for the row-walking kernel: fp32 tensor {w, h, S*C}, one box = the block's tile of all
+// classes.  False if the shape does not allow it (w not a multiple of 4, C > 32) or the driver entry point is
+// missing; the kernel then fetches its tile with plain loads.
+bool make_logit_tile_map(CUtensorMap* m, const float* z, int S, int C, int h, int w);
+// general form: any element type and swizzle; dims innermost first, strides (bytes) for dimensions 1..rank-1
+bool encode_tensor_map(CUtensorMap* m, CUtensorMapDataType dtype, CUtensorMapSwizzle swizzle, const void* base, int rank,
+                       const uint64_t* dims, const uint64_t* strides, const uint32_t* box, char* err, size_t err_len,
+                       const char* what);
 int upsample_ce_blocks(int h, int w, int C);   // blocks per stream (sizes loss_part / db_part)
 cudaError_t prepare_upsample_ce(int C);   // once per device and class count, outside any stream capture
-void launch_upsample_ce(const UpsampleCeArgs& a, cudaStream_t s);
+void launch_upsample_ce(const UpsampleCeArgs& a, const CUtensorMap* z_map, cudaStream_t s);   // z_map: host copy, used if a.has_map
 // register-resident variant for C <= 32 (k_upsample_ce_rows.cu); launch_upsample_ce dispatches to it
 bool upsample_ce_rows_supported(int C);
 int upsample_ce_rows_blocks(int h, int w);
 cudaError_t prepare_upsample_ce_rows(int C);
-void launch_upsample_ce_rows(const UpsampleCeArgs& a, cudaStream_t s);
+void launch_upsample_ce_rows(const UpsampleCeArgs& a, const CUtensorMap* z_map, cudaStream_t s);
 // student mask: argmax_c of the upsampled logits, uint8 [H][W]; with `labels` also the confusion matrix of
 // (label, mask) added into `conf`, and with `miou` the mean IoU written by the last block (k_student_mask.cu)
 struct StudentMaskArgs {
