@@ -18,8 +18,8 @@
  *     context's CUDA stream during work enqueued by that call; it keeps no reference
  *     afterwards.  Inputs must stay alive until the stream has passed that work.
  *   - Calls enqueue work on `cuda_stream` and return.  Only calls with a host out-value
- *     (`st_pack_updated_params` with a host destination, `st_agreement`'s `miou`,
- *     `st_read_tensor`) wait for the stream.
+ *     (`st_pack_updated_params` with a host destination, `st_agreement` unless its `miou` is a
+ *     device pointer, `st_read_tensor`) wait for the stream.
  *   - Errors are status codes; nothing aborts, throws or traps.  `st_last_error` gives a
  *     text for the most recent failure on that context (or, with NULL, of the last failed
  *     `st_init_head` on this thread).  All shapes are validated on the host before any
@@ -150,10 +150,12 @@ ST_API st_status st_student_mask(st_ctx *ctx, int32_t stream, uint8_t *mask_out)
  *   pred   host or device uint8 [H][W], or NULL = the current student's mask (fresh forward).
  *   label  host or device uint8 [H][W], or NULL = the stored teacher labels of `stream`.
  *   conf   host or device, or NULL; int64 [C][C], conf[l][q] = #pixels with label l and prediction q.
- *   miou   host, or NULL; mean IoU in double.
+ *   miou   host or device, or NULL; mean IoU in double.
  * Pixels whose label or prediction is >= n_classes are skipped and the call returns
  * ST_ERR_INVALID_ARG (the counts of the valid pixels are still delivered).
- * Waits for the stream.
+ * Waits for the stream, unless `miou` points to device memory: then the value is written there by
+ * work enqueued on the stream, the call returns at once, and skipped pixels are reported by the next
+ * call that does wait.
  */
 ST_API st_status st_agreement(st_ctx *ctx, int32_t stream, const uint8_t *pred, const uint8_t *label,
                        int64_t *conf, double *miou);
@@ -181,9 +183,12 @@ ST_API st_status st_read_tensor(st_ctx *ctx, int32_t stream, st_tensor which, fl
 /*
  * st_profile_step — time the kernels of the step one by one.  Runs n_steps ordinary steps of
  * Algorithm 1's loop body (they do update the parameters) without graph replay, with a CUDA event
- * recorded on the context's stream after every kernel, and returns the mean time per kernel.
+ * recorded on the context's stream after every kernel, and returns the mean time per launch.
+ * Every kernel except the parameter update is launched 8 times back to back between two events (its
+ * result does not depend on how often it runs), so that the launch gap of a 10-microsecond kernel
+ * does not dominate its figure; the update is launched once and its figure includes that gap.
  *   n_stages   host; receives the number of kernels in one step (<= ST_MAX_STAGES).
- *   ms_out     host float[ST_MAX_STAGES]; mean milliseconds of each kernel, in launch order.
+ *   ms_out     host float[ST_MAX_STAGES]; mean milliseconds per launch of each kernel, in launch order.
  *   names_out  host const char*[ST_MAX_STAGES]; static strings naming the kernels.
  * Waits for the stream after every step.  A measuring aid, not part of the method.
  */

@@ -89,7 +89,7 @@ def load_library() -> ctypes.CDLL:
     lib.st_student_mask.restype = ctypes.c_int
     lib.st_student_mask.argtypes = [vp, i32, vp]
     lib.st_agreement.restype = ctypes.c_int
-    lib.st_agreement.argtypes = [vp, i32, vp, vp, vp, ctypes.POINTER(ctypes.c_double)]
+    lib.st_agreement.argtypes = [vp, i32, vp, vp, vp, vp]
     lib.st_read_tensor.restype = ctypes.c_int
     lib.st_read_tensor.argtypes = [vp, i32, ctypes.c_int, vp, ctypes.c_size_t, ctypes.POINTER(ctypes.c_size_t)]
     lib.st_profile_step.restype = ctypes.c_int
@@ -213,12 +213,23 @@ def st_student_mask(ctx: _Ctx, stream: int, mask_out) -> None:
     _check(load_library().st_student_mask(ctx.handle, stream, _ptr(mask_out, "uint8", ctx.P, "mask_out")), ctx)
 
 
-def st_agreement(ctx: _Ctx, stream: int, pred=None, label=None, conf=None) -> float:
-    """Returns the mean IoU; `conf` (int64 [C][C]) is filled if given."""
+def st_agreement(ctx: _Ctx, stream: int, pred=None, label=None, conf=None, miou_out=None):
+    """Returns the mean IoU; `conf` (int64 [C][C]) is filled if given.  With `miou_out` (a CUDA float64
+    tensor) the mean IoU is written there by work on the context's stream, the call does not wait and
+    returns None."""
+    if miou_out is not None:
+        if not getattr(miou_out, "is_cuda", False) or str(miou_out.dtype) != "torch.float64" or miou_out.numel() < 1:
+            raise TypeError("miou_out: need a CUDA float64 tensor with one element")
+        _check(load_library().st_agreement(ctx.handle, stream, _ptr(pred, "uint8", ctx.P, "pred"),
+                                           _ptr(label, "uint8", ctx.P, "label"),
+                                           _ptr(conf, "int64", ctx.C * ctx.C, "conf"),
+                                           ctypes.c_void_p(miou_out.data_ptr())), ctx)
+        return None
     miou = ctypes.c_double(0.0)
     _check(load_library().st_agreement(ctx.handle, stream, _ptr(pred, "uint8", ctx.P, "pred"),
                                        _ptr(label, "uint8", ctx.P, "label"),
-                                       _ptr(conf, "int64", ctx.C * ctx.C, "conf"), ctypes.byref(miou)), ctx)
+                                       _ptr(conf, "int64", ctx.C * ctx.C, "conf"),
+                                       ctypes.cast(ctypes.byref(miou), ctypes.c_void_p)), ctx)
     return float(miou.value)
 
 

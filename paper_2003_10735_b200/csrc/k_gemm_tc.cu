@@ -740,37 +740,37 @@ int tc_forward(const TcPlan* P, cudaStream_t s, StageTimer* t)
     if (b.c_hidden) {
         const int tiles = ((b.w + kTileW - 1) / kTileW) * ((b.h + kTileH - 1) / kTileH);
         const int total = tiles * b.S;
-        launch_chain(tc_fwd3x3_kernel<4>, dim3(total < P->n_sms ? total : P->n_sms), dim3(kFwd3Threads), P->smem_fwd3, s,
+        ST_REPEAT(t) launch_chain(tc_fwd3x3_kernel<4>, dim3(total < P->n_sms ? total : P->n_sms), dim3(kFwd3Threads), P->smem_fwd3, s,
             P->x_fwd3, P->w1_map, b.theta, b.n_params, b.b1_off, b.hidden, b.relu_bits, b.c_in, b.c_hidden, b.h, b.w,
             total, pow2_cols(b.c_hidden), b.err);
-        if (t) t->mark("tc_fwd3x3", s);
-        ++n;
+        if (t) t->mark("tc_fwd3x3", s, st_repeats(t));
+        n += st_repeats(t);
     }
     const int tiles1 = (P->p + kTileM - 1) / kTileM;
-    launch_chain(tc_fwd1x1_kernel, dim3(tiles1, b.S), dim3(kThreadsTc), P->smem_fwd1, s,
+    ST_REPEAT(t) launch_chain(tc_fwd1x1_kernel, dim3(tiles1, b.S), dim3(kThreadsTc), P->smem_fwd1, s,
         P->act_fwd, P->w2_map, b.theta, b.n_params, b.b2_off, b.z, b.C, P->p, P->c_last / kBlockK, b.err);
-    if (t) t->mark("tc_fwd1x1", s);
-    return n + 1;
+    if (t) t->mark("tc_fwd1x1", s, st_repeats(t));
+    return n + st_repeats(t);
 }
 
 int tc_backward(const TcPlan* P, cudaStream_t s, StageTimer* t)
 {
     const TcBuffers& b = P->b;
     int n = 0;
-    launch_chain(tc_wgrad1x1_kernel<3>, dim3(P->split2, b.S), dim3(kThreadsTc), P->smem_wg1, s,
+    ST_REPEAT(t) launch_chain(tc_wgrad1x1_kernel<3>, dim3(P->split2, b.S), dim3(kThreadsTc), P->smem_wg1, s,
         P->act_wg, P->dz_map, b.w2_partials, P->c_last, P->chunks2, P->per2, P->cols2, b.err);
-    if (t) t->mark("tc_wgrad1x1", s);
-    ++n;
+    if (t) t->mark("tc_wgrad1x1", s, st_repeats(t));
+    n += st_repeats(t);
     if (b.c_hidden) {
         const int blocks = tc_b1_partials(b.h, b.w);
-        launch_chain(tc_dgrad_kernel, dim3(blocks, b.S), dim3(kThreadsTc), P->smem_dgrad, s,
+        ST_REPEAT(t) launch_chain(tc_dgrad_kernel, dim3(blocks, b.S), dim3(kThreadsTc), P->smem_dgrad, s,
             P->dz_map, P->w2_map, b.relu_bits, b.dhidden, b.b1_partials, b.c_hidden, P->p, pow2_cols(b.c_hidden), b.err);
-        if (t) t->mark("tc_dgrad", s);
-        launch_chain(tc_wgrad3x3_kernel<3>, dim3(9 * P->split1, b.S), dim3(kThreadsTc), P->smem_wg3, s,
+        if (t) t->mark("tc_dgrad", s, st_repeats(t));
+        ST_REPEAT(t) launch_chain(tc_wgrad3x3_kernel<3>, dim3(9 * P->split1, b.S), dim3(kThreadsTc), P->smem_wg3, s,
             P->x_wg3, P->dh_wg3, b.w1_partials, b.c_in, b.c_hidden, b.h, b.w, P->chunks1, P->per1, P->split1,
             P->cols1, b.err);
-        if (t) t->mark("tc_wgrad3x3", s);
-        n += 2;
+        if (t) t->mark("tc_wgrad3x3", s, st_repeats(t));
+        n += 2 * st_repeats(t);
     }
     return n;
 }

@@ -190,21 +190,21 @@ st_status enqueue_forward(st_ctx* c, StageTimer* t = nullptr)
     if (c->bf16_mode) {
         c->launches += tc_forward(c->plan, s, t);
     } else if (c->Ch == 0) {
-        launch_conv_fwd_f32(c->x_f32, c->Cin, c->h, c->w, c->theta + c->layout.w_off[0], c->theta + c->layout.b_off[0],
+        ST_REPEAT(t) launch_conv_fwd_f32(c->x_f32, c->Cin, c->h, c->w, c->theta + c->layout.w_off[0], c->theta + c->layout.b_off[0],
                             c->C, 1, false, c->z, c->S, (int64_t)c->Cin * c->p, c->n_params, c->n_params,
                             (int64_t)c->C * c->p, s);
-        if (t) t->mark("conv1x1_fwd_f32", s);
-        c->launches += 1;
+        if (t) t->mark("conv1x1_fwd_f32", s, st_repeats(t));
+        c->launches += st_repeats(t);
     } else {
-        launch_conv_fwd_f32(c->x_f32, c->Cin, c->h, c->w, c->theta + c->layout.w_off[0], c->theta + c->layout.b_off[0],
+        ST_REPEAT(t) launch_conv_fwd_f32(c->x_f32, c->Cin, c->h, c->w, c->theta + c->layout.w_off[0], c->theta + c->layout.b_off[0],
                             c->Ch, 3, true, c->hid_f32, c->S, (int64_t)c->Cin * c->p, c->n_params, c->n_params,
                             (int64_t)c->Ch * c->p, s);
-        if (t) t->mark("conv3x3_fwd_f32", s);
-        launch_conv_fwd_f32(c->hid_f32, c->Ch, c->h, c->w, c->theta + c->layout.w_off[1], c->theta + c->layout.b_off[1],
+        if (t) t->mark("conv3x3_fwd_f32", s, st_repeats(t));
+        ST_REPEAT(t) launch_conv_fwd_f32(c->hid_f32, c->Ch, c->h, c->w, c->theta + c->layout.w_off[1], c->theta + c->layout.b_off[1],
                             c->C, 1, false, c->z, c->S, (int64_t)c->Ch * c->p, c->n_params, c->n_params,
                             (int64_t)c->C * c->p, s);
-        if (t) t->mark("conv1x1_fwd_f32", s);
-        c->launches += 2;
+        if (t) t->mark("conv1x1_fwd_f32", s, st_repeats(t));
+        c->launches += 2 * st_repeats(t);
     }
     return check_launch(c, "head forward");
 }
@@ -235,19 +235,19 @@ st_status enqueue_step(st_ctx* c, int slot, bool want_conf, StageTimer* t = null
     if (st != ST_OK) return st;
 
     const UpsampleCeArgs k3 = k3_args(c, !c->bf16_mode, c->bf16_mode, want_conf ? c->conf_buf + (int64_t)slot * c->C * c->C : nullptr);
-    launch_upsample_ce(k3, &c->k3_map, s);
-    if (t) t->mark("upsample_ce", s);
-    c->launches += 1;
+    ST_REPEAT(t) launch_upsample_ce(k3, &c->k3_map, s);
+    if (t) t->mark("upsample_ce", s, st_repeats(t));
+    c->launches += st_repeats(t);
     st = check_launch(c, "upsample + cross-entropy");
     if (st != ST_OK) return st;
 
     if (c->bf16_mode) {
         c->launches += tc_backward(c->plan, s, t);
     } else if (c->Ch == 0) {
-        launch_conv_wgrad_f32(c->x_f32, c->dz, c->Cin, c->C, c->h, c->w, 1, c->grad + c->layout.w_off[0], c->S,
+        ST_REPEAT(t) launch_conv_wgrad_f32(c->x_f32, c->dz, c->Cin, c->C, c->h, c->w, 1, c->grad + c->layout.w_off[0], c->S,
                               (int64_t)c->Cin * c->p, (int64_t)c->C * c->p, c->n_params, s);
-        if (t) t->mark("conv1x1_wgrad_f32", s);
-        c->launches += 1;
+        if (t) t->mark("conv1x1_wgrad_f32", s, st_repeats(t));
+        c->launches += st_repeats(t);
     } else {
         const int64_t hs = (int64_t)c->Ch * c->p;
         launch_conv_wgrad_f32(c->hid_f32, c->dz, c->Ch, c->C, c->h, c->w, 1, c->grad + c->layout.w_off[1], c->S,
@@ -257,14 +257,14 @@ st_status enqueue_step(st_ctx* c, int slot, bool want_conf, StageTimer* t = null
         launch_conv_wgrad_f32(c->x_f32, c->dhid_f32, c->Cin, c->Ch, c->h, c->w, 3, c->grad + c->layout.w_off[0], c->S,
                               (int64_t)c->Cin * c->p, hs, c->n_params, s);
         launch_bias_grad_f32(c->dhid_f32, c->Ch, c->p, c->grad + c->layout.b_off[0], c->S, hs, c->n_params, s);
-        if (t) t->mark("backward_f32", s);
+        if (t) t->mark("backward_f32", s, 4);
         c->launches += 4;
     }
     st = check_launch(c, "head backward");
     if (st != ST_OK) return st;
 
     c->launches += launch_sgd_update(make_update_args(c, slot), s);
-    if (t) t->mark("sgd_update", s);
+    if (t) t->mark("sgd_update", s, 1);
     return check_launch(c, "sgd update");
 }
 
@@ -585,6 +585,7 @@ st_status st_profile_step(st_ctx* ctx, int32_t n_steps, int32_t* n_stages, float
         if (!ctx->has_feat[s] || !ctx->has_labels[s])
             return fail(ctx, ST_ERR_BAD_STATE, "st_profile_step: stream %d has no features or labels yet", s);
     StageTimer t;
+    t.repeat = 8;
     for (int i = 0; i <= StageTimer::kMax; ++i) ST_CUDA(ctx, cudaEventCreate(&t.ev[i]));
     double acc[StageTimer::kMax] = {0};
     st_status st = ST_OK;
@@ -599,7 +600,7 @@ st_status st_profile_step(st_ctx* ctx, int32_t n_steps, int32_t* n_stages, float
         for (int i = 0; i < n; ++i) {
             float ms = 0.f;
             cudaEventElapsedTime(&ms, t.ev[i], t.ev[i + 1]);
-            acc[i] += ms;
+            acc[i] += ms / t.launches[i];
         }
     }
     for (int i = 0; i <= StageTimer::kMax; ++i) cudaEventDestroy(t.ev[i]);
@@ -723,6 +724,11 @@ st_status st_agreement(st_ctx* ctx, int32_t stream, const uint8_t* pred, const u
     st = check_launch(ctx, "confusion");
     if (st != ST_OK) return st;
     if (conf) ST_CUDA(ctx, cudaMemcpyAsync(conf, ctx->conf_tmp, cbytes, cudaMemcpyDefault, ctx->stream));
+    if (miou && is_device_ptr(miou)) {
+        // device destination: nothing to wait for; bad labels surface at the next call that does wait
+        ST_CUDA(ctx, cudaMemcpyAsync(miou, ctx->miou_tmp, sizeof(double), cudaMemcpyDeviceToDevice, ctx->stream));
+        return ST_OK;
+    }
     st = fetch_status(ctx);
     if (st != ST_OK) return st;
     if (miou) *miou = ctx->status_host[0];

@@ -183,14 +183,20 @@ int tc_b1_partials(int h, int w);
 int tc_dz_pitch(int h, int w);      // row pitch (elements) of the bf16 logit gradient [S][kClassPad][pitch]
 TcPlan* tc_plan_create(const TcBuffers& b, char* err, size_t err_len);
 void tc_plan_destroy(TcPlan*);
-// Optional per-kernel timing: an event is recorded on the stream after each kernel launch.
+// Optional per-kernel timing: an event is recorded on the stream after each kernel's launches.  Kernels whose
+// result does not depend on how often they run (everything but the parameter update) are launched `repeat` times
+// back to back, so that the time between two events is `repeat` kernel durations plus one launch gap.
 struct StageTimer {
     static constexpr int kMax = 12;
     cudaEvent_t ev[kMax + 1];
     const char* name[kMax];
+    int launches[kMax];
+    int repeat = 1;
     int n = 0;
-    void mark(const char* what, cudaStream_t s) { if (n < kMax) { name[n] = what; cudaEventRecord(ev[n + 1], s); ++n; } }
+    void mark(const char* what, cudaStream_t s, int n_launches) { if (n < kMax) { name[n] = what; launches[n] = n_launches; cudaEventRecord(ev[n + 1], s); ++n; } }
 };
+#define ST_REPEAT(t) for (int r_ = 0, R_ = (t) ? (t)->repeat : 1; r_ < R_; ++r_)
+inline int st_repeats(const StageTimer* t) { return t ? t->repeat : 1; }
 int tc_forward(const TcPlan*, cudaStream_t s, StageTimer* t = nullptr);    // returns the number of kernels launched
 int tc_backward(const TcPlan*, cudaStream_t s, StageTimer* t = nullptr);
 

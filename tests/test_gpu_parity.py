@@ -94,6 +94,10 @@ def test_confusion_and_miou_bit_exact(C, h, w):
     m2 = st.st_agreement(ctx, 0, pred, lab, conf_h)                # host masks
     np.testing.assert_array_equal(conf_h, ref_conf)
     assert m2 == ref_m
+    m_dev = torch.zeros(1, dtype=torch.float64, device="cuda")     # device destination: written on the stream, no wait
+    assert st.st_agreement(ctx, 0, dev(pred), dev(lab), conf, miou_out=m_dev) is None
+    torch.cuda.current_stream().synchronize()
+    assert float(m_dev.item()) == ref_m
     st.st_destroy(ctx)
 
 
