@@ -302,3 +302,54 @@ def pack(head: Head) -> bytes:
 def agreement(labels: np.ndarray, pred: np.ndarray, C: int):
     conf, bad = confusion(labels, pred, C)
     return conf, miou(conf), bad
+
+
+# ----------------------------------------------------------------------------
+# Algorithm 1 as a whole: Train(student, frame, label)
+# ----------------------------------------------------------------------------
+@dataclass
+class TrainResult:
+    best_metric: float            # the metric returned with best_student
+    n_updates: int                # optimisation steps taken before the loop ended
+    best_iter: int                # number of updates behind best_student (0 = the incoming student)
+    metrics: List[float]          # metric of every prediction: metrics[i] after i updates
+    losses: List[float]           # loss of every prediction the loop computed a loss for (one per update)
+    masks: List[np.ndarray] = field(default_factory=list)   # the predictions themselves (kept on request)
+
+
+def train_key_frame(head: Head, feat: np.ndarray, labels: np.ndarray, threshold: float, max_updates: int,
+                    keep_masks: bool = False) -> TrainResult:
+    """Algorithm 1, Train(student, frame, label), in the paper's order and names.
+
+    The metric is the mean IoU of Section 3.2 between the student's mask and the pseudo-label.
+    On return ``head.theta`` holds best_student (Algorithm 3 continues with the returned student);
+    the momentum buffer is optimiser state, not part of the student, and keeps running.
+    """
+    C = head.n_classes
+    prediction = student_mask(head, feat)                               # prediction <- Forward(student, frame)
+    best_metric = agreement(labels, prediction, C)[1]                   # best_metric <- ComputeMetric(prediction, label)
+    best_student = head.theta.copy()                                    # best_student <- student
+    res = TrainResult(best_metric, 0, 0, [best_metric], [])
+    if keep_masks:
+        res.masks.append(prediction)
+    if best_metric < threshold:                                         # skip distillation when already good enough
+        for i in range(1, max_updates + 1):
+            # loss <- ComputeLoss(prediction, label); gradients <- PartialBackward(loss); student <- OptimStep(...)
+            # (the loss is a function of the same parameters that produced `prediction`)
+            loss, _ = distill_step(head, feat, labels)
+            res.losses.append(loss)
+            res.n_updates = i
+            prediction = student_mask(head, feat)                       # prediction <- Forward(student, frame)
+            metric = agreement(labels, prediction, C)[1]                # metric <- ComputeMetric(prediction, label)
+            res.metrics.append(metric)
+            if keep_masks:
+                res.masks.append(prediction)
+            if metric > best_metric:
+                best_metric = metric
+                best_student = head.theta.copy()
+                res.best_iter = i
+            if metric > threshold:
+                break
+    head.theta[:] = best_student
+    res.best_metric = best_metric
+    return res

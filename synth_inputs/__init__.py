@@ -92,6 +92,19 @@ def frozen_features(c_in: int, h: int, w: int, seed: int) -> np.ndarray:
     return x
 
 
+def label_informed_features(c_in: int, h: int, w: int, class_map: np.ndarray, up: int, seed: int,
+                            strength: float = 2.0) -> np.ndarray:
+    """ReLU(N(0,1)) features plus `strength` on channel c wherever the frame's class map shows class c at the
+    centre of the feature pixel: a stand-in for a frozen front part whose output says something about the
+    frame, so that the trainable part can actually improve its agreement with the labels (the plain noise
+    features cannot).  `class_map` is uint8 [h*up][w*up] with values below c_in."""
+    x = frozen_features(c_in, h, w, seed)
+    low = class_map[up // 2::up, up // 2::up][:h, :w].astype(np.int64)
+    yy, xx = np.meshgrid(np.arange(h), np.arange(w), indexing="ij")
+    x[low, yy, xx] += np.float32(strength)
+    return x
+
+
 # ----------------------------------------------------------------------------
 # teacher logits
 # ----------------------------------------------------------------------------
