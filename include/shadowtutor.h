@@ -125,6 +125,37 @@ ST_API st_status st_set_labels(st_ctx *ctx, int32_t stream, const uint8_t *label
 ST_API st_status st_distill_step(st_ctx *ctx, int32_t n_steps, float *loss_out, int64_t *conf_out);
 
 /*
+ * st_train_key_frame — Train(student, frame, label), the whole of Algorithm 1, on all S streams, each
+ * stream with its own control flow, decided on the device:
+ *     prediction <- Forward(student, frame); best_metric <- ComputeMetric(prediction, label); best_student <- student
+ *     if best_metric < THRESHOLD: for i = 1 .. MAX_UPDATES:
+ *         one iteration as in st_distill_step; prediction <- Forward; metric <- ComputeMetric(prediction, label)
+ *         if metric > best_metric: best_metric, best_student <- metric, student
+ *         if metric > THRESHOLD: break
+ * The metric is the mean IoU of Section 3.2 between the student's mask (arg-max of the upsampled logits) and the
+ * stored labels; THRESHOLD and MAX_UPDATES are the algorithm's two parameters (Section 4.1.3).
+ * On return the context's parameters are best_student (Algorithm 3: student, metric <- Train(...)); the momentum
+ * buffer is optimiser state and keeps its latest value.
+ *   threshold        THRESHOLD.
+ *   max_updates      MAX_UPDATES, 0..63.
+ *   n_updates_out    host or device, or NULL; int32 [S]: optimisation steps taken before the loop ended.
+ *   best_metric_out  host or device, or NULL; double [S]: best_metric.
+ *   metric_out       host or device, or NULL; double [S][max_updates + 1]: metric of the prediction after i updates;
+ *                    -1 for predictions the algorithm did not make (i > n_updates).
+ *   loss_out         host or device, or NULL; fp32 [S][max_updates + 1]: loss of the prediction after i updates,
+ *                    meaningful for i <= n_updates.
+ *   conf_out         host or device, or NULL; int64 [S][max_updates + 1][C][C]: confusion matrix of each prediction,
+ *                    meaningful for i <= n_updates.
+ * The work is enqueued on the context's stream (a replayed CUDA graph per (max_updates, threshold)); the call waits
+ * for the stream only if an output pointer is host memory.  Once a stream's loop has ended its later updates are
+ * no-ops; the kernels of the remaining iterations still run.
+ * ST_ERR_BAD_STATE if a stream has no features or labels yet; ST_ERR_INVALID_ARG for max_updates outside 0..63 or a
+ * NaN threshold.
+ */
+ST_API st_status st_train_key_frame(st_ctx *ctx, double threshold, int32_t max_updates, int32_t *n_updates_out,
+                                    double *best_metric_out, double *metric_out, float *loss_out, int64_t *conf_out);
+
+/*
  * st_pack_updated_params — UpdatedPart(student) (Algorithm 3; Table 4 sizes are fp32):
  * the current values of every trainable tensor of `stream`, fp32 little-endian, per layer in
  * forward order weight [Cout][Cin][kh][kw] then bias [Cout]; no header, no padding.

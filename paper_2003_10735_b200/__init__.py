@@ -37,7 +37,7 @@ EXPORTED = [
     "st_param_count", "st_init_head", "st_set_frozen_features", "st_teacher_labels", "st_set_labels",
     "st_distill_step", "st_pack_updated_params", "st_student_mask", "st_agreement", "st_read_tensor",
     "st_launch_count", "st_destroy", "st_last_error", "st_status_name", "st_profile_step",
-    "st_agreement_noalloc",
+    "st_agreement_noalloc", "st_train_key_frame",
 ]
 ST_NOALLOC_MAX_CLASSES = 64
 ST_MAX_STAGES = 12
@@ -84,6 +84,8 @@ def load_library() -> ctypes.CDLL:
     lib.st_set_labels.argtypes = [vp, i32, vp]
     lib.st_distill_step.restype = ctypes.c_int
     lib.st_distill_step.argtypes = [vp, i32, vp, vp]
+    lib.st_train_key_frame.restype = ctypes.c_int
+    lib.st_train_key_frame.argtypes = [vp, ctypes.c_double, i32, vp, vp, vp, vp, vp]
     lib.st_pack_updated_params.restype = ctypes.c_int
     lib.st_pack_updated_params.argtypes = [vp, i32, vp, ctypes.c_size_t, ctypes.POINTER(ctypes.c_size_t)]
     lib.st_student_mask.restype = ctypes.c_int
@@ -110,7 +112,7 @@ def load_library() -> ctypes.CDLL:
 
 
 # ---------------------------------------------------------------------------- marshalling
-_NP_OF = {"float32": np.float32, "uint8": np.uint8, "int64": np.int64}
+_NP_OF = {"float32": np.float32, "float64": np.float64, "uint8": np.uint8, "int32": np.int32, "int64": np.int64}
 
 
 def _ptr(buf, dtype: str, min_elems: int, what: str) -> Optional[int]:
@@ -194,6 +196,18 @@ def st_distill_step(ctx: _Ctx, n_steps: int, loss_out=None, conf_out=None) -> No
     _check(load_library().st_distill_step(ctx.handle, n_steps,
                                           _ptr(loss_out, "float32", ctx.S * max(n_steps, 0), "loss_out"),
                                           _ptr(conf_out, "int64", ctx.S * max(n_steps, 0) * ctx.C * ctx.C, "conf_out")), ctx)
+
+
+def st_train_key_frame(ctx: _Ctx, threshold: float, max_updates: int, n_updates=None, best_metric=None,
+                       metrics=None, losses=None, conf=None) -> None:
+    """Algorithm 1 (Train) on all streams.  Outputs (each optional; numpy array or tensor):
+    n_updates int32 [S], best_metric float64 [S], metrics float64 [S][max_updates+1],
+    losses float32 [S][max_updates+1], conf int64 [S][max_updates+1][C][C]."""
+    n = max(max_updates, 0) + 1
+    _check(load_library().st_train_key_frame(
+        ctx.handle, float(threshold), int(max_updates), _ptr(n_updates, "int32", ctx.S, "n_updates"),
+        _ptr(best_metric, "float64", ctx.S, "best_metric"), _ptr(metrics, "float64", ctx.S * n, "metrics"),
+        _ptr(losses, "float32", ctx.S * n, "losses"), _ptr(conf, "int64", ctx.S * n * ctx.C * ctx.C, "conf")), ctx)
 
 
 def st_pack_updated_params(ctx: _Ctx, stream: int, dst, dst_capacity: Optional[int] = None) -> int:

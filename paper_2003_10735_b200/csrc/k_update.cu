@@ -41,7 +41,9 @@ sgd_update_kernel(UpdateArgs a, int n_param_blocks, int64_t range_begin)
     pdl_launch_dependents();
     const int s = blockIdx.y;
     const int64_t base = (int64_t)s * a.n_params;
+    const bool skip = a.skip && a.skip[(int64_t)s * a.skip_stride];   // block-uniform
     if ((int)blockIdx.x < n_param_blocks) {
+        if (skip) return;
         const int col = threadIdx.x % kRow, g = threadIdx.x / kRow;
         int layer[E];
         bool is_weight[E], has_partials[E];
@@ -126,7 +128,7 @@ sgd_update_kernel(UpdateArgs a, int n_param_blocks, int64_t range_begin)
             }
 #pragma unroll
             for (int o = 16; o > 0; o >>= 1) g += __shfl_xor_sync(0xffffffffu, g, o);
-            if (lane == 0) apply_update(a, base + ly.b_off + item, g);
+            if (lane == 0 && !skip) apply_update(a, base + ly.b_off + item, g);
             return;
         }
         item -= ly.cout;
@@ -162,6 +164,7 @@ sgd_update_stream_kernel(UpdateArgs a, int L)
     pdl_launch_dependents();
     const LayerUpdate& ly = a.layer[L];
     const int s = blockIdx.y;
+    if (a.skip && a.skip[(int64_t)s * a.skip_stride]) return;
     const int64_t nw = (int64_t)ly.cout * ly.cin * ly.taps;
     const int64_t e = ((int64_t)blockIdx.x * 256 + threadIdx.x) * VEC;
     if (e >= nw) return;
@@ -255,10 +258,9 @@ void launch_refresh_shadow(const UpdateArgs& a, cudaStream_t s)
 
 // Mean IoU (Section 3.2): IoU_c = conf[c][c] / (row_c + col_c - conf[c][c]), averaged over the
 // classes present in the label (row_c > 0).  Integer counts, double arithmetic, fixed order.
-__global__ void miou_kernel(const unsigned long long* __restrict__ conf, int C, double* out)
+// Called by all 256 threads of a block; the value is returned to thread 0 only.
+__device__ __forceinline__ double block_miou(const unsigned long long* __restrict__ conf, int C, double* iou, int* present)
 {
-    __shared__ double iou[256];
-    __shared__ int present[256];
     const int c = threadIdx.x;
     double v = 0.0; int pr = 0;
     if (c < C) {
@@ -272,16 +274,90 @@ __global__ void miou_kernel(const unsigned long long* __restrict__ conf, int C, 
     }
     iou[c] = v; present[c] = pr;
     __syncthreads();
+    double m = 0.0;
     if (c == 0) {
         double sum = 0.0; int n = 0;
         for (int k = 0; k < C; ++k) { sum += iou[k]; n += present[k]; }
-        *out = n ? sum / n : 0.0;
+        m = n ? sum / n : 0.0;
     }
+    return m;
+}
+
+__global__ void __launch_bounds__(256) miou_kernel(const unsigned long long* __restrict__ conf, int C, double* out)
+{
+    __shared__ double iou[256];
+    __shared__ int present[256];
+    const double m = block_miou(conf, C, iou, present);
+    if (threadIdx.x == 0) *out = m;
+}
+
+// ---- Algorithm 1, the lines after "metric <- ComputeMetric(prediction, label)" ------------------------
+// One launch per prediction; blockIdx.y = stream.  Every block computes the stream's mean IoU from the confusion
+// matrix of the prediction (same arithmetic as miou_kernel), all blocks together copy the parameters into
+// best_student if the metric is a new best, and block 0 records the decisions:
+//   prediction 0 (the incoming student):  best_metric <- metric; the loop is entered iff best_metric < THRESHOLD
+//   prediction i > 0 (after i updates):   if metric > best_metric: best_metric, best_student <- metric, student;
+//                                         if metric > THRESHOLD: break;  the loop also ends at i = MAX_UPDATES.
+__global__ void __launch_bounds__(256) train_decide_kernel(TrainCtl t)
+{
+    __shared__ double iou[256];
+    __shared__ int present[256];
+    __shared__ double m_sh;
+    const int s = blockIdx.y, i = t.iter;
+    int* done = t.done + (int64_t)s * kCtlPitch;
+    double* best = t.best + (int64_t)s * kCtlPitch;
+    double* metric = t.metric + (int64_t)s * kCtlPitch;
+    const bool ended = i > 0 && done[i] != 0;                 // block-uniform
+    if (ended) {
+        if (blockIdx.x == 0 && threadIdx.x == 0) { done[i + 1] = 1; best[i + 1] = best[i]; metric[i] = -1.0; }
+        return;
+    }
+    const double m0 = block_miou(t.conf + (int64_t)s * t.conf_stream_stride, t.C, iou, present);
+    if (threadIdx.x == 0) m_sh = m0;
+    __syncthreads();
+    const double m = m_sh;
+    const double prev_best = i > 0 ? best[i] : 0.0;
+    const bool better = i == 0 || m > prev_best;
+    if (better) {
+        const float* src = t.theta + (int64_t)s * t.n_params;
+        float* dst = t.best_theta + (int64_t)s * t.n_params;
+        for (int64_t e = (int64_t)blockIdx.x * 256 + threadIdx.x; e < t.n_params; e += (int64_t)gridDim.x * 256) dst[e] = src[e];
+    }
+    if (blockIdx.x == 0 && threadIdx.x == 0) {
+        metric[i] = m;
+        best[i + 1] = better ? m : prev_best;
+        const bool stop = i == 0 ? !(m < t.threshold) : (m > t.threshold);
+        done[i + 1] = (stop || i >= t.max_updates) ? 1 : 0;
+        t.n_updates[s] = i;                                      // overwritten by the next prediction if the loop goes on
+        if (better) t.best_iter[s] = i;
+    }
+}
+
+__global__ void __launch_bounds__(256) train_commit_kernel(const float* __restrict__ best_theta, float* __restrict__ theta, int64_t n_params)
+{
+    const int64_t base = (int64_t)blockIdx.y * n_params;
+    for (int64_t e = (int64_t)blockIdx.x * 256 + threadIdx.x; e < n_params; e += (int64_t)gridDim.x * 256) theta[base + e] = best_theta[base + e];
 }
 
 void launch_miou(const unsigned long long* conf, int C, double* out, cudaStream_t s)
 {
     miou_kernel<<<1, 256, 0, s>>>(conf, C, out);
+}
+
+static unsigned copy_blocks(int64_t n_params)
+{
+    const int64_t b = (n_params + 256 * 8 - 1) / (256 * 8);      // about 8 values per thread
+    return (unsigned)(b < 1 ? 1 : (b > 592 ? 592 : b));
+}
+
+void launch_train_decide(const TrainCtl& t, cudaStream_t s)
+{
+    train_decide_kernel<<<dim3(copy_blocks(t.n_params), (unsigned)t.S), 256, 0, s>>>(t);
+}
+
+void launch_train_commit(const TrainCtl& t, float* theta, cudaStream_t s)
+{
+    train_commit_kernel<<<dim3(copy_blocks(t.n_params), (unsigned)t.S), 256, 0, s>>>(t.best_theta, theta, t.n_params);
 }
 
 // ---- pack / unpack ---------------------------------------------------------------------------------

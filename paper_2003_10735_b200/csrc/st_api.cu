@@ -8,6 +8,7 @@
 #include <cstdio>
 #include <cstring>
 #include <map>
+#include <tuple>
 #include <new>
 #include <string>
 #include <vector>
@@ -17,7 +18,12 @@ using namespace st;
 namespace {
 thread_local std::string g_init_error;
 
-struct GraphKey { int n_steps; bool conf; bool operator<(const GraphKey& o) const { return n_steps != o.n_steps ? n_steps < o.n_steps : conf < o.conf; } };
+// A replayable graph: n_steps plain iterations (train = false), or Train with MAX_UPDATES = n_steps and the
+// threshold whose bit pattern is `thr` (train = true).
+struct GraphKey {
+    int n_steps; bool conf; bool train; uint64_t thr;
+    bool operator<(const GraphKey& o) const { return std::tie(n_steps, conf, train, thr) < std::tie(o.n_steps, o.conf, o.train, o.thr); }
+};
 }  // namespace
 
 struct st_ctx {
@@ -48,6 +54,13 @@ struct st_ctx {
     int k3_has_map = 0;
     float* loss_buf = nullptr;              // [S][kMaxSteps]
     unsigned long long* conf_buf = nullptr; // [S][kMaxSteps][C][C], allocated on first use
+    // Train (Algorithm 1), allocated on first use
+    float* best_theta = nullptr;            // [S][n_params] best_student
+    int* ctl_done = nullptr;                // [S][kCtlPitch]
+    double* ctl_best = nullptr;             // [S][kCtlPitch]
+    double* ctl_metric = nullptr;           // [S][kCtlPitch]
+    int* ctl_n_updates = nullptr;           // [S]
+    int* ctl_best_iter = nullptr;           // [S]
     unsigned int* bad = nullptr;            // [3]: labels >= C met by a step / by st_agreement; [2] = first device wait that gave up
     uint8_t* mask_tmp = nullptr;            // [P]
     uint8_t* mask_tmp2 = nullptr;           // [P]
@@ -149,7 +162,7 @@ st_status check_launch(st_ctx* ctx, const char* what)
     return ST_OK;
 }
 
-UpdateArgs make_update_args(st_ctx* c, int slot)
+UpdateArgs make_update_args(st_ctx* c, int slot, const int* skip = nullptr, int64_t skip_stride = 0)
 {
     UpdateArgs u;
     memset(&u, 0, sizeof u);
@@ -180,6 +193,7 @@ UpdateArgs make_update_args(st_ctx* c, int slot)
     u.loss_part = c->loss_part; u.n_loss_part = c->n_k3_blocks;
     u.loss_buf = c->loss_buf; u.loss_slot = slot;
     u.inv_P = 1.0 / (double)c->P;
+    u.skip = skip; u.skip_stride = skip_stride;
     return u;
 }
 
@@ -228,19 +242,22 @@ UpsampleCeArgs k3_args(st_ctx* c, bool fp32_grad, bool bf16_grad, unsigned long 
     return k3;
 }
 
-st_status enqueue_step(st_ctx* c, int slot, bool want_conf, StageTimer* t = nullptr)
+// ComputeLoss and the first half of PartialBackward: loss partials, logit gradient, optionally the confusion matrix
+// of this prediction.
+st_status enqueue_loss(st_ctx* c, unsigned long long* conf, StageTimer* t = nullptr)
 {
     cudaStream_t s = c->stream;
-    st_status st = enqueue_forward(c, t);
-    if (st != ST_OK) return st;
-
-    const UpsampleCeArgs k3 = k3_args(c, !c->bf16_mode, c->bf16_mode, want_conf ? c->conf_buf + (int64_t)slot * c->C * c->C : nullptr);
+    const UpsampleCeArgs k3 = k3_args(c, !c->bf16_mode, c->bf16_mode, conf);
     ST_REPEAT(t) launch_upsample_ce(k3, &c->k3_map, s);
     if (t) t->mark("upsample_ce", s, st_repeats(t));
     c->launches += st_repeats(t);
-    st = check_launch(c, "upsample + cross-entropy");
-    if (st != ST_OK) return st;
+    return check_launch(c, "upsample + cross-entropy");
+}
 
+// The rest of PartialBackward: gradients of the head's tensors (as split-K partial sums with bf16 GEMMs).
+st_status enqueue_backward(st_ctx* c, StageTimer* t = nullptr)
+{
+    cudaStream_t s = c->stream;
     if (c->bf16_mode) {
         c->launches += tc_backward(c->plan, s, t);
     } else if (c->Ch == 0) {
@@ -260,12 +277,24 @@ st_status enqueue_step(st_ctx* c, int slot, bool want_conf, StageTimer* t = null
         if (t) t->mark("backward_f32", s, 4);
         c->launches += 4;
     }
-    st = check_launch(c, "head backward");
-    if (st != ST_OK) return st;
+    return check_launch(c, "head backward");
+}
 
-    c->launches += launch_sgd_update(make_update_args(c, slot), s);
-    if (t) t->mark("sgd_update", s, 1);
+// OptimStep, and the loss of this prediction into loss_buf[slot].  `skip`: per-stream flags (see UpdateArgs).
+st_status enqueue_update(st_ctx* c, int slot, const int* skip, int64_t skip_stride, StageTimer* t = nullptr)
+{
+    c->launches += launch_sgd_update(make_update_args(c, slot, skip, skip_stride), c->stream);
+    if (t) t->mark("sgd_update", c->stream, 1);
     return check_launch(c, "sgd update");
+}
+
+st_status enqueue_step(st_ctx* c, int slot, bool want_conf, StageTimer* t = nullptr)
+{
+    st_status st = enqueue_forward(c, t);
+    if (st == ST_OK) st = enqueue_loss(c, want_conf ? c->conf_buf + (int64_t)slot * c->C * c->C : nullptr, t);
+    if (st == ST_OK) st = enqueue_backward(c, t);
+    if (st == ST_OK) st = enqueue_update(c, slot, nullptr, 0, t);
+    return st;
 }
 
 // One 32-byte device-to-host copy and one wait: the mean IoU of the last st_agreement and the error words.
@@ -541,7 +570,7 @@ st_status st_distill_step(st_ctx* ctx, int32_t n_steps, float* loss_out, int64_t
 
     st_status st = ST_OK;
     if (ctx->use_graphs) {
-        GraphKey key{n_steps, want_conf};
+        GraphKey key{n_steps, want_conf, false, 0};
         auto it = ctx->graphs.find(key);
         if (it == ctx->graphs.end()) {
             cudaGraph_t graph = nullptr;
@@ -573,6 +602,127 @@ st_status st_distill_step(st_ctx* ctx, int32_t n_steps, float* loss_out, int64_t
     if (conf_out)
         ST_CUDA(ctx, cudaMemcpy2DAsync(conf_out, (size_t)n_steps * cc * 8, ctx->conf_buf, (size_t)kMaxSteps * cc * 8,
                                        (size_t)n_steps * cc * 8, ctx->S, cudaMemcpyDefault, ctx->stream));
+    return ST_OK;
+}
+
+namespace {
+TrainCtl train_ctl(st_ctx* c, int iter, int max_updates, double threshold)
+{
+    TrainCtl t;
+    t.conf = c->conf_buf + (int64_t)iter * c->C * c->C;
+    t.conf_stream_stride = (int64_t)kMaxSteps * c->C * c->C;
+    t.C = c->C; t.iter = iter; t.max_updates = max_updates; t.threshold = threshold;
+    t.done = c->ctl_done; t.best = c->ctl_best; t.metric = c->ctl_metric;
+    t.n_updates = c->ctl_n_updates; t.best_iter = c->ctl_best_iter;
+    t.theta = c->theta; t.best_theta = c->best_theta; t.n_params = c->n_params; t.S = c->S;
+    return t;
+}
+
+// Train of Algorithm 1 for all streams: one prediction per pass (forward, loss + gradient + confusion, decision),
+// then backward and the update, which is a no-op for streams whose loop has ended.
+st_status enqueue_train(st_ctx* c, int max_updates, double threshold)
+{
+    st_status st = ST_OK;
+    for (int i = 0; i <= max_updates && st == ST_OK; ++i) {
+        st = enqueue_forward(c);                                                          // prediction <- Forward(student, frame)
+        if (st == ST_OK) st = enqueue_loss(c, c->conf_buf + (int64_t)i * c->C * c->C);   // loss, gradient, confusion of it
+        if (st != ST_OK) break;
+        launch_train_decide(train_ctl(c, i, max_updates, threshold), c->stream);         // metric, best_student, break
+        c->launches += 1;
+        st = check_launch(c, "train control");
+        if (st == ST_OK && i < max_updates) st = enqueue_backward(c);
+        // after the last prediction every loop has ended: the launch only finalises that prediction's loss
+        if (st == ST_OK) st = enqueue_update(c, i, c->ctl_done + i + 1, kCtlPitch);
+    }
+    if (st != ST_OK) return st;
+    launch_train_commit(train_ctl(c, 0, max_updates, threshold), c->theta, c->stream);    // student <- best_student
+    launch_refresh_shadow(make_update_args(c, 0), c->stream);
+    c->launches += 2;
+    return check_launch(c, "train commit");
+}
+}  // namespace
+
+st_status st_train_key_frame(st_ctx* ctx, double threshold, int32_t max_updates, int32_t* n_updates_out,
+                             double* best_metric_out, double* metric_out, float* loss_out, int64_t* conf_out)
+{
+    if (!ctx) return ST_ERR_INVALID_ARG;
+    if (max_updates < 0 || max_updates > kMaxSteps - 1)
+        return fail(ctx, ST_ERR_INVALID_ARG, "st_train_key_frame: max_updates %d outside 0..%d", max_updates, kMaxSteps - 1);
+    if (!(threshold == threshold))
+        return fail(ctx, ST_ERR_INVALID_ARG, "st_train_key_frame: threshold is not a number");
+    for (int s = 0; s < ctx->S; ++s)
+        if (!ctx->has_feat[s] || !ctx->has_labels[s])
+            return fail(ctx, ST_ERR_BAD_STATE, "st_train_key_frame: stream %d has no %s yet", s,
+                        ctx->has_feat[s] ? "labels" : "frozen features");
+    const size_t cc = (size_t)ctx->C * ctx->C;
+    cudaError_t e = cudaSuccess;
+    if (!ctx->conf_buf) e = dev_alloc(ctx, &ctx->conf_buf, (size_t)ctx->S * kMaxSteps * cc);
+    if (e == cudaSuccess && !ctx->best_theta) {
+        e = dev_alloc(ctx, &ctx->best_theta, (size_t)ctx->S * ctx->n_params);
+        if (e == cudaSuccess) e = dev_alloc(ctx, &ctx->ctl_done, (size_t)ctx->S * kCtlPitch);
+        if (e == cudaSuccess) e = dev_alloc(ctx, &ctx->ctl_best, (size_t)ctx->S * kCtlPitch);
+        if (e == cudaSuccess) e = dev_alloc(ctx, &ctx->ctl_metric, (size_t)ctx->S * kCtlPitch);
+        if (e == cudaSuccess) e = dev_alloc(ctx, &ctx->ctl_n_updates, (size_t)ctx->S);
+        if (e == cudaSuccess) e = dev_alloc(ctx, &ctx->ctl_best_iter, (size_t)ctx->S);
+    }
+    if (e != cudaSuccess) return fail(ctx, ST_ERR_OOM, "st_train_key_frame: %s", cudaGetErrorString(e));
+    ST_CUDA(ctx, cudaMemsetAsync(ctx->conf_buf, 0, (size_t)ctx->S * kMaxSteps * cc * sizeof(unsigned long long), ctx->stream));
+
+    st_status st = ST_OK;
+    if (ctx->use_graphs) {
+        uint64_t thr_bits;
+        memcpy(&thr_bits, &threshold, sizeof thr_bits);
+        GraphKey key{max_updates, true, true, thr_bits};
+        auto it = ctx->graphs.find(key);
+        if (it == ctx->graphs.end()) {
+            cudaGraph_t graph = nullptr;
+            const int64_t before = ctx->launches;
+            ST_CUDA(ctx, cudaStreamBeginCapture(ctx->stream, cudaStreamCaptureModeThreadLocal));
+            st = enqueue_train(ctx, max_updates, threshold);
+            e = cudaStreamEndCapture(ctx->stream, &graph);
+            const int64_t n_launches = ctx->launches - before;
+            ctx->launches = before;
+            if (st != ST_OK) { if (graph) cudaGraphDestroy(graph); return st; }
+            if (e != cudaSuccess) return fail(ctx, ST_ERR_CUDA, "st_train_key_frame: graph capture: %s", cudaGetErrorString(e));
+            cudaGraphExec_t exec = nullptr;
+            e = cudaGraphInstantiate(&exec, graph, 0);
+            cudaGraphDestroy(graph);
+            if (e != cudaSuccess) return fail(ctx, ST_ERR_CUDA, "st_train_key_frame: graph instantiate: %s", cudaGetErrorString(e));
+            it = ctx->graphs.emplace(key, st_ctx::StepGraph{exec, n_launches}).first;
+        }
+        ctx->launches += it->second.n_launches;
+        ST_CUDA(ctx, cudaGraphLaunch(it->second.exec, ctx->stream));
+    } else {
+        st = enqueue_train(ctx, max_updates, threshold);
+        if (st != ST_OK) return st;
+    }
+    const int n_pred = max_updates + 1;
+    bool host_out = false;
+    if (n_updates_out) {
+        ST_CUDA(ctx, cudaMemcpyAsync(n_updates_out, ctx->ctl_n_updates, (size_t)ctx->S * sizeof(int), cudaMemcpyDefault, ctx->stream));
+        host_out |= !is_device_ptr(n_updates_out);
+    }
+    if (best_metric_out) {     // best_metric after the last prediction was judged
+        ST_CUDA(ctx, cudaMemcpy2DAsync(best_metric_out, sizeof(double), ctx->ctl_best + n_pred, kCtlPitch * sizeof(double),
+                                       sizeof(double), ctx->S, cudaMemcpyDefault, ctx->stream));
+        host_out |= !is_device_ptr(best_metric_out);
+    }
+    if (metric_out) {
+        ST_CUDA(ctx, cudaMemcpy2DAsync(metric_out, (size_t)n_pred * sizeof(double), ctx->ctl_metric, kCtlPitch * sizeof(double),
+                                       (size_t)n_pred * sizeof(double), ctx->S, cudaMemcpyDefault, ctx->stream));
+        host_out |= !is_device_ptr(metric_out);
+    }
+    if (loss_out) {
+        ST_CUDA(ctx, cudaMemcpy2DAsync(loss_out, (size_t)n_pred * sizeof(float), ctx->loss_buf, kMaxSteps * sizeof(float),
+                                       (size_t)n_pred * sizeof(float), ctx->S, cudaMemcpyDefault, ctx->stream));
+        host_out |= !is_device_ptr(loss_out);
+    }
+    if (conf_out) {
+        ST_CUDA(ctx, cudaMemcpy2DAsync(conf_out, (size_t)n_pred * cc * 8, ctx->conf_buf, (size_t)kMaxSteps * cc * 8,
+                                       (size_t)n_pred * cc * 8, ctx->S, cudaMemcpyDefault, ctx->stream));
+        host_out |= !is_device_ptr(conf_out);
+    }
+    if (host_out) ST_CUDA(ctx, cudaStreamSynchronize(ctx->stream));
     return ST_OK;
 }
 

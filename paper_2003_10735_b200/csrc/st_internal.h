@@ -144,12 +144,40 @@ struct UpdateArgs {
     float* loss_buf;         // [S][kMaxSteps]
     int loss_slot;           // slot of loss_buf written by this step
     double inv_P;
+    const int* skip;         // nullptr, or one flag per stream (skip[s * skip_stride]): non-zero = leave the stream's
+    int64_t skip_stride;     //   parameters and momentum untouched (the loss is still finalised)
 };
 int launch_sgd_update(const UpdateArgs& a, cudaStream_t s);   // returns the number of kernels launched
 // refresh the bf16 shadows from the fp32 master parameters (after init)
 void launch_refresh_shadow(const UpdateArgs& a, cudaStream_t s);
 // mean IoU (Section 3.2) from an int64 confusion matrix, in double, one block
 void launch_miou(const unsigned long long* conf, int C, double* out, cudaStream_t s);
+
+// ---- control of Algorithm 1 (Train): judged once per prediction, per stream ----------------------
+// History arrays are indexed by the number of updates behind a prediction, so that a launch reads only what
+// earlier launches wrote: done[s][i] = the loop of stream s had ended before prediction i was made,
+// best[s][i] = best_metric before prediction i was judged.
+constexpr int kCtlPitch = kMaxSteps + 2;
+struct TrainCtl {
+    const unsigned long long* conf;   // confusion matrix of this prediction, stream 0
+    int64_t conf_stream_stride;       // elements between the matrices of consecutive streams
+    int C;
+    int iter;                         // i: number of updates behind this prediction
+    int max_updates;                  // MAX_UPDATES
+    double threshold;                 // THRESHOLD
+    int* done;                        // [S][kCtlPitch]
+    double* best;                     // [S][kCtlPitch]
+    double* metric;                   // [S][kCtlPitch]  metric of prediction i; -1 where the loop had ended before
+    int* n_updates;                   // [S] updates taken when the loop ended
+    int* best_iter;                   // [S] updates behind best_student
+    const float* theta;               // [S][n_params]
+    float* best_theta;                // [S][n_params]  best_student
+    int64_t n_params;
+    int S;
+};
+void launch_train_decide(const TrainCtl& t, cudaStream_t s);
+// student <- best_student (the caller refreshes the bf16 copies afterwards)
+void launch_train_commit(const TrainCtl& t, float* theta, cudaStream_t s);
 
 // ---- K7: packed parameter buffer <-> internal order ---------------------------------------------
 // packed: per layer weight [cout][cin][kh][kw] then bias; internal: weight [tap][cout][cin] then bias.
