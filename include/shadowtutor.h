@@ -147,8 +147,9 @@ ST_API st_status st_distill_step(st_ctx *ctx, int32_t n_steps, float *loss_out, 
  *   conf_out         host or device, or NULL; int64 [S][max_updates + 1][C][C]: confusion matrix of each prediction,
  *                    meaningful for i <= n_updates.
  * The work is enqueued on the context's stream (a replayed CUDA graph per (max_updates, threshold)); the call waits
- * for the stream only if an output pointer is host memory.  Once a stream's loop has ended its later updates are
- * no-ops; the kernels of the remaining iterations still run.
+ * for the stream only if an output pointer is host memory.  The launches of all max_updates iterations are always
+ * enqueued; once a stream's loop has ended, the blocks of its later kernels return at once (with gemm_precision 0
+ * the fp32 convolutions still run and only the update is suppressed).
  * ST_ERR_BAD_STATE if a stream has no features or labels yet; ST_ERR_INVALID_ARG for max_updates outside 0..63 or a
  * NaN threshold.
  */

@@ -48,8 +48,9 @@ __global__ void __launch_bounds__(kThreadsTc)
 tc_fwd1x1_kernel(const __grid_constant__ CUtensorMap tmA,   // {K, p, S}  box {64, 128, 1}
                  const __grid_constant__ CUtensorMap tmB,   // {K, 32, S} box {64, 32, 1}
                  const float* __restrict__ theta, int64_t n_params, int64_t b_off,
-                 float* __restrict__ z, int C, int p, int kblocks, unsigned int* err)
+                 float* __restrict__ z, int C, int p, int kblocks, unsigned int* err, const int* __restrict__ skip, int64_t skip_stride)
 {
+    if (skip && skip[(int64_t)blockIdx.y * skip_stride]) return;   // this stream's training loop has ended (block-uniform)
     extern __shared__ uint8_t smem_raw[];
     uint8_t* smem = align_smem(smem_raw);
     const uint32_t a_base = smem_u32(smem);
@@ -126,8 +127,9 @@ __global__ void __launch_bounds__(kThreadsTc)
 tc_wgrad1x1_kernel(const __grid_constant__ CUtensorMap tmA,   // {K, p, S}      box {64, 64, 1}
                    const __grid_constant__ CUtensorMap tmB,   // {p, 32, S}     box {64, 32, 1}
                    float* __restrict__ partials,              // [S][n_split][32][K]
-                   int K, int n_chunks, int chunks_per_block, int tmem_cols, unsigned int* err)
+                   int K, int n_chunks, int chunks_per_block, int tmem_cols, unsigned int* err, const int* __restrict__ skip, int64_t skip_stride)
 {
+    if (skip && skip[(int64_t)blockIdx.y * skip_stride]) return;   // this stream's training loop has ended (block-uniform)
     extern __shared__ uint8_t smem_raw[];
     uint8_t* smem = align_smem(smem_raw);
     const int m_tiles = (K + kTileM - 1) / kTileM;   // accumulators (128 channels each)
@@ -230,7 +232,7 @@ tc_fwd3x3_kernel(const __grid_constant__ CUtensorMap tmA,   // {Cin, w, h, S}   
                  const float* __restrict__ theta, int64_t n_params, int64_t b_off,
                  bf16* __restrict__ hidden,                  // [S][p][Ch]
                  uint32_t* __restrict__ relu_bits,           // [S][p][Ch/32]: bit k of word j = hidden[32j + k] > 0
-                 int Cin, int Ch, int h, int w, int n_tiles_total, int acc_cols, unsigned int* err)
+                 int Cin, int Ch, int h, int w, int n_tiles_total, int acc_cols, unsigned int* err, const int* __restrict__ skip, int64_t skip_stride)
 {
     extern __shared__ uint8_t smem_raw[];
     uint8_t* smem = align_smem(smem_raw);
@@ -262,6 +264,7 @@ tc_fwd3x3_kernel(const __grid_constant__ CUtensorMap tmA,   // {Cin, w, h, S}   
         int g = 0;
         for (int t = blockIdx.x; t < n_tiles_total && ok; t += gridDim.x) {
             const int s = t / tiles_per_stream, tt = t % tiles_per_stream;
+            if (skip && skip[(int64_t)s * skip_stride]) continue;     // all three roles leave out the same tiles
             const int x0 = (tt % tiles_x) * kTileW, y0 = (tt / tiles_x) * kTileH;
             for (int it = 0; it < n_iter; ++it, ++g) {
                 const int st = g % STAGES, tap = it / kblocks, kb = it % kblocks;
@@ -277,7 +280,8 @@ tc_fwd3x3_kernel(const __grid_constant__ CUtensorMap tmA,   // {Cin, w, h, S}   
         // ---- MMA issuer
         const uint32_t idesc = instr_desc(kTileM, Ch, 0, 0);
         int g = 0, j = 0;
-        for (int t = blockIdx.x; t < n_tiles_total && ok; t += gridDim.x, ++j) {
+        for (int t = blockIdx.x; t < n_tiles_total && ok; t += gridDim.x) {
+            if (skip && skip[(int64_t)(t / tiles_per_stream) * skip_stride]) continue;
             const int buf = j & 1;
             if (j >= 2) ok = mbar_wait(smem_u32(&acc_empty[buf]), ((j >> 1) - 1) & 1, err, kWaitEmpty);
             if (!ok) break;
@@ -295,14 +299,16 @@ tc_fwd3x3_kernel(const __grid_constant__ CUtensorMap tmA,   // {Cin, w, h, S}   
                 umma_commit(smem_u32(&empty[st]));
             }
             if (ok) umma_commit(smem_u32(&acc_full[buf]));
+            ++j;                                                       // j counts the tiles this block works on
         }
     } else if (warp >= 2) {
         // ---- epilogue warps: TMEM lanes 32*(warp % 4) .. +31 = pixel rows of the tile
         const int q = warp & 3, row = q * 32 + lane;
         int j = 0;
-        for (int t = blockIdx.x; t < n_tiles_total && ok; t += gridDim.x, ++j) {
-            const int buf = j & 1;
+        for (int t = blockIdx.x; t < n_tiles_total && ok; t += gridDim.x) {
             const int s = t / tiles_per_stream, tt = t % tiles_per_stream;
+            if (skip && skip[(int64_t)s * skip_stride]) continue;
+            const int buf = j & 1;
             const int x = (tt % tiles_x) * kTileW + row % kTileW, y = (tt / tiles_x) * kTileH + row / kTileW;
             ok = mbar_wait(smem_u32(&acc_full[buf]), (j >> 1) & 1, err, kWaitDone);
             if (!ok) break;
@@ -334,6 +340,7 @@ tc_fwd3x3_kernel(const __grid_constant__ CUtensorMap tmA,   // {Cin, w, h, S}   
             tc_fence_before_sync();
             __syncwarp();
             if (lane == 0) mbar_arrive(smem_u32(&acc_empty[buf]));     // this warp's quarter of the accumulator is free
+            ++j;
         }
     }
     if (!ok) drain_after_error();
@@ -354,8 +361,9 @@ tc_wgrad3x3_kernel(const __grid_constant__ CUtensorMap tmA,   // X   {Cin, w, h,
                    const __grid_constant__ CUtensorMap tmB,   // dHd {Ch,  w, h, S} box {64, 32, 2, 1}
                    float* __restrict__ partials,              // [S][n_split][9][Ch][Cin]
                    int Cin, int Ch, int h, int w, int n_chunks, int chunks_per_block, int n_split,
-                   int tmem_cols, unsigned int* err)
+                   int tmem_cols, unsigned int* err, const int* __restrict__ skip, int64_t skip_stride)
 {
+    if (skip && skip[(int64_t)blockIdx.y * skip_stride]) return;   // this stream's training loop has ended (block-uniform)
     extern __shared__ uint8_t smem_raw[];
     uint8_t* smem = align_smem(smem_raw);
     const uint32_t base = smem_u32(smem);
@@ -454,8 +462,9 @@ tc_dgrad_kernel(const __grid_constant__ CUtensorMap tmA,   // dz  {p, 32, S}  bo
                 const uint32_t* __restrict__ relu_bits,     // [S][p][Ch/32]
                 bf16* __restrict__ dhidden,                 // [S][p][Ch]
                 float* __restrict__ b1_partials,            // [S][n_blocks][Ch]
-                int Ch, int p, int tmem_cols, unsigned int* err)
+                int Ch, int p, int tmem_cols, unsigned int* err, const int* __restrict__ skip, int64_t skip_stride)
 {
+    if (skip && skip[(int64_t)blockIdx.y * skip_stride]) return;   // this stream's training loop has ended (block-uniform)
     extern __shared__ uint8_t smem_raw[];
     uint8_t* smem = align_smem(smem_raw);
     const uint32_t a_base = smem_u32(smem);
@@ -733,7 +742,7 @@ TcPlan* tc_plan_create(const TcBuffers& b, char* err, size_t err_len)
 
 void tc_plan_destroy(TcPlan* P) { delete P; }
 
-int tc_forward(const TcPlan* P, cudaStream_t s, StageTimer* t)
+int tc_forward(const TcPlan* P, cudaStream_t s, StageTimer* t, const int* skip, int64_t skip_stride)
 {
     const TcBuffers& b = P->b;
     int n = 0;
@@ -742,33 +751,33 @@ int tc_forward(const TcPlan* P, cudaStream_t s, StageTimer* t)
         const int total = tiles * b.S;
         ST_REPEAT(t) launch_chain(tc_fwd3x3_kernel<4>, dim3(total < P->n_sms ? total : P->n_sms), dim3(kFwd3Threads), P->smem_fwd3, s,
             P->x_fwd3, P->w1_map, b.theta, b.n_params, b.b1_off, b.hidden, b.relu_bits, b.c_in, b.c_hidden, b.h, b.w,
-            total, pow2_cols(b.c_hidden), b.err);
+            total, pow2_cols(b.c_hidden), b.err, skip, skip_stride);
         if (t) t->mark("tc_fwd3x3", s, st_repeats(t));
         n += st_repeats(t);
     }
     const int tiles1 = (P->p + kTileM - 1) / kTileM;
     ST_REPEAT(t) launch_chain(tc_fwd1x1_kernel, dim3(tiles1, b.S), dim3(kThreadsTc), P->smem_fwd1, s,
-        P->act_fwd, P->w2_map, b.theta, b.n_params, b.b2_off, b.z, b.C, P->p, P->c_last / kBlockK, b.err);
+        P->act_fwd, P->w2_map, b.theta, b.n_params, b.b2_off, b.z, b.C, P->p, P->c_last / kBlockK, b.err, skip, skip_stride);
     if (t) t->mark("tc_fwd1x1", s, st_repeats(t));
     return n + st_repeats(t);
 }
 
-int tc_backward(const TcPlan* P, cudaStream_t s, StageTimer* t)
+int tc_backward(const TcPlan* P, cudaStream_t s, StageTimer* t, const int* skip, int64_t skip_stride)
 {
     const TcBuffers& b = P->b;
     int n = 0;
     ST_REPEAT(t) launch_chain(tc_wgrad1x1_kernel<3>, dim3(P->split2, b.S), dim3(kThreadsTc), P->smem_wg1, s,
-        P->act_wg, P->dz_map, b.w2_partials, P->c_last, P->chunks2, P->per2, P->cols2, b.err);
+        P->act_wg, P->dz_map, b.w2_partials, P->c_last, P->chunks2, P->per2, P->cols2, b.err, skip, skip_stride);
     if (t) t->mark("tc_wgrad1x1", s, st_repeats(t));
     n += st_repeats(t);
     if (b.c_hidden) {
         const int blocks = tc_b1_partials(b.h, b.w);
         ST_REPEAT(t) launch_chain(tc_dgrad_kernel, dim3(blocks, b.S), dim3(kThreadsTc), P->smem_dgrad, s,
-            P->dz_map, P->w2_map, b.relu_bits, b.dhidden, b.b1_partials, b.c_hidden, P->p, pow2_cols(b.c_hidden), b.err);
+            P->dz_map, P->w2_map, b.relu_bits, b.dhidden, b.b1_partials, b.c_hidden, P->p, pow2_cols(b.c_hidden), b.err, skip, skip_stride);
         if (t) t->mark("tc_dgrad", s, st_repeats(t));
         ST_REPEAT(t) launch_chain(tc_wgrad3x3_kernel<3>, dim3(9 * P->split1, b.S), dim3(kThreadsTc), P->smem_wg3, s,
             P->x_wg3, P->dh_wg3, b.w1_partials, b.c_in, b.c_hidden, b.h, b.w, P->chunks1, P->per1, P->split1,
-            P->cols1, b.err);
+            P->cols1, b.err, skip, skip_stride);
         if (t) t->mark("tc_wgrad3x3", s, st_repeats(t));
         n += 2 * st_repeats(t);
     }

@@ -68,6 +68,7 @@ upsample_ce_kernel(UpsampleCeArgs a, int chunk)
     const int tid = threadIdx.x;
     pdl_wait();
     pdl_launch_dependents();
+    if (a.skip && a.skip[(int64_t)s * a.skip_stride]) return;     // this stream's training loop has ended (block-uniform)
 
     // ---- z tile with replicated borders
     for (int idx = tid; idx < C * ZT_H * ZT_W; idx += kThreads) {

@@ -172,6 +172,7 @@ upsample_ce_rows_kernel(UpsampleCeArgs a, const __grid_constant__ CUtensorMap z_
                                                 //                  (their exponentials are 0)
     int* corr = (int*)(zt + CB * TZ);           // [C][TZ_H][36]    -64 * (adjoint of onehot)
     float2* acc = (float2*)(corr + C * TZ);     // [R_WARPS][C][32] (x, y): the cell's pull on its upper / lower node row
+    unsigned int* hist = (unsigned int*)(acc + R_WARPS * C * 32);   // [C][C] (CONF): the block's share of the confusion matrix
     __shared__ float red[R_WARPS], red_m[R_WARPS];
     __shared__ __align__(8) uint64_t tile_bar;
 
@@ -185,6 +186,7 @@ upsample_ce_rows_kernel(UpsampleCeArgs a, const __grid_constant__ CUtensorMap z_
     const uint8_t* labels = a.labels + (int64_t)s * H * W;
     const int tid = threadIdx.x, wi = tid >> 5, l = tid & 31;
     pdl_wait();                  // the logits come from the previous kernel of the step
+    if (a.skip && a.skip[(int64_t)s * a.skip_stride]) return;     // this stream's training loop has ended (block-uniform)
     pdl_launch_dependents();
 
     // ---- tile: node rows y0-1 .. y0+RN_Y, node columns xa .. xa+35 where xa = (x0-1) rounded down to a
@@ -243,6 +245,7 @@ upsample_ce_rows_kernel(UpsampleCeArgs a, const __grid_constant__ CUtensorMap z_
             const uint32_t bar = tc::smem_u32(&tile_bar);
             for (int e = tid; e < (CB - C) * kQuads; e += R_THREADS) zt4[C * kQuads + e] = make_float4(-1e30f, -1e30f, -1e30f, -1e30f);
             for (int e = tid; e < C * TZ / 4; e += R_THREADS) reinterpret_cast<int4*>(corr)[e] = make_int4(0, 0, 0, 0);
+            if (CONF) for (int e = tid; e < C * C; e += R_THREADS) hist[e] = 0;
             __syncthreads();                                   // the barrier's initialisation is visible to every waiter
             bool ok = false;
             for (uint32_t it = 0; it < 2 * tc::kSpinLimit && !ok; ++it) ok = tc::mbar_try_wait(bar, 0);
@@ -310,6 +313,7 @@ upsample_ce_rows_kernel(UpsampleCeArgs a, const __grid_constant__ CUtensorMap z_
                 if (g < kPlanes && c < CB) zt4[c * kQuads + q] = v[it];
             }
             for (int e = tid; e < C * TZ / 4; e += R_THREADS) reinterpret_cast<int4*>(corr)[e] = make_int4(0, 0, 0, 0);
+            if (CONF) for (int e = tid; e < C * C; e += R_THREADS) hist[e] = 0;
         }
     }
 #pragma unroll
@@ -357,7 +361,7 @@ upsample_ce_rows_kernel(UpsampleCeArgs a, const __grid_constant__ CUtensorMap z_
                     const float vl = fmaf(ly, q[TZ_W] - q[0], q[0]), vr = fmaf(ly, q[TZ_W + 1] - q[1], q[1]);
                     const float ul = fmaf(fmaf((2 * k + 1) * 0.125f, vr - vl, vl), kLog2e, -rc.M) - sk[k];
                     loss += (__log2f(Zs[k]) - ul) * kLn2;
-                    if (CONF) atomicAdd(a.conf + (int64_t)s * a.conf_stream_stride + lab[k] * C + arg[k], 1ull);
+                    if (CONF) atomicAdd(&hist[lab[k] * C + arg[k]], 1u);
                 }
             }
             const float fr = (2 * k + 1) * 0.125f;
@@ -428,7 +432,7 @@ upsample_ce_rows_kernel(UpsampleCeArgs a, const __grid_constant__ CUtensorMap z_
 #pragma unroll
                     for (int k = 0; k < 4; ++k)
                         if (own_cell && ((rem[r] >> (8 * k)) & 1u))
-                            atomicAdd(a.conf + (int64_t)s * a.conf_stream_stride + ((labw[r] >> (8 * k)) & 0xffu) * C + ar4[k], 1ull);
+                            atomicAdd(&hist[((labw[r] >> (8 * k)) & 0xffu) * C + ar4[k]], 1u);
                 }
             }
             float lz = 0.f;
@@ -543,6 +547,10 @@ upsample_ce_rows_kernel(UpsampleCeArgs a, const __grid_constant__ CUtensorMap z_
     if (l == 0) red[wi] = loss;
     if (n_bad) atomicAdd(a.bad, n_bad);
     __syncthreads();
+    if (CONF) {                                  // one global update per non-empty counter of the block
+        for (int e = tid; e < C * C; e += R_THREADS)
+            if (hist[e]) atomicAdd(a.conf + (int64_t)s * a.conf_stream_stride + e, (unsigned long long)hist[e]);
+    }
 
     // ---- node row y0-1+wi (warps 1..RN_Y): own upper part + lower part of the warp above + onehot part.
     // All shared-memory reads of the 21 classes are issued before the first store.
@@ -613,25 +621,25 @@ upsample_ce_rows_kernel(UpsampleCeArgs a, const __grid_constant__ CUtensorMap z_
 }
 
 template <int CB>
-size_t rows_smem_bytes(int C)
+size_t rows_smem_bytes(int C, bool conf)
 {
-    return ((size_t)CB * TZ + (size_t)C * TZ + (size_t)R_WARPS * C * 32 * 2) * sizeof(float) + 128;
+    return ((size_t)CB * TZ + (size_t)C * TZ + (size_t)R_WARPS * C * 32 * 2 + (conf ? (size_t)C * C : 0)) * sizeof(float) + 128;
 }
 
 template <int CB>
 cudaError_t prepare_cb(int C)
 {
-    cudaError_t e = cudaFuncSetAttribute(upsample_ce_rows_kernel<CB, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)rows_smem_bytes<CB>(C));
+    cudaError_t e = cudaFuncSetAttribute(upsample_ce_rows_kernel<CB, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)rows_smem_bytes<CB>(C, false));
     if (e != cudaSuccess) return e;
-    return cudaFuncSetAttribute(upsample_ce_rows_kernel<CB, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)rows_smem_bytes<CB>(C));
+    return cudaFuncSetAttribute(upsample_ce_rows_kernel<CB, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)rows_smem_bytes<CB>(C, true));
 }
 
 template <int CB>
 cudaError_t launch_cb(const UpsampleCeArgs& a, const CUtensorMap& z_map, cudaStream_t s)
 {
     dim3 grid((unsigned)((a.w + RN_X - 1) / RN_X), (unsigned)((a.h + RN_Y - 1) / RN_Y), (unsigned)a.S);
-    if (a.conf) return launch_chain(upsample_ce_rows_kernel<CB, true>, grid, dim3(R_THREADS), rows_smem_bytes<CB>(a.C), s, a, z_map);
-    return launch_chain(upsample_ce_rows_kernel<CB, false>, grid, dim3(R_THREADS), rows_smem_bytes<CB>(a.C), s, a, z_map);
+    if (a.conf) return launch_chain(upsample_ce_rows_kernel<CB, true>, grid, dim3(R_THREADS), rows_smem_bytes<CB>(a.C, true), s, a, z_map);
+    return launch_chain(upsample_ce_rows_kernel<CB, false>, grid, dim3(R_THREADS), rows_smem_bytes<CB>(a.C, false), s, a, z_map);
 }
 
 // class-count buckets: the two workload sizes exactly, multiples of four otherwise

@@ -198,11 +198,12 @@ UpdateArgs make_update_args(st_ctx* c, int slot, const int* skip = nullptr, int6
 }
 
 // Forward of the trainable part for all streams: z (and the hidden activation).
-st_status enqueue_forward(st_ctx* c, StageTimer* t = nullptr)
+// `skip` (tensor-core kernels only): per-stream flags, see tc_forward.
+st_status enqueue_forward(st_ctx* c, StageTimer* t = nullptr, const int* skip = nullptr, int64_t skip_stride = 0)
 {
     cudaStream_t s = c->stream;
     if (c->bf16_mode) {
-        c->launches += tc_forward(c->plan, s, t);
+        c->launches += tc_forward(c->plan, s, t, skip, skip_stride);
     } else if (c->Ch == 0) {
         ST_REPEAT(t) launch_conv_fwd_f32(c->x_f32, c->Cin, c->h, c->w, c->theta + c->layout.w_off[0], c->theta + c->layout.b_off[0],
                             c->C, 1, false, c->z, c->S, (int64_t)c->Cin * c->p, c->n_params, c->n_params,
@@ -226,7 +227,8 @@ st_status enqueue_forward(st_ctx* c, StageTimer* t = nullptr)
 // Arguments of the fused upsample + cross-entropy kernel.  With bf16 GEMMs the weight gradient and the dgrad read the
 // bf16 copy of the logit gradient only, so the fp32 copy is not written during a step (st_read_tensor produces it on
 // demand by running the kernel once more on the same logits and labels).
-UpsampleCeArgs k3_args(st_ctx* c, bool fp32_grad, bool bf16_grad, unsigned long long* conf)
+UpsampleCeArgs k3_args(st_ctx* c, bool fp32_grad, bool bf16_grad, unsigned long long* conf, const int* skip = nullptr,
+                       int64_t skip_stride = 0)
 {
     UpsampleCeArgs k3;
     k3.z = c->z; k3.labels = c->labels;
@@ -239,15 +241,16 @@ UpsampleCeArgs k3_args(st_ctx* c, bool fp32_grad, bool bf16_grad, unsigned long 
     k3.bad = c->bad; k3.err = c->bad + 2;
     k3.S = c->S; k3.C = c->C; k3.h = c->h; k3.w = c->w;
     k3.has_map = c->k3_has_map;
+    k3.skip = skip; k3.skip_stride = skip_stride;
     return k3;
 }
 
 // ComputeLoss and the first half of PartialBackward: loss partials, logit gradient, optionally the confusion matrix
 // of this prediction.
-st_status enqueue_loss(st_ctx* c, unsigned long long* conf, StageTimer* t = nullptr)
+st_status enqueue_loss(st_ctx* c, unsigned long long* conf, StageTimer* t = nullptr, const int* skip = nullptr, int64_t skip_stride = 0)
 {
     cudaStream_t s = c->stream;
-    const UpsampleCeArgs k3 = k3_args(c, !c->bf16_mode, c->bf16_mode, conf);
+    const UpsampleCeArgs k3 = k3_args(c, !c->bf16_mode, c->bf16_mode, conf, skip, skip_stride);
     ST_REPEAT(t) launch_upsample_ce(k3, &c->k3_map, s);
     if (t) t->mark("upsample_ce", s, st_repeats(t));
     c->launches += st_repeats(t);
@@ -255,11 +258,11 @@ st_status enqueue_loss(st_ctx* c, unsigned long long* conf, StageTimer* t = null
 }
 
 // The rest of PartialBackward: gradients of the head's tensors (as split-K partial sums with bf16 GEMMs).
-st_status enqueue_backward(st_ctx* c, StageTimer* t = nullptr)
+st_status enqueue_backward(st_ctx* c, StageTimer* t = nullptr, const int* skip = nullptr, int64_t skip_stride = 0)
 {
     cudaStream_t s = c->stream;
     if (c->bf16_mode) {
-        c->launches += tc_backward(c->plan, s, t);
+        c->launches += tc_backward(c->plan, s, t, skip, skip_stride);
     } else if (c->Ch == 0) {
         ST_REPEAT(t) launch_conv_wgrad_f32(c->x_f32, c->dz, c->Cin, c->C, c->h, c->w, 1, c->grad + c->layout.w_off[0], c->S,
                               (int64_t)c->Cin * c->p, (int64_t)c->C * c->p, c->n_params, s);
@@ -619,20 +622,23 @@ TrainCtl train_ctl(st_ctx* c, int iter, int max_updates, double threshold)
 }
 
 // Train of Algorithm 1 for all streams: one prediction per pass (forward, loss + gradient + confusion, decision),
-// then backward and the update, which is a no-op for streams whose loop has ended.
+// then backward and the update.  The update is a no-op for streams whose loop has ended; so are the blocks of the
+// tensor-core GEMMs and of the loss kernel (the fp32 convolutions still run: their results are simply not used).
 st_status enqueue_train(st_ctx* c, int max_updates, double threshold)
 {
     st_status st = ST_OK;
     for (int i = 0; i <= max_updates && st == ST_OK; ++i) {
-        st = enqueue_forward(c);                                                          // prediction <- Forward(student, frame)
-        if (st == ST_OK) st = enqueue_loss(c, c->conf_buf + (int64_t)i * c->C * c->C);   // loss, gradient, confusion of it
+        const int* ended_before = i > 0 ? c->ctl_done + i : nullptr;        // done[s][i]: no prediction i for stream s
+        const int* ended_now = c->ctl_done + i + 1;                         // done[s][i+1]: no update i+1 for stream s
+        st = enqueue_forward(c, nullptr, ended_before, kCtlPitch);                        // prediction <- Forward(student, frame)
+        if (st == ST_OK) st = enqueue_loss(c, c->conf_buf + (int64_t)i * c->C * c->C, nullptr, ended_before, kCtlPitch);   // loss, gradient, confusion
         if (st != ST_OK) break;
         launch_train_decide(train_ctl(c, i, max_updates, threshold), c->stream);         // metric, best_student, break
         c->launches += 1;
         st = check_launch(c, "train control");
-        if (st == ST_OK && i < max_updates) st = enqueue_backward(c);
+        if (st == ST_OK && i < max_updates) st = enqueue_backward(c, nullptr, ended_now, kCtlPitch);
         // after the last prediction every loop has ended: the launch only finalises that prediction's loss
-        if (st == ST_OK) st = enqueue_update(c, i, c->ctl_done + i + 1, kCtlPitch);
+        if (st == ST_OK) st = enqueue_update(c, i, ended_now, kCtlPitch);
     }
     if (st != ST_OK) return st;
     launch_train_commit(train_ctl(c, 0, max_updates, threshold), c->theta, c->stream);    // student <- best_student

@@ -70,6 +70,8 @@ struct UpsampleCeArgs {
     unsigned int* err;       // device word: first wait that gave up (0 = none)
     int S, C, h, w;
     int has_map;             // the launch carries a tile map of z (see make_logit_tile_map)
+    const int* skip;         // nullptr, or one flag per stream (skip[s * skip_stride]): non-zero = the stream's blocks return at once
+    int64_t skip_stride;
 };
 // Tile map of the logits for the row-walking kernel: fp32 tensor {w, h, S*C}, one box = the block's tile of all
 // classes.  False if the shape does not allow it (w not a multiple of 4, C > 32) or the driver entry point is
@@ -225,7 +227,8 @@ struct StageTimer {
 };
 #define ST_REPEAT(t) for (int r_ = 0, R_ = (t) ? (t)->repeat : 1; r_ < R_; ++r_)
 inline int st_repeats(const StageTimer* t) { return t ? t->repeat : 1; }
-int tc_forward(const TcPlan*, cudaStream_t s, StageTimer* t = nullptr);    // returns the number of kernels launched
-int tc_backward(const TcPlan*, cudaStream_t s, StageTimer* t = nullptr);
+// `skip`: nullptr, or one flag per stream (skip[s * skip_stride]); the blocks of a flagged stream return at once.
+int tc_forward(const TcPlan*, cudaStream_t s, StageTimer* t = nullptr, const int* skip = nullptr, int64_t skip_stride = 0);    // returns the number of kernels launched
+int tc_backward(const TcPlan*, cudaStream_t s, StageTimer* t = nullptr, const int* skip = nullptr, int64_t skip_stride = 0);
 
 }  // namespace st

@@ -172,3 +172,57 @@ def test_config5_sixteen_streams_grouped():
         np.testing.assert_array_equal(gconf, oconf)
         assert m == om
     st.st_destroy(ctx)
+
+
+def test_train_key_frame_720p_early_exit_is_cheaper_than_the_full_loop():
+    """Algorithm 1 at frame size (720p, 1x1 head, bf16 GEMMs) on label-informed features: the loop ends as soon as
+    the mean IoU passes THRESHOLD, the result is the plain loop's iterate, and the ended loop costs little."""
+    cfg = si.get_config(2)
+    C, K = cfg.n_classes, 8
+    cls = si.voronoi_map(cfg.frame_h, cfg.frame_w, cfg.n_regions, C, 2000)
+    feat = si.label_informed_features(cfg.c_in, cfg.feat_h, cfg.feat_w, cls, 4, 0, strength=3.0)
+    theta = si.initial_head_params(cfg.c_in, 0, C, 1000)
+    stream = torch.cuda.current_stream()
+
+    def fresh():
+        ctx = st.st_init_head(n_streams=1, c_in=cfg.c_in, c_hidden=0, n_classes=C, feat_h=cfg.feat_h, feat_w=cfg.feat_w,
+                              gemm_precision=1, lr=0.5, momentum=0.9, cuda_stream=stream.cuda_stream, init_params=theta)
+        st.st_set_frozen_features(ctx, 0, torch.from_numpy(feat).cuda())
+        st.st_set_labels(ctx, 0, torch.from_numpy(cls).cuda())
+        return ctx
+
+    def timed(ctx, thr):
+        n_upd = np.zeros(1, np.int32); best = np.zeros(1, np.float64); met = np.zeros((1, K + 1), np.float64)
+        st.st_train_key_frame(ctx, thr, K, n_upd, best, met)            # first call: captures the graph
+        out = (int(n_upd[0]), float(best[0]), met[0].copy())
+        ts = []
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        d_n = torch.zeros(1, dtype=torch.int32, device="cuda")
+        for _ in range(3):
+            e0.record(stream); st.st_train_key_frame(ctx, thr, K, d_n); e1.record(stream); stream.synchronize()
+            ts.append(e0.elapsed_time(e1))
+        return out, min(ts)
+
+    ctx = fresh()
+    (n_full, best_full, met_full), _ = timed(ctx, 2.0)
+    assert n_full == K and met_full[-1] > met_full[0] + 0.3, met_full      # the student learns the frame
+    st.st_destroy(ctx)
+    thr = 0.5 * (met_full[1] + met_full[2])                                  # passed after the second update
+    ctx = fresh()
+    (n, best, met), _ = timed(ctx, thr)
+    assert n == 2 and best == met[2] > thr and (met[3:] == -1).all()
+    ref = fresh()
+    st.st_distill_step(ref, 2)
+    a, b = np.empty(ctx.n_params, np.float32), np.empty(ctx.n_params, np.float32)
+    st.st_pack_updated_params(ctx, 0, a); st.st_pack_updated_params(ref, 0, b)
+    # (the timed replays above ran Train again from the returned student: with the threshold already met they take
+    # no step, so the parameters are still those of the first call)
+    assert a.tobytes() == b.tobytes()
+    # cost of a call whose loop ends at once (threshold met by the incoming student) vs the full loop
+    _, t_done = timed(ctx, thr)
+    full = fresh()
+    _, t_full = timed(full, 2.0)
+    print(f"Train 720p K=8: full loop {t_full * 1e3:.0f} us, loop ended at once {t_done * 1e3:.0f} us")
+    assert t_done < 0.5 * t_full
+    for c in (ctx, ref, full):
+        st.st_destroy(c)
