@@ -169,6 +169,17 @@ ST_API st_status st_train_key_frame(st_ctx *ctx, double threshold, int32_t max_u
 ST_API st_status st_pack_updated_params(st_ctx *ctx, int32_t stream, void *dst, size_t dst_capacity, size_t *nbytes);
 
 /*
+ * st_apply_update — ApplyUpdate(student, student_diff) (Algorithm 4): install a buffer produced by
+ * st_pack_updated_params as the parameters of `stream`.  The updated part carries values, not differences, so the
+ * trainable tensors are simply replaced; the momentum buffer is left as it is.  This is what the client does with
+ * the server's reply, and what a server does to move a student between contexts.
+ *   src     host or device; the packed buffer (layout of st_pack_updated_params).
+ *   nbytes  its size; must equal st_param_count * 4, else ST_ERR_INVALID_ARG.
+ * pack -> apply -> pack reproduces the buffer bit for bit.
+ */
+ST_API st_status st_apply_update(st_ctx *ctx, int32_t stream, const void *src, size_t nbytes);
+
+/*
  * st_student_mask — prediction of the current student at frame resolution:
  * argmax over classes of the upsampled head logits (fresh forward of the current parameters).
  *   mask_out  host or device; uint8 [H][W].
@@ -256,6 +267,57 @@ ST_API st_status st_profile_step(st_ctx *ctx, int32_t n_steps, int32_t *n_stages
 ST_API st_status st_agreement_noalloc(const uint8_t *pred, const uint8_t *label, int64_t n_pixels,
                                       int32_t n_classes, void *cuda_stream, int64_t *conf_out,
                                       double *miou_out);
+
+/* ---- host-side pieces around the step: no device work, callable without a GPU ------------------------ */
+
+/*
+ * st_next_stride — NextStride (Algorithm 2): distance to the next key frame from the current stride and the
+ * student's metric in [0, 1].  ratio = metric / THRESHOLD below the threshold (the line through (0,0) and
+ * (THRESHOLD,1)), (metric - 2 THRESHOLD + 1) / (1 - THRESHOLD) from the threshold on (the line through
+ * (THRESHOLD,1) and (1,2)); stride <- ratio * stride, cut to whole frames, clamped to [min_stride, max_stride].
+ */
+ST_API int32_t st_next_stride(int32_t stride, double metric, double threshold, int32_t min_stride, int32_t max_stride);
+
+/*
+ * st_client_schedule — the key frames the client's loop (Algorithm 4) picks among n_frames frames: the first
+ * frame is a key frame; after a key frame the reply (updated part, metric) is complete `delay` frames later, at
+ * step = MIN_STRIDE at the latest (the client then waits for it), and the stride is recomputed with
+ * st_next_stride when it completes; the next key frame is the frame at which step = stride.
+ *   metrics       host; metrics[j] = metric returned for the j-th key frame; n_metrics entries.
+ *   delay         frames until a reply is complete, >= 1.
+ *   key_frames    host, capacity entries; receives the frame indices.
+ *   n_key_frames  host; receives their number (also when capacity is too small: ST_ERR_BUFFER_TOO_SMALL).
+ * ST_ERR_INVALID_ARG: bad parameters (threshold must lie strictly between 0 and 1), or fewer metrics than key frames.
+ */
+ST_API st_status st_client_schedule(int64_t n_frames, const double *metrics, int64_t n_metrics, double threshold,
+                                    int32_t min_stride, int32_t max_stride, int32_t delay, int64_t *key_frames,
+                                    int64_t capacity, int64_t *n_key_frames);
+
+/* Latencies of Section 4.4 (Table 1), in seconds. */
+typedef struct st_latencies {
+    double t_si;  /* student inference */
+    double t_sd;  /* one student distillation step */
+    double t_ti;  /* teacher inference */
+    double t_net; /* network latency of one key frame */
+} st_latencies;
+
+/*
+ * st_throughput_bounds — frames per second the system can reach at least and at most (Section 4.4):
+ *   lower = MIN_STRIDE / (MIN_STRIDE t_si + MAX_UPDATES t_sd + t_ti + t_net)
+ *   upper = MAX_STRIDE / ((MAX_STRIDE - MIN_STRIDE) t_si + max(MIN_STRIDE t_si, t_net + t_ti))
+ * st_traffic_bounds — networked data per second, in the unit of s_net (data per key frame) per second:
+ *   lower = s_net / (MAX_STRIDE t_si + MAX_UPDATES t_sd + t_ti + t_net)
+ *   upper = s_net / max(MIN_STRIDE t_si, t_net + t_ti)
+ * st_choose_max_updates — Section 5.3's rule: the largest MAX_UPDATES whose throughput lower bound is still
+ * above fps_floor; -1 if none is (or on bad arguments).
+ * Output pointers are host and may be NULL.  ST_ERR_INVALID_ARG on non-positive t_si, negative values or
+ * min_stride > max_stride.
+ */
+ST_API st_status st_throughput_bounds(const st_latencies *lat, int32_t min_stride, int32_t max_stride,
+                                      int32_t max_updates, double *fps_lower, double *fps_upper);
+ST_API st_status st_traffic_bounds(const st_latencies *lat, double s_net, int32_t min_stride, int32_t max_stride,
+                                   int32_t max_updates, double *per_second_lower, double *per_second_upper);
+ST_API int32_t st_choose_max_updates(const st_latencies *lat, int32_t min_stride, int32_t max_stride, double fps_floor);
 
 /* Number of kernels this library has launched on the context so far. */
 ST_API int64_t st_launch_count(const st_ctx *ctx);

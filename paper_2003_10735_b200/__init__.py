@@ -37,7 +37,8 @@ EXPORTED = [
     "st_param_count", "st_init_head", "st_set_frozen_features", "st_teacher_labels", "st_set_labels",
     "st_distill_step", "st_pack_updated_params", "st_student_mask", "st_agreement", "st_read_tensor",
     "st_launch_count", "st_destroy", "st_last_error", "st_status_name", "st_profile_step",
-    "st_agreement_noalloc", "st_train_key_frame",
+    "st_agreement_noalloc", "st_train_key_frame", "st_next_stride", "st_client_schedule", "st_throughput_bounds",
+    "st_traffic_bounds", "st_choose_max_updates", "st_apply_update",
 ]
 ST_NOALLOC_MAX_CLASSES = 64
 ST_MAX_STAGES = 12
@@ -86,6 +87,19 @@ def load_library() -> ctypes.CDLL:
     lib.st_distill_step.argtypes = [vp, i32, vp, vp]
     lib.st_train_key_frame.restype = ctypes.c_int
     lib.st_train_key_frame.argtypes = [vp, ctypes.c_double, i32, vp, vp, vp, vp, vp]
+    dbl = ctypes.c_double
+    lib.st_next_stride.restype = i32
+    lib.st_next_stride.argtypes = [i32, dbl, dbl, i32, i32]
+    lib.st_client_schedule.restype = ctypes.c_int
+    lib.st_client_schedule.argtypes = [i64, vp, i64, dbl, i32, i32, i32, vp, i64, ctypes.POINTER(i64)]
+    lib.st_throughput_bounds.restype = ctypes.c_int
+    lib.st_throughput_bounds.argtypes = [vp, i32, i32, i32, ctypes.POINTER(dbl), ctypes.POINTER(dbl)]
+    lib.st_traffic_bounds.restype = ctypes.c_int
+    lib.st_traffic_bounds.argtypes = [vp, dbl, i32, i32, i32, ctypes.POINTER(dbl), ctypes.POINTER(dbl)]
+    lib.st_choose_max_updates.restype = i32
+    lib.st_choose_max_updates.argtypes = [vp, i32, i32, dbl]
+    lib.st_apply_update.restype = ctypes.c_int
+    lib.st_apply_update.argtypes = [vp, i32, vp, ctypes.c_size_t]
     lib.st_pack_updated_params.restype = ctypes.c_int
     lib.st_pack_updated_params.argtypes = [vp, i32, vp, ctypes.c_size_t, ctypes.POINTER(ctypes.c_size_t)]
     lib.st_student_mask.restype = ctypes.c_int
@@ -223,6 +237,12 @@ def st_pack_updated_params(ctx: _Ctx, stream: int, dst, dst_capacity: Optional[i
     return int(nbytes.value)
 
 
+def st_apply_update(ctx: _Ctx, stream: int, src) -> None:
+    """ApplyUpdate (Algorithm 4): install a packed parameter buffer (float32, numpy or tensor) for `stream`."""
+    _check(load_library().st_apply_update(ctx.handle, stream, _ptr(src, "float32", ctx.n_params, "src"),
+                                          ctx.n_params * 4), ctx)
+
+
 def st_student_mask(ctx: _Ctx, stream: int, mask_out) -> None:
     _check(load_library().st_student_mask(ctx.handle, stream, _ptr(mask_out, "uint8", ctx.P, "mask_out")), ctx)
 
@@ -286,6 +306,49 @@ def st_agreement_noalloc(pred, label, n_classes: int, cuda_stream: int, conf_out
         _ptr(conf_out, "int64", max(n_classes, 0) ** 2, "conf_out"), miou_out.data_ptr())
     if status != ST_OK:
         raise StError(status, load_library().st_status_name(status).decode(), "st_agreement_noalloc")
+
+
+class st_latencies(ctypes.Structure):
+    _fields_ = [("t_si", ctypes.c_double), ("t_sd", ctypes.c_double), ("t_ti", ctypes.c_double), ("t_net", ctypes.c_double)]
+
+
+def _status_only(status: int, what: str) -> None:
+    if status != ST_OK:
+        raise StError(status, load_library().st_status_name(status).decode(), what)
+
+
+def st_next_stride(stride: int, metric: float, threshold: float, min_stride: int, max_stride: int) -> int:
+    """NextStride (Algorithm 2)."""
+    return int(load_library().st_next_stride(stride, metric, threshold, min_stride, max_stride))
+
+
+def st_client_schedule(n_frames: int, metrics, threshold: float, min_stride: int, max_stride: int, delay: int):
+    """Key-frame indices picked by the client's loop (Algorithm 4) as a list."""
+    m = np.ascontiguousarray(metrics, dtype=np.float64)
+    cap = n_frames // max(min_stride, 1) + 2
+    out = np.zeros(cap, np.int64)
+    n = ctypes.c_int64(0)
+    _status_only(load_library().st_client_schedule(n_frames, m.ctypes.data, m.size, threshold, min_stride, max_stride, delay,
+                                                   out.ctypes.data, cap, ctypes.byref(n)), "st_client_schedule")
+    return out[:n.value].tolist()
+
+
+def st_throughput_bounds(lat: st_latencies, min_stride: int, max_stride: int, max_updates: int):
+    lo, hi = ctypes.c_double(0), ctypes.c_double(0)
+    _status_only(load_library().st_throughput_bounds(ctypes.byref(lat), min_stride, max_stride, max_updates,
+                                                     ctypes.byref(lo), ctypes.byref(hi)), "st_throughput_bounds")
+    return lo.value, hi.value
+
+
+def st_traffic_bounds(lat: st_latencies, s_net: float, min_stride: int, max_stride: int, max_updates: int):
+    lo, hi = ctypes.c_double(0), ctypes.c_double(0)
+    _status_only(load_library().st_traffic_bounds(ctypes.byref(lat), s_net, min_stride, max_stride, max_updates,
+                                                  ctypes.byref(lo), ctypes.byref(hi)), "st_traffic_bounds")
+    return lo.value, hi.value
+
+
+def st_choose_max_updates(lat: st_latencies, min_stride: int, max_stride: int, fps_floor: float) -> int:
+    return int(load_library().st_choose_max_updates(ctypes.byref(lat), min_stride, max_stride, fps_floor))
 
 
 def st_launch_count(ctx: _Ctx) -> int:

@@ -793,6 +793,22 @@ st_status st_pack_updated_params(st_ctx* ctx, int32_t stream, void* dst, size_t 
     return ST_OK;
 }
 
+st_status st_apply_update(st_ctx* ctx, int32_t stream, const void* src, size_t nbytes)
+{
+    st_status st = check_stream_index(ctx, stream);
+    if (st != ST_OK) return st;
+    const size_t need = (size_t)ctx->n_params * sizeof(float);
+    if (!src) return fail(ctx, ST_ERR_INVALID_ARG, "st_apply_update: NULL source");
+    if (nbytes != need) return fail(ctx, ST_ERR_INVALID_ARG, "st_apply_update: %zu bytes given, the updated part has %zu", nbytes, need);
+    const void* dev = nullptr;
+    st = to_device(ctx, src, need, &dev);
+    if (st != ST_OK) return st;
+    launch_unpack((const float*)dev, ctx->theta + (int64_t)stream * ctx->n_params, ctx->layout, 1, ctx->stream);
+    ctx->launches += 1;
+    if (ctx->bf16_mode) { launch_refresh_shadow(make_update_args(ctx, -1), ctx->stream); ctx->launches += 1; }
+    return check_launch(ctx, "apply update");
+}
+
 namespace {
 // forward of all streams with the current parameters, then the mask kernel on `stream`
 st_status student_forward(st_ctx* ctx, int32_t stream, const char* who)

@@ -366,3 +366,40 @@ def test_profile_step_times_every_kernel_and_takes_real_steps():
     np.testing.assert_allclose(packed(ctx), head.theta, rtol=1e-4, atol=1e-6)     # the profiled steps are ordinary steps
     assert st.st_launch_count(ctx) >= 8
     st.st_destroy(ctx)
+
+
+# ---------------------------------------------------------------------------- ApplyUpdate (Algorithm 4)
+@pytest.mark.parametrize("c_hidden,prec", [(0, 0), (64, 1)])
+def test_apply_update_moves_a_student_between_contexts(c_hidden, prec):
+    c_in, C, h, w = 64, 5, 9, 12
+    feat, T = rand_problem(3, c_in, C, h, w)
+    lab = oracle.teacher_labels(T)
+    theta = si.initial_head_params(c_in, c_hidden, C, 7)
+    server = make_ctx(c_in, c_hidden, C, h, w, theta, prec=prec, lr=0.05, mu=0.9)
+    st.st_set_frozen_features(server, 0, dev(feat)); st.st_set_labels(server, 0, dev(lab))
+    st.st_distill_step(server, 3)
+    update = packed(server)                                        # UpdatedPart(student)
+    client = make_ctx(c_in, c_hidden, C, h, w, theta, prec=prec)   # still holds the old student
+    st.st_set_frozen_features(client, 0, dev(feat))
+    m_old = torch.empty((4 * h, 4 * w), dtype=torch.uint8, device="cuda")
+    st.st_student_mask(client, 0, m_old)
+    st.st_apply_update(client, 0, update)                          # host buffer
+    assert packed(client).tobytes() == update.tobytes()
+    m_new, m_srv = torch.empty_like(m_old), torch.empty_like(m_old)
+    st.st_student_mask(client, 0, m_new); st.st_student_mask(server, 0, m_srv)
+    assert torch.equal(m_new, m_srv)                               # the client now predicts what the server's student predicts
+    # the oracle's student after the same three steps predicts the same mask up to near-ties
+    head = oracle.Head(c_in, c_hidden, C, lr=0.05, momentum=0.9, theta=theta, quantize_bf16=bool(prec))
+    for _ in range(3):
+        oracle.distill_step(head, feat, lab)
+    assert (m_new.cpu().numpy() != oracle.student_mask(head, feat)).mean() <= (1e-3 if prec == 0 else 2e-2)
+    st.st_apply_update(client, 0, dev(theta))                      # device buffer: back to the old student
+    assert packed(client).tobytes() == np.asarray(theta, np.float32).tobytes()
+    back = torch.empty_like(m_old)
+    st.st_student_mask(client, 0, back)
+    assert torch.equal(back, m_old)
+    with pytest.raises(st.StError) as ei:
+        st.load_library().st_apply_update  # symbol exists
+        st._check(st.load_library().st_apply_update(client.handle, 0, update.ctypes.data, update.nbytes - 4), client)
+    assert ei.value.status == st.ST_ERR_INVALID_ARG
+    st.st_destroy(server); st.st_destroy(client)
