@@ -170,6 +170,15 @@ def sgd_(theta: np.ndarray, v: np.ndarray, g: np.ndarray, lr: float, mu: float) 
     _lib(theta.dtype).so_sgd(_p(theta), _p(v), _p(g), _c_i64(theta.size), R(lr), R(mu))
 
 
+def adam_(theta: np.ndarray, m: np.ndarray, v: np.ndarray, g: np.ndarray, lr: float, b1: float, b2: float, eps: float,
+          t: int) -> None:
+    """Step t (1-based) of Adam on theta in place; m, v are the two moment buffers."""
+    assert theta.flags.c_contiguous and m.flags.c_contiguous and v.flags.c_contiguous
+    g = _c(g, theta.dtype)
+    _lib(theta.dtype).so_adam(_p(theta), _p(m), _p(v), _p(g), _c_i64(theta.size), ctypes.c_double(lr), ctypes.c_double(b1),
+                              ctypes.c_double(b2), ctypes.c_double(eps), _c_i64(t))
+
+
 def confusion(labels: np.ndarray, pred: np.ndarray, C: int):
     """(conf int64 [C][C] with conf[label][pred], number of skipped pixels)."""
     labels = _c(labels, np.uint8)
@@ -211,7 +220,12 @@ class Head:
     dtype: type = np.float32
     quantize_bf16: bool = False      # test-only: round GEMM operands to bf16 like the tensor-core path
     theta: np.ndarray = None         # flat parameters in packed order
-    vel: np.ndarray = None           # momentum, same order, starts at zero
+    vel: np.ndarray = None           # momentum (SGD) / first moment (Adam), same order, starts at zero
+    optimizer: str = "sgd"           # "sgd" (heavy-ball momentum) or "adam" (Section 5.2)
+    betas: Tuple[float, float] = (0.9, 0.999)   # Adam's decay rates and epsilon: not stated in the paper,
+    eps: float = 1e-8                #   the constants of the published algorithm are assumed
+    vel2: np.ndarray = None          # Adam's second moment
+    t: int = 0                       # optimisation steps taken so far (Adam's bias correction)
 
     def __post_init__(self):
         n = sum(int(np.prod(ws)) + int(np.prod(bs))
@@ -221,6 +235,16 @@ class Head:
         self.theta = np.ascontiguousarray(self.theta, dtype=self.dtype).copy()
         assert self.theta.size == n, (self.theta.size, n)
         self.vel = np.zeros(n, dtype=self.dtype)
+        self.vel2 = np.zeros(n, dtype=self.dtype)
+        assert self.optimizer in ("sgd", "adam")
+
+    def optim_step(self, grad: np.ndarray) -> None:
+        """student <- OptimStep(student, gradients)."""
+        self.t += 1
+        if self.optimizer == "adam":
+            adam_(self.theta, self.vel, self.vel2, grad.astype(self.dtype), self.lr, self.betas[0], self.betas[1], self.eps, self.t)
+        else:
+            sgd_(self.theta, self.vel, grad.astype(self.dtype), self.lr, self.momentum)
 
     def layers(self) -> List[Tuple[np.ndarray, np.ndarray]]:
         """Views (weight, bias) into theta, forward order."""
@@ -289,7 +313,7 @@ def distill_step(head: Head, feat: np.ndarray, labels: np.ndarray):
     """One iteration of Algorithm 1's loop: loss and gradients at the current
     parameters, then one optimiser step.  Returns (loss, student mask before the update)."""
     loss, grad, mask = gradients(head, feat, labels)
-    sgd_(head.theta, head.vel, grad.astype(head.dtype), head.lr, head.momentum)
+    head.optim_step(grad)
     return loss, mask
 
 

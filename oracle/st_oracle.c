@@ -280,6 +280,28 @@ void so_sgd(real *theta, real *v, const real *g, int64_t n, real lr, real mu)
 }
 
 /* ---------------------------------------------------------------------------
+ * OptimStep with Adam, the optimiser the paper's experiments use (Section 5.2: "the Adam optimizer with a
+ * learning rate of 0.01"; the other constants are not stated and are passed in).  Step t (1-based) of the
+ * published algorithm, epsilon added to the root of the bias-corrected second moment:
+ *   m <- b1 m + (1 - b1) g;   v <- b2 v + (1 - b2) g^2
+ *   theta <- theta - lr * (m / (1 - b1^t)) / (sqrt(v / (1 - b2^t)) + eps)
+ * Each element is computed in double and stored in the storage type.
+ * ------------------------------------------------------------------------- */
+void so_adam(real *theta, real *m, real *v, const real *g, int64_t n, double lr, double b1, double b2, double eps, int64_t t)
+{
+    const double c1 = 1.0 - pow(b1, (double)t), c2 = 1.0 - pow(b2, (double)t);
+    for (int64_t i = 0; i < n; ++i) {
+        const double gi = (double)g[i];
+        const double mi = b1 * (double)m[i] + (1.0 - b1) * gi;
+        const double vi = b2 * (double)v[i] + (1.0 - b2) * gi * gi;
+        m[i] = (real)mi;
+        v[i] = (real)vi;
+        const double mhat = mi / c1, vhat = vi / c2;
+        theta[i] = (real)((double)theta[i] - lr * mhat / (sqrt(vhat) + eps));
+    }
+}
+
+/* ---------------------------------------------------------------------------
  * ComputeMetric (Algorithm 1): mean IoU of prediction vs. label (Section 3.2):
  *   IoU_c = |pred_c ∩ label_c| / |pred_c ∪ label_c|, averaged over the classes
  *   present in the label.

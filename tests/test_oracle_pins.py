@@ -382,3 +382,61 @@ def test_round_bf16_ties_to_even():
     torch = pytest.importorskip("torch")
     ref = torch.from_numpy(x).to(torch.bfloat16).to(torch.float32).numpy()
     np.testing.assert_array_equal(oracle.round_bf16(x), ref)
+
+
+# ---------------------------------------------------------------------------- Adam (Section 5.2)
+def test_adam_first_step_moves_every_weight_by_lr_against_its_gradient_sign():
+    # step 1: m_hat = g, v_hat = g^2, so theta moves by lr * g / (|g| + eps): the sign of g, whatever its size
+    rng = np.random.default_rng(0)
+    for dtype in (np.float32, np.float64):
+        theta = rng.standard_normal(50).astype(dtype); g = (rng.standard_normal(50) * 10 ** rng.uniform(-3, 3, 50)).astype(dtype)
+        th, m, v = theta.copy(), np.zeros(50, dtype), np.zeros(50, dtype)
+        oracle.adam_(th, m, v, g, 0.01, 0.9, 0.999, 1e-8, 1)
+        np.testing.assert_allclose(th, theta - 0.01 * g / (np.abs(g) + 1e-8), rtol=0, atol=2e-6 if dtype == np.float32 else 1e-12)
+        big = np.abs(g) > 1e-2                                   # there eps / |g| < 1e-6: a plain sign step
+        np.testing.assert_allclose(th[big], (theta - 0.01 * np.sign(g))[big], rtol=0, atol=2e-6 if dtype == np.float32 else 2e-8)
+        np.testing.assert_allclose(m, 0.1 * g, rtol=1e-6); np.testing.assert_allclose(v, 0.001 * g * g, rtol=1e-6)
+
+
+def test_adam_constant_gradient_keeps_unit_steps_and_zero_gradient_does_not_move():
+    # constant g: m_hat = g and v_hat = g^2 at every step, so every step has length lr
+    th, m, v = np.zeros(3), np.zeros(3), np.zeros(3)
+    g = np.array([2.0, -0.5, 1e-3])
+    for t in range(1, 8):
+        oracle.adam_(th, m, v, g, 0.01, 0.9, 0.999, 1e-12, t)
+        np.testing.assert_allclose(th, -0.01 * t * np.sign(g), rtol=1e-6)
+    th0 = np.ones(4); m, v = np.zeros(4), np.zeros(4)
+    oracle.adam_(th0, m, v, np.zeros(4), 0.01, 0.9, 0.999, 1e-8, 1)
+    assert (th0 == 1.0).all()
+
+
+def test_adam_matches_torch_adam_over_several_steps():
+    torch = pytest.importorskip("torch")
+    rng = np.random.default_rng(1)
+    theta0 = rng.standard_normal(40)
+    grads = [rng.standard_normal(40) * (1 + k) for k in range(6)]
+    th, m, v = theta0.copy(), np.zeros(40), np.zeros(40)
+    p = torch.tensor(theta0, dtype=torch.float64, requires_grad=True)
+    opt = torch.optim.Adam([p], lr=0.01, betas=(0.8, 0.99), eps=1e-6)
+    for t, g in enumerate(grads, 1):
+        oracle.adam_(th, m, v, g, 0.01, 0.8, 0.99, 1e-6, t)
+        p.grad = torch.tensor(g, dtype=torch.float64)
+        opt.step()
+        np.testing.assert_allclose(th, p.detach().numpy(), rtol=1e-12, atol=1e-14)
+
+
+def test_head_with_adam_takes_textbook_steps_on_the_real_gradient():
+    rng = np.random.default_rng(2)
+    feat = np.maximum(rng.standard_normal((6, 4, 5)), 0).astype(np.float32)
+    labels = rng.integers(0, 3, (16, 20)).astype(np.uint8)
+    theta = si.initial_head_params(6, 0, 3, 5)
+    head = oracle.Head(6, 0, 3, lr=0.01, optimizer="adam", theta=theta)
+    th, m, v = np.asarray(theta, np.float64).copy(), np.zeros(theta.size), np.zeros(theta.size)
+    for t in range(1, 4):
+        _, g, _ = oracle.gradients(head, feat, labels)                 # gradient at the current parameters
+        oracle.distill_step(head, feat, labels)
+        m = 0.9 * m + 0.1 * g; v = 0.999 * v + 0.001 * g * g            # the update written out once more in numpy
+        th = th - 0.01 * (m / (1 - 0.9 ** t)) / (np.sqrt(v / (1 - 0.999 ** t)) + 1e-8)
+        np.testing.assert_allclose(head.theta, th, rtol=2e-5, atol=2e-7)
+        th = head.theta.astype(np.float64)                               # follow the fp32 trajectory
+        m, v = head.vel.astype(np.float64), head.vel2.astype(np.float64)
