@@ -66,8 +66,13 @@ typedef struct st_head_desc {
     int32_t up;             /* frame = feature map * up, bilinear (half-pixel centres); must be 4 */
     int32_t gemm_precision; /* 0: fp32 FMA convolutions; 1: bf16 operands on tensor cores, fp32 accumulate */
     float lr;               /* learning rate of OptimStep */
-    float momentum;         /* heavy-ball momentum; 0 = plain gradient descent */
+    float momentum;         /* heavy-ball momentum; 0 = plain gradient descent (optimizer 0 only) */
     void *cuda_stream;      /* cudaStream_t on which all work is enqueued (NULL = default stream) */
+    int32_t optimizer;      /* 0: gradient descent with momentum (Section 4.1.4); 1: Adam (the optimiser of the
+                               paper's experiments, Section 5.2) */
+    double adam_beta1;      /* Adam's decay rates and epsilon; the paper does not state them.  0 selects the */
+    double adam_beta2;      /*   constants of the published algorithm: 0.9, 0.999, 1e-8.                       */
+    double adam_eps;        /* epsilon is added to the root of the bias-corrected second moment */
 } st_head_desc;
 
 /* Number of fp32 values in one head's packed parameter buffer:

@@ -19,11 +19,36 @@ bool pdl_enabled()
 
 constexpr int kUpdThreads = 256;
 
-__device__ __forceinline__ void apply_update(const UpdateArgs& a, int64_t gi, float g)
+// Bias corrections of Adam's step t: (1 - b1^t, 1 - b2^t), t = steps taken before this call + position in the call.
+struct AdamCorr { double c1, c2; };
+__device__ __forceinline__ AdamCorr adam_corrections(const UpdateArgs& a, int s)
 {
+    AdamCorr c = {1.0, 1.0};
+    if (a.adam) {
+        const double t = (double)(a.step_base[s] + a.loss_slot + 1);
+        c.c1 = 1.0 - exp(t * a.ln_b1);
+        c.c2 = 1.0 - exp(t * a.ln_b2);
+    }
+    return c;
+}
+
+// OptimStep on one parameter.  Gradient descent with momentum: v <- mu v + g; theta <- theta - lr v.
+// Adam (each element in double, stored as fp32): m <- b1 m + (1 - b1) g; v <- b2 v + (1 - b2) g^2;
+// theta <- theta - lr (m / c1) / (sqrt(v / c2) + eps).
+__device__ __forceinline__ void apply_update(const UpdateArgs& a, int64_t gi, float g, const AdamCorr& k)
+{
+    a.grad[gi] = g;
+    if (a.adam) {
+        const double gd = (double)g;
+        const double m = a.b1 * (double)a.vel[gi] + (1.0 - a.b1) * gd;
+        const double v = a.b2 * (double)a.vel2[gi] + (1.0 - a.b2) * gd * gd;
+        a.vel[gi] = (float)m;
+        a.vel2[gi] = (float)v;
+        a.theta[gi] = (float)((double)a.theta[gi] - (double)a.lr * (m / k.c1) / (sqrt(v / k.c2) + a.eps));
+        return;
+    }
     float v = fmaf(a.mu, a.vel[gi], g);
     a.vel[gi] = v;
-    a.grad[gi] = g;
     a.theta[gi] = fmaf(-a.lr, v, a.theta[gi]);
 }
 
@@ -42,6 +67,7 @@ sgd_update_kernel(UpdateArgs a, int n_param_blocks, int64_t range_begin)
     const int s = blockIdx.y;
     const int64_t base = (int64_t)s * a.n_params;
     const bool skip = a.skip && a.skip[(int64_t)s * a.skip_stride];   // block-uniform
+    const AdamCorr corr = adam_corrections(a, s);
     if ((int)blockIdx.x < n_param_blocks) {
         if (skip) return;
         const int col = threadIdx.x % kRow, g = threadIdx.x / kRow;
@@ -98,10 +124,10 @@ sgd_update_kernel(UpdateArgs a, int n_param_blocks, int64_t range_begin)
                 } else {
                     gr = a.grad[base + i];
                 }
-                apply_update(a, base + i, gr);
+                apply_update(a, base + i, gr, corr);
                 if (ly.shadow) ly.shadow[(int64_t)s * ly.shadow_stream_stride + (i - ly.w_off)] = __float2bfloat16_rn(a.theta[base + i]);
             } else if (!ly.b_partials) {
-                apply_update(a, base + i, a.grad[base + i]);
+                apply_update(a, base + i, a.grad[base + i], corr);
             }   // biases with partial sums are finished by the reduction warps below
         }
         return;
@@ -128,7 +154,7 @@ sgd_update_kernel(UpdateArgs a, int n_param_blocks, int64_t range_begin)
             }
 #pragma unroll
             for (int o = 16; o > 0; o >>= 1) g += __shfl_xor_sync(0xffffffffu, g, o);
-            if (lane == 0 && !skip) apply_update(a, base + ly.b_off + item, g);
+            if (lane == 0 && !skip) apply_update(a, base + ly.b_off + item, g, corr);
             return;
         }
         item -= ly.cout;
@@ -190,9 +216,10 @@ sgd_update_stream_kernel(UpdateArgs a, int L)
         }
     }
     const int64_t gi = (int64_t)s * a.n_params + ly.w_off + e;
+    const AdamCorr corr = adam_corrections(a, s);
 #pragma unroll
     for (int j = 0; j < VEC; ++j) {
-        apply_update(a, gi + j, g[j]);
+        apply_update(a, gi + j, g[j], corr);
         if (ly.shadow) ly.shadow[(int64_t)s * ly.shadow_stream_stride + e + j] = __float2bfloat16_rn(a.theta[gi + j]);
     }
 }
@@ -235,6 +262,18 @@ int launch_sgd_update(const UpdateArgs& a, cudaStream_t s)
     else if (E == 1) launch_chain(sgd_update_kernel<8, 1>, grid, blk, 0, s, a, n_param_blocks, range_begin);
     else launch_chain(sgd_update_kernel<8, 4>, grid, blk, 0, s, a, n_param_blocks, range_begin);
     return n_launches;
+}
+
+__global__ void step_tick_kernel(long long* step_base, int S, int add, const int* add_per_stream)
+{
+    const int s = threadIdx.x;
+    if (s < S) step_base[s] += add_per_stream ? add_per_stream[s] : add;
+}
+
+void launch_step_tick(long long* step_base, int S, int add, const int* add_per_stream, cudaStream_t s)
+{
+    for (int s0 = 0; s0 < S; s0 += 256)
+        step_tick_kernel<<<1, 256, 0, s>>>(step_base + s0, S - s0 < 256 ? S - s0 : 256, add, add_per_stream ? add_per_stream + s0 : nullptr);
 }
 
 __global__ void refresh_shadow_kernel(UpdateArgs a)

@@ -4,6 +4,7 @@
 #include "../../include/shadowtutor.h"
 #include "st_internal.h"
 
+#include <cmath>
 #include <cstdarg>
 #include <cstdio>
 #include <cstring>
@@ -36,6 +37,10 @@ struct st_ctx {
     PackLayout layout;
 
     float *theta = nullptr, *vel = nullptr, *grad = nullptr;
+    float* vel2 = nullptr;                  // Adam's second moment
+    long long* step_base = nullptr;         // [S] optimisation steps taken so far (Adam's bias correction)
+    bool adam = false;
+    double b1 = 0.9, b2 = 0.999, eps = 1e-8;
     float* x_f32 = nullptr;
     bf16* x_bf16 = nullptr;
     uint8_t* labels = nullptr;
@@ -194,6 +199,8 @@ UpdateArgs make_update_args(st_ctx* c, int slot, const int* skip = nullptr, int6
     u.loss_buf = c->loss_buf; u.loss_slot = slot;
     u.inv_P = 1.0 / (double)c->P;
     u.skip = skip; u.skip_stride = skip_stride;
+    u.adam = c->adam ? 1 : 0; u.vel2 = c->vel2; u.step_base = c->step_base;
+    u.b1 = c->b1; u.b2 = c->b2; u.eps = c->eps; u.ln_b1 = log(c->b1); u.ln_b2 = log(c->b2);
     return u;
 }
 
@@ -384,6 +391,12 @@ st_status st_init_head(const st_head_desc* desc, const float* init_params, st_ct
         return fail(nullptr, ST_ERR_INVALID_ARG, "st_init_head: n_classes %d outside 2..255", d.n_classes);
     if (!(d.lr >= 0.f) || !(d.momentum >= 0.f) || !(d.momentum < 1.f))
         return fail(nullptr, ST_ERR_INVALID_ARG, "st_init_head: lr must be >= 0 and momentum in [0, 1)");
+    if (d.optimizer != 0 && d.optimizer != 1)
+        return fail(nullptr, ST_ERR_INVALID_ARG, "st_init_head: optimizer must be 0 (gradient descent) or 1 (Adam)");
+    const double ab1 = d.adam_beta1 == 0.0 ? 0.9 : d.adam_beta1, ab2 = d.adam_beta2 == 0.0 ? 0.999 : d.adam_beta2;
+    const double aeps = d.adam_eps == 0.0 ? 1e-8 : d.adam_eps;
+    if (d.optimizer == 1 && (!(ab1 > 0.0 && ab1 < 1.0) || !(ab2 > 0.0 && ab2 < 1.0) || !(aeps > 0.0)))
+        return fail(nullptr, ST_ERR_INVALID_ARG, "st_init_head: Adam needs beta1, beta2 in (0, 1) and eps > 0");
     if (d.gemm_precision != 0 && d.gemm_precision != 1)
         return fail(nullptr, ST_ERR_INVALID_ARG, "st_init_head: gemm_precision must be 0 or 1");
     if (d.up != kUp) return fail(nullptr, ST_ERR_UNSUPPORTED, "st_init_head: up must be 4");
@@ -406,6 +419,7 @@ st_status st_init_head(const st_head_desc* desc, const float* init_params, st_ct
     c->p = (int64_t)c->h * c->w; c->P = (int64_t)c->H * c->W;
     c->n_params = (int64_t)st_param_count(d.c_in, d.c_hidden, d.n_classes);
     c->bf16_mode = d.gemm_precision == 1;
+    c->adam = d.optimizer == 1; c->b1 = ab1; c->b2 = ab2; c->eps = aeps;
     c->has_feat.assign(c->S, 0); c->has_labels.assign(c->S, 0);
     // The legacy default stream cannot be captured: steps are then enqueued kernel by kernel.
     c->use_graphs = c->stream != nullptr && c->stream != cudaStreamLegacy && c->stream != cudaStreamPerThread;
@@ -430,6 +444,8 @@ st_status st_init_head(const st_head_desc* desc, const float* init_params, st_ct
     cudaError_t e = cudaSuccess;
 #define ALLOC(ptr, count) if (e == cudaSuccess) e = dev_alloc(c, &c->ptr, (size_t)(count))
     ALLOC(theta, S * c->n_params); ALLOC(vel, S * c->n_params); ALLOC(grad, S * c->n_params);
+    ALLOC(step_base, S);
+    if (c->adam) ALLOC(vel2, S * c->n_params);
     ALLOC(labels, S * c->P);
     ALLOC(z, S * c->C * c->p); ALLOC(dz, S * c->C * c->p);
     ALLOC(loss_part, S * c->n_k3_blocks); ALLOC(db_part, (size_t)S * c->n_k3_blocks * c->C);
@@ -580,6 +596,7 @@ st_status st_distill_step(st_ctx* ctx, int32_t n_steps, float* loss_out, int64_t
             const int64_t before = ctx->launches;
             ST_CUDA(ctx, cudaStreamBeginCapture(ctx->stream, cudaStreamCaptureModeThreadLocal));
             for (int k = 0; k < n_steps && st == ST_OK; ++k) st = enqueue_step(ctx, k, want_conf);
+            if (st == ST_OK && ctx->adam) { launch_step_tick(ctx->step_base, ctx->S, n_steps, nullptr, ctx->stream); ctx->launches += 1; }
             cudaError_t e = cudaStreamEndCapture(ctx->stream, &graph);
             const int64_t n_launches = ctx->launches - before;
             ctx->launches = before;
@@ -598,6 +615,7 @@ st_status st_distill_step(st_ctx* ctx, int32_t n_steps, float* loss_out, int64_t
             st = enqueue_step(ctx, k, want_conf);
             if (st != ST_OK) return st;
         }
+        if (ctx->adam) { launch_step_tick(ctx->step_base, ctx->S, n_steps, nullptr, ctx->stream); ctx->launches += 1; }
     }
     if (loss_out)
         ST_CUDA(ctx, cudaMemcpy2DAsync(loss_out, (size_t)n_steps * sizeof(float), ctx->loss_buf, kMaxSteps * sizeof(float),
@@ -644,6 +662,7 @@ st_status enqueue_train(st_ctx* c, int max_updates, double threshold)
     launch_train_commit(train_ctl(c, 0, max_updates, threshold), c->theta, c->stream);    // student <- best_student
     launch_refresh_shadow(make_update_args(c, 0), c->stream);
     c->launches += 2;
+    if (c->adam) { launch_step_tick(c->step_base, c->S, 0, c->ctl_n_updates, c->stream); c->launches += 1; }   // steps taken
     return check_launch(c, "train commit");
 }
 }  // namespace
@@ -751,6 +770,7 @@ st_status st_profile_step(st_ctx* ctx, int32_t n_steps, int32_t* n_stages, float
         cudaEventRecord(t.ev[0], ctx->stream);
         st = enqueue_step(ctx, 0, false, &t);
         if (st != ST_OK) break;
+        if (ctx->adam) { launch_step_tick(ctx->step_base, ctx->S, 1, nullptr, ctx->stream); ctx->launches += 1; }
         if (cudaStreamSynchronize(ctx->stream) != cudaSuccess) { st = fail(ctx, ST_ERR_CUDA, "st_profile_step: synchronize failed"); break; }
         n = t.n;
         for (int i = 0; i < n; ++i) {

@@ -148,7 +148,14 @@ struct UpdateArgs {
     double inv_P;
     const int* skip;         // nullptr, or one flag per stream (skip[s * skip_stride]): non-zero = leave the stream's
     int64_t skip_stride;     //   parameters and momentum untouched (the loss is still finalised)
+    // Adam (optimizer 1): `vel` is the first moment, `vel2` the second; step number t = step_base[s] + loss_slot + 1
+    int adam;
+    float* vel2;             // [S][n_params]
+    double b1, b2, eps, ln_b1, ln_b2;
+    const long long* step_base;   // [S] optimisation steps taken before this call
 };
+// step_base[s] += add (add_per_stream == nullptr) or += add_per_stream[s]
+void launch_step_tick(long long* step_base, int S, int add, const int* add_per_stream, cudaStream_t s);
 int launch_sgd_update(const UpdateArgs& a, cudaStream_t s);   // returns the number of kernels launched
 // refresh the bf16 shadows from the fp32 master parameters (after init)
 void launch_refresh_shadow(const UpdateArgs& a, cudaStream_t s);
