@@ -116,16 +116,29 @@ def upsample_adjoint(g: np.ndarray, s: int) -> np.ndarray:
     return dz
 
 
-def softmax_ce(u: np.ndarray, labels: np.ndarray, want_grad: bool = True):
-    """(mean loss as float, gradient [C][H][W] or None, number of out-of-range labels)."""
+def softmax_ce(u: np.ndarray, labels: np.ndarray, want_grad: bool = True, weights: Optional[np.ndarray] = None):
+    """(mean loss as float, gradient [C][H][W] or None, number of out-of-range labels).
+    `weights` (uint8 [H][W]) scales each pixel's loss and gradient (Section 5.2's loss weighting)."""
     u = _c(u)
     labels = _c(labels, np.uint8)
     C, H, W = u.shape
     g = np.empty_like(u) if want_grad else None
     loss = ctypes.c_double(0.0)
-    bad = _lib(u.dtype).so_softmax_ce(_p(u), _p(labels), _c_int(C), _c_i64(H * W),
-                                      _p(g) if want_grad else None, ctypes.byref(loss))
+    lib = _lib(u.dtype)
+    lib.so_softmax_ce_weighted.restype = _c_i64
+    wg = _c(weights, np.uint8) if weights is not None else None
+    bad = lib.so_softmax_ce_weighted(_p(u), _p(labels), _p(wg) if wg is not None else None, _c_int(C), _c_i64(H * W),
+                                     _p(g) if want_grad else None, ctypes.byref(loss))
     return loss.value, g, int(bad)
+
+
+def object_weights(labels: np.ndarray, background: int, radius: int, factor: int) -> np.ndarray:
+    """uint8 [H][W]: `factor` for pixels within `radius` (square window) of a non-background pixel, else 1."""
+    labels = _c(labels, np.uint8)
+    H, W = labels.shape
+    out = np.empty((H, W), np.uint8)
+    _lib(np.float32).so_object_weights(_p(labels), _c_int(H), _c_int(W), _c_int(background), _c_int(radius), _c_int(factor), _p(out))
+    return out
 
 
 def conv_wgrad(x: np.ndarray, dout: np.ndarray, ks: int):
@@ -226,6 +239,9 @@ class Head:
     eps: float = 1e-8                #   the constants of the published algorithm are assumed
     vel2: np.ndarray = None          # Adam's second moment
     t: int = 0                       # optimisation steps taken so far (Adam's bias correction)
+    object_weight: int = 1           # Section 5.2's loss weighting: factor for pixels near / within non-background
+    object_radius: int = 0           #   objects (5 in the paper), the distance that counts as "near" (not stated
+    background: int = 0              #   in the paper) and the background class
 
     def __post_init__(self):
         n = sum(int(np.prod(ws)) + int(np.prod(bs))
@@ -289,7 +305,8 @@ def gradients(head: Head, feat: np.ndarray, labels: np.ndarray):
     layers = head.layers()
     z, Hd = head_forward(head, feat)
     u = upsample(z, head.up)
-    loss, g, _ = softmax_ce(u, labels)
+    wgt = object_weights(labels, head.background, head.object_radius, head.object_weight) if head.object_weight > 1 else None
+    loss, g, _ = softmax_ce(u, labels, weights=wgt)
     mask = teacher_labels(u)
     dz = upsample_adjoint(g, head.up)
     if head.c_hidden == 0:

@@ -166,7 +166,20 @@ void so_upsample_adjoint(const real *g, int C, int h, int w, int s, real *dz)
  * u is [C][P]; g (may be NULL) is [C][P]; *loss = (1/P) sum_p loss_p.
  * Returns the number of labels >= C (those pixels are skipped).
  * ------------------------------------------------------------------------- */
+int64_t so_softmax_ce_weighted(const real *u, const uint8_t *lab, const uint8_t *wgt, int C, int64_t P, real *g, double *loss);
+
 int64_t so_softmax_ce(const real *u, const uint8_t *lab, int C, int64_t P, real *g, double *loss)
+{
+    return so_softmax_ce_weighted(u, lab, NULL, C, P, g, loss);
+}
+
+/* ---------------------------------------------------------------------------
+ * Loss weighting against class imbalance (Section 5.2): the cross-entropy of pixels "near and within
+ * non-background objects" is scaled by a factor (5 in the paper).  wgt[p] is that factor per pixel
+ * (NULL: 1 everywhere); the loss of a pixel and its gradient are both multiplied by it, the normaliser stays P:
+ *   loss = (1/P) sum_p wgt_p loss_p,   g_c = wgt_p (softmax_c - [c == label]) / P.
+ * ------------------------------------------------------------------------- */
+int64_t so_softmax_ce_weighted(const real *u, const uint8_t *lab, const uint8_t *wgt, int C, int64_t P, real *g, double *loss)
 {
     double total = 0.0;
     int64_t bad = 0;
@@ -185,15 +198,37 @@ int64_t so_softmax_ce(const real *u, const uint8_t *lab, int C, int64_t P, real 
         }
         double Z = 0.0;
         for (int c = 0; c < C; ++c) Z += exp((double)u[(int64_t)c * P + p] - m);
-        total += m + log(Z) - (double)u[(int64_t)l * P + p];
+        const double wp = wgt ? (double)wgt[p] : 1.0;
+        total += wp * (m + log(Z) - (double)u[(int64_t)l * P + p]);
         if (g)
             for (int c = 0; c < C; ++c) {
                 double pc = exp((double)u[(int64_t)c * P + p] - m) / Z;
-                g[(int64_t)c * P + p] = (real)((pc - (c == l ? 1.0 : 0.0)) / (double)P);
+                g[(int64_t)c * P + p] = (real)(wp * (pc - (c == l ? 1.0 : 0.0)) / (double)P);
             }
     }
     *loss = total / (double)P;
     return bad;
+}
+
+/* ---------------------------------------------------------------------------
+ * Which pixels are "near and within non-background objects" (Section 5.2; the paper gives no distance):
+ * a pixel gets weight `factor` if any pixel within `radius` rows and columns of it (a square window, cut at the
+ * frame border) carries a label other than `background`, weight 1 otherwise.  Brute force over the window.
+ * ------------------------------------------------------------------------- */
+void so_object_weights(const uint8_t *lab, int H, int W, int background, int radius, int factor, uint8_t *wgt)
+{
+#pragma omp parallel for
+    for (int y = 0; y < H; ++y)
+        for (int x = 0; x < W; ++x) {
+            int near = 0;
+            for (int dy = -radius; dy <= radius && !near; ++dy)
+                for (int dx = -radius; dx <= radius; ++dx) {
+                    const int yy = y + dy, xx = x + dx;
+                    if (yy < 0 || yy >= H || xx < 0 || xx >= W) continue;
+                    if (lab[(int64_t)yy * W + xx] != background) { near = 1; break; }
+                }
+            wgt[(int64_t)y * W + x] = (uint8_t)(near ? factor : 1);
+        }
 }
 
 /* ---------------------------------------------------------------------------

@@ -440,3 +440,70 @@ def test_head_with_adam_takes_textbook_steps_on_the_real_gradient():
         np.testing.assert_allclose(head.theta, th, rtol=2e-5, atol=2e-7)
         th = head.theta.astype(np.float64)                               # follow the fp32 trajectory
         m, v = head.vel.astype(np.float64), head.vel2.astype(np.float64)
+
+
+# ---------------------------------------------------------------------------- loss weighting near objects (Section 5.2)
+def test_object_weights_are_a_square_dilation_of_the_non_background_mask():
+    ndimage = pytest.importorskip("scipy.ndimage")
+    rng = np.random.default_rng(21)
+    for H, W, r, bg in [(9, 13, 1, 0), (20, 17, 3, 2), (6, 6, 0, 0), (5, 30, 8, 1)]:
+        lab = np.full((H, W), bg, np.uint8)
+        for _ in range(3):
+            y, x = rng.integers(0, H), rng.integers(0, W)
+            lab[y:y + rng.integers(1, 3), x:x + rng.integers(1, 4)] = (bg + 1 + rng.integers(0, 3)) % 5 if bg != 4 else 0
+        got = oracle.object_weights(lab, bg, r, 5)
+        near = ndimage.maximum_filter((lab != bg).astype(np.uint8), size=2 * r + 1, mode="constant", cval=0).astype(bool)
+        np.testing.assert_array_equal(got, np.where(near, 5, 1))
+        assert ((got == 5) | (got == 1)).all() and (got[lab != bg] == 5).all()      # "within" objects is always weighted
+    # hand case: one object pixel in the middle of a 5x7 background, radius 1 -> a 3x3 block of fives
+    lab = np.zeros((5, 7), np.uint8); lab[2, 3] = 4
+    exp = np.ones((5, 7), np.uint8); exp[1:4, 2:5] = 5
+    np.testing.assert_array_equal(oracle.object_weights(lab, 0, 1, 5), exp)
+    # at the frame corner the window is cut, not wrapped
+    lab = np.zeros((4, 4), np.uint8); lab[0, 0] = 1
+    exp = np.ones((4, 4), np.uint8); exp[:3, :3] = 5
+    np.testing.assert_array_equal(oracle.object_weights(lab, 0, 2, 5), exp)
+
+
+def test_weighted_loss_is_the_plain_loss_plus_four_times_the_near_object_part():
+    rng = np.random.default_rng(22)
+    C, H, W = 4, 12, 16
+    u = rng.standard_normal((C, H, W)) * 2
+    lab = rng.integers(0, C, (H, W)).astype(np.uint8)
+    wgt = np.where(rng.random((H, W)) < 0.3, 5, 1).astype(np.uint8)
+    loss_w, g_w, _ = oracle.softmax_ce(u, lab, weights=wgt)
+    loss_1, g_1, _ = oracle.softmax_ce(u, lab)                               # the unweighted function, pinned above
+    heavy = wgt == 5
+    n = int(heavy.sum())
+    loss_h, _, _ = oracle.softmax_ce(u[:, heavy].reshape(C, 1, n), lab[heavy].reshape(1, n))   # mean over the heavy pixels alone
+    assert loss_w == pytest.approx(loss_1 + 4.0 * loss_h * n / (H * W), rel=1e-12)
+    np.testing.assert_allclose(g_w, g_1 * wgt[None], rtol=1e-12, atol=1e-18)
+    # factor 1 everywhere is the plain loss, bit for bit
+    l1, g1, _ = oracle.softmax_ce(u, lab, weights=np.ones((H, W), np.uint8))
+    assert l1 == pytest.approx(loss_1, rel=1e-14) and g1.tobytes() == g_1.tobytes()
+
+
+def test_weighted_head_gradient_by_finite_differences_and_background_only_frames():
+    rng = np.random.default_rng(23)
+    cin, C, h, w = 3, 3, 3, 5
+    feat = np.abs(rng.standard_normal((cin, h, w))) + 0.1
+    lab = np.zeros((4 * h, 4 * w), np.uint8); lab[3:6, 4:9] = 1; lab[8, 15] = 2
+    n = si.head_param_count(cin, 0, C)
+    theta = rng.standard_normal(n) * 0.5
+    kw = dict(dtype=np.float64, object_weight=5, object_radius=2, background=0)
+    loss, grad, _ = oracle.gradients(oracle.Head(cin, 0, C, theta=theta, **kw), feat, lab)
+    wgt = oracle.object_weights(lab, 0, 2, 5)
+    assert 0 < (wgt == 5).mean() < 1
+
+    def f(th):
+        z, _ = oracle.head_forward(oracle.Head(cin, 0, C, dtype=np.float64, theta=th), feat)
+        return oracle.softmax_ce(oracle.upsample(z, 4), lab, want_grad=False, weights=wgt)[0]
+
+    fd = np.array([(f(theta + 1e-6 * e) - f(theta - 1e-6 * e)) / 2e-6 for e in np.eye(n)])
+    assert np.abs(fd - grad).max() / np.abs(fd).max() < 1e-6
+    assert loss == pytest.approx(f(theta), rel=1e-12)
+    # a frame with no object: the weighted head computes exactly what the plain head computes
+    bgl = np.zeros_like(lab)
+    a = oracle.gradients(oracle.Head(cin, 0, C, theta=theta, **kw), feat, bgl)
+    b = oracle.gradients(oracle.Head(cin, 0, C, theta=theta, dtype=np.float64), feat, bgl)
+    assert a[0] == pytest.approx(b[0], rel=1e-14) and a[1].tobytes() == b[1].tobytes()   # (the loss is an OpenMP reduction)
