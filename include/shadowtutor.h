@@ -73,6 +73,13 @@ typedef struct st_head_desc {
     double adam_beta1;      /* Adam's decay rates and epsilon; the paper does not state them.  0 selects the */
     double adam_beta2;      /*   constants of the published algorithm: 0.9, 0.999, 1e-8.                       */
     double adam_eps;        /* epsilon is added to the root of the bias-corrected second moment */
+    int32_t object_weight;  /* loss weighting against class imbalance (Section 5.2): the cross-entropy of pixels near
+                               and within non-background objects is scaled by this factor (5 in the paper; whole
+                               numbers 2..5; 0 or 1 = off, plain mean cross-entropy).  The normaliser stays the
+                               number of pixels.  Needs n_classes <= 32. */
+    int32_t object_radius;  /* what counts as "near" (the paper gives no distance): within this many rows and
+                               columns of a pixel whose label is not the background class; 0..64 */
+    int32_t background_class; /* the background class, below n_classes */
 } st_head_desc;
 
 /* Number of fp32 values in one head's packed parameter buffer:

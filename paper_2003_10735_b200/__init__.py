@@ -51,7 +51,8 @@ class st_head_desc(ctypes.Structure):
         ("up", ctypes.c_int32), ("gemm_precision", ctypes.c_int32),
         ("lr", ctypes.c_float), ("momentum", ctypes.c_float), ("cuda_stream", ctypes.c_void_p),
         ("optimizer", ctypes.c_int32), ("adam_beta1", ctypes.c_double), ("adam_beta2", ctypes.c_double),
-        ("adam_eps", ctypes.c_double),
+        ("adam_eps", ctypes.c_double), ("object_weight", ctypes.c_int32), ("object_radius", ctypes.c_int32),
+        ("background_class", ctypes.c_int32),
     ]
 
 
@@ -184,10 +185,12 @@ def st_param_count(c_in: int, c_hidden: int, n_classes: int) -> int:
 def st_init_head(*, n_streams: int = 1, c_in: int, c_hidden: int = 0, n_classes: int, feat_h: int,
                  feat_w: int, up: int = 4, gemm_precision: int = 0, lr: float = 0.01, momentum: float = 0.0,
                  cuda_stream: int = 0, init_params, optimizer: int = 0, adam_beta1: float = 0.0,
-                 adam_beta2: float = 0.0, adam_eps: float = 0.0) -> _Ctx:
+                 adam_beta2: float = 0.0, adam_eps: float = 0.0, object_weight: int = 0, object_radius: int = 0,
+                 background_class: int = 0) -> _Ctx:
     lib = load_library()
     desc = st_head_desc(n_streams, c_in, c_hidden, n_classes, feat_h, feat_w, up, gemm_precision,
-                        lr, momentum, cuda_stream or None, optimizer, adam_beta1, adam_beta2, adam_eps)
+                        lr, momentum, cuda_stream or None, optimizer, adam_beta1, adam_beta2, adam_eps,
+                        object_weight, object_radius, background_class)
     n = n_streams * int(lib.st_param_count(c_in, c_hidden, n_classes))
     out = ctypes.c_void_p()
     status = lib.st_init_head(ctypes.byref(desc), _ptr(init_params, "float32", n, "init_params"), ctypes.byref(out))

@@ -233,6 +233,13 @@ upsample_ce_rows_kernel(UpsampleCeArgs a, const __grid_constant__ CUtensorMap z_
         labw[r] = lo | (hi << 16);
         vb[r] = (((vmask >> (4 * r)) & 0x3u) ? 0x00000101u : 0u) | (((vmask >> (4 * r)) & 0xcu) ? 0x01010000u : 0u);
     }
+    // loss weighting (Section 5.2): bit 7 of a label byte marks a pixel near / within a non-background object
+    uint32_t hv[4] = {0, 0, 0, 0};                         // 0x01 in the byte of each weighted pixel
+    const int hw1 = a.heavy_w - 1;                         // what a weighted pixel counts on top of 1
+    if (hw1 > 0) {                                         // block-uniform
+#pragma unroll
+        for (int r = 0; r < 4; ++r) { hv[r] = (labw[r] >> 7) & 0x01010101u; labw[r] &= 0x7f7f7f7fu; }
+    }
     float m_loc = -INFINITY;                               // largest logit of this thread's share of the tile
     {
         // a thread keeps one 16-byte group of the tile plane (81 groups) and walks the classes three at a time
@@ -354,13 +361,14 @@ upsample_ce_rows_kernel(UpsampleCeArgs a, const __grid_constant__ CUtensorMap z_
             if (valid && lab[k] >= C) { if (own) n_bad++; lab[k] = -1; }
             if (!valid) lab[k] = -1;
             float rz = 0.f;
+            const float wk = ((hv[r] >> (8 * k)) & 1u) ? (float)a.heavy_w : 1.0f;
             if (lab[k] >= 0) {
-                rz = rcp_approx(Zs[k]);
+                rz = rcp_approx(Zs[k]) * wk;
                 if (own) {
                     const float* q = rc.za + lab[k] * TZ;
                     const float vl = fmaf(ly, q[TZ_W] - q[0], q[0]), vr = fmaf(ly, q[TZ_W + 1] - q[1], q[1]);
                     const float ul = fmaf(fmaf((2 * k + 1) * 0.125f, vr - vl, vl), kLog2e, -rc.M) - sk[k];
-                    loss += (__log2f(Zs[k]) - ul) * kLn2;
+                    loss += wk * (__log2f(Zs[k]) - ul) * kLn2;
                     if (CONF) atomicAdd(&hist[lab[k] * C + arg[k]], 1u);
                 }
             }
@@ -369,7 +377,7 @@ upsample_ce_rows_kernel(UpsampleCeArgs a, const __grid_constant__ CUtensorMap z_
             wr[k] = (fold_r ? 0.f : (fold_l ? 1.0f : fr)) * rz;
         }
         // four valid pixels with one label (the usual case): their onehot parts add up to 16 eighths per side
-        if (lab[0] >= 0 && lab[0] == lab[1] && lab[1] == lab[2] && lab[2] == lab[3]) {
+        if (hw1 == 0 && lab[0] >= 0 && lab[0] == lab[1] && lab[1] == lab[2] && lab[2] == lab[3]) {
             int* cc = corr + lab[0] * TZ;
             atomicAdd(cc + ry_top * TZ_W + rx_l, -wy0 * 16);
             atomicAdd(cc + ry_top * TZ_W + rx_r, -wy0 * 16);
@@ -379,7 +387,8 @@ upsample_ce_rows_kernel(UpsampleCeArgs a, const __grid_constant__ CUtensorMap z_
 #pragma unroll
             for (int k = 0; k < 4; ++k)
                 if (lab[k] >= 0) {
-                    const int wb = 2 * k + 1, wa = 8 - wb;       // eighths toward node columns n+1 / n
+                    const int iw = ((hv[r] >> (8 * k)) & 1u) ? a.heavy_w : 1;
+                    const int wb = (2 * k + 1) * iw, wa = (7 - 2 * k) * iw;       // eighths toward node columns n+1 / n, times the weight
                     int* cc = corr + lab[k] * TZ;
                     atomicAdd(cc + ry_top * TZ_W + rx_l, -wy0 * wa);
                     atomicAdd(cc + ry_top * TZ_W + rx_r, -wy0 * wb);
@@ -419,7 +428,7 @@ upsample_ce_rows_kernel(UpsampleCeArgs a, const __grid_constant__ CUtensorMap z_
 #pragma unroll
             for (int r = 0; r < 4; ++r) {
                 rem[r] = __vcmpltu4(labw[r], C4) & vb[r];
-                n_ok += __popc(rem[r]);
+                n_ok += __popc(rem[r]) + hw1 * __popc(rem[r] & hv[r]);      // the weights of the pixels that count
                 if (own_cell) n_bad += __popc(rem[r] ^ vb[r]);
             }
             if (CONF) {                                              // the student's class: arg-max of the interpolated logits
@@ -440,8 +449,9 @@ upsample_ce_rows_kernel(UpsampleCeArgs a, const __grid_constant__ CUtensorMap z_
             for (int j = 0; j < 16; ++j) {
                 const bool ok = (rem[j >> 2] >> (8 * (j & 3))) & 1u;
                 const float fr = (2 * (j & 3) + 1) * 0.125f;
-                const float rz = ok ? rcp_approx(Z[j]) : 0.f;
-                lz += ok ? __log2f(Z[j]) : 0.f;
+                const float wj = ((hv[j >> 2] >> (8 * (j & 3))) & 1u) ? (float)a.heavy_w : 1.0f;
+                const float rz = ok ? rcp_approx(Z[j]) * wj : 0.f;
+                lz += ok ? wj * __log2f(Z[j]) : 0.f;
                 wl[j] = (fold_l ? 0.f : (fold_r ? 1.0f : 1.0f - fr)) * rz;
                 wr[j] = (fold_r ? 0.f : (fold_l ? 1.0f : fr)) * rz;
             }
@@ -461,10 +471,11 @@ upsample_ce_rows_kernel(UpsampleCeArgs a, const __grid_constant__ CUtensorMap z_
                 for (int r = 0; r < 4; ++r) {
                     const uint32_t eq = __vcmpeq4(labw[r], cur4) & rem[r];
                     rem[r] ^= eq;
-                    tl = __dp4a(eq, corner_weights(7 - 2 * r, false), tl);
-                    tr = __dp4a(eq, corner_weights(7 - 2 * r, true), tr);
-                    bl = __dp4a(eq, corner_weights(2 * r + 1, false), bl);
-                    br = __dp4a(eq, corner_weights(2 * r + 1, true), br);
+                    const uint32_t ew = eq + (eq & hv[r]) * (uint32_t)hw1;          // each byte: the pixel's weight (1..5) or 0
+                    tl = __dp4a(ew, corner_weights(7 - 2 * r, false), tl);
+                    tr = __dp4a(ew, corner_weights(7 - 2 * r, true), tr);
+                    bl = __dp4a(ew, corner_weights(2 * r + 1, false), bl);
+                    br = __dp4a(ew, corner_weights(2 * r + 1, true), br);
                 }
                 int* cc = c_tl + cur * TZ;
                 atomicAdd(cc, -(int)tl);

@@ -44,6 +44,8 @@ struct st_ctx {
     float* x_f32 = nullptr;
     bf16* x_bf16 = nullptr;
     uint8_t* labels = nullptr;
+    uint8_t* labels_tagged = nullptr;       // [S][P] labels with bit 7 = near / within an object (loss weighting on)
+    int heavy_w = 1, heavy_radius = 0, background = 0;
     float *z = nullptr, *dz = nullptr;
     bf16* dz_bf16 = nullptr;
     int64_t dz_pitch = 0;
@@ -234,11 +236,22 @@ st_status enqueue_forward(st_ctx* c, StageTimer* t = nullptr, const int* skip = 
 // Arguments of the fused upsample + cross-entropy kernel.  With bf16 GEMMs the weight gradient and the dgrad read the
 // bf16 copy of the logit gradient only, so the fp32 copy is not written during a step (st_read_tensor produces it on
 // demand by running the kernel once more on the same logits and labels).
+// With the loss weighting on, the per-key-frame pass that marks the pixels near / within non-background objects.
+st_status tag_labels(st_ctx* c, int32_t stream)
+{
+    if (c->heavy_w <= 1) return ST_OK;
+    launch_object_weight_tags(c->labels + (int64_t)stream * c->P, c->H, c->W, c->background, c->heavy_radius, c->mask_tmp,
+                              c->labels_tagged + (int64_t)stream * c->P, c->stream);
+    c->launches += 2;
+    return check_launch(c, "object weights");
+}
+
 UpsampleCeArgs k3_args(st_ctx* c, bool fp32_grad, bool bf16_grad, unsigned long long* conf, const int* skip = nullptr,
                        int64_t skip_stride = 0)
 {
     UpsampleCeArgs k3;
-    k3.z = c->z; k3.labels = c->labels;
+    k3.z = c->z; k3.labels = c->heavy_w > 1 ? c->labels_tagged : c->labels;
+    k3.heavy_w = c->heavy_w;
     k3.dz = fp32_grad ? c->dz : nullptr;
     k3.dz_bf16 = bf16_grad ? c->dz_bf16 : nullptr;
     k3.dz_bf16_pitch = c->dz_pitch;
@@ -397,6 +410,12 @@ st_status st_init_head(const st_head_desc* desc, const float* init_params, st_ct
     const double aeps = d.adam_eps == 0.0 ? 1e-8 : d.adam_eps;
     if (d.optimizer == 1 && (!(ab1 > 0.0 && ab1 < 1.0) || !(ab2 > 0.0 && ab2 < 1.0) || !(aeps > 0.0)))
         return fail(nullptr, ST_ERR_INVALID_ARG, "st_init_head: Adam needs beta1, beta2 in (0, 1) and eps > 0");
+    if (d.object_weight > 1) {
+        if (d.object_radius < 0 || d.background_class < 0 || d.background_class >= d.n_classes)
+            return fail(nullptr, ST_ERR_INVALID_ARG, "st_init_head: loss weighting needs object_radius >= 0 and a background class below n_classes");
+        if (d.object_weight > 5 || d.object_radius > 64 || !upsample_ce_rows_supported(d.n_classes))
+            return fail(nullptr, ST_ERR_UNSUPPORTED, "st_init_head: loss weighting covers weights 2..5, radii up to 64 and at most 32 classes");
+    }
     if (d.gemm_precision != 0 && d.gemm_precision != 1)
         return fail(nullptr, ST_ERR_INVALID_ARG, "st_init_head: gemm_precision must be 0 or 1");
     if (d.up != kUp) return fail(nullptr, ST_ERR_UNSUPPORTED, "st_init_head: up must be 4");
@@ -420,6 +439,7 @@ st_status st_init_head(const st_head_desc* desc, const float* init_params, st_ct
     c->n_params = (int64_t)st_param_count(d.c_in, d.c_hidden, d.n_classes);
     c->bf16_mode = d.gemm_precision == 1;
     c->adam = d.optimizer == 1; c->b1 = ab1; c->b2 = ab2; c->eps = aeps;
+    c->heavy_w = d.object_weight > 1 ? d.object_weight : 1; c->heavy_radius = d.object_radius; c->background = d.background_class;
     c->has_feat.assign(c->S, 0); c->has_labels.assign(c->S, 0);
     // The legacy default stream cannot be captured: steps are then enqueued kernel by kernel.
     c->use_graphs = c->stream != nullptr && c->stream != cudaStreamLegacy && c->stream != cudaStreamPerThread;
@@ -447,6 +467,7 @@ st_status st_init_head(const st_head_desc* desc, const float* init_params, st_ct
     ALLOC(step_base, S);
     if (c->adam) ALLOC(vel2, S * c->n_params);
     ALLOC(labels, S * c->P);
+    if (c->heavy_w > 1) ALLOC(labels_tagged, S * c->P);
     ALLOC(z, S * c->C * c->p); ALLOC(dz, S * c->C * c->p);
     ALLOC(loss_part, S * c->n_k3_blocks); ALLOC(db_part, (size_t)S * c->n_k3_blocks * c->C);
     ALLOC(loss_buf, S * kMaxSteps);
@@ -555,7 +576,7 @@ st_status st_teacher_labels(st_ctx* ctx, int32_t stream, const float* logits_chw
     if (st != ST_OK) return st;
     if (labels_out) ST_CUDA(ctx, cudaMemcpyAsync(labels_out, dst, (size_t)ctx->P, cudaMemcpyDefault, ctx->stream));
     ctx->has_labels[stream] = 1;
-    return ST_OK;
+    return tag_labels(ctx, stream);
 }
 
 st_status st_set_labels(st_ctx* ctx, int32_t stream, const uint8_t* labels)
@@ -565,7 +586,7 @@ st_status st_set_labels(st_ctx* ctx, int32_t stream, const uint8_t* labels)
     if (!labels) return fail(ctx, ST_ERR_INVALID_ARG, "st_set_labels: NULL labels");
     ST_CUDA(ctx, cudaMemcpyAsync(ctx->labels + (int64_t)stream * ctx->P, labels, (size_t)ctx->P, cudaMemcpyDefault, ctx->stream));
     ctx->has_labels[stream] = 1;
-    return ST_OK;
+    return tag_labels(ctx, stream);
 }
 
 st_status st_distill_step(st_ctx* ctx, int32_t n_steps, float* loss_out, int64_t* conf_out)

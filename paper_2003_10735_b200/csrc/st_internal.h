@@ -55,6 +55,11 @@ void launch_feat_to_bf16_nhwc(const float* feat_chw, int Cin, int64_t p, bf16* o
 // reverse (verification only): bf16 [p][C] -> fp32 [C][p]
 void launch_nhwc_bf16_to_chw(const bf16* in, int C, int64_t p, float* out, cudaStream_t s);
 
+// ---- loss weighting near objects: labels [H][W] of one stream -> labels with bit 7 set where the pixel is within
+// `radius` of a non-background pixel; tmp is a scratch map of H*W bytes
+void launch_object_weight_tags(const uint8_t* labels, int H, int W, int background, int radius, uint8_t* tmp, uint8_t* tagged,
+                               cudaStream_t s);
+
 // ---- K3: upsample x4 + softmax cross-entropy + gradient w.r.t. the low-res logits ---------------
 struct UpsampleCeArgs {
     const float* z;          // [S][C][h][w]
@@ -72,6 +77,8 @@ struct UpsampleCeArgs {
     int has_map;             // the launch carries a tile map of z (see make_logit_tile_map)
     const int* skip;         // nullptr, or one flag per stream (skip[s * skip_stride]): non-zero = the stream's blocks return at once
     int64_t skip_stride;
+    int heavy_w;             // 1, or the integer weight (2..5) of the pixels whose label byte has bit 7 set
+                             //   (`labels` is then the tagged map made by launch_object_weight_tags)
 };
 // Tile map of the logits for the row-walking kernel: fp32 tensor {w, h, S*C}, one box = the block's tile of all
 // classes.  False if the shape does not allow it (w not a multiple of 4, C > 32) or the driver entry point is
