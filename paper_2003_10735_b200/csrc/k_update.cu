@@ -21,10 +21,11 @@ constexpr int kUpdThreads = 256;
 
 // Bias corrections of Adam's step t: (1 - b1^t, 1 - b2^t), t = steps taken before this call + position in the call.
 struct AdamCorr { double c1, c2; };
+template <bool ADAM>
 __device__ __forceinline__ AdamCorr adam_corrections(const UpdateArgs& a, int s)
 {
     AdamCorr c = {1.0, 1.0};
-    if (a.adam) {
+    if (ADAM) {
         const double t = (double)(a.step_base[s] + a.loss_slot + 1);
         c.c1 = 1.0 - exp(t * a.ln_b1);
         c.c2 = 1.0 - exp(t * a.ln_b2);
@@ -35,10 +36,11 @@ __device__ __forceinline__ AdamCorr adam_corrections(const UpdateArgs& a, int s)
 // OptimStep on one parameter.  Gradient descent with momentum: v <- mu v + g; theta <- theta - lr v.
 // Adam (each element in double, stored as fp32): m <- b1 m + (1 - b1) g; v <- b2 v + (1 - b2) g^2;
 // theta <- theta - lr (m / c1) / (sqrt(v / c2) + eps).
+template <bool ADAM>
 __device__ __forceinline__ void apply_update(const UpdateArgs& a, int64_t gi, float g, const AdamCorr& k)
 {
     a.grad[gi] = g;
-    if (a.adam) {
+    if (ADAM) {
         const double gd = (double)g;
         const double m = a.b1 * (double)a.vel[gi] + (1.0 - a.b1) * gd;
         const double v = a.b2 * (double)a.vel2[gi] + (1.0 - a.b2) * gd * gd;
@@ -55,7 +57,7 @@ __device__ __forceinline__ void apply_update(const UpdateArgs& a, int64_t gi, fl
 // Parameter blocks: a block covers kUpdThreads / G consecutive parameters; the G thread groups of a
 // block each sum every G-th split-K partial of "their" parameter (coalesced along the parameters),
 // the group sums are added in group order through shared memory, and group 0 applies the update.
-template <int G, int E>
+template <int G, int E, bool ADAM>
 __global__ void __launch_bounds__(kUpdThreads)
 sgd_update_kernel(UpdateArgs a, int n_param_blocks, int64_t range_begin)
 {
@@ -67,7 +69,7 @@ sgd_update_kernel(UpdateArgs a, int n_param_blocks, int64_t range_begin)
     const int s = blockIdx.y;
     const int64_t base = (int64_t)s * a.n_params;
     const bool skip = a.skip && a.skip[(int64_t)s * a.skip_stride];   // block-uniform
-    const AdamCorr corr = adam_corrections(a, s);
+    const AdamCorr corr = adam_corrections<ADAM>(a, s);
     if ((int)blockIdx.x < n_param_blocks) {
         if (skip) return;
         const int col = threadIdx.x % kRow, g = threadIdx.x / kRow;
@@ -124,10 +126,10 @@ sgd_update_kernel(UpdateArgs a, int n_param_blocks, int64_t range_begin)
                 } else {
                     gr = a.grad[base + i];
                 }
-                apply_update(a, base + i, gr, corr);
+                apply_update<ADAM>(a, base + i, gr, corr);
                 if (ly.shadow) ly.shadow[(int64_t)s * ly.shadow_stream_stride + (i - ly.w_off)] = __float2bfloat16_rn(a.theta[base + i]);
             } else if (!ly.b_partials) {
-                apply_update(a, base + i, a.grad[base + i], corr);
+                apply_update<ADAM>(a, base + i, a.grad[base + i], corr);
             }   // biases with partial sums are finished by the reduction warps below
         }
         return;
@@ -154,7 +156,7 @@ sgd_update_kernel(UpdateArgs a, int n_param_blocks, int64_t range_begin)
             }
 #pragma unroll
             for (int o = 16; o > 0; o >>= 1) g += __shfl_xor_sync(0xffffffffu, g, o);
-            if (lane == 0 && !skip) apply_update(a, base + ly.b_off + item, g, corr);
+            if (lane == 0 && !skip) apply_update<ADAM>(a, base + ly.b_off + item, g, corr);
             return;
         }
         item -= ly.cout;
@@ -182,7 +184,7 @@ sgd_update_kernel(UpdateArgs a, int n_param_blocks, int64_t range_begin)
 
 // A large weight tensor with a moderate number of split-K partials (the 3x3 layer): a pure stream.
 // Each thread owns VEC consecutive weights and reads them from every partial with all loads in flight.
-template <int VEC>
+template <int VEC, bool ADAM>
 __global__ void __launch_bounds__(256)
 sgd_update_stream_kernel(UpdateArgs a, int L)
 {
@@ -216,15 +218,16 @@ sgd_update_stream_kernel(UpdateArgs a, int L)
         }
     }
     const int64_t gi = (int64_t)s * a.n_params + ly.w_off + e;
-    const AdamCorr corr = adam_corrections(a, s);
+    const AdamCorr corr = adam_corrections<ADAM>(a, s);
 #pragma unroll
     for (int j = 0; j < VEC; ++j) {
-        apply_update(a, gi + j, g[j], corr);
+        apply_update<ADAM>(a, gi + j, g[j], corr);
         if (ly.shadow) ly.shadow[(int64_t)s * ly.shadow_stream_stride + e + j] = __float2bfloat16_rn(a.theta[gi + j]);
     }
 }
 
-int launch_sgd_update(const UpdateArgs& a, cudaStream_t s)
+template <bool ADAM>
+static int launch_sgd_update_t(const UpdateArgs& a, cudaStream_t s)
 {
     int n_launches = 1;
     // large layers with partial sums go through the streaming kernel; everything else (small layers, biases,
@@ -236,8 +239,8 @@ int launch_sgd_update(const UpdateArgs& a, cudaStream_t s)
         if (ly.w_partials && nw >= 65536 && ly.w_off == range_begin) {
             const bool vec = nw % 4 == 0 && ly.w_split_stride % 4 == 0 && ly.w_stream_stride % 4 == 0 &&
                              ((uintptr_t)ly.w_partials % 16 == 0);
-            if (vec) launch_chain(sgd_update_stream_kernel<4>, dim3((unsigned)((nw / 4 + 255) / 256), (unsigned)a.S), dim3(256), 0, s, a, L);
-            else launch_chain(sgd_update_stream_kernel<1>, dim3((unsigned)((nw + 255) / 256), (unsigned)a.S), dim3(256), 0, s, a, L);
+            if (vec) launch_chain(sgd_update_stream_kernel<4, ADAM>, dim3((unsigned)((nw / 4 + 255) / 256), (unsigned)a.S), dim3(256), 0, s, a, L);
+            else launch_chain(sgd_update_stream_kernel<1, ADAM>, dim3((unsigned)((nw + 255) / 256), (unsigned)a.S), dim3(256), 0, s, a, L);
             range_begin = ly.w_off + nw;
             ++n_launches;
         }
@@ -256,12 +259,17 @@ int launch_sgd_update(const UpdateArgs& a, cudaStream_t s)
     const int n_param_blocks = (int)((n_rest + per - 1) / per);
     const dim3 grid((unsigned)(n_param_blocks + n_red_blocks), (unsigned)a.S);
     const dim3 blk(kUpdThreads);
-    if (G == 1 && E == 1) launch_chain(sgd_update_kernel<1, 1>, grid, blk, 0, s, a, n_param_blocks, range_begin);
-    else if (G == 1) launch_chain(sgd_update_kernel<1, 4>, grid, blk, 0, s, a, n_param_blocks, range_begin);
-    else if (G == 16) launch_chain(sgd_update_kernel<16, 1>, grid, blk, 0, s, a, n_param_blocks, range_begin);
-    else if (E == 1) launch_chain(sgd_update_kernel<8, 1>, grid, blk, 0, s, a, n_param_blocks, range_begin);
-    else launch_chain(sgd_update_kernel<8, 4>, grid, blk, 0, s, a, n_param_blocks, range_begin);
+    if (G == 1 && E == 1) launch_chain(sgd_update_kernel<1, 1, ADAM>, grid, blk, 0, s, a, n_param_blocks, range_begin);
+    else if (G == 1) launch_chain(sgd_update_kernel<1, 4, ADAM>, grid, blk, 0, s, a, n_param_blocks, range_begin);
+    else if (G == 16) launch_chain(sgd_update_kernel<16, 1, ADAM>, grid, blk, 0, s, a, n_param_blocks, range_begin);
+    else if (E == 1) launch_chain(sgd_update_kernel<8, 1, ADAM>, grid, blk, 0, s, a, n_param_blocks, range_begin);
+    else launch_chain(sgd_update_kernel<8, 4, ADAM>, grid, blk, 0, s, a, n_param_blocks, range_begin);
     return n_launches;
+}
+
+int launch_sgd_update(const UpdateArgs& a, cudaStream_t s)
+{
+    return a.adam ? launch_sgd_update_t<true>(a, s) : launch_sgd_update_t<false>(a, s);
 }
 
 __global__ void step_tick_kernel(long long* step_base, int S, int add, const int* add_per_stream)
