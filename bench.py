@@ -361,7 +361,7 @@ def run_ours(args, cfg):
         result = None
         if rank == 0:
             ms_step = ms_total / args.steps
-            value = whole_job_rate(K * args.steps, world, ms_total)
+            value = whole_job_rate(K * S * args.steps, world, ms_total)      # SGD iterations of all streams of all ranks
             dominant = max((n for n in kernels if "frac" in kernels[n] or True),
                            key=lambda n: kernels[n]["ms"] * kernels[n]["per_key_frame"])
             dk = kernels[dominant]
@@ -382,12 +382,12 @@ def run_ours(args, cfg):
                            "l2": f"inputs rotate over {N_SETS} key frames ({N_SETS * S * (cfg.c_in * p + C * P) * 4 / 1e6:.0f} MB) > 126 MB L2",
                            "parallelism": f"replicas x{world}, no collective"},
                 "clocks": clock_info,
-                "e2e": {"value": world * K * e2e_steps / (ms_e2e / 1e3), "unit": "steps/s", "h2d_bytes_per_step": h2d,
+                "e2e": {"value": world * K * S * e2e_steps / (ms_e2e / 1e3), "unit": "steps/s", "h2d_bytes_per_step": h2d,
                         "d2h_bytes_per_step": d2h, "ms_per_step": ms_e2e / e2e_steps},
                 "gpu_launches": int(launches),
                 "roofline": roofline,
                 "key_frames_per_s": world * args.steps / (ms_total / 1e3),
-                "distill_loop_only": {"steps_per_s": K / (ms_loop / 1e3), "ms_per_k_steps": ms_loop},
+                "distill_loop_only": {"steps_per_s": K * S / (ms_loop / 1e3), "ms_per_k_steps": ms_loop},
                 "kernels": kernels,
                 "last_loss": float(loss_d[0, -1].item()), "last_miou": mious[0], "last_miou_device_run": last_miou_dev,
             }

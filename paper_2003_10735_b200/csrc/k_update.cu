@@ -305,9 +305,18 @@ void launch_refresh_shadow(const UpdateArgs& a, cudaStream_t s)
 
 // Mean IoU (Section 3.2): IoU_c = conf[c][c] / (row_c + col_c - conf[c][c]), averaged over the
 // classes present in the label (row_c > 0).  Integer counts, double arithmetic, fixed order.
-// Called by all 256 threads of a block; the value is returned to thread 0 only.
-__device__ __forceinline__ double block_miou(const unsigned long long* __restrict__ conf, int C, double* iou, int* present)
+// Called by all 256 threads of a block; the value is returned to thread 0 only.  Matrices of up to kMiouStage classes
+// are first copied to shared memory in one coalesced pass (one memory latency instead of one per row element).
+constexpr int kMiouStage = 32;
+__device__ __forceinline__ double block_miou(const unsigned long long* __restrict__ conf_g, int C, double* iou, int* present)
 {
+    __shared__ unsigned long long staged[kMiouStage * kMiouStage];
+    const unsigned long long* conf = conf_g;
+    if (C <= kMiouStage) {                                 // block-uniform
+        for (int e = threadIdx.x; e < C * C; e += blockDim.x) staged[e] = conf_g[e];
+        __syncthreads();
+        conf = staged;
+    }
     const int c = threadIdx.x;
     double v = 0.0; int pr = 0;
     if (c < C) {

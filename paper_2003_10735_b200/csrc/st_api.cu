@@ -77,6 +77,7 @@ struct st_ctx {
     float* read_tmp = nullptr; size_t read_tmp_bytes = 0;
     void* staging = nullptr; size_t staging_bytes = 0;
     std::vector<char> has_feat, has_labels;
+    bool z_current = false;                 // z holds the forward of the current parameters and features of every stream
     TcPlan* plan = nullptr;
     struct StepGraph { cudaGraphExec_t exec; int64_t n_launches; };
     std::map<GraphKey, StepGraph> graphs;
@@ -558,6 +559,7 @@ st_status st_set_frozen_features(st_ctx* ctx, int32_t stream, const float* feat_
         ST_CUDA(ctx, cudaMemcpyAsync(ctx->x_f32 + (int64_t)stream * ctx->Cin * ctx->p, feat_chw, bytes, cudaMemcpyDefault, ctx->stream));
     }
     ctx->has_feat[stream] = 1;
+    ctx->z_current = false;
     return ST_OK;
 }
 
@@ -600,6 +602,7 @@ st_status st_distill_step(st_ctx* ctx, int32_t n_steps, float* loss_out, int64_t
                         ctx->has_feat[s] ? "labels" : "frozen features");
     const bool want_conf = conf_out != nullptr;
     const size_t cc = (size_t)ctx->C * ctx->C;
+    ctx->z_current = false;                 // the steps leave z at the forward before the last update
     if (want_conf) {
         if (!ctx->conf_buf) {
             cudaError_t e = dev_alloc(ctx, &ctx->conf_buf, (size_t)ctx->S * kMaxSteps * cc);
@@ -701,6 +704,7 @@ st_status st_train_key_frame(st_ctx* ctx, double threshold, int32_t max_updates,
             return fail(ctx, ST_ERR_BAD_STATE, "st_train_key_frame: stream %d has no %s yet", s,
                         ctx->has_feat[s] ? "labels" : "frozen features");
     const size_t cc = (size_t)ctx->C * ctx->C;
+    ctx->z_current = false;
     cudaError_t e = cudaSuccess;
     if (!ctx->conf_buf) e = dev_alloc(ctx, &ctx->conf_buf, (size_t)ctx->S * kMaxSteps * cc);
     if (e == cudaSuccess && !ctx->best_theta) {
@@ -780,6 +784,7 @@ st_status st_profile_step(st_ctx* ctx, int32_t n_steps, int32_t* n_stages, float
     for (int s = 0; s < ctx->S; ++s)
         if (!ctx->has_feat[s] || !ctx->has_labels[s])
             return fail(ctx, ST_ERR_BAD_STATE, "st_profile_step: stream %d has no features or labels yet", s);
+    ctx->z_current = false;
     StageTimer t;
     t.repeat = 8;
     for (int i = 0; i <= StageTimer::kMax; ++i) ST_CUDA(ctx, cudaEventCreate(&t.ev[i]));
@@ -844,6 +849,7 @@ st_status st_apply_update(st_ctx* ctx, int32_t stream, const void* src, size_t n
     const void* dev = nullptr;
     st = to_device(ctx, src, need, &dev);
     if (st != ST_OK) return st;
+    ctx->z_current = false;
     launch_unpack((const float*)dev, ctx->theta + (int64_t)stream * ctx->n_params, ctx->layout, 1, ctx->stream);
     ctx->launches += 1;
     if (ctx->bf16_mode) { launch_refresh_shadow(make_update_args(ctx, -1), ctx->stream); ctx->launches += 1; }
@@ -857,7 +863,10 @@ st_status student_forward(st_ctx* ctx, int32_t stream, const char* who)
     if (!ctx->has_feat[stream]) return fail(ctx, ST_ERR_BAD_STATE, "%s: stream %d has no frozen features yet", who, stream);
     for (int s = 0; s < ctx->S; ++s)
         if (!ctx->has_feat[s]) return fail(ctx, ST_ERR_BAD_STATE, "%s: the forward runs on all streams; stream %d has no features", who, s);
-    return enqueue_forward(ctx);
+    if (ctx->z_current) return ST_OK;       // an earlier call already ran it and nothing has changed since
+    st_status st = enqueue_forward(ctx);
+    ctx->z_current = st == ST_OK;
+    return st;
 }
 
 StudentMaskArgs mask_args(st_ctx* ctx, int32_t stream, uint8_t* mask)

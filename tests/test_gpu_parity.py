@@ -403,3 +403,41 @@ def test_apply_update_moves_a_student_between_contexts(c_hidden, prec):
         st._check(st.load_library().st_apply_update(client.handle, 0, update.ctypes.data, update.nbytes - 4), client)
     assert ei.value.status == st.ST_ERR_INVALID_ARG
     st.st_destroy(server); st.st_destroy(client)
+
+
+def test_agreement_of_several_streams_reuses_one_forward_and_notices_changes():
+    c_in, C, h, w, S = 8, 4, 9, 12, 3
+    probs = [rand_problem(10 + s, c_in, C, h, w) for s in range(S)]
+    thetas = [si.initial_head_params(c_in, 0, C, 20 + s) for s in range(S)]
+    ctx = make_ctx(c_in, 0, C, h, w, np.concatenate(thetas), S=S, lr=0.1)
+    labs = []
+    for s, (feat, T) in enumerate(probs):
+        st.st_set_frozen_features(ctx, s, dev(feat)); st.st_teacher_labels(ctx, s, dev(T))
+        labs.append(oracle.teacher_labels(T))
+
+    def check(thetas_now):
+        before = st.st_launch_count(ctx)
+        for s, (feat, _) in enumerate(probs):
+            conf = np.zeros((C, C), np.int64)
+            m = st.st_agreement(ctx, s, None, None, conf)
+            mask = torch.empty((4 * h, 4 * w), dtype=torch.uint8, device="cuda")
+            st.st_student_mask(ctx, s, mask)
+            oconf, om, _ = oracle.agreement(labs[s], mask.cpu().numpy(), C)
+            np.testing.assert_array_equal(conf, oconf)
+            assert m == om
+            ref = oracle.student_mask(oracle.Head(c_in, 0, C, theta=thetas_now[s]), feat)
+            assert (mask.cpu().numpy() != ref).mean() < 1e-3
+        return st.st_launch_count(ctx) - before
+
+    n1 = check(thetas)
+    n2 = check(thetas)                       # nothing changed: no forward at all this time
+    assert n2 == n1 - 1
+    st.st_apply_update(ctx, 1, thetas[0])   # stream 1 gets stream 0's student: the cached forward is stale
+    check([thetas[0], thetas[0], thetas[2]])
+    st.st_distill_step(ctx, 2)              # so it is after training steps
+    heads = [oracle.Head(c_in, 0, C, lr=0.1, theta=t) for t in (thetas[0], thetas[0], thetas[2])]
+    for s, (feat, _) in enumerate(probs):
+        for _ in range(2):
+            oracle.distill_step(heads[s], feat, labs[s])
+    check([hd.theta for hd in heads])
+    st.st_destroy(ctx)
