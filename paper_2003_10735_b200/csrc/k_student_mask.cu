@@ -4,8 +4,9 @@
 //
 // Geometry as in the fused upsample + cross-entropy kernel: the frame pixels 4n+2 .. 4n+5 lie between node
 // columns n and n+1 ("cell" n) with weights 1/8, 3/8, 5/8, 7/8 toward n+1, rows alike; cells -1 and w-1 / h-1
-// are the clamped borders.  A block covers 4 cell rows x 32 cell columns (one warp per cell row, one lane per
-// cell, 16 pixels each) with the logits of the 5 x 34 surrounding nodes in shared memory, borders replicated.
+// are the clamped borders.  A block covers 4 cell rows x 32 cell columns with the logits of the 5 x 34 surrounding
+// nodes in shared memory, borders replicated.  Two warps share a cell row: one lane per cell and half of its four
+// frame rows, 8 pixels each (the kernel is latency-bound in a single wave, so more and shorter warps finish sooner).
 // Per class a lane reads the cell's four corner logits and interpolates vertically, then horizontally, with one
 // fused multiply-add per step.  No pixel is shared between cells, so blocks are independent.
 #include "st_internal.h"
@@ -14,7 +15,12 @@ namespace st {
 
 namespace {
 
-constexpr int SM_WARPS = 4, SM_THREADS = SM_WARPS * 32;
+constexpr int SM_WARPS = 4;                                              // cell rows per block
+#ifndef ST_MASK_SPLIT
+#define ST_MASK_SPLIT 2
+#endif
+constexpr int SM_SPLIT = ST_MASK_SPLIT, SM_RW = 4 / SM_SPLIT;           // warps per cell row, frame rows per warp
+constexpr int SM_THREADS = SM_WARPS * SM_SPLIT * 32;
 constexpr int SM_TH = SM_WARPS + 1, SM_TW = 40, SM_T = SM_TH * SM_TW;   // tile: 5 node rows x 40 columns (34 used, start at a multiple of 4)
 constexpr int kMaxChunk = 32;                                            // classes held in shared memory at a time
 
@@ -36,7 +42,8 @@ student_mask_kernel(StudentMaskArgs a, int chunk)
     __shared__ bool is_last;
     const int C = a.C, h = a.h, w = a.w, H = h * kUp, W = w * kUp;
     const int64_t p = (int64_t)h * w;
-    const int tid = threadIdx.x, wi = tid >> 5, l = tid & 31;
+    const int tid = threadIdx.x, wi = tid / (32 * SM_SPLIT), l = tid & 31;   // wi: cell row inside the block
+    const int r0 = ((tid >> 5) % SM_SPLIT) * SM_RW;                 // this warp's frame rows of the cell: r0 .. r0 + SM_RW - 1
     const int ya = blockIdx.y * SM_WARPS - 1, xa = blockIdx.x * 32 - 4;   // node row / column of the tile's first element
     const int i = ya + wi, n = blockIdx.x * 32 - 1 + l;                   // cell row / column
     const bool cell_ok = i <= h - 1 && n <= w - 1;
@@ -45,11 +52,11 @@ student_mask_kernel(StudentMaskArgs a, int chunk)
 
     if (CONF) for (int e = tid; e < C * C; e += SM_THREADS) hist[e] = 0;
     // labels of the lane's 16 pixels, fetched before the sweep over the classes (two aligned 16-bit loads per row)
-    uint32_t labw[4] = {0, 0, 0, 0};
+    uint32_t labw[SM_RW] = {};
     if (CONF) {
 #pragma unroll
-        for (int r = 0; r < 4; ++r) {
-            const int Y = 4 * i + 2 + r;
+        for (int r = 0; r < SM_RW; ++r) {
+            const int Y = 4 * i + 2 + r0 + r;
             if (Y >= 0 && Y < H) {
                 uint32_t llo = 0, lhi = 0;
                 if (v01) llo = __ldg(reinterpret_cast<const unsigned short*>(a.labels + (int64_t)Y * W + X0));
@@ -59,10 +66,10 @@ student_mask_kernel(StudentMaskArgs a, int chunk)
         }
     }
 
-    float best[16];
-    uint32_t arg[16];
+    float best[4 * SM_RW];
+    uint32_t arg[4 * SM_RW];
 #pragma unroll
-    for (int k = 0; k < 16; ++k) { best[k] = -INFINITY; arg[k] = 0; }
+    for (int k = 0; k < 4 * SM_RW; ++k) { best[k] = -INFINITY; arg[k] = 0; }
 
     const bool vec_ok = (w % 4 == 0) && ((uintptr_t)a.z % 16 == 0);
     for (int c0 = 0; c0 < C; c0 += chunk) {                      // classes in chunks that fit shared memory
@@ -89,8 +96,8 @@ student_mask_kernel(StudentMaskArgs a, int chunk)
                 const float tl = q[0], bl = q[SM_TW], tr = q[1], br = q[SM_TW + 1];
                 const float dl = bl - tl, dr = br - tr;
 #pragma unroll
-                for (int r = 0; r < 4; ++r) {
-                    const float ly = (2 * r + 1) * 0.125f;
+                for (int r = 0; r < SM_RW; ++r) {
+                    const float ly = (float)(2 * (r0 + r) + 1) * 0.125f;
                     const float vl = fmaf(ly, dl, tl), vr = fmaf(ly, dr, tr), d = vr - vl;
 #pragma unroll
                     for (int k = 0; k < 4; ++k) {
@@ -104,8 +111,8 @@ student_mask_kernel(StudentMaskArgs a, int chunk)
 
     unsigned int n_bad = 0;
 #pragma unroll
-    for (int r = 0; r < 4; ++r) {
-        const int Y = 4 * i + 2 + r;
+    for (int r = 0; r < SM_RW; ++r) {
+        const int Y = 4 * i + 2 + r0 + r;
         const bool row_ok = Y >= 0 && Y < H;
         const uint32_t lo = arg[4 * r] | (arg[4 * r + 1] << 8), hi = arg[4 * r + 2] | (arg[4 * r + 3] << 8);
         if (MASK && row_ok) {
@@ -148,12 +155,22 @@ student_mask_kernel(StudentMaskArgs a, int chunk)
     __threadfence();
     double* iou = reinterpret_cast<double*>(zs);                  // [C] then present [C] (the tile is no longer needed)
     int* present = reinterpret_cast<int*>(iou + C);
+    // the matrix goes to shared memory in one coalesced pass if it fits behind them (the tile region is free now)
+    unsigned long long* cm = reinterpret_cast<unsigned long long*>(present + C + (C & 1));
+    const bool staged = (size_t)C * (sizeof(double) + sizeof(int)) + 8 + (size_t)C * C * 8 <= (size_t)chunk * SM_T * sizeof(float);
+    if (staged) {
+        for (int e = tid; e < C * C; e += SM_THREADS) cm[e] = __ldcg(&a.conf[e]);
+        __syncthreads();
+    }
     for (int c = tid; c < C; c += SM_THREADS) {
         unsigned long long row = 0, col = 0;
-        for (int q = 0; q < C; ++q) { row += __ldcg(&a.conf[c * C + q]); col += __ldcg(&a.conf[q * C + c]); }
+        for (int q = 0; q < C; ++q) {
+            row += staged ? cm[c * C + q] : __ldcg(&a.conf[c * C + q]);
+            col += staged ? cm[q * C + c] : __ldcg(&a.conf[q * C + c]);
+        }
         double v = 0.0; int pr = 0;
         if (row > 0) {
-            const unsigned long long inter = __ldcg(&a.conf[c * C + c]);
+            const unsigned long long inter = staged ? cm[c * C + c] : __ldcg(&a.conf[c * C + c]);
             v = (double)inter / (double)(row + col - inter);
             pr = 1;
         }
