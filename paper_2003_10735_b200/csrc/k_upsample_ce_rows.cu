@@ -431,18 +431,34 @@ upsample_ce_rows_kernel(UpsampleCeArgs a, const __grid_constant__ CUtensorMap z_
                 n_ok += __popc(rem[r]) + hw1 * __popc(rem[r] & hv[r]);      // the weights of the pixels that count
                 if (own_cell) n_bad += __popc(rem[r] ^ vb[r]);
             }
-            if (CONF) {                                              // the student's class: arg-max of the interpolated logits
+            if (CONF) {
+                // the student's class: arg-max over the classes of the cell's 16 interpolated logits (lowest class on
+                // ties), one class at a time: own node column vertically, the right-hand one likewise, then horizontally
+                float bestv[16];
+                uint32_t argv[16];
 #pragma unroll
-                for (int r = 0; r < 4; ++r) {
-                    float Zd[4];
-                    uint32_t ar4[4] = {0, 0, 0, 0};
-                    rc.ly = (2 * r + 1) * 0.125f;
-                    pass1<CB, true, false>(rc, zero4, Zd, ar4);
+                for (int j = 0; j < 16; ++j) { bestv[j] = -INFINITY; argv[j] = 0; }
+#pragma unroll kClassUnroll
+                for (int c = 0; c < CB; ++c) {
+                    const float* q = rc.za + c * TZ;
+                    const float a0 = q[0], b0 = q[TZ_W], a1 = q[1], b1 = q[TZ_W + 1];
+                    const float da = b0 - a0, db = b1 - a1;
 #pragma unroll
-                    for (int k = 0; k < 4; ++k)
-                        if (own_cell && ((rem[r] >> (8 * k)) & 1u))
-                            atomicAdd(&hist[((labw[r] >> (8 * k)) & 0xffu) * C + ar4[k]], 1u);
+                    for (int r = 0; r < 4; ++r) {
+                        const float ly = (2 * r + 1) * 0.125f;
+                        const float vl = fmaf(fmaf(ly, da, a0), kLog2e, -rc.M), vr = fmaf(fmaf(ly, db, a1), kLog2e, -rc.M);
+                        const float d = vr - vl;
+#pragma unroll
+                        for (int k = 0; k < 4; ++k) {
+                            const float u = fmaf((2 * k + 1) * 0.125f, d, vl);
+                            if (u > bestv[4 * r + k]) { bestv[4 * r + k] = u; argv[4 * r + k] = c; }
+                        }
+                    }
                 }
+#pragma unroll
+                for (int j = 0; j < 16; ++j)
+                    if (own_cell && ((rem[j >> 2] >> (8 * (j & 3))) & 1u))
+                        atomicAdd(&hist[((labw[j >> 2] >> (8 * (j & 3))) & 0xffu) * C + argv[j]], 1u);
             }
             float lz = 0.f;
 #pragma unroll
