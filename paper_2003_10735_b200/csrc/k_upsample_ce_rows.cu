@@ -404,12 +404,29 @@ upsample_ce_rows_kernel(UpsampleCeArgs a, const __grid_constant__ CUtensorMap z_
 #pragma unroll
         for (int k = 0; k < 4; ++k) Z01[k] = Z23[k] = make_float2(0.f, 0.f);
         float wmax = 0.f;
+        // CONF: the student's class of each pixel rides on the same sweep.  The exponentials are positive and monotone
+        // in the logits, so the largest one marks the arg-max; its bit pattern with the low five bits replaced by
+        // 31 - c is compared as an integer (equal values: the lowest class wins).  Dropping five bits can only swap
+        // classes whose logits differ by less than 3e-6 relative.
+        uint32_t key[16];
+#pragma unroll
+        for (int j = 0; j < 16; ++j) key[j] = 0;
 #pragma unroll kClassUnroll
         for (int c = 0; c < CB; ++c) {
             float2 X01[4], X23[4];
             wmax = fmaxf(wmax, cell_exponentials(rc.za + c * TZ, rc.M, X01, X23));
 #pragma unroll
             for (int k = 0; k < 4; ++k) { Z01[k] = __fadd2_rn(Z01[k], X01[k]); Z23[k] = __fadd2_rn(Z23[k], X23[k]); }
+            if (CONF) {
+                const uint32_t tag = 31u - (uint32_t)c;
+#pragma unroll
+                for (int k = 0; k < 4; ++k) {
+                    key[k] = max(key[k], (__float_as_uint(X01[k].x) & ~31u) | tag);
+                    key[4 + k] = max(key[4 + k], (__float_as_uint(X01[k].y) & ~31u) | tag);
+                    key[8 + k] = max(key[8 + k], (__float_as_uint(X23[k].x) & ~31u) | tag);
+                    key[12 + k] = max(key[12 + k], (__float_as_uint(X23[k].y) & ~31u) | tag);
+                }
+            }
         }
         float Z[16];                                                 // Z[4r + k]
 #pragma unroll
@@ -432,33 +449,10 @@ upsample_ce_rows_kernel(UpsampleCeArgs a, const __grid_constant__ CUtensorMap z_
                 if (own_cell) n_bad += __popc(rem[r] ^ vb[r]);
             }
             if (CONF) {
-                // the student's class: arg-max over the classes of the cell's 16 interpolated logits (lowest class on
-                // ties), one class at a time: own node column vertically, the right-hand one likewise, then horizontally
-                float bestv[16];
-                uint32_t argv[16];
-#pragma unroll
-                for (int j = 0; j < 16; ++j) { bestv[j] = -INFINITY; argv[j] = 0; }
-#pragma unroll kClassUnroll
-                for (int c = 0; c < CB; ++c) {
-                    const float* q = rc.za + c * TZ;
-                    const float a0 = q[0], b0 = q[TZ_W], a1 = q[1], b1 = q[TZ_W + 1];
-                    const float da = b0 - a0, db = b1 - a1;
-#pragma unroll
-                    for (int r = 0; r < 4; ++r) {
-                        const float ly = (2 * r + 1) * 0.125f;
-                        const float vl = fmaf(fmaf(ly, da, a0), kLog2e, -rc.M), vr = fmaf(fmaf(ly, db, a1), kLog2e, -rc.M);
-                        const float d = vr - vl;
-#pragma unroll
-                        for (int k = 0; k < 4; ++k) {
-                            const float u = fmaf((2 * k + 1) * 0.125f, d, vl);
-                            if (u > bestv[4 * r + k]) { bestv[4 * r + k] = u; argv[4 * r + k] = c; }
-                        }
-                    }
-                }
 #pragma unroll
                 for (int j = 0; j < 16; ++j)
                     if (own_cell && ((rem[j >> 2] >> (8 * (j & 3))) & 1u))
-                        atomicAdd(&hist[((labw[j >> 2] >> (8 * (j & 3))) & 0xffu) * C + argv[j]], 1u);
+                        atomicAdd(&hist[((labw[j >> 2] >> (8 * (j & 3))) & 0xffu) * C + (31u - (key[j] & 31u))], 1u);
             }
             float lz = 0.f;
 #pragma unroll

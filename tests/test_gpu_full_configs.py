@@ -212,7 +212,7 @@ def test_train_key_frame_720p_early_exit_is_cheaper_than_the_full_loop():
     (n, best, met), _ = timed(ctx, thr)
     assert n == 2 and best == met[2] > thr and (met[3:] == -1).all()
     ref = fresh()
-    st.st_distill_step(ref, 2)
+    st.st_distill_step(ref, 2, None, torch.zeros((1, 2, C, C), dtype=torch.int64, device="cuda"))   # same loss-kernel instantiation as Train
     a, b = np.empty(ctx.n_params, np.float32), np.empty(ctx.n_params, np.float32)
     st.st_pack_updated_params(ctx, 0, a); st.st_pack_updated_params(ref, 0, b)
     # (the timed replays above ran Train again from the returned student: with the threshold already met they take

@@ -4,7 +4,8 @@ The loop's decisions compare mean IoUs with THRESHOLD and with each other; the G
 oracle's in a few near-tie pixels, so (i) the decisions are checked exactly by replaying Algorithm 1's rules on the
 GPU's own confusion matrices with the oracle's metric, (ii) the metrics are compared with the oracle's within a small
 tolerance, and where the oracle's decisions are robust to that tolerance the control flow must be identical,
-(iii) the returned parameters must be bit-identical to the GPU's own plain loop of best_iter steps."""
+(iii) the returned parameters must be bit-identical to the GPU's own plain loop of best_iter steps when that loop also
+asks for the per-step confusion matrices (the same instantiation of the loss kernel), and equal to rounding otherwise."""
 import numpy as np
 import pytest
 
@@ -114,12 +115,19 @@ def test_train_key_frame_matches_algorithm_1(c_in, c_hidden, C, h, w, prec, lr, 
         robust = all(abs(x - thr) > 2 * tol for x in m_ref[:n_o + 1])
         if robust:
             assert n == n_o, (thr, m_ref, m_gpu)
-        # (iii) the returned student is the GPU's own iterate after best_iter plain steps, bit for bit
+        # (iii) the returned student is the GPU's own iterate after best_iter plain steps: bit for bit against the loop
+        # that also computes the per-step confusion (the loss kernel is instantiated with and without it, and the two
+        # instantiations round a few gradient values differently in the last place), to rounding against the other
         ctx2 = make_ctx(c_in, c_hidden, C, h, w, [theta], 1, prec, lr, mu)
         st.st_set_frozen_features(ctx2, 0, dev(feat)); st.st_set_labels(ctx2, 0, dev(labels))
+        ctx3 = make_ctx(c_in, c_hidden, C, h, w, [theta], 1, prec, lr, mu)
+        st.st_set_frozen_features(ctx3, 0, dev(feat)); st.st_set_labels(ctx3, 0, dev(labels))
         if bi_r > 0:
-            st.st_distill_step(ctx2, bi_r)
+            st.st_distill_step(ctx2, bi_r, None, torch.zeros((1, bi_r, C, C), dtype=torch.int64, device="cuda"))
+            st.st_distill_step(ctx3, bi_r)
         assert packed(ctx).tobytes() == packed(ctx2).tobytes(), (thr, bi_r)
+        np.testing.assert_allclose(packed(ctx), packed(ctx3), rtol=0, atol=(1e-5 if prec == 0 else 1e-3) * np.abs(packed(ctx3)).max())
+        st.st_destroy(ctx3)
         # the stored student is usable at once: its mask reproduces best_metric
         cf = np.zeros((C, C), np.int64)
         assert st.st_agreement(ctx, 0, None, None, cf) == float(best[0])
