@@ -16,7 +16,7 @@
 // and 18 multiplications replace 16 exp2.  Pass 1 sums them per pixel; pass 2 forms them again,
 // multiplies by the adjoint interpolation weights / Z and reduces them to the cell's contribution to
 // its upper node row (kept in registers) and lower node row (shared memory).
-// Slow path (a class changing by more than 16 log2-units across a cell, or a sum that underflows): the
+// Slow path (a class changing by more than kFastRange log2-units across a cell, or a sum that underflows): the
 // warp walks its four frame rows one by one with exact per-pixel maxima:
 //   pass 1  each lane interpolates its own node column vertically, takes the right neighbour's by
 //           shuffle, interpolates its four pixels horizontally, and sums exp2(u - M) over the classes
@@ -48,6 +48,14 @@ constexpr float kLog2e = 1.4426950408889634f, kLn2 = 0.6931471805599453f;
 #define ST_K3_CLASS_UNROLL 3
 #endif
 constexpr int kClassUnroll = ST_K3_CLASS_UNROLL;
+// Largest change of a class's logit between two corners of a cell (in log2 units) for which the cell stays on the
+// fast path.  All 16 products of the progressions are exponentials of the cell's own pixels (at most 1 after the
+// shift), the step factors stay below 2^20, and the relative error of a product grows with the size of the exponent
+// arguments: about 5e-6 at this limit, below the tolerance of the logit gradient.
+#ifndef ST_K3_FAST_RANGE
+#define ST_K3_FAST_RANGE 40.0f
+#endif
+constexpr float kFastRange = ST_K3_FAST_RANGE;
 
 __device__ __forceinline__ float ex2_approx(float x)
 {
@@ -114,7 +122,7 @@ __device__ __forceinline__ void pass1(const RowCtx& rc, const float (&sk)[4], fl
 // With ly_r = (2r+1)/8 and fr_k = (2k+1)/8:  u(r,k) = A + B k + G r + D k r, so the values are geometric
 // progressions along k and r: 4 exp2 and 12 multiplications (8 of them packed: X01[k] = (E(0,k), E(1,k)),
 // X23[k] = (E(2,k), E(3,k))).  Returns the largest corner difference
-// in the logits' own units (the caller leaves the fast path if a class changes by more than 16 log2-units across
+// in the logits' own units (the caller leaves the fast path if a class changes by more than kFastRange log2-units across
 // the cell: the progressions would lose their small terms).  q points at raw logits; M is in log2 units.
 __device__ __forceinline__ float cell_exponentials(const float* q, float M, float2 (&X01)[4], float2 (&X23)[4])
 {
@@ -431,7 +439,7 @@ upsample_ce_rows_kernel(UpsampleCeArgs a, const __grid_constant__ CUtensorMap z_
         float Z[16];                                                 // Z[4r + k]
 #pragma unroll
         for (int k = 0; k < 4; ++k) { Z[k] = Z01[k].x; Z[4 + k] = Z01[k].y; Z[8 + k] = Z23[k].x; Z[12 + k] = Z23[k].y; }
-        bool bad = !(wmax <= 16.0f / kLog2e);                       // 16 log2-units
+        bool bad = !(wmax <= kFastRange / kLog2e);
 #pragma unroll
         for (int j = 0; j < 16; ++j) bad |= ((vmask >> j) & 1u) && !(Z[j] > 1e-18f);
         const bool slow = __any_sync(0xffffffffu, bad);
