@@ -470,7 +470,10 @@ tc_dgrad_kernel(const __grid_constant__ CUtensorMap tmA,   // dz  {p, 32, S}  bo
     const uint32_t a_base = smem_u32(smem);
     const uint32_t blk_bytes = kClassPad * 128;                 // 32 class rows x 64 elements
     const uint32_t b_base = a_base + 2 * blk_bytes;
-    const int b_blocks = Ch / kBlockK;
+    // gridDim.z blocks share a pixel tile, each with its own range of Ch / gridDim.z hidden channels (more and
+    // shorter blocks: the kernel's time is the latency of one block's epilogue)
+    const int Chb = Ch / (int)gridDim.z, ch0 = (int)blockIdx.z * Chb;
+    const int b_blocks = Chb / kBlockK;
     __shared__ float part[4 * 256];                             // per-warp channel sums
     __shared__ __align__(8) uint64_t full, done;
     __shared__ uint32_t tmem_slot;
@@ -495,9 +498,9 @@ tc_dgrad_kernel(const __grid_constant__ CUtensorMap tmA,   // dz  {p, 32, S}  bo
         mbar_expect_tx(bar, (2 + b_blocks) * blk_bytes);
         tma_load_3d(a_base, &tmA, bar, pix0, 0, s);
         tma_load_3d(a_base + blk_bytes, &tmA, bar, pix0 + 64, 0, s);
-        for (int cb = 0; cb < b_blocks; ++cb) tma_load_3d(b_base + cb * blk_bytes, &tmB, bar, cb * kBlockK, 0, s);
+        for (int cb = 0; cb < b_blocks; ++cb) tma_load_3d(b_base + cb * blk_bytes, &tmB, bar, ch0 + cb * kBlockK, 0, s);
     } else if (tid == 32) {
-        const uint32_t idesc = instr_desc(kTileM, Ch, 1, 1);
+        const uint32_t idesc = instr_desc(kTileM, Chb, 1, 1);
         ok = mbar_wait(smem_u32(&full), 0, err, kWaitFull);
         if (ok) {
             tc_fence_after_sync();
@@ -516,14 +519,14 @@ tc_dgrad_kernel(const __grid_constant__ CUtensorMap tmA,   // dz  {p, 32, S}  bo
     if (in) {
         const uint32_t* mp = relu_bits + ((int64_t)s * p + pix) * (Ch / 32);
 #pragma unroll
-        for (int j = 0; j < 8; ++j) if (j < Ch / 32) mbits[j] = __ldg(mp + j);
+        for (int j = 0; j < 8; ++j) if (j < Chb / 32) mbits[j] = __ldg(mp + ch0 / 32 + j);
     }
     ok = mbar_wait(smem_u32(&done), 0, err, kWaitDone);
     tc_fence_after_sync();
     ok = __syncthreads_and(ok);          // the epilogue below synchronises the block: all or none
     if (ok) {
         const int64_t row = ((int64_t)s * p + (in ? pix : 0)) * Ch;
-        for (int n0 = 0; n0 < Ch; n0 += 32) {
+        for (int n0 = 0; n0 < Chb; n0 += 32) {
             float v[32];
             tmem_ld_32x32(tmem + ((uint32_t)(warp * 32) << 16) + n0, v);
             if (in) {
@@ -539,7 +542,7 @@ tc_dgrad_kernel(const __grid_constant__ CUtensorMap tmA,   // dz  {p, 32, S}  bo
                     o2[k] = __floats2bfloat162_rn(v[2 * k], v[2 * k + 1]);
                 }
 #pragma unroll
-                for (int k = 0; k < 4; ++k) reinterpret_cast<uint4*>(dhidden + row + n0)[k] = out[k];
+                for (int k = 0; k < 4; ++k) reinterpret_cast<uint4*>(dhidden + row + ch0 + n0)[k] = out[k];
             } else {
 #pragma unroll
                 for (int k = 0; k < 32; ++k) v[k] = 0.f;
@@ -560,8 +563,8 @@ tc_dgrad_kernel(const __grid_constant__ CUtensorMap tmA,   // dz  {p, 32, S}  bo
             part[warp * 256 + n0 + lane] = v[0];
         }
         __syncthreads();
-        for (int k = tid; k < Ch; k += kThreadsTc)
-            b1_partials[((int64_t)s * gridDim.x + blockIdx.x) * Ch + k] =
+        for (int k = tid; k < Chb; k += kThreadsTc)
+            b1_partials[((int64_t)s * gridDim.x + blockIdx.x) * Ch + ch0 + k] =
                 (part[k] + part[256 + k]) + (part[512 + k] + part[768 + k]);
     } else {
         drain_after_error();
@@ -772,8 +775,9 @@ int tc_backward(const TcPlan* P, cudaStream_t s, StageTimer* t, const int* skip,
     n += st_repeats(t);
     if (b.c_hidden) {
         const int blocks = tc_b1_partials(b.h, b.w);
-        ST_REPEAT(t) launch_chain(tc_dgrad_kernel, dim3(blocks, b.S), dim3(kThreadsTc), P->smem_dgrad, s,
-            P->dz_map, P->w2_map, b.relu_bits, b.dhidden, b.b1_partials, b.c_hidden, P->p, pow2_cols(b.c_hidden), b.err, skip, skip_stride);
+        const int n_ch_split = (b.c_hidden % 128 == 0) ? 2 : 1;      // each block: a multiple of 64 channels (four ways measured no better)
+        ST_REPEAT(t) launch_chain(tc_dgrad_kernel, dim3(blocks, b.S, n_ch_split), dim3(kThreadsTc), P->smem_dgrad, s,
+            P->dz_map, P->w2_map, b.relu_bits, b.dhidden, b.b1_partials, b.c_hidden, P->p, pow2_cols(b.c_hidden / n_ch_split), b.err, skip, skip_stride);
         if (t) t->mark("tc_dgrad", s, st_repeats(t));
         ST_REPEAT(t) launch_chain(tc_wgrad3x3_kernel<3>, dim3(9 * P->split1, b.S), dim3(kThreadsTc), P->smem_wg3, s,
             P->x_wg3, P->dh_wg3, b.w1_partials, b.c_in, b.c_hidden, b.h, b.w, P->chunks1, P->per1, P->split1,
