@@ -229,6 +229,9 @@ template <int STAGES>
 __global__ void __launch_bounds__(kFwd3Threads)
 tc_fwd3x3_kernel(const __grid_constant__ CUtensorMap tmA,   // {Cin, w, h, S}    box {64, 32, 4, 1}
                  const __grid_constant__ CUtensorMap tmB,   // {Cin, 9*Ch, S}    box {64, Ch, 1}
+                 const __grid_constant__ CUtensorMap tmBq,  // same tensor, box {64, 64, 1}: one block of 64 output channels
+                 int tail_split,                             // the tiles of the last, partly filled round are cut into this many
+                                                             // ranges of output channels (1, 2 or 4), one work item each
                  const float* __restrict__ theta, int64_t n_params, int64_t b_off,
                  bf16* __restrict__ hidden,                  // [S][p][Ch]
                  uint32_t* __restrict__ relu_bits,           // [S][p][Ch/32]: bit k of word j = hidden[32j + k] > 0
@@ -244,6 +247,17 @@ tc_fwd3x3_kernel(const __grid_constant__ CUtensorMap tmA,   // {Cin, w, h, S}   
     const int tiles_x = (w + kTileW - 1) / kTileW, tiles_y = (h + kTileH - 1) / kTileH;
     const int tiles_per_stream = tiles_x * tiles_y;
     const int kblocks = Cin / kBlockK, n_iter = 9 * kblocks;
+    // Work items: whole tiles while every block has one, then the remaining tiles in tail_split pieces each, so that
+    // the last round is short instead of leaving most blocks idle for a full tile's time.
+    const int n_full = tail_split > 1 ? (n_tiles_total / (int)gridDim.x) * (int)gridDim.x : n_tiles_total;
+    const int n_items = n_full + (n_tiles_total - n_full) * tail_split;
+    struct Item { int tile, ch0, chn; };
+    auto item_of = [&](int wi) {
+        Item it;
+        if (wi < n_full) { it.tile = wi; it.ch0 = 0; it.chn = Ch; }
+        else { const int q = wi - n_full; it.tile = n_full + q / tail_split; it.chn = Ch / tail_split; it.ch0 = (q % tail_split) * it.chn; }
+        return it;
+    };
 
     if (warp == 0) tmem_alloc(smem_u32(&tmem_slot), 2 * acc_cols);
     if (tid == 0) {
@@ -262,26 +276,31 @@ tc_fwd3x3_kernel(const __grid_constant__ CUtensorMap tmA,   // {Cin, w, h, S}   
     if (tid == 0) {
         // ---- producer: the ring index runs on across tiles
         int g = 0;
-        for (int t = blockIdx.x; t < n_tiles_total && ok; t += gridDim.x) {
-            const int s = t / tiles_per_stream, tt = t % tiles_per_stream;
-            if (skip && skip[(int64_t)s * skip_stride]) continue;     // all three roles leave out the same tiles
+        for (int wi = blockIdx.x; wi < n_items && ok; wi += gridDim.x) {
+            const Item im = item_of(wi);
+            const int s = im.tile / tiles_per_stream, tt = im.tile % tiles_per_stream;
+            if (skip && skip[(int64_t)s * skip_stride]) continue;     // all three roles leave out the same items
             const int x0 = (tt % tiles_x) * kTileW, y0 = (tt / tiles_x) * kTileH;
             for (int it = 0; it < n_iter; ++it, ++g) {
                 const int st = g % STAGES, tap = it / kblocks, kb = it % kblocks;
                 if (g >= STAGES) ok = mbar_wait(smem_u32(&empty[st]), ((g / STAGES) - 1) & 1, err, kWaitEmpty);
                 if (!ok) break;
                 const uint32_t bar = smem_u32(&full[st]), sa = base + st * stage_bytes;
-                mbar_expect_tx(bar, stage_bytes);
+                mbar_expect_tx(bar, a_bytes + (uint32_t)im.chn * 128);
                 tma_load_4d(sa, &tmA, bar, kb * kBlockK, x0 + tap % 3 - 1, y0 + tap / 3 - 1, s);
-                tma_load_3d(sa + a_bytes, &tmB, bar, kb * kBlockK, tap * Ch, s);
+                if (im.chn == Ch) tma_load_3d(sa + a_bytes, &tmB, bar, kb * kBlockK, tap * Ch, s);
+                else
+                    for (int j = 0; j < im.chn / 64; ++j)        // 64 weight rows per copy, laid out like the single copy
+                        tma_load_3d(sa + a_bytes + j * (64 * 128), &tmBq, bar, kb * kBlockK, tap * Ch + im.ch0 + j * 64, s);
             }
         }
     } else if (tid == 32) {
         // ---- MMA issuer
-        const uint32_t idesc = instr_desc(kTileM, Ch, 0, 0);
         int g = 0, j = 0;
-        for (int t = blockIdx.x; t < n_tiles_total && ok; t += gridDim.x) {
-            if (skip && skip[(int64_t)(t / tiles_per_stream) * skip_stride]) continue;
+        for (int wi = blockIdx.x; wi < n_items && ok; wi += gridDim.x) {
+            const Item im = item_of(wi);
+            if (skip && skip[(int64_t)(im.tile / tiles_per_stream) * skip_stride]) continue;
+            const uint32_t idesc = instr_desc(kTileM, im.chn, 0, 0);
             const int buf = j & 1;
             if (j >= 2) ok = mbar_wait(smem_u32(&acc_empty[buf]), ((j >> 1) - 1) & 1, err, kWaitEmpty);
             if (!ok) break;
@@ -305,8 +324,9 @@ tc_fwd3x3_kernel(const __grid_constant__ CUtensorMap tmA,   // {Cin, w, h, S}   
         // ---- epilogue warps: TMEM lanes 32*(warp % 4) .. +31 = pixel rows of the tile
         const int q = warp & 3, row = q * 32 + lane;
         int j = 0;
-        for (int t = blockIdx.x; t < n_tiles_total && ok; t += gridDim.x) {
-            const int s = t / tiles_per_stream, tt = t % tiles_per_stream;
+        for (int wi = blockIdx.x; wi < n_items && ok; wi += gridDim.x) {
+            const Item im = item_of(wi);
+            const int s = im.tile / tiles_per_stream, tt = im.tile % tiles_per_stream;
             if (skip && skip[(int64_t)s * skip_stride]) continue;
             const int buf = j & 1;
             const int x = (tt % tiles_x) * kTileW + row % kTileW, y = (tt / tiles_x) * kTileH + row / kTileW;
@@ -316,8 +336,9 @@ tc_fwd3x3_kernel(const __grid_constant__ CUtensorMap tmA,   // {Cin, w, h, S}   
             const bool in = y < h && x < w;
             const float* bias = theta + (int64_t)s * n_params + b_off;
             const int64_t pixel = (int64_t)s * h * w + (int64_t)y * w + x;
-            bf16* dst = hidden + pixel * Ch;
-            for (int n0 = 0; n0 < Ch; n0 += 32) {
+            bf16* dst = hidden + pixel * Ch + im.ch0;
+            bias += im.ch0;
+            for (int n0 = 0; n0 < im.chn; n0 += 32) {
                 float v[32];
                 tmem_ld_32x32(tmem + ((uint32_t)(q * 32) << 16) + buf * acc_cols + n0, v);
                 if (in) {
@@ -334,7 +355,7 @@ tc_fwd3x3_kernel(const __grid_constant__ CUtensorMap tmA,   // {Cin, w, h, S}   
                     }
 #pragma unroll
                     for (int k = 0; k < 4; ++k) reinterpret_cast<uint4*>(dst + n0)[k] = out[k];
-                    relu_bits[pixel * (Ch / 32) + n0 / 32] = bits;
+                    relu_bits[pixel * (Ch / 32) + (im.ch0 + n0) / 32] = bits;
                 }
             }
             tc_fence_before_sync();
@@ -637,6 +658,7 @@ struct TcPlan {
     CUtensorMap x_fwd3;      // {Cin, w, h, S} box {64, 32, 4, 1}
     CUtensorMap x_wg3;       // box {64, 32, 2, 1}
     CUtensorMap w1_map;      // {Cin, 9*Ch, S} box {64, Ch, 1}
+    CUtensorMap w1_map_q;    // same tensor, box {64, 64, 1}
     CUtensorMap dh_wg3;      // {Ch, w, h, S} box {64, 32, 2, 1}
     int split2, chunks2, per2, cols2;
     int split1, chunks1, per1, cols1;
@@ -704,6 +726,8 @@ TcPlan* tc_plan_create(const TcBuffers& b, char* err, size_t err_len)
         uint64_t dw[3] = {ci, 9 * ch, S}, sw[2] = {ci * 2, 9 * ch * ci * 2};
         uint32_t bwt[3] = {64, (uint32_t)b.c_hidden, 1};
         ok = ok && make_map(&P->w1_map, b.w1, 3, dw, sw, bwt, err, err_len, "3x3 weight");
+        uint32_t bwq[3] = {64, 64, 1};
+        ok = ok && make_map(&P->w1_map_q, b.w1, 3, dw, sw, bwq, err, err_len, "3x3 weight (64 rows)");
     }
     if (!ok) { delete P; return nullptr; }
 
@@ -752,8 +776,17 @@ int tc_forward(const TcPlan* P, cudaStream_t s, StageTimer* t, const int* skip, 
     if (b.c_hidden) {
         const int tiles = ((b.w + kTileW - 1) / kTileW) * ((b.h + kTileH - 1) / kTileH);
         const int total = tiles * b.S;
-        ST_REPEAT(t) launch_chain(tc_fwd3x3_kernel<4>, dim3(total < P->n_sms ? total : P->n_sms), dim3(kFwd3Threads), P->smem_fwd3, s,
-            P->x_fwd3, P->w1_map, b.theta, b.n_params, b.b1_off, b.hidden, b.relu_bits, b.c_in, b.c_hidden, b.h, b.w,
+        const int grid = total < P->n_sms ? total : P->n_sms;
+        // the tiles of a partly filled last round are cut into 4 or 2 ranges of output channels if that lets every
+        // piece have its own block (pieces are multiples of 64 channels)
+        const int tail = total > grid ? total % grid : 0;
+        int tail_split = 1;
+        if (tail > 0) {
+            if (b.c_hidden % 256 == 0 && tail * 4 <= grid) tail_split = 4;
+            else if (b.c_hidden % 128 == 0 && tail * 2 <= grid) tail_split = 2;
+        }
+        ST_REPEAT(t) launch_chain(tc_fwd3x3_kernel<4>, dim3(grid), dim3(kFwd3Threads), P->smem_fwd3, s,
+            P->x_fwd3, P->w1_map, P->w1_map_q, tail_split, b.theta, b.n_params, b.b1_off, b.hidden, b.relu_bits, b.c_in, b.c_hidden, b.h, b.w,
             total, pow2_cols(b.c_hidden), b.err, skip, skip_stride);
         if (t) t->mark("tc_fwd3x3", s, st_repeats(t));
         n += st_repeats(t);

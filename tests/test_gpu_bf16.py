@@ -244,3 +244,37 @@ def test_bf16_steps_are_bit_reproducible():
         outs.append(packed(ctx))
         st.st_destroy(ctx)
     assert outs[0].tobytes() == outs[1].tobytes()
+
+
+@pytest.mark.parametrize("c_in,ch,h,w", [
+    (64, 128, 72, 352),     # 198 tiles of 128 pixels: on 148 SMs the last 50 are cut into two channel ranges each
+    (64, 256, 56, 352),     # 154 tiles: the last 6 are cut into four channel ranges each
+])
+def test_two_layer_forward_with_a_partly_filled_last_round(c_in, ch, h, w):
+    C = 5
+    rng = np.random.default_rng(9)
+    feat = np.maximum(rng.standard_normal((c_in, h, w)), 0).astype(np.float32)
+    theta = si.initial_head_params(c_in, ch, C, 8)
+    nb1 = ch * c_in * 9
+    theta[nb1:nb1 + ch] = np.linspace(-0.2, 0.3, ch)
+    ctx = make_ctx(c_in, ch, C, h, w, theta)
+    st.st_set_frozen_features(ctx, 0, dev(feat))
+    mask = torch.empty((4 * h, 4 * w), dtype=torch.uint8, device="cuda")
+    st.st_student_mask(ctx, 0, mask)                              # runs the forward
+    hq = oracle.Head(c_in, ch, C, theta=theta, quantize_bf16=True)
+    z_ref, hd_ref = oracle.head_forward(hq, feat)
+    hd = st.st_read_tensor(ctx, 0, st.ST_TENSOR_HIDDEN)
+    d = np.abs(hd - hd_ref.ravel())
+    assert (d <= 2.0 ** -7 * np.maximum(np.abs(hd_ref.ravel()), 1e-3)).all()
+    assert (d > 0).mean() < 0.02
+    z = st.st_read_tensor(ctx, 0, st.ST_TENSOR_LOGITS)
+    np.testing.assert_allclose(z, z_ref.ravel(), rtol=1e-3, atol=5e-3)
+    # the ReLU bits written by the same epilogue drive the backward pass: one step's hidden gradient is zero exactly
+    # where the hidden activation is zero
+    lab = rng.integers(0, C, (4 * h, 4 * w)).astype(np.uint8)
+    st.st_set_labels(ctx, 0, dev(lab))
+    st.st_distill_step(ctx, 1)
+    hd1 = st.st_read_tensor(ctx, 0, st.ST_TENSOR_HIDDEN)
+    dh = st.st_read_tensor(ctx, 0, st.ST_TENSOR_HIDDEN_GRAD)
+    assert (dh[hd1 == 0] == 0).all() and (dh[hd1 > 0] != 0).mean() > 0.9
+    st.st_destroy(ctx)
