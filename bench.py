@@ -37,7 +37,6 @@ ALU_FLOP_PER_CLASS_PIXEL = 20.0   # algorithmic fp32 work of the fused upsample+
 # An entry is removed whenever its kernel changes and put back after the next capture.
 NCU_DRAM_BYTES = {
     (2, "upsample_ce"): 5.85e6,      # profiles/upsample_ce_rows_720p.md
-    (3, "tc_fwd3x3"): 31.2e6,        # profiles/tc_fwd3x3_tc_dgrad_tc_wgrad3x3_720p.md
 }
 
 
