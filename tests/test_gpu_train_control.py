@@ -181,3 +181,43 @@ def test_train_key_frame_argument_errors_and_replay():
     b = run_train(ctx, 1, C, 2.0, 3)
     assert a[0][0] == 3 and b[0][0] == 3 and b[2][0, 0] == a[1][0]      # the second call starts from the first one's best
     st.st_destroy(ctx)
+
+
+@pytest.mark.parametrize("c_hidden", [0, 64])
+def test_streams_end_independently_with_tensor_core_kernels(c_hidden):
+    """Three streams with bf16 GEMMs: once a stream's loop has ended, the blocks of its GEMMs and of its loss kernel
+    return at once (the persistent 3x3 forward leaves its tiles out) while the other streams keep training."""
+    c_in, C, h, w, K, lr, mu = 64, 5, 24, 40, 6, 0.3, 0.9
+    strengths = [3.0, 0.0, 2.0]                                       # stream 1 cannot learn: its loop runs to the end
+    probs = [problem(s, c_in, c_hidden, C, h, w, strength=strengths[s]) for s in range(3)]
+    mk = lambda s: oracle.Head(c_in, c_hidden, C, lr=lr, momentum=mu, theta=probs[s][2], quantize_bf16=True)
+    full = [oracle.train_key_frame(mk(s), probs[s][0], probs[s][1], 2.0, K).metrics for s in range(3)]
+    thr = 0.5 * (full[0][1] + full[0][2]) if full[0][2] > full[0][1] else 0.5 * (full[0][0] + max(full[0]))
+    ctx = make_ctx(c_in, c_hidden, C, h, w, [p[2] for p in probs], 3, 1, lr, mu)
+    for s, (feat, labels, _) in enumerate(probs):
+        st.st_set_frozen_features(ctx, s, dev(feat)); st.st_set_labels(ctx, s, dev(labels))
+    n_upd, best, met, los, conf = run_train(ctx, 3, C, thr, K)
+    exits = []
+    for s, (feat, labels, theta) in enumerate(probs):
+        n = int(n_upd[s])
+        m_gpu = [oracle.miou(conf[s, i]) for i in range(n + 1)]
+        n_r, bi_r, best_r = rules(m_gpu + [0.0] * K, thr, K)
+        assert (n, float(best[s])) == (n_r, best_r), (s, m_gpu)      # the device followed Algorithm 1 on its own metrics
+        assert (met[s, n + 1:] == -1.0).all()
+        # the stream's returned student: its own plain loop of best_iter steps (same kernels, no other stream involved)
+        solo = make_ctx(c_in, c_hidden, C, h, w, [theta], 1, 1, lr, mu)
+        st.st_set_frozen_features(solo, 0, dev(feat)); st.st_set_labels(solo, 0, dev(labels))
+        if bi_r > 0:
+            st.st_distill_step(solo, bi_r, None, torch.zeros((1, bi_r, C, C), dtype=torch.int64, device="cuda"))
+        assert packed(ctx, s).tobytes() == packed(solo).tobytes(), s
+        st.st_destroy(solo)
+        np.testing.assert_allclose(m_gpu, full[s][:n + 1], atol=3e-2)
+        exits.append(n)
+    assert len(set(exits)) >= 2, exits                               # some loops went on after others had ended
+    # a second call starts from the returned students: those already past the threshold take no step
+    n2 = np.zeros(3, np.int32)
+    st.st_train_key_frame(ctx, thr, K, n2)
+    for s in range(3):
+        if best[s] >= thr:
+            assert n2[s] == 0, (s, n2)
+    st.st_destroy(ctx)
