@@ -310,7 +310,7 @@ def run_ours(args, cfg):
         d2h = S * (n_params * 4 + 8)
 
         # ---- per-kernel times with CUDA events on the launching stream
-        kernels = {}
+        kernels, train = {}, {}
         if rank == 0:
             def timed(fn, reps=20):
                 ev0.record(stream)
@@ -356,6 +356,14 @@ def run_ours(args, cfg):
             for k in kernels.values():
                 if "achieved" in k and k.get("peak"):
                     k["frac"] = k["achieved"] / k["peak"]
+            # Train of Algorithm 1 (forward, metric, break test and best-student snapshot per update, all on the device):
+            # the full loop (a threshold no mean IoU reaches) and a loop that ends on the first metric
+            train = {}
+            for name, thr in (("full_loop", 2.0), ("ends_at_once", 0.0)):
+                for _ in range(3):
+                    st.st_train_key_frame(ctx, thr, K)
+                train[name + "_ms"] = timed(lambda r: st.st_train_key_frame(ctx, thr, K), reps=20)
+            train["max_updates"] = K
 
         result = None
         if rank == 0:
@@ -387,7 +395,7 @@ def run_ours(args, cfg):
                 "roofline": roofline,
                 "key_frames_per_s": world * args.steps / (ms_total / 1e3),
                 "distill_loop_only": {"steps_per_s": K * S / (ms_loop / 1e3), "ms_per_k_steps": ms_loop},
-                "kernels": kernels,
+                "kernels": kernels, "train_key_frame": train,
                 "last_loss": float(loss_d[0, -1].item()), "last_miou": mious[0], "last_miou_device_run": last_miou_dev,
             }
         st.st_destroy(ctx)
