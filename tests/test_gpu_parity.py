@@ -441,3 +441,28 @@ def test_agreement_of_several_streams_reuses_one_forward_and_notices_changes():
             oracle.distill_step(heads[s], feat, labs[s])
     check([hd.theta for hd in heads])
     st.st_destroy(ctx)
+
+
+@pytest.mark.parametrize("scale", [3.5, 4.2])
+def test_steep_logits_inside_the_fast_range_keep_fp32_accuracy(scale):
+    """Logits that change by 20 to 28 nats between neighbouring nodes: most cells still take the geometric-progression
+    path of the fused loss kernel (its limit is 40 log2-units = 27.7 nats per cell), a few the row-by-row one; the
+    gradient must agree with the oracle as on gentle logits."""
+    c_in, C, h, w = 32, 21, 45, 80
+    cls = si.voronoi_map(4 * h, 4 * w, 24, C, 2005)
+    feat = si.label_informed_features(c_in, h, w, cls, 4, 7, strength=3.0)
+    theta = (si.initial_head_params(c_in, 0, C, 5) * scale).astype(np.float32)
+    ctx = make_ctx(c_in, 0, C, h, w, theta, lr=0.0)
+    st.st_set_frozen_features(ctx, 0, dev(feat)); st.st_set_labels(ctx, 0, dev(cls))
+    loss = np.zeros(1, np.float32)
+    st.st_distill_step(ctx, 1, loss)
+    head = oracle.Head(c_in, 0, C, theta=theta)
+    z, _ = oracle.head_forward(head, feat)
+    steps = max(np.abs(np.diff(z, axis=1)).max(), np.abs(np.diff(z, axis=2)).max())
+    assert 18.0 < steps < 40.0, steps                               # the case is what it is meant to be
+    ref_loss, g, _ = oracle.softmax_ce(oracle.upsample(z, 4), cls)
+    ref = oracle.upsample_adjoint(g, 4).ravel()
+    dz = st.st_read_tensor(ctx, 0, st.ST_TENSOR_LOGIT_GRAD)
+    assert np.linalg.norm(dz - ref) / np.linalg.norm(ref) < 2e-6
+    assert abs(loss[0] - ref_loss) <= 1e-5 * abs(ref_loss)
+    st.st_destroy(ctx)
