@@ -6,29 +6,33 @@
 // Geometry.  With half-pixel centres and factor 4 the frame pixels 4n+2 .. 4n+5 lie between node
 // columns n and n+1 ("cell" n) with weights 1/8, 3/8, 5/8, 7/8 toward n+1; rows alike.  Cells -1 and
 // w-1 are the clamped borders (their outer node is the inner one).
-// A block owns RN_Y rows x 30 columns of nodes and runs RN_Y+1 warps.  Warp i walks the four frame rows
-// of cell row y0-1+i; lane l owns node column x0-1+l and handles the four pixels of the cell to its
-// right.  Warp 0, lane 0 and lane 31 are halo (recomputed by the neighbouring block) so that a block
-// finishes its nodes alone, in a fixed summation order, without floating-point atomics.
-// Fast path (smooth logits, the usual case), class by class for all 16 pixels of the lane's cell at once:
-// inside a cell the interpolated logit of a class is u(r,k) = A + B k + G r + D k r (r = frame row,
-// k = pixel in the row), so its 16 exponentials form geometric progressions: four exp2 (of A, B, G, D)
-// and 18 multiplications replace 16 exp2.  Pass 1 sums them per pixel; pass 2 forms them again,
-// multiplies by the adjoint interpolation weights / Z and reduces them to the cell's contribution to
-// its upper node row (kept in registers) and lower node row (shared memory).
-// Slow path (a class changing by more than kFastRange log2-units across a cell, or a sum that underflows): the
-// warp walks its four frame rows one by one with exact per-pixel maxima:
-//   pass 1  each lane interpolates its own node column vertically, takes the right neighbour's by
-//           shuffle, interpolates its four pixels horizontally, and sums exp2(u - M) over the classes
-//           (logits are pre-scaled by log2 e; M is the largest logit of the block's tile);
-//   pass 2  the exponentials are formed again (cheaper than keeping 4 x C registers alive: two
-//           or three blocks per SM stay resident), multiplied by the adjoint interpolation weights / Z, the
-//           right-hand part is handed to the next lane by shuffle, and the row is added into two
-//           per-class accumulators: toward the upper and the lower node row.
-// If a pixel's sum underflows (logits varying by more than ~100 inside the block's tile) the warp
-// redoes that row with the exact per-pixel maximum.
-// The "- onehot(label)" part of the gradient is exact in units of 1/64, so it is accumulated with
-// integer shared-memory atomics (order-independent).
+// A block owns RN_Y rows x 30 columns of nodes and runs RN_Y+1 warps.  Warp i owns cell row y0-1+i (the 4 x 4
+// frame pixels between node rows i and i+1); lane l owns node column x0-1+l and the 16 pixels of the cell to its
+// right.  Warp 0, lane 0 and lane 31 are halo (recomputed by the neighbouring block) so that a block finishes its
+// nodes alone, in a fixed summation order, without floating-point atomics.
+// The block's logit tile (RN_Y+2 node rows x 36 columns x C classes) arrives by one TMA tile copy issued before
+// anything else; rows and columns outside the map arrive as zeros and border blocks overwrite them with the clamped
+// border values.  Shapes the tile map cannot describe are fetched with plain loads.
+// Fast path (the usual case), class by class for all 16 pixels of the lane's cell at once: inside a cell the
+// interpolated logit of a class is u(r,k) = A + B k + G r + D k r (r = frame row, k = pixel in the row), so its 16
+// exponentials form geometric progressions: four exp2 (of A, B, G, D) and 12 multiplications (packed fp32x2) replace
+// 16 exp2.  Pass 1 sums them per pixel; pass 2 forms them again (cheaper than keeping 16 x C registers alive),
+// multiplies by the adjoint interpolation weights / Z and reduces them to the cell's pull on its upper and lower
+// node row, both stored in shared memory.  Both sweeps are rolled loops over the classes.
+// Slow path (a class changing by more than kFastRange log2-units between two corners of a cell, or a sum that
+// underflows): the warp walks its four frame rows one by one with exact per-pixel maxima:
+//   pass 1  each lane interpolates its own node column vertically, takes the right neighbour's by shuffle,
+//           interpolates its four pixels horizontally, and sums exp2(u - max) over the classes (logits pre-scaled
+//           by log2 e);
+//   pass 2  the exponentials are formed again, multiplied by the adjoint interpolation weights / Z, the right-hand
+//           part is handed to the next lane by shuffle, and the row is added into the two shared-memory slots.
+// The "- onehot(label)" part of the gradient is exact in units of 1/64, so it is accumulated with integer
+// shared-memory atomics (order-independent), one round per distinct label of a cell.  Pixels tagged for the loss
+// weighting (bit 7 of the label byte) count with an integer weight in the loss, in 1/Z and in those integers.
+// The epilogue adds, per node row, the own cell row's upper part, the lower part of the cell row above and the
+// integer part, writes the bf16 (and on request the fp32) gradient, and reduces the block's bias-gradient partial by
+// a lane reduce-scatter.  With CONF the student's class of every pixel (arg-max of the interpolated logits) is taken
+// from pass 1's exponentials and counted against the label in a shared-memory confusion matrix.
 #include "st_internal.h"
 #include "tc_common.cuh"
 
