@@ -127,12 +127,17 @@ __global__ void __launch_bounds__(kThreadsTc)
 tc_wgrad1x1_kernel(const __grid_constant__ CUtensorMap tmA,   // {K, p, S}      box {64, 64, 1}
                    const __grid_constant__ CUtensorMap tmB,   // {p, 32, S}     box {64, 32, 1}
                    float* __restrict__ partials,              // [S][n_split][32][K]
-                   int K, int n_chunks, int chunks_per_block, int tmem_cols, unsigned int* err, const int* __restrict__ skip, int64_t skip_stride)
+                   int K, int n_chunks, int chunks_per_block, int m_split, int tmem_cols, unsigned int* err,
+                   const int* __restrict__ skip, int64_t skip_stride)
 {
     if (skip && skip[(int64_t)blockIdx.y * skip_stride]) return;   // this stream's training loop has ended (block-uniform)
     extern __shared__ uint8_t smem_raw[];
     uint8_t* smem = align_smem(smem_raw);
-    const int m_tiles = (K + kTileM - 1) / kTileM;   // accumulators (128 channels each)
+    // m_split blocks share a pixel range, each with its own 128-channel accumulators: with the channels divided the
+    // pixel ranges are longer and fewer, and the update has that many fewer partial sums to add per weight
+    const int m_all = (K + kTileM - 1) / kTileM;     // accumulators (128 channels each) of the whole layer
+    const int m_tiles = m_all / m_split;             // ... of this block
+    const int m0 = ((int)blockIdx.x % m_split) * m_tiles;
     const int a_blocks = m_tiles * 2;                // 64-channel blocks loaded per stage (absent ones are zero-filled)
     const uint32_t a_stage_bytes = a_blocks * (kChunkPix * 128);
     const uint32_t stage_bytes = a_stage_bytes + kClassPad * 128;
@@ -140,7 +145,7 @@ tc_wgrad1x1_kernel(const __grid_constant__ CUtensorMap tmA,   // {K, p, S}      
     __shared__ __align__(8) uint64_t full[STAGES], empty[STAGES], done;
     __shared__ uint32_t tmem_slot;
     const int tid = threadIdx.x, warp = tid >> 5;
-    const int s = blockIdx.y, split = blockIdx.x, n_split = gridDim.x;
+    const int s = blockIdx.y, split = (int)blockIdx.x / m_split, n_split = (int)gridDim.x / m_split;
     const int c_begin = split * chunks_per_block;
     const int c_end = min(n_chunks, c_begin + chunks_per_block);
 
@@ -167,7 +172,7 @@ tc_wgrad1x1_kernel(const __grid_constant__ CUtensorMap tmA,   // {K, p, S}      
             const uint32_t sa = base + st * stage_bytes;
             mbar_expect_tx(bar, stage_bytes);
             for (int cb = 0; cb < a_blocks; ++cb)
-                tma_load_3d(sa + cb * (kChunkPix * 128), &tmA, bar, cb * kBlockK, i * kChunkPix, s);
+                tma_load_3d(sa + cb * (kChunkPix * 128), &tmA, bar, (2 * m0 + cb) * kBlockK, i * kChunkPix, s);
             tma_load_3d(sa + a_stage_bytes, &tmB, bar, i * kChunkPix, 0, s);
         }
     } else if (tid == 32) {
@@ -198,7 +203,7 @@ tc_wgrad1x1_kernel(const __grid_constant__ CUtensorMap tmA,   // {K, p, S}      
         for (int m = 0; m < m_tiles; ++m) {
             float v[32];
             tmem_ld_32x32(tmem + ((uint32_t)(warp * 32) << 16) + m * kClassPad, v);
-            const int k = m * kTileM + tid;
+            const int k = (m0 + m) * kTileM + tid;
             if (k < K)
 #pragma unroll
                 for (int c = 0; c < kClassPad; ++c) dst[(int64_t)c * K + k] = any ? v[c] : 0.f;
@@ -660,19 +665,22 @@ struct TcPlan {
     CUtensorMap w1_map;      // {Cin, 9*Ch, S} box {64, Ch, 1}
     CUtensorMap w1_map_q;    // same tensor, box {64, 64, 1}
     CUtensorMap dh_wg3;      // {Ch, w, h, S} box {64, 32, 2, 1}
-    int split2, chunks2, per2, cols2;
+    int split2, chunks2, per2, cols2, msplit2;
     int split1, chunks1, per1, cols1;
     size_t smem_fwd1, smem_wg1, smem_fwd3, smem_wg3, smem_dgrad;
     int n_sms;
 };
 
+// blocks per pixel range of the 1x1 weight gradient: one per 128-channel accumulator
+static int wgrad1x1_m_split(int c_last) { const int m = (c_last + kTileM - 1) / kTileM; return m < 1 ? 1 : m; }
+
 int tc_wgrad_splits(int layer, int c_in, int c_hidden, int h, int w)
 {
-    (void)c_in; (void)c_hidden;
     int per, n;
     if (layer == 2) {
         const int64_t p = (int64_t)h * w;
-        split_geometry((int)((p + kChunkPix - 1) / kChunkPix), 148, &per, &n);
+        const int c_last = c_hidden ? c_hidden : c_in;
+        split_geometry((int)((p + kChunkPix - 1) / kChunkPix), 148 / wgrad1x1_m_split(c_last), &per, &n);
     } else {
         const int chunks = ((w + kChunkW - 1) / kChunkW) * ((h + kChunkH - 1) / kChunkH);
         split_geometry(chunks, 148 / 9, &per, &n);
@@ -733,10 +741,11 @@ TcPlan* tc_plan_create(const TcBuffers& b, char* err, size_t err_len)
 
     const int m_last = (P->c_last + kTileM - 1) / kTileM;
     P->chunks2 = (P->p + kChunkPix - 1) / kChunkPix;
-    split_geometry(P->chunks2, 148, &P->per2, &P->split2);
-    P->cols2 = pow2_cols(m_last * kClassPad);
+    P->msplit2 = wgrad1x1_m_split(P->c_last);
+    split_geometry(P->chunks2, 148 / P->msplit2, &P->per2, &P->split2);
+    P->cols2 = pow2_cols((m_last / P->msplit2) * kClassPad);
     P->smem_fwd1 = (size_t)(P->c_last / kBlockK) * (kTileM * 128 + kClassPad * 128) + kSmemAlign;
-    P->smem_wg1 = 3 * ((size_t)m_last * 2 * kChunkPix * 128 + kClassPad * 128) + kSmemAlign;
+    P->smem_wg1 = 3 * ((size_t)(m_last / P->msplit2) * 2 * kChunkPix * 128 + kClassPad * 128) + kSmemAlign;
     if (b.c_hidden) {
         const int m_in = (b.c_in + kTileM - 1) / kTileM;
         P->chunks1 = ((b.w + kChunkW - 1) / kChunkW) * ((b.h + kChunkH - 1) / kChunkH);
@@ -802,8 +811,8 @@ int tc_backward(const TcPlan* P, cudaStream_t s, StageTimer* t, const int* skip,
 {
     const TcBuffers& b = P->b;
     int n = 0;
-    ST_REPEAT(t) launch_chain(tc_wgrad1x1_kernel<3>, dim3(P->split2, b.S), dim3(kThreadsTc), P->smem_wg1, s,
-        P->act_wg, P->dz_map, b.w2_partials, P->c_last, P->chunks2, P->per2, P->cols2, b.err, skip, skip_stride);
+    ST_REPEAT(t) launch_chain(tc_wgrad1x1_kernel<3>, dim3(P->split2 * P->msplit2, b.S), dim3(kThreadsTc), P->smem_wg1, s,
+        P->act_wg, P->dz_map, b.w2_partials, P->c_last, P->chunks2, P->per2, P->msplit2, P->cols2, b.err, skip, skip_stride);
     if (t) t->mark("tc_wgrad1x1", s, st_repeats(t));
     n += st_repeats(t);
     if (b.c_hidden) {
