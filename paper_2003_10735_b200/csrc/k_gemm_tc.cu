@@ -34,6 +34,10 @@ constexpr int kTileW = 32, kTileH = 4;   // 3x3 forward: 128 pixels = 4 rows x 3
 constexpr int kChunkW = 32, kChunkH = 2; // 3x3 wgrad: 64 pixels = 2 rows x 32 columns
 constexpr int kSmemAlign = 1024;
 constexpr int kMaxKBlocks = 16;
+#ifndef ST_WG1_STAGES
+#define ST_WG1_STAGES 3
+#endif
+constexpr int kWg1Stages = ST_WG1_STAGES;   // pipeline depth of the 1x1 weight gradient (20 KB per stage at 128 channels per block)
 
 __device__ __forceinline__ uint8_t* align_smem(uint8_t* p)
 {
@@ -745,7 +749,7 @@ TcPlan* tc_plan_create(const TcBuffers& b, char* err, size_t err_len)
     split_geometry(P->chunks2, 148 / P->msplit2, &P->per2, &P->split2);
     P->cols2 = pow2_cols((m_last / P->msplit2) * kClassPad);
     P->smem_fwd1 = (size_t)(P->c_last / kBlockK) * (kTileM * 128 + kClassPad * 128) + kSmemAlign;
-    P->smem_wg1 = 3 * ((size_t)(m_last / P->msplit2) * 2 * kChunkPix * 128 + kClassPad * 128) + kSmemAlign;
+    P->smem_wg1 = kWg1Stages * ((size_t)(m_last / P->msplit2) * 2 * kChunkPix * 128 + kClassPad * 128) + kSmemAlign;
     if (b.c_hidden) {
         const int m_in = (b.c_in + kTileM - 1) / kTileM;
         P->chunks1 = ((b.w + kChunkW - 1) / kChunkW) * ((b.h + kChunkH - 1) / kChunkH);
@@ -766,7 +770,7 @@ TcPlan* tc_plan_create(const TcBuffers& b, char* err, size_t err_len)
         delete P; return nullptr;
     }
     cudaError_t e = cudaFuncSetAttribute(tc_fwd1x1_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)P->smem_fwd1);
-    if (e == cudaSuccess) e = cudaFuncSetAttribute(tc_wgrad1x1_kernel<3>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)P->smem_wg1);
+    if (e == cudaSuccess) e = cudaFuncSetAttribute(tc_wgrad1x1_kernel<kWg1Stages>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)P->smem_wg1);
     if (b.c_hidden) {
         if (e == cudaSuccess) e = cudaFuncSetAttribute(tc_fwd3x3_kernel<4>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)P->smem_fwd3);
         if (e == cudaSuccess) e = cudaFuncSetAttribute(tc_wgrad3x3_kernel<3>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)P->smem_wg3);
@@ -811,7 +815,7 @@ int tc_backward(const TcPlan* P, cudaStream_t s, StageTimer* t, const int* skip,
 {
     const TcBuffers& b = P->b;
     int n = 0;
-    ST_REPEAT(t) launch_chain(tc_wgrad1x1_kernel<3>, dim3(P->split2 * P->msplit2, b.S), dim3(kThreadsTc), P->smem_wg1, s,
+    ST_REPEAT(t) launch_chain(tc_wgrad1x1_kernel<kWg1Stages>, dim3(P->split2 * P->msplit2, b.S), dim3(kThreadsTc), P->smem_wg1, s,
         P->act_wg, P->dz_map, b.w2_partials, P->c_last, P->chunks2, P->per2, P->msplit2, P->cols2, b.err, skip, skip_stride);
     if (t) t->mark("tc_wgrad1x1", s, st_repeats(t));
     n += st_repeats(t);
