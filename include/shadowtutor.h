@@ -125,7 +125,8 @@ ST_API st_status st_set_labels(st_ctx *ctx, int32_t stream, const uint8_t *label
  * st_distill_step — n_steps iterations of Algorithm 1's loop body on all S streams:
  * head forward, bilinear x4 upsample, mean per-pixel softmax cross-entropy against the
  * stored labels (Section 5.2), gradients of the head only (PartialBackward, Section 4.2),
- * SGD(+momentum) update (OptimStep).
+ * OptimStep with the descriptor's optimiser (gradient descent with momentum, or Adam).  With object_weight > 1 the
+ * cross-entropy is the weighted one of Section 5.2.
  *   n_steps   1..64.
  *   loss_out  host or device, or NULL; fp32 [S][n_steps]: loss of each step's forward.
  *   conf_out  host or device, or NULL; int64 [S][n_steps][C][C]: conf[label][prediction] of the
