@@ -234,6 +234,122 @@ __device__ __forceinline__ void mbar_arrive(uint32_t bar)
     asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
 }
 
+// ------------------------------------------------------------------------------------------------
+// fwd 1x1, persistent: gridDim.x blocks per stream walk the stream's 128-pixel tiles.  Three roles as in the 3x3
+// forward: one thread feeds a ring of shared-memory stages by TMA across tile boundaries (one 128-pixel x 64-channel
+// block per stage, 128 KB in flight), one thread issues the MMAs into one of two tensor-memory accumulators, the
+// epilogue warps drain the other one (bias, fp32 logits, planar) meanwhile.  The classifier weights are loaded once
+// per block.
+// ------------------------------------------------------------------------------------------------
+#ifndef ST_F1_STAGES
+#define ST_F1_STAGES 8
+#endif
+constexpr int kF1Threads = 192, kF1Stages = ST_F1_STAGES;
+constexpr uint32_t kF1StageBytes = kTileM * 128;
+
+__global__ void __launch_bounds__(kF1Threads)
+tc_fwd1x1p_kernel(const __grid_constant__ CUtensorMap tmA,   // {K, p, S}  box {64, 128, 1}
+                  const __grid_constant__ CUtensorMap tmB,   // {K, 32, S} box {64, 32, 1}
+                  const float* __restrict__ theta, int64_t n_params, int64_t b_off,
+                  float* __restrict__ z, int C, int p, int kblocks, unsigned int* err,
+                  const int* __restrict__ skip, int64_t skip_stride)
+{
+    if (skip && skip[(int64_t)blockIdx.y * skip_stride]) return;   // this stream's training loop has ended (block-uniform)
+    extern __shared__ uint8_t smem_raw[];
+    uint8_t* smem = align_smem(smem_raw);
+    const uint32_t a_base = smem_u32(smem);
+    const uint32_t b_base = a_base + kF1Stages * kF1StageBytes;
+    __shared__ __align__(8) uint64_t full[kF1Stages], empty[kF1Stages], b_full, acc_full[2], acc_empty[2];
+    __shared__ uint32_t tmem_slot;
+    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+    const int s = blockIdx.y;
+    const int n_items = (p + kTileM - 1) / kTileM;
+
+    if (warp == 0) tmem_alloc(smem_u32(&tmem_slot), 2 * kClassPad);
+    if (tid == 0) {
+        for (int i = 0; i < kF1Stages; ++i) { mbar_init(smem_u32(&full[i]), 1); mbar_init(smem_u32(&empty[i]), 1); }
+        mbar_init(smem_u32(&b_full), 1);
+        for (int i = 0; i < 2; ++i) { mbar_init(smem_u32(&acc_full[i]), 1); mbar_init(smem_u32(&acc_empty[i]), 4); }
+        fence_barrier_init();
+    }
+    tc_fence_before_sync();
+    __syncthreads();
+    tc_fence_after_sync();
+    const uint32_t tmem = tmem_slot;
+    pdl_wait();                  // inputs come from the previous kernel of the step
+    pdl_launch_dependents();
+    bool ok = true;
+
+    if (tid == 0) {
+        // ---- producer
+        const uint32_t bb = smem_u32(&b_full);
+        mbar_expect_tx(bb, (uint32_t)kblocks * kClassPad * 128);
+        for (int kb = 0; kb < kblocks; ++kb) tma_load_3d(b_base + kb * (kClassPad * 128), &tmB, bb, kb * kBlockK, 0, s);
+        int g = 0;
+        for (int it = blockIdx.x; it < n_items && ok; it += gridDim.x) {
+            for (int kb = 0; kb < kblocks; ++kb, ++g) {
+                const int st = g % kF1Stages;
+                if (g >= kF1Stages) ok = mbar_wait(smem_u32(&empty[st]), ((g / kF1Stages) - 1) & 1, err, kWaitEmpty);
+                if (!ok) break;
+                const uint32_t bar = smem_u32(&full[st]);
+                mbar_expect_tx(bar, kF1StageBytes);
+                tma_load_3d(a_base + st * kF1StageBytes, &tmA, bar, kb * kBlockK, it * kTileM, s);
+            }
+        }
+    } else if (tid == 32) {
+        // ---- MMA issuer
+        constexpr uint32_t idesc = instr_desc(kTileM, kClassPad, 0, 0);
+        ok = mbar_wait(smem_u32(&b_full), 0, err, kWaitFull);
+        int g = 0, j = 0;
+        for (int it = blockIdx.x; it < n_items && ok; it += gridDim.x, ++j) {
+            const int buf = j & 1;
+            if (j >= 2) ok = mbar_wait(smem_u32(&acc_empty[buf]), ((j >> 1) - 1) & 1, err, kWaitEmpty);
+            if (!ok) break;
+            tc_fence_after_sync();
+            const uint32_t acc = tmem + buf * kClassPad;
+            for (int kb = 0; kb < kblocks; ++kb, ++g) {
+                const int st = g % kF1Stages;
+                ok = mbar_wait(smem_u32(&full[st]), (g / kF1Stages) & 1, err, kWaitFull);
+                if (!ok) break;
+                tc_fence_after_sync();
+                const uint32_t sa = a_base + st * kF1StageBytes, sb = b_base + kb * (kClassPad * 128);
+#pragma unroll
+                for (int k = 0; k < 4; ++k)
+                    umma(acc, smem_desc(sa + k * 32, 16, 1024), smem_desc(sb + k * 32, 16, 1024), idesc, (kb | k) != 0);
+                umma_commit(smem_u32(&empty[st]));
+            }
+            if (ok) umma_commit(smem_u32(&acc_full[buf]));
+        }
+    } else if (warp >= 2) {
+        // ---- epilogue warps: TMEM lanes 32*(warp % 4) .. +31 = pixels of the tile
+        const int q = warp & 3;
+        const float* bias = theta + (int64_t)s * n_params + b_off;
+        int j = 0;
+        for (int it = blockIdx.x; it < n_items && ok; it += gridDim.x, ++j) {
+            const int buf = j & 1;
+            ok = mbar_wait(smem_u32(&acc_full[buf]), (j >> 1) & 1, err, kWaitDone);
+            if (!ok) break;
+            tc_fence_after_sync();
+            float v[32];
+            tmem_ld_32x32(tmem + ((uint32_t)(q * 32) << 16) + buf * kClassPad, v);
+            const int pix = it * kTileM + q * 32 + lane;
+            if (pix < p) {
+                float* dst = z + (int64_t)s * C * p + pix;
+#pragma unroll
+                for (int c = 0; c < kClassPad; ++c)
+                    if (c < C) dst[(int64_t)c * p] = v[c] + __ldg(bias + c);
+            }
+            tc_fence_before_sync();
+            __syncwarp();
+            if (lane == 0) mbar_arrive(smem_u32(&acc_empty[buf]));
+        }
+    }
+    if (!ok) drain_after_error();
+    tc_fence_before_sync();
+    __syncthreads();
+    if (warp == 0) tmem_dealloc(tmem, 2 * kClassPad);
+}
+
 template <int STAGES>
 __global__ void __launch_bounds__(kFwd3Threads)
 tc_fwd3x3_kernel(const __grid_constant__ CUtensorMap tmA,   // {Cin, w, h, S}    box {64, 32, 4, 1}
@@ -671,7 +787,8 @@ struct TcPlan {
     CUtensorMap dh_wg3;      // {Ch, w, h, S} box {64, 32, 2, 1}
     int split2, chunks2, per2, cols2, msplit2;
     int split1, chunks1, per1, cols1;
-    size_t smem_fwd1, smem_wg1, smem_fwd3, smem_wg3, smem_dgrad;
+    size_t smem_fwd1, smem_fwd1p, smem_wg1, smem_fwd3, smem_wg3, smem_dgrad;
+    bool fwd1_persistent;
     int n_sms;
 };
 
@@ -749,6 +866,16 @@ TcPlan* tc_plan_create(const TcBuffers& b, char* err, size_t err_len)
     split_geometry(P->chunks2, 148 / P->msplit2, &P->per2, &P->split2);
     P->cols2 = pow2_cols((m_last / P->msplit2) * kClassPad);
     P->smem_fwd1 = (size_t)(P->c_last / kBlockK) * (kTileM * 128 + kClassPad * 128) + kSmemAlign;
+    P->smem_fwd1p = (size_t)kF1Stages * kF1StageBytes + (size_t)(P->c_last / kBlockK) * kClassPad * 128 + kSmemAlign;
+    {
+        // The persistent form wins where every block has many tiles to stream (16 streams at 720p: 90 us against
+        // 110 us, 0.93 of the HBM copy bandwidth); with about three tiles per SM (one 720p stream) its partly filled
+        // last round costs more than the one-tile blocks' second wave.  ST_FWD1X1_PERSISTENT=0/1 forces a choice.
+        const int64_t tiles = (int64_t)((P->p + kTileM - 1) / kTileM) * b.S;
+        bool use = tiles >= (int64_t)6 * 148;
+        if (const char* e = getenv("ST_FWD1X1_PERSISTENT")) { if (e[0] == '0') use = false; else if (e[0] == '1') use = true; }
+        P->fwd1_persistent = use && P->smem_fwd1p <= (size_t)227 * 1024;
+    }
     P->smem_wg1 = kWg1Stages * ((size_t)(m_last / P->msplit2) * 2 * kChunkPix * 128 + kClassPad * 128) + kSmemAlign;
     if (b.c_hidden) {
         const int m_in = (b.c_in + kTileM - 1) / kTileM;
@@ -770,6 +897,7 @@ TcPlan* tc_plan_create(const TcBuffers& b, char* err, size_t err_len)
         delete P; return nullptr;
     }
     cudaError_t e = cudaFuncSetAttribute(tc_fwd1x1_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)P->smem_fwd1);
+    if (e == cudaSuccess && P->fwd1_persistent) e = cudaFuncSetAttribute(tc_fwd1x1p_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)P->smem_fwd1p);
     if (e == cudaSuccess) e = cudaFuncSetAttribute(tc_wgrad1x1_kernel<kWg1Stages>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)P->smem_wg1);
     if (b.c_hidden) {
         if (e == cudaSuccess) e = cudaFuncSetAttribute(tc_fwd3x3_kernel<4>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)P->smem_fwd3);
@@ -805,8 +933,16 @@ int tc_forward(const TcPlan* P, cudaStream_t s, StageTimer* t, const int* skip, 
         n += st_repeats(t);
     }
     const int tiles1 = (P->p + kTileM - 1) / kTileM;
-    ST_REPEAT(t) launch_chain(tc_fwd1x1_kernel, dim3(tiles1, b.S), dim3(kThreadsTc), P->smem_fwd1, s,
-        P->act_fwd, P->w2_map, b.theta, b.n_params, b.b2_off, b.z, b.C, P->p, P->c_last / kBlockK, b.err, skip, skip_stride);
+    if (P->fwd1_persistent) {
+        int gx = P->n_sms / b.S;
+        if (gx < 1) gx = 1;
+        if (gx > tiles1) gx = tiles1;
+        ST_REPEAT(t) launch_chain(tc_fwd1x1p_kernel, dim3(gx, b.S), dim3(kF1Threads), P->smem_fwd1p, s,
+            P->act_fwd, P->w2_map, b.theta, b.n_params, b.b2_off, b.z, b.C, P->p, P->c_last / kBlockK, b.err, skip, skip_stride);
+    } else {
+        ST_REPEAT(t) launch_chain(tc_fwd1x1_kernel, dim3(tiles1, b.S), dim3(kThreadsTc), P->smem_fwd1, s,
+            P->act_fwd, P->w2_map, b.theta, b.n_params, b.b2_off, b.z, b.C, P->p, P->c_last / kBlockK, b.err, skip, skip_stride);
+    }
     if (t) t->mark("tc_fwd1x1", s, st_repeats(t));
     return n + st_repeats(t);
 }
