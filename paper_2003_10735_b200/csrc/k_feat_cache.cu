@@ -3,63 +3,42 @@
 // the head's GEMMs read): fp32 [Cin][p] planar -> bf16 [p][Cin] (pixel-major, channels contiguous),
 // round-to-nearest-even.
 //
-// A dtype/layout change: Cin*p*4 bytes in, Cin*p*2 bytes out.  Tiles of 64 channels x 64 pixels go
-// through shared memory so that both the reads (along pixels) and the writes (along channels) are
-// full 128-byte lines: reads are 16-byte vectors of 4 pixels, writes 16-byte vectors of 8 channels.
+// A dtype/layout change: Cin*p*4 bytes in, Cin*p*2 bytes out.  A thread owns one pixel and 16 consecutive channels:
+// it reads 16 planes (each warp 128 contiguous bytes per plane, all 16 loads in flight) and writes one full 32-byte
+// sector of the pixel-major output.  No shared memory, no barrier (a version that transposed 64 x 64 tiles through
+// shared memory took 20.4 us at 720p against 18.5 us).  The tensor-core path only exists for channel counts that are
+// multiples of 64, so 16 always divides Cin here.
 #include "st_internal.h"
 
 namespace st {
 
-constexpr int kTileC = 64, kTileP = 64;
+constexpr int kFeatGroup = 16;
 
 __global__ void __launch_bounds__(256)
 feat_to_bf16_nhwc_kernel(const float* __restrict__ in, int Cin, int64_t p, bf16* __restrict__ out)
 {
-    __shared__ float tile[kTileC][kTileP + 1];
-    const int64_t p0 = (int64_t)blockIdx.x * kTileP;
-    const int c0 = blockIdx.y * kTileC;
-    const bool vec_in = (p % 4 == 0) && ((uintptr_t)in % 16 == 0);
-    // load: 64 channels x 16 quads
-    for (int i = threadIdx.x; i < kTileC * (kTileP / 4); i += 256) {
-        int c = i / (kTileP / 4), q = i % (kTileP / 4);
-        int64_t pp = p0 + q * 4;
-        float4 v = make_float4(0.f, 0.f, 0.f, 0.f);
-        if (c0 + c < Cin) {
-            const float* src = in + (int64_t)(c0 + c) * p + pp;
-            if (vec_in && pp + 3 < p) v = __ldcs(reinterpret_cast<const float4*>(src));
-            else {
-                if (pp + 0 < p) v.x = src[0];
-                if (pp + 1 < p) v.y = src[1];
-                if (pp + 2 < p) v.z = src[2];
-                if (pp + 3 < p) v.w = src[3];
-            }
-        }
-        tile[c][q * 4 + 0] = v.x; tile[c][q * 4 + 1] = v.y; tile[c][q * 4 + 2] = v.z; tile[c][q * 4 + 3] = v.w;
-    }
-    __syncthreads();
-    // store: 64 pixels x 8 groups of 8 channels
-    const bool vec_out = (Cin % 8 == 0) && ((uintptr_t)out % 16 == 0);
-    for (int i = threadIdx.x; i < kTileP * (kTileC / 8); i += 256) {
-        int px = i / (kTileC / 8), g = i % (kTileC / 8);
-        int64_t pp = p0 + px;
-        if (pp >= p) continue;
-        int c = c0 + g * 8;
-        if (vec_out && c + 7 < Cin) {
-            __nv_bfloat162 h[4];
+    const int64_t pix = (int64_t)blockIdx.x * 256 + threadIdx.x;
+    const int c0 = blockIdx.y * kFeatGroup;
+    if (pix >= p) return;
+    float v[kFeatGroup];
 #pragma unroll
-            for (int k = 0; k < 4; ++k)
-                h[k] = __floats2bfloat162_rn(tile[g * 8 + 2 * k][px], tile[g * 8 + 2 * k + 1][px]);
-            *reinterpret_cast<uint4*>(out + pp * Cin + c) = *reinterpret_cast<uint4*>(h);
-        } else {
-            for (int k = 0; k < 8; ++k)
-                if (c + k < Cin) out[pp * Cin + c + k] = __float2bfloat16_rn(tile[g * 8 + k][px]);
-        }
+    for (int k = 0; k < kFeatGroup; ++k) v[k] = (c0 + k < Cin) ? __ldcs(in + (int64_t)(c0 + k) * p + pix) : 0.f;
+    if (c0 + kFeatGroup <= Cin && ((uintptr_t)(out + pix * Cin + c0) % 16 == 0)) {
+        __nv_bfloat162 h[kFeatGroup / 2];
+#pragma unroll
+        for (int k = 0; k < kFeatGroup / 2; ++k) h[k] = __floats2bfloat162_rn(v[2 * k], v[2 * k + 1]);
+        uint4* dst = reinterpret_cast<uint4*>(out + pix * Cin + c0);
+#pragma unroll
+        for (int k = 0; k < kFeatGroup / 8; ++k) dst[k] = reinterpret_cast<uint4*>(h)[k];
+    } else {                                   // ragged channel count or unaligned output: element by element
+        for (int k = 0; k < kFeatGroup; ++k)
+            if (c0 + k < Cin) out[pix * Cin + c0 + k] = __float2bfloat16_rn(v[k]);
     }
 }
 
 void launch_feat_to_bf16_nhwc(const float* feat_chw, int Cin, int64_t p, bf16* out, cudaStream_t s)
 {
-    dim3 grid((unsigned)((p + kTileP - 1) / kTileP), (unsigned)((Cin + kTileC - 1) / kTileC));
+    dim3 grid((unsigned)((p + 255) / 256), (unsigned)((Cin + kFeatGroup - 1) / kFeatGroup));
     feat_to_bf16_nhwc_kernel<<<grid, 256, 0, s>>>(feat_chw, Cin, p, out);
 }
 
