@@ -478,8 +478,8 @@ tc_fwd3x3_kernel(const __grid_constant__ CUtensorMap tmA,   // {Cin, w, h, S}   
                         bits |= (__low2float(o2[k]) > 0.f ? 1u : 0u) << (2 * k);
                         bits |= (__high2float(o2[k]) > 0.f ? 1u : 0u) << (2 * k + 1);
                     }
-#pragma unroll
-                    for (int k = 0; k < 4; ++k) reinterpret_cast<uint4*>(dst + n0)[k] = out[k];
+                    store_256(dst + n0, reinterpret_cast<const uint32_t*>(out));            // 32 channels = 64 bytes
+                    store_256(dst + n0 + 16, reinterpret_cast<const uint32_t*>(out) + 8);
                     relu_bits[pixel * (Ch / 32) + (im.ch0 + n0) / 32] = bits;
                 }
             }
@@ -687,8 +687,8 @@ tc_dgrad_kernel(const __grid_constant__ CUtensorMap tmA,   // dz  {p, 32, S}  bo
                     if (!((bits >> (2 * k + 1)) & 1u)) v[2 * k + 1] = 0.f;
                     o2[k] = __floats2bfloat162_rn(v[2 * k], v[2 * k + 1]);
                 }
-#pragma unroll
-                for (int k = 0; k < 4; ++k) reinterpret_cast<uint4*>(dhidden + row + ch0 + n0)[k] = out[k];
+                store_256(dhidden + row + ch0 + n0, reinterpret_cast<const uint32_t*>(out));
+                store_256(dhidden + row + ch0 + n0 + 16, reinterpret_cast<const uint32_t*>(out) + 8);
             } else {
 #pragma unroll
                 for (int k = 0; k < 32; ++k) v[k] = 0.f;

@@ -20,6 +20,16 @@ typedef __nv_bfloat16 bf16;
 // pdl_wait() returns once the predecessor grid has completed and its writes are visible; no global
 // memory is read or written before it.  pdl_launch_dependents() lets the successor start launching.
 #ifdef __CUDACC__
+// One 32-byte store (a whole sector) from eight 32-bit registers; the address must be 32-byte aligned.  Where the
+// lanes of a warp write to rows that lie far apart (pixel-major activations), a sector written as two 16-byte halves
+// reaches L2 as two partial writes; this store writes it once.
+__device__ __forceinline__ void store_256(void* dst, const uint32_t* r)
+{
+    asm volatile("st.global.v8.b32 [%0], {%1, %2, %3, %4, %5, %6, %7, %8};"
+                 :: "l"(dst), "r"(r[0]), "r"(r[1]), "r"(r[2]), "r"(r[3]), "r"(r[4]), "r"(r[5]), "r"(r[6]), "r"(r[7])
+                 : "memory");
+}
+
 __device__ __forceinline__ void pdl_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
 __device__ __forceinline__ void pdl_launch_dependents() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
 
