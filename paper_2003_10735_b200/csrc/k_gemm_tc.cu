@@ -52,7 +52,8 @@ __global__ void __launch_bounds__(kThreadsTc)
 tc_fwd1x1_kernel(const __grid_constant__ CUtensorMap tmA,   // {K, p, S}  box {64, 128, 1}
                  const __grid_constant__ CUtensorMap tmB,   // {K, 32, S} box {64, 32, 1}
                  const float* __restrict__ theta, int64_t n_params, int64_t b_off,
-                 float* __restrict__ z, int C, int p, int kblocks, unsigned int* err, const int* __restrict__ skip, int64_t skip_stride)
+                 float* __restrict__ z, int C, int p, int kblocks, unsigned int* err, const int* __restrict__ skip, int64_t skip_stride,
+                 int a_early)
 {
     if (skip && skip[(int64_t)blockIdx.y * skip_stride]) return;   // this stream's training loop has ended (block-uniform)
     extern __shared__ uint8_t smem_raw[];
@@ -73,7 +74,17 @@ tc_fwd1x1_kernel(const __grid_constant__ CUtensorMap tmA,   // {K, p, S}  box {6
     __syncthreads();
     tc_fence_after_sync();
     const uint32_t tmem = tmem_slot;
-    pdl_wait();                  // inputs come from the previous kernel of the step
+    // a_early: the kernel before this one on the stream (the previous iteration's parameter update) writes the weights
+    // but not the activations, and this kernel was launched to start while that one still runs: the activation tile
+    // is fetched now, the weights after the wait.  Each barrier expects both parts.
+    if (a_early && tid == 0) {
+        for (int kb = 0; kb < kblocks; ++kb) {
+            const uint32_t bar = smem_u32(&bars[kb]);
+            mbar_expect_tx(bar, kTileM * 128 + kClassPad * 128);
+            tma_load_3d(a_base + kb * (kTileM * 128), &tmA, bar, kb * kBlockK, pix0, s);
+        }
+    }
+    pdl_wait();                  // the weights (and, without a_early, the activations) come from the previous kernel
     pdl_launch_dependents();
     const uint32_t done_bar = smem_u32(&bars[kblocks]);
     bool ok = true;
@@ -81,8 +92,10 @@ tc_fwd1x1_kernel(const __grid_constant__ CUtensorMap tmA,   // {K, p, S}  box {6
     if (tid == 0) {
         for (int kb = 0; kb < kblocks; ++kb) {
             const uint32_t bar = smem_u32(&bars[kb]);
-            mbar_expect_tx(bar, kTileM * 128 + kClassPad * 128);
-            tma_load_3d(a_base + kb * (kTileM * 128), &tmA, bar, kb * kBlockK, pix0, s);
+            if (!a_early) {
+                mbar_expect_tx(bar, kTileM * 128 + kClassPad * 128);
+                tma_load_3d(a_base + kb * (kTileM * 128), &tmA, bar, kb * kBlockK, pix0, s);
+            }
             tma_load_3d(b_base + kb * (kClassPad * 128), &tmB, bar, kb * kBlockK, 0, s);
         }
     } else if (tid == 32) {
@@ -910,7 +923,13 @@ TcPlan* tc_plan_create(const TcBuffers& b, char* err, size_t err_len)
 
 void tc_plan_destroy(TcPlan* P) { delete P; }
 
-int tc_forward(const TcPlan* P, cudaStream_t s, StageTimer* t, const int* skip, int64_t skip_stride)
+static bool fwd1_early_enabled()     // ST_FWD1_EARLY=0 switches the early activation fetch off
+{
+    static const bool on = [] { const char* e = getenv("ST_FWD1_EARLY"); return !(e && e[0] == '0'); }();
+    return on;
+}
+
+int tc_forward(const TcPlan* P, cudaStream_t s, StageTimer* t, const int* skip, int64_t skip_stride, bool after_update)
 {
     const TcBuffers& b = P->b;
     int n = 0;
@@ -940,8 +959,12 @@ int tc_forward(const TcPlan* P, cudaStream_t s, StageTimer* t, const int* skip, 
         ST_REPEAT(t) launch_chain(tc_fwd1x1p_kernel, dim3(gx, b.S), dim3(kF1Threads), P->smem_fwd1p, s,
             P->act_fwd, P->w2_map, b.theta, b.n_params, b.b2_off, b.z, b.C, P->p, P->c_last / kBlockK, b.err, skip, skip_stride);
     } else {
-        ST_REPEAT(t) launch_chain(tc_fwd1x1_kernel, dim3(tiles1, b.S), dim3(kThreadsTc), P->smem_fwd1, s,
-            P->act_fwd, P->w2_map, b.theta, b.n_params, b.b2_off, b.z, b.C, P->p, P->c_last / kBlockK, b.err, skip, skip_stride);
+        // one-layer head, no per-stream skip flags to wait for, not a timing run: the activations are the frozen
+        // features, which no kernel of the loop writes
+        const bool a_early = after_update && !b.c_hidden && !skip && !t && fwd1_early_enabled();
+        ST_REPEAT(t) launch_early(a_early || pdl_enabled(), tc_fwd1x1_kernel, dim3(tiles1, b.S), dim3(kThreadsTc), P->smem_fwd1, s,
+            P->act_fwd, P->w2_map, b.theta, b.n_params, b.b2_off, b.z, b.C, P->p, P->c_last / kBlockK, b.err, skip, skip_stride,
+            a_early ? 1 : 0);
     }
     if (t) t->mark("tc_fwd1x1", s, st_repeats(t));
     return n + st_repeats(t);

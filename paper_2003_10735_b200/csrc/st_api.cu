@@ -209,11 +209,12 @@ UpdateArgs make_update_args(st_ctx* c, int slot, const int* skip = nullptr, int6
 
 // Forward of the trainable part for all streams: z (and the hidden activation).
 // `skip` (tensor-core kernels only): per-stream flags, see tc_forward.
-st_status enqueue_forward(st_ctx* c, StageTimer* t = nullptr, const int* skip = nullptr, int64_t skip_stride = 0)
+st_status enqueue_forward(st_ctx* c, StageTimer* t = nullptr, const int* skip = nullptr, int64_t skip_stride = 0,
+                          bool after_update = false)
 {
     cudaStream_t s = c->stream;
     if (c->bf16_mode) {
-        c->launches += tc_forward(c->plan, s, t, skip, skip_stride);
+        c->launches += tc_forward(c->plan, s, t, skip, skip_stride, after_update);
     } else if (c->Ch == 0) {
         ST_REPEAT(t) launch_conv_fwd_f32(c->x_f32, c->Cin, c->h, c->w, c->theta + c->layout.w_off[0], c->theta + c->layout.b_off[0],
                             c->C, 1, false, c->z, c->S, (int64_t)c->Cin * c->p, c->n_params, c->n_params,
@@ -314,7 +315,8 @@ st_status enqueue_update(st_ctx* c, int slot, const int* skip, int64_t skip_stri
 
 st_status enqueue_step(st_ctx* c, int slot, bool want_conf, StageTimer* t = nullptr)
 {
-    st_status st = enqueue_forward(c, t);
+    // iterations after the first follow the previous iteration's update directly
+    st_status st = enqueue_forward(c, t, nullptr, 0, slot > 0 && !t);
     if (st == ST_OK) st = enqueue_loss(c, want_conf ? c->conf_buf + (int64_t)slot * c->C * c->C : nullptr, t);
     if (st == ST_OK) st = enqueue_backward(c, t);
     if (st == ST_OK) st = enqueue_update(c, slot, nullptr, 0, t);

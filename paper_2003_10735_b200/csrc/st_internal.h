@@ -35,16 +35,24 @@ __device__ __forceinline__ void pdl_launch_dependents() { asm volatile("griddepc
 
 bool pdl_enabled();   // true if the environment variable ST_PDL is set to 1 (off by default: it measured no gain)
 
+// `early`: launch with the programmatic-serialization attribute, i.e. the kernel may start before its predecessor on
+// the stream has completed and must call pdl_wait() before it touches anything the predecessor writes.
 template <typename... KArgs, typename... Args>
-inline cudaError_t launch_chain(void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t smem, cudaStream_t s, Args&&... args)
+inline cudaError_t launch_early(bool early, void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t smem, cudaStream_t s, Args&&... args)
 {
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = grid; cfg.blockDim = block; cfg.dynamicSmemBytes = smem; cfg.stream = s;
     cudaLaunchAttribute at[1];
     at[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
     at[0].val.programmaticStreamSerializationAllowed = 1;
-    cfg.attrs = at; cfg.numAttrs = pdl_enabled() ? 1 : 0;
+    cfg.attrs = at; cfg.numAttrs = early ? 1 : 0;
     return cudaLaunchKernelEx(&cfg, kernel, std::forward<Args>(args)...);
+}
+
+template <typename... KArgs, typename... Args>
+inline cudaError_t launch_chain(void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t smem, cudaStream_t s, Args&&... args)
+{
+    return launch_early(pdl_enabled(), kernel, grid, block, smem, s, std::forward<Args>(args)...);
 }
 #endif
 
@@ -252,7 +260,11 @@ struct StageTimer {
 #define ST_REPEAT(t) for (int r_ = 0, R_ = (t) ? (t)->repeat : 1; r_ < R_; ++r_)
 inline int st_repeats(const StageTimer* t) { return t ? t->repeat : 1; }
 // `skip`: nullptr, or one flag per stream (skip[s * skip_stride]); the blocks of a flagged stream return at once.
-int tc_forward(const TcPlan*, cudaStream_t s, StageTimer* t = nullptr, const int* skip = nullptr, int64_t skip_stride = 0);    // returns the number of kernels launched
+// Returns the number of kernels launched.  `after_update`: the kernel launched just before on this stream is the
+// parameter update of the previous iteration, which writes weights but no activations; the forward of a one-layer head
+// may then fetch its activation tiles while that update is still running.
+int tc_forward(const TcPlan*, cudaStream_t s, StageTimer* t = nullptr, const int* skip = nullptr, int64_t skip_stride = 0,
+               bool after_update = false);
 int tc_backward(const TcPlan*, cudaStream_t s, StageTimer* t = nullptr, const int* skip = nullptr, int64_t skip_stride = 0);
 
 }  // namespace st
