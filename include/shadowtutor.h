@@ -292,12 +292,14 @@ ST_API st_status st_agreement_noalloc(const uint8_t *pred, const uint8_t *label,
 ST_API int32_t st_next_stride(int32_t stride, double metric, double threshold, int32_t min_stride, int32_t max_stride);
 
 /*
- * st_client_schedule — the key frames the client's loop (Algorithm 4) picks among n_frames frames: the first
- * frame is a key frame; after a key frame the reply (updated part, metric) is complete `delay` frames later, at
- * step = MIN_STRIDE at the latest (the client then waits for it), and the stride is recomputed with
- * st_next_stride when it completes; the next key frame is the frame at which step = stride.
+ * st_client_schedule — the key frames the client's loop (Algorithm 4) picks among n_frames frames.  The first
+ * frame is a key frame.  The reply to a key frame (updated part, metric) is applied min(delay, MIN_STRIDE) frames
+ * after it: when it has arrived, or when the client stops to wait for it (Section 4.3).  The stride is recomputed with
+ * st_next_stride at that moment and counts from the key frame, so the next key frame is NextStride(stride, metric)
+ * frames after the last one, whatever the delay.
  *   metrics       host; metrics[j] = metric returned for the j-th key frame; n_metrics entries.
- *   delay         frames until a reply is complete, >= 1.
+ *   delay         frames until a reply is complete, >= 1 (it decides when an update is applied, not where the key
+ *                 frames fall).
  *   key_frames    host, capacity entries; receives the frame indices.
  *   n_key_frames  host; receives their number (also when capacity is too small: ST_ERR_BUFFER_TOO_SMALL).
  * ST_ERR_INVALID_ARG: bad parameters (threshold must lie strictly between 0 and 1), or fewer metrics than key frames.

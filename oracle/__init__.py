@@ -296,25 +296,22 @@ def student_mask(head: Head, feat: np.ndarray) -> np.ndarray:
     return teacher_labels(upsample(z, head.up))
 
 
-def gradients(head: Head, feat: np.ndarray, labels: np.ndarray):
-    """Loss and gradient of every trainable tensor (flat, packed order) at the current parameters.
+def head_backward(head: Head, x: np.ndarray, Hd: Optional[np.ndarray], dz: np.ndarray) -> np.ndarray:
+    """PartialBackward from the logit gradient on (Algorithm 1; Section 4.2): the gradient of every trainable
+    tensor, flat, in packed order.  `x` is the frozen part's output as the forward saw it, `Hd` the hidden
+    activation of that forward (None for the 1x1 head), `dz` the gradient of the loss with respect to the
+    head's logits.  No gradient is formed for `x`.
 
-    Also returns the student mask of this forward (the prediction the loss was computed from).
+    With ``quantize_bf16`` the operands of the products are rounded where the tensor-core path rounds them:
+    dz where it meets the activations (weight gradient) and the weights (gradient passed back), the 1x1
+    weight, and the hidden gradient where it meets `x`.  The bias gradients are sums of the unrounded values.
     """
-    x = head._q(np.ascontiguousarray(feat, dtype=head.dtype))
     layers = head.layers()
-    z, Hd = head_forward(head, feat)
-    u = upsample(z, head.up)
-    wgt = object_weights(labels, head.background, head.object_radius, head.object_weight) if head.object_weight > 1 else None
-    loss, g, _ = softmax_ce(u, labels, weights=wgt)
-    mask = teacher_labels(u)
-    dz = upsample_adjoint(g, head.up)
     if head.c_hidden == 0:
         dW, db = conv_wgrad(x, head._q(dz), 1)
         if head.quantize_bf16:
             db = bias_grad(dz)
-        grad = np.concatenate([dW.ravel(), db.ravel()])
-        return loss, grad, mask
+        return np.concatenate([dW.ravel(), db.ravel()])
     (W1, b1), (W2, b2) = layers
     dW2, db2 = conv_wgrad(Hd, head._q(dz), 1)
     dH = conv1x1_dgrad(head._q(W2.reshape(W2.shape[0], W2.shape[1])), head._q(dz))
@@ -322,8 +319,22 @@ def gradients(head: Head, feat: np.ndarray, labels: np.ndarray):
     dW1, db1 = conv_wgrad(x, head._q(dH), 3)
     if head.quantize_bf16:
         db2, db1 = bias_grad(dz), bias_grad(dH)
-    grad = np.concatenate([dW1.ravel(), db1.ravel(), dW2.ravel(), db2.ravel()])
-    return loss, grad, mask
+    return np.concatenate([dW1.ravel(), db1.ravel(), dW2.ravel(), db2.ravel()])
+
+
+def gradients(head: Head, feat: np.ndarray, labels: np.ndarray):
+    """Loss and gradient of every trainable tensor (flat, packed order) at the current parameters.
+
+    Also returns the student mask of this forward (the prediction the loss was computed from).
+    """
+    x = head._q(np.ascontiguousarray(feat, dtype=head.dtype))
+    z, Hd = head_forward(head, feat)
+    u = upsample(z, head.up)
+    wgt = object_weights(labels, head.background, head.object_radius, head.object_weight) if head.object_weight > 1 else None
+    loss, g, _ = softmax_ce(u, labels, weights=wgt)
+    mask = teacher_labels(u)
+    dz = upsample_adjoint(g, head.up)
+    return loss, head_backward(head, x, Hd, dz), mask
 
 
 def distill_step(head: Head, feat: np.ndarray, labels: np.ndarray):
@@ -360,28 +371,31 @@ class TrainResult:
 
 def train_key_frame(head: Head, feat: np.ndarray, labels: np.ndarray, threshold: float, max_updates: int,
                     keep_masks: bool = False) -> TrainResult:
-    """Algorithm 1, Train(student, frame, label), in the paper's order and names.
+    """Train(student, frame, label) of Algorithm 1.
 
+    The incoming student is judged first and is the first best_student; distillation is skipped when it
+    already meets the threshold.  Otherwise up to `max_updates` optimisation steps follow, each judged by
+    the metric of the prediction made after it; the best iterate so far is remembered (a later one has to
+    be strictly better) and the loop ends at the first metric above the threshold.
     The metric is the mean IoU of Section 3.2 between the student's mask and the pseudo-label.
     On return ``head.theta`` holds best_student (Algorithm 3 continues with the returned student);
     the momentum buffer is optimiser state, not part of the student, and keeps running.
     """
     C = head.n_classes
-    prediction = student_mask(head, feat)                               # prediction <- Forward(student, frame)
-    best_metric = agreement(labels, prediction, C)[1]                   # best_metric <- ComputeMetric(prediction, label)
-    best_student = head.theta.copy()                                    # best_student <- student
+    prediction = student_mask(head, feat)
+    best_metric = agreement(labels, prediction, C)[1]
+    best_student = head.theta.copy()
     res = TrainResult(best_metric, 0, 0, [best_metric], [])
     if keep_masks:
         res.masks.append(prediction)
-    if best_metric < threshold:                                         # skip distillation when already good enough
+    if best_metric < threshold:
         for i in range(1, max_updates + 1):
-            # loss <- ComputeLoss(prediction, label); gradients <- PartialBackward(loss); student <- OptimStep(...)
-            # (the loss is a function of the same parameters that produced `prediction`)
+            # the loss is a function of the same parameters that produced the prediction judged last
             loss, _ = distill_step(head, feat, labels)
             res.losses.append(loss)
             res.n_updates = i
-            prediction = student_mask(head, feat)                       # prediction <- Forward(student, frame)
-            metric = agreement(labels, prediction, C)[1]                # metric <- ComputeMetric(prediction, label)
+            prediction = student_mask(head, feat)
+            metric = agreement(labels, prediction, C)[1]
             res.metrics.append(metric)
             if keep_masks:
                 res.masks.append(prediction)

@@ -24,29 +24,19 @@ st_status st_client_schedule(int64_t n_frames, const double* metrics, int64_t n_
     if (n_frames < 0 || !n_key_frames || min_stride < 1 || max_stride < min_stride || delay < 1 || !(threshold > 0.0 && threshold < 1.0))
         return ST_ERR_INVALID_ARG;
     if ((n_metrics > 0 && !metrics) || (capacity > 0 && !key_frames)) return ST_ERR_INVALID_ARG;
+    // Key frame to key frame, no per-frame bookkeeping.  The reply to the key frame at frame f (updated part and
+    // metric) is applied min(delay, MIN_STRIDE) frames later: when it has arrived, or when the client stops to
+    // wait for it.  The stride recomputed at that moment is at least MIN_STRIDE, so the frames counted since f
+    // have not passed it yet, and the next key frame is frame f + NextStride(stride, metric) whatever the delay.
     int64_t n_keys = 0;
-    int32_t stride = min_stride, step = stride;           // the first frame is a key frame
-    bool updated = true;
-    double metric = 0.0;
+    int32_t stride = min_stride;
     st_status status = ST_OK;
-    for (int64_t f = 0; f < n_frames; ++f) {
-        if (step == stride) {                              // key frame: frame goes out, the reply is awaited
-            if (n_keys >= n_metrics) { status = ST_ERR_INVALID_ARG; break; }      // ran out of metrics
-            metric = metrics[n_keys];
-            if (n_keys < capacity) key_frames[n_keys] = f;
-            else status = ST_ERR_BUFFER_TOO_SMALL;         // keep counting
-            ++n_keys;
-            step = 0;
-            updated = false;
-        }
-        ++step;                                            // student inference on this frame
-        if (!updated) {
-            const bool completed = step >= delay || step == min_stride;   // at MIN_STRIDE the client waits for the reply
-            if (completed) {
-                stride = st_next_stride(stride, metric, threshold, min_stride, max_stride);
-                updated = true;
-            }
-        }
+    for (int64_t f = 0; f < n_frames; f += stride) {
+        if (n_keys >= n_metrics) { status = ST_ERR_INVALID_ARG; break; }          // this key frame has no metric
+        if (n_keys < capacity) key_frames[n_keys] = f;
+        else status = ST_ERR_BUFFER_TOO_SMALL;                                     // keep counting
+        stride = st_next_stride(stride, metrics[n_keys], threshold, min_stride, max_stride);
+        ++n_keys;
     }
     *n_key_frames = n_keys;
     return status;

@@ -7,7 +7,7 @@ import pytest
 
 import paper_2003_10735_b200 as st
 from oracle import schedule as sch
-from test_schedule_pins import G, L, MIN, MAX
+from test_schedule_pins import G, L, MIN, MAX, hand_traces
 
 
 def lat():
@@ -29,7 +29,11 @@ def test_client_schedule_matches_the_oracle(delay):
     metrics = [rnd.random() for _ in range(700)]
     for n in (0, 1, 7, 8, 9, 500, 5000):
         assert st.st_client_schedule(n, metrics, 0.8, MIN, MAX, delay) == sch.client_schedule(n, metrics, 0.8, MIN, MAX, delay)
-    assert st.st_client_schedule(200, [1.0] * 10, 0.8, 8, 64, 1) == [0, 16, 48, 112, 176]     # the hand trace
+
+
+def test_client_schedule_reproduces_the_hand_worked_sequences():
+    for n, delay, metrics, keys in hand_traces():
+        assert st.st_client_schedule(n, metrics, G["threshold"], MIN, MAX, delay) == keys, (n, delay, metrics)
 
 
 def test_client_schedule_errors():

@@ -78,16 +78,24 @@ def test_next_stride_clamps_and_truncates():
     assert sch.next_stride(16, T, T, MIN, MAX) == 16                     # at the threshold the stride stays
 
 
+def hand_traces():
+    """(n_frames, delay, metrics, key frames) of every case in tests/golden/client_schedule_traces.txt."""
+    out = []
+    with open(os.path.join(os.path.dirname(GOLDEN), "client_schedule_traces.txt")) as f:
+        for line in f:
+            if not line.strip() or line.startswith("#"):
+                continue
+            head, metrics, keys = line.split("|")
+            n, delay = (int(t) for t in head.split())
+            out.append((n, delay, [float(t) for t in metrics.split()], [int(t) for t in keys.split()]))
+    return out
+
+
 def test_client_schedule_hand_traces():
-    T = 0.8
-    # metric always at the threshold: the stride stays MIN_STRIDE, every 8th frame is a key frame
-    assert sch.client_schedule(40, [T] * 10, T, 8, 64, delay=3) == [0, 8, 16, 24, 32]
-    # perfect student: 8 -> 16 -> 32 -> 64 -> 64: key frames at 0, then 16 later, 32 later, 64 later ...
-    assert sch.client_schedule(200, [1.0] * 10, T, 8, 64, delay=1) == [0, 16, 48, 112, 176]
-    # the new stride applies to the running count: a reply that lands late (at step = MIN_STRIDE) still stretches it
-    assert sch.client_schedule(200, [1.0] * 10, T, 8, 64, delay=100) == [0, 16, 48, 112, 176]
-    # a poor student after a good one: 8 -> 16, then metric 0.4 halves it back to 8
-    assert sch.client_schedule(60, [1.0, 0.4, 0.4, 0.4, 0.4, 0.4, 0.4], T, 8, 64, delay=2) == [0, 16, 24, 32, 40, 48, 56]
+    traces = hand_traces()
+    assert len(traces) >= 9
+    for n, delay, metrics, keys in traces:
+        assert sch.client_schedule(n, metrics, G["threshold"], MIN, MAX, delay) == keys, (n, delay, metrics)
 
 
 @pytest.mark.parametrize("delay", [1, 4, 8, 50])
