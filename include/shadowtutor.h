@@ -17,6 +17,8 @@
  *   - The caller owns every buffer it passes.  The library reads or writes it only on the
  *     context's CUDA stream during work enqueued by that call; it keeps no reference
  *     afterwards.  Inputs must stay alive until the stream has passed that work.
+ *   - No pointer needs more than the alignment of its element type (one byte for label maps and masks, four
+ *     for fp32 tensors); 16-byte aligned, contiguous buffers take the fastest paths.
  *   - Calls enqueue work on `cuda_stream` and return.  Only calls with a host out-value
  *     (`st_pack_updated_params` with a host destination, `st_agreement` unless its `miou` is a
  *     device pointer, `st_read_tensor`) wait for the stream.

@@ -887,6 +887,9 @@ TcPlan* tc_plan_create(const TcBuffers& b, char* err, size_t err_len)
         const int64_t tiles = (int64_t)((P->p + kTileM - 1) / kTileM) * b.S;
         bool use = tiles >= (int64_t)6 * 148;
         if (const char* e = getenv("ST_FWD1X1_PERSISTENT")) { if (e[0] == '0') use = false; else if (e[0] == '1') use = true; }
+        // the one-tile form keeps the whole channel extent of its tile in shared memory: beyond 704 channels it no
+        // longer fits, and the persistent form (a ring of eight stages, whatever the channel count) takes over
+        if (P->smem_fwd1 > (size_t)227 * 1024) use = true;
         P->fwd1_persistent = use && P->smem_fwd1p <= (size_t)227 * 1024;
     }
     P->smem_wg1 = kWg1Stages * ((size_t)(m_last / P->msplit2) * 2 * kChunkPix * 128 + kClassPad * 128) + kSmemAlign;
@@ -904,12 +907,13 @@ TcPlan* tc_plan_create(const TcBuffers& b, char* err, size_t err_len)
         }
     }
     const size_t lim = 227 * 1024;
-    if (P->c_last / kBlockK > kMaxKBlocks || P->smem_fwd1 > lim || P->smem_wg1 > lim || P->smem_fwd3 > lim ||
+    if (P->c_last / kBlockK > kMaxKBlocks || (!P->fwd1_persistent && P->smem_fwd1 > lim) || P->smem_wg1 > lim || P->smem_fwd3 > lim ||
         P->smem_wg3 > lim || P->smem_dgrad > lim) {
         snprintf(err, err_len, "shared memory per block exceeds 227 KB for these channel counts");
         delete P; return nullptr;
     }
-    cudaError_t e = cudaFuncSetAttribute(tc_fwd1x1_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)P->smem_fwd1);
+    cudaError_t e = cudaSuccess;
+    if (!P->fwd1_persistent) e = cudaFuncSetAttribute(tc_fwd1x1_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)P->smem_fwd1);
     if (e == cudaSuccess && P->fwd1_persistent) e = cudaFuncSetAttribute(tc_fwd1x1p_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)P->smem_fwd1p);
     if (e == cudaSuccess) e = cudaFuncSetAttribute(tc_wgrad1x1_kernel<kWg1Stages>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)P->smem_wg1);
     if (b.c_hidden) {

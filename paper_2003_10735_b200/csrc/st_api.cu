@@ -889,15 +889,16 @@ st_status st_student_mask(st_ctx* ctx, int32_t stream, uint8_t* mask_out)
     st = student_forward(ctx, stream, "st_student_mask");
     if (st != ST_OK) return st;
     const bool dev = is_device_ptr(mask_out);
-    uint8_t* dst = dev ? mask_out : ctx->mask_tmp;
+    // the kernel writes the mask two pixels (16 bits) at a time: a destination at an odd address gets its
+    // mask through the context's own buffer
+    const bool direct = dev && ((uintptr_t)mask_out & 1u) == 0;
+    uint8_t* dst = direct ? mask_out : ctx->mask_tmp;
     launch_student_mask(mask_args(ctx, stream, dst), ctx->stream);
     ctx->launches += 1;
     st = check_launch(ctx, "student mask");
     if (st != ST_OK) return st;
-    if (!dev) {
-        ST_CUDA(ctx, cudaMemcpyAsync(mask_out, dst, (size_t)ctx->P, cudaMemcpyDeviceToHost, ctx->stream));
-        ST_CUDA(ctx, cudaStreamSynchronize(ctx->stream));
-    }
+    if (!direct) ST_CUDA(ctx, cudaMemcpyAsync(mask_out, dst, (size_t)ctx->P, cudaMemcpyDefault, ctx->stream));
+    if (!dev) ST_CUDA(ctx, cudaStreamSynchronize(ctx->stream));
     return ST_OK;
 }
 
@@ -908,9 +909,11 @@ st_status st_agreement(st_ctx* ctx, int32_t stream, const uint8_t* pred, const u
     const uint8_t* d_label = nullptr;
     const uint8_t* d_pred = nullptr;
     if (label) {
-        if (is_device_ptr(label)) d_label = label;
+        // the fused kernel reads labels two pixels (16 bits) at a time: a device map at an odd address is copied
+        // into the context's buffer like a host map (the plain confusion kernel takes any address)
+        if (is_device_ptr(label) && (pred || ((uintptr_t)label & 1u) == 0)) d_label = label;
         else {
-            ST_CUDA(ctx, cudaMemcpyAsync(ctx->mask_tmp2, label, (size_t)ctx->P, cudaMemcpyHostToDevice, ctx->stream));
+            ST_CUDA(ctx, cudaMemcpyAsync(ctx->mask_tmp2, label, (size_t)ctx->P, cudaMemcpyDefault, ctx->stream));
             d_label = ctx->mask_tmp2;
         }
     } else {

@@ -57,6 +57,7 @@ def test_status_names(lib):
     (dict(gemm_precision=1, c_in=48), st.ST_ERR_UNSUPPORTED),
     (dict(gemm_precision=1, c_in=64, n_classes=40), st.ST_ERR_UNSUPPORTED),
     (dict(gemm_precision=1, c_in=64, c_hidden=320), st.ST_ERR_UNSUPPORTED),
+    (dict(gemm_precision=1, c_in=1088), st.ST_ERR_UNSUPPORTED),         # the advertised bound of the bf16 path: c_in <= 1024
 ])
 def test_init_rejects_bad_descriptions_on_the_host(lib, kw, status):
     args = dict(n_streams=1, c_in=8, c_hidden=0, n_classes=3, feat_h=4, feat_w=4, up=4, gemm_precision=0,

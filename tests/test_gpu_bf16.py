@@ -79,6 +79,8 @@ def test_feature_cache_rounds_to_nearest_even(c_in, h, w):
     (128, 21, 24, 40),   # several tiles and a half one
     (256, 32, 17, 31),   # all 32 class rows in use, two channel accumulators
     (192, 2, 8, 8),      # channel count that is not a multiple of 128
+    (768, 21, 10, 30),   # more channels than the one-tile forward can hold in shared memory: the persistent form serves
+    (1024, 4, 6, 9),     # the largest channel count the path accepts
 ])
 def test_1x1_head_single_step_intermediates(c_in, C, h, w):
     feat, T = problem(3, c_in, C, h, w)

@@ -101,6 +101,41 @@ def test_confusion_and_miou_bit_exact(C, h, w):
     st.st_destroy(ctx)
 
 
+def test_masks_at_odd_addresses_give_the_same_results():
+    """Label maps and masks are byte arrays: a view that starts at an odd address (a tensor sliced by one byte) must
+    give the same mask, confusion matrix and mean IoU as an aligned buffer."""
+    C, c_in, h, w = 5, 8, 9, 14
+    P = 16 * h * w
+    feat, T = rand_problem(3, c_in, C, h, w)
+    ctx = make_ctx(c_in, 0, C, h, w, si.initial_head_params(c_in, 0, C, 4))
+    st.st_set_frozen_features(ctx, 0, dev(feat))
+    st.st_teacher_labels(ctx, 0, dev(T))
+    lab = oracle.teacher_labels(T)
+    mask = torch.empty((4 * h, 4 * w), dtype=torch.uint8, device="cuda")
+    st.st_student_mask(ctx, 0, mask)
+    conf = torch.zeros((C, C), dtype=torch.int64, device="cuda")
+    m = st.st_agreement(ctx, 0, None, dev(lab), conf)
+    for shift in (1, 3):
+        raw = torch.zeros(P + 16, dtype=torch.uint8, device="cuda")
+        mask_odd = raw[shift:shift + P]
+        assert mask_odd.data_ptr() % 2 == 1
+        st.st_student_mask(ctx, 0, mask_odd)
+        assert torch.equal(mask_odd.view(4 * h, 4 * w), mask) and int(raw[:shift].sum()) == 0 and int(raw[shift + P:].sum()) == 0
+        lab_raw = torch.zeros(P + 16, dtype=torch.uint8, device="cuda")
+        lab_odd = lab_raw[shift:shift + P]
+        lab_odd.copy_(dev(lab).view(-1))
+        conf2 = torch.zeros_like(conf)
+        assert st.st_agreement(ctx, 0, None, lab_odd, conf2) == m               # the student's own mask, fused kernel
+        assert torch.equal(conf2, conf)
+        conf3 = torch.zeros_like(conf)
+        assert st.st_agreement(ctx, 0, mask_odd, lab_odd, conf3) == m           # two masks, both at odd addresses
+        assert torch.equal(conf3, conf)
+    ref_conf, ref_m, _ = oracle.agreement(lab, mask.cpu().numpy(), C)
+    np.testing.assert_array_equal(conf.cpu().numpy(), ref_conf)
+    assert m == ref_m
+    st.st_destroy(ctx)
+
+
 def test_agreement_reports_out_of_range_labels():
     C, h, w = 3, 2, 2
     lab = np.zeros((8, 8), np.uint8)

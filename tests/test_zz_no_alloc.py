@@ -55,3 +55,33 @@ def test_noalloc_rejects_sizes_beyond_its_fixed_scratch():
     with pytest.raises(st.StError) as ei:
         st.st_agreement_noalloc(d, d, 1, 0, conf, miou)
     assert ei.value.status == st.ST_ERR_INVALID_ARG
+
+
+def test_noalloc_allocates_nothing_and_takes_any_length_and_address():
+    """Once the first call on the device has looked the internal array up, a call leaves the device's free memory
+    as it found it.  Masks whose length is not a multiple of 16 and that start at an odd address go through the
+    kernel's pixel-by-pixel path and are checked against a count made with numpy."""
+    C, n = 7, 16 * 1000 + 11
+    rng = np.random.default_rng(5)
+    lab = rng.integers(0, C, n).astype(np.uint8)
+    pred = np.where(rng.random(n) < 0.5, lab, rng.integers(0, C, n)).astype(np.uint8)
+    stream = torch.cuda.Stream()
+    with torch.cuda.stream(stream):
+        raw_l = torch.zeros(n + 16, dtype=torch.uint8, device="cuda")
+        raw_p = torch.zeros(n + 16, dtype=torch.uint8, device="cuda")
+        d_lab, d_pred = raw_l[1:1 + n], raw_p[3:3 + n]
+        d_lab.copy_(torch.from_numpy(lab).cuda()); d_pred.copy_(torch.from_numpy(pred).cuda())
+        assert d_lab.data_ptr() % 2 == 1 and d_pred.data_ptr() % 2 == 1
+        conf = torch.empty((C, C), dtype=torch.int64, device="cuda")
+        miou = torch.empty(1, dtype=torch.float64, device="cuda")
+        st.st_agreement_noalloc(d_pred, d_lab, C, stream.cuda_stream, conf, miou)     # the set-up call, if none came before
+        stream.synchronize()
+        free_before = torch.cuda.mem_get_info()[0]
+        st.st_agreement_noalloc(d_pred, d_lab, C, stream.cuda_stream, conf, miou)
+        stream.synchronize()
+        assert torch.cuda.mem_get_info()[0] == free_before
+    ref = np.bincount(lab.astype(np.int64) * C + pred, minlength=C * C).reshape(C, C)
+    np.testing.assert_array_equal(conf.cpu().numpy(), ref)
+    rows, cols, diag = ref.sum(1), ref.sum(0), np.diag(ref)
+    present = rows > 0
+    assert miou.item() == pytest.approx(float(np.mean(diag[present] / (rows + cols - diag)[present])), rel=1e-14)
