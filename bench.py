@@ -32,7 +32,12 @@ import synth_inputs as si  # noqa: E402
 
 METRIC = "720p key-frame partial-distill steps/s (K=8)"
 N_SETS = 4            # distinct key frames the device-resident run rotates over (4 x 136 MB > 126 MB L2)
-ALU_FLOP_PER_CLASS_PIXEL = 20.0   # algorithmic fp32 work of the fused upsample+CE kernel (10 FMA-equivalents)
+# Algorithmic work of the fused upsample + cross-entropy kernel per class and frame pixel: two horizontal and one vertical
+# interpolation step, exponent scale and shift, the sum, the normalisation and three adjoint multiply-adds -- 10
+# multiply-add equivalents = 20 flop (12 to 16 separate fp32 operations when written without fused multiply-adds) --
+# and one exponential.
+ALU_FLOP_PER_CLASS_PIXEL = 20.0
+EX2_PER_CLASS_PIXEL = 1.0
 # dram__bytes_read.sum + dram__bytes_write.sum per launch, ncu capture of (workload, kernel); see profiles/.
 # An entry is removed whenever its kernel changes and put back after the next capture.
 NCU_DRAM_BYTES = {
@@ -66,7 +71,7 @@ class ClockSampler:
         try:
             self.proc = subprocess.Popen(
                 ["nvidia-smi", "-i", str(gpu_index), f"--query-gpu={self.FIELDS}", "--format=csv,noheader,nounits",
-                 "-lms", "100"], stdout=open(self.path, "w"), stderr=subprocess.DEVNULL)
+                 "-lms", "50"], stdout=open(self.path, "w"), stderr=subprocess.DEVNULL)
         except OSError:
             self.proc = None
         self.t0 = self.t1 = None
@@ -198,6 +203,137 @@ def whole_job_rate(units_per_rank: float, world: int, ms_max: float) -> float:
 # --------------------------------------------------------------------------------------------
 # the CUDA path
 # --------------------------------------------------------------------------------------------
+def timed_blocks(torch, stream, barrier, n_blocks, steps, body, between=None):
+    """ms of each of n_blocks timed regions of `steps` calls of body(i), each bracketed by barrier + synchronize
+    and timed with CUDA events on the launching stream; `between` runs outside the timed regions."""
+    ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    out, i = [], 0
+    for _ in range(n_blocks):
+        if between is not None:
+            between()
+        barrier()
+        ev0.record(stream)
+        for _ in range(steps):
+            body(i)
+            i += 1
+        ev1.record(stream)
+        barrier()
+        out.append(ev0.elapsed_time(ev1))
+    return out
+
+
+def kernel_table(st, ctx, cfg, peaks, arith, n_profile_steps):
+    """Per-kernel CUDA-event times of one step (st_profile_step) with the roofline each kernel is held against."""
+    S, C, K = cfg.n_streams, cfg.n_classes, cfg.k_steps
+    p, P = cfg.feat_h * cfg.feat_w, cfg.frame_h * cfg.frame_w
+    c_last = cfg.c_hidden or cfg.c_in
+    hbm, tensor_peak = peaks["hbm_gbs"], peaks["bf16_tflops"]
+    kernels = {}
+    for name, ms in st.st_profile_step(ctx, n_profile_steps):
+        k = {"ms": ms, "per_key_frame": K}
+        if name == "upsample_ce":
+            class_pixels = float(C) * P * S
+            k.update(bound="alu", achieved=ALU_FLOP_PER_CLASS_PIXEL * class_pixels / ms / 1e9, peak=arith["fma_tflops"],
+                     unit="TFLOP/s", hbm_gbs=S * (2 * C * p * 4 + P) / ms / 1e6,
+                     xu={"achieved": EX2_PER_CLASS_PIXEL * class_pixels / ms / 1e9, "peak": arith["ex2_tops"],
+                         "unit": "1e12 exp2/s", "frac": EX2_PER_CLASS_PIXEL * class_pixels / ms / 1e9 / arith["ex2_tops"]})
+        elif name == "tc_fwd1x1":
+            k.update(bound="hbm", achieved=S * (p * c_last * 2 + C * p * 4) / ms / 1e6, peak=hbm, unit="GB/s",
+                     tflops=2.0 * S * p * C * c_last / ms / 1e9)
+        elif name == "tc_wgrad1x1":
+            k.update(bound="hbm", achieved=S * (p * c_last * 2 + C * p * 2) / ms / 1e6, peak=hbm, unit="GB/s",
+                     tflops=2.0 * S * p * C * c_last / ms / 1e9)
+        elif name in ("tc_fwd3x3", "tc_wgrad3x3"):
+            k.update(bound="tensor", achieved=2.0 * S * p * cfg.c_hidden * cfg.c_in * 9 / ms / 1e9, peak=tensor_peak,
+                     unit="TFLOP/s")
+        elif name == "tc_dgrad":
+            k.update(bound="hbm", achieved=S * (2 * p * cfg.c_hidden * 2 + C * p * 4) / ms / 1e6, peak=hbm, unit="GB/s")
+        else:
+            k.update(bound="latency")
+        kernels[name] = k
+    for k in kernels.values():
+        if "achieved" in k and k.get("peak"):
+            k["frac"] = k["achieved"] / k["peak"]
+    return kernels
+
+
+def make_context(st, stream, cfg, theta0, **kw):
+    args = dict(n_streams=cfg.n_streams, c_in=cfg.c_in, c_hidden=cfg.c_hidden, n_classes=cfg.n_classes, feat_h=cfg.feat_h,
+                feat_w=cfg.feat_w, gemm_precision=cfg.gemm_precision, lr=cfg.lr, momentum=cfg.momentum,
+                cuda_stream=stream.cuda_stream, init_params=theta0)
+    args.update(kw)
+    return st.st_init_head(**args)
+
+
+def run_other_workload(st, torch, stream, idx, feats_d, logits_d, peaks, arith, local_rank):
+    """A few key frames of another workload of the same frame size (the two-layer head, the 16-stream 1x1 head) on the
+    input sets already on the device (stream s takes set s mod N_SETS); no CPU baseline."""
+    cfg = si.get_config(idx)
+    S, C, K = cfg.n_streams, cfg.n_classes, cfg.k_steps
+    theta0 = np.concatenate([si.initial_head_params(cfg.c_in, cfg.c_hidden, C, 1000 + s) for s in range(S)])
+    ctx = make_context(st, stream, cfg, theta0)
+    packed = torch.empty((S, ctx.n_params), dtype=torch.float32, device="cuda")
+    conf = torch.zeros((S, C, C), dtype=torch.int64, device="cuda")
+    miou = torch.zeros(S, dtype=torch.float64, device="cuda")
+    loss = torch.zeros((S, K), dtype=torch.float32, device="cuda")
+
+    def key_frame(i):
+        for s in range(S):
+            st.st_set_frozen_features(ctx, s, feats_d[(i + s) % N_SETS][0])
+            st.st_teacher_labels(ctx, s, logits_d[(i + s) % N_SETS][0])
+        st.st_distill_step(ctx, K, loss)
+        for s in range(S):
+            st.st_pack_updated_params(ctx, s, packed[s])
+            st.st_agreement(ctx, s, None, None, conf[s], miou_out=miou[s:s + 1])
+
+    def sync():
+        torch.cuda.synchronize()
+
+    for i in range(3):
+        key_frame(i)
+    steps = 10 if S == 1 else 4
+    clocks = ClockSampler(local_rank)
+    clocks.begin()
+    ms = timed_blocks(torch, stream, sync, 5, steps, key_frame)
+    ms_loop = timed_blocks(torch, stream, sync, 5, steps, lambda i: st.st_distill_step(ctx, K, loss))
+    clocks.end()
+    kernels = kernel_table(st, ctx, cfg, peaks, arith, 5)
+    st.st_destroy(ctx)
+    med = statistics.median(ms) / steps
+    return {"workload": cfg.name, "steps_per_s": K * S / (med / 1e3), "ms_per_key_frame": med,
+            "ms_per_key_frame_min": min(ms) / steps,
+            "distill_loop_only": {"steps_per_s": K * S / (statistics.median(ms_loop) / steps / 1e3),
+                                  "ms_per_step": statistics.median(ms_loop) / steps / K},
+            "streams": S, "c_hidden": cfg.c_hidden, "kernels": kernels, "clocks": clocks.finish(),
+            "inputs": f"the {N_SETS} input sets of the main run, stream s on set (key frame + s) mod {N_SETS}"}
+
+
+def run_confident_student(st, torch, stream, cfg, peaks, arith):
+    """The main workload with a student that has learnt its frame: features that carry the class map, trained until the
+    mean IoU passes the paper's THRESHOLD of 0.8 (Section 5.3).  Its logits are steep at class boundaries, which is the
+    expensive case of the fused upsample + cross-entropy kernel."""
+    C, K = cfg.n_classes, cfg.k_steps
+    cls = si.voronoi_map(cfg.frame_h, cfg.frame_w, cfg.n_regions, C, 2000)
+    feat = si.label_informed_features(cfg.c_in, cfg.feat_h, cfg.feat_w, cls, cfg.up, 0, strength=3.0)
+    theta0 = si.initial_head_params(cfg.c_in, cfg.c_hidden, C, 1000)
+    ctx = make_context(st, stream, cfg, theta0, lr=0.5)
+    st.st_set_frozen_features(ctx, 0, torch.from_numpy(feat).cuda())
+    st.st_set_labels(ctx, 0, torch.from_numpy(cls).cuda())
+    miou, n_steps = 0.0, 0
+    while miou <= 0.8 and n_steps < 200:
+        st.st_distill_step(ctx, K)
+        n_steps += K
+        miou = st.st_agreement(ctx, 0, None, None, None)
+    loss = torch.zeros((1, K), dtype=torch.float32, device="cuda")
+    ms = timed_blocks(torch, stream, torch.cuda.synchronize, 5, 20, lambda i: st.st_distill_step(ctx, K, loss))
+    kernels = kernel_table(st, ctx, cfg, peaks, arith, 10)
+    out = {"miou_when_timed": miou, "steps_to_get_there": n_steps, "ms_per_step": statistics.median(ms) / 20 / K,
+           "upsample_ce_ms": kernels["upsample_ce"]["ms"], "upsample_ce_frac": kernels["upsample_ce"].get("frac"),
+           "miou_after": st.st_agreement(ctx, 0, None, None, None)}
+    st.st_destroy(ctx)
+    return out
+
+
 def run_ours(args, cfg):
     import torch
     import paper_2003_10735_b200 as st
@@ -217,6 +353,9 @@ def run_ours(args, cfg):
     H, W, p, P = cfg.frame_h, cfg.frame_w, cfg.feat_h * cfg.feat_w, cfg.frame_h * cfg.frame_w
 
     with torch.cuda.stream(stream):
+        # ---- this device's plain-arithmetic ceilings (fp32 multiply-add, exp2), measured, a few milliseconds
+        fma_tflops, ex2_tops = st.st_measure_arithmetic_peaks(stream.cuda_stream)
+        arith = {"fma_tflops": fma_tflops, "ex2_tops": ex2_tops}
         # ---- seeded synthetic inputs (each rank its own streams: the path shards by stream, no exchange)
         feats_h, logits_h, thetas = [], [], []
         for i in range(N_SETS):
@@ -231,11 +370,10 @@ def run_ours(args, cfg):
         for s in range(S):
             thetas.append(si.initial_head_params(cfg.c_in, cfg.c_hidden, C, 1000 + s))
         theta0 = np.concatenate(thetas)
+        theta0_d = torch.from_numpy(theta0).cuda().reshape(S, -1)
         feats_d = [[f.cuda(non_blocking=True) for f in fs] for fs in feats_h]
         logits_d = [[t.cuda(non_blocking=True) for t in ts] for ts in logits_h]
-        ctx = st.st_init_head(n_streams=S, c_in=cfg.c_in, c_hidden=cfg.c_hidden, n_classes=C, feat_h=cfg.feat_h,
-                              feat_w=cfg.feat_w, gemm_precision=cfg.gemm_precision, lr=cfg.lr, momentum=cfg.momentum,
-                              cuda_stream=stream.cuda_stream, init_params=theta0)
+        ctx = make_context(st, stream, cfg, theta0)
         n_params = ctx.n_params
         packed_d = torch.empty((S, n_params), dtype=torch.float32, device="cuda")
         packed_h = torch.empty((S, n_params), dtype=torch.float32).pin_memory()
@@ -262,56 +400,54 @@ def run_ours(args, cfg):
                 dist.barrier()
             torch.cuda.synchronize()
 
+        def reset_parameters():             # outside every timed region: each block starts from the initial student
+            for s in range(S):
+                st.st_apply_update(ctx, s, theta0_d[s])
+
+        # A timed block is exactly --steps key frames.  Short blocks are repeated so that about two thousand key frames
+        # are timed in all; the reported value is the median block (the minimum is given beside it).
+        n_blocks = args.blocks if args.blocks > 0 else max(1, min(101, -(-2000 // args.steps)))
+        if n_blocks > 1 and n_blocks % 2 == 0:
+            n_blocks += 1
+
         # ---- device-resident run
         for i in range(args.warmup):
             key_frame(i, feats_d, logits_d, packed_d)
         clocks = ClockSampler(local_rank) if rank == 0 else None
         barrier()
         launches0 = st.st_launch_count(ctx)
-        ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
         if clocks:
             clocks.begin()
-        ev0.record(stream)
-        for i in range(args.steps):
-            key_frame(i, feats_d, logits_d, packed_d)
-        ev1.record(stream)
-        barrier()
+        block_ms = timed_blocks(torch, stream, barrier, n_blocks, args.steps,
+                                lambda i: key_frame(i, feats_d, logits_d, packed_d), between=reset_parameters)
         if clocks:
             clocks.end()
-        ms_total = ev0.elapsed_time(ev1)
+        launches = (st.st_launch_count(ctx) - launches0 - n_blocks * S * (2 if cfg.gemm_precision == 1 else 1)) // n_blocks
         last_miou_dev = float(miou_d[0].item())
-        launches = st.st_launch_count(ctx) - launches0
-        ms_total = max_over_ranks(ms_total, dist, "cuda")
+        block_ms = [max_over_ranks(m, dist, "cuda") for m in block_ms]
+        ms_total = statistics.median(block_ms)
         clock_info = clocks.finish() if clocks else None
 
         # ---- the K-step loop alone (inputs already cached), for the per-step view
-        barrier()
-        n_loop = max(10, min(args.steps, 500))
-        ev0.record(stream)
-        for i in range(n_loop):
-            st.st_distill_step(ctx, K, loss_d)
-        ev1.record(stream)
-        torch.cuda.synchronize()
-        ms_loop = ev0.elapsed_time(ev1) / n_loop
+        n_loop = max(10, min(args.steps, 200))
+        ms_loop = statistics.median(timed_blocks(torch, stream, barrier, 5, n_loop, lambda i: st.st_distill_step(ctx, K, loss_d),
+                                                 between=reset_parameters)) / n_loop
 
         # ---- end to end through the C ABI with host buffers (pinned): H2D of the inputs, D2H of the results
         e2e_steps = max(3, min(args.steps, 100))
         for i in range(min(args.warmup, 3)):
             key_frame(i, feats_h, logits_h, packed_h, results_on_device=False)
-        barrier()
-        ev0.record(stream)
-        for i in range(e2e_steps):
-            key_frame(i, feats_h, logits_h, packed_h, results_on_device=False)
-        ev1.record(stream)
-        barrier()
-        ms_e2e = ev0.elapsed_time(ev1)
-        ms_e2e = max_over_ranks(ms_e2e, dist, "cuda")
+        e2e_ms = timed_blocks(torch, stream, barrier, 3, e2e_steps,
+                              lambda i: key_frame(i, feats_h, logits_h, packed_h, results_on_device=False), between=reset_parameters)
+        ms_e2e = statistics.median([max_over_ranks(m, dist, "cuda") for m in e2e_ms])
         h2d = S * (cfg.c_in * p * 4 + C * P * 4)
         d2h = S * (n_params * 4 + 8)
 
         # ---- per-kernel times with CUDA events on the launching stream
-        kernels, train = {}, {}
+        kernels, train, others, confident = {}, {}, {}, None
         if rank == 0:
+            ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+
             def timed(fn, reps=20):
                 ev0.record(stream)
                 for r in range(reps):
@@ -321,44 +457,31 @@ def run_ours(args, cfg):
                 return ev0.elapsed_time(ev1) / reps
             t_arg = timed(lambda r: st.st_teacher_labels(ctx, 0, logits_d[r % N_SETS][0]))
             t_feat = timed(lambda r: st.st_set_frozen_features(ctx, 0, feats_d[r % N_SETS][0]))
-            masks = [torch.randint(0, C, (H, W), dtype=torch.uint8, device="cuda") for _ in range(2)]
-            t_agree = timed(lambda r: st.st_agreement(ctx, 0, masks[0], masks[1], conf_d[0]))
             hbm = peaks["hbm_gbs"]
             kernels["argmax_u8"] = {"ms": t_arg, "bound": "hbm", "achieved": (C * P * 4 + P) / t_arg / 1e6,
                                     "peak": hbm, "unit": "GB/s", "per_key_frame": S}
             if cfg.gemm_precision == 1:
                 kernels["feat_to_bf16_nhwc"] = {"ms": t_feat, "bound": "hbm", "achieved": cfg.c_in * p * 6 / t_feat / 1e6,
                                                 "peak": hbm, "unit": "GB/s", "per_key_frame": S}
-            kernels["agreement(confusion+miou+sync)"] = {"ms": t_agree, "bound": "latency", "achieved": 2 * P / t_agree / 1e6,
-                                                         "peak": hbm, "unit": "GB/s", "per_key_frame": S}
-            c_last = cfg.c_hidden or cfg.c_in
-            alu_peak = 148 * 128 * 2 * peaks["sm_max_mhz"] * 1e6 / 1e12          # fp32 FMA lanes x 2 flop x clock
-            tensor_peak = peaks["bf16_tflops"]
-            for name, ms in st.st_profile_step(ctx, 20):
-                k = {"ms": ms, "per_key_frame": K}
-                if name == "upsample_ce":
-                    k.update(bound="alu", achieved=ALU_FLOP_PER_CLASS_PIXEL * C * P * S / ms / 1e9, peak=alu_peak, unit="TFLOP/s",
-                             hbm_gbs=S * (2 * C * p * 4 + P) / ms / 1e6)
-                elif name == "tc_fwd1x1":
-                    k.update(bound="hbm", achieved=S * (p * c_last * 2 + C * p * 4) / ms / 1e6, peak=hbm, unit="GB/s",
-                             tflops=2.0 * S * p * C * c_last / ms / 1e9)
-                elif name == "tc_wgrad1x1":
-                    k.update(bound="hbm", achieved=S * (p * c_last * 2 + C * p * 2) / ms / 1e6, peak=hbm, unit="GB/s",
-                             tflops=2.0 * S * p * C * c_last / ms / 1e9)
-                elif name in ("tc_fwd3x3", "tc_wgrad3x3"):
-                    k.update(bound="tensor", achieved=2.0 * S * p * cfg.c_hidden * cfg.c_in * 9 / ms / 1e9, peak=tensor_peak,
-                             unit="TFLOP/s")
-                elif name == "tc_dgrad":
-                    k.update(bound="hbm", achieved=S * (2 * p * cfg.c_hidden * 2 + C * p * 4) / ms / 1e6, peak=hbm, unit="GB/s")
-                else:
-                    k.update(bound="latency")
-                kernels[name] = k
-            for k in kernels.values():
-                if "achieved" in k and k.get("peak"):
-                    k["frac"] = k["achieved"] / k["peak"]
+            # agreement of two given masks: the kernel alone (results delivered into device buffers: one launch, no copy,
+            # no wait; launched back to back) and the whole call with the mean IoU read back by the host
+            rng = np.random.default_rng(0)
+            lab_map = si.voronoi_map(H, W, cfg.n_regions, C, 2000)
+            noisy = np.where(rng.random((H, W)) < 0.9, lab_map, rng.integers(0, C, (H, W))).astype(np.uint8)
+            m_coh = [torch.from_numpy(lab_map).cuda(), torch.from_numpy(noisy).cuda()]
+            m_rnd = [torch.randint(0, C, (H, W), dtype=torch.uint8, device="cuda") for _ in range(2)]
+            agree = {}
+            for name, (a, b) in (("coherent_masks", m_coh), ("random_masks", m_rnd)):
+                t_k = timed(lambda r: st.st_agreement(ctx, 0, a, b, conf_d[0], miou_out=miou_d[0:1]), reps=50)
+                t_c = timed(lambda r: st.st_agreement(ctx, 0, a, b, conf_d[0]), reps=20)
+                agree[name] = {"kernel_us": t_k * 1e3, "call_us": t_c * 1e3, "kernel_gbs": 2 * P / t_k / 1e6,
+                               "kernel_frac_of_hbm": 2 * P / t_k / 1e6 / hbm}
+            t_own = timed(lambda r: st.st_agreement(ctx, 0, None, None, conf_d[0], miou_out=miou_d[0:1]), reps=50)
+            agree["student_mask_fused"] = {"kernel_us": t_own * 1e3, "note": "arg-max of the upsampled logits + confusion + mean IoU, forward reused"}
+            kernels["agreement"] = {"ms": agree["coherent_masks"]["kernel_us"] / 1e3, "bound": "latency", "per_key_frame": S, **agree}
+            kernels.update(kernel_table(st, ctx, cfg, peaks, arith, 20))
             # Train of Algorithm 1 (forward, metric, break test and best-student snapshot per update, all on the device):
             # the full loop (a threshold no mean IoU reaches) and a loop that ends on the first metric
-            train = {}
             for name, thr in (("full_loop", 2.0), ("ends_at_once", 0.0)):
                 for _ in range(3):
                     st.st_train_key_frame(ctx, thr, K)
@@ -369,16 +492,18 @@ def run_ours(args, cfg):
         if rank == 0:
             ms_step = ms_total / args.steps
             value = whole_job_rate(K * S * args.steps, world, ms_total)      # SGD iterations of all streams of all ranks
-            dominant = max((n for n in kernels if "frac" in kernels[n] or True),
-                           key=lambda n: kernels[n]["ms"] * kernels[n]["per_key_frame"])
+            dominant = max(kernels, key=lambda n: kernels[n]["ms"] * kernels[n]["per_key_frame"])
             dk = kernels[dominant]
             # DRAM bytes per launch from the ncu capture summarised in profiles/ (same kernel, same workload)
             traffic = NCU_DRAM_BYTES.get((args.workload, dominant))
             roofline = {"kernel": dominant, "bound": dk.get("bound"), "achieved": dk.get("achieved"), "peak": dk.get("peak"),
                         "unit": dk.get("unit"), "frac": dk.get("frac"), "traffic": traffic,
                         "peak_source": f"of {peaks['source']}" if dk.get("bound") in ("hbm", "tensor") else
-                                       "148 SMs x 128 fp32 lanes x 2 flop x max SM clock",
+                                       "fp32 multiply-add rate measured on this device by st_measure_arithmetic_peaks",
                         "ms_per_launch": dk["ms"]}
+            if dk.get("bound") == "alu":
+                roofline.update(algorithmic_flop_per_class_pixel=ALU_FLOP_PER_CLASS_PIXEL, xu=dk.get("xu"),
+                                derived_fma_peak_tflops=148 * 128 * 2 * peaks["sm_max_mhz"] * 1e6 / 1e12)
             result = {
                 "metric": METRIC, "value": value, "unit": "steps/s", "n_gpus": world, "steps": args.steps,
                 "warmup": args.warmup, "ms_per_step": ms_step, "higher_is_better": True, "scaling": "weak",
@@ -387,18 +512,28 @@ def run_ours(args, cfg):
                            "classes": C, "streams_per_gpu": S, "c_hidden": cfg.c_hidden,
                            "step": "features cache + labels + K SGD iterations + pack + agreement per key frame",
                            "l2": f"inputs rotate over {N_SETS} key frames ({N_SETS * S * (cfg.c_in * p + C * P) * 4 / 1e6:.0f} MB) > 126 MB L2",
-                           "parallelism": f"replicas x{world}, no collective"},
+                           "parallelism": f"replicas x{world}, no collective",
+                           "timed_blocks": f"{n_blocks} blocks of {args.steps} key frames, parameters reset before each; value = median block"},
+                "timed_blocks": {"n": n_blocks, "ms_median": ms_total, "ms_min": min(block_ms), "ms_max": max(block_ms),
+                                 "value_of_fastest_block": whole_job_rate(K * S * args.steps, world, min(block_ms))},
                 "clocks": clock_info,
                 "e2e": {"value": world * K * S * e2e_steps / (ms_e2e / 1e3), "unit": "steps/s", "h2d_bytes_per_step": h2d,
                         "d2h_bytes_per_step": d2h, "ms_per_step": ms_e2e / e2e_steps},
                 "gpu_launches": int(launches),
                 "roofline": roofline,
+                "arithmetic_peaks": arith,
                 "key_frames_per_s": world * args.steps / (ms_total / 1e3),
                 "distill_loop_only": {"steps_per_s": K * S / (ms_loop / 1e3), "ms_per_k_steps": ms_loop},
                 "kernels": kernels, "train_key_frame": train,
                 "last_loss": float(loss_d[0, -1].item()), "last_miou": mious[0], "last_miou_device_run": last_miou_dev,
             }
         st.st_destroy(ctx)
+
+        # ---- beside the headline: the same workload with a trained student, and the other workloads of this frame size
+        if rank == 0 and world == 1 and not args.headline_only and args.workload == 2:
+            result["confident_student"] = run_confident_student(st, torch, stream, cfg, peaks, arith)
+            result["other_workloads"] = {str(idx): run_other_workload(st, torch, stream, idx, feats_d, logits_d, peaks, arith, local_rank)
+                                         for idx in (3, 5)}
 
     if rank == 0:
         if world == 1 and not args.no_cpu_baseline:
@@ -429,6 +564,8 @@ def main():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--workload", type=int, default=2, help="index into the synthetic workload table (2 = 720p, 1x1 head, K=8)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--blocks", type=int, default=0, help="timed blocks of --steps key frames (0: enough for about 2000 key frames)")
+    ap.add_argument("--headline-only", action="store_true", help="skip the trained-student and other-workload runs")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
     cfg = si.get_config(args.workload)

@@ -255,6 +255,18 @@ ST_API st_status st_profile_step(st_ctx *ctx, int32_t n_steps, int32_t *n_stages
                                  const char **names_out);
 
 /*
+ * st_measure_arithmetic_peaks — what this device sustains in plain fp32 multiply-adds and in exp2 evaluations
+ * (special-function unit), measured with two register-only kernels of a few hundred microseconds each.  These
+ * are the ceilings of the fused upsample + cross-entropy kernel (ComputeLoss and the start of PartialBackward
+ * of Algorithm 1), which is bound by arithmetic, not by memory.  A measuring aid, not part of the method.
+ *   cuda_stream  cudaStream_t on which the kernels run (NULL = default stream).
+ *   fma_tflops   host, may be NULL; 10^12 fp32 operations per second, a multiply-add counted as two.
+ *   ex2_tops     host, may be NULL; 10^12 exp2 evaluations per second.
+ * Allocates four bytes of device memory for the duration of the call and waits for the stream.
+ */
+ST_API st_status st_measure_arithmetic_peaks(void *cuda_stream, double *fma_tflops, double *ex2_tops);
+
+/*
  * st_agreement_noalloc — confusion matrix and mean IoU of two masks without any allocation.
  * (The paper has no counterpart: this entry point exists for the sake of callers, not of the method.)
  *

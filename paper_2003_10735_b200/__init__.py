@@ -38,7 +38,7 @@ EXPORTED = [
     "st_distill_step", "st_pack_updated_params", "st_student_mask", "st_agreement", "st_read_tensor",
     "st_launch_count", "st_destroy", "st_last_error", "st_status_name", "st_profile_step",
     "st_agreement_noalloc", "st_train_key_frame", "st_next_stride", "st_client_schedule", "st_throughput_bounds",
-    "st_traffic_bounds", "st_choose_max_updates", "st_apply_update",
+    "st_traffic_bounds", "st_choose_max_updates", "st_apply_update", "st_measure_arithmetic_peaks",
 ]
 ST_NOALLOC_MAX_CLASSES = 64
 ST_MAX_STAGES = 12
@@ -116,6 +116,8 @@ def load_library() -> ctypes.CDLL:
                                     ctypes.POINTER(ctypes.c_char_p)]
     lib.st_agreement_noalloc.restype = ctypes.c_int
     lib.st_agreement_noalloc.argtypes = [vp, vp, i64, i32, vp, vp, vp]
+    lib.st_measure_arithmetic_peaks.restype = ctypes.c_int
+    lib.st_measure_arithmetic_peaks.argtypes = [vp, ctypes.POINTER(dbl), ctypes.POINTER(dbl)]
     lib.st_launch_count.restype = i64
     lib.st_launch_count.argtypes = [vp]
     lib.st_destroy.restype = None
@@ -312,6 +314,14 @@ def st_agreement_noalloc(pred, label, n_classes: int, cuda_stream: int, conf_out
         _ptr(conf_out, "int64", max(n_classes, 0) ** 2, "conf_out"), miou_out.data_ptr())
     if status != ST_OK:
         raise StError(status, load_library().st_status_name(status).decode(), "st_agreement_noalloc")
+
+
+def st_measure_arithmetic_peaks(cuda_stream: int = 0):
+    """(fp32 multiply-add rate in TFLOP/s, exp2 rate in 10^12 per second) measured on the current device."""
+    fma, ex2 = ctypes.c_double(0), ctypes.c_double(0)
+    _status_only(load_library().st_measure_arithmetic_peaks(cuda_stream or None, ctypes.byref(fma), ctypes.byref(ex2)),
+                 "st_measure_arithmetic_peaks")
+    return fma.value, ex2.value
 
 
 class st_latencies(ctypes.Structure):

@@ -9,6 +9,7 @@
 // key per warp instead of 32 conflicting ones.  Blocks then add their counters to the
 // 64-bit global matrix.  Pixels with a label or prediction >= C are skipped and counted.
 #include "st_internal.h"
+#include "miou.cuh"
 
 namespace st {
 
@@ -30,7 +31,7 @@ __device__ __forceinline__ void warp_count(CounterT* hist, int key, bool valid)
 template <int MODE>
 __global__ void __launch_bounds__(kConfThreads)
 confusion_kernel(const uint8_t* __restrict__ label, const uint8_t* __restrict__ pred, int64_t P, int C,
-                 unsigned long long* __restrict__ conf, unsigned int* __restrict__ bad)
+                 unsigned long long* __restrict__ conf, unsigned int* __restrict__ bad, ConfusionFinish fin)
 {
     extern __shared__ unsigned int hist_all[];
     const int CC = C * C;
@@ -86,21 +87,45 @@ confusion_kernel(const uint8_t* __restrict__ label, const uint8_t* __restrict__ 
         if (sum) atomicAdd(&conf[i], sum);
     }
     if (n_bad) atomicAdd(bad, n_bad);
+    if (!fin.ticket) return;
+
+    // ---- the last block to finish delivers the matrix and its mean IoU and leaves the counters at zero for the next launch
+    __shared__ bool is_last;
+    __shared__ double iou[kConfThreads];
+    __shared__ int present[kConfThreads];
+    __threadfence();
+    __syncthreads();
+    if (threadIdx.x == 0) is_last = atomicAdd(fin.ticket, 1u) == gridDim.x - 1;
+    __syncthreads();
+    if (!is_last) return;
+    __threadfence();
+    const double m = block_miou(conf, C, iou, present);
+    for (int i = threadIdx.x; i < CC; i += kConfThreads) {
+        fin.result[i] = __ldcg(conf + i);
+        conf[i] = 0;
+    }
+    if (threadIdx.x == 0) { *fin.miou = m; *fin.ticket = 0; }
 }
 
 void launch_confusion(const uint8_t* label, const uint8_t* pred, int64_t P, int C,
-                      unsigned long long* conf, unsigned int* bad, cudaStream_t s)
+                      unsigned long long* conf, unsigned int* bad, cudaStream_t s, const ConfusionFinish* finish)
 {
-    if (P <= 0) return;
+    ConfusionFinish fin = {nullptr, nullptr, nullptr};
+    if (finish) fin = *finish;
+    if (P <= 0 && !fin.ticket) return;
+    if (P < 0) P = 0;
     const size_t one = (size_t)C * C * sizeof(unsigned int);
     int64_t work = (P / 16 + kConfThreads - 1) / kConfThreads;
     int blocks = (int)(work < 1 ? 1 : (work > 148 * 4 ? 148 * 4 : work));
-    if (one * kConfWarps <= 48 * 1024)
-        confusion_kernel<0><<<blocks, kConfThreads, one * kConfWarps, s>>>(label, pred, P, C, conf, bad);
-    else if (one <= 48 * 1024)
-        confusion_kernel<1><<<blocks, kConfThreads, one, s>>>(label, pred, P, C, conf, bad);
+    // dynamic shared memory stays below 36 KB: the kernel's static arrays (mean IoU of the last block) take 11 KB of
+    // the 48 KB a block gets without opting in
+    constexpr size_t kDynLimit = 36 * 1024;
+    if (one * kConfWarps <= kDynLimit)
+        confusion_kernel<0><<<blocks, kConfThreads, one * kConfWarps, s>>>(label, pred, P, C, conf, bad, fin);
+    else if (one <= kDynLimit)
+        confusion_kernel<1><<<blocks, kConfThreads, one, s>>>(label, pred, P, C, conf, bad, fin);
     else
-        confusion_kernel<2><<<blocks, kConfThreads, 0, s>>>(label, pred, P, C, conf, bad);
+        confusion_kernel<2><<<blocks, kConfThreads, 0, s>>>(label, pred, P, C, conf, bad, fin);
 }
 
 }  // namespace st

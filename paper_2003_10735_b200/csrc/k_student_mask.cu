@@ -177,6 +177,12 @@ student_mask_kernel(StudentMaskArgs a, int chunk)
         iou[c] = v; present[c] = pr;
     }
     __syncthreads();
+    if (a.conf_out) {                                             // deliver the matrix, leave the counters at zero
+        for (int e = tid; e < C * C; e += SM_THREADS) {
+            a.conf_out[e] = staged ? cm[e] : __ldcg(&a.conf[e]);
+            a.conf[e] = 0;
+        }
+    }
     if (tid == 0) {
         double sum = 0.0; int cnt = 0;
         for (int k = 0; k < C; ++k) { sum += iou[k]; cnt += present[k]; }

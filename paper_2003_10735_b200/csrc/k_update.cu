@@ -6,6 +6,7 @@
 // per-block partial sums of the bias gradients, and the per-block loss partials.
 // K7 — UpdatedPart(student) (Algorithm 3): the packed fp32 buffer of all trainable tensors.
 #include "st_internal.h"
+#include "miou.cuh"
 
 #include <cstdlib>
 
@@ -301,42 +302,6 @@ __global__ void refresh_shadow_kernel(UpdateArgs a)
 void launch_refresh_shadow(const UpdateArgs& a, cudaStream_t s)
 {
     refresh_shadow_kernel<<<dim3((unsigned)((a.n_params + 255) / 256), (unsigned)a.S), 256, 0, s>>>(a);
-}
-
-// Mean IoU (Section 3.2): IoU_c = conf[c][c] / (row_c + col_c - conf[c][c]), averaged over the
-// classes present in the label (row_c > 0).  Integer counts, double arithmetic, fixed order.
-// Called by all 256 threads of a block; the value is returned to thread 0 only.  Matrices of up to kMiouStage classes
-// are first copied to shared memory in one coalesced pass (one memory latency instead of one per row element).
-constexpr int kMiouStage = 32;
-__device__ __forceinline__ double block_miou(const unsigned long long* __restrict__ conf_g, int C, double* iou, int* present)
-{
-    __shared__ unsigned long long staged[kMiouStage * kMiouStage];
-    const unsigned long long* conf = conf_g;
-    if (C <= kMiouStage) {                                 // block-uniform
-        for (int e = threadIdx.x; e < C * C; e += blockDim.x) staged[e] = conf_g[e];
-        __syncthreads();
-        conf = staged;
-    }
-    const int c = threadIdx.x;
-    double v = 0.0; int pr = 0;
-    if (c < C) {
-        unsigned long long row = 0, col = 0;
-        for (int q = 0; q < C; ++q) { row += conf[c * C + q]; col += conf[q * C + c]; }
-        if (row > 0) {
-            const unsigned long long inter = conf[c * C + c];
-            v = (double)inter / (double)(row + col - inter);
-            pr = 1;
-        }
-    }
-    iou[c] = v; present[c] = pr;
-    __syncthreads();
-    double m = 0.0;
-    if (c == 0) {
-        double sum = 0.0; int n = 0;
-        for (int k = 0; k < C; ++k) { sum += iou[k]; n += present[k]; }
-        m = n ? sum / n : 0.0;
-    }
-    return m;
 }
 
 __global__ void __launch_bounds__(256) miou_kernel(const unsigned long long* __restrict__ conf, int C, double* out)

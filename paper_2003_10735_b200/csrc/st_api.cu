@@ -474,7 +474,7 @@ st_status st_init_head(const st_head_desc* desc, const float* init_params, st_ct
     ALLOC(z, S * c->C * c->p); ALLOC(dz, S * c->C * c->p);
     ALLOC(loss_part, S * c->n_k3_blocks); ALLOC(db_part, (size_t)S * c->n_k3_blocks * c->C);
     ALLOC(loss_buf, S * kMaxSteps);
-    ALLOC(miou_tmp, 4); ALLOC(mask_tmp, c->P); ALLOC(mask_tmp2, c->P); ALLOC(conf_tmp, c->C * c->C + 1);   // + the block counter of the fused agreement kernel
+    ALLOC(miou_tmp, 4); ALLOC(mask_tmp, c->P); ALLOC(mask_tmp2, c->P); ALLOC(conf_tmp, 2 * c->C * c->C + 1);   // counters (zero between calls), the block counter, the delivered matrix
     if (e == cudaSuccess) { c->bad = reinterpret_cast<unsigned int*>(c->miou_tmp + 1); e = cudaHostAlloc((void**)&c->status_host, 32, cudaHostAllocDefault); }
     if (c->bf16_mode) {
         ALLOC(x_bf16, S * c->p * c->Cin);
@@ -920,15 +920,21 @@ st_status st_agreement(st_ctx* ctx, int32_t stream, const uint8_t* pred, const u
         if (!ctx->has_labels[stream]) return fail(ctx, ST_ERR_BAD_STATE, "st_agreement: stream %d has no labels yet", stream);
         d_label = ctx->labels + (int64_t)stream * ctx->P;
     }
-    const size_t cbytes = (size_t)ctx->C * ctx->C * sizeof(unsigned long long);
+    const size_t cc = (size_t)ctx->C * ctx->C, cbytes = cc * sizeof(unsigned long long);
+    // Where the kernel delivers the finished matrix and the mean IoU: straight into the caller's device buffers where
+    // it gave some (the call is then one kernel and nothing else), else into the context's, to be copied out below.
+    const bool conf_direct = conf && is_device_ptr(conf) && ((uintptr_t)conf & 7u) == 0;
+    const bool miou_direct = miou && is_device_ptr(miou) && ((uintptr_t)miou & 7u) == 0;
+    unsigned long long* conf_res = conf_direct ? reinterpret_cast<unsigned long long*>(conf) : ctx->conf_tmp + cc + 1;
+    double* miou_res = miou_direct ? miou : ctx->miou_tmp;
     if (!pred && student_mask_fused_supported(ctx->C)) {
         // the student's own mask: arg-max, confusion and mean IoU in one kernel, the mask itself is not stored
         st = student_forward(ctx, stream, "st_agreement");
         if (st != ST_OK) return st;
-        ST_CUDA(ctx, cudaMemsetAsync(ctx->conf_tmp, 0, cbytes, ctx->stream));
         StudentMaskArgs a = mask_args(ctx, stream, nullptr);
-        a.labels = d_label; a.conf = ctx->conf_tmp; a.bad = ctx->bad + 1; a.miou = ctx->miou_tmp;
-        a.ticket = reinterpret_cast<unsigned int*>(ctx->conf_tmp + (size_t)ctx->C * ctx->C);
+        a.labels = d_label; a.conf = ctx->conf_tmp; a.bad = ctx->bad + 1; a.miou = miou_res;
+        a.ticket = reinterpret_cast<unsigned int*>(ctx->conf_tmp + cc);
+        a.conf_out = conf_res;
         launch_student_mask(a, ctx->stream);
         ctx->launches += 1;
     } else {
@@ -943,17 +949,17 @@ st_status st_agreement(st_ctx* ctx, int32_t stream, const uint8_t* pred, const u
             if (st != ST_OK) return st;
             d_pred = ctx->mask_tmp;
         }
-        ST_CUDA(ctx, cudaMemsetAsync(ctx->conf_tmp, 0, cbytes, ctx->stream));
-        launch_confusion(d_label, d_pred, ctx->P, ctx->C, ctx->conf_tmp, ctx->bad + 1, ctx->stream);
-        launch_miou(ctx->conf_tmp, ctx->C, ctx->miou_tmp, ctx->stream);
-        ctx->launches += 2;
+        // one kernel: its last block turns the counts into the mean IoU, delivers the matrix and clears the counters
+        const ConfusionFinish fin = {conf_res, miou_res, reinterpret_cast<unsigned int*>(ctx->conf_tmp + cc)};
+        launch_confusion(d_label, d_pred, ctx->P, ctx->C, ctx->conf_tmp, ctx->bad + 1, ctx->stream, &fin);
+        ctx->launches += 1;
     }
     st = check_launch(ctx, "confusion");
     if (st != ST_OK) return st;
-    if (conf) ST_CUDA(ctx, cudaMemcpyAsync(conf, ctx->conf_tmp, cbytes, cudaMemcpyDefault, ctx->stream));
+    if (conf && !conf_direct) ST_CUDA(ctx, cudaMemcpyAsync(conf, conf_res, cbytes, cudaMemcpyDefault, ctx->stream));
     if (miou && is_device_ptr(miou)) {
         // device destination: nothing to wait for; bad labels surface at the next call that does wait
-        ST_CUDA(ctx, cudaMemcpyAsync(miou, ctx->miou_tmp, sizeof(double), cudaMemcpyDeviceToDevice, ctx->stream));
+        if (!miou_direct) ST_CUDA(ctx, cudaMemcpyAsync(miou, ctx->miou_tmp, sizeof(double), cudaMemcpyDeviceToDevice, ctx->stream));
         return ST_OK;
     }
     st = fetch_status(ctx);

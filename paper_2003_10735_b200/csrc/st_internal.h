@@ -65,8 +65,12 @@ void launch_argmax_u8(const float* logits, int C, int64_t P, uint8_t* labels, cu
 
 // ---- K6: confusion matrix of two uint8 masks ---------------------------------------------------
 // conf: int64 [C][C], accumulated into (caller zeroes it); bad: count of pixels with l or q >= C.
+// With `finish` the kernel completes the measurement by itself: its last block writes the matrix to `result` and the
+// mean IoU (Section 3.2) to `miou`, then clears `conf` and the ticket, so that the next launch needs no memset
+// (`conf` and `*ticket` must be zero before the first launch).
+struct ConfusionFinish { unsigned long long* result; double* miou; unsigned int* ticket; };
 void launch_confusion(const uint8_t* label, const uint8_t* pred, int64_t P, int C,
-                      unsigned long long* conf, unsigned int* bad, cudaStream_t s);
+                      unsigned long long* conf, unsigned int* bad, cudaStream_t s, const ConfusionFinish* finish = nullptr);
 
 // ---- K8: frozen features fp32 [Cin][p] -> bf16 [p][Cin] ---------------------------------------
 void launch_feat_to_bf16_nhwc(const float* feat_chw, int Cin, int64_t p, bf16* out, cudaStream_t s);
@@ -121,10 +125,11 @@ struct StudentMaskArgs {
     int C, h, w;
     uint8_t* mask;             // [H][W] or nullptr (confusion only)
     const uint8_t* labels;     // [H][W] or nullptr (mask only)
-    unsigned long long* conf;  // [C][C], zeroed by the caller
+    unsigned long long* conf;  // [C][C], zero on entry
     unsigned int* bad;         // count of labels >= C
     double* miou;              // nullptr: no mean IoU
     unsigned int* ticket;      // zero between launches (block counter for the mean IoU)
+    unsigned long long* conf_out;  // with `miou`: the last block writes the finished matrix here and clears `conf`
 };
 bool student_mask_fused_supported(int C);   // confusion counters fit shared memory
 cudaError_t prepare_student_mask(int C);    // once per device and class count, outside any stream capture
