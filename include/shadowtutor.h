@@ -120,6 +120,27 @@ ST_API st_status st_set_frozen_features(st_ctx *ctx, int32_t stream, const float
  */
 ST_API st_status st_teacher_labels(st_ctx *ctx, int32_t stream, const float *logits_chw, uint8_t *labels_out);
 
+/*
+ * st_prefetch_key_frame / st_use_prefetched_key_frame — bring the next key frame's inputs to the device while the
+ * current key frame is still being trained.  In the server loop (Algorithm 3) a key frame arrives from the client
+ * while the previous one may still be in Train; the copy of its inputs from host memory is by far the longest part
+ * of handling it (136 MB against 0.35 ms of kernels at 720p), so it runs on a CUDA stream of the library's own, beside
+ * the context's stream.
+ *   st_prefetch_key_frame   feat_chw, logits_chw: host (pinned memory makes the copy asynchronous) or device, shapes
+ *                           as in st_set_frozen_features / st_teacher_labels.  Returns at once; the buffers must stay
+ *                           alive and unchanged until st_use_prefetched_key_frame for this stream has returned and the
+ *                           context's stream has passed its work.  A second prefetch for the same stream before the
+ *                           first is used replaces it.  Device memory for one key frame's inputs is allocated per
+ *                           stream on first use (ST_ERR_OOM / ST_ERR_CUDA on failure).
+ *   st_use_prefetched_key_frame   makes the prefetched inputs the current key frame of `stream`: the context's stream
+ *                           waits for the copy (the host does not), then runs what st_set_frozen_features and
+ *                           st_teacher_labels run.  labels_out as in st_teacher_labels.  ST_ERR_BAD_STATE if nothing
+ *                           was prefetched for the stream.
+ * Everything else about the two inputs is as documented for the two plain calls.
+ */
+ST_API st_status st_prefetch_key_frame(st_ctx *ctx, int32_t stream, const float *feat_chw, const float *logits_chw);
+ST_API st_status st_use_prefetched_key_frame(st_ctx *ctx, int32_t stream, uint8_t *labels_out);
+
 /* Install an existing label map (uint8 [H][W], host or device) as the training target. */
 ST_API st_status st_set_labels(st_ctx *ctx, int32_t stream, const uint8_t *labels);
 

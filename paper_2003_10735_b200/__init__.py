@@ -39,6 +39,7 @@ EXPORTED = [
     "st_launch_count", "st_destroy", "st_last_error", "st_status_name", "st_profile_step",
     "st_agreement_noalloc", "st_train_key_frame", "st_next_stride", "st_client_schedule", "st_throughput_bounds",
     "st_traffic_bounds", "st_choose_max_updates", "st_apply_update", "st_measure_arithmetic_peaks",
+    "st_prefetch_key_frame", "st_use_prefetched_key_frame",
 ]
 ST_NOALLOC_MAX_CLASSES = 64
 ST_MAX_STAGES = 12
@@ -84,6 +85,10 @@ def load_library() -> ctypes.CDLL:
     lib.st_set_frozen_features.argtypes = [vp, i32, vp]
     lib.st_teacher_labels.restype = ctypes.c_int
     lib.st_teacher_labels.argtypes = [vp, i32, vp, vp]
+    lib.st_prefetch_key_frame.restype = ctypes.c_int
+    lib.st_prefetch_key_frame.argtypes = [vp, i32, vp, vp]
+    lib.st_use_prefetched_key_frame.restype = ctypes.c_int
+    lib.st_use_prefetched_key_frame.argtypes = [vp, i32, vp]
     lib.st_set_labels.restype = ctypes.c_int
     lib.st_set_labels.argtypes = [vp, i32, vp]
     lib.st_distill_step.restype = ctypes.c_int
@@ -208,6 +213,17 @@ def st_set_frozen_features(ctx: _Ctx, stream: int, feat_chw) -> None:
 def st_teacher_labels(ctx: _Ctx, stream: int, logits_chw, labels_out=None) -> None:
     _check(load_library().st_teacher_labels(ctx.handle, stream, _ptr(logits_chw, "float32", ctx.C * ctx.P, "logits_chw"),
                                             _ptr(labels_out, "uint8", ctx.P, "labels_out")), ctx)
+
+
+def st_prefetch_key_frame(ctx: _Ctx, stream: int, feat_chw, logits_chw) -> None:
+    """Start copying the next key frame's inputs to the device on the library's own copy stream."""
+    _check(load_library().st_prefetch_key_frame(ctx.handle, stream, _ptr(feat_chw, "float32", ctx.desc.c_in * ctx.p, "feat_chw"),
+                                                _ptr(logits_chw, "float32", ctx.C * ctx.P, "logits_chw")), ctx)
+
+
+def st_use_prefetched_key_frame(ctx: _Ctx, stream: int, labels_out=None) -> None:
+    """Make the prefetched inputs the current key frame of `stream` (feature cache + labels)."""
+    _check(load_library().st_use_prefetched_key_frame(ctx.handle, stream, _ptr(labels_out, "uint8", ctx.P, "labels_out")), ctx)
 
 
 def st_set_labels(ctx: _Ctx, stream: int, labels) -> None:

@@ -55,7 +55,6 @@ tc_fwd1x1_kernel(const __grid_constant__ CUtensorMap tmA,   // {K, p, S}  box {6
                  float* __restrict__ z, int C, int p, int kblocks, unsigned int* err, const int* __restrict__ skip, int64_t skip_stride,
                  int a_early)
 {
-    if (skip && skip[(int64_t)blockIdx.y * skip_stride]) return;   // this stream's training loop has ended (block-uniform)
     extern __shared__ uint8_t smem_raw[];
     uint8_t* smem = align_smem(smem_raw);
     const uint32_t a_base = smem_u32(smem);
@@ -85,7 +84,12 @@ tc_fwd1x1_kernel(const __grid_constant__ CUtensorMap tmA,   // {K, p, S}  box {6
         }
     }
     pdl_wait();                  // the weights (and, without a_early, the activations) come from the previous kernel
-    pdl_launch_dependents();
+    if (skip && skip[(int64_t)blockIdx.y * skip_stride]) {     // this stream's training loop has ended (block-uniform; the flag
+        tc_fence_before_sync();                                 // comes from an earlier kernel, so it is read after the wait)
+        __syncthreads();
+        if (warp == 0) tmem_dealloc(tmem, 32);
+        return;
+    }
     const uint32_t done_bar = smem_u32(&bars[kblocks]);
     bool ok = true;
 
@@ -115,6 +119,7 @@ tc_fwd1x1_kernel(const __grid_constant__ CUtensorMap tmA,   // {K, p, S}  box {6
     }
     __syncwarp();
     ok = mbar_wait(done_bar, 0, err, kWaitDone);
+    pdl_launch_dependents();     // only the epilogue is left
     tc_fence_after_sync();
     if (ok) {
         float v[32];
@@ -145,9 +150,8 @@ tc_wgrad1x1_kernel(const __grid_constant__ CUtensorMap tmA,   // {K, p, S}      
                    const __grid_constant__ CUtensorMap tmB,   // {p, 32, S}     box {64, 32, 1}
                    float* __restrict__ partials,              // [S][n_split][32][K]
                    int K, int n_chunks, int chunks_per_block, int m_split, int tmem_cols, unsigned int* err,
-                   const int* __restrict__ skip, int64_t skip_stride)
+                   const int* __restrict__ skip, int64_t skip_stride, int a_early)
 {
-    if (skip && skip[(int64_t)blockIdx.y * skip_stride]) return;   // this stream's training loop has ended (block-uniform)
     extern __shared__ uint8_t smem_raw[];
     uint8_t* smem = align_smem(smem_raw);
     // m_split blocks share a pixel range, each with its own 128-channel accumulators: with the channels divided the
@@ -176,8 +180,24 @@ tc_wgrad1x1_kernel(const __grid_constant__ CUtensorMap tmA,   // {K, p, S}      
     __syncthreads();
     tc_fence_after_sync();
     const uint32_t tmem = tmem_slot;
+    // a_early: the activations are the frozen features, which no kernel of the loop writes, and this kernel may have been
+    // launched while its predecessor (which produces the logit gradient) is still running: the activation part of the
+    // first stages is fetched now, the gradient part after the wait.  Each barrier expects both parts.
+    const int n_pre = a_early ? min(STAGES, c_end - c_begin) : 0;
+    if (tid == 0)
+        for (int it = 0; it < n_pre; ++it) {
+            const uint32_t bar = smem_u32(&full[it]), sa = base + it * stage_bytes;
+            mbar_expect_tx(bar, stage_bytes);
+            for (int cb = 0; cb < a_blocks; ++cb)
+                tma_load_3d(sa + cb * (kChunkPix * 128), &tmA, bar, (2 * m0 + cb) * kBlockK, (c_begin + it) * kChunkPix, s);
+        }
     pdl_wait();                  // inputs come from the previous kernel of the step
-    pdl_launch_dependents();
+    if (skip && skip[(int64_t)blockIdx.y * skip_stride]) {     // this stream's training loop has ended (block-uniform; the flag
+        tc_fence_before_sync();                                 // comes from an earlier kernel, so it is read after the wait)
+        __syncthreads();
+        if (warp == 0) tmem_dealloc(tmem, tmem_cols);
+        return;
+    }
     bool ok = true;
 
     if (tid == 0) {
@@ -187,9 +207,11 @@ tc_wgrad1x1_kernel(const __grid_constant__ CUtensorMap tmA,   // {K, p, S}      
             if (!ok) break;
             const uint32_t bar = smem_u32(&full[st]);
             const uint32_t sa = base + st * stage_bytes;
-            mbar_expect_tx(bar, stage_bytes);
-            for (int cb = 0; cb < a_blocks; ++cb)
-                tma_load_3d(sa + cb * (kChunkPix * 128), &tmA, bar, (2 * m0 + cb) * kBlockK, i * kChunkPix, s);
+            if (it >= n_pre) {
+                mbar_expect_tx(bar, stage_bytes);
+                for (int cb = 0; cb < a_blocks; ++cb)
+                    tma_load_3d(sa + cb * (kChunkPix * 128), &tmA, bar, (2 * m0 + cb) * kBlockK, i * kChunkPix, s);
+            }
             tma_load_3d(sa + a_stage_bytes, &tmB, bar, i * kChunkPix, 0, s);
         }
     } else if (tid == 32) {
@@ -213,6 +235,7 @@ tc_wgrad1x1_kernel(const __grid_constant__ CUtensorMap tmA,   // {K, p, S}      
     }
     __syncwarp();
     ok = mbar_wait(smem_u32(&done), 0, err, kWaitDone);
+    pdl_launch_dependents();     // only the epilogue is left
     tc_fence_after_sync();
     if (ok) {
         float* dst = partials + ((int64_t)s * n_split + split) * kClassPad * K;
@@ -267,7 +290,6 @@ tc_fwd1x1p_kernel(const __grid_constant__ CUtensorMap tmA,   // {K, p, S}  box {
                   float* __restrict__ z, int C, int p, int kblocks, unsigned int* err,
                   const int* __restrict__ skip, int64_t skip_stride)
 {
-    if (skip && skip[(int64_t)blockIdx.y * skip_stride]) return;   // this stream's training loop has ended (block-uniform)
     extern __shared__ uint8_t smem_raw[];
     uint8_t* smem = align_smem(smem_raw);
     const uint32_t a_base = smem_u32(smem);
@@ -290,7 +312,12 @@ tc_fwd1x1p_kernel(const __grid_constant__ CUtensorMap tmA,   // {K, p, S}  box {
     tc_fence_after_sync();
     const uint32_t tmem = tmem_slot;
     pdl_wait();                  // inputs come from the previous kernel of the step
-    pdl_launch_dependents();
+    if (skip && skip[(int64_t)blockIdx.y * skip_stride]) {     // this stream's training loop has ended (block-uniform; the flag
+        tc_fence_before_sync();                                 // comes from an earlier kernel, so it is read after the wait)
+        __syncthreads();
+        if (warp == 0) tmem_dealloc(tmem, 2 * kClassPad);
+        return;
+    }
     bool ok = true;
 
     if (tid == 0) {
@@ -309,6 +336,7 @@ tc_fwd1x1p_kernel(const __grid_constant__ CUtensorMap tmA,   // {K, p, S}  box {
                 tma_load_3d(a_base + st * kF1StageBytes, &tmA, bar, kb * kBlockK, it * kTileM, s);
             }
         }
+        pdl_launch_dependents();     // every load is issued: the next kernel of the step may set itself up
     } else if (tid == 32) {
         // ---- MMA issuer
         constexpr uint32_t idesc = instr_desc(kTileM, kClassPad, 0, 0);
@@ -408,7 +436,6 @@ tc_fwd3x3_kernel(const __grid_constant__ CUtensorMap tmA,   // {Cin, w, h, S}   
     tc_fence_after_sync();
     const uint32_t tmem = tmem_slot;
     pdl_wait();                  // inputs come from the previous kernel of the step
-    pdl_launch_dependents();
     bool ok = true;
 
     if (tid == 0) {
@@ -432,6 +459,7 @@ tc_fwd3x3_kernel(const __grid_constant__ CUtensorMap tmA,   // {Cin, w, h, S}   
                         tma_load_3d(sa + a_bytes + j * (64 * 128), &tmBq, bar, kb * kBlockK, tap * Ch + im.ch0 + j * 64, s);
             }
         }
+        pdl_launch_dependents();     // every load is issued: the next kernel of the step may set itself up
     } else if (tid == 32) {
         // ---- MMA issuer
         int g = 0, j = 0;
@@ -522,7 +550,6 @@ tc_wgrad3x3_kernel(const __grid_constant__ CUtensorMap tmA,   // X   {Cin, w, h,
                    int Cin, int Ch, int h, int w, int n_chunks, int chunks_per_block, int n_split,
                    int tmem_cols, unsigned int* err, const int* __restrict__ skip, int64_t skip_stride)
 {
-    if (skip && skip[(int64_t)blockIdx.y * skip_stride]) return;   // this stream's training loop has ended (block-uniform)
     extern __shared__ uint8_t smem_raw[];
     uint8_t* smem = align_smem(smem_raw);
     const uint32_t base = smem_u32(smem);
@@ -548,7 +575,12 @@ tc_wgrad3x3_kernel(const __grid_constant__ CUtensorMap tmA,   // X   {Cin, w, h,
     tc_fence_after_sync();
     const uint32_t tmem = tmem_slot;
     pdl_wait();                  // inputs come from the previous kernel of the step
-    pdl_launch_dependents();
+    if (skip && skip[(int64_t)blockIdx.y * skip_stride]) {     // this stream's training loop has ended (block-uniform; the flag
+        tc_fence_before_sync();                                 // comes from an earlier kernel, so it is read after the wait)
+        __syncthreads();
+        if (warp == 0) tmem_dealloc(tmem, tmem_cols);
+        return;
+    }
     bool ok = true;
 
     if (tid == 0) {
@@ -585,6 +617,7 @@ tc_wgrad3x3_kernel(const __grid_constant__ CUtensorMap tmA,   // X   {Cin, w, h,
     }
     __syncwarp();
     ok = mbar_wait(smem_u32(&done), 0, err, kWaitDone);
+    pdl_launch_dependents();     // only the epilogue is left
     tc_fence_after_sync();
     if (ok) {
         float* dst = partials + (((int64_t)s * n_split + split) * 9 + tap) * Ch * Cin;
@@ -623,7 +656,6 @@ tc_dgrad_kernel(const __grid_constant__ CUtensorMap tmA,   // dz  {p, 32, S}  bo
                 float* __restrict__ b1_partials,            // [S][n_blocks][Ch]
                 int Ch, int p, int tmem_cols, unsigned int* err, const int* __restrict__ skip, int64_t skip_stride)
 {
-    if (skip && skip[(int64_t)blockIdx.y * skip_stride]) return;   // this stream's training loop has ended (block-uniform)
     extern __shared__ uint8_t smem_raw[];
     uint8_t* smem = align_smem(smem_raw);
     const uint32_t a_base = smem_u32(smem);
@@ -649,7 +681,12 @@ tc_dgrad_kernel(const __grid_constant__ CUtensorMap tmA,   // dz  {p, 32, S}  bo
     tc_fence_after_sync();
     const uint32_t tmem = tmem_slot;
     pdl_wait();                  // inputs come from the previous kernel of the step
-    pdl_launch_dependents();
+    if (skip && skip[(int64_t)blockIdx.y * skip_stride]) {     // this stream's training loop has ended (block-uniform; the flag
+        tc_fence_before_sync();                                 // comes from an earlier kernel, so it is read after the wait)
+        __syncthreads();
+        if (warp == 0) tmem_dealloc(tmem, tmem_cols);
+        return;
+    }
     bool ok = true;
 
     if (tid == 0) {
@@ -681,6 +718,7 @@ tc_dgrad_kernel(const __grid_constant__ CUtensorMap tmA,   // dz  {p, 32, S}  bo
         for (int j = 0; j < 8; ++j) if (j < Chb / 32) mbits[j] = __ldg(mp + ch0 / 32 + j);
     }
     ok = mbar_wait(smem_u32(&done), 0, err, kWaitDone);
+    pdl_launch_dependents();             // only the epilogue is left
     tc_fence_after_sync();
     ok = __syncthreads_and(ok);          // the epilogue below synchronises the block: all or none
     if (ok) {
@@ -949,7 +987,7 @@ int tc_forward(const TcPlan* P, cudaStream_t s, StageTimer* t, const int* skip, 
             if (b.c_hidden % 256 == 0 && tail * 4 <= grid) tail_split = 4;
             else if (b.c_hidden % 128 == 0 && tail * 2 <= grid) tail_split = 2;
         }
-        ST_REPEAT(t) launch_chain(tc_fwd3x3_kernel<4>, dim3(grid), dim3(kFwd3Threads), P->smem_fwd3, s,
+        ST_REPEAT(t) launch_chain(b.chain_early != 0, tc_fwd3x3_kernel<4>, dim3(grid), dim3(kFwd3Threads), P->smem_fwd3, s,
             P->x_fwd3, P->w1_map, P->w1_map_q, tail_split, b.theta, b.n_params, b.b1_off, b.hidden, b.relu_bits, b.c_in, b.c_hidden, b.h, b.w,
             total, pow2_cols(b.c_hidden), b.err, skip, skip_stride);
         if (t) t->mark("tc_fwd3x3", s, st_repeats(t));
@@ -960,13 +998,13 @@ int tc_forward(const TcPlan* P, cudaStream_t s, StageTimer* t, const int* skip, 
         int gx = P->n_sms / b.S;
         if (gx < 1) gx = 1;
         if (gx > tiles1) gx = tiles1;
-        ST_REPEAT(t) launch_chain(tc_fwd1x1p_kernel, dim3(gx, b.S), dim3(kF1Threads), P->smem_fwd1p, s,
+        ST_REPEAT(t) launch_chain(b.chain_early != 0, tc_fwd1x1p_kernel, dim3(gx, b.S), dim3(kF1Threads), P->smem_fwd1p, s,
             P->act_fwd, P->w2_map, b.theta, b.n_params, b.b2_off, b.z, b.C, P->p, P->c_last / kBlockK, b.err, skip, skip_stride);
     } else {
         // one-layer head, no per-stream skip flags to wait for, not a timing run: the activations are the frozen
         // features, which no kernel of the loop writes
         const bool a_early = after_update && !b.c_hidden && !skip && !t && fwd1_early_enabled();
-        ST_REPEAT(t) launch_early(a_early || pdl_enabled(), tc_fwd1x1_kernel, dim3(tiles1, b.S), dim3(kThreadsTc), P->smem_fwd1, s,
+        ST_REPEAT(t) launch_early(a_early || b.chain_early, tc_fwd1x1_kernel, dim3(tiles1, b.S), dim3(kThreadsTc), P->smem_fwd1, s,
             P->act_fwd, P->w2_map, b.theta, b.n_params, b.b2_off, b.z, b.C, P->p, P->c_last / kBlockK, b.err, skip, skip_stride,
             a_early ? 1 : 0);
     }
@@ -978,17 +1016,19 @@ int tc_backward(const TcPlan* P, cudaStream_t s, StageTimer* t, const int* skip,
 {
     const TcBuffers& b = P->b;
     int n = 0;
-    ST_REPEAT(t) launch_chain(tc_wgrad1x1_kernel<kWg1Stages>, dim3(P->split2 * P->msplit2, b.S), dim3(kThreadsTc), P->smem_wg1, s,
-        P->act_wg, P->dz_map, b.w2_partials, P->c_last, P->chunks2, P->per2, P->msplit2, P->cols2, b.err, skip, skip_stride);
+    // one-layer head: the activations are the frozen features, which no kernel of the loop writes
+    const int a_early = (!b.c_hidden && !skip && !t && b.chain_early) ? 1 : 0;
+    ST_REPEAT(t) launch_chain(b.chain_early != 0, tc_wgrad1x1_kernel<kWg1Stages>, dim3(P->split2 * P->msplit2, b.S), dim3(kThreadsTc), P->smem_wg1, s,
+        P->act_wg, P->dz_map, b.w2_partials, P->c_last, P->chunks2, P->per2, P->msplit2, P->cols2, b.err, skip, skip_stride, a_early);
     if (t) t->mark("tc_wgrad1x1", s, st_repeats(t));
     n += st_repeats(t);
     if (b.c_hidden) {
         const int blocks = tc_b1_partials(b.h, b.w);
         const int n_ch_split = (b.c_hidden % 128 == 0) ? 2 : 1;      // each block: a multiple of 64 channels (four ways measured no better)
-        ST_REPEAT(t) launch_chain(tc_dgrad_kernel, dim3(blocks, b.S, n_ch_split), dim3(kThreadsTc), P->smem_dgrad, s,
+        ST_REPEAT(t) launch_chain(b.chain_early != 0, tc_dgrad_kernel, dim3(blocks, b.S, n_ch_split), dim3(kThreadsTc), P->smem_dgrad, s,
             P->dz_map, P->w2_map, b.relu_bits, b.dhidden, b.b1_partials, b.c_hidden, P->p, pow2_cols(b.c_hidden / n_ch_split), b.err, skip, skip_stride);
         if (t) t->mark("tc_dgrad", s, st_repeats(t));
-        ST_REPEAT(t) launch_chain(tc_wgrad3x3_kernel<3>, dim3(9 * P->split1, b.S), dim3(kThreadsTc), P->smem_wg3, s,
+        ST_REPEAT(t) launch_chain(b.chain_early != 0, tc_wgrad3x3_kernel<3>, dim3(9 * P->split1, b.S), dim3(kThreadsTc), P->smem_wg3, s,
             P->x_wg3, P->dh_wg3, b.w1_partials, b.c_in, b.c_hidden, b.h, b.w, P->chunks1, P->per1, P->split1,
             P->cols1, b.err, skip, skip_stride);
         if (t) t->mark("tc_wgrad3x3", s, st_repeats(t));

@@ -14,7 +14,7 @@ namespace st {
 
 bool pdl_enabled()
 {
-    static const bool on = [] { const char* e = getenv("ST_PDL"); return e && e[0] == '1'; }();
+    static const bool on = [] { const char* e = getenv("ST_PDL"); return !(e && e[0] == '0'); }();
     return on;
 }
 
@@ -37,22 +37,41 @@ __device__ __forceinline__ AdamCorr adam_corrections(const UpdateArgs& a, int s)
 // OptimStep on one parameter.  Gradient descent with momentum: v <- mu v + g; theta <- theta - lr v.
 // Adam (each element in double, stored as fp32): m <- b1 m + (1 - b1) g; v <- b2 v + (1 - b2) g^2;
 // theta <- theta - lr (m / c1) / (sqrt(v / c2) + eps).
+// The state of one parameter (value, momentum or first moment, second moment), which the gradient kernels before the
+// update never write: it can be fetched before their results are waited for.
+struct ParamState { float theta, vel, vel2; };
 template <bool ADAM>
-__device__ __forceinline__ void apply_update(const UpdateArgs& a, int64_t gi, float g, const AdamCorr& k)
+__device__ __forceinline__ ParamState load_state(const UpdateArgs& a, int64_t gi)
+{
+    ParamState p;
+    p.theta = a.theta[gi]; p.vel = a.vel[gi]; p.vel2 = ADAM ? a.vel2[gi] : 0.f;
+    return p;
+}
+
+template <bool ADAM>
+__device__ __forceinline__ float apply_update(const UpdateArgs& a, int64_t gi, float g, const AdamCorr& k, const ParamState& p)
 {
     a.grad[gi] = g;
     if (ADAM) {
         const double gd = (double)g;
-        const double m = a.b1 * (double)a.vel[gi] + (1.0 - a.b1) * gd;
-        const double v = a.b2 * (double)a.vel2[gi] + (1.0 - a.b2) * gd * gd;
+        const double m = a.b1 * (double)p.vel + (1.0 - a.b1) * gd;
+        const double v = a.b2 * (double)p.vel2 + (1.0 - a.b2) * gd * gd;
         a.vel[gi] = (float)m;
         a.vel2[gi] = (float)v;
-        a.theta[gi] = (float)((double)a.theta[gi] - (double)a.lr * (m / k.c1) / (sqrt(v / k.c2) + a.eps));
-        return;
+        const float t = (float)((double)p.theta - (double)a.lr * (m / k.c1) / (sqrt(v / k.c2) + a.eps));
+        a.theta[gi] = t;
+        return t;
     }
-    float v = fmaf(a.mu, a.vel[gi], g);
+    float v = fmaf(a.mu, p.vel, g);
     a.vel[gi] = v;
-    a.theta[gi] = fmaf(-a.lr, v, a.theta[gi]);
+    const float t = fmaf(-a.lr, v, p.theta);
+    a.theta[gi] = t;
+    return t;
+}
+template <bool ADAM>
+__device__ __forceinline__ float apply_update(const UpdateArgs& a, int64_t gi, float g, const AdamCorr& k)
+{
+    return apply_update<ADAM>(a, gi, g, k, load_state<ADAM>(a, gi));
 }
 
 // Parameter blocks: a block covers kUpdThreads / G consecutive parameters; the G thread groups of a
@@ -65,23 +84,21 @@ sgd_update_kernel(UpdateArgs a, int n_param_blocks, int64_t range_begin)
     constexpr int kRow = kUpdThreads / G;      // consecutive parameters covered by one thread group
     constexpr int kPer = kRow * E;             // parameters per block
     __shared__ float part[G][kPer];
-    pdl_wait();
-    pdl_launch_dependents();
     const int s = blockIdx.y;
     const int64_t base = (int64_t)s * a.n_params;
-    const bool skip = a.skip && a.skip[(int64_t)s * a.skip_stride];   // block-uniform
-    const AdamCorr corr = adam_corrections<ADAM>(a, s);
-    if ((int)blockIdx.x < n_param_blocks) {
-        if (skip) return;
-        const int col = threadIdx.x % kRow, g = threadIdx.x / kRow;
-        int layer[E];
-        bool is_weight[E], has_partials[E];
-        float sum[E];
-        // E parameters per thread, all of their split-K loads issued before any is consumed
+    const bool param_block = (int)blockIdx.x < n_param_blocks;
+    const int col = threadIdx.x % kRow, g = threadIdx.x / kRow;
+    int layer[E];
+    bool is_weight[E], has_partials[E];
+    ParamState state[E];
+    // which parameters this thread looks after, and (first thread group) their current state: none of it comes from the
+    // kernels just before this one, so it is done before their completion is waited for
+    if (param_block) {
 #pragma unroll
         for (int e = 0; e < E; ++e) {
             const int64_t i = range_begin + (int64_t)blockIdx.x * kPer + e * kRow + col;
-            layer[e] = -1; is_weight[e] = false; has_partials[e] = false; sum[e] = 0.f;
+            layer[e] = -1; is_weight[e] = false; has_partials[e] = false;
+            state[e].theta = state[e].vel = state[e].vel2 = 0.f;
             if (i < a.n_params) {
                 for (int L = 0; L < a.n_layers; ++L) {
                     const LayerUpdate& ly = a.layer[L];
@@ -90,6 +107,21 @@ sgd_update_kernel(UpdateArgs a, int n_param_blocks, int64_t range_begin)
                     if (i >= ly.b_off && i < ly.b_off + ly.cout) { layer[e] = L; is_weight[e] = false; }
                 }
             }
+            if (g == 0 && layer[e] >= 0 && (is_weight[e] || !a.layer[layer[e]].b_partials)) state[e] = load_state<ADAM>(a, base + i);
+        }
+    }
+    pdl_wait();
+    pdl_launch_dependents();
+    const bool skip = a.skip && a.skip[(int64_t)s * a.skip_stride];   // block-uniform
+    const AdamCorr corr = adam_corrections<ADAM>(a, s);
+    if (param_block) {
+        if (skip) return;
+        float sum[E];
+        // E parameters per thread, all of their split-K loads issued before any is consumed
+#pragma unroll
+        for (int e = 0; e < E; ++e) {
+            const int64_t i = range_begin + (int64_t)blockIdx.x * kPer + e * kRow + col;
+            sum[e] = 0.f;
             if (layer[e] >= 0 && is_weight[e] && a.layer[layer[e]].w_partials) {
                 const LayerUpdate& ly = a.layer[layer[e]];
                 has_partials[e] = true;
@@ -127,10 +159,10 @@ sgd_update_kernel(UpdateArgs a, int n_param_blocks, int64_t range_begin)
                 } else {
                     gr = a.grad[base + i];
                 }
-                apply_update<ADAM>(a, base + i, gr, corr);
-                if (ly.shadow) ly.shadow[(int64_t)s * ly.shadow_stream_stride + (i - ly.w_off)] = __float2bfloat16_rn(a.theta[base + i]);
+                const float t = apply_update<ADAM>(a, base + i, gr, corr, state[e]);
+                if (ly.shadow) ly.shadow[(int64_t)s * ly.shadow_stream_stride + (i - ly.w_off)] = __float2bfloat16_rn(t);
             } else if (!ly.b_partials) {
-                apply_update<ADAM>(a, base + i, a.grad[base + i], corr);
+                apply_update<ADAM>(a, base + i, a.grad[base + i], corr, state[e]);
             }   // biases with partial sums are finished by the reduction warps below
         }
         return;
@@ -240,8 +272,8 @@ static int launch_sgd_update_t(const UpdateArgs& a, cudaStream_t s)
         if (ly.w_partials && nw >= 65536 && ly.w_off == range_begin) {
             const bool vec = nw % 4 == 0 && ly.w_split_stride % 4 == 0 && ly.w_stream_stride % 4 == 0 &&
                              ((uintptr_t)ly.w_partials % 16 == 0);
-            if (vec) launch_chain(sgd_update_stream_kernel<4, ADAM>, dim3((unsigned)((nw / 4 + 255) / 256), (unsigned)a.S), dim3(256), 0, s, a, L);
-            else launch_chain(sgd_update_stream_kernel<1, ADAM>, dim3((unsigned)((nw + 255) / 256), (unsigned)a.S), dim3(256), 0, s, a, L);
+            if (vec) launch_chain(a.chain_early != 0, sgd_update_stream_kernel<4, ADAM>, dim3((unsigned)((nw / 4 + 255) / 256), (unsigned)a.S), dim3(256), 0, s, a, L);
+            else launch_chain(a.chain_early != 0, sgd_update_stream_kernel<1, ADAM>, dim3((unsigned)((nw + 255) / 256), (unsigned)a.S), dim3(256), 0, s, a, L);
             range_begin = ly.w_off + nw;
             ++n_launches;
         }
@@ -260,11 +292,11 @@ static int launch_sgd_update_t(const UpdateArgs& a, cudaStream_t s)
     const int n_param_blocks = (int)((n_rest + per - 1) / per);
     const dim3 grid((unsigned)(n_param_blocks + n_red_blocks), (unsigned)a.S);
     const dim3 blk(kUpdThreads);
-    if (G == 1 && E == 1) launch_chain(sgd_update_kernel<1, 1, ADAM>, grid, blk, 0, s, a, n_param_blocks, range_begin);
-    else if (G == 1) launch_chain(sgd_update_kernel<1, 4, ADAM>, grid, blk, 0, s, a, n_param_blocks, range_begin);
-    else if (G == 16) launch_chain(sgd_update_kernel<16, 1, ADAM>, grid, blk, 0, s, a, n_param_blocks, range_begin);
-    else if (E == 1) launch_chain(sgd_update_kernel<8, 1, ADAM>, grid, blk, 0, s, a, n_param_blocks, range_begin);
-    else launch_chain(sgd_update_kernel<8, 4, ADAM>, grid, blk, 0, s, a, n_param_blocks, range_begin);
+    if (G == 1 && E == 1) launch_chain(a.chain_early != 0, sgd_update_kernel<1, 1, ADAM>, grid, blk, 0, s, a, n_param_blocks, range_begin);
+    else if (G == 1) launch_chain(a.chain_early != 0, sgd_update_kernel<1, 4, ADAM>, grid, blk, 0, s, a, n_param_blocks, range_begin);
+    else if (G == 16) launch_chain(a.chain_early != 0, sgd_update_kernel<16, 1, ADAM>, grid, blk, 0, s, a, n_param_blocks, range_begin);
+    else if (E == 1) launch_chain(a.chain_early != 0, sgd_update_kernel<8, 1, ADAM>, grid, blk, 0, s, a, n_param_blocks, range_begin);
+    else launch_chain(a.chain_early != 0, sgd_update_kernel<8, 4, ADAM>, grid, blk, 0, s, a, n_param_blocks, range_begin);
     return n_launches;
 }
 

@@ -266,8 +266,8 @@ void launch_upsample_ce(const UpsampleCeArgs& a, const CUtensorMap* z_map, cudaS
     size_t smem = 0;
     const int chunk = chunk_classes(a.C, &smem);
     dim3 grid((unsigned)((a.w + NX - 1) / NX), (unsigned)((a.h + NY - 1) / NY), (unsigned)a.S);
-    if (a.conf) launch_chain(upsample_ce_kernel<true>, grid, dim3(kThreads), smem, s, a, chunk);
-    else launch_chain(upsample_ce_kernel<false>, grid, dim3(kThreads), smem, s, a, chunk);
+    if (a.conf) launch_chain(a.chain_early != 0, upsample_ce_kernel<true>, grid, dim3(kThreads), smem, s, a, chunk);
+    else launch_chain(a.chain_early != 0, upsample_ce_kernel<false>, grid, dim3(kThreads), smem, s, a, chunk);
 }
 
 }  // namespace st

@@ -197,9 +197,6 @@ upsample_ce_rows_kernel(UpsampleCeArgs a, const __grid_constant__ CUtensorMap z_
     const float* z = a.z + (int64_t)s * C * p;
     const uint8_t* labels = a.labels + (int64_t)s * H * W;
     const int tid = threadIdx.x, wi = tid >> 5, l = tid & 31;
-    pdl_wait();                  // the logits come from the previous kernel of the step
-    if (a.skip && a.skip[(int64_t)s * a.skip_stride]) return;     // this stream's training loop has ended (block-uniform)
-    pdl_launch_dependents();
 
     // ---- tile: node rows y0-1 .. y0+RN_Y, node columns xa .. xa+35 where xa = (x0-1) rounded down to a
     // multiple of 4 (so that rows are fetched as 16-byte vectors), clamped at the borders, scaled by
@@ -207,16 +204,6 @@ upsample_ce_rows_kernel(UpsampleCeArgs a, const __grid_constant__ CUtensorMap z_
     const bool vec_ok = (w % 4 == 0) && ((uintptr_t)z % 16 == 0);
     const int xa = vec_ok ? ((x0 - 1) & ~3) : x0 - 1;      // x0-1 >= -1; (-1 & ~3) = -4
     const int off = (x0 - 1) - xa;                         // column of node x0-1 inside the tile
-    if (a.has_map && tid == 0) {                           // block-uniform flag (implies vec_ok)
-        // one tile copy for the whole block, started before anything else: box {36 columns, RN_Y + 2 node rows,
-        // C classes} at (xa, y0 - 1, s C).  Rows and columns outside the map arrive as zeros and are replaced
-        // below by the clamped border values.
-        const uint32_t bar = tc::smem_u32(&tile_bar);
-        tc::mbar_init(bar, 1);
-        tc::fence_barrier_init();
-        tc::mbar_expect_tx(bar, (uint32_t)(C * TZ * sizeof(float)));
-        tc::tma_load_3d(tc::smem_u32(zt), &z_map, bar, xa, y0 - 1, s * C);
-    }
     const int i = y0 - 1 + wi;                  // cell row: frame rows 4i+2 .. 4i+5, node rows (i, i+1)
     const int n = x0 - 1 + l;                   // own node column; cell n lies between node columns n and n+1
     const bool cell_row_valid = i <= h - 1;
@@ -259,12 +246,28 @@ upsample_ce_rows_kernel(UpsampleCeArgs a, const __grid_constant__ CUtensorMap z_
         constexpr int kIter = (CB + kPlanes - 1) / kPlanes;
         const int g = tid / kQuads, q = tid % kQuads;
         float4* zt4 = reinterpret_cast<float4*>(zt);
-        if (a.has_map) {
-            // ---- the tile copy is in flight since the start of the block
-            const uint32_t bar = tc::smem_u32(&tile_bar);
+        if (a.has_map) {                                       // shared memory the tile copy does not write
             for (int e = tid; e < (CB - C) * kQuads; e += R_THREADS) zt4[C * kQuads + e] = make_float4(-1e30f, -1e30f, -1e30f, -1e30f);
             for (int e = tid; e < C * TZ / 4; e += R_THREADS) reinterpret_cast<int4*>(corr)[e] = make_int4(0, 0, 0, 0);
             if (CONF) for (int e = tid; e < C * C; e += R_THREADS) hist[e] = 0;
+        }
+        // The logits come from the previous kernel of the step; nothing before this line depends on them, so a launch that
+        // started while that kernel was still running has used the time.
+        pdl_wait();
+        if (a.skip && a.skip[(int64_t)s * a.skip_stride]) return;     // this stream's training loop has ended (block-uniform)
+        if (a.has_map && tid == 0) {                           // block-uniform flag (implies vec_ok)
+            // one tile copy for the whole block, started before anything else that needs the logits: box {36 columns,
+            // RN_Y + 2 node rows, C classes} at (xa, y0 - 1, s C).  Rows and columns outside the map arrive as zeros and
+            // are replaced below by the clamped border values.
+            const uint32_t bar = tc::smem_u32(&tile_bar);
+            tc::mbar_init(bar, 1);
+            tc::fence_barrier_init();
+            tc::mbar_expect_tx(bar, (uint32_t)(C * TZ * sizeof(float)));
+            tc::tma_load_3d(tc::smem_u32(zt), &z_map, bar, xa, y0 - 1, s * C);
+        }
+        if (a.has_map) {
+            // ---- the tile copy is in flight
+            const uint32_t bar = tc::smem_u32(&tile_bar);
             __syncthreads();                                   // the barrier's initialisation is visible to every waiter
             bool ok = false;
             for (uint32_t it = 0; it < 2 * tc::kSpinLimit && !ok; ++it) ok = tc::mbar_try_wait(bar, 0);
@@ -580,6 +583,7 @@ upsample_ce_rows_kernel(UpsampleCeArgs a, const __grid_constant__ CUtensorMap z_
     if (l == 0) red[wi] = loss;
     if (n_bad) atomicAdd(a.bad, n_bad);
     __syncthreads();
+    pdl_launch_dependents();                     // only the epilogue is left: the next kernel of the step may set itself up
     if (CONF) {                                  // one global update per non-empty counter of the block
         for (int e = tid; e < C * C; e += R_THREADS)
             if (hist[e]) atomicAdd(a.conf + (int64_t)s * a.conf_stream_stride + e, (unsigned long long)hist[e]);
@@ -671,8 +675,8 @@ template <int CB>
 cudaError_t launch_cb(const UpsampleCeArgs& a, const CUtensorMap& z_map, cudaStream_t s)
 {
     dim3 grid((unsigned)((a.w + RN_X - 1) / RN_X), (unsigned)((a.h + RN_Y - 1) / RN_Y), (unsigned)a.S);
-    if (a.conf) return launch_chain(upsample_ce_rows_kernel<CB, true>, grid, dim3(R_THREADS), rows_smem_bytes<CB>(a.C, true), s, a, z_map);
-    return launch_chain(upsample_ce_rows_kernel<CB, false>, grid, dim3(R_THREADS), rows_smem_bytes<CB>(a.C, false), s, a, z_map);
+    if (a.conf) return launch_chain(a.chain_early != 0, upsample_ce_rows_kernel<CB, true>, grid, dim3(R_THREADS), rows_smem_bytes<CB>(a.C, true), s, a, z_map);
+    return launch_chain(a.chain_early != 0, upsample_ce_rows_kernel<CB, false>, grid, dim3(R_THREADS), rows_smem_bytes<CB>(a.C, false), s, a, z_map);
 }
 
 // class-count buckets: the two workload sizes exactly, multiples of four otherwise

@@ -77,11 +77,17 @@ struct st_ctx {
     float* read_tmp = nullptr; size_t read_tmp_bytes = 0;
     void* staging = nullptr; size_t staging_bytes = 0;
     std::vector<char> has_feat, has_labels;
+    // inputs of the next key frame, copied from host memory on a stream of the library's own while the current key
+    // frame is trained (st_prefetch_key_frame); all created on first use
+    cudaStream_t copy_stream = nullptr;
+    struct Prefetch { float* feat = nullptr; float* logits = nullptr; cudaEvent_t copied = nullptr, consumed = nullptr; bool pending = false, used_once = false; };
+    std::vector<Prefetch> prefetch;
     bool z_current = false;                 // z holds the forward of the current parameters and features of every stream
     TcPlan* plan = nullptr;
     struct StepGraph { cudaGraphExec_t exec; int64_t n_launches; };
     std::map<GraphKey, StepGraph> graphs;
     bool use_graphs = true;
+    bool chain_early = false;               // kernels of a step may start while their predecessor drains (one-layer heads)
     std::string err;
     int64_t launches = 0;
     std::vector<void*> allocs;
@@ -204,6 +210,7 @@ UpdateArgs make_update_args(st_ctx* c, int slot, const int* skip = nullptr, int6
     u.skip = skip; u.skip_stride = skip_stride;
     u.adam = c->adam ? 1 : 0; u.vel2 = c->vel2; u.step_base = c->step_base;
     u.b1 = c->b1; u.b2 = c->b2; u.eps = c->eps; u.ln_b1 = log(c->b1); u.ln_b2 = log(c->b2);
+    u.chain_early = c->chain_early ? 1 : 0;
     return u;
 }
 
@@ -264,6 +271,7 @@ UpsampleCeArgs k3_args(st_ctx* c, bool fp32_grad, bool bf16_grad, unsigned long 
     k3.S = c->S; k3.C = c->C; k3.h = c->h; k3.w = c->w;
     k3.has_map = c->k3_has_map;
     k3.skip = skip; k3.skip_stride = skip_stride;
+    k3.chain_early = c->chain_early ? 1 : 0;
     return k3;
 }
 
@@ -391,6 +399,14 @@ void st_destroy(st_ctx* ctx)
     if (ctx->plan) tc_plan_destroy(ctx->plan);
     for (void* q : ctx->allocs) cudaFree(q);
     if (ctx->staging) cudaFree(ctx->staging);
+    if (ctx->copy_stream) cudaStreamSynchronize(ctx->copy_stream);
+    for (auto& pf : ctx->prefetch) {
+        if (pf.feat) cudaFree(pf.feat);
+        if (pf.logits) cudaFree(pf.logits);
+        if (pf.copied) cudaEventDestroy(pf.copied);
+        if (pf.consumed) cudaEventDestroy(pf.consumed);
+    }
+    if (ctx->copy_stream) cudaStreamDestroy(ctx->copy_stream);
     if (ctx->read_tmp) cudaFree(ctx->read_tmp);
     if (ctx->status_host) cudaFreeHost(ctx->status_host);
     delete ctx;
@@ -447,6 +463,11 @@ st_status st_init_head(const st_head_desc* desc, const float* init_params, st_ct
     // The legacy default stream cannot be captured: steps are then enqueued kernel by kernel.
     c->use_graphs = c->stream != nullptr && c->stream != cudaStreamLegacy && c->stream != cudaStreamPerThread;
     if (const char* e = getenv("ST_NO_GRAPH")) if (e[0] == '1') c->use_graphs = false;
+    // Programmatic dependent launch along the step's chain: with the one-layer head every kernel has something to do
+    // before its predecessor's results are needed (label fetch, feature tiles) and the step is 2 us shorter; the
+    // two-layer head's kernels fill the SMs to the end and gain nothing (measured: 1 us slower).  ST_PDL=0 / 1 force it.
+    c->chain_early = pdl_enabled() && c->Ch == 0;
+    if (const char* e = getenv("ST_PDL")) if (e[0] == '1') c->chain_early = true;
 
     PackLayout& L = c->layout;
     memset(&L, 0, sizeof L);
@@ -520,6 +541,7 @@ st_status st_init_head(const st_head_desc* desc, const float* init_params, st_ct
         b.x = c->x_bf16; b.w1 = c->w1_shadow; b.w2 = c->w2_shadow; b.theta = c->theta; b.n_params = c->n_params;
         b.b1_off = c->Ch ? L.b_off[0] : 0; b.b2_off = L.b_off[L.n_layers - 1]; b.w2_off = L.w_off[L.n_layers - 1];
         b.err = c->bad + 2;
+        b.chain_early = c->chain_early ? 1 : 0;
         b.z = c->z; b.hidden = c->hid_bf16; b.relu_bits = c->relu_bits; b.dz = c->dz; b.dz_bf16 = c->dz_bf16; b.dhidden = c->dhid_bf16;
         b.w1_partials = c->w1_partials; b.w2_partials = c->w2_partials; b.b1_partials = c->b1_partials;
         char msg[256] = {0};
@@ -581,6 +603,47 @@ st_status st_teacher_labels(st_ctx* ctx, int32_t stream, const float* logits_chw
     if (labels_out) ST_CUDA(ctx, cudaMemcpyAsync(labels_out, dst, (size_t)ctx->P, cudaMemcpyDefault, ctx->stream));
     ctx->has_labels[stream] = 1;
     return tag_labels(ctx, stream);
+}
+
+st_status st_prefetch_key_frame(st_ctx* ctx, int32_t stream, const float* feat_chw, const float* logits_chw)
+{
+    st_status st = check_stream_index(ctx, stream);
+    if (st != ST_OK) return st;
+    if (!feat_chw || !logits_chw) return fail(ctx, ST_ERR_INVALID_ARG, "st_prefetch_key_frame: NULL input");
+    if (ctx->prefetch.empty()) ctx->prefetch.resize(ctx->S);
+    st_ctx::Prefetch& pf = ctx->prefetch[stream];
+    const size_t fbytes = (size_t)ctx->Cin * ctx->p * sizeof(float), lbytes = (size_t)ctx->C * ctx->P * sizeof(float);
+    if (!ctx->copy_stream) ST_CUDA(ctx, cudaStreamCreateWithFlags(&ctx->copy_stream, cudaStreamNonBlocking));
+    if (!pf.feat) {
+        ST_CUDA(ctx, cudaMalloc((void**)&pf.feat, fbytes));
+        ST_CUDA(ctx, cudaMalloc((void**)&pf.logits, lbytes));
+        ST_CUDA(ctx, cudaEventCreateWithFlags(&pf.copied, cudaEventDisableTiming));
+        ST_CUDA(ctx, cudaEventCreateWithFlags(&pf.consumed, cudaEventDisableTiming));
+    }
+    // the kernels that read the previous contents of the two buffers must have run before they are overwritten
+    if (pf.used_once) ST_CUDA(ctx, cudaStreamWaitEvent(ctx->copy_stream, pf.consumed, 0));
+    ST_CUDA(ctx, cudaMemcpyAsync(pf.feat, feat_chw, fbytes, cudaMemcpyDefault, ctx->copy_stream));
+    ST_CUDA(ctx, cudaMemcpyAsync(pf.logits, logits_chw, lbytes, cudaMemcpyDefault, ctx->copy_stream));
+    ST_CUDA(ctx, cudaEventRecord(pf.copied, ctx->copy_stream));
+    pf.pending = true;
+    return ST_OK;
+}
+
+st_status st_use_prefetched_key_frame(st_ctx* ctx, int32_t stream, uint8_t* labels_out)
+{
+    st_status st = check_stream_index(ctx, stream);
+    if (st != ST_OK) return st;
+    if (ctx->prefetch.empty() || !ctx->prefetch[stream].pending)
+        return fail(ctx, ST_ERR_BAD_STATE, "st_use_prefetched_key_frame: stream %d has no prefetched key frame", stream);
+    st_ctx::Prefetch& pf = ctx->prefetch[stream];
+    ST_CUDA(ctx, cudaStreamWaitEvent(ctx->stream, pf.copied, 0));      // the device waits for the copy, the host does not
+    st = st_set_frozen_features(ctx, stream, pf.feat);
+    if (st == ST_OK) st = st_teacher_labels(ctx, stream, pf.logits, labels_out);
+    if (st != ST_OK) return st;
+    ST_CUDA(ctx, cudaEventRecord(pf.consumed, ctx->stream));
+    pf.pending = false;
+    pf.used_once = true;
+    return ST_OK;
 }
 
 st_status st_set_labels(st_ctx* ctx, int32_t stream, const uint8_t* labels)

@@ -33,7 +33,7 @@ __device__ __forceinline__ void store_256(void* dst, const uint32_t* r)
 __device__ __forceinline__ void pdl_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
 __device__ __forceinline__ void pdl_launch_dependents() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
 
-bool pdl_enabled();   // true if the environment variable ST_PDL is set to 1 (off by default: it measured no gain)
+bool pdl_enabled();   // true unless the environment variable ST_PDL is set to 0
 
 // `early`: launch with the programmatic-serialization attribute, i.e. the kernel may start before its predecessor on
 // the stream has completed and must call pdl_wait() before it touches anything the predecessor writes.
@@ -49,10 +49,11 @@ inline cudaError_t launch_early(bool early, void (*kernel)(KArgs...), dim3 grid,
     return cudaLaunchKernelEx(&cfg, kernel, std::forward<Args>(args)...);
 }
 
+// A kernel of the step's chain; `early` is the context's choice (the `chain_early` field of the argument structs).
 template <typename... KArgs, typename... Args>
-inline cudaError_t launch_chain(void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t smem, cudaStream_t s, Args&&... args)
+inline cudaError_t launch_chain(bool early, void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t smem, cudaStream_t s, Args&&... args)
 {
-    return launch_early(pdl_enabled(), kernel, grid, block, smem, s, std::forward<Args>(args)...);
+    return launch_early(early, kernel, grid, block, smem, s, std::forward<Args>(args)...);
 }
 #endif
 
@@ -101,6 +102,7 @@ struct UpsampleCeArgs {
     int64_t skip_stride;
     int heavy_w;             // 1, or the integer weight (2..5) of the pixels whose label byte has bit 7 set
                              //   (`labels` is then the tagged map made by launch_object_weight_tags)
+    int chain_early;         // launch so that the kernel may start while its predecessor on the stream drains
 };
 // Tile map of the logits for the row-walking kernel: fp32 tensor {w, h, S*C}, one box = the block's tile of all
 // classes.  False if the shape does not allow it (w not a multiple of 4, C > 32) or the driver entry point is
@@ -183,6 +185,7 @@ struct UpdateArgs {
     float* vel2;             // [S][n_params]
     double b1, b2, eps, ln_b1, ln_b2;
     const long long* step_base;   // [S] optimisation steps taken before this call
+    int chain_early;         // launch so that the kernel may start while its predecessor on the stream drains
 };
 // step_base[s] += add (add_per_stream == nullptr) or += add_per_stream[s]
 void launch_step_tick(long long* step_base, int S, int add, const int* add_per_stream, cudaStream_t s);
@@ -243,6 +246,7 @@ struct TcBuffers {
     float* w2_partials;   // [S][n_split2][kClassPad][c_last]
     float* b1_partials;   // [S][n_b1part][c_hidden]
     unsigned int* err;    // device word: first wait that gave up (0 = none)
+    int chain_early;      // launch the kernels so that each may start while its predecessor on the stream drains
 };
 // Geometry is fixed by the shapes alone, so scratch can be sized before the plan exists.
 int tc_wgrad_splits(int layer /*1: 3x3, 2: 1x1*/, int c_in, int c_hidden, int h, int w);

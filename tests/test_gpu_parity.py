@@ -101,6 +101,37 @@ def test_confusion_and_miou_bit_exact(C, h, w):
     st.st_destroy(ctx)
 
 
+def test_prefetched_key_frames_equal_plain_ones():
+    """Inputs brought in by st_prefetch_key_frame (the library's copy stream, while the previous key frame trains) give
+    exactly the labels, losses and parameters of the plain calls."""
+    C, c_in, h, w, K = 6, 8, 11, 19, 3
+    theta = si.initial_head_params(c_in, 0, C, 3)
+    frames = [rand_problem(20 + f, c_in, C, h, w) for f in range(3)]
+    pinned = [(torch.from_numpy(f).pin_memory(), torch.from_numpy(T).pin_memory()) for f, T in frames]
+    plain, pre = make_ctx(c_in, 0, C, h, w, theta, lr=0.05, mu=0.9), make_ctx(c_in, 0, C, h, w, theta, lr=0.05, mu=0.9)
+    with pytest.raises(st.StError) as ei:
+        st.st_use_prefetched_key_frame(pre, 0)
+    assert ei.value.status == st.ST_ERR_BAD_STATE
+    st.st_prefetch_key_frame(pre, 0, *pinned[0])
+    for f in range(3):
+        lab_a = torch.empty((4 * h, 4 * w), dtype=torch.uint8, device="cuda")
+        lab_b = torch.empty_like(lab_a)
+        st.st_set_frozen_features(plain, 0, pinned[f][0]); st.st_teacher_labels(plain, 0, pinned[f][1], lab_a)
+        st.st_use_prefetched_key_frame(pre, 0, lab_b)
+        if f + 1 < 3:
+            st.st_prefetch_key_frame(pre, 0, *pinned[f + 1])          # copied while the steps below run
+        la, lb = np.zeros(K, np.float32), np.zeros(K, np.float32)
+        st.st_distill_step(plain, K, la); st.st_distill_step(pre, K, lb)
+        torch.cuda.synchronize()
+        assert torch.equal(lab_a, lab_b)
+        np.testing.assert_array_equal(lab_a.cpu().numpy(), oracle.teacher_labels(frames[f][1]))
+        assert la.tobytes() == lb.tobytes()
+        assert packed(plain).tobytes() == packed(pre).tobytes()
+    with pytest.raises(st.StError):
+        st.st_use_prefetched_key_frame(pre, 0)                         # nothing pending any more
+    st.st_destroy(plain); st.st_destroy(pre)
+
+
 def test_masks_at_odd_addresses_give_the_same_results():
     """Label maps and masks are byte arrays: a view that starts at an odd address (a tensor sliced by one byte) must
     give the same mask, confusion matrix and mean IoU as an aligned buffer."""
