@@ -53,20 +53,25 @@ tc_fwd1x1_kernel(const __grid_constant__ CUtensorMap tmA,   // {K, p, S}  box {6
                  const __grid_constant__ CUtensorMap tmB,   // {K, 32, S} box {64, 32, 1}
                  const float* __restrict__ theta, int64_t n_params, int64_t b_off,
                  float* __restrict__ z, int C, int p, int kblocks, unsigned int* err, const int* __restrict__ skip, int64_t skip_stride,
-                 int a_early)
+                 int a_early, uint32_t spin_limit, uint32_t stall_bytes)
 {
+    // spin_limit / stall_bytes: kSpinLimit and 0 in normal use.  A test of the give-up path lowers the limit and makes
+    // the first barrier expect stall_bytes more than its copies deliver, so that the wait on it runs out: every copy
+    // that was issued still lands, the kernel records where it gave up, writes nothing, frees its tensor memory and
+    // returns.
     extern __shared__ uint8_t smem_raw[];
     uint8_t* smem = align_smem(smem_raw);
     const uint32_t a_base = smem_u32(smem);
     const uint32_t b_base = a_base + kblocks * (kTileM * 128);
     __shared__ __align__(8) uint64_t bars[kMaxKBlocks + 1];
-    __shared__ uint32_t tmem_slot;
+    __shared__ uint32_t tmem_slot, gave_up;
     const int tid = threadIdx.x, warp = tid >> 5;
     const int s = blockIdx.y, pix0 = blockIdx.x * kTileM;
 
     if (warp == 0) tmem_alloc(smem_u32(&tmem_slot), 32);
     if (tid == 0) {
         for (int i = 0; i <= kblocks; ++i) mbar_init(smem_u32(&bars[i]), 1);
+        gave_up = 0;
         fence_barrier_init();
     }
     tc_fence_before_sync();
@@ -79,7 +84,7 @@ tc_fwd1x1_kernel(const __grid_constant__ CUtensorMap tmA,   // {K, p, S}  box {6
     if (a_early && tid == 0) {
         for (int kb = 0; kb < kblocks; ++kb) {
             const uint32_t bar = smem_u32(&bars[kb]);
-            mbar_expect_tx(bar, kTileM * 128 + kClassPad * 128);
+            mbar_expect_tx(bar, kTileM * 128 + kClassPad * 128 + (kb == 0 ? stall_bytes : 0u));
             tma_load_3d(a_base + kb * (kTileM * 128), &tmA, bar, kb * kBlockK, pix0, s);
         }
     }
@@ -97,7 +102,7 @@ tc_fwd1x1_kernel(const __grid_constant__ CUtensorMap tmA,   // {K, p, S}  box {6
         for (int kb = 0; kb < kblocks; ++kb) {
             const uint32_t bar = smem_u32(&bars[kb]);
             if (!a_early) {
-                mbar_expect_tx(bar, kTileM * 128 + kClassPad * 128);
+                mbar_expect_tx(bar, kTileM * 128 + kClassPad * 128 + (kb == 0 ? stall_bytes : 0u));
                 tma_load_3d(a_base + kb * (kTileM * 128), &tmA, bar, kb * kBlockK, pix0, s);
             }
             tma_load_3d(b_base + kb * (kClassPad * 128), &tmB, bar, kb * kBlockK, 0, s);
@@ -105,8 +110,8 @@ tc_fwd1x1_kernel(const __grid_constant__ CUtensorMap tmA,   // {K, p, S}  box {6
     } else if (tid == 32) {
         constexpr uint32_t idesc = instr_desc(kTileM, kClassPad, 0, 0);
         for (int kb = 0; kb < kblocks; ++kb) {
-            ok = mbar_wait(smem_u32(&bars[kb]), 0, err, kWaitFull);
-            if (!ok) break;
+            ok = mbar_wait(smem_u32(&bars[kb]), 0, err, kWaitFull, spin_limit);
+            if (!ok) { gave_up = 1; break; }
             tc_fence_after_sync();
 #pragma unroll
             for (int k = 0; k < 4; ++k) {
@@ -121,6 +126,8 @@ tc_fwd1x1_kernel(const __grid_constant__ CUtensorMap tmA,   // {K, p, S}  box {6
     ok = mbar_wait(done_bar, 0, err, kWaitDone);
     pdl_launch_dependents();     // only the epilogue is left
     tc_fence_after_sync();
+    __syncthreads();
+    if (gave_up) ok = false;     // the issuing thread ran out of patience: nothing was multiplied, nothing is written
     if (ok) {
         float v[32];
         tmem_ld_32x32(tmem + ((uint32_t)(warp * 32) << 16), v);
@@ -841,6 +848,7 @@ struct TcPlan {
     size_t smem_fwd1, smem_fwd1p, smem_wg1, smem_fwd3, smem_wg3, smem_dgrad;
     bool fwd1_persistent;
     int n_sms;
+    bool test_stall;         // test of the give-up path (environment ST_TEST_STALL_FWD1X1=1 when the plan is made)
 };
 
 // blocks per pixel range of the 1x1 weight gradient: one per 128-channel accumulator
@@ -925,6 +933,7 @@ TcPlan* tc_plan_create(const TcBuffers& b, char* err, size_t err_len)
         const int64_t tiles = (int64_t)((P->p + kTileM - 1) / kTileM) * b.S;
         bool use = tiles >= (int64_t)6 * 148;
         if (const char* e = getenv("ST_FWD1X1_PERSISTENT")) { if (e[0] == '0') use = false; else if (e[0] == '1') use = true; }
+        if (const char* e = getenv("ST_TEST_STALL_FWD1X1")) if (e[0] == '1') { P->test_stall = true; use = false; }
         // the one-tile form keeps the whole channel extent of its tile in shared memory: beyond 704 channels it no
         // longer fits, and the persistent form (a ring of eight stages, whatever the channel count) takes over
         if (P->smem_fwd1 > (size_t)227 * 1024) use = true;
@@ -1006,7 +1015,7 @@ int tc_forward(const TcPlan* P, cudaStream_t s, StageTimer* t, const int* skip, 
         const bool a_early = after_update && !b.c_hidden && !skip && !t && fwd1_early_enabled();
         ST_REPEAT(t) launch_early(a_early || b.chain_early, tc_fwd1x1_kernel, dim3(tiles1, b.S), dim3(kThreadsTc), P->smem_fwd1, s,
             P->act_fwd, P->w2_map, b.theta, b.n_params, b.b2_off, b.z, b.C, P->p, P->c_last / kBlockK, b.err, skip, skip_stride,
-            a_early ? 1 : 0);
+            a_early ? 1 : 0, P->test_stall ? (1u << 12) : kSpinLimit, P->test_stall ? 16u : 0u);
     }
     if (t) t->mark("tc_fwd1x1", s, st_repeats(t));
     return n + st_repeats(t);

@@ -40,9 +40,10 @@ __device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity)
     return ok != 0;
 }
 // Bounded wait; on give-up writes `code` (tagged with the block) into *err and returns false.
-__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, unsigned int* err, unsigned int code)
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, unsigned int* err, unsigned int code,
+                                          uint32_t limit = kSpinLimit)
 {
-    for (uint32_t it = 0; it < kSpinLimit; ++it)
+    for (uint32_t it = 0; it < limit; ++it)
         if (mbar_try_wait(bar, parity)) return true;
     atomicCAS(err, 0u, code | (blockIdx.x << 8));
     return false;

@@ -280,3 +280,32 @@ def test_two_layer_forward_with_a_partly_filled_last_round(c_in, ch, h, w):
     dh = st.st_read_tensor(ctx, 0, st.ST_TENSOR_HIDDEN_GRAD)
     assert (dh[hd1 == 0] == 0).all() and (dh[hd1 > 0] != 0).mean() > 0.9
     st.st_destroy(ctx)
+
+
+def test_a_wait_that_runs_out_is_reported_and_nothing_else_breaks(monkeypatch):
+    """Every wait inside the tensor-core kernels is bounded.  A test-only switch makes the forward's first barrier
+    expect 16 bytes more than its copies deliver and shortens the limit: the wait runs out, the kernel records where,
+    writes nothing, frees its tensor memory and returns; the host reports ST_ERR_CUDA at the next call that waits.
+    Nothing faults or hangs, the device stays usable, and a context made without the switch works as ever."""
+    c_in, C, h, w = 64, 5, 9, 13
+    feat, T = problem(12, c_in, C, h, w)
+    theta = si.initial_head_params(c_in, 0, C, 5)
+    monkeypatch.setenv("ST_TEST_STALL_FWD1X1", "1")
+    ctx = make_ctx(c_in, 0, C, h, w, theta, lr=0.05)
+    monkeypatch.delenv("ST_TEST_STALL_FWD1X1")
+    st.st_set_frozen_features(ctx, 0, dev(feat)); st.st_teacher_labels(ctx, 0, dev(T))
+    st.st_distill_step(ctx, 1)
+    with pytest.raises(st.StError) as ei:
+        st.st_read_tensor(ctx, 0, st.ST_TENSOR_LOGITS)
+    assert ei.value.status == st.ST_ERR_CUDA
+    assert "gave up waiting (code 1, block 0)" in str(ei.value)         # code 1: a wait for data to arrive
+    assert (st.st_read_tensor(ctx, 0, st.ST_TENSOR_FEATURES) == oracle.round_bf16(feat).ravel()).all()   # reported once; the context answers
+    st.st_destroy(ctx)
+    good = make_ctx(c_in, 0, C, h, w, theta, lr=0.05)
+    st.st_set_frozen_features(good, 0, dev(feat)); st.st_teacher_labels(good, 0, dev(T))
+    loss = np.zeros(1, np.float32)
+    st.st_distill_step(good, 1, loss)
+    hq = oracle.Head(c_in, 0, C, lr=0.05, theta=theta, quantize_bf16=True)
+    l_ref, _, _ = oracle.gradients(hq, feat, oracle.teacher_labels(T))
+    assert abs(loss[0] - l_ref) <= 2e-5 * abs(l_ref)
+    st.st_destroy(good)
