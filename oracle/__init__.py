@@ -171,6 +171,18 @@ def conv1x1_dgrad(W2: np.ndarray, dz: np.ndarray) -> np.ndarray:
     return dH
 
 
+def conv_dgrad(dout: np.ndarray, W: np.ndarray, c_take: Optional[int] = None) -> np.ndarray:
+    """Gradient with respect to the first `c_take` input channels of a convolution layer (all of them by default)."""
+    dout = _c(dout)
+    W = _c(W, dout.dtype)
+    Cout, Cin, ks, _ = W.shape
+    _, h, w = dout.shape
+    take = Cin if c_take is None else int(c_take)
+    din = np.empty((take, h, w), dtype=dout.dtype)
+    _lib(dout.dtype).so_conv_dgrad(_p(dout), _p(W), _c_int(Cin), _c_int(take), _c_int(Cout), _c_int(h), _c_int(w), _c_int(ks), _p(din))
+    return din
+
+
 def relu_mask_(dH: np.ndarray, Hact: np.ndarray) -> None:
     assert dH.flags.c_contiguous and Hact.flags.c_contiguous and dH.dtype == Hact.dtype
     _lib(dH.dtype).so_relu_mask(_p(dH), _p(Hact), _c_i64(dH.size))
@@ -354,6 +366,139 @@ def pack(head: Head) -> bytes:
 def agreement(labels: np.ndarray, pred: np.ndarray, C: int):
     conf, bad = confusion(labels, pred, C)
     return conf, miou(conf), bad
+
+
+# ----------------------------------------------------------------------------
+# a deeper trainable subset: a stack of student blocks with skip inputs and a freeze boundary inside it
+# ----------------------------------------------------------------------------
+@dataclass
+class StackHead:
+    """The back part of the student as a stack of blocks (Section 5.2: blocks SB5 and SB6, each fed by the block before
+    it and by a feature map of the frozen front part -- SB2's and SB1's -- concatenated to its input, then the
+    classifier), with the freeze boundary of partial distillation (Section 4.2) anywhere inside it.
+
+    The paper's drawing of a student block is not in its text.  Reading taken: block b is a 3x3 convolution with zero
+    padding 1 over concat(previous block's output or the frozen part's output, skip input b) followed by ReLU; all
+    blocks and their skip inputs share the resolution of the frozen part's output (whatever resampling the skip maps
+    need belongs to the frozen part); the classifier is a 1x1 convolution.  Layers before `first_trained` keep their
+    parameters: no gradient is formed for them and none is passed back into them ("the gradient computation can stop
+    in the middle", Section 4.2).  first_trained = 0 trains every block; = len(blocks) trains the classifier alone.
+    """
+    c_in: int
+    blocks: List[Tuple[int, int]]    # per block (output channels, skip-input channels)
+    n_classes: int
+    first_trained: int = 0
+    up: int = 4
+    lr: float = 0.01
+    momentum: float = 0.0
+    dtype: type = np.float32
+    quantize_bf16: bool = False      # test-only: round GEMM operands to bf16 like the tensor-core path
+    theta: np.ndarray = None         # flat parameters of ALL layers, forward order: per layer weight then bias
+    vel: np.ndarray = None
+
+    def shapes(self):
+        out, prev = [], self.c_in
+        for c_out, c_skip in self.blocks:
+            out.append(((c_out, prev + c_skip, 3, 3), (c_out,)))
+            prev = c_out
+        out.append(((self.n_classes, prev, 1, 1), (self.n_classes,)))
+        return out
+
+    def __post_init__(self):
+        n = sum(int(np.prod(ws)) + int(np.prod(bs)) for ws, bs in self.shapes())
+        if self.theta is None:
+            self.theta = np.zeros(n, dtype=self.dtype)
+        self.theta = np.ascontiguousarray(self.theta, dtype=self.dtype).copy()
+        assert self.theta.size == n, (self.theta.size, n)
+        self.vel = np.zeros(n, dtype=self.dtype)
+        assert 0 <= self.first_trained <= len(self.blocks)
+
+    def layers(self):
+        out, off = [], 0
+        for ws, bs in self.shapes():
+            nw, nb = int(np.prod(ws)), int(np.prod(bs))
+            out.append((self.theta[off:off + nw].reshape(ws), self.theta[off + nw:off + nw + nb]))
+            off += nw + nb
+        return out
+
+    def trained_slice(self) -> slice:
+        """Where the trained layers sit in theta (they are the last ones): what UpdatedPart carries."""
+        off = 0
+        for ws, bs in self.shapes()[:self.first_trained]:
+            off += int(np.prod(ws)) + int(np.prod(bs))
+        return slice(off, self.theta.size)
+
+    def _q(self, a):
+        return round_bf16(a) if self.quantize_bf16 else a
+
+
+def stack_forward(head: StackHead, feat: np.ndarray, skips: List[Optional[np.ndarray]]):
+    """(logits [C][h][w], inputs of every block as the convolution saw them, outputs of every block)."""
+    layers = head.layers()
+    prev = head._q(np.ascontiguousarray(feat, dtype=head.dtype))
+    ins, outs = [], []
+    for b, (c_out, c_skip) in enumerate(head.blocks):
+        x = prev if c_skip == 0 else np.concatenate([prev, head._q(np.ascontiguousarray(skips[b], dtype=head.dtype))], axis=0)
+        W, bias = layers[b]
+        prev = head._q(conv_fwd(x, head._q(W), bias, relu=True))
+        ins.append(x); outs.append(prev)
+    Wc, bc = layers[-1]
+    return conv_fwd(prev, head._q(Wc), bc), ins, outs
+
+
+def stack_student_mask(head: StackHead, feat, skips) -> np.ndarray:
+    return teacher_labels(upsample(stack_forward(head, feat, skips)[0], head.up))
+
+
+def stack_gradients(head: StackHead, feat, skips, labels):
+    """Loss, gradient of every parameter (zero for the frozen layers) and the student mask of this forward."""
+    z, ins, outs = stack_forward(head, feat, skips)
+    u = upsample(z, head.up)
+    loss, g, _ = softmax_ce(u, labels)
+    mask = teacher_labels(u)
+    dz = upsample_adjoint(g, head.up)
+    layers = head.layers()
+    B = len(head.blocks)
+    grads = [None] * (B + 1)
+    Wc, _ = layers[-1]
+    last = outs[-1] if B else head._q(np.ascontiguousarray(feat, dtype=head.dtype))
+    dWc, dbc = conv_wgrad(last, head._q(dz), 1)
+    if head.quantize_bf16:
+        dbc = bias_grad(dz)
+    grads[B] = (dWc, dbc)
+    if head.first_trained < B:
+        dH = conv1x1_dgrad(head._q(Wc.reshape(Wc.shape[0], Wc.shape[1])), head._q(dz))
+        relu_mask_(dH, outs[-1])
+        for b in range(B - 1, head.first_trained - 1, -1):
+            W, _ = layers[b]
+            dW, db = conv_wgrad(ins[b], head._q(dH), 3)
+            if head.quantize_bf16:
+                db = bias_grad(dH)
+            grads[b] = (dW, db)
+            if b > head.first_trained:             # pass the gradient on to the block before (its own output channels only)
+                c_prev = head.blocks[b - 1][0]
+                dH = conv_dgrad(head._q(dH), head._q(W), c_prev)
+                relu_mask_(dH, outs[b - 1])
+    flat = []
+    for (ws, bs), gr in zip(head.shapes(), grads):
+        if gr is None:
+            flat += [np.zeros(int(np.prod(ws)), head.dtype), np.zeros(int(np.prod(bs)), head.dtype)]
+        else:
+            flat += [gr[0].ravel(), gr[1].ravel()]
+    return loss, np.concatenate(flat), mask
+
+
+def stack_distill_step(head: StackHead, feat, skips, labels):
+    """One iteration of Algorithm 1's loop on the trained layers (gradient descent with momentum)."""
+    loss, grad, mask = stack_gradients(head, feat, skips, labels)
+    sl = head.trained_slice()
+    sgd_(head.theta[sl], head.vel[sl], grad[sl].astype(head.dtype), head.lr, head.momentum)
+    return loss, mask
+
+
+def stack_pack(head: StackHead) -> bytes:
+    """UpdatedPart(student) (Algorithm 3): the trained layers only, forward order, weight then bias, fp32."""
+    return np.ascontiguousarray(head.theta[head.trained_slice()], dtype="<f4").tobytes()
 
 
 # ----------------------------------------------------------------------------

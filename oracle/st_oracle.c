@@ -292,6 +292,35 @@ void so_conv1x1_dgrad(const real *W2, const real *dz, int C, int Ch, int64_t P, 
         }
 }
 
+/* Gradient passed back through a convolution layer to its input (needed between trained layers only; nothing is
+ * passed back into a frozen layer's output, Section 4.2).  Transpose of so_conv_fwd:
+ *   din[ci][y][x] = sum_{co,ky,kx} dout[co][y - ky + r][x - kx + r] * Wt[co][ci][ky][kx]
+ * (output pixel (yo, xo) read input pixel (yo + ky - r, xo + kx - r), so input pixel (y, x) was read by output pixel
+ * (y - ky + r, x - kx + r); positions outside the map contribute nothing).  Only the first Cin_take input channels
+ * are formed (those of the preceding trained layer when the input is a concatenation). */
+void so_conv_dgrad(const real *dout, const real *Wt, int Cin, int Cin_take, int Cout, int h, int w, int ks, real *din)
+{
+    const int r = ks / 2;
+#pragma omp parallel for
+    for (int ci = 0; ci < Cin_take; ++ci)
+        for (int y = 0; y < h; ++y)
+            for (int x = 0; x < w; ++x) {
+                double acc = 0.0;
+                for (int co = 0; co < Cout; ++co)
+                    for (int ky = 0; ky < ks; ++ky) {
+                        const int yo = y - ky + r;
+                        if (yo < 0 || yo >= h) continue;
+                        for (int kx = 0; kx < ks; ++kx) {
+                            const int xo = x - kx + r;
+                            if (xo < 0 || xo >= w) continue;
+                            acc += (double)dout[((int64_t)co * h + yo) * w + xo] *
+                                   (double)Wt[(((int64_t)co * Cin + ci) * ks + ky) * ks + kx];
+                        }
+                    }
+                din[((int64_t)ci * h + y) * w + x] = (real)acc;
+            }
+}
+
 /* ReLU backward: the gradient passes where the activation is > 0 (0 at exactly 0). */
 void so_relu_mask(real *dH, const real *Hact, int64_t n)
 {
