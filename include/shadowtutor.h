@@ -82,11 +82,29 @@ typedef struct st_head_desc {
     int32_t object_radius;  /* what counts as "near" (the paper gives no distance): within this many rows and
                                columns of a pixel whose label is not the background class; 0..64 */
     int32_t background_class; /* the background class, below n_classes */
+    /* The back part as a stack of student blocks (Section 5.2: the blocks SB5 and SB6, each fed by the block before
+       it and by a feature map of the frozen front part concatenated to its input), with the freeze boundary of partial
+       distillation (Section 4.2) anywhere inside it.  The paper's drawing of a block is not in its text; reading
+       taken: block b = 3x3 convolution with zero padding 1 over the concatenation (channels of the previous block's
+       output, or of the frozen part's output for block 0, first; then the channels of skip input b), followed by ReLU;
+       blocks and skip inputs share the resolution feat_h x feat_w; the classifier is a 1x1 convolution. */
+    int32_t n_blocks;         /* 0: the head given by c_hidden.  1..ST_MAX_BLOCKS: this many blocks, then the classifier
+                                 (c_hidden must be 0, gemm_precision 1) */
+    int32_t block_c_out[2];   /* output channels of each block: multiples of 64, at most 256 */
+    int32_t block_c_skip[2];  /* channels of each block's skip input (0: none): multiples of 64 */
+    int32_t first_trained;    /* blocks before this index keep their parameters: no gradient is formed for them and none
+                                 is passed back into them.  0 trains every block, n_blocks the classifier alone. */
 } st_head_desc;
+#define ST_MAX_BLOCKS 2
 
 /* Number of fp32 values in one head's packed parameter buffer:
  * per layer in forward order, weight [Cout][Cin][kh][kw] then bias [Cout]. */
 ST_API size_t st_param_count(int32_t c_in, int32_t c_hidden, int32_t n_classes);
+
+/* The same for any description: *n_all (may be NULL) = values of all layers of the back part, which st_init_head
+ * takes; *n_trained (may be NULL) = values of the layers behind the freeze boundary, which UpdatedPart carries.  For a
+ * head without blocks both equal st_param_count.  ST_ERR_INVALID_ARG on a NULL or inconsistent description. */
+ST_API st_status st_head_param_counts(const st_head_desc *desc, size_t *n_all, size_t *n_trained);
 
 /*
  * st_init_head — create the server-side copy of the student's trainable part
@@ -110,6 +128,15 @@ ST_API st_status st_init_head(const st_head_desc *desc, const float *init_params
  *   feat_chw  host or device; fp32 [c_in][feat_h][feat_w], contiguous.
  */
 ST_API st_status st_set_frozen_features(st_ctx *ctx, int32_t stream, const float *feat_chw);
+
+/*
+ * st_set_skip_features — cache the skip input of one block for one key frame: the feature map of the frozen front
+ * part that Section 5.2 concatenates to the block's input (SB2's output for SB5, SB1's for SB6), already at the
+ * resolution feat_h x feat_w.  Like the frozen part's output it does not change while the back part is trained.
+ *   block     0 <= block < n_blocks, a block with block_c_skip > 0.
+ *   feat_chw  host or device; fp32 [block_c_skip][feat_h][feat_w], contiguous.
+ */
+ST_API st_status st_set_skip_features(st_ctx *ctx, int32_t stream, int32_t block, const float *feat_chw);
 
 /*
  * st_teacher_labels — pseudo-label of the key frame (Algorithm 3: label <- Forward(teacher)):
@@ -245,9 +272,11 @@ typedef enum st_tensor {
     ST_TENSOR_LOGIT_GRAD = 1,  /* dz, fp32 [C][h][w]: gradient of the mean loss w.r.t. z */
     ST_TENSOR_PARAM_GRAD = 2,  /* fp32, packed order: gradient applied by the last update */
     ST_TENSOR_MOMENTUM = 3,    /* fp32, packed order */
-    ST_TENSOR_HIDDEN = 4,      /* fp32 [c_hidden][h][w]: ReLU output of the 3x3 layer (two-layer head) */
+    ST_TENSOR_HIDDEN = 4,      /* fp32 [c_hidden][h][w]: ReLU output of the 3x3 layer (two-layer head; last block of a stack) */
     ST_TENSOR_HIDDEN_GRAD = 5, /* fp32 [c_hidden][h][w]: gradient w.r.t. the hidden activation (after the ReLU mask) */
-    ST_TENSOR_FEATURES = 6     /* fp32 [c_in][h][w]: the cached features as the GEMMs see them */
+    ST_TENSOR_FEATURES = 6,    /* fp32 [c_in][h][w]: the cached features as the GEMMs see them */
+    ST_TENSOR_HIDDEN_FIRST = 7,      /* a stack of two blocks: output of block 0, fp32 [block_c_out[0]][h][w] */
+    ST_TENSOR_HIDDEN_GRAD_FIRST = 8  /* ... and the gradient with respect to it (after the ReLU mask) */
 } st_tensor;
 
 /*

@@ -32,6 +32,9 @@ ST_TENSOR_MOMENTUM = 3
 ST_TENSOR_HIDDEN = 4
 ST_TENSOR_HIDDEN_GRAD = 5
 ST_TENSOR_FEATURES = 6
+ST_TENSOR_HIDDEN_FIRST = 7
+ST_TENSOR_HIDDEN_GRAD_FIRST = 8
+ST_MAX_BLOCKS = 2
 
 EXPORTED = [
     "st_param_count", "st_init_head", "st_set_frozen_features", "st_teacher_labels", "st_set_labels",
@@ -39,7 +42,7 @@ EXPORTED = [
     "st_launch_count", "st_destroy", "st_last_error", "st_status_name", "st_profile_step",
     "st_agreement_noalloc", "st_train_key_frame", "st_next_stride", "st_client_schedule", "st_throughput_bounds",
     "st_traffic_bounds", "st_choose_max_updates", "st_apply_update", "st_measure_arithmetic_peaks",
-    "st_prefetch_key_frame", "st_use_prefetched_key_frame",
+    "st_prefetch_key_frame", "st_use_prefetched_key_frame", "st_head_param_counts", "st_set_skip_features",
 ]
 ST_NOALLOC_MAX_CLASSES = 64
 ST_MAX_STAGES = 12
@@ -54,6 +57,8 @@ class st_head_desc(ctypes.Structure):
         ("optimizer", ctypes.c_int32), ("adam_beta1", ctypes.c_double), ("adam_beta2", ctypes.c_double),
         ("adam_eps", ctypes.c_double), ("object_weight", ctypes.c_int32), ("object_radius", ctypes.c_int32),
         ("background_class", ctypes.c_int32),
+        ("n_blocks", ctypes.c_int32), ("block_c_out", ctypes.c_int32 * 2), ("block_c_skip", ctypes.c_int32 * 2),
+        ("first_trained", ctypes.c_int32),
     ]
 
 
@@ -79,6 +84,10 @@ def load_library() -> ctypes.CDLL:
     vp, i32, i64 = ctypes.c_void_p, ctypes.c_int32, ctypes.c_int64
     lib.st_param_count.restype = ctypes.c_size_t
     lib.st_param_count.argtypes = [i32, i32, i32]
+    lib.st_head_param_counts.restype = ctypes.c_int
+    lib.st_head_param_counts.argtypes = [ctypes.POINTER(st_head_desc), ctypes.POINTER(ctypes.c_size_t), ctypes.POINTER(ctypes.c_size_t)]
+    lib.st_set_skip_features.restype = ctypes.c_int
+    lib.st_set_skip_features.argtypes = [vp, i32, i32, vp]
     lib.st_init_head.restype = ctypes.c_int
     lib.st_init_head.argtypes = [ctypes.POINTER(st_head_desc), vp, ctypes.POINTER(vp)]
     lib.st_set_frozen_features.restype = ctypes.c_int
@@ -167,7 +176,8 @@ class _Ctx:
         self.S, self.C = desc.n_streams, desc.n_classes
         self.p = desc.feat_h * desc.feat_w
         self.P = self.p * desc.up * desc.up
-        self.n_params = st_param_count(desc.c_in, desc.c_hidden, desc.n_classes)
+        # n_params: the values UpdatedPart carries (the trained layers); n_params_all: every layer of the back part
+        self.n_params_all, self.n_params = st_head_param_counts(desc)
 
     def __del__(self):
         try:
@@ -189,16 +199,33 @@ def st_param_count(c_in: int, c_hidden: int, n_classes: int) -> int:
     return int(load_library().st_param_count(c_in, c_hidden, n_classes))
 
 
+def st_head_param_counts(desc: st_head_desc):
+    """(values of all layers of the back part, values of the trained layers) for a description."""
+    n_all, n_trained = ctypes.c_size_t(0), ctypes.c_size_t(0)
+    _status_only(load_library().st_head_param_counts(ctypes.byref(desc), ctypes.byref(n_all), ctypes.byref(n_trained)),
+                 "st_head_param_counts")
+    return int(n_all.value), int(n_trained.value)
+
+
 def st_init_head(*, n_streams: int = 1, c_in: int, c_hidden: int = 0, n_classes: int, feat_h: int,
                  feat_w: int, up: int = 4, gemm_precision: int = 0, lr: float = 0.01, momentum: float = 0.0,
                  cuda_stream: int = 0, init_params, optimizer: int = 0, adam_beta1: float = 0.0,
                  adam_beta2: float = 0.0, adam_eps: float = 0.0, object_weight: int = 0, object_radius: int = 0,
-                 background_class: int = 0) -> _Ctx:
+                 background_class: int = 0, blocks=(), first_trained: int = 0) -> _Ctx:
+    """`blocks`: (c_out, c_skip) per student block in front of the classifier (at most ST_MAX_BLOCKS); `init_params`
+    holds every layer of the back part, frozen ones included."""
     lib = load_library()
+    if len(blocks) > ST_MAX_BLOCKS:
+        raise ValueError(f"at most {ST_MAX_BLOCKS} blocks")
+    c_out = (ctypes.c_int32 * 2)(*([b[0] for b in blocks] + [0] * (2 - len(blocks))))
+    c_skip = (ctypes.c_int32 * 2)(*([b[1] for b in blocks] + [0] * (2 - len(blocks))))
     desc = st_head_desc(n_streams, c_in, c_hidden, n_classes, feat_h, feat_w, up, gemm_precision,
                         lr, momentum, cuda_stream or None, optimizer, adam_beta1, adam_beta2, adam_eps,
-                        object_weight, object_radius, background_class)
-    n = n_streams * int(lib.st_param_count(c_in, c_hidden, n_classes))
+                        object_weight, object_radius, background_class, len(blocks), c_out, c_skip, first_trained)
+    counts_all, _ = ctypes.c_size_t(0), None
+    if lib.st_head_param_counts(ctypes.byref(desc), ctypes.byref(counts_all), None) != ST_OK:
+        counts_all = ctypes.c_size_t(int(lib.st_param_count(c_in, c_hidden, n_classes)))    # the library reports what is wrong
+    n = n_streams * int(counts_all.value)
     out = ctypes.c_void_p()
     status = lib.st_init_head(ctypes.byref(desc), _ptr(init_params, "float32", n, "init_params"), ctypes.byref(out))
     _check(status, None)
@@ -208,6 +235,11 @@ def st_init_head(*, n_streams: int = 1, c_in: int, c_hidden: int = 0, n_classes:
 def st_set_frozen_features(ctx: _Ctx, stream: int, feat_chw) -> None:
     n = ctx.desc.c_in * ctx.p
     _check(load_library().st_set_frozen_features(ctx.handle, stream, _ptr(feat_chw, "float32", n, "feat_chw")), ctx)
+
+
+def st_set_skip_features(ctx: _Ctx, stream: int, block: int, feat_chw) -> None:
+    n = ctx.desc.block_c_skip[block] * ctx.p if 0 <= block < ST_MAX_BLOCKS else 0
+    _check(load_library().st_set_skip_features(ctx.handle, stream, block, _ptr(feat_chw, "float32", n, "feat_chw")), ctx)
 
 
 def st_teacher_labels(ctx: _Ctx, stream: int, logits_chw, labels_out=None) -> None:

@@ -398,17 +398,29 @@ tc_fwd1x1p_kernel(const __grid_constant__ CUtensorMap tmA,   // {K, p, S}  box {
     if (warp == 0) tmem_dealloc(tmem, 2 * kClassPad);
 }
 
-template <int STAGES>
+// MODE 0: the layer's forward (bias, ReLU, bf16 output, one ReLU bit per output value).
+// MODE 1: the gradient passed back through the layer to the block before it: the same tile walk over the layer's output
+//         gradient with the weights transposed and their taps mirrored (prepared by the update kernel); the epilogue
+//         applies the ReLU mask of the receiving block, writes bf16 and emits per-tile channel sums of the unrounded
+//         values (the receiving block's bias gradient).
+// The K loop runs over 9 taps x (kblocks1 + kblocks2) channel blocks: the first kblocks1 come from tmA (the previous
+// block's output, or the frozen part's), the others from tmA2 (the block's skip input): the concatenation of
+// Section 5.2 is never materialised.
+template <int STAGES, int MODE>
 __global__ void __launch_bounds__(kFwd3Threads)
-tc_fwd3x3_kernel(const __grid_constant__ CUtensorMap tmA,   // {Cin, w, h, S}    box {64, 32, 4, 1}
-                 const __grid_constant__ CUtensorMap tmB,   // {Cin, 9*Ch, S}    box {64, Ch, 1}
+tc_fwd3x3_kernel(const __grid_constant__ CUtensorMap tmA,   // {C1, w, h, S}     box {64, 32, 4, 1}
+                 const __grid_constant__ CUtensorMap tmA2,  // {C2, w, h, S}     box {64, 32, 4, 1} (unused if kblocks2 == 0)
+                 int kblocks1, int kblocks2,
+                 const __grid_constant__ CUtensorMap tmB,   // {C1+C2, 9*Ch, S}  box {64, Ch, 1}
                  const __grid_constant__ CUtensorMap tmBq,  // same tensor, box {64, 64, 1}: one block of 64 output channels
                  int tail_split,                             // the tiles of the last, partly filled round are cut into this many
                                                              // ranges of output channels (1, 2 or 4), one work item each
-                 const float* __restrict__ theta, int64_t n_params, int64_t b_off,
-                 bf16* __restrict__ hidden,                  // [S][p][Ch]
-                 uint32_t* __restrict__ relu_bits,           // [S][p][Ch/32]: bit k of word j = hidden[32j + k] > 0
-                 int Cin, int Ch, int h, int w, int n_tiles_total, int acc_cols, unsigned int* err, const int* __restrict__ skip, int64_t skip_stride)
+                 const float* __restrict__ theta, int64_t n_params, int64_t b_off,   // MODE 0: bias
+                 bf16* __restrict__ out,                     // [S][p][Ch]
+                 uint32_t* __restrict__ relu_bits,           // [S][p][Ch/32]: bit k of word j = out[32j + k] > 0 (MODE 0: written;
+                                                             //   MODE 1: the receiving block's bits, read)
+                 float* __restrict__ b_partials,             // MODE 1: [S][tiles per stream][Ch] channel sums of each tile
+                 int Ch, int h, int w, int n_tiles_total, int acc_cols, unsigned int* err, const int* __restrict__ skip, int64_t skip_stride)
 {
     extern __shared__ uint8_t smem_raw[];
     uint8_t* smem = align_smem(smem_raw);
@@ -416,10 +428,11 @@ tc_fwd3x3_kernel(const __grid_constant__ CUtensorMap tmA,   // {Cin, w, h, S}   
     const uint32_t a_bytes = kTileM * 128, b_bytes = (uint32_t)Ch * 128, stage_bytes = a_bytes + b_bytes;
     __shared__ __align__(8) uint64_t full[STAGES], empty[STAGES], acc_full[2], acc_empty[2];
     __shared__ uint32_t tmem_slot;
+    __shared__ float part[MODE == 1 ? 4 * 256 : 1];             // MODE 1: per-warp channel sums of the tile
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     const int tiles_x = (w + kTileW - 1) / kTileW, tiles_y = (h + kTileH - 1) / kTileH;
     const int tiles_per_stream = tiles_x * tiles_y;
-    const int kblocks = Cin / kBlockK, n_iter = 9 * kblocks;
+    const int kblocks = kblocks1 + kblocks2, n_iter = 9 * kblocks;
     // Work items: whole tiles while every block has one, then the remaining tiles in tail_split pieces each, so that
     // the last round is short instead of leaving most blocks idle for a full tile's time.
     const int n_full = tail_split > 1 ? (n_tiles_total / (int)gridDim.x) * (int)gridDim.x : n_tiles_total;
@@ -453,18 +466,28 @@ tc_fwd3x3_kernel(const __grid_constant__ CUtensorMap tmA,   // {Cin, w, h, S}   
             const int s = im.tile / tiles_per_stream, tt = im.tile % tiles_per_stream;
             if (skip && skip[(int64_t)s * skip_stride]) continue;     // all three roles leave out the same items
             const int x0 = (tt % tiles_x) * kTileW, y0 = (tt / tiles_x) * kTileH;
-            for (int it = 0; it < n_iter; ++it, ++g) {
-                const int st = g % STAGES, tap = it / kblocks, kb = it % kblocks;
-                if (g >= STAGES) ok = mbar_wait(smem_u32(&empty[st]), ((g / STAGES) - 1) & 1, err, kWaitEmpty);
-                if (!ok) break;
-                const uint32_t bar = smem_u32(&full[st]), sa = base + st * stage_bytes;
-                mbar_expect_tx(bar, a_bytes + (uint32_t)im.chn * 128);
-                tma_load_4d(sa, &tmA, bar, kb * kBlockK, x0 + tap % 3 - 1, y0 + tap / 3 - 1, s);
-                if (im.chn == Ch) tma_load_3d(sa + a_bytes, &tmB, bar, kb * kBlockK, tap * Ch, s);
-                else
-                    for (int j = 0; j < im.chn / 64; ++j)        // 64 weight rows per copy, laid out like the single copy
-                        tma_load_3d(sa + a_bytes + j * (64 * 128), &tmBq, bar, kb * kBlockK, tap * Ch + im.ch0 + j * 64, s);
+            // One stage: wait for its slot, then the activation block (from `src`, whose tensor map is fixed at each of
+            // the two places this is expanded: a map chosen at run time costs every copy a slow look-up) and the weights.
+#define ST_FWD3_STAGE(src, a_coord)                                                                                       \
+            {                                                                                                             \
+                const int st = g % STAGES;                                                                                \
+                if (g >= STAGES) ok = mbar_wait(smem_u32(&empty[st]), ((g / STAGES) - 1) & 1, err, kWaitEmpty);          \
+                if (!ok) break;                                                                                           \
+                const uint32_t bar = smem_u32(&full[st]), sa = base + st * stage_bytes;                                   \
+                mbar_expect_tx(bar, a_bytes + (uint32_t)im.chn * 128);                                                    \
+                tma_load_4d(sa, &(src), bar, (a_coord), x0 + tap % 3 - 1, y0 + tap / 3 - 1, s);                          \
+                if (im.chn == Ch) tma_load_3d(sa + a_bytes, &tmB, bar, kb * kBlockK, tap * Ch, s);                        \
+                else                                                                                                      \
+                    for (int j = 0; j < im.chn / 64; ++j)        /* 64 weight rows per copy, laid out like the single copy */ \
+                        tma_load_3d(sa + a_bytes + j * (64 * 128), &tmBq, bar, kb * kBlockK, tap * Ch + im.ch0 + j * 64, s); \
+                ++g;                                                                                                      \
             }
+            for (int tap = 0; tap < 9 && ok; ++tap) {
+                int kb = 0;
+                for (; kb < kblocks1; ++kb) ST_FWD3_STAGE(tmA, kb * kBlockK)
+                for (; kb < kblocks && ok; ++kb) ST_FWD3_STAGE(tmA2, (kb - kblocks1) * kBlockK)
+            }
+#undef ST_FWD3_STAGE
         }
         pdl_launch_dependents();     // every load is issued: the next kernel of the step may set itself up
     } else if (tid == 32) {
@@ -504,36 +527,81 @@ tc_fwd3x3_kernel(const __grid_constant__ CUtensorMap tmA,   // {Cin, w, h, S}   
             const int buf = j & 1;
             const int x = (tt % tiles_x) * kTileW + row % kTileW, y = (tt / tiles_x) * kTileH + row / kTileW;
             ok = mbar_wait(smem_u32(&acc_full[buf]), (j >> 1) & 1, err, kWaitDone);
+            if (MODE == 1) {                                           // the four epilogue warps stay together: they share `part`
+                int all_ok;
+                asm volatile("{\n\t.reg .pred p, q;\n\tsetp.ne.b32 p, %1, 0;\n\tbarrier.cta.red.and.pred q, 1, 128, p;\n\tselp.u32 %0, 1, 0, q;\n\t}"
+                             : "=r"(all_ok) : "r"((int)ok) : "memory");
+                ok = all_ok != 0;
+            }
             if (!ok) break;
             tc_fence_after_sync();
             const bool in = y < h && x < w;
-            const float* bias = theta + (int64_t)s * n_params + b_off;
             const int64_t pixel = (int64_t)s * h * w + (int64_t)y * w + x;
-            bf16* dst = hidden + pixel * Ch + im.ch0;
-            bias += im.ch0;
+            bf16* dst = out + pixel * Ch + im.ch0;
+            const float* bias = theta + (int64_t)s * n_params + b_off + im.ch0;
             for (int n0 = 0; n0 < im.chn; n0 += 32) {
                 float v[32];
                 tmem_ld_32x32(tmem + ((uint32_t)(q * 32) << 16) + buf * acc_cols + n0, v);
-                if (in) {
-                    uint4 out[4];
-                    __nv_bfloat162* o2 = reinterpret_cast<__nv_bfloat162*>(out);
-                    uint32_t bits = 0;
+                if (MODE == 0) {
+                    if (in) {
+                        uint4 o4[4];
+                        __nv_bfloat162* o2 = reinterpret_cast<__nv_bfloat162*>(o4);
+                        uint32_t bits = 0;
 #pragma unroll
-                    for (int k = 0; k < 16; ++k) {
-                        const float a = fmaxf(v[2 * k] + __ldg(bias + n0 + 2 * k), 0.f), b = fmaxf(v[2 * k + 1] + __ldg(bias + n0 + 2 * k + 1), 0.f);
-                        o2[k] = __floats2bfloat162_rn(a, b);
-                        // the mask is taken on the stored (rounded) activation, the value the next layer sees
-                        bits |= (__low2float(o2[k]) > 0.f ? 1u : 0u) << (2 * k);
-                        bits |= (__high2float(o2[k]) > 0.f ? 1u : 0u) << (2 * k + 1);
+                        for (int k = 0; k < 16; ++k) {
+                            const float a = fmaxf(v[2 * k] + __ldg(bias + n0 + 2 * k), 0.f), b = fmaxf(v[2 * k + 1] + __ldg(bias + n0 + 2 * k + 1), 0.f);
+                            o2[k] = __floats2bfloat162_rn(a, b);
+                            // the mask is taken on the stored (rounded) activation, the value the next layer sees
+                            bits |= (__low2float(o2[k]) > 0.f ? 1u : 0u) << (2 * k);
+                            bits |= (__high2float(o2[k]) > 0.f ? 1u : 0u) << (2 * k + 1);
+                        }
+                        store_256(dst + n0, reinterpret_cast<const uint32_t*>(o4));            // 32 channels = 64 bytes
+                        store_256(dst + n0 + 16, reinterpret_cast<const uint32_t*>(o4) + 8);
+                        relu_bits[pixel * (Ch / 32) + (im.ch0 + n0) / 32] = bits;
                     }
-                    store_256(dst + n0, reinterpret_cast<const uint32_t*>(out));            // 32 channels = 64 bytes
-                    store_256(dst + n0 + 16, reinterpret_cast<const uint32_t*>(out) + 8);
-                    relu_bits[pixel * (Ch / 32) + (im.ch0 + n0) / 32] = bits;
+                } else {
+                    if (in) {
+                        const uint32_t bits = __ldg(relu_bits + pixel * (Ch / 32) + (im.ch0 + n0) / 32);
+                        uint4 o4[4];
+                        __nv_bfloat162* o2 = reinterpret_cast<__nv_bfloat162*>(o4);
+#pragma unroll
+                        for (int k = 0; k < 16; ++k) {
+                            if (!((bits >> (2 * k)) & 1u)) v[2 * k] = 0.f;
+                            if (!((bits >> (2 * k + 1)) & 1u)) v[2 * k + 1] = 0.f;
+                            o2[k] = __floats2bfloat162_rn(v[2 * k], v[2 * k + 1]);
+                        }
+                        store_256(dst + n0, reinterpret_cast<const uint32_t*>(o4));
+                        store_256(dst + n0 + 16, reinterpret_cast<const uint32_t*>(o4) + 8);
+                    } else {
+#pragma unroll
+                        for (int k = 0; k < 32; ++k) v[k] = 0.f;
+                    }
+                    // sums over the warp's 32 pixels in a fixed order: a reduce-scatter over the lanes, after which lane c
+                    // holds the sum of channel n0 + c
+#pragma unroll
+                    for (int half = 16; half >= 1; half >>= 1) {
+                        const bool up = (lane & half) != 0;
+#pragma unroll
+                        for (int k = 0; k < half; ++k) {
+                            const float keep = up ? v[k + half] : v[k];
+                            const float send = up ? v[k] : v[k + half];
+                            v[k] = keep + __shfl_xor_sync(0xffffffffu, send, half);
+                        }
+                    }
+                    part[q * 256 + n0 + lane] = v[0];
                 }
             }
             tc_fence_before_sync();
             __syncwarp();
             if (lane == 0) mbar_arrive(smem_u32(&acc_empty[buf]));     // this warp's quarter of the accumulator is free
+            if (MODE == 1) {
+                asm volatile("barrier.cta.sync 1, 128;" ::: "memory");
+                const int e = (warp - 2) * 32 + lane;                  // 0..127 over the four epilogue warps
+                for (int k = e; k < im.chn; k += 128)
+                    b_partials[((int64_t)s * tiles_per_stream + tt) * Ch + im.ch0 + k] =
+                        (part[k] + part[256 + k]) + (part[512 + k] + part[768 + k]);
+                asm volatile("barrier.cta.sync 1, 128;" ::: "memory");
+            }
             ++j;
         }
     }
@@ -551,12 +619,15 @@ tc_fwd3x3_kernel(const __grid_constant__ CUtensorMap tmA,   // {Cin, w, h, S}   
 // ------------------------------------------------------------------------------------------------
 template <int STAGES>
 __global__ void __launch_bounds__(kThreadsTc)
-tc_wgrad3x3_kernel(const __grid_constant__ CUtensorMap tmA,   // X   {Cin, w, h, S} box {64, 32, 2, 1}
+tc_wgrad3x3_kernel(const __grid_constant__ CUtensorMap tmA,   // previous output {C1, w, h, S} box {64, 32, 2, 1}
+                   const __grid_constant__ CUtensorMap tmA2,  // skip input      {C2, w, h, S} box {64, 32, 2, 1} (unused if C2 == 0)
+                   int blocks1,                                // C1 / 64: input-channel blocks that come from tmA
                    const __grid_constant__ CUtensorMap tmB,   // dHd {Ch,  w, h, S} box {64, 32, 2, 1}
                    float* __restrict__ partials,              // [S][n_split][9][Ch][Cin]
                    int Cin, int Ch, int h, int w, int n_chunks, int chunks_per_block, int n_split,
                    int tmem_cols, unsigned int* err, const int* __restrict__ skip, int64_t skip_stride)
 {
+    // Cin = C1 + C2: the layer's input is the concatenation (previous output, skip input), read from its two sources
     extern __shared__ uint8_t smem_raw[];
     uint8_t* smem = align_smem(smem_raw);
     const uint32_t base = smem_u32(smem);
@@ -598,8 +669,14 @@ tc_wgrad3x3_kernel(const __grid_constant__ CUtensorMap tmA,   // X   {Cin, w, h,
             const int x0 = (i % chunks_x) * kChunkW, y0 = (i / chunks_x) * kChunkH;
             const uint32_t bar = smem_u32(&full[st]), sa = base + st * stage_bytes;
             mbar_expect_tx(bar, stage_bytes);
-            for (int cb = 0; cb < a_blocks; ++cb)
+            // blocks past the last channel arrive as zeros (out-of-range fill); two loops, each with its own tensor map
+            // (a map chosen at run time costs every copy a slow look-up)
+            const int n_first = blocks1 * kBlockK == Cin ? a_blocks : blocks1;
+            int cb = 0;
+            for (; cb < n_first; ++cb)
                 tma_load_4d(sa + cb * blk_bytes, &tmA, bar, cb * kBlockK, x0 + tap % 3 - 1, y0 + tap / 3 - 1, s);
+            for (; cb < a_blocks; ++cb)
+                tma_load_4d(sa + cb * blk_bytes, &tmA2, bar, (cb - blocks1) * kBlockK, x0 + tap % 3 - 1, y0 + tap / 3 - 1, s);
             for (int cb = 0; cb < b_blocks; ++cb)
                 tma_load_4d(sa + a_bytes + cb * blk_bytes, &tmB, bar, cb * kBlockK, x0, y0, s);
         }
@@ -831,6 +908,17 @@ bool encode_tensor_map(CUtensorMap* m, CUtensorMapDataType dtype, CUtensorMapSwi
     return true;
 }
 
+struct TcBlockPlan {
+    CUtensorMap in_fwd, skip_fwd;    // the block's two inputs {C, w, h, S}, box {64, 32, 4, 1} (forward tiles)
+    CUtensorMap in_wg, skip_wg;      // same tensors, box {64, 32, 2, 1} (weight-gradient chunks)
+    CUtensorMap w_map, w_map_q;      // {c_tot, 9*c_out, S}, boxes {64, c_out, 1} and {64, 64, 1}
+    CUtensorMap wt_map, wt_map_q;    // mirrored, transposed weights {c_out, 9*c_prev, S}, boxes {64, c_prev, 1} and {64, 64, 1}
+    CUtensorMap dout_fwd;            // the block's output gradient {c_out, w, h, S}, box {64, 32, 4, 1} (A operand when passed back)
+    CUtensorMap dout_wg;             // same tensor, box {64, 32, 2, 1} (B operand of the weight gradient)
+    int cols_wg;                     // tensor-memory columns of the weight gradient
+    size_t smem_fwd, smem_back, smem_wg;
+};
+
 struct TcPlan {
     TcBuffers b;
     int p, p_pad, c_last;
@@ -838,14 +926,10 @@ struct TcPlan {
     CUtensorMap act_wg;      // same tensor, box {64, 64, 1}
     CUtensorMap w2_map;      // {c_last, 32, S} box {64, 32, 1}
     CUtensorMap dz_map;      // {p, 32, S} box {64, 32, 1}
-    CUtensorMap x_fwd3;      // {Cin, w, h, S} box {64, 32, 4, 1}
-    CUtensorMap x_wg3;       // box {64, 32, 2, 1}
-    CUtensorMap w1_map;      // {Cin, 9*Ch, S} box {64, Ch, 1}
-    CUtensorMap w1_map_q;    // same tensor, box {64, 64, 1}
-    CUtensorMap dh_wg3;      // {Ch, w, h, S} box {64, 32, 2, 1}
+    TcBlockPlan blk[kMaxBlocks];
     int split2, chunks2, per2, cols2, msplit2;
-    int split1, chunks1, per1, cols1;
-    size_t smem_fwd1, smem_fwd1p, smem_wg1, smem_fwd3, smem_wg3, smem_dgrad;
+    int split1, chunks1, per1;          // pixel chunks of the 3x3 weight gradients (the same for every block)
+    size_t smem_fwd1, smem_fwd1p, smem_wg1, smem_dgrad;
     bool fwd1_persistent;
     int n_sms;
     bool test_stall;         // test of the give-up path (environment ST_TEST_STALL_FWD1X1=1 when the plan is made)
@@ -854,12 +938,11 @@ struct TcPlan {
 // blocks per pixel range of the 1x1 weight gradient: one per 128-channel accumulator
 static int wgrad1x1_m_split(int c_last) { const int m = (c_last + kTileM - 1) / kTileM; return m < 1 ? 1 : m; }
 
-int tc_wgrad_splits(int layer, int c_in, int c_hidden, int h, int w)
+int tc_wgrad_splits(int layer, int c_last, int h, int w)
 {
     int per, n;
     if (layer == 2) {
         const int64_t p = (int64_t)h * w;
-        const int c_last = c_hidden ? c_hidden : c_in;
         split_geometry((int)((p + kChunkPix - 1) / kChunkPix), 148 / wgrad1x1_m_split(c_last), &per, &n);
     } else {
         const int chunks = ((w + kChunkW - 1) / kChunkW) * ((h + kChunkH - 1) / kChunkH);
@@ -869,6 +952,8 @@ int tc_wgrad_splits(int layer, int c_in, int c_hidden, int h, int w)
 }
 
 int tc_b1_partials(int h, int w) { return (int)(((int64_t)h * w + kTileM - 1) / kTileM); }
+
+int tc_tile3_count(int h, int w) { return ((w + kTileW - 1) / kTileW) * ((h + kTileH - 1) / kTileH); }
 
 int tc_dz_pitch(int h, int w) { return (int)((((int64_t)h * w + 63) / 64) * 64); }
 
@@ -883,9 +968,10 @@ TcPlan* tc_plan_create(const TcBuffers& b, char* err, size_t err_len)
         cudaGetDevice(&dev);
         if (cudaDeviceGetAttribute(&P->n_sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || P->n_sms < 1) P->n_sms = 148;
     }
-    P->c_last = b.c_hidden ? b.c_hidden : b.c_in;
+    const int nb = b.n_blocks;
+    P->c_last = nb ? b.blk[nb - 1].c_out : b.c_in;
     const uint64_t S = (uint64_t)b.S, p = (uint64_t)P->p, cl = (uint64_t)P->c_last;
-    const bf16* act = b.c_hidden ? b.hidden : b.x;
+    const bf16* act = nb ? b.blk[nb - 1].out : b.x;
     bool ok = true;
     {
         uint64_t dims[3] = {cl, p, S}, str[2] = {cl * 2, p * cl * 2};
@@ -903,19 +989,49 @@ TcPlan* tc_plan_create(const TcBuffers& b, char* err, size_t err_len)
         uint32_t box[3] = {64, (uint32_t)kClassPad, 1};
         ok = make_map(&P->dz_map, b.dz_bf16, 3, dims, str, box, err, err_len, "logit gradient");
     }
-    if (ok && b.c_hidden) {
-        const uint64_t ci = (uint64_t)b.c_in, ch = (uint64_t)b.c_hidden, w = (uint64_t)b.w, h = (uint64_t)b.h;
-        uint64_t dx[4] = {ci, w, h, S}, sx[3] = {ci * 2, w * ci * 2, h * w * ci * 2};
-        uint32_t bf[4] = {64, (uint32_t)kTileW, (uint32_t)kTileH, 1}, bw[4] = {64, (uint32_t)kChunkW, (uint32_t)kChunkH, 1};
-        ok = ok && make_map(&P->x_fwd3, b.x, 4, dx, sx, bf, err, err_len, "features (3x3 forward)");
-        ok = ok && make_map(&P->x_wg3, b.x, 4, dx, sx, bw, err, err_len, "features (3x3 wgrad)");
-        uint64_t dh[4] = {ch, w, h, S}, sh[3] = {ch * 2, w * ch * 2, h * w * ch * 2};
-        ok = ok && make_map(&P->dh_wg3, b.dhidden, 4, dh, sh, bw, err, err_len, "hidden gradient");
-        uint64_t dw[3] = {ci, 9 * ch, S}, sw[2] = {ci * 2, 9 * ch * ci * 2};
-        uint32_t bwt[3] = {64, (uint32_t)b.c_hidden, 1};
-        ok = ok && make_map(&P->w1_map, b.w1, 3, dw, sw, bwt, err, err_len, "3x3 weight");
-        uint32_t bwq[3] = {64, 64, 1};
-        ok = ok && make_map(&P->w1_map_q, b.w1, 3, dw, sw, bwq, err, err_len, "3x3 weight (64 rows)");
+    const size_t lim = 227 * 1024;
+    for (int i = 0; ok && i < nb; ++i) {
+        const TcBlock& k = b.blk[i];
+        TcBlockPlan& q = P->blk[i];
+        const uint64_t w = (uint64_t)b.w, h = (uint64_t)b.h, c1 = (uint64_t)k.c_prev, c2 = (uint64_t)k.c_skip, co = (uint64_t)k.c_out,
+                       ct = c1 + c2;
+        const uint32_t bf[4] = {64, (uint32_t)kTileW, (uint32_t)kTileH, 1}, bw[4] = {64, (uint32_t)kChunkW, (uint32_t)kChunkH, 1};
+        auto act_maps = [&](const bf16* base, uint64_t c, CUtensorMap* fwd, CUtensorMap* wg, const char* what) {
+            uint64_t d[4] = {c, w, h, S}, st[3] = {c * 2, w * c * 2, h * w * c * 2};
+            bool r = true;
+            if (fwd) r = r && make_map(fwd, base, 4, d, st, bf, err, err_len, what);
+            if (wg) r = r && make_map(wg, base, 4, d, st, bw, err, err_len, what);
+            return r;
+        };
+        ok = ok && act_maps(k.in_prev, c1, &q.in_fwd, &q.in_wg, "block input");
+        if (c2) ok = ok && act_maps(k.in_skip, c2, &q.skip_fwd, &q.skip_wg, "skip input");
+        else { q.skip_fwd = q.in_fwd; q.skip_wg = q.in_wg; }
+        ok = ok && act_maps(k.dout, co, &q.dout_fwd, &q.dout_wg, "block output gradient");
+        {
+            uint64_t dw[3] = {ct, 9 * co, S}, sw[2] = {ct * 2, 9 * co * ct * 2};
+            uint32_t bwt[3] = {64, (uint32_t)co, 1}, bwq[3] = {64, 64, 1};
+            ok = ok && make_map(&q.w_map, k.w, 3, dw, sw, bwt, err, err_len, "3x3 weight");
+            ok = ok && make_map(&q.w_map_q, k.w, 3, dw, sw, bwq, err, err_len, "3x3 weight (64 rows)");
+        }
+        if (ok && k.pass_back) {
+            uint64_t dw[3] = {co, 9 * c1, S}, sw[2] = {co * 2, 9 * c1 * co * 2};
+            uint32_t bwt[3] = {64, (uint32_t)c1, 1}, bwq[3] = {64, 64, 1};
+            ok = ok && make_map(&q.wt_map, k.w_t, 3, dw, sw, bwt, err, err_len, "3x3 weight, transposed");
+            ok = ok && make_map(&q.wt_map_q, k.w_t, 3, dw, sw, bwq, err, err_len, "3x3 weight, transposed (64 rows)");
+        }
+        const int m_in = ((int)ct + kTileM - 1) / kTileM;
+        q.cols_wg = pow2_cols(m_in * k.c_out);
+        q.smem_fwd = 4 * ((size_t)kTileM * 128 + (size_t)k.c_out * 128) + kSmemAlign;
+        q.smem_back = 4 * ((size_t)kTileM * 128 + (size_t)k.c_prev * 128) + kSmemAlign;
+        q.smem_wg = 3 * ((size_t)(m_in * 2 + k.c_out / kBlockK) * kChunkPix * 128) + kSmemAlign;
+        if (ok && q.cols_wg > 512) {
+            snprintf(err, err_len, "a block with %d input and %d output channels needs %d TMEM columns (> 512)", (int)ct, k.c_out, q.cols_wg);
+            ok = false;
+        }
+        if (ok && (q.smem_fwd > lim || q.smem_wg > lim || (k.pass_back && (q.smem_back > lim || k.c_prev > 256)))) {
+            snprintf(err, err_len, "shared memory per block exceeds 227 KB for these channel counts");
+            ok = false;
+        }
     }
     if (!ok) { delete P; return nullptr; }
 
@@ -940,33 +1056,39 @@ TcPlan* tc_plan_create(const TcBuffers& b, char* err, size_t err_len)
         P->fwd1_persistent = use && P->smem_fwd1p <= (size_t)227 * 1024;
     }
     P->smem_wg1 = kWg1Stages * ((size_t)(m_last / P->msplit2) * 2 * kChunkPix * 128 + kClassPad * 128) + kSmemAlign;
-    if (b.c_hidden) {
-        const int m_in = (b.c_in + kTileM - 1) / kTileM;
+    size_t smem_fwd3 = 0, smem_back3 = 0, smem_wg3 = 0;
+    if (nb) {
         P->chunks1 = ((b.w + kChunkW - 1) / kChunkW) * ((b.h + kChunkH - 1) / kChunkH);
         split_geometry(P->chunks1, 148 / 9, &P->per1, &P->split1);
-        P->cols1 = pow2_cols(m_in * b.c_hidden);
-        P->smem_fwd3 = 4 * ((size_t)kTileM * 128 + (size_t)b.c_hidden * 128) + kSmemAlign;
-        P->smem_wg3 = 3 * ((size_t)(m_in * 2 + b.c_hidden / kBlockK) * kChunkPix * 128) + kSmemAlign;
-        P->smem_dgrad = (size_t)(2 + b.c_hidden / kBlockK) * kClassPad * 128 + kSmemAlign;
-        if (P->cols1 > 512) {
-            snprintf(err, err_len, "c_in %d with c_hidden %d needs %d TMEM columns (> 512)", b.c_in, b.c_hidden, P->cols1);
-            delete P; return nullptr;
+        P->smem_dgrad = (size_t)(2 + P->c_last / kBlockK) * kClassPad * 128 + kSmemAlign;
+        for (int i = 0; i < nb; ++i) {
+            if (P->blk[i].smem_fwd > smem_fwd3) smem_fwd3 = P->blk[i].smem_fwd;
+            if (b.blk[i].pass_back && P->blk[i].smem_back > smem_back3) smem_back3 = P->blk[i].smem_back;
+            if (P->blk[i].smem_wg > smem_wg3) smem_wg3 = P->blk[i].smem_wg;
         }
     }
-    const size_t lim = 227 * 1024;
-    if (P->c_last / kBlockK > kMaxKBlocks || (!P->fwd1_persistent && P->smem_fwd1 > lim) || P->smem_wg1 > lim || P->smem_fwd3 > lim ||
-        P->smem_wg3 > lim || P->smem_dgrad > lim) {
+    if (P->c_last / kBlockK > kMaxKBlocks || (!P->fwd1_persistent && P->smem_fwd1 > lim) || P->smem_wg1 > lim || P->smem_dgrad > lim) {
         snprintf(err, err_len, "shared memory per block exceeds 227 KB for these channel counts");
         delete P; return nullptr;
     }
+    // Raise a kernel's shared-memory allowance to what this plan launches it with, never lower it: the attribute belongs
+    // to the function, not to a plan, and an earlier plan with larger layers may still be in use.
+    auto allow = [&](const void* fn, size_t need) -> cudaError_t {
+        cudaFuncAttributes at;
+        cudaError_t r = cudaFuncGetAttributes(&at, fn);
+        if (r != cudaSuccess) return r;
+        if (need <= (size_t)at.maxDynamicSharedSizeBytes) return cudaSuccess;
+        return cudaFuncSetAttribute(fn, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)need);
+    };
     cudaError_t e = cudaSuccess;
-    if (!P->fwd1_persistent) e = cudaFuncSetAttribute(tc_fwd1x1_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)P->smem_fwd1);
-    if (e == cudaSuccess && P->fwd1_persistent) e = cudaFuncSetAttribute(tc_fwd1x1p_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)P->smem_fwd1p);
-    if (e == cudaSuccess) e = cudaFuncSetAttribute(tc_wgrad1x1_kernel<kWg1Stages>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)P->smem_wg1);
-    if (b.c_hidden) {
-        if (e == cudaSuccess) e = cudaFuncSetAttribute(tc_fwd3x3_kernel<4>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)P->smem_fwd3);
-        if (e == cudaSuccess) e = cudaFuncSetAttribute(tc_wgrad3x3_kernel<3>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)P->smem_wg3);
-        if (e == cudaSuccess) e = cudaFuncSetAttribute(tc_dgrad_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)P->smem_dgrad);
+    if (!P->fwd1_persistent) e = allow((const void*)tc_fwd1x1_kernel, P->smem_fwd1);
+    if (e == cudaSuccess && P->fwd1_persistent) e = allow((const void*)tc_fwd1x1p_kernel, P->smem_fwd1p);
+    if (e == cudaSuccess) e = allow((const void*)tc_wgrad1x1_kernel<kWg1Stages>, P->smem_wg1);
+    if (nb) {
+        if (e == cudaSuccess) e = allow((const void*)tc_fwd3x3_kernel<4, 0>, smem_fwd3);
+        if (e == cudaSuccess && smem_back3) e = allow((const void*)tc_fwd3x3_kernel<4, 1>, smem_back3);
+        if (e == cudaSuccess) e = allow((const void*)tc_wgrad3x3_kernel<3>, smem_wg3);
+        if (e == cudaSuccess) e = allow((const void*)tc_dgrad_kernel, P->smem_dgrad);
     }
     if (e != cudaSuccess) { snprintf(err, err_len, "shared-memory attribute: %s", cudaGetErrorString(e)); delete P; return nullptr; }
     return P;
@@ -980,28 +1102,46 @@ static bool fwd1_early_enabled()     // ST_FWD1_EARLY=0 switches the early activ
     return on;
 }
 
-int tc_forward(const TcPlan* P, cudaStream_t s, StageTimer* t, const int* skip, int64_t skip_stride, bool after_update)
+static const char* const kFwd3Names[kMaxBlocks] = {"tc_fwd3x3", "tc_fwd3x3#2"};
+static const char* const kWg3Names[kMaxBlocks] = {"tc_wgrad3x3", "tc_wgrad3x3#2"};
+
+// the tile walk of a 3x3 layer over `total` tiles: grid size and how the tiles of a partly filled last round are cut
+static void tile_walk(const TcPlan* P, int total, int n_out, int* grid, int* tail_split)
+{
+    *grid = total < P->n_sms ? total : P->n_sms;
+    // the tiles of a partly filled last round are cut into 4 or 2 ranges of output channels if that lets every
+    // piece have its own block (pieces are multiples of 64 channels)
+    const int tail = total > *grid ? total % *grid : 0;
+    *tail_split = 1;
+    if (tail > 0) {
+        if (n_out % 256 == 0 && tail * 4 <= *grid) *tail_split = 4;
+        else if (n_out % 128 == 0 && tail * 2 <= *grid) *tail_split = 2;
+    }
+}
+
+int tc_forward_blocks(const TcPlan* P, int first, int last, cudaStream_t s, StageTimer* t, const int* skip, int64_t skip_stride)
 {
     const TcBuffers& b = P->b;
     int n = 0;
-    if (b.c_hidden) {
-        const int tiles = ((b.w + kTileW - 1) / kTileW) * ((b.h + kTileH - 1) / kTileH);
-        const int total = tiles * b.S;
-        const int grid = total < P->n_sms ? total : P->n_sms;
-        // the tiles of a partly filled last round are cut into 4 or 2 ranges of output channels if that lets every
-        // piece have its own block (pieces are multiples of 64 channels)
-        const int tail = total > grid ? total % grid : 0;
-        int tail_split = 1;
-        if (tail > 0) {
-            if (b.c_hidden % 256 == 0 && tail * 4 <= grid) tail_split = 4;
-            else if (b.c_hidden % 128 == 0 && tail * 2 <= grid) tail_split = 2;
-        }
-        ST_REPEAT(t) launch_chain(b.chain_early != 0, tc_fwd3x3_kernel<4>, dim3(grid), dim3(kFwd3Threads), P->smem_fwd3, s,
-            P->x_fwd3, P->w1_map, P->w1_map_q, tail_split, b.theta, b.n_params, b.b1_off, b.hidden, b.relu_bits, b.c_in, b.c_hidden, b.h, b.w,
-            total, pow2_cols(b.c_hidden), b.err, skip, skip_stride);
-        if (t) t->mark("tc_fwd3x3", s, st_repeats(t));
+    const int total = tc_tile3_count(b.h, b.w) * b.S;
+    for (int i = first; i < last; ++i) {
+        const TcBlock& k = b.blk[i];
+        const TcBlockPlan& q = P->blk[i];
+        int grid, tail_split;
+        tile_walk(P, total, k.c_out, &grid, &tail_split);
+        ST_REPEAT(t) launch_chain(b.chain_early != 0, tc_fwd3x3_kernel<4, 0>, dim3(grid), dim3(kFwd3Threads), q.smem_fwd, s,
+            q.in_fwd, q.skip_fwd, k.c_prev / kBlockK, k.c_skip / kBlockK, q.w_map, q.w_map_q, tail_split, b.theta, b.n_params, k.b_off,
+            k.out, k.relu_bits, (float*)nullptr, k.c_out, b.h, b.w, total, pow2_cols(k.c_out), b.err, skip, skip_stride);
+        if (t) t->mark(kFwd3Names[i], s, st_repeats(t));
         n += st_repeats(t);
     }
+    return n;
+}
+
+int tc_forward(const TcPlan* P, cudaStream_t s, StageTimer* t, const int* skip, int64_t skip_stride, bool after_update, int first_block)
+{
+    const TcBuffers& b = P->b;
+    int n = tc_forward_blocks(P, first_block, b.n_blocks, s, t, skip, skip_stride);
     const int tiles1 = (P->p + kTileM - 1) / kTileM;
     if (P->fwd1_persistent) {
         int gx = P->n_sms / b.S;
@@ -1012,7 +1152,7 @@ int tc_forward(const TcPlan* P, cudaStream_t s, StageTimer* t, const int* skip, 
     } else {
         // one-layer head, no per-stream skip flags to wait for, not a timing run: the activations are the frozen
         // features, which no kernel of the loop writes
-        const bool a_early = after_update && !b.c_hidden && !skip && !t && fwd1_early_enabled();
+        const bool a_early = after_update && !b.n_blocks && !skip && !t && fwd1_early_enabled();
         ST_REPEAT(t) launch_early(a_early || b.chain_early, tc_fwd1x1_kernel, dim3(tiles1, b.S), dim3(kThreadsTc), P->smem_fwd1, s,
             P->act_fwd, P->w2_map, b.theta, b.n_params, b.b2_off, b.z, b.C, P->p, P->c_last / kBlockK, b.err, skip, skip_stride,
             a_early ? 1 : 0, P->test_stall ? (1u << 12) : kSpinLimit, P->test_stall ? 16u : 0u);
@@ -1026,22 +1166,43 @@ int tc_backward(const TcPlan* P, cudaStream_t s, StageTimer* t, const int* skip,
     const TcBuffers& b = P->b;
     int n = 0;
     // one-layer head: the activations are the frozen features, which no kernel of the loop writes
-    const int a_early = (!b.c_hidden && !skip && !t && b.chain_early) ? 1 : 0;
+    const int a_early = (!b.n_blocks && !skip && !t && b.chain_early) ? 1 : 0;
     ST_REPEAT(t) launch_chain(b.chain_early != 0, tc_wgrad1x1_kernel<kWg1Stages>, dim3(P->split2 * P->msplit2, b.S), dim3(kThreadsTc), P->smem_wg1, s,
         P->act_wg, P->dz_map, b.w2_partials, P->c_last, P->chunks2, P->per2, P->msplit2, P->cols2, b.err, skip, skip_stride, a_early);
     if (t) t->mark("tc_wgrad1x1", s, st_repeats(t));
     n += st_repeats(t);
-    if (b.c_hidden) {
+    const int nb = b.n_blocks;
+    if (!nb || !b.blk[nb - 1].trained) return n;          // nothing is passed back into a frozen block (Section 4.2)
+    {
+        const TcBlock& k = b.blk[nb - 1];
         const int blocks = tc_b1_partials(b.h, b.w);
-        const int n_ch_split = (b.c_hidden % 128 == 0) ? 2 : 1;      // each block: a multiple of 64 channels (four ways measured no better)
+        const int n_ch_split = (k.c_out % 128 == 0) ? 2 : 1;      // each block: a multiple of 64 channels (four ways measured no better)
         ST_REPEAT(t) launch_chain(b.chain_early != 0, tc_dgrad_kernel, dim3(blocks, b.S, n_ch_split), dim3(kThreadsTc), P->smem_dgrad, s,
-            P->dz_map, P->w2_map, b.relu_bits, b.dhidden, b.b1_partials, b.c_hidden, P->p, pow2_cols(b.c_hidden / n_ch_split), b.err, skip, skip_stride);
+            P->dz_map, P->w2_map, k.relu_bits, k.dout, k.b_partials, k.c_out, P->p, pow2_cols(k.c_out / n_ch_split), b.err, skip, skip_stride);
         if (t) t->mark("tc_dgrad", s, st_repeats(t));
-        ST_REPEAT(t) launch_chain(b.chain_early != 0, tc_wgrad3x3_kernel<3>, dim3(9 * P->split1, b.S), dim3(kThreadsTc), P->smem_wg3, s,
-            P->x_wg3, P->dh_wg3, b.w1_partials, b.c_in, b.c_hidden, b.h, b.w, P->chunks1, P->per1, P->split1,
-            P->cols1, b.err, skip, skip_stride);
-        if (t) t->mark("tc_wgrad3x3", s, st_repeats(t));
-        n += 2 * st_repeats(t);
+        n += st_repeats(t);
+    }
+    const int total = tc_tile3_count(b.h, b.w) * b.S;
+    for (int i = nb - 1; i >= 0 && b.blk[i].trained; --i) {
+        const TcBlock& k = b.blk[i];
+        const TcBlockPlan& q = P->blk[i];
+        ST_REPEAT(t) launch_chain(b.chain_early != 0, tc_wgrad3x3_kernel<3>, dim3(9 * P->split1, b.S), dim3(kThreadsTc), q.smem_wg, s,
+            q.in_wg, q.skip_wg, k.c_prev / kBlockK, q.dout_wg, k.w_partials, k.c_prev + k.c_skip, k.c_out, b.h, b.w, P->chunks1, P->per1,
+            P->split1, q.cols_wg, b.err, skip, skip_stride);
+        if (t) t->mark(kWg3Names[i], s, st_repeats(t));
+        n += st_repeats(t);
+        if (k.pass_back) {
+            // gradient with respect to the previous block's output: the tile walk of the forward over this block's
+            // output gradient, with the mirrored and transposed weights; masked by the previous block's ReLU bits
+            const TcBlock& r = b.blk[i - 1];
+            int grid, tail_split;
+            tile_walk(P, total, k.c_prev, &grid, &tail_split);
+            ST_REPEAT(t) launch_chain(b.chain_early != 0, tc_fwd3x3_kernel<4, 1>, dim3(grid), dim3(kFwd3Threads), q.smem_back, s,
+                q.dout_fwd, q.dout_fwd, k.c_out / kBlockK, 0, q.wt_map, q.wt_map_q, tail_split, (const float*)nullptr, (int64_t)0, (int64_t)0,
+                r.dout, r.relu_bits, r.b_partials, k.c_prev, b.h, b.w, total, pow2_cols(k.c_prev), b.err, skip, skip_stride);
+            if (t) t->mark("tc_dgrad3x3", s, st_repeats(t));
+            n += st_repeats(t);
+        }
     }
     return n;
 }

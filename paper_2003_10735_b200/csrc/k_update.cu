@@ -20,6 +20,22 @@ bool pdl_enabled()
 
 constexpr int kUpdThreads = 256;
 
+// bf16 copies of weight element e (internal order [tap][cout][cin]) of a layer: the one the forward and the weight
+// gradient read, and, for a 3x3 layer whose gradient is passed back, the mirrored and transposed one
+__device__ __forceinline__ void write_shadows(const LayerUpdate& ly, int s, int64_t e, float value)
+{
+    const bf16 v = __float2bfloat16_rn(value);
+    if (ly.shadow) ly.shadow[(int64_t)s * ly.shadow_stream_stride + e] = v;
+    if (ly.shadow_t) {
+        const int ci = (int)(e % ly.cin);
+        if (ci < ly.c_take) {
+            const int64_t r = e / ly.cin;
+            const int co = (int)(r % ly.cout), tap = (int)(r / ly.cout);
+            ly.shadow_t[(int64_t)s * ly.shadow_t_stream_stride + ((int64_t)(ly.taps - 1 - tap) * ly.c_take + ci) * ly.cout + co] = v;
+        }
+    }
+}
+
 // Bias corrections of Adam's step t: (1 - b1^t, 1 - b2^t), t = steps taken before this call + position in the call.
 struct AdamCorr { double c1, c2; };
 template <bool ADAM>
@@ -160,7 +176,7 @@ sgd_update_kernel(UpdateArgs a, int n_param_blocks, int64_t range_begin)
                     gr = a.grad[base + i];
                 }
                 const float t = apply_update<ADAM>(a, base + i, gr, corr, state[e]);
-                if (ly.shadow) ly.shadow[(int64_t)s * ly.shadow_stream_stride + (i - ly.w_off)] = __float2bfloat16_rn(t);
+                write_shadows(ly, s, i - ly.w_off, t);
             } else if (!ly.b_partials) {
                 apply_update<ADAM>(a, base + i, a.grad[base + i], corr, state[e]);
             }   // biases with partial sums are finished by the reduction warps below
@@ -253,10 +269,7 @@ sgd_update_stream_kernel(UpdateArgs a, int L)
     const int64_t gi = (int64_t)s * a.n_params + ly.w_off + e;
     const AdamCorr corr = adam_corrections<ADAM>(a, s);
 #pragma unroll
-    for (int j = 0; j < VEC; ++j) {
-        apply_update<ADAM>(a, gi + j, g[j], corr);
-        if (ly.shadow) ly.shadow[(int64_t)s * ly.shadow_stream_stride + e + j] = __float2bfloat16_rn(a.theta[gi + j]);
-    }
+    for (int j = 0; j < VEC; ++j) write_shadows(ly, s, e + j, apply_update<ADAM>(a, gi + j, g[j], corr));
 }
 
 template <bool ADAM>
@@ -265,7 +278,7 @@ static int launch_sgd_update_t(const UpdateArgs& a, cudaStream_t s)
     int n_launches = 1;
     // large layers with partial sums go through the streaming kernel; everything else (small layers, biases,
     // loss) through the grouped kernel, which then starts after the streamed range
-    int64_t range_begin = 0;
+    int64_t range_begin = a.param_begin;
     for (int L = 0; L < a.n_layers; ++L) {
         const LayerUpdate& ly = a.layer[L];
         const int64_t nw = (int64_t)ly.cout * ly.cin * ly.taps;
@@ -325,9 +338,7 @@ __global__ void refresh_shadow_kernel(UpdateArgs a)
     for (int L = 0; L < a.n_layers; ++L) {
         const LayerUpdate& ly = a.layer[L];
         const int64_t nw = (int64_t)ly.cout * ly.cin * ly.taps;
-        if (ly.shadow && i >= ly.w_off && i < ly.w_off + nw)
-            ly.shadow[(int64_t)s * ly.shadow_stream_stride + (i - ly.w_off)] =
-                __float2bfloat16_rn(a.theta[(int64_t)s * a.n_params + i]);
+        if (i >= ly.w_off && i < ly.w_off + nw) write_shadows(ly, s, i - ly.w_off, a.theta[(int64_t)s * a.n_params + i]);
     }
 }
 
@@ -415,12 +426,13 @@ void launch_train_commit(const TrainCtl& t, float* theta, cudaStream_t s)
 
 // ---- pack / unpack ---------------------------------------------------------------------------------
 template <bool TO_PACKED>
-__global__ void pack_kernel(const float* __restrict__ src, float* __restrict__ dst, PackLayout L)
+__global__ void pack_kernel(const float* __restrict__ src, float* __restrict__ dst, PackLayout L, int64_t begin, int64_t count)
 {
-    const int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;   // index in packed order
-    if (i >= L.n_params) return;
+    const int64_t q = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;   // index in the packed buffer
+    if (q >= count) return;
+    const int64_t i = begin + q;                                         // the parameter's index in packed order
     const int64_t base = (int64_t)blockIdx.y * L.n_params;
-    int64_t j = i;                                                       // index in internal order
+    int64_t j = i;                                                       // its index in internal order
     for (int k = 0; k < L.n_layers; ++k) {
         const int64_t nw = (int64_t)L.cout[k] * L.cin[k] * L.taps[k];
         if (i >= L.w_off[k] && i < L.w_off[k] + nw) {
@@ -431,18 +443,20 @@ __global__ void pack_kernel(const float* __restrict__ src, float* __restrict__ d
             j = L.w_off[k] + ((int64_t)tap * L.cout[k] + co) * L.cin[k] + ci;
         }
     }
-    if (TO_PACKED) dst[base + i] = src[base + j];
-    else dst[base + j] = src[base + i];
+    if (TO_PACKED) dst[(int64_t)blockIdx.y * count + q] = src[base + j];
+    else dst[base + j] = src[(int64_t)blockIdx.y * count + q];
 }
 
-void launch_pack(const float* internal, float* packed, const PackLayout& L, int n_bufs, cudaStream_t s)
+void launch_pack(const float* internal, float* packed, const PackLayout& L, int64_t begin, int64_t count, int n_bufs, cudaStream_t s)
 {
-    pack_kernel<true><<<dim3((unsigned)((L.n_params + 255) / 256), (unsigned)n_bufs), 256, 0, s>>>(internal, packed, L);
+    if (count <= 0) return;
+    pack_kernel<true><<<dim3((unsigned)((count + 255) / 256), (unsigned)n_bufs), 256, 0, s>>>(internal, packed, L, begin, count);
 }
 
-void launch_unpack(const float* packed, float* internal, const PackLayout& L, int n_bufs, cudaStream_t s)
+void launch_unpack(const float* packed, float* internal, const PackLayout& L, int64_t begin, int64_t count, int n_bufs, cudaStream_t s)
 {
-    pack_kernel<false><<<dim3((unsigned)((L.n_params + 255) / 256), (unsigned)n_bufs), 256, 0, s>>>(packed, internal, L);
+    if (count <= 0) return;
+    pack_kernel<false><<<dim3((unsigned)((count + 255) / 256), (unsigned)n_bufs), 256, 0, s>>>(packed, internal, L, begin, count);
 }
 
 }  // namespace st

@@ -50,11 +50,22 @@ struct st_ctx {
     bf16* dz_bf16 = nullptr;
     int64_t dz_pitch = 0;
     float *hid_f32 = nullptr, *dhid_f32 = nullptr;
-    bf16 *hid_bf16 = nullptr, *dhid_bf16 = nullptr;
-    uint32_t* relu_bits = nullptr;
-    bf16 *w1_shadow = nullptr, *w2_shadow = nullptr;
-    float *w1_partials = nullptr, *w2_partials = nullptr, *b1_partials = nullptr;
-    int n_split1 = 0, n_split2 = 0, n_b1part = 0;
+    // student blocks in front of the classifier (bf16 tensor-core path): the head with one hidden layer is one block
+    // without a skip input
+    int n_blocks = 0, first_trained = 0;    // blocks before first_trained are frozen (Section 4.2)
+    struct Block {
+        int c_prev = 0, c_skip = 0, c_out = 0;
+        bf16 *skip = nullptr, *out = nullptr, *dout = nullptr, *w = nullptr, *w_t = nullptr;
+        uint32_t* relu_bits = nullptr;
+        float *w_partials = nullptr, *b_partials = nullptr;
+        int n_bpart = 0;
+        std::vector<char> has_skip;
+    } blk[kMaxBlocks];
+    bool prefix_current = false;            // the frozen blocks' outputs belong to the current features and skip inputs
+    int64_t trained_begin = 0, n_trained = 0;   // where the trained layers start in one stream's parameters; how many values
+    bf16* w2_shadow = nullptr;
+    float* w2_partials = nullptr;
+    int n_split1 = 0, n_split2 = 0;
     float *loss_part = nullptr, *db_part = nullptr;
     int n_k3_blocks = 0;
     CUtensorMap k3_map;        // tile map of z for the fused upsample + cross-entropy kernel
@@ -176,18 +187,22 @@ st_status check_launch(st_ctx* ctx, const char* what)
     return ST_OK;
 }
 
-UpdateArgs make_update_args(st_ctx* c, int slot, const int* skip = nullptr, int64_t skip_stride = 0)
+// Arguments of the update kernels.  `all_layers`: every layer including the frozen ones (refreshing the bf16 copies);
+// otherwise the layers behind the freeze boundary only.
+UpdateArgs make_update_args(st_ctx* c, int slot, const int* skip = nullptr, int64_t skip_stride = 0, bool all_layers = false)
 {
     UpdateArgs u;
     memset(&u, 0, sizeof u);
     u.theta = c->theta; u.vel = c->vel; u.grad = c->grad;
     u.n_params = c->n_params; u.S = c->S; u.lr = c->d.lr; u.mu = c->d.momentum;
-    u.n_layers = c->layout.n_layers;
-    for (int L = 0; L < u.n_layers; ++L) {
-        LayerUpdate& ly = u.layer[L];
+    const int n_all = c->layout.n_layers, first = all_layers ? 0 : (c->bf16_mode ? c->first_trained : 0);
+    u.n_layers = n_all - first;
+    u.param_begin = all_layers ? 0 : c->trained_begin;
+    for (int L = first; L < n_all; ++L) {
+        LayerUpdate& ly = u.layer[L - first];
         ly.w_off = c->layout.w_off[L]; ly.b_off = c->layout.b_off[L];
         ly.cout = c->layout.cout[L]; ly.cin = c->layout.cin[L]; ly.taps = c->layout.taps[L];
-        const bool last = (L == u.n_layers - 1);
+        const bool last = (L == n_all - 1);
         if (last) { ly.b_partials = c->db_part; ly.n_bpart = c->n_k3_blocks; }
         if (c->bf16_mode) {
             if (last) {
@@ -196,11 +211,13 @@ UpdateArgs make_update_args(st_ctx* c, int slot, const int* skip = nullptr, int6
                 ly.w_stream_stride = ly.w_split_stride * c->n_split2;
                 ly.shadow = c->w2_shadow; ly.shadow_stream_stride = (int64_t)kClassPad * ly.cin;
             } else {
-                ly.w_partials = c->w1_partials; ly.n_split = c->n_split1;
+                const st_ctx::Block& k = c->blk[L];
+                ly.w_partials = k.w_partials; ly.n_split = c->n_split1;
                 ly.w_split_stride = (int64_t)9 * ly.cout * ly.cin;
                 ly.w_stream_stride = ly.w_split_stride * c->n_split1;
-                ly.shadow = c->w1_shadow; ly.shadow_stream_stride = (int64_t)9 * ly.cout * ly.cin;
-                ly.b_partials = c->b1_partials; ly.n_bpart = c->n_b1part;
+                ly.shadow = k.w; ly.shadow_stream_stride = (int64_t)9 * ly.cout * ly.cin;
+                ly.shadow_t = k.w_t; ly.shadow_t_stream_stride = (int64_t)9 * k.c_prev * ly.cout; ly.c_take = k.c_prev;
+                ly.b_partials = k.b_partials; ly.n_bpart = k.n_bpart;
             }
         }
     }
@@ -214,6 +231,21 @@ UpdateArgs make_update_args(st_ctx* c, int slot, const int* skip = nullptr, int6
     return u;
 }
 
+// The outputs of the frozen blocks do not change while the blocks behind them are trained (Section 4.2): they are
+// computed once per key frame, outside the replayed step.
+st_status ensure_prefix(st_ctx* c)
+{
+    if (!c->bf16_mode || c->prefix_current) return ST_OK;
+    const int n = c->first_trained < c->n_blocks ? c->first_trained : c->n_blocks;
+    if (n > 0) {
+        c->launches += tc_forward_blocks(c->plan, 0, n, c->stream);
+        cudaError_t e = cudaGetLastError();
+        if (e != cudaSuccess) return ST_ERR_CUDA;
+    }
+    c->prefix_current = true;
+    return ST_OK;
+}
+
 // Forward of the trainable part for all streams: z (and the hidden activation).
 // `skip` (tensor-core kernels only): per-stream flags, see tc_forward.
 st_status enqueue_forward(st_ctx* c, StageTimer* t = nullptr, const int* skip = nullptr, int64_t skip_stride = 0,
@@ -221,7 +253,7 @@ st_status enqueue_forward(st_ctx* c, StageTimer* t = nullptr, const int* skip = 
 {
     cudaStream_t s = c->stream;
     if (c->bf16_mode) {
-        c->launches += tc_forward(c->plan, s, t, skip, skip_stride, after_update);
+        c->launches += tc_forward(c->plan, s, t, skip, skip_stride, after_update, c->first_trained < c->n_blocks ? c->first_trained : c->n_blocks);
     } else if (c->Ch == 0) {
         ST_REPEAT(t) launch_conv_fwd_f32(c->x_f32, c->Cin, c->h, c->w, c->theta + c->layout.w_off[0], c->theta + c->layout.b_off[0],
                             c->C, 1, false, c->z, c->S, (int64_t)c->Cin * c->p, c->n_params, c->n_params,
@@ -373,6 +405,30 @@ size_t st_param_count(int32_t c_in, int32_t c_hidden, int32_t n_classes)
     return (size_t)c_hidden * c_in * 9 + c_hidden + (size_t)n_classes * c_hidden + n_classes;
 }
 
+st_status st_head_param_counts(const st_head_desc* d, size_t* n_all, size_t* n_trained)
+{
+    if (!d || d->c_in < 1 || d->n_classes < 1 || d->c_hidden < 0) return ST_ERR_INVALID_ARG;
+    size_t all = 0, frozen = 0;
+    int prev = d->c_in;
+    if (d->n_blocks != 0) {
+        if (d->n_blocks < 0 || d->n_blocks > kMaxBlocks || d->c_hidden != 0 || d->first_trained < 0 || d->first_trained > d->n_blocks)
+            return ST_ERR_INVALID_ARG;
+        for (int i = 0; i < d->n_blocks; ++i) {
+            if (d->block_c_out[i] < 1 || d->block_c_skip[i] < 0) return ST_ERR_INVALID_ARG;
+            all += (size_t)d->block_c_out[i] * (prev + d->block_c_skip[i]) * 9 + d->block_c_out[i];
+            if (i < d->first_trained) frozen = all;
+            prev = d->block_c_out[i];
+        }
+    } else if (d->c_hidden > 0) {
+        all += (size_t)d->c_hidden * prev * 9 + d->c_hidden;
+        prev = d->c_hidden;
+    }
+    all += (size_t)d->n_classes * prev + d->n_classes;
+    if (n_all) *n_all = all;
+    if (n_trained) *n_trained = all - frozen;
+    return ST_OK;
+}
+
 const char* st_status_name(st_status s)
 {
     switch (s) {
@@ -446,17 +502,47 @@ st_status st_init_head(const st_head_desc* desc, const float* init_params, st_ct
                         "st_init_head: the bf16 tensor-core path needs c_in and c_hidden multiples of 64, "
                         "c_hidden <= 256, c_in <= 1024 and n_classes <= %d", kClassPad);
     }
+    // the back part as a stack of student blocks (n_blocks > 0), or the head given by c_hidden (n_blocks == 0)
+    int n_blocks = 0, first_trained = 0, blk_out[kMaxBlocks] = {0}, blk_skip[kMaxBlocks] = {0};
+    if (d.n_blocks != 0) {
+        if (d.n_blocks < 0 || d.n_blocks > kMaxBlocks || d.c_hidden != 0 || d.first_trained < 0 || d.first_trained > d.n_blocks)
+            return fail(nullptr, ST_ERR_INVALID_ARG, "st_init_head: n_blocks must be 0..%d with c_hidden 0, and first_trained 0..n_blocks", kMaxBlocks);
+        if (d.gemm_precision != 1)
+            return fail(nullptr, ST_ERR_UNSUPPORTED, "st_init_head: a stack of blocks needs gemm_precision 1 (bf16 tensor cores)");
+        int prev = d.c_in;
+        for (int i = 0; i < d.n_blocks; ++i) {
+            const int co = d.block_c_out[i], cs = d.block_c_skip[i];
+            if (co < 1 || cs < 0) return fail(nullptr, ST_ERR_INVALID_ARG, "st_init_head: block %d needs c_out >= 1 and c_skip >= 0", i);
+            const int tot = prev + cs;
+            if (co % 64 != 0 || cs % 64 != 0 || prev % 64 != 0 || co > 256 || prev > 256 || ((tot + 127) / 128) * co > 512)
+                return fail(nullptr, ST_ERR_UNSUPPORTED,
+                            "st_init_head: block %d: channel counts must be multiples of 64, at most 256 for the block's output and for "
+                            "the previous output it reads, and ceil((c_prev + c_skip) / 128) * c_out at most 512", i);
+            blk_out[i] = co; blk_skip[i] = cs; prev = co;
+        }
+        n_blocks = d.n_blocks; first_trained = d.first_trained;
+    } else if (d.c_hidden > 0 && d.gemm_precision == 1) {
+        if (((d.c_in + 127) / 128) * d.c_hidden > 512)
+            return fail(nullptr, ST_ERR_UNSUPPORTED, "st_init_head: ceil(c_in / 128) * c_hidden must be at most 512 on the bf16 path");
+        n_blocks = 1; blk_out[0] = d.c_hidden;
+    }
 
     st_ctx* c = new (std::nothrow) st_ctx();
     if (!c) return fail(nullptr, ST_ERR_OOM, "st_init_head: host allocation failed");
     c->d = d;
     c->stream = (cudaStream_t)d.cuda_stream;
     cudaGetDevice(&c->device);
-    c->S = d.n_streams; c->C = d.n_classes; c->Cin = d.c_in; c->Ch = d.c_hidden;
+    c->S = d.n_streams; c->C = d.n_classes; c->Cin = d.c_in;
+    c->Ch = n_blocks ? blk_out[n_blocks - 1] : d.c_hidden;      // channels in front of the classifier (0: the features themselves)
     c->h = d.feat_h; c->w = d.feat_w; c->H = d.feat_h * kUp; c->W = d.feat_w * kUp;
     c->p = (int64_t)c->h * c->w; c->P = (int64_t)c->H * c->W;
-    c->n_params = (int64_t)st_param_count(d.c_in, d.c_hidden, d.n_classes);
     c->bf16_mode = d.gemm_precision == 1;
+    c->n_blocks = n_blocks; c->first_trained = first_trained;
+    for (int i = 0, prev = d.c_in; i < n_blocks; ++i) {
+        c->blk[i].c_prev = prev; c->blk[i].c_skip = blk_skip[i]; c->blk[i].c_out = blk_out[i];
+        c->blk[i].has_skip.assign(d.n_streams, blk_skip[i] ? 0 : 1);
+        prev = blk_out[i];
+    }
     c->adam = d.optimizer == 1; c->b1 = ab1; c->b2 = ab2; c->eps = aeps;
     c->heavy_w = d.object_weight > 1 ? d.object_weight : 1; c->heavy_radius = d.object_radius; c->background = d.background_class;
     c->has_feat.assign(c->S, 0); c->has_labels.assign(c->S, 0);
@@ -469,17 +555,25 @@ st_status st_init_head(const st_head_desc* desc, const float* init_params, st_ct
     c->chain_early = pdl_enabled() && c->Ch == 0;
     if (const char* e = getenv("ST_PDL")) if (e[0] == '1') c->chain_early = true;
 
+    // layers in forward order: the 3x3 layers (blocks, or the fp32 path's hidden layer), then the classifier
     PackLayout& L = c->layout;
     memset(&L, 0, sizeof L);
-    L.n_params = c->n_params;
-    if (c->Ch == 0) {
-        L.n_layers = 1; L.cout[0] = c->C; L.cin[0] = c->Cin; L.taps[0] = 1;
-        L.w_off[0] = 0; L.b_off[0] = (int64_t)c->C * c->Cin;
-    } else {
-        L.n_layers = 2;
-        L.cout[0] = c->Ch; L.cin[0] = c->Cin; L.taps[0] = 9; L.w_off[0] = 0; L.b_off[0] = (int64_t)c->Ch * c->Cin * 9;
-        L.cout[1] = c->C; L.cin[1] = c->Ch; L.taps[1] = 1; L.w_off[1] = L.b_off[0] + c->Ch;
-        L.b_off[1] = L.w_off[1] + (int64_t)c->C * c->Ch;
+    {
+        int64_t off = 0;
+        int n = 0, prev = c->Cin;
+        const int n3 = c->bf16_mode ? n_blocks : (d.c_hidden ? 1 : 0);
+        for (int i = 0; i < n3; ++i, ++n) {
+            const int co = c->bf16_mode ? blk_out[i] : d.c_hidden, ci = prev + (c->bf16_mode ? blk_skip[i] : 0);
+            L.cout[n] = co; L.cin[n] = ci; L.taps[n] = 9; L.w_off[n] = off; off += (int64_t)co * ci * 9;
+            L.b_off[n] = off; off += co;
+            if (i < first_trained) c->trained_begin = off;
+            prev = co;
+        }
+        L.cout[n] = c->C; L.cin[n] = prev; L.taps[n] = 1; L.w_off[n] = off; off += (int64_t)c->C * prev;
+        L.b_off[n] = off; off += c->C;
+        L.n_layers = n + 1;
+        L.n_params = c->n_params = off;
+        c->n_trained = off - c->trained_begin;
     }
 
     const int S = c->S;
@@ -502,16 +596,26 @@ st_status st_init_head(const st_head_desc* desc, const float* init_params, st_ct
         c->dz_pitch = tc_dz_pitch(c->h, c->w);
         ALLOC(dz_bf16, (size_t)S * kClassPad * c->dz_pitch);
         ALLOC(w2_shadow, (size_t)S * kClassPad * c_last);
-        c->n_split2 = tc_wgrad_splits(2, c->Cin, c->Ch, c->h, c->w);
+        c->n_split2 = tc_wgrad_splits(2, c_last, c->h, c->w);
         ALLOC(w2_partials, (size_t)S * c->n_split2 * kClassPad * c_last);
-        if (c->Ch) {
-            ALLOC(hid_bf16, S * c->p * c->Ch); ALLOC(dhid_bf16, S * c->p * c->Ch);
-            ALLOC(relu_bits, S * c->p * (c->Ch / 32));
-            ALLOC(w1_shadow, (size_t)S * 9 * c->Ch * c->Cin);
-            c->n_split1 = tc_wgrad_splits(1, c->Cin, c->Ch, c->h, c->w);
-            ALLOC(w1_partials, (size_t)S * c->n_split1 * 9 * c->Ch * c->Cin);
-            c->n_b1part = tc_b1_partials(c->h, c->w);
-            ALLOC(b1_partials, (size_t)S * c->n_b1part * c->Ch);
+        c->n_split1 = n_blocks ? tc_wgrad_splits(1, 0, c->h, c->w) : 0;
+        for (int i = 0; i < n_blocks; ++i) {
+            st_ctx::Block& k = c->blk[i];
+            const size_t tot = (size_t)k.c_prev + k.c_skip;
+            const bool trained = i >= first_trained;
+            if (k.c_skip) ALLOC(blk[i].skip, S * c->p * k.c_skip);
+            ALLOC(blk[i].out, S * c->p * k.c_out);
+            ALLOC(blk[i].relu_bits, S * c->p * (k.c_out / 32));
+            ALLOC(blk[i].w, (size_t)S * 9 * k.c_out * tot);
+            if (trained) {
+                ALLOC(blk[i].dout, S * c->p * k.c_out);
+                ALLOC(blk[i].w_partials, (size_t)S * c->n_split1 * 9 * k.c_out * tot);
+                // the block in front of the classifier gets its gradient from the 128-pixel tiles of the 1x1 layer's
+                // kernel, the others from the 4 x 32 tiles of the 3x3 tile walk
+                k.n_bpart = i == n_blocks - 1 ? tc_b1_partials(c->h, c->w) : tc_tile3_count(c->h, c->w);
+                ALLOC(blk[i].b_partials, (size_t)S * k.n_bpart * k.c_out);
+                if (i > first_trained) ALLOC(blk[i].w_t, (size_t)S * 9 * k.c_prev * k.c_out);
+            }
         }
     } else {
         ALLOC(x_f32, S * c->Cin * c->p);
@@ -532,18 +636,28 @@ st_status st_init_head(const st_head_desc* desc, const float* init_params, st_ct
     // parameters: packed order -> internal order (the momentum buffer serves as scratch, then is zeroed)
     const size_t pbytes = (size_t)S * c->n_params * sizeof(float);
     e = cudaMemcpyAsync(c->vel, init_params, pbytes, cudaMemcpyDefault, c->stream);
-    if (e == cudaSuccess) { launch_unpack(c->vel, c->theta, c->layout, S, c->stream); e = cudaGetLastError(); }
+    if (e == cudaSuccess) { launch_unpack(c->vel, c->theta, c->layout, 0, c->n_params, S, c->stream); e = cudaGetLastError(); }
     if (e == cudaSuccess) e = cudaMemsetAsync(c->vel, 0, pbytes, c->stream);
     if (e == cudaSuccess && c->bf16_mode) {
         TcBuffers b;
         memset(&b, 0, sizeof b);
-        b.S = S; b.c_in = c->Cin; b.c_hidden = c->Ch; b.C = c->C; b.h = c->h; b.w = c->w;
-        b.x = c->x_bf16; b.w1 = c->w1_shadow; b.w2 = c->w2_shadow; b.theta = c->theta; b.n_params = c->n_params;
-        b.b1_off = c->Ch ? L.b_off[0] : 0; b.b2_off = L.b_off[L.n_layers - 1]; b.w2_off = L.w_off[L.n_layers - 1];
+        b.S = S; b.c_in = c->Cin; b.C = c->C; b.h = c->h; b.w = c->w;
+        b.x = c->x_bf16; b.w2 = c->w2_shadow; b.theta = c->theta; b.n_params = c->n_params;
+        b.b2_off = L.b_off[L.n_layers - 1]; b.w2_off = L.w_off[L.n_layers - 1];
         b.err = c->bad + 2;
         b.chain_early = c->chain_early ? 1 : 0;
-        b.z = c->z; b.hidden = c->hid_bf16; b.relu_bits = c->relu_bits; b.dz = c->dz; b.dz_bf16 = c->dz_bf16; b.dhidden = c->dhid_bf16;
-        b.w1_partials = c->w1_partials; b.w2_partials = c->w2_partials; b.b1_partials = c->b1_partials;
+        b.z = c->z; b.dz = c->dz; b.dz_bf16 = c->dz_bf16; b.w2_partials = c->w2_partials;
+        b.n_blocks = n_blocks;
+        for (int i = 0; i < n_blocks; ++i) {
+            const st_ctx::Block& k = c->blk[i];
+            TcBlock& q = b.blk[i];
+            q.c_prev = k.c_prev; q.c_skip = k.c_skip; q.c_out = k.c_out;
+            q.in_prev = i ? c->blk[i - 1].out : c->x_bf16; q.in_skip = k.skip;
+            q.w = k.w; q.w_t = k.w_t; q.b_off = L.b_off[i];
+            q.out = k.out; q.relu_bits = k.relu_bits; q.dout = k.dout;
+            q.w_partials = k.w_partials; q.b_partials = k.b_partials;
+            q.trained = i >= first_trained ? 1 : 0; q.pass_back = i > first_trained ? 1 : 0;
+        }
         char msg[256] = {0};
         c->plan = tc_plan_create(b, msg, sizeof msg);
         if (!c->plan) {
@@ -551,7 +665,7 @@ st_status st_init_head(const st_head_desc* desc, const float* init_params, st_ct
             st_destroy(c);
             return code;
         }
-        launch_refresh_shadow(make_update_args(c, -1), c->stream);
+        launch_refresh_shadow(make_update_args(c, -1, nullptr, 0, true), c->stream);
         e = cudaGetLastError();
     }
     if (e == cudaSuccess) e = cudaStreamSynchronize(c->stream);   // init_params may be released on return
@@ -584,6 +698,28 @@ st_status st_set_frozen_features(st_ctx* ctx, int32_t stream, const float* feat_
     }
     ctx->has_feat[stream] = 1;
     ctx->z_current = false;
+    ctx->prefix_current = false;
+    return ST_OK;
+}
+
+st_status st_set_skip_features(st_ctx* ctx, int32_t stream, int32_t block, const float* feat_chw)
+{
+    st_status st = check_stream_index(ctx, stream);
+    if (st != ST_OK) return st;
+    if (block < 0 || block >= ctx->n_blocks || ctx->blk[block].c_skip == 0)
+        return fail(ctx, ST_ERR_INVALID_ARG, "st_set_skip_features: block %d has no skip input", block);
+    if (!feat_chw) return fail(ctx, ST_ERR_INVALID_ARG, "st_set_skip_features: NULL features");
+    st_ctx::Block& k = ctx->blk[block];
+    const void* src = nullptr;
+    st = to_device(ctx, feat_chw, (size_t)k.c_skip * ctx->p * sizeof(float), &src);
+    if (st != ST_OK) return st;
+    launch_feat_to_bf16_nhwc((const float*)src, k.c_skip, ctx->p, k.skip + (int64_t)stream * ctx->p * k.c_skip, ctx->stream);
+    ctx->launches += 1;
+    st = check_launch(ctx, "skip feature cache");
+    if (st != ST_OK) return st;
+    k.has_skip[stream] = 1;
+    ctx->z_current = false;
+    ctx->prefix_current = false;
     return ST_OK;
 }
 
@@ -656,15 +792,30 @@ st_status st_set_labels(st_ctx* ctx, int32_t stream, const uint8_t* labels)
     return tag_labels(ctx, stream);
 }
 
+namespace {
+// every stream has its features (and skip inputs) and, if asked for, its labels; the frozen blocks' outputs are current
+st_status ready_to_run(st_ctx* ctx, const char* who, bool need_labels)
+{
+    for (int s = 0; s < ctx->S; ++s) {
+        if (!ctx->has_feat[s]) return fail(ctx, ST_ERR_BAD_STATE, "%s: stream %d has no frozen features yet", who, s);
+        for (int b = 0; b < ctx->n_blocks; ++b)
+            if (!ctx->blk[b].has_skip[s]) return fail(ctx, ST_ERR_BAD_STATE, "%s: stream %d has no skip input for block %d yet", who, s, b);
+        if (need_labels && !ctx->has_labels[s]) return fail(ctx, ST_ERR_BAD_STATE, "%s: stream %d has no labels yet", who, s);
+    }
+    if (ensure_prefix(ctx) != ST_OK) return fail(ctx, ST_ERR_CUDA, "%s: forward of the frozen blocks failed", who);
+    return ST_OK;
+}
+}  // namespace
+
 st_status st_distill_step(st_ctx* ctx, int32_t n_steps, float* loss_out, int64_t* conf_out)
 {
     if (!ctx) return ST_ERR_INVALID_ARG;
     if (n_steps < 1 || n_steps > kMaxSteps)
         return fail(ctx, ST_ERR_INVALID_ARG, "st_distill_step: n_steps %d outside 1..%d", n_steps, kMaxSteps);
-    for (int s = 0; s < ctx->S; ++s)
-        if (!ctx->has_feat[s] || !ctx->has_labels[s])
-            return fail(ctx, ST_ERR_BAD_STATE, "st_distill_step: stream %d has no %s yet", s,
-                        ctx->has_feat[s] ? "labels" : "frozen features");
+    {
+        const st_status ready = ready_to_run(ctx, "st_distill_step", true);
+        if (ready != ST_OK) return ready;
+    }
     const bool want_conf = conf_out != nullptr;
     const size_t cc = (size_t)ctx->C * ctx->C;
     ctx->z_current = false;                 // the steps leave z at the forward before the last update
@@ -764,10 +915,10 @@ st_status st_train_key_frame(st_ctx* ctx, double threshold, int32_t max_updates,
         return fail(ctx, ST_ERR_INVALID_ARG, "st_train_key_frame: max_updates %d outside 0..%d", max_updates, kMaxSteps - 1);
     if (!(threshold == threshold))
         return fail(ctx, ST_ERR_INVALID_ARG, "st_train_key_frame: threshold is not a number");
-    for (int s = 0; s < ctx->S; ++s)
-        if (!ctx->has_feat[s] || !ctx->has_labels[s])
-            return fail(ctx, ST_ERR_BAD_STATE, "st_train_key_frame: stream %d has no %s yet", s,
-                        ctx->has_feat[s] ? "labels" : "frozen features");
+    {
+        const st_status ready = ready_to_run(ctx, "st_train_key_frame", true);
+        if (ready != ST_OK) return ready;
+    }
     const size_t cc = (size_t)ctx->C * ctx->C;
     ctx->z_current = false;
     cudaError_t e = cudaSuccess;
@@ -846,9 +997,10 @@ st_status st_profile_step(st_ctx* ctx, int32_t n_steps, int32_t* n_stages, float
     if (!ctx) return ST_ERR_INVALID_ARG;
     if (n_steps < 1 || !n_stages || !ms_out || !names_out)
         return fail(ctx, ST_ERR_INVALID_ARG, "st_profile_step: n_steps >= 1 and non-NULL outputs are required");
-    for (int s = 0; s < ctx->S; ++s)
-        if (!ctx->has_feat[s] || !ctx->has_labels[s])
-            return fail(ctx, ST_ERR_BAD_STATE, "st_profile_step: stream %d has no features or labels yet", s);
+    {
+        const st_status ready = ready_to_run(ctx, "st_profile_step", true);
+        if (ready != ST_OK) return ready;
+    }
     ctx->z_current = false;
     StageTimer t;
     t.repeat = 8;
@@ -881,21 +1033,21 @@ st_status st_pack_updated_params(st_ctx* ctx, int32_t stream, void* dst, size_t 
 {
     st_status st = check_stream_index(ctx, stream);
     if (st != ST_OK) return st;
-    const size_t need = (size_t)ctx->n_params * sizeof(float);
+    const size_t need = (size_t)ctx->n_trained * sizeof(float);      // UpdatedPart: the layers behind the freeze boundary
     if (nbytes) *nbytes = need;
     if (!dst) return fail(ctx, ST_ERR_INVALID_ARG, "st_pack_updated_params: NULL destination");
     if (dst_capacity < need)
         return fail(ctx, ST_ERR_BUFFER_TOO_SMALL, "st_pack_updated_params: capacity %zu < %zu bytes", dst_capacity, need);
     const float* src = ctx->theta + (int64_t)stream * ctx->n_params;
     if (is_device_ptr(dst)) {
-        launch_pack(src, (float*)dst, ctx->layout, 1, ctx->stream);
+        launch_pack(src, (float*)dst, ctx->layout, ctx->trained_begin, ctx->n_trained, 1, ctx->stream);
         ctx->launches += 1;
         return check_launch(ctx, "pack");
     }
     // host destination: pack into the staging buffer, then copy out
     st = ensure_staging(ctx, need);
     if (st != ST_OK) return st;
-    launch_pack(src, (float*)ctx->staging, ctx->layout, 1, ctx->stream);
+    launch_pack(src, (float*)ctx->staging, ctx->layout, ctx->trained_begin, ctx->n_trained, 1, ctx->stream);
     ctx->launches += 1;
     st = check_launch(ctx, "pack");
     if (st != ST_OK) return st;
@@ -908,14 +1060,14 @@ st_status st_apply_update(st_ctx* ctx, int32_t stream, const void* src, size_t n
 {
     st_status st = check_stream_index(ctx, stream);
     if (st != ST_OK) return st;
-    const size_t need = (size_t)ctx->n_params * sizeof(float);
+    const size_t need = (size_t)ctx->n_trained * sizeof(float);
     if (!src) return fail(ctx, ST_ERR_INVALID_ARG, "st_apply_update: NULL source");
     if (nbytes != need) return fail(ctx, ST_ERR_INVALID_ARG, "st_apply_update: %zu bytes given, the updated part has %zu", nbytes, need);
     const void* dev = nullptr;
     st = to_device(ctx, src, need, &dev);
     if (st != ST_OK) return st;
     ctx->z_current = false;
-    launch_unpack((const float*)dev, ctx->theta + (int64_t)stream * ctx->n_params, ctx->layout, 1, ctx->stream);
+    launch_unpack((const float*)dev, ctx->theta + (int64_t)stream * ctx->n_params, ctx->layout, ctx->trained_begin, ctx->n_trained, 1, ctx->stream);
     ctx->launches += 1;
     if (ctx->bf16_mode) { launch_refresh_shadow(make_update_args(ctx, -1), ctx->stream); ctx->launches += 1; }
     return check_launch(ctx, "apply update");
@@ -925,9 +1077,9 @@ namespace {
 // forward of all streams with the current parameters, then the mask kernel on `stream`
 st_status student_forward(st_ctx* ctx, int32_t stream, const char* who)
 {
-    if (!ctx->has_feat[stream]) return fail(ctx, ST_ERR_BAD_STATE, "%s: stream %d has no frozen features yet", who, stream);
-    for (int s = 0; s < ctx->S; ++s)
-        if (!ctx->has_feat[s]) return fail(ctx, ST_ERR_BAD_STATE, "%s: the forward runs on all streams; stream %d has no features", who, s);
+    (void)stream;                           // the forward runs on all streams
+    st_status ready = ready_to_run(ctx, who, false);
+    if (ready != ST_OK) return ready;
     if (ctx->z_current) return ST_OK;       // an earlier call already ran it and nothing has changed since
     st_status st = enqueue_forward(ctx);
     ctx->z_current = st == ST_OK;
@@ -1041,7 +1193,14 @@ st_status st_read_tensor(st_ctx* ctx, int32_t stream, st_tensor which, float* ds
         case ST_TENSOR_PARAM_GRAD: case ST_TENSOR_MOMENTUM: count = (size_t)ctx->n_params; break;
         case ST_TENSOR_HIDDEN: case ST_TENSOR_HIDDEN_GRAD:
             if (!ctx->Ch) return fail(ctx, ST_ERR_INVALID_ARG, "st_read_tensor: the head has no hidden layer");
+            if (which == ST_TENSOR_HIDDEN_GRAD && ctx->bf16_mode && !ctx->blk[ctx->n_blocks - 1].dout)
+                return fail(ctx, ST_ERR_INVALID_ARG, "st_read_tensor: the last block is frozen, no gradient is formed for it");
             count = (size_t)ctx->Ch * ctx->p; break;
+        case ST_TENSOR_HIDDEN_FIRST: case ST_TENSOR_HIDDEN_GRAD_FIRST:
+            if (ctx->n_blocks < 2) return fail(ctx, ST_ERR_INVALID_ARG, "st_read_tensor: the head has no second block");
+            if (which == ST_TENSOR_HIDDEN_GRAD_FIRST && !ctx->blk[0].dout)
+                return fail(ctx, ST_ERR_INVALID_ARG, "st_read_tensor: the first block is frozen, no gradient is formed for it");
+            count = (size_t)ctx->blk[0].c_out * ctx->p; break;
         case ST_TENSOR_FEATURES: count = (size_t)ctx->Cin * ctx->p; break;
         default: return fail(ctx, ST_ERR_INVALID_ARG, "st_read_tensor: unknown tensor %d", (int)which);
     }
@@ -1067,15 +1226,23 @@ st_status st_read_tensor(st_ctx* ctx, int32_t stream, st_tensor which, float* ds
             }
             src = ctx->dz + s * ctx->C * ctx->p;
             break;
-        case ST_TENSOR_PARAM_GRAD: launch_pack(ctx->grad + s * ctx->n_params, ctx->read_tmp, ctx->layout, 1, ctx->stream); src = ctx->read_tmp; break;
-        case ST_TENSOR_MOMENTUM: launch_pack(ctx->vel + s * ctx->n_params, ctx->read_tmp, ctx->layout, 1, ctx->stream); src = ctx->read_tmp; break;
+        case ST_TENSOR_PARAM_GRAD: launch_pack(ctx->grad + s * ctx->n_params, ctx->read_tmp, ctx->layout, 0, ctx->n_params, 1, ctx->stream); src = ctx->read_tmp; break;
+        case ST_TENSOR_MOMENTUM: launch_pack(ctx->vel + s * ctx->n_params, ctx->read_tmp, ctx->layout, 0, ctx->n_params, 1, ctx->stream); src = ctx->read_tmp; break;
         case ST_TENSOR_HIDDEN:
-            if (ctx->bf16_mode) { launch_nhwc_bf16_to_chw(ctx->hid_bf16 + s * ctx->p * ctx->Ch, ctx->Ch, ctx->p, ctx->read_tmp, ctx->stream); src = ctx->read_tmp; }
+            if (ctx->bf16_mode) { launch_nhwc_bf16_to_chw(ctx->blk[ctx->n_blocks - 1].out + s * ctx->p * ctx->Ch, ctx->Ch, ctx->p, ctx->read_tmp, ctx->stream); src = ctx->read_tmp; }
             else src = ctx->hid_f32 + s * ctx->Ch * ctx->p;
             break;
         case ST_TENSOR_HIDDEN_GRAD:
-            if (ctx->bf16_mode) { launch_nhwc_bf16_to_chw(ctx->dhid_bf16 + s * ctx->p * ctx->Ch, ctx->Ch, ctx->p, ctx->read_tmp, ctx->stream); src = ctx->read_tmp; }
+            if (ctx->bf16_mode) { launch_nhwc_bf16_to_chw(ctx->blk[ctx->n_blocks - 1].dout + s * ctx->p * ctx->Ch, ctx->Ch, ctx->p, ctx->read_tmp, ctx->stream); src = ctx->read_tmp; }
             else src = ctx->dhid_f32 + s * ctx->Ch * ctx->p;
+            break;
+        case ST_TENSOR_HIDDEN_FIRST:
+            launch_nhwc_bf16_to_chw(ctx->blk[0].out + s * ctx->p * ctx->blk[0].c_out, ctx->blk[0].c_out, ctx->p, ctx->read_tmp, ctx->stream);
+            src = ctx->read_tmp;
+            break;
+        case ST_TENSOR_HIDDEN_GRAD_FIRST:
+            launch_nhwc_bf16_to_chw(ctx->blk[0].dout + s * ctx->p * ctx->blk[0].c_out, ctx->blk[0].c_out, ctx->p, ctx->read_tmp, ctx->stream);
+            src = ctx->read_tmp;
             break;
         case ST_TENSOR_FEATURES:
             if (ctx->bf16_mode) { launch_nhwc_bf16_to_chw(ctx->x_bf16 + s * ctx->p * ctx->Cin, ctx->Cin, ctx->p, ctx->read_tmp, ctx->stream); src = ctx->read_tmp; }

@@ -60,6 +60,8 @@ inline cudaError_t launch_chain(bool early, void (*kernel)(KArgs...), dim3 grid,
 constexpr int kUp = 4;            // bilinear upsample factor of the head (frame = feature map * 4)
 constexpr int kMaxSteps = 64;     // upper bound of n_steps in one st_distill_step call
 constexpr int kClassPad = 32;     // class rows of bf16 GEMM operands are padded to this (UMMA N)
+constexpr int kMaxBlocks = 2;     // student blocks in front of the classifier (Section 5.2: SB5, SB6)
+constexpr int kMaxLayers = kMaxBlocks + 1;
 
 // ---- K1: teacher logits -> uint8 labels -------------------------------------------------------
 void launch_argmax_u8(const float* logits, int C, int64_t P, uint8_t* labels, cudaStream_t s);
@@ -163,6 +165,9 @@ struct LayerUpdate {
     int n_bpart;
     bf16* shadow;              // nullptr or the bf16 copy of the weight read by the GEMMs (same linear index)
     int64_t shadow_stream_stride;
+    bf16* shadow_t;            // nullptr, or a second bf16 copy [9][c_take][cout] with the taps mirrored and the channels
+    int64_t shadow_t_stream_stride;   // transposed, for the first c_take input channels: what the gradient passed back
+    int c_take;                //   through this 3x3 layer multiplies
 };
 struct UpdateArgs {
     float* theta;      // [S][n_params]   internal order
@@ -171,8 +176,9 @@ struct UpdateArgs {
     int64_t n_params;
     int S;
     float lr, mu;
-    LayerUpdate layer[2];
+    LayerUpdate layer[kMaxLayers];
     int n_layers;
+    int64_t param_begin;     // parameters before this index belong to frozen layers and are left alone
     const float* loss_part;  // [S][n_loss_part] per-block sums of per-pixel losses
     int n_loss_part;
     float* loss_buf;         // [S][kMaxSteps]
@@ -223,34 +229,50 @@ void launch_train_commit(const TrainCtl& t, float* theta, cudaStream_t s);
 
 // ---- K7: packed parameter buffer <-> internal order ---------------------------------------------
 // packed: per layer weight [cout][cin][kh][kw] then bias; internal: weight [tap][cout][cin] then bias.
-struct PackLayout { int n_layers; int64_t w_off[2], b_off[2]; int cout[2], cin[2], taps[2]; int64_t n_params; };
-void launch_pack(const float* internal, float* packed, const PackLayout& L, int n_bufs, cudaStream_t s);
-void launch_unpack(const float* packed, float* internal, const PackLayout& L, int n_bufs, cudaStream_t s);
+// `begin`, `count`: the range of one stream's parameters that the packed buffer carries (all of them at initialisation;
+// the trained layers, which come last, in UpdatedPart); packed buffers of consecutive streams lie `count` floats apart.
+struct PackLayout { int n_layers; int64_t w_off[kMaxLayers], b_off[kMaxLayers]; int cout[kMaxLayers], cin[kMaxLayers], taps[kMaxLayers]; int64_t n_params; };
+void launch_pack(const float* internal, float* packed, const PackLayout& L, int64_t begin, int64_t count, int n_bufs, cudaStream_t s);
+void launch_unpack(const float* packed, float* internal, const PackLayout& L, int64_t begin, int64_t count, int n_bufs, cudaStream_t s);
 
 // ---- bf16 tensor-core GEMMs (gemm_precision 1) -------------------------------------------------
 struct TcPlan;   // tensor maps and launch geometry; built once per context
+// One student block of the trainable back part: 3x3 convolution (zero padding 1) over the concatenation of the previous
+// block's output (the frozen part's output for the first block) and the block's skip input, then ReLU.
+struct TcBlock {
+    int c_prev, c_skip, c_out;
+    const bf16* in_prev;     // [S][p][c_prev]
+    const bf16* in_skip;     // [S][p][c_skip] or nullptr
+    const bf16* w;           // [S][9][c_out][c_prev + c_skip]  bf16 copy of the weight, tap-major
+    const bf16* w_t;         // [S][9][c_prev][c_out]  taps mirrored, channels transposed (pass_back only)
+    int64_t b_off;           // offset of the bias in one stream's parameters
+    bf16* out;               // [S][p][c_out]
+    uint32_t* relu_bits;     // [S][p][c_out/32]: one bit per output value, set where it is > 0
+    bf16* dout;              // [S][p][c_out]     gradient with respect to the output, after the ReLU mask
+    float* w_partials;       // [S][n_split1][9][c_out][c_prev + c_skip]
+    float* b_partials;       // [S][n_bpart][c_out]: 128-pixel tiles for the last block, 4 x 32 tiles for the others
+    int trained;             // the block lies behind the freeze boundary: its gradients are formed
+    int pass_back;           // ... and so does the block before it: the gradient is passed on to it
+};
 struct TcBuffers {
-    int S, c_in, c_hidden, C, h, w;
+    int S, c_in, C, h, w;
+    int n_blocks;
+    TcBlock blk[kMaxBlocks];
     const bf16* x;        // [S][p][c_in]     cached features, pixel-major
-    const bf16* w1;       // [S][9][c_hidden][c_in]  (two-layer head) bf16 copy of the 3x3 weight
     const bf16* w2;       // [S][kClassPad][c_last]  bf16 copy of the 1x1 weight, rows >= C zero
     const float* theta;   // [S][n_params]    biases are read from the master parameters
-    int64_t n_params, b1_off, b2_off, w2_off;
+    int64_t n_params, b2_off, w2_off;
     float* z;             // [S][C][p]
-    bf16* hidden;         // [S][p][c_hidden]
-    uint32_t* relu_bits;  // [S][p][c_hidden/32]: one bit per hidden value, set where it is > 0
     const float* dz;      // [S][C][p]
     const bf16* dz_bf16;  // [S][kClassPad][tc_dz_pitch]
-    bf16* dhidden;        // [S][p][c_hidden]
-    float* w1_partials;   // [S][n_split1][9][c_hidden][c_in]
     float* w2_partials;   // [S][n_split2][kClassPad][c_last]
-    float* b1_partials;   // [S][n_b1part][c_hidden]
     unsigned int* err;    // device word: first wait that gave up (0 = none)
     int chain_early;      // launch the kernels so that each may start while its predecessor on the stream drains
 };
 // Geometry is fixed by the shapes alone, so scratch can be sized before the plan exists.
-int tc_wgrad_splits(int layer /*1: 3x3, 2: 1x1*/, int c_in, int c_hidden, int h, int w);
-int tc_b1_partials(int h, int w);
+int tc_wgrad_splits(int layer /*1: 3x3, 2: 1x1*/, int c_last, int h, int w);
+int tc_b1_partials(int h, int w);   // 128-pixel tiles (bias-gradient partials of the block in front of the classifier)
+int tc_tile3_count(int h, int w);   // 4 x 32 pixel tiles of a 3x3 layer per stream (bias-gradient partials of earlier blocks)
 int tc_dz_pitch(int h, int w);      // row pitch (elements) of the bf16 logit gradient [S][kClassPad][pitch]
 TcPlan* tc_plan_create(const TcBuffers& b, char* err, size_t err_len);
 void tc_plan_destroy(TcPlan*);
@@ -271,9 +293,12 @@ inline int st_repeats(const StageTimer* t) { return t ? t->repeat : 1; }
 // `skip`: nullptr, or one flag per stream (skip[s * skip_stride]); the blocks of a flagged stream return at once.
 // Returns the number of kernels launched.  `after_update`: the kernel launched just before on this stream is the
 // parameter update of the previous iteration, which writes weights but no activations; the forward of a one-layer head
-// may then fetch its activation tiles while that update is still running.
+// may then fetch its activation tiles while that update is still running.  `first_block`: the blocks before it are
+// frozen and their outputs already computed for this key frame (tc_forward_blocks).
 int tc_forward(const TcPlan*, cudaStream_t s, StageTimer* t = nullptr, const int* skip = nullptr, int64_t skip_stride = 0,
-               bool after_update = false);
+               bool after_update = false, int first_block = 0);
+int tc_forward_blocks(const TcPlan*, int first, int last, cudaStream_t s, StageTimer* t = nullptr, const int* skip = nullptr,
+                      int64_t skip_stride = 0);
 int tc_backward(const TcPlan*, cudaStream_t s, StageTimer* t = nullptr, const int* skip = nullptr, int64_t skip_stride = 0);
 
 }  // namespace st
