@@ -226,7 +226,12 @@ def kernel_table(st, ctx, cfg, peaks, arith, n_profile_steps):
     """Per-kernel CUDA-event times of one step (st_profile_step) with the roofline each kernel is held against."""
     S, C, K = cfg.n_streams, cfg.n_classes, cfg.k_steps
     p, P = cfg.feat_h * cfg.feat_w, cfg.frame_h * cfg.frame_w
-    c_last = cfg.c_hidden or cfg.c_in
+    blocks = [tuple(b) for b in cfg.blocks] or ([(cfg.c_hidden, 0)] if cfg.c_hidden else [])
+    c_last = blocks[-1][0] if blocks else cfg.c_in
+
+    def block_flop(i):                  # one 3x3 layer over its concatenated input
+        c_prev = cfg.c_in if i == 0 else blocks[i - 1][0]
+        return 2.0 * S * p * blocks[i][0] * 9 * (c_prev + blocks[i][1])
     hbm, tensor_peak = peaks["hbm_gbs"], peaks["bf16_tflops"]
     kernels = {}
     for name, ms in st.st_profile_step(ctx, n_profile_steps):
@@ -243,11 +248,12 @@ def kernel_table(st, ctx, cfg, peaks, arith, n_profile_steps):
         elif name == "tc_wgrad1x1":
             k.update(bound="hbm", achieved=S * (p * c_last * 2 + C * p * 2) / ms / 1e6, peak=hbm, unit="GB/s",
                      tflops=2.0 * S * p * C * c_last / ms / 1e9)
-        elif name in ("tc_fwd3x3", "tc_wgrad3x3"):
-            k.update(bound="tensor", achieved=2.0 * S * p * cfg.c_hidden * cfg.c_in * 9 / ms / 1e9, peak=tensor_peak,
-                     unit="TFLOP/s")
+        elif name.startswith("tc_fwd3x3") or name.startswith("tc_wgrad3x3"):
+            k.update(bound="tensor", achieved=block_flop(1 if name.endswith("#2") else 0) / ms / 1e9, peak=tensor_peak, unit="TFLOP/s")
+        elif name == "tc_dgrad3x3":     # through block 1 into block 0's output channels
+            k.update(bound="tensor", achieved=2.0 * S * p * blocks[0][0] * 9 * blocks[1][0] / ms / 1e9, peak=tensor_peak, unit="TFLOP/s")
         elif name == "tc_dgrad":
-            k.update(bound="hbm", achieved=S * (2 * p * cfg.c_hidden * 2 + C * p * 4) / ms / 1e6, peak=hbm, unit="GB/s")
+            k.update(bound="hbm", achieved=S * (2 * p * c_last * 2 + C * p * 4) / ms / 1e6, peak=hbm, unit="GB/s")
         else:
             k.update(bound="latency")
         kernels[name] = k
@@ -270,8 +276,16 @@ def run_other_workload(st, torch, stream, idx, feats_d, logits_d, peaks, arith, 
     input sets already on the device (stream s takes set s mod N_SETS); no CPU baseline."""
     cfg = si.get_config(idx)
     S, C, K = cfg.n_streams, cfg.n_classes, cfg.k_steps
-    theta0 = np.concatenate([si.initial_head_params(cfg.c_in, cfg.c_hidden, C, 1000 + s) for s in range(S)])
-    ctx = make_context(st, stream, cfg, theta0)
+    if cfg.blocks:                      # the stack of blocks has its own channel counts: one input set of its own
+        theta0 = si.initial_stack_params(cfg.c_in, cfg.blocks, C, 1000)
+        ctx = make_context(st, stream, cfg, theta0, blocks=[tuple(b) for b in cfg.blocks], first_trained=cfg.first_trained)
+        own = torch.from_numpy(si.frozen_features(cfg.c_in, cfg.feat_h, cfg.feat_w, 0)).cuda()
+        feats_d = [[own]] * N_SETS
+        for b in range(len(cfg.blocks)):
+            st.st_set_skip_features(ctx, 0, b, torch.from_numpy(si.skip_features(cfg, b, 0)).cuda())
+    else:
+        theta0 = np.concatenate([si.initial_head_params(cfg.c_in, cfg.c_hidden, C, 1000 + s) for s in range(S)])
+        ctx = make_context(st, stream, cfg, theta0)
     packed = torch.empty((S, ctx.n_params), dtype=torch.float32, device="cuda")
     conf = torch.zeros((S, C, C), dtype=torch.int64, device="cuda")
     miou = torch.zeros(S, dtype=torch.float64, device="cuda")
@@ -304,7 +318,7 @@ def run_other_workload(st, torch, stream, idx, feats_d, logits_d, peaks, arith, 
             "ms_per_key_frame_min": min(ms) / steps,
             "distill_loop_only": {"steps_per_s": K * S / (statistics.median(ms_loop) / steps / 1e3),
                                   "ms_per_step": statistics.median(ms_loop) / steps / K},
-            "streams": S, "c_hidden": cfg.c_hidden, "kernels": kernels, "clocks": clocks.finish(),
+            "streams": S, "c_hidden": cfg.c_hidden, "blocks": [list(b) for b in cfg.blocks], "kernels": kernels, "clocks": clocks.finish(),
             "inputs": f"the {N_SETS} input sets of the main run, stream s on set (key frame + s) mod {N_SETS}"}
 
 
@@ -555,7 +569,7 @@ def run_ours(args, cfg):
         if rank == 0 and world == 1 and not args.headline_only and args.workload == 2:
             result["confident_student"] = run_confident_student(st, torch, stream, cfg, peaks, arith)
             result["other_workloads"] = {str(idx): run_other_workload(st, torch, stream, idx, feats_d, logits_d, peaks, arith, local_rank)
-                                         for idx in (3, 5)}
+                                         for idx in (3, 5, 6)}
 
     if rank == 0:
         if world == 1 and not args.no_cpu_baseline:

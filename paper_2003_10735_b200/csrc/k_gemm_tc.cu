@@ -908,6 +908,17 @@ bool encode_tensor_map(CUtensorMap* m, CUtensorMapDataType dtype, CUtensorMapSwi
     return true;
 }
 
+// the instantiation of a 3x3 kernel with a given pipeline depth (all depths share one function type)
+template <int MODE>
+static decltype(&tc_fwd3x3_kernel<4, MODE>) fwd3_kernel(int stages)
+{
+    return stages >= 8 ? tc_fwd3x3_kernel<8, MODE> : (stages >= 6 ? tc_fwd3x3_kernel<6, MODE> : tc_fwd3x3_kernel<4, MODE>);
+}
+static decltype(&tc_wgrad3x3_kernel<3>) wgrad3_kernel(int stages)
+{
+    return stages >= 5 ? tc_wgrad3x3_kernel<5> : (stages >= 4 ? tc_wgrad3x3_kernel<4> : tc_wgrad3x3_kernel<3>);
+}
+
 struct TcBlockPlan {
     CUtensorMap in_fwd, skip_fwd;    // the block's two inputs {C, w, h, S}, box {64, 32, 4, 1} (forward tiles)
     CUtensorMap in_wg, skip_wg;      // same tensors, box {64, 32, 2, 1} (weight-gradient chunks)
@@ -916,6 +927,7 @@ struct TcBlockPlan {
     CUtensorMap dout_fwd;            // the block's output gradient {c_out, w, h, S}, box {64, 32, 4, 1} (A operand when passed back)
     CUtensorMap dout_wg;             // same tensor, box {64, 32, 2, 1} (B operand of the weight gradient)
     int cols_wg;                     // tensor-memory columns of the weight gradient
+    int stages_fwd, stages_back, stages_wg;   // pipeline depths of the three kernels of this block
     size_t smem_fwd, smem_back, smem_wg;
 };
 
@@ -1021,9 +1033,18 @@ TcPlan* tc_plan_create(const TcBuffers& b, char* err, size_t err_len)
         }
         const int m_in = ((int)ct + kTileM - 1) / kTileM;
         q.cols_wg = pow2_cols(m_in * k.c_out);
-        q.smem_fwd = 4 * ((size_t)kTileM * 128 + (size_t)k.c_out * 128) + kSmemAlign;
-        q.smem_back = 4 * ((size_t)kTileM * 128 + (size_t)k.c_prev * 128) + kSmemAlign;
-        q.smem_wg = 3 * ((size_t)(m_in * 2 + k.c_out / kBlockK) * kChunkPix * 128) + kSmemAlign;
+        // pipeline depth: as many stages as fit in about 208 KB (a stage of a narrow layer is small, and with only four
+        // of them in flight the copies' latency, not the tensor pipe, sets the pace)
+        auto pick = [](size_t stage_bytes, int lo, int mid, int hi) {
+            const size_t fit = ((size_t)208 * 1024) / stage_bytes;
+            return fit >= (size_t)hi ? hi : (fit >= (size_t)mid ? mid : lo);
+        };
+        const size_t st_fwd = (size_t)kTileM * 128 + (size_t)k.c_out * 128, st_back = (size_t)kTileM * 128 + (size_t)k.c_prev * 128,
+                     st_wg = (size_t)(m_in * 2 + k.c_out / kBlockK) * kChunkPix * 128;
+        q.stages_fwd = pick(st_fwd, 4, 6, 8); q.stages_back = pick(st_back, 4, 6, 8); q.stages_wg = pick(st_wg, 3, 4, 5);
+        q.smem_fwd = q.stages_fwd * st_fwd + kSmemAlign;
+        q.smem_back = q.stages_back * st_back + kSmemAlign;
+        q.smem_wg = q.stages_wg * st_wg + kSmemAlign;
         if (ok && q.cols_wg > 512) {
             snprintf(err, err_len, "a block with %d input and %d output channels needs %d TMEM columns (> 512)", (int)ct, k.c_out, q.cols_wg);
             ok = false;
@@ -1056,16 +1077,10 @@ TcPlan* tc_plan_create(const TcBuffers& b, char* err, size_t err_len)
         P->fwd1_persistent = use && P->smem_fwd1p <= (size_t)227 * 1024;
     }
     P->smem_wg1 = kWg1Stages * ((size_t)(m_last / P->msplit2) * 2 * kChunkPix * 128 + kClassPad * 128) + kSmemAlign;
-    size_t smem_fwd3 = 0, smem_back3 = 0, smem_wg3 = 0;
     if (nb) {
         P->chunks1 = ((b.w + kChunkW - 1) / kChunkW) * ((b.h + kChunkH - 1) / kChunkH);
         split_geometry(P->chunks1, 148 / 9, &P->per1, &P->split1);
         P->smem_dgrad = (size_t)(2 + P->c_last / kBlockK) * kClassPad * 128 + kSmemAlign;
-        for (int i = 0; i < nb; ++i) {
-            if (P->blk[i].smem_fwd > smem_fwd3) smem_fwd3 = P->blk[i].smem_fwd;
-            if (b.blk[i].pass_back && P->blk[i].smem_back > smem_back3) smem_back3 = P->blk[i].smem_back;
-            if (P->blk[i].smem_wg > smem_wg3) smem_wg3 = P->blk[i].smem_wg;
-        }
     }
     if (P->c_last / kBlockK > kMaxKBlocks || (!P->fwd1_persistent && P->smem_fwd1 > lim) || P->smem_wg1 > lim || P->smem_dgrad > lim) {
         snprintf(err, err_len, "shared memory per block exceeds 227 KB for these channel counts");
@@ -1084,12 +1099,13 @@ TcPlan* tc_plan_create(const TcBuffers& b, char* err, size_t err_len)
     if (!P->fwd1_persistent) e = allow((const void*)tc_fwd1x1_kernel, P->smem_fwd1);
     if (e == cudaSuccess && P->fwd1_persistent) e = allow((const void*)tc_fwd1x1p_kernel, P->smem_fwd1p);
     if (e == cudaSuccess) e = allow((const void*)tc_wgrad1x1_kernel<kWg1Stages>, P->smem_wg1);
-    if (nb) {
-        if (e == cudaSuccess) e = allow((const void*)tc_fwd3x3_kernel<4, 0>, smem_fwd3);
-        if (e == cudaSuccess && smem_back3) e = allow((const void*)tc_fwd3x3_kernel<4, 1>, smem_back3);
-        if (e == cudaSuccess) e = allow((const void*)tc_wgrad3x3_kernel<3>, smem_wg3);
-        if (e == cudaSuccess) e = allow((const void*)tc_dgrad_kernel, P->smem_dgrad);
+    for (int i = 0; i < nb; ++i) {
+        const TcBlockPlan& q = P->blk[i];
+        if (e == cudaSuccess) e = allow((const void*)fwd3_kernel<0>(q.stages_fwd), q.smem_fwd);
+        if (e == cudaSuccess && b.blk[i].pass_back) e = allow((const void*)fwd3_kernel<1>(q.stages_back), q.smem_back);
+        if (e == cudaSuccess) e = allow((const void*)wgrad3_kernel(q.stages_wg), q.smem_wg);
     }
+    if (nb && e == cudaSuccess) e = allow((const void*)tc_dgrad_kernel, P->smem_dgrad);
     if (e != cudaSuccess) { snprintf(err, err_len, "shared-memory attribute: %s", cudaGetErrorString(e)); delete P; return nullptr; }
     return P;
 }
@@ -1129,7 +1145,7 @@ int tc_forward_blocks(const TcPlan* P, int first, int last, cudaStream_t s, Stag
         const TcBlockPlan& q = P->blk[i];
         int grid, tail_split;
         tile_walk(P, total, k.c_out, &grid, &tail_split);
-        ST_REPEAT(t) launch_chain(b.chain_early != 0, tc_fwd3x3_kernel<4, 0>, dim3(grid), dim3(kFwd3Threads), q.smem_fwd, s,
+        ST_REPEAT(t) launch_chain(b.chain_early != 0, fwd3_kernel<0>(q.stages_fwd), dim3(grid), dim3(kFwd3Threads), q.smem_fwd, s,
             q.in_fwd, q.skip_fwd, k.c_prev / kBlockK, k.c_skip / kBlockK, q.w_map, q.w_map_q, tail_split, b.theta, b.n_params, k.b_off,
             k.out, k.relu_bits, (float*)nullptr, k.c_out, b.h, b.w, total, pow2_cols(k.c_out), b.err, skip, skip_stride);
         if (t) t->mark(kFwd3Names[i], s, st_repeats(t));
@@ -1186,7 +1202,7 @@ int tc_backward(const TcPlan* P, cudaStream_t s, StageTimer* t, const int* skip,
     for (int i = nb - 1; i >= 0 && b.blk[i].trained; --i) {
         const TcBlock& k = b.blk[i];
         const TcBlockPlan& q = P->blk[i];
-        ST_REPEAT(t) launch_chain(b.chain_early != 0, tc_wgrad3x3_kernel<3>, dim3(9 * P->split1, b.S), dim3(kThreadsTc), q.smem_wg, s,
+        ST_REPEAT(t) launch_chain(b.chain_early != 0, wgrad3_kernel(q.stages_wg), dim3(9 * P->split1, b.S), dim3(kThreadsTc), q.smem_wg, s,
             q.in_wg, q.skip_wg, k.c_prev / kBlockK, q.dout_wg, k.w_partials, k.c_prev + k.c_skip, k.c_out, b.h, b.w, P->chunks1, P->per1,
             P->split1, q.cols_wg, b.err, skip, skip_stride);
         if (t) t->mark(kWg3Names[i], s, st_repeats(t));
@@ -1197,7 +1213,7 @@ int tc_backward(const TcPlan* P, cudaStream_t s, StageTimer* t, const int* skip,
             const TcBlock& r = b.blk[i - 1];
             int grid, tail_split;
             tile_walk(P, total, k.c_prev, &grid, &tail_split);
-            ST_REPEAT(t) launch_chain(b.chain_early != 0, tc_fwd3x3_kernel<4, 1>, dim3(grid), dim3(kFwd3Threads), q.smem_back, s,
+            ST_REPEAT(t) launch_chain(b.chain_early != 0, fwd3_kernel<1>(q.stages_back), dim3(grid), dim3(kFwd3Threads), q.smem_back, s,
                 q.dout_fwd, q.dout_fwd, k.c_out / kBlockK, 0, q.wt_map, q.wt_map_q, tail_split, (const float*)nullptr, (int64_t)0, (int64_t)0,
                 r.dout, r.relu_bits, r.b_partials, k.c_prev, b.h, b.w, total, pow2_cols(k.c_prev), b.err, skip, skip_stride);
             if (t) t->mark("tc_dgrad3x3", s, st_repeats(t));

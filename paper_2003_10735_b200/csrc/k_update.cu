@@ -119,7 +119,7 @@ sgd_update_kernel(UpdateArgs a, int n_param_blocks, int64_t range_begin)
                 for (int L = 0; L < a.n_layers; ++L) {
                     const LayerUpdate& ly = a.layer[L];
                     const int64_t nw = (int64_t)ly.cout * ly.cin * ly.taps;
-                    if (i >= ly.w_off && i < ly.w_off + nw) { layer[e] = L; is_weight[e] = true; }
+                    if (i >= ly.w_off && i < ly.w_off + nw && !ly.streamed) { layer[e] = L; is_weight[e] = true; }
                     if (i >= ly.b_off && i < ly.b_off + ly.cout) { layer[e] = L; is_weight[e] = false; }
                 }
             }
@@ -279,22 +279,24 @@ static int launch_sgd_update_t(const UpdateArgs& a, cudaStream_t s)
     // large layers with partial sums go through the streaming kernel; everything else (small layers, biases,
     // loss) through the grouped kernel, which then starts after the streamed range
     int64_t range_begin = a.param_begin;
+    UpdateArgs g = a;                    // what the grouped kernel gets: streamed layers lose their partial sums there
     for (int L = 0; L < a.n_layers; ++L) {
         const LayerUpdate& ly = a.layer[L];
         const int64_t nw = (int64_t)ly.cout * ly.cin * ly.taps;
-        if (ly.w_partials && nw >= 65536 && ly.w_off == range_begin) {
+        if (ly.w_partials && nw >= 65536) {
             const bool vec = nw % 4 == 0 && ly.w_split_stride % 4 == 0 && ly.w_stream_stride % 4 == 0 &&
                              ((uintptr_t)ly.w_partials % 16 == 0);
             if (vec) launch_chain(a.chain_early != 0, sgd_update_stream_kernel<4, ADAM>, dim3((unsigned)((nw / 4 + 255) / 256), (unsigned)a.S), dim3(256), 0, s, a, L);
             else launch_chain(a.chain_early != 0, sgd_update_stream_kernel<1, ADAM>, dim3((unsigned)((nw + 255) / 256), (unsigned)a.S), dim3(256), 0, s, a, L);
-            range_begin = ly.w_off + nw;
+            if (ly.w_off == range_begin) range_begin = ly.w_off + nw;     // the grouped kernel starts behind leading streamed layers
+            g.layer[L].streamed = 1;                                       // ... and leaves the weights of later ones alone
             ++n_launches;
         }
     }
     int items = 1, max_split = 1;
     for (int L = 0; L < a.n_layers; ++L) {
         if (a.layer[L].b_partials) items += a.layer[L].cout;
-        if (a.layer[L].w_partials && a.layer[L].n_split > max_split) max_split = a.layer[L].n_split;
+        if (a.layer[L].w_partials && !g.layer[L].streamed && a.layer[L].n_split > max_split) max_split = a.layer[L].n_split;
     }
     const int n_red_blocks = (items + kUpdThreads / 32 - 1) / (kUpdThreads / 32);
     const int64_t n_rest = a.n_params - range_begin;
@@ -305,11 +307,11 @@ static int launch_sgd_update_t(const UpdateArgs& a, cudaStream_t s)
     const int n_param_blocks = (int)((n_rest + per - 1) / per);
     const dim3 grid((unsigned)(n_param_blocks + n_red_blocks), (unsigned)a.S);
     const dim3 blk(kUpdThreads);
-    if (G == 1 && E == 1) launch_chain(a.chain_early != 0, sgd_update_kernel<1, 1, ADAM>, grid, blk, 0, s, a, n_param_blocks, range_begin);
-    else if (G == 1) launch_chain(a.chain_early != 0, sgd_update_kernel<1, 4, ADAM>, grid, blk, 0, s, a, n_param_blocks, range_begin);
-    else if (G == 16) launch_chain(a.chain_early != 0, sgd_update_kernel<16, 1, ADAM>, grid, blk, 0, s, a, n_param_blocks, range_begin);
-    else if (E == 1) launch_chain(a.chain_early != 0, sgd_update_kernel<8, 1, ADAM>, grid, blk, 0, s, a, n_param_blocks, range_begin);
-    else launch_chain(a.chain_early != 0, sgd_update_kernel<8, 4, ADAM>, grid, blk, 0, s, a, n_param_blocks, range_begin);
+    if (G == 1 && E == 1) launch_chain(a.chain_early != 0, sgd_update_kernel<1, 1, ADAM>, grid, blk, 0, s, g, n_param_blocks, range_begin);
+    else if (G == 1) launch_chain(a.chain_early != 0, sgd_update_kernel<1, 4, ADAM>, grid, blk, 0, s, g, n_param_blocks, range_begin);
+    else if (G == 16) launch_chain(a.chain_early != 0, sgd_update_kernel<16, 1, ADAM>, grid, blk, 0, s, g, n_param_blocks, range_begin);
+    else if (E == 1) launch_chain(a.chain_early != 0, sgd_update_kernel<8, 1, ADAM>, grid, blk, 0, s, g, n_param_blocks, range_begin);
+    else launch_chain(a.chain_early != 0, sgd_update_kernel<8, 4, ADAM>, grid, blk, 0, s, g, n_param_blocks, range_begin);
     return n_launches;
 }
 

@@ -168,6 +168,7 @@ struct LayerUpdate {
     bf16* shadow_t;            // nullptr, or a second bf16 copy [9][c_take][cout] with the taps mirrored and the channels
     int64_t shadow_t_stream_stride;   // transposed, for the first c_take input channels: what the gradient passed back
     int c_take;                //   through this 3x3 layer multiplies
+    int streamed;              // set by the launcher: the streaming kernel updates this layer's weights, the grouped one skips them
 };
 struct UpdateArgs {
     float* theta;      // [S][n_params]   internal order

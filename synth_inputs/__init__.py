@@ -22,7 +22,7 @@ import numpy as np
 __all__ = [
     "WorkloadConfig", "CONFIGS", "get_config", "frozen_features", "voronoi_map",
     "teacher_logits", "head_param_shapes", "head_param_count", "initial_head_params",
-    "key_frame_indices",
+    "key_frame_indices", "initial_stack_params", "skip_features",
 ]
 
 
@@ -46,6 +46,8 @@ class WorkloadConfig:
     n_frames: int = 1        # frames in the clip (drift workloads)
     key_stride: int = 0      # key frame every key_stride frames (0: only frame 0)
     drift: int = 0           # per-frame translation step in pixels
+    blocks: Tuple[Tuple[int, int], ...] = ()   # a stack of student blocks: (output channels, skip-input channels) each
+    first_trained: int = 0   # blocks before this index are frozen
 
     @property
     def frame_h(self) -> int:
@@ -68,6 +70,9 @@ CONFIGS = {
                       momentum=0.9, gemm_precision=1, n_regions=128, teacher="blur"),
     5: WorkloadConfig("720p_16_streams", 256, 0, 21, 180, 320, k_steps=8, lr=0.01, momentum=0.9,
                       n_streams=16, gemm_precision=1, n_regions=64, teacher="onehot_noise"),
+    # the trained back part in the paper's shape (Section 5.2): two blocks with skip inputs, then the classifier
+    6: WorkloadConfig("720p_stack_sb5_sb6", 128, 0, 21, 180, 320, k_steps=8, lr=0.005, momentum=0.9,
+                      gemm_precision=1, n_regions=64, teacher="onehot_noise", blocks=((128, 64), (64, 64))),
 }
 
 
@@ -219,6 +224,25 @@ def initial_head_params(c_in: int, c_hidden: int, n_classes: int, seed: int) -> 
         parts.append((rng.standard_normal(ws, dtype=np.float32) * std).ravel())
         parts.append(np.zeros(bs, dtype=np.float32))
     return np.concatenate(parts)
+
+
+def initial_stack_params(c_in: int, blocks, n_classes: int, seed: int) -> np.ndarray:
+    """The same initialisation for a stack of blocks: per block the 3x3 weight [c_out][c_prev + c_skip][3][3] and its
+    bias, then the 1x1 classifier; one flat fp32 buffer in forward order."""
+    rng = np.random.default_rng(seed)
+    parts, prev = [], c_in
+    shapes = [(co, prev_ + cs, 3) for (co, cs), prev_ in zip(blocks, [c_in] + [b[0] for b in blocks[:-1]])]
+    shapes.append((n_classes, blocks[-1][0] if blocks else c_in, 1))
+    for co, ci, k in shapes:
+        std = np.float32(np.sqrt(2.0 / (ci * k * k)))
+        parts.append((rng.standard_normal((co, ci, k, k), dtype=np.float32) * std).ravel())
+        parts.append(np.zeros(co, dtype=np.float32))
+    return np.concatenate(parts)
+
+
+def skip_features(cfg: WorkloadConfig, block: int, seed: int) -> np.ndarray:
+    """Skip input of one block: a feature map of the frozen front part, drawn like its output."""
+    return frozen_features(cfg.blocks[block][1], cfg.feat_h, cfg.feat_w, 5000 + 10 * seed + block)
 
 
 def stream_inputs(cfg: WorkloadConfig, stream: int = 0, frame: int = 0):

@@ -179,3 +179,48 @@ def test_stack_two_streams_and_a_second_key_frame():
         sl = heads[s].trained_slice()
         assert rel_l2(got - probs[s][3][sl], heads[s].theta[sl].astype(np.float64) - probs[s][3][sl]) <= 2e-2
     st.st_destroy(ctx)
+
+
+def test_stack_workload_full_width_band_and_full_frame():
+    """The stack workload (two blocks with skip inputs, 128 -> 128 -> 64 -> 21) at full width: a band of rows against
+    the oracle over K = 4 steps with momentum, then the whole 720p frame through its invariants."""
+    full = si.get_config(6)
+    blocks, C = [tuple(b) for b in full.blocks], full.n_classes
+    theta = si.initial_stack_params(full.c_in, blocks, C, 1000)
+    # ---- a band the oracle finishes in seconds
+    rows, K = 10, 4
+    cfg = si.WorkloadConfig("band", full.c_in, 0, C, rows, full.feat_w, n_regions=24, teacher="onehot_noise", blocks=full.blocks)
+    feat = si.frozen_features(cfg.c_in, rows, cfg.feat_w, 3)
+    skips = [si.skip_features(cfg, b, 3) for b in range(2)]
+    T = si.teacher_logits(cfg, stream=1)
+    ctx = make_ctx(cfg.c_in, blocks, C, rows, cfg.feat_w, theta, 0, lr=full.lr, mu=full.momentum)
+    feed(ctx, 0, feat, skips, T)
+    loss = np.zeros(K, np.float32)
+    st.st_distill_step(ctx, K, loss)
+    lab = oracle.teacher_labels(T)
+    plain = oracle.StackHead(cfg.c_in, blocks, C, lr=full.lr, momentum=full.momentum, theta=theta)
+    quant = oracle.StackHead(cfg.c_in, blocks, C, lr=full.lr, momentum=full.momentum, theta=theta, quantize_bf16=True)
+    ref = [oracle.stack_distill_step(plain, feat, skips, lab)[0] for _ in range(K)]
+    q = [oracle.stack_distill_step(quant, feat, skips, lab)[0] for _ in range(K)]
+    np.testing.assert_allclose(loss, q, rtol=3e-5)
+    np.testing.assert_allclose(loss, ref, rtol=1e-4 * np.sqrt(full.feat_h / rows))
+    got = np.empty(ctx.n_params, np.float32)
+    st.st_pack_updated_params(ctx, 0, got)
+    assert rel_l2(got - theta, quant.theta.astype(np.float64) - theta) <= 5e-3
+    assert rel_l2(got - theta, plain.theta.astype(np.float64) - theta) <= 2e-2
+    st.st_destroy(ctx)
+    # ---- the whole frame
+    K = full.k_steps
+    ctx = make_ctx(full.c_in, blocks, C, full.feat_h, full.feat_w, theta, 0, lr=full.lr, mu=full.momentum)
+    T = si.teacher_logits(full)
+    feed(ctx, 0, si.frozen_features(full.c_in, full.feat_h, full.feat_w, 0), [si.skip_features(full, b, 0) for b in range(2)], T)
+    loss = np.zeros(K, np.float32)
+    conf = np.zeros((K, C, C), np.int64)
+    st.st_distill_step(ctx, K, loss, conf)
+    lab = oracle.teacher_labels(T)
+    assert np.isfinite(loss).all() and loss[-1] < loss[0]
+    for k in range(K):
+        assert conf[k].sum() == lab.size
+        np.testing.assert_array_equal(conf[k].sum(1), np.bincount(lab.ravel(), minlength=C))
+    assert st.st_pack_updated_params(ctx, 0, np.empty(ctx.n_params, np.float32)) == theta.size * 4
+    st.st_destroy(ctx)
