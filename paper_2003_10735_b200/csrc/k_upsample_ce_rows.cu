@@ -128,6 +128,26 @@ __device__ __forceinline__ void pass1(const RowCtx& rc, const float (&sk)[4], fl
 // X23[k] = (E(2,k), E(3,k))).  Returns the largest corner difference
 // in the logits' own units (the caller leaves the fast path if a class changes by more than kFastRange log2-units across
 // the cell: the progressions would lose their small terms).  q points at raw logits; M is in log2 units.
+// The four quantities everything else is a product of: X01[0] = (E(0,0), E(1,0)), X23[0] = (E(2,0), E(3,0)) and the
+// per-row ratios between neighbouring pixels q01 = (q_0, q_1), q23 = (q_2, q_3), E(r,k) = E(r,0) q_r^k.
+__device__ __forceinline__ float cell_bases(const float* q, float M, float2& x01, float2& x23, float2& q01, float2& q23)
+{
+    const float a = q[0], b = q[TZ_W];
+    const float ar = __shfl_down_sync(0xffffffffu, a, 1), br = __shfl_down_sync(0xffffffffu, b, 1);
+    const float p = b - a, qq = br - ar, e0 = ar - a;
+    const float qp = qq - p;
+    const float wv = fmaf(qp, 0.125f, e0);
+    const float A = fmaf(wv, 0.125f, fmaf(p, 0.125f, a));
+    const float E00 = ex2_approx(fmaf(A, kLog2e, -M)), QB = ex2_approx((0.25f * kLog2e) * wv),
+                TG = ex2_approx(fmaf(qp, 0.03125f * kLog2e, (0.25f * kLog2e) * p)), SD = ex2_approx((0.0625f * kLog2e) * qp);
+    const float TG2 = TG * TG, SD2 = SD * SD;
+    q01 = make_float2(QB, QB * SD);
+    q23 = __fmul2_rn(q01, make_float2(SD2, SD2));
+    x01 = make_float2(E00, E00 * TG);
+    x23 = __fmul2_rn(x01, make_float2(TG2, TG2));
+    return fmaxf(fabsf(p), fmaxf(fabsf(qq), fabsf(e0)));
+}
+
 __device__ __forceinline__ float cell_exponentials(const float* q, float M, float2 (&X01)[4], float2 (&X23)[4])
 {
     const float a = q[0], b = q[TZ_W];
@@ -532,15 +552,18 @@ upsample_ce_rows_kernel(UpsampleCeArgs a, const __grid_constant__ CUtensorMap z_
             const float2 bw01 = make_float2(bw[0], bw[1]), bw23 = make_float2(bw[2], bw[3]);
 #pragma unroll kClassUnroll
             for (int c = 0; c < CB; ++c) {
-                float2 X01[4], X23[4];
-                cell_exponentials(rc.za + c * TZ, rc.M, X01, X23);
-                float2 aL01 = __fmul2_rn(WL01[3], X01[3]), aL23 = __fmul2_rn(WL23[3], X23[3]);
-                float2 aR01 = __fmul2_rn(WR01[3], X01[3]), aR23 = __fmul2_rn(WR23[3], X23[3]);
+                // a row's four exponentials are E(r,0) q_r^k, so the row's weighted sum is E(r,0) times a cubic in q_r
+                // with the pixel weights as coefficients: Horner's rule, the progression itself is not formed again
+                float2 x01, x23, q01, q23;
+                cell_bases(rc.za + c * TZ, rc.M, x01, x23, q01, q23);
+                float2 aL01 = WL01[3], aL23 = WL23[3], aR01 = WR01[3], aR23 = WR23[3];
 #pragma unroll
                 for (int k = 2; k >= 0; --k) {
-                    aL01 = __ffma2_rn(WL01[k], X01[k], aL01); aL23 = __ffma2_rn(WL23[k], X23[k], aL23);
-                    aR01 = __ffma2_rn(WR01[k], X01[k], aR01); aR23 = __ffma2_rn(WR23[k], X23[k], aR23);
+                    aL01 = __ffma2_rn(aL01, q01, WL01[k]); aL23 = __ffma2_rn(aL23, q23, WL23[k]);
+                    aR01 = __ffma2_rn(aR01, q01, WR01[k]); aR23 = __ffma2_rn(aR23, q23, WR23[k]);
                 }
+                aL01 = __fmul2_rn(aL01, x01); aL23 = __fmul2_rn(aL23, x23);
+                aR01 = __fmul2_rn(aR01, x01); aR23 = __fmul2_rn(aR23, x23);
                 // own cell's left part + left cell's right part, per row
                 const float2 hs01 = __fadd2_rn(aL01, make_float2(__shfl_up_sync(0xffffffffu, aR01.x, 1), __shfl_up_sync(0xffffffffu, aR01.y, 1)));
                 const float2 hs23 = __fadd2_rn(aL23, make_float2(__shfl_up_sync(0xffffffffu, aR23.x, 1), __shfl_up_sync(0xffffffffu, aR23.y, 1)));
