@@ -500,7 +500,9 @@ def run_ours(args, cfg):
             # no wait; launched back to back) and the whole call with the mean IoU read back by the host
             rng = np.random.default_rng(0)
             lab_map = si.voronoi_map(H, W, cfg.n_regions, C, 2000)
-            noisy = np.where(rng.random((H, W)) < 0.9, lab_map, rng.integers(0, C, (H, W))).astype(np.uint8)
+            # a prediction like a trained student's: the same regions with their borders a few pixels off, plus 1 % of stray pixels
+            moved = np.roll(lab_map, (3, 5), axis=(0, 1))
+            noisy = np.where(rng.random((H, W)) < 0.99, moved, rng.integers(0, C, (H, W))).astype(np.uint8)
             m_coh = [torch.from_numpy(lab_map).cuda(), torch.from_numpy(noisy).cuda()]
             m_rnd = [torch.randint(0, C, (H, W), dtype=torch.uint8, device="cuda") for _ in range(2)]
             agree = {}
@@ -509,6 +511,14 @@ def run_ours(args, cfg):
                 t_c = timed(lambda r: st.st_agreement(ctx, 0, a, b, conf_d[0]), reps=20)
                 agree[name] = {"kernel_us": t_k * 1e3, "call_us": t_c * 1e3, "kernel_gbs": 2 * P / t_k / 1e6,
                                "kernel_frac_of_hbm": 2 * P / t_k / 1e6 / hbm}
+            # the same counting kernel on sixteen frames' worth of pixels in one launch (the no-context entry point takes
+            # any length): what the kernel reaches when it has more than one wave of work
+            big = [m.repeat(16, 1) for m in m_coh]
+            t_big = timed(lambda r: st.st_agreement_noalloc(big[1], big[0], C, stream.cuda_stream, conf_d[0], miou_d[0:1]), reps=20)
+            agree["coherent_masks_16_frames"] = {"kernel_us": t_big * 1e3, "kernel_gbs": 32 * P / t_big / 1e6,
+                                                 "kernel_frac_of_hbm": 32 * P / t_big / 1e6 / hbm,
+                                                 "note": "memset + counting kernel + mean-IoU kernel of st_agreement_noalloc"}
+            del big
             t_own = timed(lambda r: st.st_agreement(ctx, 0, None, None, conf_d[0], miou_out=miou_d[0:1]), reps=50)
             agree["student_mask_fused"] = {"kernel_us": t_own * 1e3, "note": "arg-max of the upsampled logits + confusion + mean IoU, forward reused"}
             kernels["agreement"] = {"ms": agree["coherent_masks"]["kernel_us"] / 1e3, "bound": "latency", "per_key_frame": S, **agree}
