@@ -260,9 +260,9 @@ cudaError_t prepare_upsample_ce(int C)
     return cudaFuncSetAttribute(upsample_ce_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
 }
 
-void launch_upsample_ce(const UpsampleCeArgs& a, const CUtensorMap* z_map, cudaStream_t s)
+void launch_upsample_ce(const UpsampleCeArgs& a, const CUtensorMap* z_map, cudaStream_t s, const CUtensorMap* x_map, const CUtensorMap* w_map)
 {
-    if (upsample_ce_rows_supported(a.C)) { launch_upsample_ce_rows(a, z_map, s); return; }
+    if (upsample_ce_rows_supported(a.C)) { launch_upsample_ce_rows(a, z_map, s, x_map, w_map); return; }
     size_t smem = 0;
     const int chunk = chunk_classes(a.C, &smem);
     dim3 grid((unsigned)((a.w + NX - 1) / NX), (unsigned)((a.h + NY - 1) / NY), (unsigned)a.S);

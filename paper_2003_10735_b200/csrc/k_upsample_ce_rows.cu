@@ -44,7 +44,14 @@ namespace {
 
 constexpr int RN_Y = 7, RN_X = 30;
 constexpr int R_WARPS = RN_Y + 1, R_THREADS = R_WARPS * 32;
-constexpr int TZ_H = RN_Y + 2, TZ_W = 36, TZ = TZ_H * TZ_W;   // tile rows hold 36 columns: 32 used, starting at a multiple of 4
+constexpr int TZ_H = RN_Y + 2;
+// Columns of a tile row (template parameter TW of everything below): 36 when the logits are fetched from global memory
+// (32 used, starting at a multiple of 4 so that rows are whole 16-byte vectors), 32 when the block computes its logits
+// itself (kTwFused).
+constexpr int kTwLoad = 36, kTwFused = 32;
+// The block computes its own logits: one 64-channel slice of the feature tile (9 x 32 pixels, 128 bytes each) per stage
+constexpr uint32_t kStageBytes = TZ_H * kTwFused * 128, kWeightBytes = kClassPad * 128;
+constexpr int kFusedStages = 2, kFusedTmemCols = 128, kFusedMaxKBlocks = 4;
 constexpr float kLog2e = 1.4426950408889634f, kLn2 = 0.6931471805599453f;
 // Classes per iteration of the two fast-path class sweeps.  The sweeps are rolled loops: unrolled over all classes
 // they were ~70 KB of straight-line code that every warp ran through once, and instruction fetch was the main stall.
@@ -83,17 +90,22 @@ __host__ __device__ constexpr uint32_t corner_weights(int row_eighths, bool righ
                  : (uint32_t)(row_eighths * 7) | (uint32_t)(row_eighths * 5) << 8 | (uint32_t)(row_eighths * 3) << 16 | (uint32_t)(row_eighths * 1) << 24;
 }
 
+// A lane reads its cell's corner logits at clamped tile coordinates, so the clamped borders (node row -1 is row 0, node
+// column w is column w-1, ...) need no copies in the tile.
 struct RowCtx {
-    const float* za;     // own column, upper node row, class 0
+    const float* za;     // own (clamped) node column, upper (clamped) node row, class 0
+    int dq;              // elements from there to the lower node row: the tile's row pitch, or 0 where both rows clamp to one
+    int dr;              // ... to the right-hand node column: 1, or 0 at the right border
     float ly;            // weight toward the lower node row
     float M;             // warp-uniform shift
 };
 
 // interpolated, shifted logits of the lane's four pixels for class c
-template <bool SHIFT>
+template <bool SHIFT, int TW>
 __device__ __forceinline__ void pixel_logits(const RowCtx& rc, int c, const float (&sk)[4], float (&u)[4])
 {
-    const float a = rc.za[c * TZ], b = rc.za[c * TZ + TZ_W];
+    constexpr int TZ = TZ_H * TW;
+    const float a = rc.za[c * TZ], b = rc.za[c * TZ + rc.dq];
     const float vl = fmaf(fmaf(rc.ly, b - a, a), kLog2e, -rc.M);
     const float vr = __shfl_down_sync(0xffffffffu, vl, 1);
     const float d = vr - vl;
@@ -104,7 +116,7 @@ __device__ __forceinline__ void pixel_logits(const RowCtx& rc, int c, const floa
     }
 }
 
-template <int CB, bool CONF, bool SHIFT>
+template <int CB, bool CONF, bool SHIFT, int TW>
 __device__ __forceinline__ void pass1(const RowCtx& rc, const float (&sk)[4], float (&Zs)[4], uint32_t (&arg)[4])
 {
     float best[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};
@@ -112,7 +124,7 @@ __device__ __forceinline__ void pass1(const RowCtx& rc, const float (&sk)[4], fl
 #pragma unroll
     for (int c = 0; c < CB; ++c) {
         float u[4];
-        pixel_logits<SHIFT>(rc, c, sk, u);
+        pixel_logits<SHIFT, TW>(rc, c, sk, u);
 #pragma unroll
         for (int k = 0; k < 4; ++k) {
             if (CONF && !SHIFT) { if (u[k] > best[k]) { best[k] = u[k]; arg[k] = c; } }
@@ -122,7 +134,7 @@ __device__ __forceinline__ void pass1(const RowCtx& rc, const float (&sk)[4], fl
 }
 
 // The 16 exponentials exp2(u(r,k) - M) of one class inside the lane's cell, u bilinear between the four
-// corner logits (own column: rows i, i+1 from shared memory; right column from the next lane).
+// corner logits (own column: the two node rows from shared memory, dq elements apart; right column from the next lane).
 // With ly_r = (2r+1)/8 and fr_k = (2k+1)/8:  u(r,k) = A + B k + G r + D k r, so the values are geometric
 // progressions along k and r: 4 exp2 and 12 multiplications (8 of them packed: X01[k] = (E(0,k), E(1,k)),
 // X23[k] = (E(2,k), E(3,k))).  Returns the largest corner difference
@@ -130,9 +142,9 @@ __device__ __forceinline__ void pass1(const RowCtx& rc, const float (&sk)[4], fl
 // the cell: the progressions would lose their small terms).  q points at raw logits; M is in log2 units.
 // The four quantities everything else is a product of: X01[0] = (E(0,0), E(1,0)), X23[0] = (E(2,0), E(3,0)) and the
 // per-row ratios between neighbouring pixels q01 = (q_0, q_1), q23 = (q_2, q_3), E(r,k) = E(r,0) q_r^k.
-__device__ __forceinline__ float cell_bases(const float* q, float M, float2& x01, float2& x23, float2& q01, float2& q23)
+__device__ __forceinline__ float cell_bases(const float* q, int dq, float M, float2& x01, float2& x23, float2& q01, float2& q23)
 {
-    const float a = q[0], b = q[TZ_W];
+    const float a = q[0], b = q[dq];
     const float ar = __shfl_down_sync(0xffffffffu, a, 1), br = __shfl_down_sync(0xffffffffu, b, 1);
     const float p = b - a, qq = br - ar, e0 = ar - a;
     const float qp = qq - p;
@@ -148,9 +160,9 @@ __device__ __forceinline__ float cell_bases(const float* q, float M, float2& x01
     return fmaxf(fabsf(p), fmaxf(fabsf(qq), fabsf(e0)));
 }
 
-__device__ __forceinline__ float cell_exponentials(const float* q, float M, float2 (&X01)[4], float2 (&X23)[4])
+__device__ __forceinline__ float cell_exponentials(const float* q, int dq, float M, float2 (&X01)[4], float2 (&X23)[4])
 {
-    const float a = q[0], b = q[TZ_W];
+    const float a = q[0], b = q[dq];
     const float ar = __shfl_down_sync(0xffffffffu, a, 1), br = __shfl_down_sync(0xffffffffu, b, 1);
     const float p = b - a, qq = br - ar, e0 = ar - a;
     const float qp = qq - p;
@@ -175,14 +187,14 @@ __device__ __forceinline__ float cell_exponentials(const float* q, float M, floa
 // pass 2 of one row on the slow path: the exponentials are formed again, multiplied by the adjoint interpolation
 // weights / Z, the right-hand part goes to the next lane, and the row is added into this thread's shared-memory
 // slots of the upper and the lower node row
-template <int CB>
+template <int CB, int TW>
 __device__ __forceinline__ void pass2_slow(const RowCtx& rc, const float (&sk)[4], const float (&wl)[4], const float (&wr)[4],
                                            float tw, float bw, float2* my_acc, int C)
 {
 #pragma unroll
     for (int c = 0; c < CB; ++c) {
         float u[4];
-        pixel_logits<true>(rc, c, sk, u);
+        pixel_logits<true, TW>(rc, c, sk, u);
         const float e0 = ex2_approx(u[0]), e1 = ex2_approx(u[1]), e2 = ex2_approx(u[2]), e3 = ex2_approx(u[3]);
         const float aL = fmaf(wl[0], e0, fmaf(wl[1], e1, fmaf(wl[2], e2, wl[3] * e3)));
         const float aR = fmaf(wr[0], e0, fmaf(wr[1], e1, fmaf(wr[2], e2, wr[3] * e3)));
@@ -194,19 +206,24 @@ __device__ __forceinline__ void pass2_slow(const RowCtx& rc, const float (&sk)[4
     }
 }
 
-template <int CB, bool CONF>
+template <int CB, bool CONF, int TW>
 __global__ void __launch_bounds__(R_THREADS, 2)
-upsample_ce_rows_kernel(UpsampleCeArgs a, const __grid_constant__ CUtensorMap z_map)
+upsample_ce_rows_kernel(UpsampleCeArgs a, const __grid_constant__ CUtensorMap z_map, const __grid_constant__ CUtensorMap x_map,
+                        const __grid_constant__ CUtensorMap w_map)
 {
+    constexpr bool FUSED = TW == kTwFused;      // the block multiplies its own logit tile (Forward of Algorithm 1 for a 1x1 classifier)
+    constexpr int TZ_W = TW, TZ = TZ_H * TW;
     extern __shared__ __align__(128) float smem_r[];
     const int C = a.C, h = a.h, w = a.w, H = h * kUp, W = w * kUp;
-    float* zt = smem_r;                         // [CB][TZ_H][36]   logits, borders replicated; classes >= C hold -1e30
-                                                //                  (their exponentials are 0)
-    int* corr = (int*)(zt + CB * TZ);           // [C][TZ_H][36]    -64 * (adjoint of onehot)
+    // [CB][TZ_H][TW]  logits, borders replicated; classes >= C hold -1e30 (their exponentials are 0).  FUSED: the feature
+    // stages and the classifier weights lie over this and the next two arrays until the multiplication has finished.
+    float* zt = FUSED ? (float*)(((uintptr_t)smem_r + 1023) & ~(uintptr_t)1023) : smem_r;
+    int* corr = (int*)(zt + CB * TZ);           // [C][TZ_H][TW]    -64 * (adjoint of onehot)
     float2* acc = (float2*)(corr + C * TZ);     // [R_WARPS][C][32] (x, y): the cell's pull on its upper / lower node row
     unsigned int* hist = (unsigned int*)(acc + R_WARPS * C * 32);   // [C][C] (CONF): the block's share of the confusion matrix
-    __shared__ float red[R_WARPS], red_m[R_WARPS];
-    __shared__ __align__(8) uint64_t tile_bar;
+    __shared__ float red[R_WARPS], red_m[R_WARPS], sbias[kClassPad];
+    __shared__ __align__(8) uint64_t tile_bar, mm_bar[2 * kFusedStages + 2];   // FUSED: full[2], empty[2], weights, done
+    __shared__ uint32_t tmem_slot, gave_up;
 
     // Launch order: the last block row first, then rows 0, 1, ...  Blocks at the frame border do extra work, and the
     // blocks that reach an SM first finish earlier than their later companions, so the border rows go first.
@@ -221,7 +238,7 @@ upsample_ce_rows_kernel(UpsampleCeArgs a, const __grid_constant__ CUtensorMap z_
     // ---- tile: node rows y0-1 .. y0+RN_Y, node columns xa .. xa+35 where xa = (x0-1) rounded down to a
     // multiple of 4 (so that rows are fetched as 16-byte vectors), clamped at the borders, scaled by
     // log2(e).  Fully unrolled: all of a thread's loads are in flight together.
-    const bool vec_ok = (w % 4 == 0) && ((uintptr_t)z % 16 == 0);
+    const bool vec_ok = !FUSED && (w % 4 == 0) && ((uintptr_t)z % 16 == 0);
     const int xa = vec_ok ? ((x0 - 1) & ~3) : x0 - 1;      // x0-1 >= -1; (-1 & ~3) = -4
     const int off = (x0 - 1) - xa;                         // column of node x0-1 inside the tile
     const int i = y0 - 1 + wi;                  // cell row: frame rows 4i+2 .. 4i+5, node rows (i, i+1)
@@ -259,7 +276,159 @@ upsample_ce_rows_kernel(UpsampleCeArgs a, const __grid_constant__ CUtensorMap z_
 #pragma unroll
         for (int r = 0; r < 4; ++r) { hv[r] = (labw[r] >> 7) & 0x01010101u; labw[r] &= 0x7f7f7f7fu; }
     }
+    // Node rows above 0 / below h-1 and node columns left of 0 / right of w-1 repeat the border row / column (the tile
+    // holds something else there: zeros from the tile copy, or the bare bias from the block's own multiplication).
+    auto replicate_borders = [&]() {
+        float4* zt4 = reinterpret_cast<float4*>(zt);
+        const bool edge_rows = y0 == 0 || y0 + RN_Y > h - 1, edge_cols = xa < 0 || xa + TZ_W > w;
+        if (edge_rows) {                                   // block-uniform: node rows above 0 / below h-1 repeat the border row
+            const int j_lo = y0 == 0 ? 1 : 0;              // first tile row inside the map
+            const int j_hi = min(TZ_H - 1, h - y0);        // last one
+            const int n_out = TZ_H - (j_hi - j_lo + 1);    // rows to fill: 0 .. j_lo-1 and j_hi+1 .. TZ_H-1
+            for (int e = tid; e < C * n_out * (TZ_W / 4); e += R_THREADS) {
+                const int c = e / (n_out * (TZ_W / 4)), r = (e / (TZ_W / 4)) % n_out, x4 = e % (TZ_W / 4);
+                const int j = r < j_lo ? r : j_hi + 1 + (r - j_lo);
+                const int jc = j < j_lo ? j_lo : j_hi;
+                zt4[(c * TZ + j * TZ_W) / 4 + x4] = zt4[(c * TZ + jc * TZ_W) / 4 + x4];
+            }
+            __syncthreads();
+        }
+        if (edge_cols) {                                   // node columns left of 0 / right of w-1 repeat the border column
+            const int x_lo = xa < 0 ? -xa : 0;             // first tile column inside the map
+            const int x_hi = min(TZ_W - 1, w - 1 - xa);    // last one
+            const int n_out = TZ_W - (x_hi - x_lo + 1);
+            for (int e = tid; e < C * TZ_H * n_out; e += R_THREADS) {
+                const int row = e / n_out, r = e % n_out;  // row = c * TZ_H + j
+                const int x = r < x_lo ? r : x_hi + 1 + (r - x_lo);
+                zt[row * TZ_W + x] = zt[row * TZ_W + (x < x_lo ? x_lo : x_hi)];
+            }
+            __syncthreads();
+        }
+    };
     float m_loc = -INFINITY;                               // largest logit of this thread's share of the tile
+    uint32_t tmem = 0;                                     // FUSED: the block's tensor memory (given back at the very end)
+    if constexpr (FUSED) {
+        // ---- Forward for a 1x1 classifier, inside the block: z[pix][c] = b[c] + sum_k X[pix][k] W[c][k] for the 9 x 32
+        // nodes of the tile.  The feature tile arrives in 64-channel slices (one 4-d tile copy each, rows and columns
+        // outside the map arrive as zeros) through a ring of two stages, the classifier weights in one barrier's worth of
+        // copies; one thread issues three 128 x 32 x 16 tcgen05 multiplications per 16 channels (pixel rows 288 .. 383 of
+        // the third one read whatever follows the stage: their results are never looked at), the accumulators (fp32, in
+        // tensor memory) are drained into the logit tile by all warps.
+        const uint32_t ring = tc::smem_u32(zt), w_base = ring + kFusedStages * kStageBytes;
+        const uint32_t bar0 = tc::smem_u32(&mm_bar[0]);
+        auto full_bar = [&](int st) { return bar0 + 8u * (uint32_t)st; };
+        auto empty_bar = [&](int st) { return bar0 + 8u * (uint32_t)(kFusedStages + st); };
+        const uint32_t w_bar = bar0 + 8u * (2 * kFusedStages), done_bar = w_bar + 8u;
+        if (wi == 0) tc::tmem_alloc(tc::smem_u32(&tmem_slot), kFusedTmemCols);
+        if (tid == 0) {
+            for (int k = 0; k < 2 * kFusedStages + 2; ++k) tc::mbar_init(bar0 + 8u * (uint32_t)k, 1);
+            gave_up = 0;
+            tc::fence_barrier_init();
+        }
+        tc::tc_fence_before_sync();
+        __syncthreads();
+        tc::tc_fence_after_sync();
+        tmem = tmem_slot;
+        const int kblocks = a.kblocks;
+        // x_early: the kernel before this one on the stream (the previous iteration's update) does not write the features,
+        // and this launch may have started while that one still runs: the first slices are fetched before the wait
+        const int n_pre = a.x_early ? min(kFusedStages, kblocks) : 0;
+        if (tid == 0)
+            for (int kb = 0; kb < n_pre; ++kb) {
+                tc::mbar_expect_tx(full_bar(kb), kStageBytes);
+                tc::tma_load_4d(ring + kb * kStageBytes, &x_map, full_bar(kb), kb * 64, x0 - 1, y0 - 1, s);
+            }
+        pdl_wait();                                        // the weights come from the previous kernel of the stream
+        if (a.skip && a.skip[(int64_t)s * a.skip_stride]) {           // this stream's training loop has ended (block-uniform)
+            if (tid == 0)                                   // copies already on their way land before shared memory is given back
+                for (int kb = 0; kb < n_pre; ++kb) tc::mbar_wait(full_bar(kb), 0, a.err, tc::kWaitFull);
+            tc::tc_fence_before_sync();
+            __syncthreads();
+            if (wi == 0) tc::tmem_dealloc(tmem, kFusedTmemCols);
+            return;
+        }
+        if (tid < kClassPad) sbias[tid] = tid < C ? a.theta[(int64_t)s * a.n_params + a.b_off + tid] : 0.f;
+        bool ok = true;
+        if (tid == 0) {
+            tc::mbar_expect_tx(w_bar, (uint32_t)kblocks * kWeightBytes);
+            for (int kb = 0; kb < kblocks; ++kb) tc::tma_load_3d(w_base + kb * kWeightBytes, &w_map, w_bar, kb * 64, 0, s);
+            for (int kb = n_pre; kb < kblocks && ok; ++kb) {
+                const int st = kb % kFusedStages;
+                if (kb >= kFusedStages) ok = tc::mbar_wait(empty_bar(st), ((kb / kFusedStages) - 1) & 1, a.err, tc::kWaitEmpty);
+                if (ok) {
+                    tc::mbar_expect_tx(full_bar(st), kStageBytes);
+                    tc::tma_load_4d(ring + st * kStageBytes, &x_map, full_bar(st), kb * 64, x0 - 1, y0 - 1, s);
+                }
+            }
+        } else if (tid == 32) {
+            constexpr uint32_t idesc = tc::instr_desc(128, kClassPad, 0, 0);
+            ok = tc::mbar_wait(w_bar, 0, a.err, tc::kWaitFull);
+            for (int kb = 0; kb < kblocks && ok; ++kb) {
+                const int st = kb % kFusedStages;
+                ok = tc::mbar_wait(full_bar(st), (kb / kFusedStages) & 1, a.err, tc::kWaitFull);
+                if (!ok) break;
+                tc::tc_fence_after_sync();
+#pragma unroll
+                for (int m = 0; m < 3; ++m)
+#pragma unroll
+                    for (int k = 0; k < 4; ++k)
+                        tc::umma(tmem + m * kClassPad, tc::smem_desc(ring + st * kStageBytes + m * (128 * 128) + k * 32, 16, 1024),
+                                 tc::smem_desc(w_base + kb * kWeightBytes + k * 32, 16, 1024), idesc, (kb | k) != 0);
+                tc::umma_commit(empty_bar(st));
+            }
+            if (!ok) gave_up = 1;
+            tc::umma_commit(done_bar);
+        }
+        __syncwarp();
+        ok = tc::mbar_wait(done_bar, 0, a.err, tc::kWaitDone);
+        tc::tc_fence_after_sync();
+        if (!__syncthreads_and(ok) || gave_up) {           // block-uniform: a wait ran out; nothing is written
+            tc::drain_after_error();
+            tc::tc_fence_before_sync();
+            __syncthreads();
+            if (wi == 0) tc::tmem_dealloc(tmem, kFusedTmemCols);
+            return;
+        }
+        // the stages are dead: the arrays they lay over get their initial contents
+        {
+            float4* zt4 = reinterpret_cast<float4*>(zt);
+            for (int e = tid; e < (CB - C) * (TZ / 4); e += R_THREADS) zt4[C * (TZ / 4) + e] = make_float4(-1e30f, -1e30f, -1e30f, -1e30f);
+            for (int e = tid; e < C * TZ / 4; e += R_THREADS) reinterpret_cast<int4*>(corr)[e] = make_int4(0, 0, 0, 0);
+            if (CONF) for (int e = tid; e < C * C; e += R_THREADS) hist[e] = 0;
+        }
+        // accumulator m holds tile rows 4m .. 4m+3 (one row of 32 nodes per 32 lanes of tensor memory, and a warp reaches
+        // the lanes 32 (warp % 4) ..): warps 0-3 drain rows 0-3, warps 4-7 rows 4-7, warps 0 and 4 half of the classes of
+        // row 8 each
+        auto put_row = [&](const float* v, int n_cols, int c0, int j) {     // v[i]: class c0 + i of node (row j, column l)
+            const int ny = y0 - 1 + j, nx = x0 - 1 + l;
+            const bool in_frame = ny >= 0 && ny < h && nx >= 0 && nx < w;
+            // the block's own nodes go to global memory as well where the caller wants the logits kept
+            const bool keep = a.z_out && in_frame && j >= 1 && j <= RN_Y && l >= 1 && l <= RN_X;
+            float* dst = zt + c0 * TZ + j * TW + l;
+            float* zo = a.z_out + ((int64_t)s * C + c0) * p + (int64_t)ny * w + nx;
+#pragma unroll
+            for (int i = 0; i < 32; ++i)
+                if (i < n_cols && c0 + i < C) {
+                    const float t = v[i] + sbias[c0 + i];
+                    dst[i * TZ] = t;
+                    if (in_frame) m_loc = fmaxf(m_loc, t);
+                    if (keep) zo[(int64_t)i * p] = t;
+                }
+        };
+        {
+            float v[32];
+            tc::tmem_ld_32x32(tmem + ((uint32_t)((wi & 3) * 32) << 16) + (wi >> 2) * kClassPad, v);
+            put_row(v, 32, 0, wi);
+        }
+        if ((wi & 3) == 0) {
+            const int c0 = wi ? 16 : 0;
+            float v[32];
+            tc::tmem_ld_32x16(tmem + 2 * kClassPad + c0, reinterpret_cast<float(&)[16]>(v));
+            put_row(v, 16, c0, 8);
+        }
+        tc::tc_fence_before_sync();
+        __syncthreads();                                   // the tile is complete (its entries outside the frame are never read)
+    } else
     {
         // a thread keeps one 16-byte group of the tile plane (81 groups) and walks the classes three at a time
         constexpr int kQuads = TZ / 4, kPlanes = R_THREADS / kQuads;       // 81, 3
@@ -296,30 +465,7 @@ upsample_ce_rows_kernel(UpsampleCeArgs a, const __grid_constant__ CUtensorMap z_
                 tc::drain_after_error();
                 return;
             }
-            const bool edge_rows = y0 == 0 || y0 + RN_Y > h - 1, edge_cols = xa < 0 || xa + TZ_W > w;
-            if (edge_rows) {                                   // block-uniform: node rows above 0 / below h-1 repeat the border row
-                const int j_lo = y0 == 0 ? 1 : 0;              // first tile row inside the map
-                const int j_hi = min(TZ_H - 1, h - y0);        // last one
-                const int n_out = TZ_H - (j_hi - j_lo + 1);    // rows to fill: 0 .. j_lo-1 and j_hi+1 .. TZ_H-1
-                for (int e = tid; e < C * n_out * (TZ_W / 4); e += R_THREADS) {
-                    const int c = e / (n_out * (TZ_W / 4)), r = (e / (TZ_W / 4)) % n_out, x4 = e % (TZ_W / 4);
-                    const int j = r < j_lo ? r : j_hi + 1 + (r - j_lo);
-                    const int jc = j < j_lo ? j_lo : j_hi;
-                    zt4[(c * TZ + j * TZ_W) / 4 + x4] = zt4[(c * TZ + jc * TZ_W) / 4 + x4];
-                }
-                __syncthreads();
-            }
-            if (edge_cols) {                                   // node columns left of 0 / right of w-1 repeat the border column
-                const int x_lo = xa < 0 ? -xa : 0;             // first tile column inside the map
-                const int x_hi = min(TZ_W - 1, w - 1 - xa);    // last one
-                const int n_out = TZ_W - (x_hi - x_lo + 1);
-                for (int e = tid; e < C * TZ_H * n_out; e += R_THREADS) {
-                    const int row = e / n_out, r = e % n_out;  // row = c * TZ_H + j
-                    const int x = r < x_lo ? r : x_hi + 1 + (r - x_lo);
-                    zt[row * TZ_W + x] = zt[row * TZ_W + (x < x_lo ? x_lo : x_hi)];
-                }
-                __syncthreads();
-            }
+            replicate_borders();
 #pragma unroll
             for (int it = 0; it < kIter; ++it) {
                 const int c = g + it * kPlanes;
@@ -364,7 +510,9 @@ upsample_ce_rows_kernel(UpsampleCeArgs a, const __grid_constant__ CUtensorMap z_
     __syncthreads();
 
     RowCtx rc;
-    rc.za = zt + wi * TZ_W + off + l;
+    rc.za = zt + ry_top * TZ_W + rx_l;
+    rc.dq = (ry_bot - ry_top) * TZ_W;
+    rc.dr = rx_r - rx_l;
     rc.ly = 0.f;
     {
         // shift of the exponentials: the largest logit of the block's tile (a pixel whose own logits lie far below it
@@ -401,7 +549,7 @@ upsample_ce_rows_kernel(UpsampleCeArgs a, const __grid_constant__ CUtensorMap z_
                 rz = rcp_approx(Zs[k]) * wk;
                 if (own) {
                     const float* q = rc.za + lab[k] * TZ;
-                    const float vl = fmaf(ly, q[TZ_W] - q[0], q[0]), vr = fmaf(ly, q[TZ_W + 1] - q[1], q[1]);
+                    const float vl = fmaf(ly, q[rc.dq] - q[0], q[0]), vr = fmaf(ly, q[rc.dq + rc.dr] - q[rc.dr], q[rc.dr]);
                     const float ul = fmaf(fmaf((2 * k + 1) * 0.125f, vr - vl, vl), kLog2e, -rc.M) - sk[k];
                     loss += wk * (__log2f(Zs[k]) - ul) * kLn2;
                     if (CONF) atomicAdd(&hist[lab[k] * C + arg[k]], 1u);
@@ -449,7 +597,7 @@ upsample_ce_rows_kernel(UpsampleCeArgs a, const __grid_constant__ CUtensorMap z_
 #pragma unroll kClassUnroll
         for (int c = 0; c < CB; ++c) {
             float2 X01[4], X23[4];
-            wmax = fmaxf(wmax, cell_exponentials(rc.za + c * TZ, rc.M, X01, X23));
+            wmax = fmaxf(wmax, cell_exponentials(rc.za + c * TZ, rc.dq, rc.M, X01, X23));
 #pragma unroll
             for (int k = 0; k < 4; ++k) { Z01[k] = __fadd2_rn(Z01[k], X01[k]); Z23[k] = __fadd2_rn(Z23[k], X23[k]); }
             if (CONF) {
@@ -555,7 +703,7 @@ upsample_ce_rows_kernel(UpsampleCeArgs a, const __grid_constant__ CUtensorMap z_
                 // a row's four exponentials are E(r,0) q_r^k, so the row's weighted sum is E(r,0) times a cubic in q_r
                 // with the pixel weights as coefficients: Horner's rule, the progression itself is not formed again
                 float2 x01, x23, q01, q23;
-                cell_bases(rc.za + c * TZ, rc.M, x01, x23, q01, q23);
+                cell_bases(rc.za + c * TZ, rc.dq, rc.M, x01, x23, q01, q23);
                 float2 aL01 = WL01[3], aL23 = WL23[3], aR01 = WR01[3], aR23 = WR23[3];
 #pragma unroll
                 for (int k = 2; k >= 0; --k) {
@@ -582,19 +730,19 @@ upsample_ce_rows_kernel(UpsampleCeArgs a, const __grid_constant__ CUtensorMap z_
                 const float zero4[4] = {0.f, 0.f, 0.f, 0.f};
                 for (int c = 0; c < C; ++c) {
                     float u[4];
-                    pixel_logits<false>(rc, c, zero4, u);
+                    pixel_logits<false, TW>(rc, c, zero4, u);
 #pragma unroll
                     for (int k = 0; k < 4; ++k) ex[k] = fmaxf(ex[k], u[k]);
                 }
                 float Zs[4];
                 uint32_t ar4[4] = {0, 0, 0, 0};
-                if (CONF) pass1<CB, true, false>(rc, zero4, Zs, ar4);    // arg-max of the interpolated logits
-                pass1<CB, false, true>(rc, ex, Zs, ar4);
+                if (CONF) pass1<CB, true, false, TW>(rc, zero4, Zs, ar4);    // arg-max of the interpolated logits
+                pass1<CB, false, true, TW>(rc, ex, Zs, ar4);
                 float wl4[4], wr4[4];
                 finish_row(r, Zs, ex, ar4, wl4, wr4);
                 const float twr = i == -1 ? 0.f : (i == h - 1 ? 1.0f : 1.0f - rc.ly);
                 const float bwr = i == h - 1 ? 0.f : (i == -1 ? 1.0f : rc.ly);
-                pass2_slow<CB>(rc, ex, wl4, wr4, twr, bwr, my_acc, C);
+                pass2_slow<CB, TW>(rc, ex, wl4, wr4, twr, bwr, my_acc, C);
             }
         }
     } else {
@@ -678,28 +826,49 @@ upsample_ce_rows_kernel(UpsampleCeArgs a, const __grid_constant__ CUtensorMap z_
         for (int k = 0; k < R_WARPS; ++k) t += red[k];
         a.loss_part[(int64_t)s * n_blk + blk] = t;
     }
+    if constexpr (FUSED) {
+        if (wi == 0) {                           // every warp's reads of tensor memory ended before the barriers above
+            __syncwarp();
+            tc::tc_fence_after_sync();
+            tc::tmem_dealloc(tmem, kFusedTmemCols);
+        }
+    }
 }
 
-template <int CB>
+template <int CB, int TW>
 size_t rows_smem_bytes(int C, bool conf)
 {
-    return ((size_t)CB * TZ + (size_t)C * TZ + (size_t)R_WARPS * C * 32 * 2 + (conf ? (size_t)C * C : 0)) * sizeof(float) + 128;
+    constexpr size_t TZ = (size_t)TZ_H * TW;
+    const size_t plain = ((size_t)CB * TZ + (size_t)C * TZ + (size_t)R_WARPS * C * 32 * 2 + (conf ? (size_t)C * C : 0)) * sizeof(float) + 128;
+    if (TW != kTwFused) return plain;
+    // the feature stages and the weights lie over the kernel's arrays; the third multiplication of the last stage reads
+    // 384 pixel rows from the stage's start; 1 KB so that the stages can start at a multiple of 1024
+    const size_t ring = (size_t)kFusedStages * kStageBytes + (size_t)kFusedMaxKBlocks * kWeightBytes;
+    const size_t reach = (size_t)(kFusedStages - 1) * kStageBytes + 384 * 128;
+    return (plain > ring ? (plain > reach ? plain : reach) : (ring > reach ? ring : reach)) + 1024;
 }
 
 template <int CB>
 cudaError_t prepare_cb(int C)
 {
-    cudaError_t e = cudaFuncSetAttribute(upsample_ce_rows_kernel<CB, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)rows_smem_bytes<CB>(C, false));
-    if (e != cudaSuccess) return e;
-    return cudaFuncSetAttribute(upsample_ce_rows_kernel<CB, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)rows_smem_bytes<CB>(C, true));
+    cudaError_t e = cudaFuncSetAttribute(upsample_ce_rows_kernel<CB, false, kTwLoad>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)rows_smem_bytes<CB, kTwLoad>(C, false));
+    if (e == cudaSuccess) e = cudaFuncSetAttribute(upsample_ce_rows_kernel<CB, true, kTwLoad>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)rows_smem_bytes<CB, kTwLoad>(C, true));
+    if (e == cudaSuccess) e = cudaFuncSetAttribute(upsample_ce_rows_kernel<CB, false, kTwFused>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)rows_smem_bytes<CB, kTwFused>(C, false));
+    if (e == cudaSuccess) e = cudaFuncSetAttribute(upsample_ce_rows_kernel<CB, true, kTwFused>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)rows_smem_bytes<CB, kTwFused>(C, true));
+    return e;
 }
 
 template <int CB>
-cudaError_t launch_cb(const UpsampleCeArgs& a, const CUtensorMap& z_map, cudaStream_t s)
+cudaError_t launch_cb(const UpsampleCeArgs& a, const CUtensorMap& z_map, const CUtensorMap& x_map, const CUtensorMap& w_map, cudaStream_t s)
 {
     dim3 grid((unsigned)((a.w + RN_X - 1) / RN_X), (unsigned)((a.h + RN_Y - 1) / RN_Y), (unsigned)a.S);
-    if (a.conf) return launch_chain(a.chain_early != 0, upsample_ce_rows_kernel<CB, true>, grid, dim3(R_THREADS), rows_smem_bytes<CB>(a.C, true), s, a, z_map);
-    return launch_chain(a.chain_early != 0, upsample_ce_rows_kernel<CB, false>, grid, dim3(R_THREADS), rows_smem_bytes<CB>(a.C, false), s, a, z_map);
+    const bool early = a.chain_early != 0 || a.x_early != 0;
+    if (a.fused) {
+        if (a.conf) return launch_chain(early, upsample_ce_rows_kernel<CB, true, kTwFused>, grid, dim3(R_THREADS), rows_smem_bytes<CB, kTwFused>(a.C, true), s, a, z_map, x_map, w_map);
+        return launch_chain(early, upsample_ce_rows_kernel<CB, false, kTwFused>, grid, dim3(R_THREADS), rows_smem_bytes<CB, kTwFused>(a.C, false), s, a, z_map, x_map, w_map);
+    }
+    if (a.conf) return launch_chain(early, upsample_ce_rows_kernel<CB, true, kTwLoad>, grid, dim3(R_THREADS), rows_smem_bytes<CB, kTwLoad>(a.C, true), s, a, z_map, x_map, w_map);
+    return launch_chain(early, upsample_ce_rows_kernel<CB, false, kTwLoad>, grid, dim3(R_THREADS), rows_smem_bytes<CB, kTwLoad>(a.C, false), s, a, z_map, x_map, w_map);
 }
 
 // class-count buckets: the two workload sizes exactly, multiples of four otherwise
@@ -731,27 +900,51 @@ int upsample_ce_rows_blocks(int h, int w) { return ((h + RN_Y - 1) / RN_Y) * ((w
 
 cudaError_t prepare_upsample_ce_rows(int C) { ST_ROWS_DISPATCH(prepare_cb, C, C) }
 
-cudaError_t launch_rows_dispatch(const UpsampleCeArgs& a, const CUtensorMap& z_map, cudaStream_t s) { ST_ROWS_DISPATCH(launch_cb, a.C, a, z_map, s) }
-
-void launch_upsample_ce_rows(const UpsampleCeArgs& a, const CUtensorMap* z_map, cudaStream_t s)
+cudaError_t launch_rows_dispatch(const UpsampleCeArgs& a, const CUtensorMap& z_map, const CUtensorMap& x_map, const CUtensorMap& w_map, cudaStream_t s)
 {
-    if (a.has_map && z_map) { launch_rows_dispatch(a, *z_map, s); return; }
-    UpsampleCeArgs b = a;
-    b.has_map = 0;
+    ST_ROWS_DISPATCH(launch_cb, a.C, a, z_map, x_map, w_map, s)
+}
+
+void launch_upsample_ce_rows(const UpsampleCeArgs& a, const CUtensorMap* z_map, cudaStream_t s, const CUtensorMap* x_map, const CUtensorMap* w_map)
+{
     CUtensorMap none;
     memset(&none, 0, sizeof(none));
-    launch_rows_dispatch(b, none, s);
+    UpsampleCeArgs b = a;
+    if (b.fused && !(x_map && w_map && fused_forward_supported(b.C, b.h, b.w, b.kblocks * 64))) b.fused = 0;
+    if (b.fused) { b.has_map = 0; launch_rows_dispatch(b, none, *x_map, *w_map, s); return; }
+    b.x_early = 0;
+    if (!(b.has_map && z_map)) b.has_map = 0;
+    launch_rows_dispatch(b, b.has_map ? *z_map : none, none, none, s);
+}
+
+// The block multiplies its own logits when the classifier is a 1x1 layer over at most 256 channels (a multiple of 64)
+// and the feature map is at least one tile large.
+bool fused_forward_supported(int C, int h, int w, int c_in)
+{
+    return upsample_ce_rows_supported(C) && c_in >= 64 && c_in % 64 == 0 && c_in / 64 <= kFusedMaxKBlocks && w >= kTwFused && h >= TZ_H;
 }
 
 bool make_logit_tile_map(CUtensorMap* m, const float* z, int S, int C, int h, int w)
 {
-    if (!upsample_ce_rows_supported(C) || w % 4 != 0 || w < TZ_W || h < TZ_H || ((uintptr_t)z & 15u)) return false;
+    if (!upsample_ce_rows_supported(C) || w % 4 != 0 || w < kTwLoad || h < TZ_H || ((uintptr_t)z & 15u)) return false;
     const uint64_t dims[3] = {(uint64_t)w, (uint64_t)h, (uint64_t)S * C};
     const uint64_t strides[2] = {(uint64_t)w * sizeof(float), (uint64_t)h * w * sizeof(float)};
-    const uint32_t box[3] = {(uint32_t)TZ_W, (uint32_t)TZ_H, (uint32_t)C};
+    const uint32_t box[3] = {(uint32_t)kTwLoad, (uint32_t)TZ_H, (uint32_t)C};
     char err[128];
     return encode_tensor_map(m, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, CU_TENSOR_MAP_SWIZZLE_NONE, z, 3, dims, strides, box, err,
                              sizeof(err), "logit tile");
+}
+
+bool make_feature_tile_map(CUtensorMap* m, const bf16* x, int S, int c_in, int h, int w)
+{
+    if (c_in % 64 != 0 || w < kTwFused || h < TZ_H || ((uintptr_t)x & 15u)) return false;
+    const uint64_t c = (uint64_t)c_in;
+    const uint64_t dims[4] = {c, (uint64_t)w, (uint64_t)h, (uint64_t)S};
+    const uint64_t strides[3] = {c * 2, (uint64_t)w * c * 2, (uint64_t)h * w * c * 2};
+    const uint32_t box[4] = {64, (uint32_t)kTwFused, (uint32_t)TZ_H, 1};
+    char err[128];
+    return encode_tensor_map(m, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, CU_TENSOR_MAP_SWIZZLE_128B, x, 4, dims, strides, box, err,
+                             sizeof(err), "feature tile");
 }
 
 }  // namespace st

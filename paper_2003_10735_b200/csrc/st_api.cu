@@ -70,6 +70,8 @@ struct st_ctx {
     int n_k3_blocks = 0;
     CUtensorMap k3_map;        // tile map of z for the fused upsample + cross-entropy kernel
     int k3_has_map = 0;
+    CUtensorMap fx_map, fw_map; // tile maps of the features and of the bf16 classifier weights: the loss kernel multiplies its own logits
+    int fused_fwd = 0;          //   (one-layer head with bf16 GEMMs; ST_FUSED_FORWARD=0 switches it off)
     float* loss_buf = nullptr;              // [S][kMaxSteps]
     unsigned long long* conf_buf = nullptr; // [S][kMaxSteps][C][C], allocated on first use
     // Train (Algorithm 1), allocated on first use
@@ -249,9 +251,10 @@ st_status ensure_prefix(st_ctx* c)
 // Forward of the trainable part for all streams: z (and the hidden activation).
 // `skip` (tensor-core kernels only): per-stream flags, see tc_forward.
 st_status enqueue_forward(st_ctx* c, StageTimer* t = nullptr, const int* skip = nullptr, int64_t skip_stride = 0,
-                          bool after_update = false)
+                          bool after_update = false, bool loss_follows = false)
 {
     cudaStream_t s = c->stream;
+    if (c->fused_fwd && loss_follows) return ST_OK;      // the loss kernel multiplies the logits itself (and writes them)
     if (c->bf16_mode) {
         c->launches += tc_forward(c->plan, s, t, skip, skip_stride, after_update, c->first_trained < c->n_blocks ? c->first_trained : c->n_blocks);
     } else if (c->Ch == 0) {
@@ -304,16 +307,25 @@ UpsampleCeArgs k3_args(st_ctx* c, bool fp32_grad, bool bf16_grad, unsigned long 
     k3.has_map = c->k3_has_map;
     k3.skip = skip; k3.skip_stride = skip_stride;
     k3.chain_early = c->chain_early ? 1 : 0;
+    k3.fused = 0; k3.x_early = 0; k3.kblocks = 0; k3.theta = nullptr; k3.n_params = 0; k3.b_off = 0; k3.z_out = nullptr;
     return k3;
 }
 
 // ComputeLoss and the first half of PartialBackward: loss partials, logit gradient, optionally the confusion matrix
 // of this prediction.
-st_status enqueue_loss(st_ctx* c, unsigned long long* conf, StageTimer* t = nullptr, const int* skip = nullptr, int64_t skip_stride = 0)
+st_status enqueue_loss(st_ctx* c, unsigned long long* conf, StageTimer* t = nullptr, const int* skip = nullptr, int64_t skip_stride = 0,
+                       bool after_update = false, bool keep_logits = true)
 {
     cudaStream_t s = c->stream;
-    const UpsampleCeArgs k3 = k3_args(c, !c->bf16_mode, c->bf16_mode, conf, skip, skip_stride);
-    ST_REPEAT(t) launch_upsample_ce(k3, &c->k3_map, s);
+    UpsampleCeArgs k3 = k3_args(c, !c->bf16_mode, c->bf16_mode, conf, skip, skip_stride);
+    if (c->fused_fwd) {
+        // Forward as well: the features are frozen, so after a parameter update (which writes weights only) their tiles
+        // may be fetched while that update is still running
+        k3.fused = 1; k3.x_early = after_update && !t ? 1 : 0; k3.kblocks = c->Cin / 64;
+        k3.theta = c->theta; k3.n_params = c->n_params; k3.b_off = c->layout.b_off[c->layout.n_layers - 1];
+        k3.z_out = keep_logits ? c->z : nullptr;         // logits that the next iteration overwrites unread stay on the chip
+    }
+    ST_REPEAT(t) launch_upsample_ce(k3, &c->k3_map, s, &c->fx_map, &c->fw_map);
     if (t) t->mark("upsample_ce", s, st_repeats(t));
     c->launches += st_repeats(t);
     return check_launch(c, "upsample + cross-entropy");
@@ -353,11 +365,11 @@ st_status enqueue_update(st_ctx* c, int slot, const int* skip, int64_t skip_stri
     return check_launch(c, "sgd update");
 }
 
-st_status enqueue_step(st_ctx* c, int slot, bool want_conf, StageTimer* t = nullptr)
+st_status enqueue_step(st_ctx* c, int slot, bool want_conf, StageTimer* t = nullptr, bool last = true)
 {
     // iterations after the first follow the previous iteration's update directly
-    st_status st = enqueue_forward(c, t, nullptr, 0, slot > 0 && !t);
-    if (st == ST_OK) st = enqueue_loss(c, want_conf ? c->conf_buf + (int64_t)slot * c->C * c->C : nullptr, t);
+    st_status st = enqueue_forward(c, t, nullptr, 0, slot > 0 && !t, true);
+    if (st == ST_OK) st = enqueue_loss(c, want_conf ? c->conf_buf + (int64_t)slot * c->C * c->C : nullptr, t, nullptr, 0, slot > 0, last);
     if (st == ST_OK) st = enqueue_backward(c, t);
     if (st == ST_OK) st = enqueue_update(c, slot, nullptr, 0, t);
     return st;
@@ -667,6 +679,15 @@ st_status st_init_head(const st_head_desc* desc, const float* init_params, st_ct
         }
         launch_refresh_shadow(make_update_args(c, -1, nullptr, 0, true), c->stream);
         e = cudaGetLastError();
+        const char* off = getenv("ST_FUSED_FORWARD");
+        if (n_blocks == 0 && !(off && off[0] == '0') && fused_forward_supported(c->C, c->h, c->w, c->Cin)) {
+            const uint64_t ci = (uint64_t)c->Cin;
+            const uint64_t dims[3] = {ci, (uint64_t)kClassPad, (uint64_t)S}, str[2] = {ci * 2, (uint64_t)kClassPad * ci * 2};
+            const uint32_t box[3] = {64, (uint32_t)kClassPad, 1};
+            c->fused_fwd = make_feature_tile_map(&c->fx_map, c->x_bf16, S, c->Cin, c->h, c->w) &&
+                           encode_tensor_map(&c->fw_map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, CU_TENSOR_MAP_SWIZZLE_128B, c->w2_shadow, 3,
+                                             dims, str, box, msg, sizeof msg, "1x1 weight");
+        }
     }
     if (e == cudaSuccess) e = cudaStreamSynchronize(c->stream);   // init_params may be released on return
     if (e != cudaSuccess) {
@@ -835,7 +856,7 @@ st_status st_distill_step(st_ctx* ctx, int32_t n_steps, float* loss_out, int64_t
             cudaGraph_t graph = nullptr;
             const int64_t before = ctx->launches;
             ST_CUDA(ctx, cudaStreamBeginCapture(ctx->stream, cudaStreamCaptureModeThreadLocal));
-            for (int k = 0; k < n_steps && st == ST_OK; ++k) st = enqueue_step(ctx, k, want_conf);
+            for (int k = 0; k < n_steps && st == ST_OK; ++k) st = enqueue_step(ctx, k, want_conf, nullptr, k == n_steps - 1);
             if (st == ST_OK && ctx->adam) { launch_step_tick(ctx->step_base, ctx->S, n_steps, nullptr, ctx->stream); ctx->launches += 1; }
             cudaError_t e = cudaStreamEndCapture(ctx->stream, &graph);
             const int64_t n_launches = ctx->launches - before;
@@ -852,7 +873,7 @@ st_status st_distill_step(st_ctx* ctx, int32_t n_steps, float* loss_out, int64_t
         ST_CUDA(ctx, cudaGraphLaunch(it->second.exec, ctx->stream));
     } else {
         for (int k = 0; k < n_steps; ++k) {
-            st = enqueue_step(ctx, k, want_conf);
+            st = enqueue_step(ctx, k, want_conf, nullptr, k == n_steps - 1);
             if (st != ST_OK) return st;
         }
         if (ctx->adam) { launch_step_tick(ctx->step_base, ctx->S, n_steps, nullptr, ctx->stream); ctx->launches += 1; }
@@ -888,8 +909,8 @@ st_status enqueue_train(st_ctx* c, int max_updates, double threshold)
     for (int i = 0; i <= max_updates && st == ST_OK; ++i) {
         const int* ended_before = i > 0 ? c->ctl_done + i : nullptr;        // done[s][i]: no prediction i for stream s
         const int* ended_now = c->ctl_done + i + 1;                         // done[s][i+1]: no update i+1 for stream s
-        st = enqueue_forward(c, nullptr, ended_before, kCtlPitch);                        // prediction <- Forward(student, frame)
-        if (st == ST_OK) st = enqueue_loss(c, c->conf_buf + (int64_t)i * c->C * c->C, nullptr, ended_before, kCtlPitch);   // loss, gradient, confusion
+        st = enqueue_forward(c, nullptr, ended_before, kCtlPitch, false, true);           // prediction <- Forward(student, frame)
+        if (st == ST_OK) st = enqueue_loss(c, c->conf_buf + (int64_t)i * c->C * c->C, nullptr, ended_before, kCtlPitch, i > 0);   // loss, gradient, confusion
         if (st != ST_OK) break;
         launch_train_decide(train_ctl(c, i, max_updates, threshold), c->stream);         // metric, best_student, break
         c->launches += 1;

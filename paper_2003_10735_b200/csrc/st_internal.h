@@ -105,6 +105,14 @@ struct UpsampleCeArgs {
     int heavy_w;             // 1, or the integer weight (2..5) of the pixels whose label byte has bit 7 set
                              //   (`labels` is then the tagged map made by launch_object_weight_tags)
     int chain_early;         // launch so that the kernel may start while its predecessor on the stream drains
+    // The block multiplies its own logit tile instead of reading `z` (Forward for a 1x1 classifier over bf16 features,
+    // row-walking kernel only; the launch then carries tile maps of the features and of the bf16 weights):
+    int fused;               // 0, or 1: ignore `z`, compute the tile from the maps
+    int x_early;             // the features are not written by the kernel just before this one: fetch them before waiting for it
+    int kblocks;             // 64-channel slices of the classifier's input
+    const float* theta;      // parameters (for the bias: theta[s * n_params + b_off + c])
+    int64_t n_params, b_off;
+    float* z_out;            // nullptr, or [S][C][h][w]: the logits are written here as well
 };
 // Tile map of the logits for the row-walking kernel: fp32 tensor {w, h, S*C}, one box = the block's tile of all
 // classes.  False if the shape does not allow it (w not a multiple of 4, C > 32) or the driver entry point is
@@ -116,12 +124,19 @@ bool encode_tensor_map(CUtensorMap* m, CUtensorMapDataType dtype, CUtensorMapSwi
                        const char* what);
 int upsample_ce_blocks(int h, int w, int C);   // blocks per stream (sizes loss_part / db_part)
 cudaError_t prepare_upsample_ce(int C);   // once per device and class count, outside any stream capture
-void launch_upsample_ce(const UpsampleCeArgs& a, const CUtensorMap* z_map, cudaStream_t s);   // z_map: host copy, used if a.has_map
+// z_map: host copy, used if a.has_map; x_map, w_map: host copies, needed if a.fused (without them, or for a shape
+// fused_forward_supported rejects, the launch falls back to reading `z`)
+void launch_upsample_ce(const UpsampleCeArgs& a, const CUtensorMap* z_map, cudaStream_t s, const CUtensorMap* x_map = nullptr,
+                        const CUtensorMap* w_map = nullptr);
+bool fused_forward_supported(int C, int h, int w, int c_in);
+// Tile map of bf16 features [S][h][w][c_in] for the fused forward: {c_in, w, h, S}, one box = 64 channels of the block's tile
+bool make_feature_tile_map(CUtensorMap* m, const bf16* x, int S, int c_in, int h, int w);
 // register-resident variant for C <= 32 (k_upsample_ce_rows.cu); launch_upsample_ce dispatches to it
 bool upsample_ce_rows_supported(int C);
 int upsample_ce_rows_blocks(int h, int w);
 cudaError_t prepare_upsample_ce_rows(int C);
-void launch_upsample_ce_rows(const UpsampleCeArgs& a, const CUtensorMap* z_map, cudaStream_t s);
+void launch_upsample_ce_rows(const UpsampleCeArgs& a, const CUtensorMap* z_map, cudaStream_t s, const CUtensorMap* x_map = nullptr,
+                             const CUtensorMap* w_map = nullptr);
 // student mask: argmax_c of the upsampled logits, uint8 [H][W]; with `labels` also the confusion matrix of
 // (label, mask) added into `conf`, and with `miou` the mean IoU written by the last block (k_student_mask.cu)
 struct StudentMaskArgs {
