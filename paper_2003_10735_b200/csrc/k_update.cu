@@ -90,6 +90,41 @@ __device__ __forceinline__ float apply_update(const UpdateArgs& a, int64_t gi, f
     return apply_update<ADAM>(a, gi, g, k, load_state<ADAM>(a, gi));
 }
 
+// Train (Algorithm 1), judged by every block of the update that follows prediction i: metric <- mIoU of the prediction;
+// better = the metric is the best so far (best_student <- student); skip = the loop ends here or had ended before
+// (no OptimStep).  Block-uniform; called by all 256 threads.  `writer` (one block per stream) records the history.
+__device__ __forceinline__ void train_decision(const TrainCtl& t, int s, bool writer, bool& skip, bool& better)
+{
+    __shared__ double iou[256];
+    __shared__ int present[256];
+    __shared__ double m_sh;
+    const int i = t.iter;
+    int* done = t.done + (int64_t)s * kCtlPitch;
+    double* best = t.best + (int64_t)s * kCtlPitch;
+    double* metric = t.metric + (int64_t)s * kCtlPitch;
+    better = false;
+    if (i > 0 && done[i] != 0) {                                 // the loop had ended before this prediction
+        skip = true;
+        if (writer && threadIdx.x == 0) { done[i + 1] = 1; best[i + 1] = best[i]; metric[i] = -1.0; }
+        return;
+    }
+    const double m0 = block_miou(t.conf + (int64_t)s * t.conf_stream_stride, t.C, iou, present);
+    if (threadIdx.x == 0) m_sh = m0;
+    __syncthreads();
+    const double m = m_sh;
+    const double prev_best = i > 0 ? best[i] : 0.0;
+    better = i == 0 || m > prev_best;
+    const bool stop = i == 0 ? !(m < t.threshold) : (m > t.threshold);
+    skip = stop || i >= t.max_updates;
+    if (writer && threadIdx.x == 0) {
+        metric[i] = m;
+        best[i + 1] = better ? m : prev_best;
+        done[i + 1] = skip ? 1 : 0;
+        t.n_updates[s] = i;                                      // overwritten by the next prediction if the loop goes on
+        if (better) t.best_iter[s] = i;
+    }
+}
+
 // Parameter blocks: a block covers kUpdThreads / G consecutive parameters; the G thread groups of a
 // block each sum every G-th split-K partial of "their" parameter (coalesced along the parameters),
 // the group sums are added in group order through shared memory, and group 0 applies the update.
@@ -128,10 +163,13 @@ sgd_update_kernel(UpdateArgs a, int n_param_blocks, int64_t range_begin)
     }
     pdl_wait();
     pdl_launch_dependents();
-    const bool skip = a.skip && a.skip[(int64_t)s * a.skip_stride];   // block-uniform
+    bool skip = a.skip && a.skip[(int64_t)s * a.skip_stride];   // block-uniform
+    bool better = false;                                         // Train: this prediction is the best so far
+    if (a.has_ctl) train_decision(a.ctl, s, blockIdx.x == 0, skip, better);
+    float* best_theta = a.has_ctl ? a.ctl.best_theta : nullptr;
     const AdamCorr corr = adam_corrections<ADAM>(a, s);
     if (param_block) {
-        if (skip) return;
+        if (skip && !better) return;
         float sum[E];
         // E parameters per thread, all of their split-K loads issued before any is consumed
 #pragma unroll
@@ -175,10 +213,11 @@ sgd_update_kernel(UpdateArgs a, int n_param_blocks, int64_t range_begin)
                 } else {
                     gr = a.grad[base + i];
                 }
-                const float t = apply_update<ADAM>(a, base + i, gr, corr, state[e]);
-                write_shadows(ly, s, i - ly.w_off, t);
+                if (better) best_theta[base + i] = state[e].theta;
+                if (!skip) write_shadows(ly, s, i - ly.w_off, apply_update<ADAM>(a, base + i, gr, corr, state[e]));
             } else if (!ly.b_partials) {
-                apply_update<ADAM>(a, base + i, a.grad[base + i], corr, state[e]);
+                if (better) best_theta[base + i] = state[e].theta;
+                if (!skip) apply_update<ADAM>(a, base + i, a.grad[base + i], corr, state[e]);
             }   // biases with partial sums are finished by the reduction warps below
         }
         return;
@@ -205,7 +244,10 @@ sgd_update_kernel(UpdateArgs a, int n_param_blocks, int64_t range_begin)
             }
 #pragma unroll
             for (int o = 16; o > 0; o >>= 1) g += __shfl_xor_sync(0xffffffffu, g, o);
-            if (lane == 0 && !skip) apply_update<ADAM>(a, base + ly.b_off + item, g, corr);
+            if (lane == 0) {
+                if (better) best_theta[base + ly.b_off + item] = a.theta[base + ly.b_off + item];
+                if (!skip) apply_update<ADAM>(a, base + ly.b_off + item, g, corr);
+            }
             return;
         }
         item -= ly.cout;
@@ -241,7 +283,9 @@ sgd_update_stream_kernel(UpdateArgs a, int L)
     pdl_launch_dependents();
     const LayerUpdate& ly = a.layer[L];
     const int s = blockIdx.y;
-    if (a.skip && a.skip[(int64_t)s * a.skip_stride]) return;
+    bool skip = a.skip && a.skip[(int64_t)s * a.skip_stride], better = false;
+    if (a.has_ctl) train_decision(a.ctl, s, false, skip, better);      // the grouped kernel's block 0 writes the history
+    if (skip && !better) return;
     const int64_t nw = (int64_t)ly.cout * ly.cin * ly.taps;
     const int64_t e = ((int64_t)blockIdx.x * 256 + threadIdx.x) * VEC;
     if (e >= nw) return;
@@ -269,7 +313,10 @@ sgd_update_stream_kernel(UpdateArgs a, int L)
     const int64_t gi = (int64_t)s * a.n_params + ly.w_off + e;
     const AdamCorr corr = adam_corrections<ADAM>(a, s);
 #pragma unroll
-    for (int j = 0; j < VEC; ++j) write_shadows(ly, s, e + j, apply_update<ADAM>(a, gi + j, g[j], corr));
+    for (int j = 0; j < VEC; ++j) {
+        if (better) a.ctl.best_theta[gi + j] = a.theta[gi + j];
+        if (!skip) write_shadows(ly, s, e + j, apply_update<ADAM>(a, gi + j, g[j], corr));
+    }
 }
 
 template <bool ADAM>
@@ -364,45 +411,11 @@ __global__ void __launch_bounds__(256) miou_kernel(const unsigned long long* __r
 //   prediction 0 (the incoming student):  best_metric <- metric; the loop is entered iff best_metric < THRESHOLD
 //   prediction i > 0 (after i updates):   if metric > best_metric: best_metric, best_student <- metric, student;
 //                                         if metric > THRESHOLD: break;  the loop also ends at i = MAX_UPDATES.
-__global__ void __launch_bounds__(256) train_decide_kernel(TrainCtl t)
-{
-    __shared__ double iou[256];
-    __shared__ int present[256];
-    __shared__ double m_sh;
-    const int s = blockIdx.y, i = t.iter;
-    int* done = t.done + (int64_t)s * kCtlPitch;
-    double* best = t.best + (int64_t)s * kCtlPitch;
-    double* metric = t.metric + (int64_t)s * kCtlPitch;
-    const bool ended = i > 0 && done[i] != 0;                 // block-uniform
-    if (ended) {
-        if (blockIdx.x == 0 && threadIdx.x == 0) { done[i + 1] = 1; best[i + 1] = best[i]; metric[i] = -1.0; }
-        return;
-    }
-    const double m0 = block_miou(t.conf + (int64_t)s * t.conf_stream_stride, t.C, iou, present);
-    if (threadIdx.x == 0) m_sh = m0;
-    __syncthreads();
-    const double m = m_sh;
-    const double prev_best = i > 0 ? best[i] : 0.0;
-    const bool better = i == 0 || m > prev_best;
-    if (better) {
-        const float* src = t.theta + (int64_t)s * t.n_params;
-        float* dst = t.best_theta + (int64_t)s * t.n_params;
-        for (int64_t e = (int64_t)blockIdx.x * 256 + threadIdx.x; e < t.n_params; e += (int64_t)gridDim.x * 256) dst[e] = src[e];
-    }
-    if (blockIdx.x == 0 && threadIdx.x == 0) {
-        metric[i] = m;
-        best[i + 1] = better ? m : prev_best;
-        const bool stop = i == 0 ? !(m < t.threshold) : (m > t.threshold);
-        done[i + 1] = (stop || i >= t.max_updates) ? 1 : 0;
-        t.n_updates[s] = i;                                      // overwritten by the next prediction if the loop goes on
-        if (better) t.best_iter[s] = i;
-    }
-}
-
-__global__ void __launch_bounds__(256) train_commit_kernel(const float* __restrict__ best_theta, float* __restrict__ theta, int64_t n_params)
+__global__ void __launch_bounds__(256) train_commit_kernel(const float* __restrict__ best_theta, float* __restrict__ theta, int64_t n_params,
+                                                           int64_t begin)
 {
     const int64_t base = (int64_t)blockIdx.y * n_params;
-    for (int64_t e = (int64_t)blockIdx.x * 256 + threadIdx.x; e < n_params; e += (int64_t)gridDim.x * 256) theta[base + e] = best_theta[base + e];
+    for (int64_t e = begin + (int64_t)blockIdx.x * 256 + threadIdx.x; e < n_params; e += (int64_t)gridDim.x * 256) theta[base + e] = best_theta[base + e];
 }
 
 void launch_miou(const unsigned long long* conf, int C, double* out, cudaStream_t s)
@@ -416,14 +429,9 @@ static unsigned copy_blocks(int64_t n_params)
     return (unsigned)(b < 1 ? 1 : (b > 592 ? 592 : b));
 }
 
-void launch_train_decide(const TrainCtl& t, cudaStream_t s)
-{
-    train_decide_kernel<<<dim3(copy_blocks(t.n_params), (unsigned)t.S), 256, 0, s>>>(t);
-}
-
 void launch_train_commit(const TrainCtl& t, float* theta, cudaStream_t s)
 {
-    train_commit_kernel<<<dim3(copy_blocks(t.n_params), (unsigned)t.S), 256, 0, s>>>(t.best_theta, theta, t.n_params);
+    train_commit_kernel<<<dim3(copy_blocks(t.n_params - t.param_begin), (unsigned)t.S), 256, 0, s>>>(t.best_theta, theta, t.n_params, t.param_begin);
 }
 
 // ---- pack / unpack ---------------------------------------------------------------------------------

@@ -358,9 +358,11 @@ st_status enqueue_backward(st_ctx* c, StageTimer* t = nullptr, const int* skip =
 }
 
 // OptimStep, and the loss of this prediction into loss_buf[slot].  `skip`: per-stream flags (see UpdateArgs).
-st_status enqueue_update(st_ctx* c, int slot, const int* skip, int64_t skip_stride, StageTimer* t = nullptr)
+st_status enqueue_update(st_ctx* c, int slot, const int* skip, int64_t skip_stride, StageTimer* t = nullptr, const TrainCtl* ctl = nullptr)
 {
-    c->launches += launch_sgd_update(make_update_args(c, slot, skip, skip_stride), c->stream);
+    UpdateArgs u = make_update_args(c, slot, skip, skip_stride);
+    if (ctl) { u.has_ctl = 1; u.ctl = *ctl; u.skip = nullptr; }      // Train: the update judges the prediction itself
+    c->launches += launch_sgd_update(u, c->stream);
     if (t) t->mark("sgd_update", c->stream, 1);
     return check_launch(c, "sgd update");
 }
@@ -897,27 +899,26 @@ TrainCtl train_ctl(st_ctx* c, int iter, int max_updates, double threshold)
     t.done = c->ctl_done; t.best = c->ctl_best; t.metric = c->ctl_metric;
     t.n_updates = c->ctl_n_updates; t.best_iter = c->ctl_best_iter;
     t.theta = c->theta; t.best_theta = c->best_theta; t.n_params = c->n_params; t.S = c->S;
+    t.param_begin = c->trained_begin;
     return t;
 }
 
-// Train of Algorithm 1 for all streams: one prediction per pass (forward, loss + gradient + confusion, decision),
-// then backward and the update.  The update is a no-op for streams whose loop has ended; so are the blocks of the
-// tensor-core GEMMs and of the loss kernel (the fp32 convolutions still run: their results are simply not used).
+// Train of Algorithm 1 for all streams: one prediction per pass (forward, loss + gradient + confusion), the backward,
+// then the update kernel, which first judges the prediction (metric, best_student, break) and takes the step only
+// where the loop goes on.  The backward of the pass in which a loop ends is therefore computed and not used; from the
+// next pass on the stream's blocks of the tensor-core GEMMs and of the loss kernel return at once (the fp32
+// convolutions still run: their results are simply not used).
 st_status enqueue_train(st_ctx* c, int max_updates, double threshold)
 {
     st_status st = ST_OK;
     for (int i = 0; i <= max_updates && st == ST_OK; ++i) {
         const int* ended_before = i > 0 ? c->ctl_done + i : nullptr;        // done[s][i]: no prediction i for stream s
-        const int* ended_now = c->ctl_done + i + 1;                         // done[s][i+1]: no update i+1 for stream s
         st = enqueue_forward(c, nullptr, ended_before, kCtlPitch, false, true);           // prediction <- Forward(student, frame)
         if (st == ST_OK) st = enqueue_loss(c, c->conf_buf + (int64_t)i * c->C * c->C, nullptr, ended_before, kCtlPitch, i > 0);   // loss, gradient, confusion
-        if (st != ST_OK) break;
-        launch_train_decide(train_ctl(c, i, max_updates, threshold), c->stream);         // metric, best_student, break
-        c->launches += 1;
-        st = check_launch(c, "train control");
-        if (st == ST_OK && i < max_updates) st = enqueue_backward(c, nullptr, ended_now, kCtlPitch);
-        // after the last prediction every loop has ended: the launch only finalises that prediction's loss
-        if (st == ST_OK) st = enqueue_update(c, i, ended_now, kCtlPitch);
+        if (st == ST_OK && i < max_updates) st = enqueue_backward(c, nullptr, ended_before, kCtlPitch);
+        // after the last prediction every loop ends: the launch judges it and finalises its loss
+        const TrainCtl ctl = train_ctl(c, i, max_updates, threshold);
+        if (st == ST_OK) st = enqueue_update(c, i, nullptr, 0, nullptr, &ctl);           // metric, best_student, break, OptimStep
     }
     if (st != ST_OK) return st;
     launch_train_commit(train_ctl(c, 0, max_updates, threshold), c->theta, c->stream);    // student <- best_student

@@ -168,6 +168,31 @@ void launch_conv1x1_dgrad_relu_f32(const float* W2, const float* dz, const float
 void launch_bias_grad_f32(const float* d, int C, int64_t p, float* db, int S, int64_t d_stride,
                           int64_t db_stride, cudaStream_t s);
 
+// ---- control of Algorithm 1 (Train): judged once per prediction, per stream, by the update kernel that follows the
+// prediction (metric of the prediction, best_student, the break) ----------------------------------------------
+// History arrays are indexed by the number of updates behind a prediction, so that a launch reads only what
+// earlier launches wrote: done[s][i] = the loop of stream s had ended before prediction i was made,
+// best[s][i] = best_metric before prediction i was judged.
+constexpr int kCtlPitch = kMaxSteps + 2;
+struct TrainCtl {
+    const unsigned long long* conf;   // confusion matrix of this prediction, stream 0
+    int64_t conf_stream_stride;       // elements between the matrices of consecutive streams
+    int C;
+    int iter;                         // i: number of updates behind this prediction
+    int max_updates;                  // MAX_UPDATES
+    double threshold;                 // THRESHOLD
+    int* done;                        // [S][kCtlPitch]
+    double* best;                     // [S][kCtlPitch]
+    double* metric;                   // [S][kCtlPitch]  metric of prediction i; -1 where the loop had ended before
+    int* n_updates;                   // [S] updates taken when the loop ended
+    int* best_iter;                   // [S] updates behind best_student
+    const float* theta;               // [S][n_params]
+    float* best_theta;                // [S][n_params]  best_student
+    int64_t n_params;
+    int64_t param_begin;              // parameters before this index are frozen: best_student never differs from the student there
+    int S;
+};
+
 // ---- K5: SGD(+momentum) update, loss finalisation, bf16 shadow refresh -------------------------
 struct LayerUpdate {
     int64_t w_off, b_off;      // offsets (floats) of weight / bias in one stream's parameter buffer
@@ -208,6 +233,12 @@ struct UpdateArgs {
     double b1, b2, eps, ln_b1, ln_b2;
     const long long* step_base;   // [S] optimisation steps taken before this call
     int chain_early;         // launch so that the kernel may start while its predecessor on the stream drains
+    // Train (Algorithm 1): the update also judges the prediction it follows.  Every block works the metric out from the
+    // prediction's confusion matrix (same counts, same arithmetic, same answer), keeps the old value of its parameters
+    // as best_student's where the metric is the best so far, and leaves them alone where the loop has ended; block 0
+    // writes the history.  `skip` is then not used.
+    int has_ctl;
+    TrainCtl ctl;
 };
 // step_base[s] += add (add_per_stream == nullptr) or += add_per_stream[s]
 void launch_step_tick(long long* step_base, int S, int add, const int* add_per_stream, cudaStream_t s);
@@ -216,32 +247,9 @@ int launch_sgd_update(const UpdateArgs& a, cudaStream_t s);   // returns the num
 void launch_refresh_shadow(const UpdateArgs& a, cudaStream_t s);
 // mean IoU (Section 3.2) from an int64 confusion matrix, in double, one block
 void launch_miou(const unsigned long long* conf, int C, double* out, cudaStream_t s);
-
-// ---- control of Algorithm 1 (Train): judged once per prediction, per stream ----------------------
-// History arrays are indexed by the number of updates behind a prediction, so that a launch reads only what
-// earlier launches wrote: done[s][i] = the loop of stream s had ended before prediction i was made,
-// best[s][i] = best_metric before prediction i was judged.
-constexpr int kCtlPitch = kMaxSteps + 2;
-struct TrainCtl {
-    const unsigned long long* conf;   // confusion matrix of this prediction, stream 0
-    int64_t conf_stream_stride;       // elements between the matrices of consecutive streams
-    int C;
-    int iter;                         // i: number of updates behind this prediction
-    int max_updates;                  // MAX_UPDATES
-    double threshold;                 // THRESHOLD
-    int* done;                        // [S][kCtlPitch]
-    double* best;                     // [S][kCtlPitch]
-    double* metric;                   // [S][kCtlPitch]  metric of prediction i; -1 where the loop had ended before
-    int* n_updates;                   // [S] updates taken when the loop ended
-    int* best_iter;                   // [S] updates behind best_student
-    const float* theta;               // [S][n_params]
-    float* best_theta;                // [S][n_params]  best_student
-    int64_t n_params;
-    int S;
-};
-void launch_train_decide(const TrainCtl& t, cudaStream_t s);
-// student <- best_student (the caller refreshes the bf16 copies afterwards)
+// student <- best_student for the trained parameters (the caller refreshes the bf16 copies afterwards)
 void launch_train_commit(const TrainCtl& t, float* theta, cudaStream_t s);
+
 
 // ---- K7: packed parameter buffer <-> internal order ---------------------------------------------
 // packed: per layer weight [cout][cin][kh][kw] then bias; internal: weight [tap][cout][cin] then bias.
