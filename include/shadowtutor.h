@@ -268,7 +268,9 @@ ST_API st_status st_agreement(st_ctx *ctx, int32_t stream, const uint8_t *pred, 
 
 /* Intermediate tensors of the most recent step, for verification. */
 typedef enum st_tensor {
-    ST_TENSOR_LOGITS = 0,      /* z, fp32 [C][h][w]: head output of the last forward */
+    ST_TENSOR_LOGITS = 0,      /* z, fp32 [C][h][w]: head output of the last forward (after st_distill_step: of its last
+                                  step, before that step's update; after st_train_key_frame: of the student the call
+                                  leaves behind, computed when asked for) */
     ST_TENSOR_LOGIT_GRAD = 1,  /* dz, fp32 [C][h][w]: gradient of the mean loss w.r.t. z */
     ST_TENSOR_PARAM_GRAD = 2,  /* fp32, packed order: gradient applied by the last update */
     ST_TENSOR_MOMENTUM = 3,    /* fp32, packed order */

@@ -16,6 +16,7 @@
 // shifted (x, y) coordinates of a [channel][x][y][stream] tensor map.
 #include "st_internal.h"
 #include "tc_common.cuh"
+#include "train_ctl.cuh"
 
 #include <cstdio>
 #include <cstring>
@@ -157,8 +158,20 @@ tc_wgrad1x1_kernel(const __grid_constant__ CUtensorMap tmA,   // {K, p, S}      
                    const __grid_constant__ CUtensorMap tmB,   // {p, 32, S}     box {64, 32, 1}
                    float* __restrict__ partials,              // [S][n_split][32][K]
                    int K, int n_chunks, int chunks_per_block, int m_split, int tmem_cols, unsigned int* err,
-                   const int* __restrict__ skip, int64_t skip_stride, int a_early)
+                   const int* __restrict__ skip, int64_t skip_stride, int a_early, int has_ctl, const TrainCtl ctl)
 {
+    // Train: the block after the last one of the weight gradient judges the prediction (metric, best so far, break)
+    // while the others multiply; it takes no part in anything below
+    if (has_ctl && blockIdx.x == gridDim.x - 1) {
+        const int s = blockIdx.y;
+        const TrainHistory hist = train_history(ctl, s);
+        pdl_wait();
+        bool stop, better;
+        train_decision(ctl, s, true, hist, nullptr, stop, better);
+        pdl_launch_dependents();
+        return;
+    }
+    const int n_blocks_x = (int)gridDim.x - (has_ctl ? 1 : 0);
     extern __shared__ uint8_t smem_raw[];
     uint8_t* smem = align_smem(smem_raw);
     // m_split blocks share a pixel range, each with its own 128-channel accumulators: with the channels divided the
@@ -173,7 +186,7 @@ tc_wgrad1x1_kernel(const __grid_constant__ CUtensorMap tmA,   // {K, p, S}      
     __shared__ __align__(8) uint64_t full[STAGES], empty[STAGES], done;
     __shared__ uint32_t tmem_slot;
     const int tid = threadIdx.x, warp = tid >> 5;
-    const int s = blockIdx.y, split = (int)blockIdx.x / m_split, n_split = (int)gridDim.x / m_split;
+    const int s = blockIdx.y, split = (int)blockIdx.x / m_split, n_split = n_blocks_x / m_split;
     const int c_begin = split * chunks_per_block;
     const int c_end = min(n_chunks, c_begin + chunks_per_block);
 
@@ -1177,14 +1190,17 @@ int tc_forward(const TcPlan* P, cudaStream_t s, StageTimer* t, const int* skip, 
     return n + st_repeats(t);
 }
 
-int tc_backward(const TcPlan* P, cudaStream_t s, StageTimer* t, const int* skip, int64_t skip_stride)
+int tc_backward(const TcPlan* P, cudaStream_t s, StageTimer* t, const int* skip, int64_t skip_stride, const TrainCtl* ctl)
 {
     const TcBuffers& b = P->b;
     int n = 0;
     // one-layer head: the activations are the frozen features, which no kernel of the loop writes
     const int a_early = (!b.n_blocks && !skip && !t && b.chain_early) ? 1 : 0;
-    ST_REPEAT(t) launch_chain(b.chain_early != 0, tc_wgrad1x1_kernel<kWg1Stages>, dim3(P->split2 * P->msplit2, b.S), dim3(kThreadsTc), P->smem_wg1, s,
-        P->act_wg, P->dz_map, b.w2_partials, P->c_last, P->chunks2, P->per2, P->msplit2, P->cols2, b.err, skip, skip_stride, a_early);
+    TrainCtl no_ctl;
+    memset(&no_ctl, 0, sizeof no_ctl);
+    ST_REPEAT(t) launch_chain(b.chain_early != 0, tc_wgrad1x1_kernel<kWg1Stages>, dim3(P->split2 * P->msplit2 + (ctl ? 1 : 0), b.S), dim3(kThreadsTc),
+        P->smem_wg1, s, P->act_wg, P->dz_map, b.w2_partials, P->c_last, P->chunks2, P->per2, P->msplit2, P->cols2, b.err, skip, skip_stride,
+        a_early, ctl ? 1 : 0, ctl ? *ctl : no_ctl);
     if (t) t->mark("tc_wgrad1x1", s, st_repeats(t));
     n += st_repeats(t);
     const int nb = b.n_blocks;

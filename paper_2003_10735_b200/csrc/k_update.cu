@@ -7,6 +7,7 @@
 // K7 — UpdatedPart(student) (Algorithm 3): the packed fp32 buffer of all trainable tensors.
 #include "st_internal.h"
 #include "miou.cuh"
+#include "train_ctl.cuh"
 
 #include <cstdlib>
 
@@ -90,41 +91,6 @@ __device__ __forceinline__ float apply_update(const UpdateArgs& a, int64_t gi, f
     return apply_update<ADAM>(a, gi, g, k, load_state<ADAM>(a, gi));
 }
 
-// Train (Algorithm 1), judged by every block of the update that follows prediction i: metric <- mIoU of the prediction;
-// better = the metric is the best so far (best_student <- student); skip = the loop ends here or had ended before
-// (no OptimStep).  Block-uniform; called by all 256 threads.  `writer` (one block per stream) records the history.
-__device__ __forceinline__ void train_decision(const TrainCtl& t, int s, bool writer, bool& skip, bool& better)
-{
-    __shared__ double iou[256];
-    __shared__ int present[256];
-    __shared__ double m_sh;
-    const int i = t.iter;
-    int* done = t.done + (int64_t)s * kCtlPitch;
-    double* best = t.best + (int64_t)s * kCtlPitch;
-    double* metric = t.metric + (int64_t)s * kCtlPitch;
-    better = false;
-    if (i > 0 && done[i] != 0) {                                 // the loop had ended before this prediction
-        skip = true;
-        if (writer && threadIdx.x == 0) { done[i + 1] = 1; best[i + 1] = best[i]; metric[i] = -1.0; }
-        return;
-    }
-    const double m0 = block_miou(t.conf + (int64_t)s * t.conf_stream_stride, t.C, iou, present);
-    if (threadIdx.x == 0) m_sh = m0;
-    __syncthreads();
-    const double m = m_sh;
-    const double prev_best = i > 0 ? best[i] : 0.0;
-    better = i == 0 || m > prev_best;
-    const bool stop = i == 0 ? !(m < t.threshold) : (m > t.threshold);
-    skip = stop || i >= t.max_updates;
-    if (writer && threadIdx.x == 0) {
-        metric[i] = m;
-        best[i + 1] = better ? m : prev_best;
-        done[i + 1] = skip ? 1 : 0;
-        t.n_updates[s] = i;                                      // overwritten by the next prediction if the loop goes on
-        if (better) t.best_iter[s] = i;
-    }
-}
-
 // Parameter blocks: a block covers kUpdThreads / G consecutive parameters; the G thread groups of a
 // block each sum every G-th split-K partial of "their" parameter (coalesced along the parameters),
 // the group sums are added in group order through shared memory, and group 0 applies the update.
@@ -161,15 +127,24 @@ sgd_update_kernel(UpdateArgs a, int n_param_blocks, int64_t range_begin)
             if (g == 0 && layer[e] >= 0 && (is_weight[e] || !a.layer[layer[e]].b_partials)) state[e] = load_state<ADAM>(a, base + i);
         }
     }
+    TrainHistory hist{};
+    if (a.has_ctl) hist = train_history(a.ctl, s);
     pdl_wait();
     pdl_launch_dependents();
     bool skip = a.skip && a.skip[(int64_t)s * a.skip_stride];   // block-uniform
     bool better = false;                                         // Train: this prediction is the best so far
-    if (a.has_ctl) train_decision(a.ctl, s, blockIdx.x == 0, skip, better);
+    MiouFetch fetched{};
+    const bool decide_here = a.has_ctl == 1;                     // 2: the backward before this kernel has judged the prediction
+    if (decide_here) fetched = train_fetch(a.ctl, s, hist);      // on their way while the partial sums are fetched and added
+    if (a.has_ctl == 2 && !hist.ended) train_outcome(a.ctl, s, skip, better);
     float* best_theta = a.has_ctl ? a.ctl.best_theta : nullptr;
     const AdamCorr corr = adam_corrections<ADAM>(a, s);
     if (param_block) {
-        if (skip && !better) return;
+        if (a.has_ctl && hist.ended) {                  // nothing to judge, nothing to update: the history goes on
+            if (decide_here) train_decision(a.ctl, s, blockIdx.x == 0, hist, &fetched, skip, better);
+            return;
+        }
+        if (skip && !decide_here && !better) return;
         float sum[E];
         // E parameters per thread, all of their split-K loads issued before any is consumed
 #pragma unroll
@@ -197,8 +172,9 @@ sgd_update_kernel(UpdateArgs a, int n_param_blocks, int64_t range_begin)
         }
 #pragma unroll
         for (int e = 0; e < E; ++e) part[g][e * kRow + col] = sum[e];
+        if (decide_here) train_decision(a.ctl, s, blockIdx.x == 0, hist, &fetched, skip, better);
         __syncthreads();
-        if (g != 0) return;
+        if (g != 0 || (skip && !better)) return;
 #pragma unroll
         for (int e = 0; e < E; ++e) {
             if (layer[e] < 0) continue;
@@ -223,6 +199,8 @@ sgd_update_kernel(UpdateArgs a, int n_param_blocks, int64_t range_begin)
         return;
     }
     // ---- reduction warps: one warp per bias element that has partial sums, plus one for the loss
+    if (decide_here) train_decision(a.ctl, s, blockIdx.x == 0, hist, &fetched, skip, better);
+    else if (a.has_ctl && hist.ended) skip = true;
     const int warp = ((int)blockIdx.x - n_param_blocks) * (kUpdThreads / 32) + (threadIdx.x >> 5);
     const int lane = threadIdx.x & 31;
     int item = warp;
@@ -284,7 +262,12 @@ sgd_update_stream_kernel(UpdateArgs a, int L)
     const LayerUpdate& ly = a.layer[L];
     const int s = blockIdx.y;
     bool skip = a.skip && a.skip[(int64_t)s * a.skip_stride], better = false;
-    if (a.has_ctl) train_decision(a.ctl, s, false, skip, better);      // the grouped kernel's block 0 writes the history
+    if (a.has_ctl) {                                                   // the grouped kernel's block 0 writes the history
+        const TrainHistory hist = train_history(a.ctl, s);
+        if (a.has_ctl == 1) { const MiouFetch f = train_fetch(a.ctl, s, hist); train_decision(a.ctl, s, false, hist, &f, skip, better); }
+        else if (hist.ended) skip = true;
+        else train_outcome(a.ctl, s, skip, better);
+    }
     if (skip && !better) return;
     const int64_t nw = (int64_t)ly.cout * ly.cin * ly.taps;
     const int64_t e = ((int64_t)blockIdx.x * 256 + threadIdx.x) * VEC;

@@ -11,12 +11,33 @@ namespace st {
 // cache: the caller may be the last block of a kernel whose other blocks have just added to them.  Matrices of up to kMiouStage classes
 // are first copied to shared memory in one coalesced pass (one memory latency instead of one per row element).
 constexpr int kMiouStage = 32;
-__device__ __forceinline__ double block_miou(const unsigned long long* conf_g, int C, double* iou, int* present)
+// The copy to shared memory in two halves, for a caller that has other loads to issue while these are on their way:
+// miou_fetch starts the thread's share (blocks of 256 threads, C <= kMiouStage), block_miou takes it over.
+struct MiouFetch { unsigned long long v[kMiouStage * kMiouStage / 256]; };
+__device__ __forceinline__ MiouFetch miou_fetch(const unsigned long long* conf_g, int C)
+{
+    MiouFetch f;
+#pragma unroll
+    for (int k = 0; k < kMiouStage * kMiouStage / 256; ++k) {
+        const int e = threadIdx.x + 256 * k;
+        f.v[k] = e < C * C ? __ldcg(conf_g + e) : 0ull;
+    }
+    return f;
+}
+__device__ __forceinline__ double block_miou(const unsigned long long* conf_g, int C, double* iou, int* present, const MiouFetch* fetched = nullptr)
 {
     __shared__ unsigned long long staged[kMiouStage * kMiouStage];
     const unsigned long long* conf = conf_g;
     if (C <= kMiouStage) {                                 // block-uniform
-        for (int e = threadIdx.x; e < C * C; e += blockDim.x) staged[e] = __ldcg(conf_g + e);
+        if (fetched) {
+#pragma unroll
+            for (int k = 0; k < kMiouStage * kMiouStage / 256; ++k) {
+                const int e = threadIdx.x + 256 * k;
+                if (e < C * C) staged[e] = fetched->v[k];
+            }
+        } else {
+            for (int e = threadIdx.x; e < C * C; e += blockDim.x) staged[e] = __ldcg(conf_g + e);
+        }
         __syncthreads();
         conf = staged;
     }

@@ -81,6 +81,7 @@ struct st_ctx {
     double* ctl_metric = nullptr;           // [S][kCtlPitch]
     int* ctl_n_updates = nullptr;           // [S]
     int* ctl_best_iter = nullptr;           // [S]
+    int* ctl_better = nullptr;              // [S][kCtlPitch]
     unsigned int* bad = nullptr;            // [3]: labels >= C met by a step / by st_agreement; [2] = first device wait that gave up
     uint8_t* mask_tmp = nullptr;            // [P]
     uint8_t* mask_tmp2 = nullptr;           // [P]
@@ -96,6 +97,7 @@ struct st_ctx {
     struct Prefetch { float* feat = nullptr; float* logits = nullptr; cudaEvent_t copied = nullptr, consumed = nullptr; bool pending = false, used_once = false; };
     std::vector<Prefetch> prefetch;
     bool z_current = false;                 // z holds the forward of the current parameters and features of every stream
+    bool z_unkept = false;                  // the last call multiplied its logits inside the loss kernel and kept none of them
     TcPlan* plan = nullptr;
     struct StepGraph { cudaGraphExec_t exec; int64_t n_launches; };
     std::map<GraphKey, StepGraph> graphs;
@@ -332,11 +334,11 @@ st_status enqueue_loss(st_ctx* c, unsigned long long* conf, StageTimer* t = null
 }
 
 // The rest of PartialBackward: gradients of the head's tensors (as split-K partial sums with bf16 GEMMs).
-st_status enqueue_backward(st_ctx* c, StageTimer* t = nullptr, const int* skip = nullptr, int64_t skip_stride = 0)
+st_status enqueue_backward(st_ctx* c, StageTimer* t = nullptr, const int* skip = nullptr, int64_t skip_stride = 0, const TrainCtl* ctl = nullptr)
 {
     cudaStream_t s = c->stream;
     if (c->bf16_mode) {
-        c->launches += tc_backward(c->plan, s, t, skip, skip_stride);
+        c->launches += tc_backward(c->plan, s, t, skip, skip_stride, ctl);
     } else if (c->Ch == 0) {
         ST_REPEAT(t) launch_conv_wgrad_f32(c->x_f32, c->dz, c->Cin, c->C, c->h, c->w, 1, c->grad + c->layout.w_off[0], c->S,
                               (int64_t)c->Cin * c->p, (int64_t)c->C * c->p, c->n_params, s);
@@ -358,10 +360,12 @@ st_status enqueue_backward(st_ctx* c, StageTimer* t = nullptr, const int* skip =
 }
 
 // OptimStep, and the loss of this prediction into loss_buf[slot].  `skip`: per-stream flags (see UpdateArgs).
-st_status enqueue_update(st_ctx* c, int slot, const int* skip, int64_t skip_stride, StageTimer* t = nullptr, const TrainCtl* ctl = nullptr)
+st_status enqueue_update(st_ctx* c, int slot, const int* skip, int64_t skip_stride, StageTimer* t = nullptr, const TrainCtl* ctl = nullptr,
+                         int ctl_mode = 1)
 {
     UpdateArgs u = make_update_args(c, slot, skip, skip_stride);
-    if (ctl) { u.has_ctl = 1; u.ctl = *ctl; u.skip = nullptr; }      // Train: the update judges the prediction itself
+    // Train: the update judges the prediction itself (1), or reads what the backward before it has found (2)
+    if (ctl) { u.has_ctl = ctl_mode; u.ctl = *ctl; u.skip = nullptr; }
     c->launches += launch_sgd_update(u, c->stream);
     if (t) t->mark("sgd_update", c->stream, 1);
     return check_launch(c, "sgd update");
@@ -842,6 +846,7 @@ st_status st_distill_step(st_ctx* ctx, int32_t n_steps, float* loss_out, int64_t
     const bool want_conf = conf_out != nullptr;
     const size_t cc = (size_t)ctx->C * ctx->C;
     ctx->z_current = false;                 // the steps leave z at the forward before the last update
+    ctx->z_unkept = false;
     if (want_conf) {
         if (!ctx->conf_buf) {
             cudaError_t e = dev_alloc(ctx, &ctx->conf_buf, (size_t)ctx->S * kMaxSteps * cc);
@@ -897,7 +902,7 @@ TrainCtl train_ctl(st_ctx* c, int iter, int max_updates, double threshold)
     t.conf_stream_stride = (int64_t)kMaxSteps * c->C * c->C;
     t.C = c->C; t.iter = iter; t.max_updates = max_updates; t.threshold = threshold;
     t.done = c->ctl_done; t.best = c->ctl_best; t.metric = c->ctl_metric;
-    t.n_updates = c->ctl_n_updates; t.best_iter = c->ctl_best_iter;
+    t.n_updates = c->ctl_n_updates; t.best_iter = c->ctl_best_iter; t.better = c->ctl_better;
     t.theta = c->theta; t.best_theta = c->best_theta; t.n_params = c->n_params; t.S = c->S;
     t.param_begin = c->trained_begin;
     return t;
@@ -914,11 +919,14 @@ st_status enqueue_train(st_ctx* c, int max_updates, double threshold)
     for (int i = 0; i <= max_updates && st == ST_OK; ++i) {
         const int* ended_before = i > 0 ? c->ctl_done + i : nullptr;        // done[s][i]: no prediction i for stream s
         st = enqueue_forward(c, nullptr, ended_before, kCtlPitch, false, true);           // prediction <- Forward(student, frame)
-        if (st == ST_OK) st = enqueue_loss(c, c->conf_buf + (int64_t)i * c->C * c->C, nullptr, ended_before, kCtlPitch, i > 0);   // loss, gradient, confusion
-        if (st == ST_OK && i < max_updates) st = enqueue_backward(c, nullptr, ended_before, kCtlPitch);
-        // after the last prediction every loop ends: the launch judges it and finalises its loss
+        if (st == ST_OK) st = enqueue_loss(c, c->conf_buf + (int64_t)i * c->C * c->C, nullptr, ended_before, kCtlPitch, i > 0, false);   // loss, gradient, confusion
+        // metric, best_student, break: judged by an extra block of the backward's first tensor-core kernel while that
+        // kernel works, or, where there is none (fp32 convolutions; the last prediction, after which every loop ends),
+        // by the update itself, which in any case takes the step only where the loop goes on
         const TrainCtl ctl = train_ctl(c, i, max_updates, threshold);
-        if (st == ST_OK) st = enqueue_update(c, i, nullptr, 0, nullptr, &ctl);           // metric, best_student, break, OptimStep
+        const bool side = c->bf16_mode && i < max_updates;
+        if (st == ST_OK && i < max_updates) st = enqueue_backward(c, nullptr, ended_before, kCtlPitch, side ? &ctl : nullptr);
+        if (st == ST_OK) st = enqueue_update(c, i, nullptr, 0, nullptr, &ctl, side ? 2 : 1);
     }
     if (st != ST_OK) return st;
     launch_train_commit(train_ctl(c, 0, max_updates, threshold), c->theta, c->stream);    // student <- best_student
@@ -943,6 +951,7 @@ st_status st_train_key_frame(st_ctx* ctx, double threshold, int32_t max_updates,
     }
     const size_t cc = (size_t)ctx->C * ctx->C;
     ctx->z_current = false;
+    ctx->z_unkept = ctx->fused_fwd != 0;    // the loop's logits never leave the loss kernel
     cudaError_t e = cudaSuccess;
     if (!ctx->conf_buf) e = dev_alloc(ctx, &ctx->conf_buf, (size_t)ctx->S * kMaxSteps * cc);
     if (e == cudaSuccess && !ctx->best_theta) {
@@ -952,6 +961,7 @@ st_status st_train_key_frame(st_ctx* ctx, double threshold, int32_t max_updates,
         if (e == cudaSuccess) e = dev_alloc(ctx, &ctx->ctl_metric, (size_t)ctx->S * kCtlPitch);
         if (e == cudaSuccess) e = dev_alloc(ctx, &ctx->ctl_n_updates, (size_t)ctx->S);
         if (e == cudaSuccess) e = dev_alloc(ctx, &ctx->ctl_best_iter, (size_t)ctx->S);
+        if (e == cudaSuccess) e = dev_alloc(ctx, &ctx->ctl_better, (size_t)ctx->S * kCtlPitch);
     }
     if (e != cudaSuccess) return fail(ctx, ST_ERR_OOM, "st_train_key_frame: %s", cudaGetErrorString(e));
     ST_CUDA(ctx, cudaMemsetAsync(ctx->conf_buf, 0, (size_t)ctx->S * kMaxSteps * cc * sizeof(unsigned long long), ctx->stream));
@@ -1105,6 +1115,7 @@ st_status student_forward(st_ctx* ctx, int32_t stream, const char* who)
     if (ctx->z_current) return ST_OK;       // an earlier call already ran it and nothing has changed since
     st_status st = enqueue_forward(ctx);
     ctx->z_current = st == ST_OK;
+    if (st == ST_OK) ctx->z_unkept = false;
     return st;
 }
 
@@ -1239,6 +1250,10 @@ st_status st_read_tensor(st_ctx* ctx, int32_t stream, st_tensor which, float* ds
     }
     const float* src = nullptr;
     const int64_t s = stream;
+    if ((which == ST_TENSOR_LOGITS || which == ST_TENSOR_LOGIT_GRAD) && ctx->z_unkept) {
+        st = student_forward(ctx, stream, "st_read_tensor");     // the forward of the student the last call left behind
+        if (st != ST_OK) return st;
+    }
     switch (which) {
         case ST_TENSOR_LOGITS: src = ctx->z + s * ctx->C * ctx->p; break;
         case ST_TENSOR_LOGIT_GRAD:

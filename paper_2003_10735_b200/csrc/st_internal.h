@@ -184,6 +184,7 @@ struct TrainCtl {
     int* done;                        // [S][kCtlPitch]
     double* best;                     // [S][kCtlPitch]
     double* metric;                   // [S][kCtlPitch]  metric of prediction i; -1 where the loop had ended before
+    int* better;                      // [S][kCtlPitch]  prediction i was the best so far (best_student <- student)
     int* n_updates;                   // [S] updates taken when the loop ended
     int* best_iter;                   // [S] updates behind best_student
     const float* theta;               // [S][n_params]
@@ -237,7 +238,7 @@ struct UpdateArgs {
     // prediction's confusion matrix (same counts, same arithmetic, same answer), keeps the old value of its parameters
     // as best_student's where the metric is the best so far, and leaves them alone where the loop has ended; block 0
     // writes the history.  `skip` is then not used.
-    int has_ctl;
+    int has_ctl;             // 0; 1: this kernel judges the prediction; 2: the backward before it has (see tc_backward), read the outcome
     TrainCtl ctl;
 };
 // step_base[s] += add (add_per_stream == nullptr) or += add_per_stream[s]
@@ -323,6 +324,9 @@ int tc_forward(const TcPlan*, cudaStream_t s, StageTimer* t = nullptr, const int
                bool after_update = false, int first_block = 0);
 int tc_forward_blocks(const TcPlan*, int first, int last, cudaStream_t s, StageTimer* t = nullptr, const int* skip = nullptr,
                       int64_t skip_stride = 0);
-int tc_backward(const TcPlan*, cudaStream_t s, StageTimer* t = nullptr, const int* skip = nullptr, int64_t skip_stride = 0);
+// `ctl` (Train): one extra block per stream of the first kernel judges the prediction the backward belongs to, beside the
+// kernel's own work; the update that follows reads the outcome.
+int tc_backward(const TcPlan*, cudaStream_t s, StageTimer* t = nullptr, const int* skip = nullptr, int64_t skip_stride = 0,
+                const TrainCtl* ctl = nullptr);
 
 }  // namespace st
