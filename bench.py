@@ -43,6 +43,8 @@ EX2_PER_CLASS_PIXEL = 1.0
 NCU_DRAM_BYTES = {
     (2, "upsample_ce"): 5.85e6,      # profiles/upsample_ce_rows_720p.md
 }
+# st_init_head reads this when a context is made: "0" keeps the classifier's forward in a kernel of its own
+FUSED_SWITCH = "ST_FUSED_FORWARD"
 
 
 def read_peaks():
@@ -236,12 +238,20 @@ def kernel_table(st, ctx, cfg, peaks, arith, n_profile_steps):
     kernels = {}
     for name, ms in st.st_profile_step(ctx, n_profile_steps):
         k = {"ms": ms, "per_key_frame": K}
-        if name == "upsample_ce":
+        if name in ("upsample_ce", "fwd1x1_upsample_ce"):
             class_pixels = float(C) * P * S
             k.update(bound="alu", achieved=ALU_FLOP_PER_CLASS_PIXEL * class_pixels / ms / 1e9, peak=arith["fma_tflops"],
                      unit="TFLOP/s", hbm_gbs=S * (2 * C * p * 4 + P) / ms / 1e6,
                      xu={"achieved": EX2_PER_CLASS_PIXEL * class_pixels / ms / 1e9, "peak": arith["ex2_tops"],
                          "unit": "1e12 exp2/s", "frac": EX2_PER_CLASS_PIXEL * class_pixels / ms / 1e9 / arith["ex2_tops"]})
+            if name == "fwd1x1_upsample_ce":
+                # the kernel also multiplies its own logit tiles (Forward of the 1x1 classifier): every block fetches the
+                # 9 x 32 nodes around its 7 x 30 from L2, so the launch streams 288/210 of the feature map
+                n_tiles = -(-cfg.feat_h // 7) * -(-cfg.feat_w // 30)
+                k.update(hbm_gbs=S * (p * c_last * 2 + P) / ms / 1e6,
+                         forward={"tensor_tflops": 2.0 * S * n_tiles * 384 * 32 * c_last / ms / 1e9,
+                                  "feature_bytes_fetched_by_blocks": S * n_tiles * 288 * c_last * 2,
+                                  "note": "replaces tc_fwd1x1 + upsample_ce (see kernels_unfused for those two)"})
         elif name == "tc_fwd1x1":
             k.update(bound="hbm", achieved=S * (p * c_last * 2 + C * p * 4) / ms / 1e6, peak=hbm, unit="GB/s",
                      tflops=2.0 * S * p * C * c_last / ms / 1e9)
@@ -341,8 +351,10 @@ def run_confident_student(st, torch, stream, cfg, peaks, arith):
     loss = torch.zeros((1, K), dtype=torch.float32, device="cuda")
     ms = timed_blocks(torch, stream, torch.cuda.synchronize, 5, 20, lambda i: st.st_distill_step(ctx, K, loss))
     kernels = kernel_table(st, ctx, cfg, peaks, arith, 10)
+    loss_kernel = "fwd1x1_upsample_ce" if "fwd1x1_upsample_ce" in kernels else "upsample_ce"
     out = {"miou_when_timed": miou, "steps_to_get_there": n_steps, "ms_per_step": statistics.median(ms) / 20 / K,
-           "upsample_ce_ms": kernels["upsample_ce"]["ms"], "upsample_ce_frac": kernels["upsample_ce"].get("frac"),
+           "upsample_ce_ms": kernels[loss_kernel]["ms"], "upsample_ce_frac": kernels[loss_kernel].get("frac"),
+           "loss_kernel": loss_kernel,
            "miou_after": st.st_agreement(ctx, 0, None, None, None)}
     st.st_destroy(ctx)
     return out
@@ -477,7 +489,7 @@ def run_ours(args, cfg):
         d2h = S * (n_params * 4 + 8)
 
         # ---- per-kernel times with CUDA events on the launching stream
-        kernels, train, others, confident = {}, {}, {}, None
+        kernels, train, others, confident, unfused = {}, {}, {}, None, None
         if rank == 0:
             ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
 
@@ -523,6 +535,19 @@ def run_ours(args, cfg):
             agree["student_mask_fused"] = {"kernel_us": t_own * 1e3, "note": "arg-max of the upsampled logits + confusion + mean IoU, forward reused"}
             kernels["agreement"] = {"ms": agree["coherent_masks"]["kernel_us"] / 1e3, "bound": "latency", "per_key_frame": S, **agree}
             kernels.update(kernel_table(st, ctx, cfg, peaks, arith, 20))
+            if "fwd1x1_upsample_ce" in kernels:
+                # the same step with the classifier's forward in its own kernel, for the two kernels' own rooflines
+                os.environ[FUSED_SWITCH] = "0"
+                ctx_u = make_context(st, stream, cfg, theta0)
+                os.environ.pop(FUSED_SWITCH)
+                st.st_set_frozen_features(ctx_u, 0, feats_d[0][0])
+                st.st_teacher_labels(ctx_u, 0, logits_d[0][0])
+                for _ in range(3):
+                    st.st_distill_step(ctx_u, K, loss_d[0:1])
+                ms_u = statistics.median(timed_blocks(torch, stream, barrier, 5, 50, lambda i: st.st_distill_step(ctx_u, K, loss_d[0:1]))) / 50
+                unfused = kernel_table(st, ctx_u, si.get_config(args.workload), peaks, arith, 20)
+                unfused["distill_loop_only_ms_per_step"] = ms_u / K
+                st.st_destroy(ctx_u)
             # Train of Algorithm 1 (forward, metric, break test and best-student snapshot per update, all on the device):
             # the full loop (a threshold no mean IoU reaches) and a loop that ends on the first metric
             for name, thr in (("full_loop", 2.0), ("ends_at_once", 0.0)):
@@ -570,7 +595,7 @@ def run_ours(args, cfg):
                 "arithmetic_peaks": arith,
                 "key_frames_per_s": world * args.steps / (ms_total / 1e3),
                 "distill_loop_only": {"steps_per_s": K * S / (ms_loop / 1e3), "ms_per_k_steps": ms_loop},
-                "kernels": kernels, "train_key_frame": train,
+                "kernels": kernels, "kernels_unfused": unfused, "train_key_frame": train,
                 "last_loss": float(loss_d[0, -1].item()), "last_miou": mious[0], "last_miou_device_run": last_miou_dev,
             }
         st.st_destroy(ctx)

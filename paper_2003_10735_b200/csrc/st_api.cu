@@ -328,7 +328,7 @@ st_status enqueue_loss(st_ctx* c, unsigned long long* conf, StageTimer* t = null
         k3.z_out = keep_logits ? c->z : nullptr;         // logits that the next iteration overwrites unread stay on the chip
     }
     ST_REPEAT(t) launch_upsample_ce(k3, &c->k3_map, s, &c->fx_map, &c->fw_map);
-    if (t) t->mark("upsample_ce", s, st_repeats(t));
+    if (t) t->mark(k3.fused ? "fwd1x1_upsample_ce" : "upsample_ce", s, st_repeats(t));
     c->launches += st_repeats(t);
     return check_launch(c, "upsample + cross-entropy");
 }
