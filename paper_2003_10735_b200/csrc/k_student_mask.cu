@@ -223,6 +223,7 @@ cudaError_t prepare_student_mask(int C)
 
 void launch_student_mask(const StudentMaskArgs& a, cudaStream_t s)
 {
+    if (a.fused) { launch_student_eval(a, s); return; }
     int chunk;
     const bool conf = a.labels != nullptr;
     const size_t smem = mask_smem(a.C, conf, &chunk);

@@ -35,6 +35,7 @@
 // from pass 1's exponentials and counted against the label in a shared-memory confusion matrix.
 #include "st_internal.h"
 #include "tc_common.cuh"
+#include "fused_tile.cuh"
 
 #include <string.h>
 
@@ -42,16 +43,13 @@ namespace st {
 
 namespace {
 
-constexpr int RN_Y = 7, RN_X = 30;
+constexpr int RN_Y = fused::kOwnRows, RN_X = fused::kOwnCols;      // nodes a block owns: 7 rows x 30 columns
 constexpr int R_WARPS = RN_Y + 1, R_THREADS = R_WARPS * 32;
 constexpr int TZ_H = RN_Y + 2;
 // Columns of a tile row (template parameter TW of everything below): 36 when the logits are fetched from global memory
 // (32 used, starting at a multiple of 4 so that rows are whole 16-byte vectors), 32 when the block computes its logits
 // itself (kTwFused).
-constexpr int kTwLoad = 36, kTwFused = 32;
-// The block computes its own logits: one 64-channel slice of the feature tile (9 x 32 pixels, 128 bytes each) per stage
-constexpr uint32_t kStageBytes = TZ_H * kTwFused * 128, kWeightBytes = kClassPad * 128;
-constexpr int kFusedStages = 2, kFusedTmemCols = 128, kFusedMaxKBlocks = 4;
+constexpr int kTwLoad = 36, kTwFused = fused::kTileCols;
 constexpr float kLog2e = 1.4426950408889634f, kLn2 = 0.6931471805599453f;
 // Classes per iteration of the two fast-path class sweeps.  The sweeps are rolled loops: unrolled over all classes
 // they were ~70 KB of straight-line code that every warp ran through once, and instruction fetch was the main stall.
@@ -221,9 +219,9 @@ upsample_ce_rows_kernel(UpsampleCeArgs a, const __grid_constant__ CUtensorMap z_
     int* corr = (int*)(zt + CB * TZ);           // [C][TZ_H][TW]    -64 * (adjoint of onehot)
     float2* acc = (float2*)(corr + C * TZ);     // [R_WARPS][C][32] (x, y): the cell's pull on its upper / lower node row
     unsigned int* hist = (unsigned int*)(acc + R_WARPS * C * 32);   // [C][C] (CONF): the block's share of the confusion matrix
-    __shared__ float red[R_WARPS], red_m[R_WARPS], sbias[kClassPad];
-    __shared__ __align__(8) uint64_t tile_bar, mm_bar[2 * kFusedStages + 2];   // FUSED: full[2], empty[2], weights, done
-    __shared__ uint32_t tmem_slot, gave_up;
+    __shared__ float red[R_WARPS], red_m[R_WARPS];
+    __shared__ __align__(8) uint64_t tile_bar;
+    __shared__ fused::Shared fsh;               // FUSED: barriers, tensor-memory slot, bias of the block's own forward
 
     // Launch order: the last block row first, then rows 0, 1, ...  Blocks at the frame border do extra work, and the
     // blocks that reach an SM first finish earlier than their later companions, so the border rows go first.
@@ -308,126 +306,21 @@ upsample_ce_rows_kernel(UpsampleCeArgs a, const __grid_constant__ CUtensorMap z_
     float m_loc = -INFINITY;                               // largest logit of this thread's share of the tile
     uint32_t tmem = 0;                                     // FUSED: the block's tensor memory (given back at the very end)
     if constexpr (FUSED) {
-        // ---- Forward for a 1x1 classifier, inside the block: z[pix][c] = b[c] + sum_k X[pix][k] W[c][k] for the 9 x 32
-        // nodes of the tile.  The feature tile arrives in 64-channel slices (one 4-d tile copy each, rows and columns
-        // outside the map arrive as zeros) through a ring of two stages, the classifier weights in one barrier's worth of
-        // copies; one thread issues three 128 x 32 x 16 tcgen05 multiplications per 16 channels (pixel rows 288 .. 383 of
-        // the third one read whatever follows the stage: their results are never looked at), the accumulators (fp32, in
-        // tensor memory) are drained into the logit tile by all warps.
-        const uint32_t ring = tc::smem_u32(zt), w_base = ring + kFusedStages * kStageBytes;
-        const uint32_t bar0 = tc::smem_u32(&mm_bar[0]);
-        auto full_bar = [&](int st) { return bar0 + 8u * (uint32_t)st; };
-        auto empty_bar = [&](int st) { return bar0 + 8u * (uint32_t)(kFusedStages + st); };
-        const uint32_t w_bar = bar0 + 8u * (2 * kFusedStages), done_bar = w_bar + 8u;
-        if (wi == 0) tc::tmem_alloc(tc::smem_u32(&tmem_slot), kFusedTmemCols);
-        if (tid == 0) {
-            for (int k = 0; k < 2 * kFusedStages + 2; ++k) tc::mbar_init(bar0 + 8u * (uint32_t)k, 1);
-            gave_up = 0;
-            tc::fence_barrier_init();
-        }
-        tc::tc_fence_before_sync();
-        __syncthreads();
-        tc::tc_fence_after_sync();
-        tmem = tmem_slot;
-        const int kblocks = a.kblocks;
-        // x_early: the kernel before this one on the stream (the previous iteration's update) does not write the features,
-        // and this launch may have started while that one still runs: the first slices are fetched before the wait
-        const int n_pre = a.x_early ? min(kFusedStages, kblocks) : 0;
-        if (tid == 0)
-            for (int kb = 0; kb < n_pre; ++kb) {
-                tc::mbar_expect_tx(full_bar(kb), kStageBytes);
-                tc::tma_load_4d(ring + kb * kStageBytes, &x_map, full_bar(kb), kb * 64, x0 - 1, y0 - 1, s);
-            }
-        pdl_wait();                                        // the weights come from the previous kernel of the stream
-        if (a.skip && a.skip[(int64_t)s * a.skip_stride]) {           // this stream's training loop has ended (block-uniform)
-            if (tid == 0)                                   // copies already on their way land before shared memory is given back
-                for (int kb = 0; kb < n_pre; ++kb) tc::mbar_wait(full_bar(kb), 0, a.err, tc::kWaitFull);
-            tc::tc_fence_before_sync();
-            __syncthreads();
-            if (wi == 0) tc::tmem_dealloc(tmem, kFusedTmemCols);
-            return;
-        }
-        if (tid < kClassPad) sbias[tid] = tid < C ? a.theta[(int64_t)s * a.n_params + a.b_off + tid] : 0.f;
-        bool ok = true;
-        if (tid == 0) {
-            tc::mbar_expect_tx(w_bar, (uint32_t)kblocks * kWeightBytes);
-            for (int kb = 0; kb < kblocks; ++kb) tc::tma_load_3d(w_base + kb * kWeightBytes, &w_map, w_bar, kb * 64, 0, s);
-            for (int kb = n_pre; kb < kblocks && ok; ++kb) {
-                const int st = kb % kFusedStages;
-                if (kb >= kFusedStages) ok = tc::mbar_wait(empty_bar(st), ((kb / kFusedStages) - 1) & 1, a.err, tc::kWaitEmpty);
-                if (ok) {
-                    tc::mbar_expect_tx(full_bar(st), kStageBytes);
-                    tc::tma_load_4d(ring + st * kStageBytes, &x_map, full_bar(st), kb * 64, x0 - 1, y0 - 1, s);
-                }
-            }
-        } else if (tid == 32) {
-            constexpr uint32_t idesc = tc::instr_desc(128, kClassPad, 0, 0);
-            ok = tc::mbar_wait(w_bar, 0, a.err, tc::kWaitFull);
-            for (int kb = 0; kb < kblocks && ok; ++kb) {
-                const int st = kb % kFusedStages;
-                ok = tc::mbar_wait(full_bar(st), (kb / kFusedStages) & 1, a.err, tc::kWaitFull);
-                if (!ok) break;
-                tc::tc_fence_after_sync();
-#pragma unroll
-                for (int m = 0; m < 3; ++m)
-#pragma unroll
-                    for (int k = 0; k < 4; ++k)
-                        tc::umma(tmem + m * kClassPad, tc::smem_desc(ring + st * kStageBytes + m * (128 * 128) + k * 32, 16, 1024),
-                                 tc::smem_desc(w_base + kb * kWeightBytes + k * 32, 16, 1024), idesc, (kb | k) != 0);
-                tc::umma_commit(empty_bar(st));
-            }
-            if (!ok) gave_up = 1;
-            tc::umma_commit(done_bar);
-        }
-        __syncwarp();
-        ok = tc::mbar_wait(done_bar, 0, a.err, tc::kWaitDone);
-        tc::tc_fence_after_sync();
-        if (!__syncthreads_and(ok) || gave_up) {           // block-uniform: a wait ran out; nothing is written
-            tc::drain_after_error();
-            tc::tc_fence_before_sync();
-            __syncthreads();
-            if (wi == 0) tc::tmem_dealloc(tmem, kFusedTmemCols);
-            return;
-        }
-        // the stages are dead: the arrays they lay over get their initial contents
-        {
-            float4* zt4 = reinterpret_cast<float4*>(zt);
-            for (int e = tid; e < (CB - C) * (TZ / 4); e += R_THREADS) zt4[C * (TZ / 4) + e] = make_float4(-1e30f, -1e30f, -1e30f, -1e30f);
+        // ---- Forward for a 1x1 classifier, inside the block (fused_tile.cuh)
+        fused::Args fa;
+        fa.kblocks = a.kblocks; fa.x_early = a.x_early;
+        fa.skip = a.skip ? a.skip + (int64_t)s * a.skip_stride : nullptr;
+        fa.err = a.err;
+        fa.bias = a.theta + (int64_t)s * a.n_params + a.b_off;
+        fa.z_out = a.z_out ? a.z_out + (int64_t)s * C * p : nullptr;
+        fa.C = C; fa.h = h; fa.w = w;
+        auto after_mma = [&]() {                        // the arrays the stages lay over get their initial contents
             for (int e = tid; e < C * TZ / 4; e += R_THREADS) reinterpret_cast<int4*>(corr)[e] = make_int4(0, 0, 0, 0);
             if (CONF) for (int e = tid; e < C * C; e += R_THREADS) hist[e] = 0;
-        }
-        // accumulator m holds tile rows 4m .. 4m+3 (one row of 32 nodes per 32 lanes of tensor memory, and a warp reaches
-        // the lanes 32 (warp % 4) ..): warps 0-3 drain rows 0-3, warps 4-7 rows 4-7, warps 0 and 4 half of the classes of
-        // row 8 each
-        auto put_row = [&](const float* v, int n_cols, int c0, int j) {     // v[i]: class c0 + i of node (row j, column l)
-            const int ny = y0 - 1 + j, nx = x0 - 1 + l;
-            const bool in_frame = ny >= 0 && ny < h && nx >= 0 && nx < w;
-            // the block's own nodes go to global memory as well where the caller wants the logits kept
-            const bool keep = a.z_out && in_frame && j >= 1 && j <= RN_Y && l >= 1 && l <= RN_X;
-            float* dst = zt + c0 * TZ + j * TW + l;
-            float* zo = a.z_out + ((int64_t)s * C + c0) * p + (int64_t)ny * w + nx;
-#pragma unroll
-            for (int i = 0; i < 32; ++i)
-                if (i < n_cols && c0 + i < C) {
-                    const float t = v[i] + sbias[c0 + i];
-                    dst[i * TZ] = t;
-                    if (in_frame) m_loc = fmaxf(m_loc, t);
-                    if (keep) zo[(int64_t)i * p] = t;
-                }
         };
-        {
-            float v[32];
-            tc::tmem_ld_32x32(tmem + ((uint32_t)((wi & 3) * 32) << 16) + (wi >> 2) * kClassPad, v);
-            put_row(v, 32, 0, wi);
-        }
-        if ((wi & 3) == 0) {
-            const int c0 = wi ? 16 : 0;
-            float v[32];
-            tc::tmem_ld_32x16(tmem + 2 * kClassPad + c0, reinterpret_cast<float(&)[16]>(v));
-            put_row(v, 16, c0, 8);
-        }
-        tc::tc_fence_before_sync();
-        __syncthreads();                                   // the tile is complete (its entries outside the frame are never read)
+        const fused::Tile tile = fused::logit_tile<CB>(fa, &x_map, &w_map, fsh, zt, s, x0, y0, after_mma);
+        if (!tile.ok) return;
+        m_loc = tile.m_loc; tmem = tile.tmem;
     } else
     {
         // a thread keeps one 16-byte group of the tile plane (81 groups) and walks the classes three at a time
@@ -826,13 +719,7 @@ upsample_ce_rows_kernel(UpsampleCeArgs a, const __grid_constant__ CUtensorMap z_
         for (int k = 0; k < R_WARPS; ++k) t += red[k];
         a.loss_part[(int64_t)s * n_blk + blk] = t;
     }
-    if constexpr (FUSED) {
-        if (wi == 0) {                           // every warp's reads of tensor memory ended before the barriers above
-            __syncwarp();
-            tc::tc_fence_after_sync();
-            tc::tmem_dealloc(tmem, kFusedTmemCols);
-        }
-    }
+    if constexpr (FUSED) fused::free_tmem(tmem);     // every warp's reads of tensor memory ended before the barriers above
 }
 
 template <int CB, int TW>
@@ -841,11 +728,7 @@ size_t rows_smem_bytes(int C, bool conf)
     constexpr size_t TZ = (size_t)TZ_H * TW;
     const size_t plain = ((size_t)CB * TZ + (size_t)C * TZ + (size_t)R_WARPS * C * 32 * 2 + (conf ? (size_t)C * C : 0)) * sizeof(float) + 128;
     if (TW != kTwFused) return plain;
-    // the feature stages and the weights lie over the kernel's arrays; the third multiplication of the last stage reads
-    // 384 pixel rows from the stage's start; 1 KB so that the stages can start at a multiple of 1024
-    const size_t ring = (size_t)kFusedStages * kStageBytes + (size_t)kFusedMaxKBlocks * kWeightBytes;
-    const size_t reach = (size_t)(kFusedStages - 1) * kStageBytes + 384 * 128;
-    return (plain > ring ? (plain > reach ? plain : reach) : (ring > reach ? ring : reach)) + 1024;
+    return fused::smem_bytes(plain);      // the feature stages and the weights lie over the kernel's arrays
 }
 
 template <int CB>
@@ -921,7 +804,7 @@ void launch_upsample_ce_rows(const UpsampleCeArgs& a, const CUtensorMap* z_map, 
 // and the feature map is at least one tile large.
 bool fused_forward_supported(int C, int h, int w, int c_in)
 {
-    return upsample_ce_rows_supported(C) && c_in >= 64 && c_in % 64 == 0 && c_in / 64 <= kFusedMaxKBlocks && w >= kTwFused && h >= TZ_H;
+    return upsample_ce_rows_supported(C) && c_in >= 64 && c_in % 64 == 0 && c_in / 64 <= fused::kMaxKBlocks && w >= fused::kTileCols && h >= fused::kTileRows;
 }
 
 bool make_logit_tile_map(CUtensorMap* m, const float* z, int S, int C, int h, int w)

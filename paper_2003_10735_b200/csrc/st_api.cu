@@ -692,7 +692,8 @@ st_status st_init_head(const st_head_desc* desc, const float* init_params, st_ct
             const uint32_t box[3] = {64, (uint32_t)kClassPad, 1};
             c->fused_fwd = make_feature_tile_map(&c->fx_map, c->x_bf16, S, c->Cin, c->h, c->w) &&
                            encode_tensor_map(&c->fw_map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, CU_TENSOR_MAP_SWIZZLE_128B, c->w2_shadow, 3,
-                                             dims, str, box, msg, sizeof msg, "1x1 weight");
+                                             dims, str, box, msg, sizeof msg, "1x1 weight") &&
+                           prepare_student_eval(c->C) == cudaSuccess;
         }
     }
     if (e == cudaSuccess) e = cudaStreamSynchronize(c->stream);   // init_params may be released on return
@@ -1125,6 +1126,12 @@ StudentMaskArgs mask_args(st_ctx* ctx, int32_t stream, uint8_t* mask)
     a.z = ctx->z + (int64_t)stream * ctx->C * ctx->p;
     a.C = ctx->C; a.h = ctx->h; a.w = ctx->w;
     a.mask = mask;
+    if (ctx->fused_fwd) {               // the mask kernel multiplies the logits itself: no forward before it, `z` is not read
+        a.fused = 1; a.kblocks = ctx->Cin / 64; a.stream = stream;
+        a.bias = ctx->theta + (int64_t)stream * ctx->n_params + ctx->layout.b_off[ctx->layout.n_layers - 1];
+        a.err = ctx->bad + 2;
+        a.x_map = &ctx->fx_map; a.w_map = &ctx->fw_map;
+    }
     return a;
 }
 }  // namespace
@@ -1134,7 +1141,7 @@ st_status st_student_mask(st_ctx* ctx, int32_t stream, uint8_t* mask_out)
     st_status st = check_stream_index(ctx, stream);
     if (st != ST_OK) return st;
     if (!mask_out) return fail(ctx, ST_ERR_INVALID_ARG, "st_student_mask: NULL destination");
-    st = student_forward(ctx, stream, "st_student_mask");
+    st = ctx->fused_fwd ? ready_to_run(ctx, "st_student_mask", false) : student_forward(ctx, stream, "st_student_mask");
     if (st != ST_OK) return st;
     const bool dev = is_device_ptr(mask_out);
     // the kernel writes the mask two pixels (16 bits) at a time: a destination at an odd address gets its
@@ -1177,7 +1184,7 @@ st_status st_agreement(st_ctx* ctx, int32_t stream, const uint8_t* pred, const u
     double* miou_res = miou_direct ? miou : ctx->miou_tmp;
     if (!pred && student_mask_fused_supported(ctx->C)) {
         // the student's own mask: arg-max, confusion and mean IoU in one kernel, the mask itself is not stored
-        st = student_forward(ctx, stream, "st_agreement");
+        st = ctx->fused_fwd ? ready_to_run(ctx, "st_agreement", false) : student_forward(ctx, stream, "st_agreement");
         if (st != ST_OK) return st;
         StudentMaskArgs a = mask_args(ctx, stream, nullptr);
         a.labels = d_label; a.conf = ctx->conf_tmp; a.bad = ctx->bad + 1; a.miou = miou_res;

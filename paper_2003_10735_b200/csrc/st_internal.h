@@ -149,7 +149,16 @@ struct StudentMaskArgs {
     double* miou;              // nullptr: no mean IoU
     unsigned int* ticket;      // zero between launches (block counter for the mean IoU)
     unsigned long long* conf_out;  // with `miou`: the last block writes the finished matrix here and clears `conf`
+    // One-layer head with bf16 features: the kernel multiplies the logits itself (k_student_eval.cu) and `z` is not read
+    int fused;                 // 0, or 1: the fields below are set
+    int kblocks, stream;       // 64-channel slices of the features; the stream (a coordinate of the tile maps)
+    const float* bias;         // the classifier's bias of that stream (fp32 master parameters)
+    unsigned int* err;         // device word: first wait that gave up
+    const CUtensorMap* x_map;  // host copies of the tile maps of the features (make_feature_tile_map) and of the bf16 weights
+    const CUtensorMap* w_map;
 };
+cudaError_t prepare_student_eval(int C);    // once per device and class count, outside any stream capture
+cudaError_t launch_student_eval(const StudentMaskArgs& a, cudaStream_t s);
 bool student_mask_fused_supported(int C);   // confusion counters fit shared memory
 cudaError_t prepare_student_mask(int C);    // once per device and class count, outside any stream capture
 void launch_student_mask(const StudentMaskArgs& a, cudaStream_t s);
