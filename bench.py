@@ -42,6 +42,9 @@ EX2_PER_CLASS_PIXEL = 1.0
 # An entry is removed whenever its kernel changes and put back after the next capture.
 NCU_DRAM_BYTES = {
     (2, "upsample_ce"): 5.85e6,      # profiles/upsample_ce_rows_720p.md
+    # profiles/fwd1x1_upsample_ce_rows_720p.md: a capture starts with cold caches, so the feature map (29.5 MB, L2 resident
+    # over the K iterations of the step loop) is read from DRAM once; labels 0.92 MB
+    (2, "fwd1x1_upsample_ce"): 30.53e6,
 }
 # st_init_head reads this when a context is made: "0" keeps the classifier's forward in a kernel of its own
 FUSED_SWITCH = "ST_FUSED_FORWARD"
@@ -394,12 +397,17 @@ def run_ours(args, cfg):
             feats_h.append(per_stream_f)
             logits_h.append(per_stream_t)
         for s in range(S):
-            thetas.append(si.initial_head_params(cfg.c_in, cfg.c_hidden, C, 1000 + s))
+            thetas.append(si.initial_stack_params(cfg.c_in, cfg.blocks, C, 1000 + s) if cfg.blocks
+                          else si.initial_head_params(cfg.c_in, cfg.c_hidden, C, 1000 + s))
         theta0 = np.concatenate(thetas)
         theta0_d = torch.from_numpy(theta0).cuda().reshape(S, -1)
         feats_d = [[f.cuda(non_blocking=True) for f in fs] for fs in feats_h]
         logits_d = [[t.cuda(non_blocking=True) for t in ts] for ts in logits_h]
-        ctx = make_context(st, stream, cfg, theta0)
+        stack_kw = dict(blocks=[tuple(b) for b in cfg.blocks], first_trained=cfg.first_trained) if cfg.blocks else {}
+        ctx = make_context(st, stream, cfg, theta0, **stack_kw)
+        for s in range(S if cfg.blocks else 0):      # a stack of blocks: the skip inputs are cached like the features
+            for b in range(len(cfg.blocks)):
+                st.st_set_skip_features(ctx, s, b, torch.from_numpy(si.skip_features(cfg, b, s)).cuda())
         n_params = ctx.n_params
         packed_d = torch.empty((S, n_params), dtype=torch.float32, device="cuda")
         packed_h = torch.empty((S, n_params), dtype=torch.float32).pin_memory()
