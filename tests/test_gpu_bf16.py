@@ -309,3 +309,69 @@ def test_a_wait_that_runs_out_is_reported_and_nothing_else_breaks(monkeypatch):
     l_ref, _, _ = oracle.gradients(hq, feat, oracle.teacher_labels(T))
     assert abs(loss[0] - l_ref) <= 2e-5 * abs(l_ref)
     st.st_destroy(good)
+
+
+@pytest.mark.parametrize("c_in,C,h,w,S", [
+    (64, 5, 9, 32, 1),       # the smallest map the block-level forward takes: one tile, one 64-channel slice
+    (128, 21, 24, 40, 2),    # two streams, ragged tiles in both directions
+    (192, 32, 23, 95, 1),    # three slices, all 32 class rows, a last tile column of five nodes
+    (256, 19, 30, 61, 1),    # four slices (the ring of two is refilled), a last tile column of one node
+])
+def test_forward_inside_the_loss_kernel_equals_the_separate_forward(c_in, C, h, w, S, monkeypatch):
+    """A one-layer head multiplies its logits inside the loss kernel and inside the student-mask kernel.  With
+    ST_FUSED_FORWARD=0 at context creation the same steps run with the forward as a kernel of its own.  Both forms
+    multiply the same bf16 operands in the same order, so the logits agree bit by bit as long as the parameters do.
+    The loss kernel shifts its exponentials by the largest logit of the block's tile, and the two forms' tiles differ
+    (36 columns from a multiple of four against 32 from the block's first node), so sums of exponentials can round
+    differently in the last place: everything downstream is compared to a few units in the last place, integer
+    counts to a handful of pixels."""
+    K = 3
+    probs = [problem(10 + s, c_in, C, h, w) for s in range(S)]
+    theta = np.concatenate([si.initial_head_params(c_in, 0, C, 20 + s) for s in range(S)])
+
+    def run(fused):
+        if not fused:
+            monkeypatch.setenv("ST_FUSED_FORWARD", "0")
+        ctx = make_ctx(c_in, 0, C, h, w, theta, S=S, lr=0.05, mu=0.9)
+        monkeypatch.delenv("ST_FUSED_FORWARD", raising=False)
+        for s in range(S):
+            st.st_set_frozen_features(ctx, s, dev(probs[s][0]))
+            st.st_teacher_labels(ctx, s, dev(probs[s][1]))
+        loss = np.zeros((S, K), np.float32)
+        conf = np.zeros((S, K, C, C), np.int64)
+        st.st_distill_step(ctx, K, loss, conf)
+        out = {"loss": loss, "conf": conf, "launches": st.st_launch_count(ctx)}
+        out["z"] = [st.st_read_tensor(ctx, s, st.ST_TENSOR_LOGITS) for s in range(S)]
+        out["dz"] = [st.st_read_tensor(ctx, s, st.ST_TENSOR_LOGIT_GRAD) for s in range(S)]
+        out["theta"] = [packed(ctx, s) for s in range(S)]
+        masks, agree = [], []
+        for s in range(S):
+            m = torch.empty((4 * h, 4 * w), dtype=torch.uint8, device="cuda")
+            st.st_student_mask(ctx, s, m)
+            masks.append(m.cpu().numpy())
+            c = np.zeros((C, C), np.int64)
+            agree.append((st.st_agreement(ctx, s, None, None, c), c))
+        out["mask"], out["agree"] = masks, agree
+        n_upd = np.zeros(S, np.int32); best = np.zeros(S, np.float64); met = np.zeros((S, K + 1), np.float64)
+        st.st_train_key_frame(ctx, 2.0, K, n_upd, best, met)
+        out["train"] = (n_upd, best, met, [packed(ctx, s) for s in range(S)])
+        st.st_destroy(ctx)
+        return out
+
+    a, b = run(True), run(False)
+    assert a["launches"] < b["launches"]                      # the forward really was part of another kernel
+    P = 16 * h * w
+    np.testing.assert_allclose(a["loss"], b["loss"], rtol=2e-6)
+    assert np.abs(a["conf"] - b["conf"]).sum(axis=(2, 3)).max() <= 2 * max(4, P // 1000)
+    for s in range(S):
+        np.testing.assert_allclose(a["z"][s], b["z"][s], rtol=1e-5, atol=1e-5)
+        np.testing.assert_allclose(a["dz"][s], b["dz"][s], rtol=1e-4, atol=1e-10)
+        np.testing.assert_allclose(a["theta"][s], b["theta"][s], rtol=1e-5, atol=1e-7)
+        assert (a["mask"][s] != b["mask"][s]).sum() <= max(4, P // 1000)
+        assert abs(a["agree"][s][0] - b["agree"][s][0]) <= 1e-3
+        assert np.abs(a["agree"][s][1] - b["agree"][s][1]).sum() <= 2 * max(4, P // 1000)
+        assert int(a["agree"][s][1].sum()) == P and int(b["agree"][s][1].sum()) == P
+        np.testing.assert_allclose(a["train"][3][s], b["train"][3][s], rtol=1e-4, atol=1e-6)
+    assert (a["train"][0] == b["train"][0]).all()             # updates taken
+    np.testing.assert_allclose(a["train"][1], b["train"][1], atol=1e-3)
+    np.testing.assert_allclose(a["train"][2], b["train"][2], atol=1e-3)
