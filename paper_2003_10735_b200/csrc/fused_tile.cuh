@@ -35,6 +35,10 @@ struct Args {
     const float* bias;       // the classifier's bias of this block's stream (fp32 master parameters)
     float* z_out;            // nullptr, or the stream's logits [C][h][w]: the block's own nodes are written there as well
     int C, h, w;
+    // tc::kSpinLimit and 0 in normal use.  A test of the give-up path lowers the limit and makes the first barrier expect
+    // stall_bytes more than its copy delivers, so that the wait on it runs out: every copy that was issued still lands,
+    // the block records where it gave up, writes nothing, frees its tensor memory and returns.
+    uint32_t spin_limit, stall_bytes;
 };
 
 // What the block keeps in static shared memory for this
@@ -80,7 +84,7 @@ __device__ __forceinline__ Tile logit_tile(const Args& a, const CUtensorMap* x_m
     const int n_pre = a.x_early ? min(kStages, kblocks) : 0;
     if (tid == 0)
         for (int kb = 0; kb < n_pre; ++kb) {
-            tc::mbar_expect_tx(full_bar(kb), kStageBytes);
+            tc::mbar_expect_tx(full_bar(kb), kStageBytes + (kb == 0 ? a.stall_bytes : 0u));
             tc::tma_load_4d(ring + kb * kStageBytes, x_map, full_bar(kb), kb * 64, x0 - 1, y0 - 1, s);
         }
     pdl_wait();                                        // the weights come from the previous kernel of the stream
@@ -101,7 +105,7 @@ __device__ __forceinline__ Tile logit_tile(const Args& a, const CUtensorMap* x_m
             const int st = kb % kStages;
             if (kb >= kStages) ok = tc::mbar_wait(empty_bar(st), ((kb / kStages) - 1) & 1, a.err, tc::kWaitEmpty);
             if (ok) {
-                tc::mbar_expect_tx(full_bar(st), kStageBytes);
+                tc::mbar_expect_tx(full_bar(st), kStageBytes + (kb == 0 ? a.stall_bytes : 0u));
                 tc::tma_load_4d(ring + st * kStageBytes, x_map, full_bar(st), kb * 64, x0 - 1, y0 - 1, s);
             }
         }
@@ -110,7 +114,7 @@ __device__ __forceinline__ Tile logit_tile(const Args& a, const CUtensorMap* x_m
         ok = tc::mbar_wait(w_bar, 0, a.err, tc::kWaitFull);
         for (int kb = 0; kb < kblocks && ok; ++kb) {
             const int st = kb % kStages;
-            ok = tc::mbar_wait(full_bar(st), (kb / kStages) & 1, a.err, tc::kWaitFull);
+            ok = tc::mbar_wait(full_bar(st), (kb / kStages) & 1, a.err, tc::kWaitFull, a.spin_limit);
             if (!ok) break;
             tc::tc_fence_after_sync();
 #pragma unroll

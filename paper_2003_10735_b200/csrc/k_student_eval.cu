@@ -68,6 +68,7 @@ student_eval_kernel(StudentMaskArgs a, const __grid_constant__ CUtensorMap x_map
     fa.kblocks = a.kblocks; fa.x_early = 1;                // nothing that can still be running writes the features
     fa.skip = nullptr; fa.err = a.err; fa.bias = a.bias; fa.z_out = nullptr;
     fa.C = C; fa.h = h; fa.w = w;
+    fa.spin_limit = tc::kSpinLimit; fa.stall_bytes = 0;
     auto after_mma = [&]() {
         if (CONF) for (int e = tid; e < C * C; e += kThreads) hist[e] = 0;
     };

@@ -314,6 +314,7 @@ upsample_ce_rows_kernel(UpsampleCeArgs a, const __grid_constant__ CUtensorMap z_
         fa.bias = a.theta + (int64_t)s * a.n_params + a.b_off;
         fa.z_out = a.z_out ? a.z_out + (int64_t)s * C * p : nullptr;
         fa.C = C; fa.h = h; fa.w = w;
+        fa.spin_limit = a.test_stall ? (1u << 12) : tc::kSpinLimit; fa.stall_bytes = a.test_stall ? 16u : 0u;
         auto after_mma = [&]() {                        // the arrays the stages lay over get their initial contents
             for (int e = tid; e < C * TZ / 4; e += R_THREADS) reinterpret_cast<int4*>(corr)[e] = make_int4(0, 0, 0, 0);
             if (CONF) for (int e = tid; e < C * C; e += R_THREADS) hist[e] = 0;

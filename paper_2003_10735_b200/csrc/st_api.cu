@@ -72,6 +72,7 @@ struct st_ctx {
     int k3_has_map = 0;
     CUtensorMap fx_map, fw_map; // tile maps of the features and of the bf16 classifier weights: the loss kernel multiplies its own logits
     int fused_fwd = 0;          //   (one-layer head with bf16 GEMMs; ST_FUSED_FORWARD=0 switches it off)
+    int test_stall_fused = 0;   // test of the give-up path inside that kernel (environment ST_TEST_STALL_FUSED=1 at context creation)
     float* loss_buf = nullptr;              // [S][kMaxSteps]
     unsigned long long* conf_buf = nullptr; // [S][kMaxSteps][C][C], allocated on first use
     // Train (Algorithm 1), allocated on first use
@@ -309,7 +310,7 @@ UpsampleCeArgs k3_args(st_ctx* c, bool fp32_grad, bool bf16_grad, unsigned long 
     k3.has_map = c->k3_has_map;
     k3.skip = skip; k3.skip_stride = skip_stride;
     k3.chain_early = c->chain_early ? 1 : 0;
-    k3.fused = 0; k3.x_early = 0; k3.kblocks = 0; k3.theta = nullptr; k3.n_params = 0; k3.b_off = 0; k3.z_out = nullptr;
+    k3.fused = 0; k3.x_early = 0; k3.kblocks = 0; k3.theta = nullptr; k3.n_params = 0; k3.b_off = 0; k3.z_out = nullptr; k3.test_stall = 0;
     return k3;
 }
 
@@ -326,6 +327,7 @@ st_status enqueue_loss(st_ctx* c, unsigned long long* conf, StageTimer* t = null
         k3.fused = 1; k3.x_early = after_update && !t ? 1 : 0; k3.kblocks = c->Cin / 64;
         k3.theta = c->theta; k3.n_params = c->n_params; k3.b_off = c->layout.b_off[c->layout.n_layers - 1];
         k3.z_out = keep_logits ? c->z : nullptr;         // logits that the next iteration overwrites unread stay on the chip
+        k3.test_stall = c->test_stall_fused;
     }
     ST_REPEAT(t) launch_upsample_ce(k3, &c->k3_map, s, &c->fx_map, &c->fw_map);
     if (t) t->mark(k3.fused ? "fwd1x1_upsample_ce" : "upsample_ce", s, st_repeats(t));
@@ -694,6 +696,7 @@ st_status st_init_head(const st_head_desc* desc, const float* init_params, st_ct
                            encode_tensor_map(&c->fw_map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, CU_TENSOR_MAP_SWIZZLE_128B, c->w2_shadow, 3,
                                              dims, str, box, msg, sizeof msg, "1x1 weight") &&
                            prepare_student_eval(c->C) == cudaSuccess;
+            if (const char* ts = getenv("ST_TEST_STALL_FUSED")) c->test_stall_fused = ts[0] == '1' ? 1 : 0;
         }
     }
     if (e == cudaSuccess) e = cudaStreamSynchronize(c->stream);   // init_params may be released on return

@@ -113,6 +113,7 @@ struct UpsampleCeArgs {
     const float* theta;      // parameters (for the bias: theta[s * n_params + b_off + c])
     int64_t n_params, b_off;
     float* z_out;            // nullptr, or [S][C][h][w]: the logits are written here as well
+    int test_stall;          // test of the give-up path: the first wait of the block's forward runs out (see fused_tile.cuh)
 };
 // Tile map of the logits for the row-walking kernel: fp32 tensor {w, h, S*C}, one box = the block's tile of all
 // classes.  False if the shape does not allow it (w not a multiple of 4, C > 32) or the driver entry point is

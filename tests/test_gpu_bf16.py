@@ -311,6 +311,35 @@ def test_a_wait_that_runs_out_is_reported_and_nothing_else_breaks(monkeypatch):
     st.st_destroy(good)
 
 
+def test_a_wait_that_runs_out_inside_the_loss_kernels_own_forward(monkeypatch):
+    """The same for the forward that a one-layer head's loss kernel runs inside its blocks: with the test-only switch
+    the first feature slice's barrier expects 16 bytes more than the copy delivers and the limit is short.  Every block
+    gives up, writes nothing, frees its tensor memory and returns; the error is reported once and the device stays
+    usable."""
+    c_in, C, h, w = 128, 5, 20, 64
+    feat, T = problem(13, c_in, C, h, w)
+    theta = si.initial_head_params(c_in, 0, C, 5)
+    monkeypatch.setenv("ST_TEST_STALL_FUSED", "1")
+    ctx = make_ctx(c_in, 0, C, h, w, theta, lr=0.05)
+    monkeypatch.delenv("ST_TEST_STALL_FUSED")
+    st.st_set_frozen_features(ctx, 0, dev(feat)); st.st_teacher_labels(ctx, 0, dev(T))
+    st.st_distill_step(ctx, 2)
+    with pytest.raises(st.StError) as ei:
+        st.st_read_tensor(ctx, 0, st.ST_TENSOR_FEATURES)
+    assert ei.value.status == st.ST_ERR_CUDA
+    assert "gave up waiting (code 1," in str(ei.value)                    # code 1: a wait for data to arrive
+    assert (st.st_read_tensor(ctx, 0, st.ST_TENSOR_FEATURES) == oracle.round_bf16(feat).ravel()).all()   # reported once
+    st.st_destroy(ctx)
+    good = make_ctx(c_in, 0, C, h, w, theta, lr=0.05)
+    st.st_set_frozen_features(good, 0, dev(feat)); st.st_teacher_labels(good, 0, dev(T))
+    loss = np.zeros(1, np.float32)
+    st.st_distill_step(good, 1, loss)
+    hq = oracle.Head(c_in, 0, C, lr=0.05, theta=theta, quantize_bf16=True)
+    l_ref, _, _ = oracle.gradients(hq, feat, oracle.teacher_labels(T))
+    assert abs(loss[0] - l_ref) <= 2e-5 * abs(l_ref)
+    st.st_destroy(good)
+
+
 @pytest.mark.parametrize("c_in,C,h,w,S", [
     (64, 5, 9, 32, 1),       # the smallest map the block-level forward takes: one tile, one 64-channel slice
     (128, 21, 24, 40, 2),    # two streams, ragged tiles in both directions
