@@ -518,8 +518,8 @@ def train_key_frame(head: Head, feat: np.ndarray, labels: np.ndarray, threshold:
                     keep_masks: bool = False) -> TrainResult:
     """Train(student, frame, label) of Algorithm 1.
 
-    The incoming student is judged first and is the first best_student; distillation is skipped when it
-    already meets the threshold.  Otherwise up to `max_updates` optimisation steps follow, each judged by
+    The incoming student is assessed first and is the first best_student; distillation is skipped when it
+    already meets the threshold.  Otherwise up to `max_updates` optimisation steps follow, each assessed by
     the metric of the prediction made after it; the best iterate so far is remembered (a later one has to
     be strictly better) and the loop ends at the first metric above the threshold.
     The metric is the mean IoU of Section 3.2 between the student's mask and the pseudo-label.
@@ -535,7 +535,7 @@ def train_key_frame(head: Head, feat: np.ndarray, labels: np.ndarray, threshold:
         res.masks.append(prediction)
     if best_metric < threshold:
         for i in range(1, max_updates + 1):
-            # the loss is a function of the same parameters that produced the prediction judged last
+            # the loss is a function of the same parameters that produced the prediction assessed last
             loss, _ = distill_step(head, feat, labels)
             res.losses.append(loss)
             res.n_updates = i

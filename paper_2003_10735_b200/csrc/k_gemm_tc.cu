@@ -160,7 +160,7 @@ tc_wgrad1x1_kernel(const __grid_constant__ CUtensorMap tmA,   // {K, p, S}      
                    int K, int n_chunks, int chunks_per_block, int m_split, int tmem_cols, unsigned int* err,
                    const int* __restrict__ skip, int64_t skip_stride, int a_early, int has_ctl, const TrainCtl ctl)
 {
-    // Train: the block after the last one of the weight gradient judges the prediction (metric, best so far, break)
+    // Train: the block after the last one of the weight gradient assesses the prediction (metric, best so far, break)
     // while the others multiply; it takes no part in anything below
     if (has_ctl && blockIdx.x == gridDim.x - 1) {
         const int s = blockIdx.y;

@@ -134,13 +134,13 @@ sgd_update_kernel(UpdateArgs a, int n_param_blocks, int64_t range_begin)
     bool skip = a.skip && a.skip[(int64_t)s * a.skip_stride];   // block-uniform
     bool better = false;                                         // Train: this prediction is the best so far
     MiouFetch fetched{};
-    const bool decide_here = a.has_ctl == 1;                     // 2: the backward before this kernel has judged the prediction
+    const bool decide_here = a.has_ctl == 1;                     // 2: the backward before this kernel has assessed the prediction
     if (decide_here) fetched = train_fetch(a.ctl, s, hist);      // on their way while the partial sums are fetched and added
     if (a.has_ctl == 2 && !hist.ended) train_outcome(a.ctl, s, skip, better);
     float* best_theta = a.has_ctl ? a.ctl.best_theta : nullptr;
     const AdamCorr corr = adam_corrections<ADAM>(a, s);
     if (param_block) {
-        if (a.has_ctl && hist.ended) {                  // nothing to judge, nothing to update: the history goes on
+        if (a.has_ctl && hist.ended) {                  // nothing to assess, nothing to update: the history goes on
             if (decide_here) train_decision(a.ctl, s, blockIdx.x == 0, hist, &fetched, skip, better);
             return;
         }

@@ -366,7 +366,7 @@ st_status enqueue_update(st_ctx* c, int slot, const int* skip, int64_t skip_stri
                          int ctl_mode = 1)
 {
     UpdateArgs u = make_update_args(c, slot, skip, skip_stride);
-    // Train: the update judges the prediction itself (1), or reads what the backward before it has found (2)
+    // Train: the update assesses the prediction itself (1), or reads what the backward before it has found (2)
     if (ctl) { u.has_ctl = ctl_mode; u.ctl = *ctl; u.skip = nullptr; }
     c->launches += launch_sgd_update(u, c->stream);
     if (t) t->mark("sgd_update", c->stream, 1);
@@ -913,7 +913,7 @@ TrainCtl train_ctl(st_ctx* c, int iter, int max_updates, double threshold)
 }
 
 // Train of Algorithm 1 for all streams: one prediction per pass (forward, loss + gradient + confusion), the backward,
-// then the update kernel, which first judges the prediction (metric, best_student, break) and takes the step only
+// then the update kernel, which first assesses the prediction (metric, best_student, break) and takes the step only
 // where the loop goes on.  The backward of the pass in which a loop ends is therefore computed and not used; from the
 // next pass on the stream's blocks of the tensor-core GEMMs and of the loss kernel return at once (the fp32
 // convolutions still run: their results are simply not used).
@@ -924,7 +924,7 @@ st_status enqueue_train(st_ctx* c, int max_updates, double threshold)
         const int* ended_before = i > 0 ? c->ctl_done + i : nullptr;        // done[s][i]: no prediction i for stream s
         st = enqueue_forward(c, nullptr, ended_before, kCtlPitch, false, true);           // prediction <- Forward(student, frame)
         if (st == ST_OK) st = enqueue_loss(c, c->conf_buf + (int64_t)i * c->C * c->C, nullptr, ended_before, kCtlPitch, i > 0, false);   // loss, gradient, confusion
-        // metric, best_student, break: judged by an extra block of the backward's first tensor-core kernel while that
+        // metric, best_student, break: assessed by an extra block of the backward's first tensor-core kernel while that
         // kernel works, or, where there is none (fp32 convolutions; the last prediction, after which every loop ends),
         // by the update itself, which in any case takes the step only where the loop goes on
         const TrainCtl ctl = train_ctl(c, i, max_updates, threshold);
@@ -1004,7 +1004,7 @@ st_status st_train_key_frame(st_ctx* ctx, double threshold, int32_t max_updates,
         ST_CUDA(ctx, cudaMemcpyAsync(n_updates_out, ctx->ctl_n_updates, (size_t)ctx->S * sizeof(int), cudaMemcpyDefault, ctx->stream));
         host_out |= !is_device_ptr(n_updates_out);
     }
-    if (best_metric_out) {     // best_metric after the last prediction was judged
+    if (best_metric_out) {     // best_metric after the last prediction was assessed
         ST_CUDA(ctx, cudaMemcpy2DAsync(best_metric_out, sizeof(double), ctx->ctl_best + n_pred, kCtlPitch * sizeof(double),
                                        sizeof(double), ctx->S, cudaMemcpyDefault, ctx->stream));
         host_out |= !is_device_ptr(best_metric_out);

@@ -178,11 +178,11 @@ void launch_conv1x1_dgrad_relu_f32(const float* W2, const float* dz, const float
 void launch_bias_grad_f32(const float* d, int C, int64_t p, float* db, int S, int64_t d_stride,
                           int64_t db_stride, cudaStream_t s);
 
-// ---- control of Algorithm 1 (Train): judged once per prediction, per stream, by the update kernel that follows the
+// ---- control of Algorithm 1 (Train): assessed once per prediction, per stream, by the update kernel that follows the
 // prediction (metric of the prediction, best_student, the break) ----------------------------------------------
 // History arrays are indexed by the number of updates behind a prediction, so that a launch reads only what
 // earlier launches wrote: done[s][i] = the loop of stream s had ended before prediction i was made,
-// best[s][i] = best_metric before prediction i was judged.
+// best[s][i] = best_metric before prediction i was assessed.
 constexpr int kCtlPitch = kMaxSteps + 2;
 struct TrainCtl {
     const unsigned long long* conf;   // confusion matrix of this prediction, stream 0
@@ -244,11 +244,11 @@ struct UpdateArgs {
     double b1, b2, eps, ln_b1, ln_b2;
     const long long* step_base;   // [S] optimisation steps taken before this call
     int chain_early;         // launch so that the kernel may start while its predecessor on the stream drains
-    // Train (Algorithm 1): the update also judges the prediction it follows.  Every block works the metric out from the
+    // Train (Algorithm 1): the update also assesses the prediction it follows.  Every block works the metric out from the
     // prediction's confusion matrix (same counts, same arithmetic, same answer), keeps the old value of its parameters
     // as best_student's where the metric is the best so far, and leaves them alone where the loop has ended; block 0
     // writes the history.  `skip` is then not used.
-    int has_ctl;             // 0; 1: this kernel judges the prediction; 2: the backward before it has (see tc_backward), read the outcome
+    int has_ctl;             // 0; 1: this kernel assesses the prediction; 2: the backward before it has (see tc_backward), read the outcome
     TrainCtl ctl;
 };
 // step_base[s] += add (add_per_stream == nullptr) or += add_per_stream[s]
@@ -334,7 +334,7 @@ int tc_forward(const TcPlan*, cudaStream_t s, StageTimer* t = nullptr, const int
                bool after_update = false, int first_block = 0);
 int tc_forward_blocks(const TcPlan*, int first, int last, cudaStream_t s, StageTimer* t = nullptr, const int* skip = nullptr,
                       int64_t skip_stride = 0);
-// `ctl` (Train): one extra block per stream of the first kernel judges the prediction the backward belongs to, beside the
+// `ctl` (Train): one extra block per stream of the first kernel assesses the prediction the backward belongs to, beside the
 // kernel's own work; the update that follows reads the outcome.
 int tc_backward(const TcPlan*, cudaStream_t s, StageTimer* t = nullptr, const int* skip = nullptr, int64_t skip_stride = 0,
                 const TrainCtl* ctl = nullptr);

@@ -1,4 +1,4 @@
-// Train of Algorithm 1: the judgement of a prediction, shared by the kernels that take it.
+// Train of Algorithm 1: the assessment of a prediction, shared by the kernels that take it.
 #pragma once
 
 #include "st_internal.h"
@@ -6,12 +6,12 @@
 
 namespace st {
 
-// Train (Algorithm 1), the judgement of prediction i: metric <- mIoU of the prediction; better = the metric is the best
+// Train (Algorithm 1), the assessment of prediction i: metric <- mIoU of the prediction; better = the metric is the best
 // so far (best_student <- student); skip = the loop ends here or had ended before (no OptimStep).  It is taken either
 // by one extra block of the first backward kernel, beside that kernel's own work (the update then reads the outcome),
 // or, where no backward follows the prediction, by every block of the update itself (same counts, same arithmetic,
 // same answer).  In three parts so that the loads overlap what else a kernel waits for: train_history reads what the
-// previous judgement left (it may run before the kernel's predecessors have finished), train_fetch starts the loads of
+// previous assessment left (it may run before the kernel's predecessors have finished), train_fetch starts the loads of
 // the prediction's confusion matrix (blocks of 256 threads), train_decision finishes.  Block-uniform; called by all
 // threads of the block.  `writer` (one block per stream) records the history.
 struct TrainHistory { bool ended; double prev_best; };
